@@ -1,0 +1,463 @@
+"""Cost functions of the optimisation problems and their derivatives, in fp64.
+
+TEST INFRASTRUCTURE (see the package docstring).  A `Level` is one problem P_k of the
+multilevel program of Sec. 2: its own parameters theta_k, its cost C_k, one batch of data
+D_k and the list of problems whose parameters constrain it (U_k and L_k, Def. 1).
+
+Notation (own parameters x, one constraining block c):
+    g = dC/dx,  H = d2C/dx2,  M = d(g)/dc,  so that  (dx*/dc)^T v = -M^T H^{-1} v
+by the implicit function theorem at a stationary point of C in x (the base operation of
+Sec. 3.2).  Every function below is the hand-derived formula for one cost family; the tests
+pin each of them to central finite differences of `cost`.
+
+Cost families
+-------------
+logreg_wd        App. D.1 lower problem: mean logistic loss + 1/2 w^T diag(lambda) w
+logreg           App. D.1 upper problem: mean logistic loss of the lower w on validation data
+quadratic_wd     1/2 |A w - b|^2 + 1/2 w^T diag(lambda) w   (closed-form best response)
+quadratic        1/2 |A w - b|^2 of a constraining w          (upper loss for the above)
+mlp_ce_reweight  App. A "Classifier": mean_i r_i * CE_i with r_i = sigmoid(weightnet(CE_i
+                 detached)), plus 1/2 sum_l exp(lambda_l) |W_l|^2 when a log-weight-decay
+                 constraint is attached
+mlp_ce           App. A "Reweight": plain mean cross-entropy of a constraining classifier
+weightnet_detect mean_j (sigmoid(weightnet(CE_j(w))) - clean_j)^2 + mu/2 |theta|^2, where the
+                 per-sample loss is NOT detached (w is a constraining parameter of this cost)
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Optional
+
+import numpy as np
+from scipy.special import erf, expit
+
+from .bf16 import round_to_bf16
+
+WN_H = 100  # hidden width of the 1-100-1 weight net (App. C, "Meta-Weight-Network")
+
+
+@dataclass(eq=False)
+class Level:
+    loss: str
+    param_kind: str                    # 'vector' | 'mlp' | 'weightnet' | 'logwd'
+    params: np.ndarray                 # flat fp64 (master copy)
+    X: Optional[np.ndarray] = None
+    y: Optional[np.ndarray] = None
+    aux: Optional[np.ndarray] = None   # weightnet_detect: 1.0 where the given label is clean
+    widths: Optional[tuple] = None     # MLP layer widths (in, hidden..., classes)
+    activation: str = "relu"
+    lr: float = 0.1
+    mu: float = 0.0
+    bf16: bool = False                 # MLP matrices are used through a bf16-rounded copy
+    constraints: list = field(default_factory=list)
+
+    def __post_init__(self):
+        self.params = np.array(self.params, dtype=np.float64).reshape(-1)
+        if self.X is not None:
+            self.X = np.asarray(self.X, dtype=np.float64)
+        if self.y is not None and np.issubdtype(np.asarray(self.y).dtype, np.floating):
+            self.y = np.asarray(self.y, dtype=np.float64)
+        if self.aux is not None:
+            self.aux = np.asarray(self.aux, dtype=np.float64)
+
+
+def _p(level: Level, over) -> np.ndarray:
+    if over is not None and id(level) in over:
+        return np.asarray(over[id(level)], dtype=np.float64)
+    return level.params
+
+
+def _find(L: Level, kind: str, required: bool = True) -> Optional[Level]:
+    for c in [L] + list(L.constraints):
+        if c.param_kind == kind:
+            return c
+    if required:
+        raise ValueError(f"level with loss {L.loss} has no participant of kind {kind}")
+    return None
+
+
+def _find_constraint(L: Level, kind: str, required: bool = True) -> Optional[Level]:
+    for c in L.constraints:
+        if c.param_kind == kind:
+            return c
+    if required:
+        raise ValueError(f"level with loss {L.loss} has no constraint of kind {kind}")
+    return None
+
+
+# ------------------------------------------------------------------ scalar functions
+def softplus(t):
+    return np.maximum(t, 0.0) + np.log1p(np.exp(-np.abs(t)))
+
+
+def _act(name, a):
+    if name == "relu":
+        return np.maximum(a, 0.0)
+    if name == "gelu":
+        return a * 0.5 * (1.0 + erf(a / np.sqrt(2.0)))
+    raise ValueError(name)
+
+
+def _act_d1(name, a):
+    if name == "relu":
+        return (a > 0.0).astype(np.float64)          # relu'(0) = 0
+    pdf = np.exp(-0.5 * a * a) / np.sqrt(2.0 * np.pi)
+    return 0.5 * (1.0 + erf(a / np.sqrt(2.0))) + a * pdf
+
+
+def _act_d2(name, a):
+    if name == "relu":
+        return np.zeros_like(a)
+    pdf = np.exp(-0.5 * a * a) / np.sqrt(2.0 * np.pi)
+    return pdf * (2.0 - a * a)
+
+
+# ------------------------------------------------------------------ MLP pieces
+def mlp_unpack(widths, flat):
+    """Flat [W_1, b_1, W_2, b_2, ...] -> lists of W_l [out,in] and b_l [out]."""
+    Ws, bs, o = [], [], 0
+    for l in range(len(widths) - 1):
+        fin, fout = widths[l], widths[l + 1]
+        Ws.append(flat[o:o + fout * fin].reshape(fout, fin)); o += fout * fin
+        bs.append(flat[o:o + fout]); o += fout
+    assert o == flat.size, "parameter vector does not match the layer widths"
+    return Ws, bs
+
+
+def mlp_pack(Ws, bs):
+    return np.concatenate([np.concatenate([W.reshape(-1), b.reshape(-1)]) for W, b in zip(Ws, bs)])
+
+
+def _mlp_weights(level: Level, flat):
+    """The copy of the parameters the cost is evaluated at: matrices rounded to bf16 for
+    mixed-precision levels (the single quantisation point), biases as they are."""
+    Ws, bs = mlp_unpack(level.widths, flat)
+    if level.bf16:
+        Ws = [round_to_bf16(W) for W in Ws]
+    return Ws, bs
+
+
+def _mlp_forward(Ws, bs, X, act):
+    """h[l] is the input of layer l (h[0] = X), a[l] its pre-activation; logits = a[-1]."""
+    h, a = [X], []
+    for l, (W, b) in enumerate(zip(Ws, bs)):
+        a.append(h[-1] @ W.T + b)
+        if l < len(Ws) - 1:
+            h.append(_act(act, a[-1]))
+    return h, a
+
+
+def _softmax_ce(z, y):
+    zs = z - z.max(axis=1, keepdims=True)
+    logp = zs - np.log(np.exp(zs).sum(axis=1, keepdims=True))
+    p = np.exp(logp)
+    ell = -logp[np.arange(z.shape[0]), y]
+    return p, ell
+
+
+def _onehot(y, C):
+    e = np.zeros((y.shape[0], C))
+    e[np.arange(y.shape[0]), y] = 1.0
+    return e
+
+
+def _mlp_backward(Ws, h, a, delta_top, act):
+    """Reverse sweep from delta_top = dC/d(logits).  Returns gW, gb and the per-layer
+    delta_l = dC/da_l and dh_l = dC/dh_l (dh[l] pairs with a[l-1])."""
+    L = len(Ws)
+    gW, gb, deltas, dhs = [None] * L, [None] * L, [None] * L, [None] * L
+    delta = delta_top
+    for l in range(L - 1, -1, -1):
+        deltas[l] = delta
+        gW[l] = delta.T @ h[l]
+        gb[l] = delta.sum(axis=0)
+        if l > 0:
+            dhs[l] = delta @ Ws[l]
+            delta = dhs[l] * _act_d1(act, a[l - 1])
+    return gW, gb, deltas, dhs
+
+
+def _mlp_rforward(Ws, h, a, Us, cs, act):
+    """Directional derivative of the forward pass along (U_l, c_l): Ra[l] = d a_l."""
+    Rh = np.zeros_like(h[0])
+    Rhs, Ras = [], []
+    for l in range(len(Ws)):
+        Rhs.append(Rh)
+        Ra = Rh @ Ws[l].T + h[l] @ Us[l].T + cs[l]
+        Ras.append(Ra)
+        if l < len(Ws) - 1:
+            Rh = _act_d1(act, a[l]) * Ra
+    return Rhs, Ras
+
+
+# ------------------------------------------------------------------ weight net 1-100-1
+def wn_unpack(theta):
+    H = WN_H
+    return theta[0:H], theta[H:2 * H], theta[2 * H:3 * H], theta[3 * H]
+
+
+def wn_forward(theta, ell):
+    """s = a2 . relu(a1*ell + b1) + b2 ; r = sigmoid(s).  Returns r, s, hidden, mask."""
+    a1, b1, a2, b2 = wn_unpack(theta)
+    pre = ell[:, None] * a1[None, :] + b1[None, :]
+    mask = (pre > 0.0).astype(np.float64)
+    hid = pre * mask
+    s = hid @ a2 + b2
+    return expit(s), s, hid, mask
+
+
+def wn_grad_s(theta, ell, hid, mask):
+    """Per-sample d s / d theta, shape [B, 301]."""
+    a1, b1, a2, b2 = wn_unpack(theta)
+    ma2 = mask * a2[None, :]
+    return np.concatenate([ma2 * ell[:, None], ma2, hid, np.ones((ell.shape[0], 1))], axis=1)
+
+
+def wn_ds_dell(theta, mask):
+    a1, b1, a2, b2 = wn_unpack(theta)
+    return (mask * (a1 * a2)[None, :]).sum(axis=1)
+
+
+# ------------------------------------------------------------------ per-family evaluation
+def _logreg_parts(L, over):
+    if L.loss == "logreg_wd":
+        w = _p(L, over)
+        lam = _p(_find_constraint(L, "vector"), over)
+    else:
+        w = _p(_find_constraint(L, "vector"), over)
+        lam = None
+    return w, lam
+
+
+def _mlp_ce_state(L: Level, over):
+    """Forward pass of the classifier that takes part in cost L and the per-sample CE."""
+    M = _find(L, "mlp")
+    Ws, bs = _mlp_weights(M, _p(M, over))
+    h, a = _mlp_forward(Ws, bs, L.X, M.activation)
+    p, ell = _softmax_ce(a[-1], np.asarray(L.y, dtype=np.int64))
+    return M, Ws, bs, h, a, p, ell
+
+
+def _reweight_r(L: Level, ell, over):
+    T = _find_constraint(L, "weightnet", required=False)
+    if T is None:
+        return np.ones_like(ell), None
+    r, s, hid, mask = wn_forward(_p(T, over), ell)
+    return r, (T, s, hid, mask)
+
+
+def _kappas(L: Level, over, nl):
+    lamL = _find_constraint(L, "logwd", required=False)
+    if lamL is None:
+        return np.zeros(nl), None
+    return np.exp(_p(lamL, over)), lamL
+
+
+def cost(L: Level, over=None, r_fixed=None, ell_fixed=None) -> float:
+    """C_k evaluated at the current (or overridden) parameters of all participants.
+
+    mlp_ce_reweight carries a stop-gradient (the weight net sees the detached per-sample
+    loss): `r_fixed` freezes the weights r_i (the function whose w-derivatives `grad`/`hvp`
+    return) and `ell_fixed` freezes the per-sample losses (the function whose
+    theta-derivative `grad` returns)."""
+    if L.loss in ("logreg_wd", "logreg"):
+        w, lam = _logreg_parts(L, over)
+        c = softplus(-L.y * (L.X @ w)).mean()
+        if lam is not None:
+            c += 0.5 * np.sum(lam * w * w)
+        return float(c)
+    if L.loss in ("quadratic_wd", "quadratic"):
+        if L.loss == "quadratic_wd":
+            w, lam = _p(L, over), _p(_find_constraint(L, "vector"), over)
+        else:
+            w, lam = _p(_find_constraint(L, "vector"), over), None
+        rres = L.X @ w - L.y
+        c = 0.5 * rres @ rres
+        if lam is not None:
+            c += 0.5 * np.sum(lam * w * w)
+        return float(c)
+    if L.loss == "mlp_ce":
+        _, _, _, _, _, _, ell = _mlp_ce_state(L, over)
+        return float(ell.mean())
+    if L.loss == "mlp_ce_reweight":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        if ell_fixed is not None:
+            ell = np.asarray(ell_fixed, dtype=np.float64)
+        r = _reweight_r(L, ell, over)[0] if r_fixed is None else np.asarray(r_fixed)
+        kap, _ = _kappas(L, over, len(Ws))
+        return float((r * ell).mean() + 0.5 * sum(k * np.sum(W * W) for k, W in zip(kap, Ws)))
+    if L.loss == "weightnet_detect":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        T = _find(L, "weightnet")
+        th = _p(T, over)
+        r, _, _, _ = wn_forward(th, ell)
+        return float(((r - L.aux) ** 2).mean() + 0.5 * L.mu * th @ th)
+    raise ValueError(L.loss)
+
+
+def grad(L: Level, wrt: Level, over=None) -> np.ndarray:
+    """dC_L / d(params of `wrt`), `wrt` being L itself or one of its constraints.
+
+    For mlp_ce_reweight the stop-gradient of the App. A listing applies: the derivative with
+    respect to the classifier treats r_i as constants, the derivative with respect to the
+    weight net treats the per-sample losses as data."""
+    n_out = _p(wrt, over).size
+    if L.loss in ("logreg_wd", "logreg"):
+        w, lam = _logreg_parts(L, over)
+        own_w = L if L.loss == "logreg_wd" else _find_constraint(L, "vector")
+        if wrt is own_w:
+            z = L.X @ w
+            g = -(L.X.T @ (L.y * expit(-L.y * z))) / L.X.shape[0]
+            return g + lam * w if lam is not None else g
+        if L.loss == "logreg_wd" and wrt is _find_constraint(L, "vector"):
+            return 0.5 * w * w
+        return np.zeros(n_out)
+    if L.loss in ("quadratic_wd", "quadratic"):
+        own_w = L if L.loss == "quadratic_wd" else _find_constraint(L, "vector")
+        w = _p(own_w, over)
+        if wrt is own_w:
+            g = L.X.T @ (L.X @ w - L.y)
+            return g + _p(_find_constraint(L, "vector"), over) * w if L.loss == "quadratic_wd" else g
+        if L.loss == "quadratic_wd" and wrt is _find_constraint(L, "vector"):
+            return 0.5 * w * w
+        return np.zeros(n_out)
+    if L.loss == "mlp_ce":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        if wrt is not M:
+            return np.zeros(n_out)
+        B = L.X.shape[0]
+        delta = (p - _onehot(np.asarray(L.y, np.int64), p.shape[1])) / B
+        gW, gb, _, _ = _mlp_backward(Ws, h, a, delta, M.activation)
+        return mlp_pack(gW, gb)
+    if L.loss == "mlp_ce_reweight":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        B = L.X.shape[0]
+        r, wn = _reweight_r(L, ell, over)
+        kap, lamL = _kappas(L, over, len(Ws))
+        if wrt is L:
+            delta = (r / B)[:, None] * (p - _onehot(np.asarray(L.y, np.int64), p.shape[1]))
+            gW, gb, _, _ = _mlp_backward(Ws, h, a, delta, M.activation)
+            gW = [g + k * W for g, k, W in zip(gW, kap, Ws)]
+            return mlp_pack(gW, gb)
+        if wn is not None and wrt is wn[0]:
+            T, s, hid, mask = wn
+            J = wn_grad_s(_p(T, over), ell, hid, mask)
+            return ((r * (1.0 - r) * ell)[:, None] * J).sum(axis=0) / B
+        if lamL is not None and wrt is lamL:
+            return np.array([0.5 * k * np.sum(W * W) for k, W in zip(kap, Ws)])
+        return np.zeros(n_out)
+    if L.loss == "weightnet_detect":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        T = _find(L, "weightnet")
+        th = _p(T, over)
+        B = L.X.shape[0]
+        r, s, hid, mask = wn_forward(th, ell)
+        fp = 2.0 * (r - L.aux) * r * (1.0 - r)          # d/ds (sigmoid(s) - c)^2
+        if wrt is T:
+            return (fp[:, None] * wn_grad_s(th, ell, hid, mask)).sum(axis=0) / B + L.mu * th
+        if wrt is M:
+            kappa = fp * wn_ds_dell(th, mask) / B              # dC/d ell_j
+            delta = kappa[:, None] * (p - _onehot(np.asarray(L.y, np.int64), p.shape[1]))
+            gW, gb, _, _ = _mlp_backward(Ws, h, a, delta, M.activation)
+            return mlp_pack(gW, gb)
+        return np.zeros(n_out)
+    raise ValueError(L.loss)
+
+
+def hvp(L: Level, u: np.ndarray, over=None) -> np.ndarray:
+    """H u with H = d2 C_L / d(own params)^2."""
+    u = np.asarray(u, dtype=np.float64)
+    if L.loss == "logreg_wd":
+        w, lam = _logreg_parts(L, over)
+        z = L.X @ w
+        return L.X.T @ (expit(z) * expit(-z) * (L.X @ u)) / L.X.shape[0] + lam * u
+    if L.loss == "quadratic_wd":
+        lam = _p(_find_constraint(L, "vector"), over)
+        return L.X.T @ (L.X @ u) + lam * u
+    if L.loss == "mlp_ce_reweight":
+        # R-operator (forward-over-reverse) through the classifier, r_i held constant.
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        act = M.activation
+        B = L.X.shape[0]
+        r, _ = _reweight_r(L, ell, over)
+        kap, _ = _kappas(L, over, len(Ws))
+        Us, cs = mlp_unpack(M.widths, u)
+        delta_top = (r / B)[:, None] * (p - _onehot(np.asarray(L.y, np.int64), p.shape[1]))
+        _, _, deltas, dhs = _mlp_backward(Ws, h, a, delta_top, act)
+        Rhs, Ras = _mlp_rforward(Ws, h, a, Us, cs, act)
+        Rdelta = (r / B)[:, None] * (p * Ras[-1] - p * (p * Ras[-1]).sum(axis=1, keepdims=True))
+        nl = len(Ws)
+        RgW, Rgb = [None] * nl, [None] * nl
+        for l in range(nl - 1, -1, -1):
+            RgW[l] = Rdelta.T @ h[l] + deltas[l].T @ Rhs[l] + kap[l] * Us[l]
+            Rgb[l] = Rdelta.sum(axis=0)
+            if l > 0:
+                Rdh = Rdelta @ Ws[l] + deltas[l] @ Us[l]
+                Rdelta = (Rdh * _act_d1(act, a[l - 1])
+                          + dhs[l] * _act_d2(act, a[l - 1]) * Ras[l - 1])
+        return mlp_pack(RgW, Rgb)
+    if L.loss == "weightnet_detect" and L.param_kind == "weightnet":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        th = _p(L, over)
+        a1, b1, a2, b2 = wn_unpack(th)
+        ua1, ub1, ua2, ub2 = wn_unpack(u)
+        B = L.X.shape[0]
+        r, s, hid, mask = wn_forward(th, ell)
+        c = L.aux
+        rp = r * (1.0 - r)
+        fp = 2.0 * (r - c) * rp
+        fpp = 2.0 * rp * rp + 2.0 * (r - c) * rp * (1.0 - 2.0 * r)
+        J = wn_grad_s(th, ell, hid, mask)                     # [B,301]
+        Ju = J @ u
+        # second derivative of s: only the (a2_k, a1_k) and (a2_k, b1_k) pairs are non-zero
+        S2u = np.concatenate([
+            mask * ua2[None, :] * ell[:, None],
+            mask * ua2[None, :],
+            mask * (ell[:, None] * ua1[None, :] + ub1[None, :]),
+            np.zeros((B, 1))], axis=1)
+        return ((fpp * Ju)[:, None] * J + fp[:, None] * S2u).sum(axis=0) / B + L.mu * u
+    raise ValueError(f"no Hessian-vector product for loss {L.loss} / {L.param_kind}")
+
+
+def mixed_vjp(L: Level, wrt: Level, q: np.ndarray, over=None) -> np.ndarray:
+    """M^T q = d/dc < dC_L/dx , q > with q held fixed, c = params of the constraint `wrt`."""
+    q = np.asarray(q, dtype=np.float64)
+    if L.loss in ("logreg_wd", "quadratic_wd"):
+        if wrt is _find_constraint(L, "vector"):
+            return _p(L, over) * q
+        raise ValueError("unknown constraint")
+    if L.loss == "mlp_ce_reweight":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        B = L.X.shape[0]
+        r, wn = _reweight_r(L, ell, over)
+        kap, lamL = _kappas(L, over, len(Ws))
+        Qs, qc = mlp_unpack(M.widths, q)
+        if wn is not None and wrt is wn[0]:
+            T, s, hid, mask = wn
+            _, Ras = _mlp_rforward(Ws, h, a, Qs, qc, M.activation)
+            d = ((p - _onehot(np.asarray(L.y, np.int64), p.shape[1])) * Ras[-1]).sum(axis=1)
+            J = wn_grad_s(_p(T, over), ell, hid, mask)
+            return ((d * r * (1.0 - r))[:, None] * J).sum(axis=0) / B
+        if lamL is not None and wrt is lamL:
+            return np.array([k * np.sum(W * Q) for k, W, Q in zip(kap, Ws, Qs)])
+        raise ValueError("unknown constraint")
+    if L.loss == "weightnet_detect" and L.param_kind == "weightnet":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        if wrt is not M:
+            raise ValueError("unknown constraint")
+        th = _p(L, over)
+        a1, b1, a2, b2 = wn_unpack(th)
+        qa1, qb1, qa2, qb2 = wn_unpack(q)
+        B = L.X.shape[0]
+        r, s, hid, mask = wn_forward(th, ell)
+        c = L.aux
+        rp = r * (1.0 - r)
+        fp = 2.0 * (r - c) * rp
+        fpp = 2.0 * rp * rp + 2.0 * (r - c) * rp * (1.0 - 2.0 * r)
+        Jq = wn_grad_s(th, ell, hid, mask) @ q
+        dJq_dell = (mask * (a2 * qa1 + a1 * qa2)[None, :]).sum(axis=1)
+        kappa = (fpp * wn_ds_dell(th, mask) * Jq + fp * dJq_dell) / B
+        delta = kappa[:, None] * (p - _onehot(np.asarray(L.y, np.int64), p.shape[1]))
+        gW, gb, _, _ = _mlp_backward(Ws, h, a, delta, M.activation)
+        return mlp_pack(gW, gb)
+    raise ValueError(f"no mixed second derivative for loss {L.loss}")

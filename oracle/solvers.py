@@ -1,0 +1,134 @@
+"""Unrolled lower steps, best-response-Jacobian x vector products and their chaining (fp64).
+
+TEST INFRASTRUCTURE (see the package docstring).
+
+The paper names the approximations (Sec. 3.2: AID with Neumann series, AID with conjugate
+gradient, AID with finite difference) and refers to the original works for their steps; the
+steps below are the textbook form of each, applied to the implicit-function-theorem
+expression  (dx*/dc)^T v = -M^T H^{-1} v  evaluated at the current (unrolled, approximate)
+lower parameters x (Sec. 3.2; Sec. 5.4 for the finite difference being taken at the unrolled
+weights).  Readings where the paper is silent:
+  * Neumann(K, alpha): K Hessian-vector products, terms j = 0..K, the sum scaled by alpha, so
+    that it tends to H^{-1} v when the spectral radius of (I - alpha H) is below one.
+  * CG(K, tol): zero start, no preconditioner, stops after K iterations, or when the residual
+    norm has fallen to tol*|v|, or (status "breakdown") when a search direction has p^T H p <= 0.
+  * FD(eps0, alpha): eps = eps0/|v|_2; result -alpha*[dC/dc(x+eps v) - dC/dc(x-eps v)]/(2 eps),
+    i.e. H^{-1} replaced by alpha*I; alpha defaults to 1.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from . import levels as _lv
+from .levels import Level
+
+grad = _lv.grad
+hvp = _lv.hvp
+mixed_vjp = _lv.mixed_vjp
+
+
+def lower_step(L: Level, n_steps: int) -> None:
+    """x <- x - lr * dC/dx, n_steps times on the level's fixed batch (Sec. 3.2: w* is
+    approximated by a small number of unrolled gradient steps).  Updates L.params in place.
+    For mixed-precision levels the gradient is taken at the bf16-rounded copy of the
+    current master, which is re-derived at every step."""
+    for _ in range(int(n_steps)):
+        L.params = L.params - L.lr * grad(L, L)
+
+
+def neumann_solve(hv, v, K: int, alpha: float) -> np.ndarray:
+    """q = alpha * sum_{j=0..K} (I - alpha H)^j v, built with K products hv(.) = H(.)."""
+    t = np.array(v, dtype=np.float64)
+    s = t.copy()
+    for _ in range(int(K)):
+        t = t - alpha * hv(t)
+        s = s + t
+    return alpha * s
+
+
+def cg_solve(hv, v, K: int, tol: float = 0.0):
+    """Conjugate gradient on H q = v.  Returns (q, iterations done, status) with status
+    'ok' or 'breakdown'."""
+    v = np.asarray(v, dtype=np.float64)
+    q = np.zeros_like(v)
+    r = v.copy()
+    p = r.copy()
+    rho = r @ r
+    stop = (tol * tol) * (v @ v)
+    it = 0
+    for _ in range(int(K)):
+        if rho <= stop:
+            break
+        h = hv(p)
+        gamma = p @ h
+        if gamma <= 0.0:
+            return q, it, "breakdown"
+        a = rho / gamma
+        q = q + a * p
+        r = r - a * h
+        rho_new = r @ r
+        p = r + (rho_new / rho) * p
+        rho = rho_new
+        it += 1
+    return q, it, "ok"
+
+
+def brj(L: Level, wrt: Level, v, method: str, K: int = 0, alpha: float = 1.0,
+        eps0: float = 0.01, tol: float = 0.0, info: dict | None = None) -> np.ndarray:
+    """(d x*/d c)^T v for the problem L (own parameters x) and its constraint `wrt` (c):
+    the base operation of Sec. 3.2, by the chosen approximation."""
+    v = np.asarray(v, dtype=np.float64)
+    if method == "neumann":
+        q = neumann_solve(lambda t: hvp(L, t), v, K, alpha)
+        return -mixed_vjp(L, wrt, q)
+    if method == "cg":
+        q, it, status = cg_solve(lambda t: hvp(L, t), v, K, tol)
+        if info is not None:
+            info["iters"], info["status"] = it, status
+        return -mixed_vjp(L, wrt, q)
+    if method == "fd":
+        nv = np.sqrt(v @ v)
+        if nv == 0.0:
+            return np.zeros(wrt.params.size)
+        eps = eps0 / nv
+        gp = grad(L, wrt, over={id(L): L.params + eps * v})
+        gm = grad(L, wrt, over={id(L): L.params - eps * v})
+        return -alpha * (gp - gm) / (2.0 * eps)
+    raise ValueError(method)
+
+
+def _hypergrad(lower, upper, wrt, **kw):
+    """Eq. 1 for one lower problem: direct gradient + best-response Jacobian x direct gradient."""
+    v = grad(upper, lower)
+    return grad(upper, wrt) + brj(lower, wrt, v, **kw)
+
+
+def hypergrad_neumann(lower: Level, upper: Level, wrt: Level, K: int, alpha: float):
+    return _hypergrad(lower, upper, wrt, method="neumann", K=K, alpha=alpha)
+
+
+def hypergrad_cg(lower: Level, upper: Level, wrt: Level, K: int, tol: float = 0.0,
+                 info: dict | None = None):
+    return _hypergrad(lower, upper, wrt, method="cg", K=K, tol=tol, info=info)
+
+
+def hypergrad_fd(lower: Level, upper: Level, wrt: Level, eps0: float = 0.01, alpha: float = 1.0):
+    return _hypergrad(lower, upper, wrt, method="fd", eps0=eps0, alpha=alpha)
+
+
+def chain_levels(levels, path, cfgs, v_in=None) -> np.ndarray:
+    """One path term of Eq. 2, evaluated right to left (Sec. 3.2).
+
+    path = [k, q(1), ..., q(m)] are indices into `levels`: the result is with respect to the
+    parameters of levels[k]; q(1) is reached from k by the upper-to-lower edge and q(i+1)
+    from q(i) by lower-to-upper edges.  The start vector is v_in, or dC_k/d theta_{q(m)} when
+    v_in is None.  cfgs[i] (a dict of `brj` keyword arguments) configures the edge into
+    q(i+1), i.e. cfgs[0] is the upper-to-lower edge.  The direct gradient of Eq. 2 is not
+    added."""
+    k, q = path[0], list(path[1:])
+    if not q:
+        raise ValueError("path needs at least one edge")
+    v = grad(levels[k], levels[q[-1]]) if v_in is None else np.asarray(v_in, dtype=np.float64)
+    for i in range(len(q) - 1, 0, -1):
+        v = brj(levels[q[i]], levels[q[i - 1]], v, **cfgs[i])
+    return brj(levels[q[0]], levels[k], v, **cfgs[0])
