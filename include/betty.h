@@ -1,0 +1,190 @@
+/* betty.h - C ABI of the B200 hypergradient library.
+ *
+ * The library evaluates the hot path of gradient-based multilevel optimisation (MLO) as the
+ * Betty paper states it (arXiv 2207.02849): a program of problems P_1..P_n, each with own
+ * parameters theta_k, a cost C_k(theta_k, U_k, L_k; D_k) and constraining parameters from upper
+ * (U_k, non-optimal) and lower (L_k, optimal) problems (Sec. 2, Def. 1).  The gradient of an
+ * upper cost is the direct gradient plus best-response Jacobians times direct gradients (Eq. 1),
+ * a best-response Jacobian along a path being a product of per-edge Jacobians that is evaluated
+ * right to left as repeated (Jacobian x vector) products (Eq. 2 and Sec. 3.2).  The per-edge
+ * product  (d x* / d c)^T v = -M^T H^{-1} v  (x own parameters of the lower problem, c the
+ * constraining block, H = d2C/dx2, M = d(dC/dx)/dc) is approximated by implicit differentiation
+ * with a Neumann series, with conjugate gradient, or with a finite difference (Sec. 3.2), at
+ * lower parameters obtained by a few unrolled gradient steps (Sec. 3.2).
+ *
+ * Conventions
+ *  - Everything crossing this boundary is plain C: PODs, pointers, sizes.  Level descriptors and
+ *    the `widths`/`constraints`/`path`/`per_edge` arrays are HOST memory and are only read during
+ *    the call.  Every other pointer (params, X, y, aux, vectors, ws) is DEVICE memory on the
+ *    current CUDA device, owned by the caller; the library never allocates, frees or keeps a
+ *    pointer after a call returns.
+ *  - Parameter blocks and every flat vector argument (u, q, v_in, out) are fp32.  An MLP block is
+ *    [W_1, b_1, W_2, b_2, ...] with W_l of shape [widths[l+1], widths[l]] row-major and b_l of
+ *    length widths[l+1].  A weight-net block (1-100-1 net of the data-reweighting experiment) is
+ *    [a1(100), b1(100), a2(100), b2(1)].  fp32 vectors must be 16-byte aligned, X 16-byte aligned.
+ *  - `ws` is scratch of at least betty_workspace_size() bytes, 256-byte aligned.  Its first 256
+ *    bytes hold a device status block written by kernels (see betty_poll_status); contents do not
+ *    need to be preserved between calls, but calls sharing one `ws` must not overlap in time.
+ *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
+ *    synchronising.  Argument errors are returned immediately and nothing is enqueued.
+ *    Conditions found on the device (non-finite values, CG breakdown, an expired bounded wait)
+ *    are recorded in the status block and reported by betty_poll_status.
+ *  - One GPU (compute capability 10.0).  There is no CPU fallback.
+ */
+#ifndef BETTY_H_
+#define BETTY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BETTY_OK = 0,
+  BETTY_ERR_INVALID_ARG = 1,  /* null pointer, negative size, unknown enum, bad path */
+  BETTY_ERR_SHAPE = 2,        /* sizes of participants do not fit the cost family */
+  BETTY_ERR_DTYPE = 3,
+  BETTY_ERR_ALIGNMENT = 4,
+  BETTY_ERR_WORKSPACE = 5,    /* ws too small or misaligned */
+  BETTY_ERR_CUDA = 6,         /* a CUDA runtime call failed (launch error, wrong device) */
+  BETTY_ERR_NONFINITE = 7,    /* device: a reduction met Inf/NaN */
+  BETTY_ERR_BREAKDOWN = 8,    /* device: CG met a direction with p^T H p <= 0 */
+  BETTY_ERR_TIMEOUT = 9,      /* device: a bounded wait (mbarrier) expired */
+  BETTY_ERR_UNSUPPORTED = 10  /* combination not implemented */
+} betty_status;
+
+/* Cost families C_k.  "own" = the level's own parameter block. */
+typedef enum {
+  /* App. D.1 lower problem: own w[d]; constraint VECTOR lambda[d].
+   * C = (1/n) sum_i softplus(-y_i x_i.w) + 1/2 sum_j lambda_j w_j^2.  X fp32 [n,d], y fp32 +-1. */
+  BETTY_LOSS_LOGREG_WD = 0,
+  /* App. D.1 upper problem: C = (1/n) sum_i softplus(-y_i x_i.w), w = the first VECTOR constraint. */
+  BETTY_LOSS_LOGREG = 1,
+  /* C = 1/2 |X w - y|^2 + 1/2 sum_j lambda_j w_j^2 (closed-form best response; used to test
+   * solvers, and the indefinite case of CG).  own w[d]; constraint VECTOR lambda[d]; y fp32 [n]. */
+  BETTY_LOSS_QUADRATIC_WD = 2,
+  /* C = 1/2 |X w - y|^2 of the first VECTOR constraint w. */
+  BETTY_LOSS_QUADRATIC = 3,
+  /* App. A "Classifier" (data reweighting): own MLP; optional constraints WEIGHTNET theta and
+   * LOGWD lambda.  C = (1/B) sum_i r_i l_i + 1/2 sum_l exp(lambda_l) |W_l|_F^2, l_i = softmax
+   * cross-entropy of sample i, r_i = sigmoid(weightnet(l_i; theta)) with l_i detached: derivatives
+   * w.r.t. the MLP treat r_i as constants, derivatives w.r.t. theta treat l_i as data.
+   * r_i = 1 without a WEIGHTNET constraint; no decay term without a LOGWD constraint.
+   * X bf16 [n,d], y int32 class ids. */
+  BETTY_LOSS_MLP_CE_REWEIGHT = 4,
+  /* App. A "Reweight": C = (1/B) sum_i l_i of the first MLP constraint on this level's batch. */
+  BETTY_LOSS_MLP_CE = 5,
+  /* C = (1/B) sum_j (sigmoid(weightnet(l_j(w); theta)) - aux_j)^2 + mu/2 |theta|^2 with theta the
+   * WEIGHTNET participant and w the MLP participant (own block or constraints); l_j is NOT
+   * detached.  aux fp32 [n] in {0,1} (1 = label is clean).  X bf16 [n,d], y int32. */
+  BETTY_LOSS_WEIGHTNET_DETECT = 6
+} betty_loss;
+
+typedef enum {
+  BETTY_PARAM_VECTOR = 0,    /* plain vector (logistic/quadratic w, per-feature weight decay) */
+  BETTY_PARAM_MLP = 1,       /* classifier weights, layout above */
+  BETTY_PARAM_WEIGHTNET = 2, /* 301 parameters of the 1-100-1 weight net */
+  BETTY_PARAM_LOGWD = 3      /* per-layer log weight decay, one per MLP layer */
+} betty_param_kind;
+
+typedef enum { BETTY_NEUMANN = 0, BETTY_CG = 1, BETTY_FD = 2 } betty_method;
+typedef enum { BETTY_ACT_RELU = 0, BETTY_ACT_GELU = 1 } betty_activation; /* GELU: erf form */
+typedef enum { BETTY_F32 = 0, BETTY_BF16 = 1, BETTY_I32 = 2 } betty_dtype;
+
+/* Approximation of one best-response Jacobian (Sec. 3.2).
+ *  NEUMANN: q = alpha * sum_{j=0..K} (I - alpha H)^j v   (K Hessian-vector products)
+ *  CG     : K iterations of conjugate gradient on H q = v from q = 0; stops early once
+ *           |r| <= tol*|v|; p^T H p <= 0 stops it and records BETTY_ERR_BREAKDOWN
+ *  FD     : eps = eps0/|v|_2;  -alpha * [dC/dc(x + eps v) - dC/dc(x - eps v)] / (2 eps) */
+typedef struct {
+  int32_t method; /* betty_method */
+  int32_t K;
+  float alpha;
+  float eps0;
+  float tol;
+} betty_method_cfg;
+
+/* One problem P_k. */
+typedef struct betty_level {
+  int32_t loss;         /* betty_loss */
+  int32_t param_kind;   /* betty_param_kind of the own block */
+  float* params;        /* device fp32 [n_params]; updated in place by betty_lower_step */
+  int64_t n_params;
+  const void* X;        /* device, row-major [n, d]; dtype x_dtype */
+  int32_t x_dtype;      /* betty_dtype */
+  int64_t n, d;
+  const void* y;        /* device [n]: fp32 (logistic +-1, quadratic targets) or int32 class ids */
+  const float* aux;     /* device [n] fp32, WEIGHTNET_DETECT only, else NULL */
+  int32_t n_layers;     /* MLP own block: number of weight matrices; else 0 */
+  const int64_t* widths;/* host [n_layers+1]: input width, hidden widths, classes */
+  int32_t activation;   /* betty_activation (hidden layers) */
+  float lr;             /* step size of betty_lower_step */
+  float mu;             /* WEIGHTNET_DETECT ridge term */
+  int32_t n_constraints;
+  const struct betty_level* const* constraints; /* host array: U_k and L_k providers */
+} betty_level;
+
+/* Scratch bytes sufficient for any call below on these levels (Sec. 2: the whole program). */
+betty_status betty_workspace_size(const betty_level* const* levels, int32_t n_levels,
+                                  size_t* bytes);
+
+/* Zero the status block at the head of ws (enqueued on stream).  Call once before first use. */
+betty_status betty_reset_status(void* ws, size_t ws_bytes, void* stream);
+
+/* Synchronises `stream`, reads the status block and returns the first device-side condition
+ * recorded since the last reset (BETTY_OK if none).  cg_iters (host, may be NULL) receives the
+ * iteration count of the most recent CG solve. */
+betty_status betty_poll_status(const void* ws, void* stream, int32_t* cg_iters);
+
+/* Sec. 3.2 (approximating w* by unrolled gradient steps): n_steps times
+ * params <- params - lr * dC/d(params) on the level's batch.  MLP blocks: the gradient is taken
+ * at the bf16-rounded copy of the fp32 master, re-derived every step. */
+betty_status betty_lower_step(const betty_level* L, int32_t n_steps, void* ws, size_t ws_bytes,
+                              void* stream);
+
+/* Eq. 1 "direct gradient": out[wrt->n_params] = dC_L / d(params of wrt), wrt being L itself or
+ * one of its constraints (zeros when C_L does not depend on it). */
+betty_status betty_grad(const betty_level* L, const betty_level* wrt, float* out, void* ws,
+                        size_t ws_bytes, void* stream);
+
+/* Hessian-vector product of Sec. 3.2's implicit methods: Hu = (d2 C_L / d own^2) u. */
+betty_status betty_hvp(const betty_level* L, const float* u, float* Hu, void* ws, size_t ws_bytes,
+                       void* stream);
+
+/* Mixed second-derivative product (the upper-to-lower / lower-to-upper factor of Eq. 2 before the
+ * solve): out[wrt->n_params] = M^T q = d/dc <dC_L/d own, q>, c = params of constraint `wrt`. */
+betty_status betty_mixed_vjp(const betty_level* L, const betty_level* wrt, const float* q,
+                             float* out, void* ws, size_t ws_bytes, void* stream);
+
+/* Eq. 1 for one lower problem:  out[wrt->n_params] = dC_upper/d(wrt) + (d lower^opt / d wrt)^T
+ * dC_upper/d(lower), the Jacobian product by the named approximation.  `wrt` must be a
+ * constraint of `lower` (normally `upper` itself). */
+betty_status betty_hypergrad_neumann(const betty_level* lower, const betty_level* upper,
+                                     const betty_level* wrt, int32_t K, float alpha, float* out,
+                                     void* ws, size_t ws_bytes, void* stream);
+betty_status betty_hypergrad_cg(const betty_level* lower, const betty_level* upper,
+                                const betty_level* wrt, int32_t K, float tol, float* out,
+                                void* ws, size_t ws_bytes, void* stream);
+betty_status betty_hypergrad_fd(const betty_level* lower, const betty_level* upper,
+                                const betty_level* wrt, float eps0, float alpha, float* out,
+                                void* ws, size_t ws_bytes, void* stream);
+
+/* One path term of Eq. 2, evaluated right to left (Sec. 3.2).  path = [k, q(1), ..., q(m)] indexes
+ * `levels`; q(1) is reached from k by the upper-to-lower edge, q(i+1) from q(i) by lower-to-upper
+ * edges; per_edge[i] configures the edge into q(i+1) (per_edge[0]: the upper-to-lower edge).
+ * Start vector: v_in[levels[q(m)]->n_params], or dC_k/d theta_{q(m)} when v_in is NULL.
+ * out[levels[k]->n_params] receives the product (accumulate != 0: is added to out).  The direct
+ * gradient of Eq. 2 is not added.  path_len = m + 1 >= 2. */
+betty_status betty_chain_levels(const betty_level* const* levels, int32_t n_levels,
+                                const int32_t* path, int32_t path_len,
+                                const betty_method_cfg* per_edge, const float* v_in, float* out,
+                                int32_t accumulate, void* ws, size_t ws_bytes, void* stream);
+
+const char* betty_status_string(betty_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BETTY_H_ */

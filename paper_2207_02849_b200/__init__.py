@@ -1,0 +1,15 @@
+"""B200 (sm_100a) library for the hypergradient path of gradient-based multilevel optimisation
+(arXiv 2207.02849): a C-ABI shared library of hand-written CUDA kernels plus this thin ctypes
+binding.  Importing the package does not load the library; the first call does, and fails
+loudly when the library is missing (there is no CPU fallback)."""
+from .binding import (  # noqa: F401
+    BettyError, Level, MethodCfg, Workspace, betty_chain_levels, betty_grad, betty_hvp,
+    betty_hypergrad_cg, betty_hypergrad_fd, betty_hypergrad_neumann, betty_lower_step,
+    betty_mixed_vjp, betty_poll_status, betty_reset_status, betty_status_string,
+    betty_workspace_size, lib, lib_path,
+)
+from . import binding as _b
+
+for _k, _v in vars(_b).items():
+    if _k.startswith(("BETTY_", "LOSS_", "PARAM_", "ACT_")):
+        globals()[_k] = _v

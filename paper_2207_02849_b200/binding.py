@@ -1,0 +1,235 @@
+"""ctypes binding of include/betty.h.  Argument marshalling only: every computation runs in
+the CUDA library.  torch is used for device memory and the current stream."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+
+# ---- enums (mirrors of betty.h) ----
+BETTY_OK = 0
+(BETTY_ERR_INVALID_ARG, BETTY_ERR_SHAPE, BETTY_ERR_DTYPE, BETTY_ERR_ALIGNMENT, BETTY_ERR_WORKSPACE,
+ BETTY_ERR_CUDA, BETTY_ERR_NONFINITE, BETTY_ERR_BREAKDOWN, BETTY_ERR_TIMEOUT,
+ BETTY_ERR_UNSUPPORTED) = range(1, 11)
+(LOSS_LOGREG_WD, LOSS_LOGREG, LOSS_QUADRATIC_WD, LOSS_QUADRATIC, LOSS_MLP_CE_REWEIGHT, LOSS_MLP_CE,
+ LOSS_WEIGHTNET_DETECT) = range(7)
+PARAM_VECTOR, PARAM_MLP, PARAM_WEIGHTNET, PARAM_LOGWD = range(4)
+BETTY_NEUMANN, BETTY_CG, BETTY_FD = range(3)
+ACT_RELU, ACT_GELU = range(2)
+BETTY_F32, BETTY_BF16, BETTY_I32 = range(3)
+
+
+class BettyError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {betty_status_string(status)} (status {status})")
+
+
+class _MethodCfg(C.Structure):
+    _fields_ = [("method", C.c_int32), ("K", C.c_int32), ("alpha", C.c_float), ("eps0", C.c_float),
+                ("tol", C.c_float)]
+
+
+class _Level(C.Structure):
+    pass
+
+
+_Level._fields_ = [
+    ("loss", C.c_int32), ("param_kind", C.c_int32), ("params", C.c_void_p), ("n_params", C.c_int64),
+    ("X", C.c_void_p), ("x_dtype", C.c_int32), ("n", C.c_int64), ("d", C.c_int64),
+    ("y", C.c_void_p), ("aux", C.c_void_p), ("n_layers", C.c_int32), ("widths", C.POINTER(C.c_int64)),
+    ("activation", C.c_int32), ("lr", C.c_float), ("mu", C.c_float), ("n_constraints", C.c_int32),
+    ("constraints", C.POINTER(C.POINTER(_Level))),
+]
+
+_lib = None
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, "libbetty.so")
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built: nothing here falls back to
+    another implementation."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2207_02849_b200.build` "
+                           "(nvcc, sm_100a); this package has no CPU fallback")
+    L = C.CDLL(path)
+    LP, VP, I32, SZ, F = C.POINTER(_Level), C.c_void_p, C.c_int32, C.c_size_t, C.c_float
+    sig = {
+        "betty_workspace_size": [C.POINTER(LP), I32, C.POINTER(SZ)],
+        "betty_reset_status": [VP, SZ, VP],
+        "betty_poll_status": [VP, VP, C.POINTER(I32)],
+        "betty_lower_step": [LP, I32, VP, SZ, VP],
+        "betty_grad": [LP, LP, VP, VP, SZ, VP],
+        "betty_hvp": [LP, VP, VP, VP, SZ, VP],
+        "betty_mixed_vjp": [LP, LP, VP, VP, VP, SZ, VP],
+        "betty_hypergrad_neumann": [LP, LP, LP, I32, F, VP, VP, SZ, VP],
+        "betty_hypergrad_cg": [LP, LP, LP, I32, F, VP, VP, SZ, VP],
+        "betty_hypergrad_fd": [LP, LP, LP, F, F, VP, VP, SZ, VP],
+        "betty_chain_levels": [C.POINTER(LP), I32, C.POINTER(I32), I32, C.POINTER(_MethodCfg), VP, VP, I32,
+                               VP, SZ, VP],
+    }
+    for name, args in sig.items():
+        fn = getattr(L, name)
+        fn.argtypes, fn.restype = args, C.c_int
+    L.betty_status_string.argtypes, L.betty_status_string.restype = [C.c_int], C.c_char_p
+    _lib = L
+    return L
+
+
+def betty_status_string(status: int) -> str:
+    return lib().betty_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != BETTY_OK:
+        raise BettyError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("device tensors must be contiguous CUDA tensors")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+_DT = {torch.float32: BETTY_F32, torch.bfloat16: BETTY_BF16, torch.int32: BETTY_I32}
+
+
+class Level:
+    """Host-side descriptor of one problem P_k: keeps the tensors alive and owns the C struct."""
+
+    def __init__(self, loss: int, param_kind: int, params: torch.Tensor, X: Optional[torch.Tensor] = None,
+                 y: Optional[torch.Tensor] = None, aux: Optional[torch.Tensor] = None,
+                 widths: Optional[Sequence[int]] = None, activation: int = ACT_RELU, lr: float = 0.1,
+                 mu: float = 0.0):
+        self.params, self.X, self.y, self.aux = params, X, y, aux
+        self.widths = tuple(int(w) for w in widths) if widths is not None else None
+        self.constraints: list[Level] = []
+        s = _Level()
+        s.loss, s.param_kind = int(loss), int(param_kind)
+        s.params, s.n_params = _ptr(params), params.numel()
+        s.X = _ptr(X)
+        s.x_dtype = _DT.get(X.dtype, -1) if X is not None else BETTY_F32
+        s.n, s.d = (X.shape[0], X.shape[1]) if X is not None else (0, 0)
+        s.y, s.aux = _ptr(y), _ptr(aux)
+        if self.widths is not None:
+            self._widths = (C.c_int64 * len(self.widths))(*self.widths)
+            s.n_layers, s.widths = len(self.widths) - 1, self._widths
+        else:
+            s.n_layers, s.widths = 0, None
+        s.activation, s.lr, s.mu = int(activation), float(lr), float(mu)
+        s.n_constraints, s.constraints = 0, None
+        self.c = s
+
+    def set_constraints(self, levels: Sequence["Level"]) -> "Level":
+        self.constraints = list(levels)
+        self._carr = (C.POINTER(_Level) * max(1, len(levels)))(*[C.pointer(l.c) for l in levels])
+        self.c.n_constraints = len(levels)
+        self.c.constraints = self._carr if levels else None
+        return self
+
+    @property
+    def ref(self):
+        return C.byref(self.c)
+
+
+class MethodCfg:
+    def __init__(self, method: int, K: int = 0, alpha: float = 1.0, eps0: float = 0.01, tol: float = 0.0):
+        self.c = _MethodCfg(int(method), int(K), float(alpha), float(eps0), float(tol))
+
+
+def _level_array(levels: Sequence[Level]):
+    return (C.POINTER(_Level) * len(levels))(*[C.pointer(l.c) for l in levels])
+
+
+def betty_workspace_size(levels: Sequence[Level]) -> int:
+    out = C.c_size_t(0)
+    _check(lib().betty_workspace_size(_level_array(levels), len(levels), C.byref(out)), "betty_workspace_size")
+    return int(out.value)
+
+
+class Workspace:
+    """Caller-owned scratch (a torch uint8 tensor) sized by betty_workspace_size."""
+
+    def __init__(self, levels: Sequence[Level], device="cuda", extra_bytes: int = 0):
+        self.nbytes = betty_workspace_size(levels) + int(extra_bytes)
+        self.buf = torch.empty(self.nbytes + 256, dtype=torch.uint8, device=device)
+        off = (-self.buf.data_ptr()) % 256
+        self.ptr = self.buf.data_ptr() + off
+        betty_reset_status(self)
+
+
+def betty_reset_status(ws: Workspace, stream=None) -> None:
+    _check(lib().betty_reset_status(ws.ptr, ws.nbytes, _stream(stream)), "betty_reset_status")
+
+
+def betty_poll_status(ws: Workspace, stream=None, raise_on_error: bool = True):
+    """Synchronises the stream; returns (status, cg_iters)."""
+    it = C.c_int32(0)
+    st = lib().betty_poll_status(ws.ptr, _stream(stream), C.byref(it))
+    if raise_on_error:
+        _check(st, "betty_poll_status")
+    return st, int(it.value)
+
+
+def betty_lower_step(L: Level, n_steps: int, ws: Workspace, stream=None) -> None:
+    _check(lib().betty_lower_step(L.ref, int(n_steps), ws.ptr, ws.nbytes, _stream(stream)), "betty_lower_step")
+
+
+def betty_grad(L: Level, wrt: Level, out: torch.Tensor, ws: Workspace, stream=None) -> None:
+    _check(lib().betty_grad(L.ref, wrt.ref, _ptr(out), ws.ptr, ws.nbytes, _stream(stream)), "betty_grad")
+
+
+def betty_hvp(L: Level, u: torch.Tensor, Hu: torch.Tensor, ws: Workspace, stream=None) -> None:
+    _check(lib().betty_hvp(L.ref, _ptr(u), _ptr(Hu), ws.ptr, ws.nbytes, _stream(stream)), "betty_hvp")
+
+
+def betty_mixed_vjp(L: Level, wrt: Level, q: torch.Tensor, out: torch.Tensor, ws: Workspace, stream=None) -> None:
+    _check(lib().betty_mixed_vjp(L.ref, wrt.ref, _ptr(q), _ptr(out), ws.ptr, ws.nbytes, _stream(stream)),
+           "betty_mixed_vjp")
+
+
+def betty_hypergrad_neumann(lower: Level, upper: Level, wrt: Level, K: int, alpha: float, out: torch.Tensor,
+                            ws: Workspace, stream=None) -> None:
+    _check(lib().betty_hypergrad_neumann(lower.ref, upper.ref, wrt.ref, int(K), float(alpha), _ptr(out), ws.ptr,
+                                         ws.nbytes, _stream(stream)), "betty_hypergrad_neumann")
+
+
+def betty_hypergrad_cg(lower: Level, upper: Level, wrt: Level, K: int, tol: float, out: torch.Tensor,
+                       ws: Workspace, stream=None) -> None:
+    _check(lib().betty_hypergrad_cg(lower.ref, upper.ref, wrt.ref, int(K), float(tol), _ptr(out), ws.ptr, ws.nbytes,
+                                    _stream(stream)), "betty_hypergrad_cg")
+
+
+def betty_hypergrad_fd(lower: Level, upper: Level, wrt: Level, eps0: float, alpha: float, out: torch.Tensor,
+                       ws: Workspace, stream=None) -> None:
+    _check(lib().betty_hypergrad_fd(lower.ref, upper.ref, wrt.ref, float(eps0), float(alpha), _ptr(out), ws.ptr,
+                                    ws.nbytes, _stream(stream)), "betty_hypergrad_fd")
+
+
+def betty_chain_levels(levels: Sequence[Level], path: Sequence[int], per_edge: Sequence[MethodCfg],
+                       v_in: Optional[torch.Tensor], out: torch.Tensor, accumulate: bool, ws: Workspace,
+                       stream=None) -> None:
+    arr = _level_array(levels)
+    p = (C.c_int32 * len(path))(*[int(i) for i in path])
+    cfgs = (_MethodCfg * len(per_edge))(*[m.c for m in per_edge])
+    _check(lib().betty_chain_levels(arr, len(levels), p, len(path), cfgs, _ptr(v_in), _ptr(out),
+                                    1 if accumulate else 0, ws.ptr, ws.nbytes, _stream(stream)), "betty_chain_levels")

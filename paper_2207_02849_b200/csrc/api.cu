@@ -1,0 +1,357 @@
+// C ABI entry points: argument validation, dispatch on the cost family, and the host-side
+// drivers of Sec. 3.2's approximations (Neumann series, conjugate gradient, finite difference),
+// Eq. 1 and the right-to-left product along one path of Eq. 2.  Drivers only enqueue kernels;
+// every scalar of the iterations stays on the device.
+#include "ops.cuh"
+
+namespace betty {
+
+// ------------------------------------------------------------------ small kernels
+// out (+)= scale * x
+__global__ void k_scale_into(float* out, const float* x, float scale, int accumulate, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    out[i] = (accumulate ? out[i] : 0.f) + scale * x[i];
+}
+// weight-decay constraint: dC/d(lambda) = 1/2 w^2, so the central difference is evaluated as written,
+// in double to keep the cancellation exact:  out (+)= -alpha*[(w+ev)^2 - (w-ev)^2]/(4e)
+__global__ void k_fd_weight_decay(float* out, const float* w, const float* v, const float* vnorm2, float eps0,
+                                  float alpha, int accumulate, int64_t n) {
+  const double nv = sqrt((double)*vnorm2);
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    float base = accumulate ? out[i] : 0.f;
+    if (nv > 0.0) {
+      const double eps = (double)eps0 / nv;
+      const double wp = (double)w[i] + eps * (double)v[i], wm = (double)w[i] - eps * (double)v[i];
+      base += (float)(-(double)alpha * (0.5 * wp * wp - 0.5 * wm * wm) / (2.0 * eps));
+    }
+    out[i] = base;
+  }
+}
+static inline int ew_grid(int64_t n) {
+  int64_t b = (n + 1023) / 1024;
+  return (int)(b < 1 ? 1 : (b > 2368 ? 2368 : b));
+}
+
+// ------------------------------------------------------------------ vector families
+static const betty_level* vec_w_level(const betty_level* L) {
+  if (L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_QUADRATIC_WD) return L;
+  return find_constraint(L, BETTY_PARAM_VECTOR);
+}
+static inline int vec_family(const betty_level* L) {
+  return (L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_LOGREG) ? 0 : 1;
+}
+static inline bool vec_has_wd(const betty_level* L) {
+  return L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_QUADRATIC_WD;
+}
+
+betty_status vecfam_validate(const betty_level* L) {
+  if (L->n < 0 || L->d <= 0) return BETTY_ERR_SHAPE;
+  if (L->x_dtype != BETTY_F32) return BETTY_ERR_DTYPE;
+  if ((L->n > 0 && (!L->X || !L->y))) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(L->X)) return BETTY_ERR_ALIGNMENT;
+  const betty_level* wl = vec_w_level(L);
+  if (!wl || !wl->params) return BETTY_ERR_INVALID_ARG;
+  if (wl->n_params != L->d) return BETTY_ERR_SHAPE;
+  if (!aligned16(wl->params)) return BETTY_ERR_ALIGNMENT;
+  if (vec_has_wd(L)) {
+    if (L->param_kind != BETTY_PARAM_VECTOR) return BETTY_ERR_INVALID_ARG;
+    const betty_level* lam = find_constraint(L, BETTY_PARAM_VECTOR);
+    if (!lam || !lam->params) return BETTY_ERR_INVALID_ARG;
+    if (lam->n_params != L->d) return BETTY_ERR_SHAPE;
+  }
+  return BETTY_OK;
+}
+
+betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out) {
+  const betty_level* wl = vec_w_level(L);
+  if (wrt == wl) {
+    const float* lam = vec_has_wd(L) ? find_constraint(L, BETTY_PARAM_VECTOR)->params : nullptr;
+    return logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, wl->params, nullptr, lam,
+                       out, nullptr, 0.f);
+  }
+  if (vec_has_wd(L) && wrt == find_constraint(L, BETTY_PARAM_VECTOR))
+    return vec_mul(c, out, 0.5f, L->params, L->params, L->d);
+  return vec_zero(c, out, wrt->n_params);
+}
+
+betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu) {
+  if (!vec_has_wd(L)) return BETTY_ERR_UNSUPPORTED;
+  return logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, u,
+                     find_constraint(L, BETTY_PARAM_VECTOR)->params, Hu, nullptr, 0.f);
+}
+
+betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, const float* q, float* out) {
+  if (!vec_has_wd(L) || wrt != find_constraint(L, BETTY_PARAM_VECTOR)) return BETTY_ERR_INVALID_ARG;
+  return vec_mul(c, out, 1.0f, L->params, q, L->d);
+}
+
+betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps) {
+  if (!vec_has_wd(L)) return BETTY_ERR_UNSUPPORTED;
+  const float* lam = find_constraint(L, BETTY_PARAM_VECTOR)->params;
+  for (int s = 0; s < n_steps; ++s)
+    BETTY_TRY(logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, nullptr, lam,
+                          nullptr, L->params, L->lr));
+  return BETTY_OK;
+}
+
+betty_status vecfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
+                       float eps0, float alpha, float* out, bool accumulate) {
+  if (!vec_has_wd(L) || wrt != find_constraint(L, BETTY_PARAM_VECTOR)) return BETTY_ERR_INVALID_ARG;
+  k_fd_weight_decay<<<ew_grid(L->d), 256, 0, c.stream>>>(out, L->params, v, vnorm2, eps0, alpha, accumulate ? 1 : 0, L->d);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
+// ------------------------------------------------------------------ dispatch
+static betty_status validate_level(const betty_level* L) {
+  if (!L) return BETTY_ERR_INVALID_ARG;
+  if (L->n_constraints < 0 || (L->n_constraints > 0 && !L->constraints)) return BETTY_ERR_INVALID_ARG;
+  for (int i = 0; i < L->n_constraints; ++i)
+    if (!L->constraints[i]) return BETTY_ERR_INVALID_ARG;
+  if (L->n_params < 0 || (L->n_params > 0 && !L->params)) return BETTY_ERR_INVALID_ARG;
+  if (L->param_kind < BETTY_PARAM_VECTOR || L->param_kind > BETTY_PARAM_LOGWD) return BETTY_ERR_INVALID_ARG;
+  if (is_vector_family(L->loss)) return vecfam_validate(L);
+  if (is_mlp_family(L->loss)) return mlpfam_validate(L);
+  return BETTY_ERR_INVALID_ARG;
+}
+
+static bool is_participant(const betty_level* L, const betty_level* wrt) {
+  if (wrt == L) return true;
+  for (int i = 0; i < L->n_constraints; ++i)
+    if (L->constraints[i] == wrt) return true;
+  return false;
+}
+
+static betty_status check_ws(void* ws, size_t ws_bytes) {
+  if (!ws || ws_bytes < sizeof(StatusBlock)) return BETTY_ERR_WORKSPACE;
+  if (((uintptr_t)ws) & 255u) return BETTY_ERR_WORKSPACE;
+  return BETTY_OK;
+}
+
+static betty_status level_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out) {
+  if (is_vector_family(L->loss)) return vecfam_grad(c, L, wrt, out);
+  return mlpfam_grad(c, L, wrt, out);
+}
+
+// (d x*/d c)^T v by the configured approximation; out (+)= result.
+static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v,
+                        const betty_method_cfg& cfg, float* out, bool accumulate) {
+  if (!is_participant(L, wrt) || wrt == L) return BETTY_ERR_INVALID_ARG;
+  const int64_t n = L->n_params, nc = wrt->n_params;
+  const bool vecfam = is_vector_family(L->loss);
+  const size_t mark = c.arena.mark();
+  BETTY_ALLOC(partials, float, c, (size_t)vec_dot_partials(n));
+  BETTY_TRY(vec_reduce_init(c, partials));
+  betty_status rc = BETTY_OK;
+  if (cfg.method == BETTY_FD) {
+    BETTY_ALLOC(st, SolveState, c, 1);
+    BETTY_TRY(vec_dot(c, v, v, n, &st->vnorm2, partials));
+    rc = vecfam ? vecfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, out, accumulate)
+                : mlpfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, out, accumulate);
+    c.arena.release(mark);
+    return rc;
+  }
+  if (cfg.method != BETTY_NEUMANN && cfg.method != BETTY_CG) return BETTY_ERR_INVALID_ARG;
+  if (cfg.K < 0) return BETTY_ERR_INVALID_ARG;
+  MlpHvpCache* cache = nullptr;
+  if (!vecfam) BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
+  BETTY_ALLOC(q, float, c, (size_t)n);
+  BETTY_ALLOC(h, float, c, (size_t)n);
+  BETTY_ALLOC(m, float, c, (size_t)nc);
+  float qscale = 1.f;
+  if (cfg.method == BETTY_NEUMANN) {
+    BETTY_ALLOC(t, float, c, (size_t)n);
+    BETTY_TRY(vec_copy(c, t, v, n));
+    BETTY_TRY(vec_copy(c, q, v, n));
+    for (int k = 0; k < cfg.K; ++k) {
+      BETTY_TRY(vecfam ? vecfam_hvp(c, L, t, h) : mlpfam_hvp(c, L, cache, t, h));
+      BETTY_TRY(neumann_update(c, t, q, h, cfg.alpha, n));
+    }
+    qscale = cfg.alpha;   // q holds the plain sum; alpha is applied with the sign below
+  } else {
+    BETTY_ALLOC(st, SolveState, c, 1);
+    BETTY_ALLOC(r, float, c, (size_t)n);
+    BETTY_ALLOC(p, float, c, (size_t)n);
+    BETTY_TRY(cg_init(c, st, v, q, r, p, cfg.tol, n, partials));
+    for (int k = 0; k < cfg.K; ++k) {
+      BETTY_TRY(vecfam ? vecfam_hvp(c, L, p, h) : mlpfam_hvp(c, L, cache, p, h));
+      BETTY_TRY(cg_step(c, st, q, r, p, h, n, partials));
+    }
+  }
+  BETTY_TRY(vecfam ? vecfam_mixed(c, L, wrt, q, m) : mlpfam_mixed(c, L, cache, wrt, q, m));
+  k_scale_into<<<ew_grid(nc), 256, 0, c.stream>>>(out, m, -qscale, accumulate ? 1 : 0, nc);
+  BETTY_LAUNCH_CHECK();
+  c.arena.release(mark);
+  return BETTY_OK;
+}
+
+static betty_status hypergrad(const betty_level* lower, const betty_level* upper, const betty_level* wrt,
+                              const betty_method_cfg& cfg, float* out, void* ws, size_t ws_bytes, void* stream) {
+  BETTY_TRY(validate_level(lower));
+  BETTY_TRY(validate_level(upper));
+  if (!wrt || !out) return BETTY_ERR_INVALID_ARG;
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  if (!is_participant(upper, lower) || !is_participant(upper, wrt) || !is_participant(lower, wrt) || wrt == lower)
+    return BETTY_ERR_INVALID_ARG;
+  Ctx c(ws, ws_bytes, stream);
+  BETTY_ALLOC(v, float, c, (size_t)lower->n_params);
+  BETTY_TRY(level_grad(c, upper, lower, v));     // dC_u / d theta_lower
+  BETTY_TRY(level_grad(c, upper, wrt, out));     // direct gradient
+  return brj(c, lower, wrt, v, cfg, out, true);
+}
+
+}  // namespace betty
+
+using namespace betty;
+
+extern "C" {
+
+const char* betty_status_string(betty_status s) {
+  switch (s) {
+    case BETTY_OK: return "ok";
+    case BETTY_ERR_INVALID_ARG: return "invalid argument";
+    case BETTY_ERR_SHAPE: return "shape mismatch";
+    case BETTY_ERR_DTYPE: return "unsupported dtype";
+    case BETTY_ERR_ALIGNMENT: return "misaligned pointer";
+    case BETTY_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case BETTY_ERR_CUDA: return "CUDA runtime error";
+    case BETTY_ERR_NONFINITE: return "non-finite value met on the device";
+    case BETTY_ERR_BREAKDOWN: return "conjugate gradient breakdown (p^T H p <= 0)";
+    case BETTY_ERR_TIMEOUT: return "bounded device wait expired";
+    case BETTY_ERR_UNSUPPORTED: return "unsupported combination";
+  }
+  return "unknown status";
+}
+
+betty_status betty_workspace_size(const betty_level* const* levels, int32_t n_levels, size_t* bytes) {
+  if (!levels || n_levels <= 0 || !bytes) return BETTY_ERR_INVALID_ARG;
+  size_t total = 1 << 20;
+  size_t maxp = 0;
+  for (int i = 0; i < n_levels; ++i) {
+    const betty_level* L = levels[i];
+    if (!L) return BETTY_ERR_INVALID_ARG;
+    if ((size_t)L->n_params > maxp) maxp = (size_t)L->n_params;
+    if (is_vector_family(L->loss)) {
+      // per-CTA column partials of the streaming pass (2 CTAs per SM) or the fallback's row scratch
+      size_t d = (size_t)(L->d > 0 ? L->d : 1), n = (size_t)(L->n > 0 ? L->n : 1);
+      size_t need = (2 * 148 + 64) * d * sizeof(float) + n * sizeof(float) + 4096;
+      if (need > total) total = need + (1 << 20);
+    } else if (is_mlp_family(L->loss)) {
+      total += mlpfam_workspace(L);
+    } else {
+      return BETTY_ERR_INVALID_ARG;
+    }
+  }
+  // solver vectors: v, q, h, t/r, p, m plus chain intermediates, each padded
+  total += 10 * (maxp * sizeof(float) + 256) + (1 << 16);
+  *bytes = (total + 255) & ~size_t(255);
+  return BETTY_OK;
+}
+
+betty_status betty_reset_status(void* ws, size_t ws_bytes, void* stream) {
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  if (cudaMemsetAsync(ws, 0, sizeof(StatusBlock), (cudaStream_t)stream) != cudaSuccess) return BETTY_ERR_CUDA;
+  return BETTY_OK;
+}
+
+betty_status betty_poll_status(const void* ws, void* stream, int32_t* cg_iters) {
+  if (!ws) return BETTY_ERR_WORKSPACE;
+  StatusBlock h;
+  if (cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess) return BETTY_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BETTY_ERR_CUDA;
+  if (cg_iters) *cg_iters = h.cg_iters;
+  if (h.code < 0 || h.code > BETTY_ERR_UNSUPPORTED) return BETTY_ERR_CUDA;
+  return (betty_status)h.code;
+}
+
+betty_status betty_lower_step(const betty_level* L, int32_t n_steps, void* ws, size_t ws_bytes, void* stream) {
+  BETTY_TRY(validate_level(L));
+  if (n_steps < 0) return BETTY_ERR_INVALID_ARG;
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  Ctx c(ws, ws_bytes, stream);
+  if (is_vector_family(L->loss)) return vecfam_lower_step(c, L, n_steps);
+  return mlpfam_lower_step(c, L, n_steps);
+}
+
+betty_status betty_grad(const betty_level* L, const betty_level* wrt, float* out, void* ws, size_t ws_bytes,
+                        void* stream) {
+  BETTY_TRY(validate_level(L));
+  if (!wrt || !out || !is_participant(L, wrt)) return BETTY_ERR_INVALID_ARG;
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  Ctx c(ws, ws_bytes, stream);
+  return level_grad(c, L, wrt, out);
+}
+
+betty_status betty_hvp(const betty_level* L, const float* u, float* Hu, void* ws, size_t ws_bytes, void* stream) {
+  BETTY_TRY(validate_level(L));
+  if (!u || !Hu) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(u) || !aligned16(Hu)) return BETTY_ERR_ALIGNMENT;
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  Ctx c(ws, ws_bytes, stream);
+  if (is_vector_family(L->loss)) return vecfam_hvp(c, L, u, Hu);
+  MlpHvpCache* cache = nullptr;
+  BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
+  return mlpfam_hvp(c, L, cache, u, Hu);
+}
+
+betty_status betty_mixed_vjp(const betty_level* L, const betty_level* wrt, const float* q, float* out, void* ws,
+                             size_t ws_bytes, void* stream) {
+  BETTY_TRY(validate_level(L));
+  if (!wrt || !q || !out || !is_participant(L, wrt) || wrt == L) return BETTY_ERR_INVALID_ARG;
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  Ctx c(ws, ws_bytes, stream);
+  if (is_vector_family(L->loss)) return vecfam_mixed(c, L, wrt, q, out);
+  MlpHvpCache* cache = nullptr;
+  BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
+  return mlpfam_mixed(c, L, cache, wrt, q, out);
+}
+
+betty_status betty_hypergrad_neumann(const betty_level* lower, const betty_level* upper, const betty_level* wrt,
+                                     int32_t K, float alpha, float* out, void* ws, size_t ws_bytes, void* stream) {
+  betty_method_cfg cfg = {BETTY_NEUMANN, K, alpha, 0.f, 0.f};
+  return hypergrad(lower, upper, wrt, cfg, out, ws, ws_bytes, stream);
+}
+
+betty_status betty_hypergrad_cg(const betty_level* lower, const betty_level* upper, const betty_level* wrt, int32_t K,
+                                float tol, float* out, void* ws, size_t ws_bytes, void* stream) {
+  betty_method_cfg cfg = {BETTY_CG, K, 0.f, 0.f, tol};
+  return hypergrad(lower, upper, wrt, cfg, out, ws, ws_bytes, stream);
+}
+
+betty_status betty_hypergrad_fd(const betty_level* lower, const betty_level* upper, const betty_level* wrt, float eps0,
+                                float alpha, float* out, void* ws, size_t ws_bytes, void* stream) {
+  if (!(eps0 > 0.f)) return BETTY_ERR_INVALID_ARG;
+  betty_method_cfg cfg = {BETTY_FD, 0, alpha, eps0, 0.f};
+  return hypergrad(lower, upper, wrt, cfg, out, ws, ws_bytes, stream);
+}
+
+betty_status betty_chain_levels(const betty_level* const* levels, int32_t n_levels, const int32_t* path,
+                                int32_t path_len, const betty_method_cfg* per_edge, const float* v_in, float* out,
+                                int32_t accumulate, void* ws, size_t ws_bytes, void* stream) {
+  if (!levels || n_levels <= 0 || !path || path_len < 2 || !per_edge || !out) return BETTY_ERR_INVALID_ARG;
+  for (int i = 0; i < path_len; ++i)
+    if (path[i] < 0 || path[i] >= n_levels || !levels[path[i]]) return BETTY_ERR_INVALID_ARG;
+  for (int i = 0; i < path_len; ++i) BETTY_TRY(validate_level(levels[path[i]]));
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  Ctx c(ws, ws_bytes, stream);
+  const betty_level* K = levels[path[0]];
+  const int m = path_len - 1;
+  const betty_level* last = levels[path[m]];
+  const float* v = v_in;
+  if (!v) {
+    if (!is_participant(K, last)) return BETTY_ERR_INVALID_ARG;
+    BETTY_ALLOC(v0, float, c, (size_t)last->n_params);
+    BETTY_TRY(level_grad(c, K, last, v0));
+    v = v0;
+  }
+  for (int i = m; i >= 2; --i) {
+    const betty_level* Li = levels[path[i]];
+    const betty_level* Lprev = levels[path[i - 1]];
+    BETTY_ALLOC(vn, float, c, (size_t)Lprev->n_params);
+    BETTY_TRY(brj(c, Li, Lprev, v, per_edge[i - 1], vn, false));
+    v = vn;
+  }
+  return brj(c, levels[path[1]], K, v, per_edge[0], out, accumulate != 0);
+}
+
+}  // extern "C"

@@ -1,0 +1,104 @@
+// Shared host/device helpers of the library: workspace arena, status block, launch checks.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "betty.h"
+
+namespace betty {
+
+typedef __nv_bfloat16 bf16;
+
+// Device status block: the first 256 bytes of the caller's workspace.
+struct StatusBlock {
+  int32_t code;      // first device-side condition (betty_status), 0 if none
+  int32_t cg_iters;  // iterations done by the most recent CG solve
+  int32_t pad[62];
+};
+static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
+
+// State of one inverse-Hessian solve, kept on the device so that no host sync is needed.
+struct SolveState {
+  float rho;       // r.r
+  float gamma;     // p.Hp
+  float rho_new;
+  float stop;      // tol^2 * v.v
+  float vnorm2;    // v.v (FD: |v|^2)
+  int32_t active;  // 1 while iterations still update the iterate
+  int32_t iters;
+  int32_t pad;
+};
+
+__device__ __forceinline__ void record_status(StatusBlock* sb, int32_t code) {
+  atomicCAS(&sb->code, 0, code);
+}
+
+// Bump allocator over the caller's workspace.  Nothing is ever freed inside a call.
+struct Arena {
+  char* base;
+  size_t size;
+  size_t off;
+  bool overflow;
+  __host__ Arena(void* b, size_t s) : base((char*)b), size(s), off(sizeof(StatusBlock)), overflow(false) {}
+  template <typename T>
+  __host__ T* alloc(size_t count) {
+    size_t bytes = (count * sizeof(T) + 255) & ~size_t(255);
+    if (off + bytes > size) { overflow = true; return nullptr; }
+    T* p = (T*)(base + off);
+    off += bytes;
+    return p;
+  }
+  __host__ size_t mark() const { return off; }
+  __host__ void release(size_t m) { off = m; }
+  __host__ StatusBlock* status() const { return (StatusBlock*)base; }
+};
+
+struct Ctx {
+  cudaStream_t stream;
+  Arena arena;
+  int sm_count;
+  __host__ Ctx(void* ws, size_t ws_bytes, void* s) : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(148) {}
+};
+
+#define BETTY_TRY(expr)                       \
+  do {                                        \
+    betty_status _s = (expr);                 \
+    if (_s != BETTY_OK) return _s;            \
+  } while (0)
+
+#define BETTY_LAUNCH_CHECK()                                   \
+  do {                                                         \
+    if (cudaPeekAtLastError() != cudaSuccess) {                \
+      (void)cudaGetLastError();                                \
+      return BETTY_ERR_CUDA;                                   \
+    }                                                          \
+  } while (0)
+
+#define BETTY_ALLOC(var, T, ctx, count)                        \
+  T* var = (ctx).arena.template alloc<T>(count);               \
+  if (!(var)) return BETTY_ERR_WORKSPACE;
+
+static inline bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
+
+// ---- vector kernels (vec.cu); all vectors fp32, scalars stay on the device ----
+betty_status vec_zero(Ctx& c, float* x, int64_t n);
+betty_status vec_copy(Ctx& c, float* dst, const float* src, int64_t n);
+// out = a*x + b*y (y may be null => a*x); in-place allowed
+betty_status vec_axpby(Ctx& c, float* out, float a, const float* x, float b, const float* y, int64_t n);
+// out = x * y (elementwise), scaled by a
+betty_status vec_mul(Ctx& c, float* out, float a, const float* x, const float* y, int64_t n);
+// *result = x.y, deterministic two-phase; records NONFINITE
+betty_status vec_dot(Ctx& c, const float* x, const float* y, int64_t n, float* result, float* partials);
+int64_t vec_dot_partials(int64_t n);
+// Neumann: t <- t - alpha*Ht ; s <- s + t
+betty_status neumann_update(Ctx& c, float* t, float* s, const float* Ht, float alpha, int64_t n);
+// CG pieces driven by a SolveState on the device
+betty_status cg_init(Ctx& c, SolveState* st, const float* v, float* q, float* r, float* p, float tol,
+                     int64_t n, float* partials);
+betty_status cg_step(Ctx& c, SolveState* st, float* q, float* r, float* p, const float* h, int64_t n,
+                     float* partials);
+// zero the ticket counters that live behind a partials buffer; once per buffer per call
+betty_status vec_reduce_init(Ctx& c, float* partials);
+
+}  // namespace betty

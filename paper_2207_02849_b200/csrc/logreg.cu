@@ -1,0 +1,305 @@
+// Fused row-streaming pass for the logistic / least-squares cost families (App. D.1 problem):
+//   gradient   g  = X^T c(z)        with z = X w,  c_i = -y_i sigmoid(-y_i z_i)/n   (logistic)
+//   HVP        Hu = X^T (s(z) . Xu) with s_i = sigmoid(z_i) sigmoid(-z_i)/n         (logistic)
+// and the analogous forms for 1/2|Xw-y|^2 (c_i = z_i - y_i, s_i = 1).  X is read from HBM exactly
+// once per pass: a tile of rows is brought into shared memory by a bulk asynchronous copy (TMA,
+// mbarrier completion), each thread keeps its columns of the tile in registers between the row dot
+// products and the scaled accumulation, and per-CTA column sums are reduced in a fixed order by a
+// small second kernel that also applies the weight-decay term and, for a lower-level step, the
+// gradient-descent update.
+#include "common.cuh"
+
+namespace betty {
+
+static constexpr int LR_THREADS = 256;
+static constexpr int LR_R = 2;       // rows per tile
+static constexpr int LR_S = 3;       // pipeline stages
+static constexpr int LR_WARPS = LR_THREADS / 32;
+static constexpr uint32_t SPIN_LIMIT = 1u << 22;
+
+struct LrArgs {
+  const float* X; const float* y; int64_t n; int64_t d;
+  const float* w; const float* u;
+  float* partials;       // [gridDim.x][d]
+  int family;            // 0 logistic, 1 least squares
+  float inv_n;
+  StatusBlock* sb;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within SPIN_LIMIT polls.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  for (uint32_t i = 0; i < SPIN_LIMIT; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ float sigmoidf_(float t) { return 1.f / (1.f + __expf(-t)); }
+
+// coefficient multiplying row i in the accumulation
+template <bool HVP>
+__device__ __forceinline__ float row_coef(int family, float z, float t, float y, float inv_n) {
+  if (family == 0) {
+    if (HVP) { float s = sigmoidf_(z); return s * (1.f - s) * t * inv_n; }
+    return -y * sigmoidf_(-y * z) * inv_n;
+  }
+  return HVP ? t : (z - y);
+}
+
+// NCH: float4 column chunks per thread (d <= 1024*NCH, d % 4 == 0)
+template <int NCH, bool HVP>
+__global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int64_t d = a.d;
+  const int d4 = (int)(d >> 2);
+  const size_t tile_floats = (size_t)LR_R * d;
+  float* tiles = (float*)smem;
+  uint64_t* full = (uint64_t*)(smem + LR_S * tile_floats * sizeof(float));
+  float* red = (float*)(full + LR_S);     // [2][LR_WARPS][2*LR_R]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  float4 wv[NCH], uv[NCH], acc[NCH];
+#pragma unroll
+  for (int k = 0; k < NCH; ++k) {
+    int c4 = tid + k * LR_THREADS;
+    wv[k] = (c4 < d4) ? __ldg((const float4*)a.w + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    uv[k] = (HVP && c4 < d4) ? __ldg((const float4*)a.u + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+
+  const int64_t ntiles = (a.n + LR_R - 1) / LR_R;
+  if (tid == 0) {
+    for (int s = 0; s < LR_S; ++s) mbar_init(&full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  auto issue = [&](int s, int64_t t) {
+    int64_t rows = a.n - t * LR_R; if (rows > LR_R) rows = LR_R;
+    uint32_t bytes = (uint32_t)(rows * d * sizeof(float));
+    mbar_expect_tx(&full[s], bytes);
+    bulk_load(tiles + (size_t)s * tile_floats, a.X + (size_t)t * LR_R * d, bytes, &full[s]);
+  };
+  if (tid == 0) {
+    for (int s = 0; s < LR_S; ++s) {
+      int64_t t = blockIdx.x + (int64_t)s * gridDim.x;
+      if (t < ntiles) issue(s, t);
+    }
+  }
+
+  int buf = 0;
+  bool timed_out = false;
+  int64_t i = 0;
+  for (;; ++i) {
+    const int64_t t = blockIdx.x + i * gridDim.x;
+    if (t >= ntiles) break;
+    const int s = (int)(i % LR_S);
+    const uint32_t parity = (uint32_t)((i / LR_S) & 1);
+    const bool landed = mbar_wait_bounded(&full[s], parity);
+    int rows = (int)((a.n - t * LR_R) < LR_R ? (a.n - t * LR_R) : LR_R);
+    const float4* tile4 = (const float4*)(tiles + (size_t)s * tile_floats);
+    float4 x[LR_R][NCH];
+    float pz[LR_R], pt[LR_R];
+#pragma unroll
+    for (int r = 0; r < LR_R; ++r) {
+      pz[r] = 0.f; pt[r] = 0.f;
+#pragma unroll
+      for (int k = 0; k < NCH; ++k) {
+        int c4 = tid + k * LR_THREADS;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c4 < d4 && r < rows) v = tile4[(size_t)r * d4 + c4];
+        x[r][k] = v;
+        pz[r] += v.x * wv[k].x + v.y * wv[k].y + v.z * wv[k].z + v.w * wv[k].w;
+        if (HVP) pt[r] += v.x * uv[k].x + v.y * uv[k].y + v.z * uv[k].z + v.w * uv[k].w;
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < LR_R; ++r) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        pz[r] += __shfl_xor_sync(0xffffffffu, pz[r], o);
+        if (HVP) pt[r] += __shfl_xor_sync(0xffffffffu, pt[r], o);
+      }
+    }
+    float* rb = red + buf * (LR_WARPS * 2 * LR_R);
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < LR_R; ++r) { rb[warp * 2 * LR_R + 2 * r] = pz[r]; rb[warp * 2 * LR_R + 2 * r + 1] = pt[r]; }
+    }
+    // every thread has copied its part of stage s into registers; the same barrier makes the
+    // verdict on an expired wait uniform across the CTA
+    if (__syncthreads_or(!landed)) { timed_out = true; break; }
+    if (tid == 0) {
+      const int64_t tn = t + (int64_t)LR_S * gridDim.x;
+      if (tn < ntiles) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        issue(s, tn);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < LR_R; ++r) {
+      float z = 0.f, tt = 0.f;
+#pragma unroll
+      for (int wi = 0; wi < LR_WARPS; ++wi) { z += rb[wi * 2 * LR_R + 2 * r]; tt += rb[wi * 2 * LR_R + 2 * r + 1]; }
+      float c = 0.f;
+      if (r < rows) c = row_coef<HVP>(a.family, z, tt, a.family == 0 && HVP ? 0.f : __ldg(a.y + t * LR_R + r), a.inv_n);
+#pragma unroll
+      for (int k = 0; k < NCH; ++k) {
+        acc[k].x += c * x[r][k].x; acc[k].y += c * x[r][k].y; acc[k].z += c * x[r][k].z; acc[k].w += c * x[r][k].w;
+      }
+    }
+    buf ^= 1;
+  }
+  if (timed_out) {
+    if (tid == 0) {
+      record_status(a.sb, BETTY_ERR_TIMEOUT);
+      // give copies that are still in flight a bounded chance to land before the CTA exits
+      for (int64_t j = i; j < i + LR_S; ++j) {
+        if (blockIdx.x + j * gridDim.x >= ntiles) break;
+        (void)mbar_wait_bounded(&full[j % LR_S], (uint32_t)((j / LR_S) & 1));
+      }
+    }
+    __syncthreads();
+  }
+  float4* out4 = (float4*)(a.partials + (size_t)blockIdx.x * d);
+#pragma unroll
+  for (int k = 0; k < NCH; ++k) {
+    int c4 = tid + k * LR_THREADS;
+    if (c4 < d4) out4[c4] = acc[k];
+  }
+}
+
+// ---- fallback for any d (odd widths, d > 4096): two passes over X with plain loads ----
+template <bool HVP>
+__global__ void k_rowcoef(LrArgs a, float* coef) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t i = warp; i < a.n; i += nwarps) {
+    const float* xr = a.X + (size_t)i * a.d;
+    float z = 0.f, t = 0.f;
+    for (int64_t j = lane; j < a.d; j += 32) {
+      float xv = xr[j];
+      z += xv * a.w[j];
+      if (HVP) t += xv * a.u[j];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      z += __shfl_xor_sync(0xffffffffu, z, o);
+      if (HVP) t += __shfl_xor_sync(0xffffffffu, t, o);
+    }
+    if (lane == 0) coef[i] = row_coef<HVP>(a.family, z, t, a.family == 0 && HVP ? 0.f : a.y[i], a.inv_n);
+  }
+}
+__global__ void k_colacc(LrArgs a, const float* coef) {
+  const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const int64_t rows_per = (a.n + gridDim.y - 1) / gridDim.y;
+  const int64_t r0 = blockIdx.y * rows_per;
+  int64_t r1 = r0 + rows_per; if (r1 > a.n) r1 = a.n;
+  if (j >= a.d) return;
+  float acc = 0.f;
+  for (int64_t i = r0; i < r1; ++i) acc += coef[i] * a.X[(size_t)i * a.d + j];
+  a.partials[(size_t)blockIdx.y * a.d + j] = acc;
+}
+
+// out_j = sum_c partials[c][j] + lam_j * vec_j ; optionally w_j <- w_j - lr * (that)
+__global__ void k_logreg_finalize(const float* partials, int nparts, int64_t d, const float* lam, const float* vec,
+                                  float* out, float* w_update, float lr) {
+  __shared__ float sh[8][32];
+  const int cx = threadIdx.x & 31, sl = threadIdx.x >> 5;
+  const int64_t j = blockIdx.x * 32 + cx;
+  float acc = 0.f;
+  if (j < d) {
+    const int per = (nparts + 7) / 8;
+    const int c0 = sl * per, c1 = min(nparts, c0 + per);
+    for (int c = c0; c < c1; ++c) acc += partials[(size_t)c * d + j];
+  }
+  sh[sl][cx] = acc;
+  __syncthreads();
+  if (sl == 0 && j < d) {
+    float g = 0.f;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) g += sh[s][cx];
+    if (lam) g += lam[j] * vec[j];
+    if (out) out[j] = g;
+    if (w_update) w_update[j] = w_update[j] - lr * g;
+  }
+}
+
+template <int NCH, bool HVP>
+static betty_status launch_stream(Ctx& c, const LrArgs& a, int grid) {
+  size_t smem = (size_t)LR_S * LR_R * a.d * sizeof(float) + LR_S * sizeof(uint64_t) + 2 * LR_WARPS * 2 * LR_R * sizeof(float);
+  auto kern = k_logreg_stream<NCH, HVP>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BETTY_ERR_CUDA;
+  kern<<<grid, LR_THREADS, smem, c.stream>>>(a);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
+// One streaming pass.  u == nullptr: gradient form, else HVP form.  lam (nullable) adds lam.*w
+// (gradient) or lam.*u (HVP).  out (nullable) receives the vector; w_update (nullable) is
+// decremented by lr times it.
+betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
+                         const float* u, const float* lam, float* out, float* w_update, float lr) {
+  if (d <= 0) return BETTY_OK;
+  LrArgs a;
+  a.X = X; a.y = y; a.n = n; a.d = d; a.w = w; a.u = u; a.family = family;
+  a.inv_n = n > 0 ? 1.0f / (float)n : 0.f;
+  a.sb = c.arena.status();
+  const size_t mark = c.arena.mark();
+  int nparts;
+  const bool fast = (d % 4 == 0) && d <= 4096 && aligned16(X) && aligned16(w) && (!u || aligned16(u));
+  if (fast) {
+    const int64_t ntiles = (n + LR_R - 1) / LR_R;
+    int grid = 2 * c.sm_count;
+    if (ntiles < grid) grid = ntiles > 0 ? (int)ntiles : 1;
+    nparts = grid;
+    BETTY_ALLOC(partials, float, c, (size_t)grid * d);
+    a.partials = partials;
+    betty_status s;
+    const bool hv = u != nullptr;
+    if (d <= 1024) s = hv ? launch_stream<1, true>(c, a, grid) : launch_stream<1, false>(c, a, grid);
+    else if (d <= 2048) s = hv ? launch_stream<2, true>(c, a, grid) : launch_stream<2, false>(c, a, grid);
+    else s = hv ? launch_stream<4, true>(c, a, grid) : launch_stream<4, false>(c, a, grid);
+    BETTY_TRY(s);
+  } else {
+    int64_t want = (n + 255) / 256; if (want < 1) want = 1; if (want > 64) want = 64;
+    nparts = (int)want;
+    BETTY_ALLOC(partials, float, c, (size_t)nparts * d);
+    BETTY_ALLOC(coef, float, c, (size_t)(n > 0 ? n : 1));
+    a.partials = partials;
+    int rb = (int)((n + 7) / 8); if (rb < 1) rb = 1; if (rb > 148 * 8) rb = 148 * 8;
+    if (u) k_rowcoef<true><<<rb, 256, 0, c.stream>>>(a, coef); else k_rowcoef<false><<<rb, 256, 0, c.stream>>>(a, coef);
+    BETTY_LAUNCH_CHECK();
+    dim3 g((unsigned)((d + 255) / 256), (unsigned)nparts);
+    k_colacc<<<g, 256, 0, c.stream>>>(a, coef);
+    BETTY_LAUNCH_CHECK();
+  }
+  k_logreg_finalize<<<(unsigned)((d + 31) / 32), 256, 0, c.stream>>>(a.partials, nparts, d, lam, u ? u : w, out, w_update, lr);
+  BETTY_LAUNCH_CHECK();
+  c.arena.release(mark);
+  return BETTY_OK;
+}
+
+}  // namespace betty

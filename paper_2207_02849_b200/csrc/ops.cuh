@@ -1,0 +1,52 @@
+// Per-cost-family operations behind the C ABI.  Each function enqueues kernels on ctx.stream
+// and allocates its scratch from ctx.arena.
+#pragma once
+#include "common.cuh"
+
+namespace betty {
+
+static inline const betty_level* find_constraint(const betty_level* L, int kind) {
+  for (int i = 0; i < L->n_constraints; ++i)
+    if (L->constraints[i] && L->constraints[i]->param_kind == kind) return L->constraints[i];
+  return nullptr;
+}
+static inline const betty_level* find_participant(const betty_level* L, int kind) {
+  if (L->param_kind == kind) return L;
+  return find_constraint(L, kind);
+}
+static inline bool is_vector_family(int loss) {
+  return loss == BETTY_LOSS_LOGREG_WD || loss == BETTY_LOSS_LOGREG || loss == BETTY_LOSS_QUADRATIC_WD ||
+         loss == BETTY_LOSS_QUADRATIC;
+}
+static inline bool is_mlp_family(int loss) {
+  return loss == BETTY_LOSS_MLP_CE_REWEIGHT || loss == BETTY_LOSS_MLP_CE || loss == BETTY_LOSS_WEIGHTNET_DETECT;
+}
+
+// logreg.cu
+betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
+                         const float* u, const float* lam, float* out, float* w_update, float lr);
+
+// ---- vector families (api.cu) ----
+betty_status vecfam_validate(const betty_level* L);
+betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);
+betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu);
+betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, const float* q, float* out);
+betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps);
+// out (+)= -alpha*[dC/dc(x+eps v) - dC/dc(x-eps v)]/(2 eps), eps = eps0/sqrt(*vnorm2) on the device
+betty_status vecfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
+                       float eps0, float alpha, float* out, bool accumulate);
+
+// ---- MLP families (mlp.cu) ----
+struct MlpHvpCache;  // base forward/backward state shared by the HVPs of one solve
+betty_status mlpfam_validate(const betty_level* L);
+size_t mlpfam_workspace(const betty_level* L);
+betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);
+betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache);
+betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* u, float* Hu);
+betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* cache, const betty_level* wrt, const float* q,
+                          float* out);
+betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps);
+betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
+                       float eps0, float alpha, float* out, bool accumulate);
+
+}  // namespace betty

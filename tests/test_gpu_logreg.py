@@ -1,0 +1,176 @@
+"""Parity of the CUDA path with the fp64 oracle for the logistic / quadratic families
+(App. D.1 problem): element-by-element on the same seeded inputs, through the C ABI.
+Tolerance: relative L2 error <= 1e-4 for fp32 hypergradients."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from tests import oracle_build as ob
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def bt():
+    import paper_2207_02849_b200 as bt
+    return bt
+
+
+def _pair(inp):
+    from tests import cuda_build as cb
+    return cb.logreg_levels(inp), ob.logreg_levels(inp)
+
+
+def _vec(n):
+    return torch.empty(n, dtype=torch.float32, device="cuda")
+
+
+SHAPES = [
+    (1024, 64, 256),      # the small configuration
+    (37, 64, 5),          # fewer rows than CTAs
+    (2051, 4096, 513),    # full width, several tiles per CTA and a ragged last tile
+    (1000, 2048, 300), (777, 1024, 100), (333, 516, 64),
+    (257, 130, 33),       # d % 4 != 0: two-pass kernels
+    (300, 4100, 40),      # d > 4096: two-pass kernels
+    (1, 8, 1),
+]
+
+
+@pytest.mark.parametrize("n,d,nv", SHAPES)
+def test_primitives_match_oracle(bt, n, d, nv):
+    from tests import cuda_build as cb
+    inp = si.logreg_bilevel(100 + n + d, n, d, nv)
+    inp.w0 = si.normal_f32(7, 1, (d,)) * np.float32(0.5 / np.sqrt(d))
+    inp.lam = (np.abs(si.normal_f32(7, 2, (d,))) * 0.05 + 0.01).astype(np.float32)
+    (w, lam), (ow, olam) = _pair(inp)
+    ws = bt.Workspace([w, lam])
+    out = _vec(d)
+    bt.betty_grad(w, w, out, ws)
+    assert cb.rel_l2(out, oracle.grad(ow, ow)) < 2e-5
+    bt.betty_grad(w, lam, out, ws)
+    assert cb.rel_l2(out, oracle.grad(ow, olam)) < 1e-6
+    bt.betty_grad(lam, w, out, ws)
+    assert cb.rel_l2(out, oracle.grad(olam, ow)) < 2e-5
+    bt.betty_grad(lam, lam, out, ws)
+    assert torch.all(out == 0)
+    u = si.normal_f32(9, 3, (d,))
+    bt.betty_hvp(w, cb.dev(u), out, ws)
+    assert cb.rel_l2(out, oracle.hvp(ow, u)) < 2e-5
+    bt.betty_mixed_vjp(w, lam, cb.dev(u), out, ws)
+    assert cb.rel_l2(out, oracle.mixed_vjp(ow, olam, u)) < 1e-6
+    bt.betty_lower_step(w, 3, ws)
+    oracle.lower_step(ow, 3)
+    assert cb.rel_l2(w.params, ow.params) < 2e-5
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+@pytest.mark.parametrize("n,d,nv,steps,K", [(1024, 64, 256, 100, 10), (2051, 4096, 513, 20, 20),
+                                             (513, 1028, 64, 10, 7)])
+def test_hypergradients_match_oracle(bt, n, d, nv, steps, K):
+    from tests import cuda_build as cb
+    inp = si.config1() if (n, d) == (1024, 64) else si.logreg_bilevel(si.BASE_SEED + 2, n, d, nv)
+    (w, lam), (ow, olam) = _pair(inp)
+    ws = bt.Workspace([w, lam])
+    bt.betty_lower_step(w, steps, ws)
+    oracle.lower_step(ow, steps)
+    assert cb.rel_l2(w.params, ow.params) < TOL
+    out = _vec(d)
+    bt.betty_hypergrad_neumann(w, lam, lam, K, 0.01, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_neumann(ow, olam, olam, K, 0.01)) < TOL
+    bt.betty_hypergrad_cg(w, lam, lam, K, 0.0, out, ws)
+    info = {}
+    ref = oracle.hypergrad_cg(ow, olam, olam, K, 0.0, info=info)
+    assert cb.rel_l2(out, ref) < TOL
+    st, iters = bt.betty_poll_status(ws)
+    assert st == bt.BETTY_OK and iters == info["iters"] == K          # integer work: exact
+    bt.betty_hypergrad_fd(w, lam, lam, 0.01, 1.0, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_fd(ow, olam, olam, 0.01, 1.0)) < TOL
+    # chain call on the one-edge path gives the Jacobian term alone (direct gradient is zero here)
+    bt.betty_chain_levels([w, lam], [1, 0], [bt.MethodCfg(bt.BETTY_CG, K=K)], None, out, False, ws)
+    assert cb.rel_l2(out, ref) < TOL
+
+
+def test_cg_early_stop_counts_iterations_like_the_oracle(bt):
+    from tests import cuda_build as cb
+    inp = si.logreg_bilevel(5, 400, 16, 100)
+    (w, lam), (ow, olam) = _pair(inp)
+    ws = bt.Workspace([w, lam])
+    bt.betty_lower_step(w, 50, ws); oracle.lower_step(ow, 50)
+    out = _vec(16)
+    bt.betty_hypergrad_cg(w, lam, lam, 64, 1e-3, out, ws)
+    info = {}
+    ref = oracle.hypergrad_cg(ow, olam, olam, 64, 1e-3, info=info)
+    st, iters = bt.betty_poll_status(ws)
+    assert st == bt.BETTY_OK and iters == info["iters"] and iters < 64
+    assert cb.rel_l2(out, ref) < TOL
+
+
+def test_quadratic_family_and_cg_breakdown_status(bt):
+    from tests import cuda_build as cb
+    rng = np.random.default_rng(11)
+    A, b = rng.standard_normal((150, 24)).astype(np.float32), rng.standard_normal(150).astype(np.float32)
+    Av, bv = rng.standard_normal((90, 24)).astype(np.float32), rng.standard_normal(90).astype(np.float32)
+    lamv = (rng.random(24) + 0.1).astype(np.float32)
+    w0 = (rng.standard_normal(24) * 0.1).astype(np.float32)
+    lo, up = cb.quadratic_levels(A, b, lamv, Av, bv, w0)
+    olo, oup = ob.quadratic_levels(A, b, lamv, Av, bv, w0)
+    ws = bt.Workspace([lo, up])
+    out = _vec(24)
+    bt.betty_hypergrad_cg(lo, up, up, 24, 0.0, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_cg(olo, oup, oup, 24, 0.0)) < 1e-3   # 24 fp32 CG steps
+    bt.betty_hypergrad_neumann(lo, up, up, 8, 1e-3, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_neumann(olo, oup, oup, 8, 1e-3)) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+    # an indefinite Hessian: the oracle reports breakdown at iteration 0, the device must too
+    lam_bad = lamv.copy(); lam_bad[:] = -500.0
+    lo2, up2 = cb.quadratic_levels(A, b, lam_bad, Av, bv, w0)
+    olo2, oup2 = ob.quadratic_levels(A, b, lam_bad, Av, bv, w0)
+    info = {}
+    ref = oracle.hypergrad_cg(olo2, oup2, oup2, 5, 0.0, info=info)
+    assert info["status"] == "breakdown"
+    ws2 = bt.Workspace([lo2, up2])
+    bt.betty_hypergrad_cg(lo2, up2, up2, 5, 0.0, out, ws2)
+    st, iters = bt.betty_poll_status(ws2, raise_on_error=False)
+    assert st == bt.BETTY_ERR_BREAKDOWN and iters == info["iters"]
+    assert cb.rel_l2(out, ref) < TOL or np.linalg.norm(ref) == 0
+    bt.betty_reset_status(ws2)
+    assert bt.betty_poll_status(ws2)[0] == bt.BETTY_OK
+
+
+def test_empty_batch_and_argument_errors(bt):
+    from tests import cuda_build as cb
+    inp = si.logreg_bilevel(3, 16, 8, 4)
+    (w, lam), _ = _pair(inp)
+    ws = bt.Workspace([w, lam])
+    out = _vec(8)
+    empty = bt.Level(bt.LOSS_LOGREG_WD, bt.PARAM_VECTOR, cb.dev(inp.w0 + 1), X=torch.empty(0, 8, dtype=torch.float32, device="cuda"),
+                     y=torch.empty(0, dtype=torch.float32, device="cuda"))
+    empty.set_constraints([lam])
+    bt.betty_grad(empty, empty, out, ws)            # only the weight-decay term is left
+    assert cb.rel_l2(out, (inp.lam * (inp.w0 + 1)).astype(np.float64)) < 1e-6
+    with pytest.raises(bt.BettyError) as e:
+        bt.betty_hypergrad_cg(w, lam, w, 3, 0.0, out, ws)      # wrt must be a constraint of lower
+    assert e.value.status == bt.BETTY_ERR_INVALID_ARG
+    bad = bt.Level(bt.LOSS_LOGREG_WD, bt.PARAM_VECTOR, cb.dev(np.zeros(7, np.float32)), X=w.X, y=w.y)
+    bad.set_constraints([lam])
+    with pytest.raises(bt.BettyError) as e:
+        bt.betty_grad(bad, bad, out, ws)
+    assert e.value.status == bt.BETTY_ERR_SHAPE
+    small = bt.Workspace([w, lam]); small.nbytes = 512
+    with pytest.raises(bt.BettyError) as e:
+        bt.betty_hvp(w, out, out, small)
+    assert e.value.status == bt.BETTY_ERR_WORKSPACE
+
+
+def test_repeated_calls_are_bitwise_identical(bt):
+    inp = si.logreg_bilevel(8, 3000, 4096, 64)
+    (w, lam), _ = _pair(inp)
+    ws = bt.Workspace([w, lam])
+    u = torch.randn(4096, dtype=torch.float32, device="cuda")
+    a, b = _vec(4096), _vec(4096)
+    bt.betty_hvp(w, u, a, ws)
+    bt.betty_hvp(w, u, b, ws)
+    assert torch.equal(a, b)

@@ -15,7 +15,6 @@ from oracle.bf16 import round_to_bf16
 import synth_inputs as si
 from tests.oracle_build import logreg_levels, quadratic_levels, reweight_levels, three_levels
 
-torch.set_default_dtype(torch.float64)
 
 
 def central_fd(f, x, eps=1e-6):

@@ -16,7 +16,6 @@ from tests.oracle_build import logreg_levels, quadratic_levels, three_levels
 from tests.test_oracle_derivatives import (_t, _tiny_three, _torch_detect_cost,
                                            _torch_reweight_cost, central_fd, rel)
 
-torch.set_default_dtype(torch.float64)
 
 
 def _spd(d, seed, lo=0.2, hi=2.0):
