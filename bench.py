@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the hypergradient hot path.
+
+`python bench.py --gpus N --steps K --warmup W` prints ONE JSON line.  A step is one pass of the
+whole hot path over one batch of synthetic input: the unrolled lower-level gradient steps, the
+direct gradients of the upper cost and the best-response-Jacobian product of the configuration's
+method (default workload: the bilevel logistic weight-decay problem with X of 262144 x 4096 fp32,
+20 lower steps, conjugate gradient with K = 20).  Inputs are resident in device memory for
+`value`; `e2e` repeats the measurement with host (pinned) inputs copied in every step and the
+result read back.  `--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+Under torchrun (N > 1) every rank runs an independent replica on its own GPU (the path has no
+exchange step); value is the aggregate, time the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "hypergradient_steps_per_sec"
+UNIT = "steps/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+        self.t0 = self.t1 = None
+
+    def mark_begin(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        inside = [ln for (t, ln) in self.lines if self.t0 is not None and self.t0 <= t <= (self.t1 or t) + 0.05]
+        if not inside:      # region shorter than one sampling period: fall back to every sample taken under load
+            inside = [ln for (_, ln) in self.lines]
+        for ln in inside:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ workloads
+class LogregWorkload:
+    """Configs 1 and 2: bilevel weight decay for logistic regression (App. D.1 problem)."""
+
+    def __init__(self, cfg: int, method: str, scale: float = 1.0):
+        import synth_inputs as si
+        self.cfg = cfg
+        self.inp = si.config1() if cfg == 1 else si.config2(scale)
+        self.method = method or ("cg" if cfg == 2 else "cg")
+        self.n, self.d = self.inp.X.shape
+        self.nv = self.inp.Xv.shape[0]
+        self.name = (f"config{cfg}: logistic weight-decay bilevel, X fp32 {self.n}x{self.d} train / "
+                     f"{self.nv}x{self.d} val, {self.inp.lower_steps} lower GD steps, {self.method} K={self.inp.K}")
+        self.dtype = "f32"
+
+    # algorithmic bytes of one streaming pass over the train matrix (the dominant kernel)
+    def pass_bytes(self):
+        return self.n * self.d * 4
+
+    def setup_device(self):
+        import torch
+        import paper_2207_02849_b200 as bt
+        from tests import cuda_build as cb
+        self.bt, self.torch = bt, torch
+        self.w, self.lam = cb.logreg_levels(self.inp)
+        self.w0 = self.w.params.clone()
+        self.out = torch.empty(self.d, dtype=torch.float32, device="cuda")
+        self.ws = bt.Workspace([self.w, self.lam])
+
+    def step(self):
+        bt = self.bt
+        self.w.params.copy_(self.w0)
+        bt.betty_lower_step(self.w, self.inp.lower_steps, self.ws)
+        if self.method == "cg":
+            bt.betty_hypergrad_cg(self.w, self.lam, self.lam, self.inp.K, 0.0, self.out, self.ws)
+        elif self.method == "neumann":
+            bt.betty_hypergrad_neumann(self.w, self.lam, self.lam, self.inp.K, self.inp.alpha, self.out, self.ws)
+        else:
+            bt.betty_hypergrad_fd(self.w, self.lam, self.lam, 0.01, 1.0, self.out, self.ws)
+
+    # -- end-to-end: host buffers in, result out, through the same C-ABI calls
+    def setup_host(self):
+        torch = self.torch
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        self.h_in = [pin(self.inp.X), pin(self.inp.y), pin(self.inp.Xv), pin(self.inp.yv), pin(self.inp.lam),
+                     pin(self.inp.w0)]
+        self.d_in = [self.w.X, self.w.y, self.lam.X, self.lam.y, self.lam.params, self.w0]
+        self.h_out = torch.empty(self.d, dtype=torch.float32).pin_memory()
+        self.h2d = sum(t.numel() * t.element_size() for t in self.h_in)
+        self.d2h = self.h_out.numel() * 4
+
+    def step_e2e(self):
+        for h, d in zip(self.h_in, self.d_in):
+            d.copy_(h, non_blocking=True)
+        self.step()
+        self.h_out.copy_(self.out, non_blocking=True)
+
+    def roofline_probe(self, reps: int):
+        """Average duration of the dominant kernel (the fused HVP row-stream pass over the train
+        matrix), timed alone with CUDA events around single betty_hvp calls; the tiny fixed-order
+        reduction kernel that follows it is inside the bracket."""
+        torch, bt = self.torch, self.bt
+        u = torch.randn(self.d, dtype=torch.float32, device="cuda")
+        hu = torch.empty_like(u)
+        for _ in range(3):
+            bt.betty_hvp(self.w, u, hu, self.ws)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in evs:
+            a.record()
+            bt.betty_hvp(self.w, u, hu, self.ws)
+            b.record()
+        torch.cuda.synchronize()
+        ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+        return {"kernel": "k_logreg_stream<HVP>", "ms": ms, "bytes": self.pass_bytes(), "bound": "hbm"}
+
+    # -- oracle on a bounded sample of the same workload
+    def oracle_sample(self, budget_rows: int):
+        import oracle
+        from tests import oracle_build as ob
+        import synth_inputs as si
+        import copy
+        n_s = min(self.n, budget_rows)
+        nv_s = max(1, min(self.nv, int(round(budget_rows * self.nv / self.n))))
+        inp = copy.copy(self.inp)
+        inp.X, inp.y, inp.Xv, inp.yv = self.inp.X[:n_s], self.inp.y[:n_s], self.inp.Xv[:nv_s], self.inp.yv[:nv_s]
+        ow, olam = ob.logreg_levels(inp)
+        t0 = time.perf_counter()
+        oracle.lower_step(ow, inp.lower_steps)
+        if self.method == "cg":
+            oracle.hypergrad_cg(ow, olam, olam, inp.K, 0.0)
+        elif self.method == "neumann":
+            oracle.hypergrad_neumann(ow, olam, olam, inp.K, inp.alpha)
+        else:
+            oracle.hypergrad_fd(ow, olam, olam, 0.01, 1.0)
+        dt = time.perf_counter() - t0
+        frac = n_s / self.n
+        return dt / frac, f"first {n_s} of {self.n} train rows and {nv_s} of {self.nv} validation rows, full step, time scaled by {1/frac:.0f}x"
+
+
+def make_workload(cfg: int, method: str, scale: float):
+    if cfg in (1, 2):
+        return LogregWorkload(cfg, method, scale)
+    raise SystemExit(f"config {cfg} is not wired into the benchmark yet")
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------ main
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    wl = make_workload(args.config, args.method, args.scale)
+    rows = args.oracle_rows
+    times = []
+    for i in range(args.warmup + args.steps):
+        t, sample = wl.oracle_sample(rows)
+        if i >= args.warmup:
+            times.append(t)
+    sec = float(np.mean(times))
+    val = 1.0 / sec
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": 0, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--method", default="")
+    ap.add_argument("--scale", type=float, default=1.0, help="row-count scale of config 2 (tests/profiling only)")
+    ap.add_argument("--oracle-rows", type=int, default=131072)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if args.steps > 3:
+            args.steps = 3
+        args.warmup = min(args.warmup, 1)
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: this path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    import paper_2207_02849_b200 as bt
+
+    wl = make_workload(args.config, args.method, args.scale)
+    wl.setup_device()
+    warm = max(args.warmup, 3)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup, sampler=None):
+        if sampler:
+            sampler.start()     # the sampler starts during warm-up; only samples inside the timed region count
+        for _ in range(warmup):
+            fn()
+        barrier()
+        if sampler:
+            sampler.mark_begin()
+        l0 = bt.betty_kernel_launches()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        if sampler:
+            sampler.mark_end()
+        launches = bt.betty_kernel_launches() - l0
+        clocks = sampler.stop() if sampler else None
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, launches, clocks
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms, launches, clocks = timed(wl.step, args.steps, warm, sampler)
+    st, _ = bt.betty_poll_status(wl.ws)
+    ms_per_step = ms / args.steps
+    value = world * 1e3 / ms_per_step
+
+    e2e = None
+    if not args.no_e2e:
+        wl.setup_host()
+        ms_e, _, _ = timed(wl.step_e2e, max(1, min(args.steps, 5)), 3)
+        e_steps = max(1, min(args.steps, 5))
+        e2e = {"value": world * 1e3 / (ms_e / e_steps), "unit": UNIT, "h2d_bytes_per_step": int(wl.h2d),
+               "d2h_bytes_per_step": int(wl.d2h)}
+
+    peaks = _peaks()
+    probe = wl.roofline_probe(20)
+    if probe["bound"] == "hbm":
+        achieved = probe["bytes"] / (probe["ms"] * 1e-3) / 1e9
+        peak, unit = peaks["hbm_gbs"], "GB/s"
+    else:
+        achieved = probe["flops"] / (probe["ms"] * 1e-3) / 1e12
+        peak, unit = peaks["bf16_tflops"], "TFLOP/s"
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            tj = json.load(f).get(probe["kernel"])
+        if tj and tj.get("valid"):
+            traffic = tj["dram_bytes_per_unit"] * (probe["bytes"] / tj["unit_bytes"])
+    roofline = {"bound": probe["bound"], "kernel": probe["kernel"], "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": traffic, "peak_source": f"{peaks['source']} (burst; kernel timed alone)",
+                "kernel_ms": probe["ms"], "algorithmic_bytes_per_launch": probe.get("bytes")}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        sec, sample = wl.oracle_sample(args.oracle_rows)
+        cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "l2": "inputs (train matrix) larger than L2; no flush between steps",
+                       "replicas": world, "device_status": bt.betty_status_string(st)},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

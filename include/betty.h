@@ -184,6 +184,10 @@ betty_status betty_chain_levels(const betty_level* const* levels, int32_t n_leve
 
 const char* betty_status_string(betty_status s);
 
+/* Number of CUDA kernels this library has launched in the calling process since it was loaded
+ * (host-side counter; used by benchmarks to report their launch count). */
+uint64_t betty_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

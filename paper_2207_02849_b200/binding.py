@@ -83,12 +83,17 @@ def lib():
         fn = getattr(L, name)
         fn.argtypes, fn.restype = args, C.c_int
     L.betty_status_string.argtypes, L.betty_status_string.restype = [C.c_int], C.c_char_p
+    L.betty_kernel_launches.argtypes, L.betty_kernel_launches.restype = [], C.c_uint64
     _lib = L
     return L
 
 
 def betty_status_string(status: int) -> str:
     return lib().betty_status_string(int(status)).decode()
+
+
+def betty_kernel_launches() -> int:
+    return int(lib().betty_kernel_launches())
 
 
 def _check(status: int, where: str):

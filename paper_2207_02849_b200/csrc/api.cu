@@ -6,6 +6,8 @@
 
 namespace betty {
 
+unsigned long long g_kernel_launches = 0;
+
 // ------------------------------------------------------------------ small kernels
 // out (+)= scale * x
 __global__ void k_scale_into(float* out, const float* x, float scale, int accumulate, int64_t n) {
@@ -222,6 +224,8 @@ const char* betty_status_string(betty_status s) {
   }
   return "unknown status";
 }
+
+uint64_t betty_kernel_launches(void) { return (uint64_t)g_kernel_launches; }
 
 betty_status betty_workspace_size(const betty_level* const* levels, int32_t n_levels, size_t* bytes) {
   if (!levels || n_levels <= 0 || !bytes) return BETTY_ERR_INVALID_ARG;

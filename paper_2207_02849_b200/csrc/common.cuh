@@ -67,8 +67,11 @@ struct Ctx {
     if (_s != BETTY_OK) return _s;            \
   } while (0)
 
+// Every kernel launch of the library passes through this check, which also counts it.
+extern unsigned long long g_kernel_launches;
 #define BETTY_LAUNCH_CHECK()                                   \
   do {                                                         \
+    ++betty::g_kernel_launches;                                \
     if (cudaPeekAtLastError() != cudaSuccess) {                \
       (void)cudaGetLastError();                                \
       return BETTY_ERR_CUDA;                                   \

@@ -159,7 +159,7 @@ def test_empty_batch_and_argument_errors(bt):
     with pytest.raises(bt.BettyError) as e:
         bt.betty_grad(bad, bad, out, ws)
     assert e.value.status == bt.BETTY_ERR_SHAPE
-    small = bt.Workspace([w, lam]); small.nbytes = 512
+    small = bt.Workspace([w, lam]); small.nbytes = 256
     with pytest.raises(bt.BettyError) as e:
         bt.betty_hvp(w, out, out, small)
     assert e.value.status == bt.BETTY_ERR_WORKSPACE
