@@ -52,7 +52,8 @@ typedef enum {
   BETTY_ERR_NONFINITE = 7,    /* device: a reduction met Inf/NaN */
   BETTY_ERR_BREAKDOWN = 8,    /* device: CG met a direction with p^T H p <= 0 */
   BETTY_ERR_TIMEOUT = 9,      /* device: a bounded wait (mbarrier) expired */
-  BETTY_ERR_UNSUPPORTED = 10  /* combination not implemented */
+  BETTY_ERR_UNSUPPORTED = 10, /* combination not implemented */
+  BETTY_ERR_CAPACITY = 11     /* size exceeds the fixed built-in scratch of an allocation-free call */
 } betty_status;
 
 /* Cost families C_k.  "own" = the level's own parameter block. */
@@ -181,6 +182,26 @@ betty_status betty_chain_levels(const betty_level* const* levels, int32_t n_leve
                                 const int32_t* path, int32_t path_len,
                                 const betty_method_cfg* per_edge, const float* v_in, float* out,
                                 int32_t accumulate, void* ws, size_t ws_bytes, void* stream);
+
+/* (No counterpart in the paper: a deployment aid.)  Hessian-vector product of the logistic
+ * weight-decay cost, Hu = (1/n) X^T (sigmoid(z) sigmoid(-z) . X u) + lam . u with z = X w, for callers
+ * that have no device memory to give as workspace and may not allocate any: a host whose GPU memory
+ * is fully reserved by another allocator or pool, or code that must not risk the device-wide
+ * synchronisation an allocation or a free can cause.  The scratch (per-CTA column sums and a status
+ * word) is a fixed array inside the library image, about 4.6 MiB, held by every GPU that loads the
+ * library until the process exits.  This call allocates and frees nothing.
+ *   X fp32 [n, d] row-major, w / lam / u / Hu fp32 [d], all DEVICE pointers, 16-byte aligned;
+ *   d a multiple of 4 and at most 4096: a larger d returns BETTY_ERR_CAPACITY, nothing is enqueued;
+ *   status_dev: DEVICE int32 owned by the caller, or NULL; receives 0 or the betty_status of a
+ *   condition met on the device (BETTY_ERR_TIMEOUT).
+ * Same kernels, launch shape and summation order as betty_hvp on a LOGREG_WD level.  The first call
+ * on each device looks up the array's device address (with that device current); make that first
+ * call outside any stream capture.  All calls on one device share the array, which keeps the previous
+ * call's contents (the call clears the part that must start at zero): two calls whose kernels can
+ * overlap on the GPU, e.g. on different streams, race on it, so serialise them. */
+betty_status betty_hvp_logreg_static(const float* X, int64_t n, int64_t d, const float* w,
+                                     const float* lam, const float* u, float* Hu,
+                                     int32_t* status_dev, void* stream);
 
 const char* betty_status_string(betty_status s);
 

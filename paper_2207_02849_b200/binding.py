@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 BETTY_OK = 0
 (BETTY_ERR_INVALID_ARG, BETTY_ERR_SHAPE, BETTY_ERR_DTYPE, BETTY_ERR_ALIGNMENT, BETTY_ERR_WORKSPACE,
  BETTY_ERR_CUDA, BETTY_ERR_NONFINITE, BETTY_ERR_BREAKDOWN, BETTY_ERR_TIMEOUT,
- BETTY_ERR_UNSUPPORTED) = range(1, 11)
+ BETTY_ERR_UNSUPPORTED, BETTY_ERR_CAPACITY) = range(1, 12)
 (LOSS_LOGREG_WD, LOSS_LOGREG, LOSS_QUADRATIC_WD, LOSS_QUADRATIC, LOSS_MLP_CE_REWEIGHT, LOSS_MLP_CE,
  LOSS_WEIGHTNET_DETECT) = range(7)
 PARAM_VECTOR, PARAM_MLP, PARAM_WEIGHTNET, PARAM_LOGWD = range(4)
@@ -79,6 +79,7 @@ def lib():
         "betty_chain_levels": [C.POINTER(LP), I32, C.POINTER(I32), I32, C.POINTER(_MethodCfg), VP, VP, I32,
                                VP, SZ, VP],
     }
+    sig["betty_hvp_logreg_static"] = [VP, C.c_int64, C.c_int64, VP, VP, VP, VP, VP, VP]
     for name, args in sig.items():
         fn = getattr(L, name)
         fn.argtypes, fn.restype = args, C.c_int
@@ -238,3 +239,12 @@ def betty_chain_levels(levels: Sequence[Level], path: Sequence[int], per_edge: S
     cfgs = (_MethodCfg * len(per_edge))(*[m.c for m in per_edge])
     _check(lib().betty_chain_levels(arr, len(levels), p, len(path), cfgs, _ptr(v_in), _ptr(out),
                                     1 if accumulate else 0, ws.ptr, ws.nbytes, _stream(stream)), "betty_chain_levels")
+
+
+def betty_hvp_logreg_static(X: torch.Tensor, w: torch.Tensor, lam: torch.Tensor, u: torch.Tensor, Hu: torch.Tensor,
+                            status_dev: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Logistic weight-decay HVP that uses the library's built-in scratch instead of a workspace
+    (for callers that cannot allocate device memory); see betty.h for the limits."""
+    n, d = X.shape
+    _check(lib().betty_hvp_logreg_static(_ptr(X) if n else None, n, d, _ptr(w), _ptr(lam), _ptr(u), _ptr(Hu),
+                                         _ptr(status_dev), _stream(stream)), "betty_hvp_logreg_static")

@@ -221,6 +221,7 @@ const char* betty_status_string(betty_status s) {
     case BETTY_ERR_BREAKDOWN: return "conjugate gradient breakdown (p^T H p <= 0)";
     case BETTY_ERR_TIMEOUT: return "bounded device wait expired";
     case BETTY_ERR_UNSUPPORTED: return "unsupported combination";
+    case BETTY_ERR_CAPACITY: return "size exceeds the fixed built-in scratch of this allocation-free call";
   }
   return "unknown status";
 }

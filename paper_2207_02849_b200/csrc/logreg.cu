@@ -303,3 +303,68 @@ betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int
 }
 
 }  // namespace betty
+
+// ------------------------------------------------------------------ allocation-free HVP
+// Scratch that belongs to the library image itself: every GPU that loads the library holds
+// these bytes until the process exits.  Layout: [StatusBlock (256 B)][per-CTA column sums].
+namespace betty {
+static constexpr int NOALLOC_MAX_D = 4096;
+static constexpr int NOALLOC_MAX_CTAS = 2 * 148;
+static constexpr size_t NOALLOC_FLOATS = sizeof(StatusBlock) / sizeof(float) + (size_t)NOALLOC_MAX_CTAS * NOALLOC_MAX_D;
+static __device__ __align__(256) float g_noalloc_scratch[NOALLOC_FLOATS];
+static constexpr int NOALLOC_MAX_DEVICES = 64;
+static float* g_noalloc_ptr[NOALLOC_MAX_DEVICES];   // device address of the array, per device ordinal
+
+__global__ void k_noalloc_report(const StatusBlock* sb, int32_t* status_dev) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) *status_dev = sb->code;
+}
+}  // namespace betty
+
+extern "C" betty_status betty_hvp_logreg_static(const float* X, int64_t n, int64_t d, const float* w,
+                                                const float* lam, const float* u, float* Hu,
+                                                int32_t* status_dev, void* stream) {
+  using namespace betty;
+  if (n < 0 || d <= 0) return BETTY_ERR_SHAPE;
+  if (!w || !lam || !u || !Hu || (n > 0 && !X)) return BETTY_ERR_INVALID_ARG;
+  if (d > NOALLOC_MAX_D) return BETTY_ERR_CAPACITY;          // beyond the fixed scratch
+  if (d % 4 != 0) return BETTY_ERR_UNSUPPORTED;               // only the single-pass kernel is offered here
+  if (!aligned16(X) || !aligned16(w) || !aligned16(u) || !aligned16(Hu)) return BETTY_ERR_ALIGNMENT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return BETTY_ERR_CUDA;
+  if (!g_noalloc_ptr[dev]) {
+    // In host code the array's name is only a handle; the device address has to be asked for,
+    // once per device, with that device current.
+    float* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) {
+      (void)cudaGetLastError();
+      return BETTY_ERR_CUDA;
+    }
+    g_noalloc_ptr[dev] = p;
+  }
+  float* base = g_noalloc_ptr[dev];
+  cudaStream_t s = (cudaStream_t)stream;
+  // the status block is the only part that must start at zero: every per-CTA row that the
+  // reduction reads is rewritten by this call's streaming kernel
+  if (cudaMemsetAsync(base, 0, sizeof(StatusBlock), s) != cudaSuccess) return BETTY_ERR_CUDA;
+  Ctx c(base, NOALLOC_FLOATS * sizeof(float), stream);
+  LrArgs a;
+  a.X = X; a.y = nullptr; a.n = n; a.d = d; a.w = w; a.u = u; a.family = 0;
+  a.inv_n = n > 0 ? 1.0f / (float)n : 0.f;
+  a.sb = c.arena.status();
+  a.partials = base + sizeof(StatusBlock) / sizeof(float);
+  const int64_t ntiles = (n + LR_R - 1) / LR_R;
+  int grid = NOALLOC_MAX_CTAS;
+  if (ntiles < grid) grid = ntiles > 0 ? (int)ntiles : 1;
+  betty_status st;
+  if (d <= 1024) st = launch_stream<1, true>(c, a, grid);
+  else if (d <= 2048) st = launch_stream<2, true>(c, a, grid);
+  else st = launch_stream<4, true>(c, a, grid);
+  if (st != BETTY_OK) return st;
+  k_logreg_finalize<<<(unsigned)((d + 31) / 32), 256, 0, s>>>(a.partials, grid, d, lam, u, Hu, nullptr, 0.f);
+  BETTY_LAUNCH_CHECK();
+  if (status_dev) {
+    k_noalloc_report<<<1, 32, 0, s>>>(a.sb, status_dev);
+    BETTY_LAUNCH_CHECK();
+  }
+  return BETTY_OK;
+}
