@@ -130,21 +130,34 @@ def mlp_pack(Ws, bs):
 
 def _mlp_weights(level: Level, flat):
     """The copy of the parameters the cost is evaluated at: matrices rounded to bf16 for
-    mixed-precision levels (the single quantisation point), biases as they are."""
+    mixed-precision levels, biases as they are."""
     Ws, bs = mlp_unpack(level.widths, flat)
     if level.bf16:
         Ws = [round_to_bf16(W) for W in Ws]
     return Ws, bs
 
 
-def _mlp_forward(Ws, bs, X, act):
-    """h[l] is the input of layer l (h[0] = X), a[l] its pre-activation; logits = a[-1]."""
-    h, a = [X], []
+def _mlp_forward(Ws, bs, X, act, quant=False, offsets=None):
+    """h[l] is the input of layer l (h[0] = X), a[l] its pre-activation; logits = a[-1].
+
+    Mixed-precision levels (quant=True) feed every matrix product bf16 operands, so each hidden
+    activation is rounded to bf16 before it enters the next layer; the rounding offsets
+    round(h) - h are returned.  With `offsets` given, those offsets are added instead of
+    rounding again: a perturbed evaluation keeps the base point's quantisation offsets frozen,
+    the same straight-through convention under which the derivatives are taken."""
+    h, a, offs = [X], [], []
     for l, (W, b) in enumerate(zip(Ws, bs)):
         a.append(h[-1] @ W.T + b)
         if l < len(Ws) - 1:
-            h.append(_act(act, a[-1]))
-    return h, a
+            hn = _act(act, a[-1])
+            if offsets is not None:
+                hn = hn + offsets[l]
+            elif quant:
+                hq = round_to_bf16(hn)
+                offs.append(hq - hn)
+                hn = hq
+            h.append(hn)
+    return h, a, offs
 
 
 def _softmax_ce(z, y):
@@ -230,10 +243,24 @@ def _logreg_parts(L, over):
 
 
 def _mlp_ce_state(L: Level, over):
-    """Forward pass of the classifier that takes part in cost L and the per-sample CE."""
+    """Forward pass of the classifier that takes part in cost L and the per-sample CE.
+
+    over["frozen"] (a set of level ids) marks the classifier's override as a perturbed
+    evaluation: its parameters are the base compute copy plus the given displacement, and
+    the activations keep the base pass's rounding offsets."""
     M = _find(L, "mlp")
-    Ws, bs = _mlp_weights(M, _p(M, over))
-    h, a = _mlp_forward(Ws, bs, L.X, M.activation)
+    flat = _p(M, over)
+    frozen = over is not None and id(M) in over.get("frozen", ())
+    if frozen and M.bf16:
+        Wb, bb = _mlp_weights(M, M.params)
+        _, _, offs = _mlp_forward(Wb, bb, L.X, M.activation, quant=True)
+        Wd, bd = mlp_unpack(M.widths, flat - M.params)
+        Ws = [W0 + dW for W0, dW in zip(Wb, Wd)]
+        bs = [b0 + db for b0, db in zip(bb, bd)]
+        h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation, offsets=offs)
+    else:
+        Ws, bs = _mlp_weights(M, flat)
+        h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation, quant=M.bf16)
     p, ell = _softmax_ce(a[-1], np.asarray(L.y, dtype=np.int64))
     return M, Ws, bs, h, a, p, ell
 

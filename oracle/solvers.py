@@ -13,7 +13,9 @@ weights).  Readings where the paper is silent:
   * CG(K, tol): zero start, no preconditioner, stops after K iterations, or when the residual
     norm has fallen to tol*|v|, or (status "breakdown") when a search direction has p^T H p <= 0.
   * FD(eps0, alpha): eps = eps0/|v|_2; result -alpha*[dC/dc(x+eps v) - dC/dc(x-eps v)]/(2 eps),
-    i.e. H^{-1} replaced by alpha*I; alpha defaults to 1.
+    i.e. H^{-1} replaced by alpha*I; alpha defaults to 1.  On mixed-precision levels the two
+    perturbed evaluations are not re-quantised: x +- eps v displaces the bf16 compute copy, and
+    the rounding offsets of weights and hidden activations stay at their base-point values.
 """
 from __future__ import annotations
 
@@ -91,8 +93,10 @@ def brj(L: Level, wrt: Level, v, method: str, K: int = 0, alpha: float = 1.0,
         if nv == 0.0:
             return np.zeros(wrt.params.size)
         eps = eps0 / nv
-        gp = grad(L, wrt, over={id(L): L.params + eps * v})
-        gm = grad(L, wrt, over={id(L): L.params - eps * v})
+        # perturbed evaluations keep the base point's bf16 rounding offsets (weights and hidden
+        # activations) frozen; for full-precision levels "frozen" has no effect
+        gp = grad(L, wrt, over={id(L): L.params + eps * v, "frozen": {id(L)}})
+        gm = grad(L, wrt, over={id(L): L.params - eps * v, "frozen": {id(L)}})
         return -alpha * (gp - gm) / (2.0 * eps)
     raise ValueError(method)
 

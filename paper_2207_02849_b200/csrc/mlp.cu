@@ -1,12 +1,789 @@
-// placeholder until the MLP families are wired in
+// MLP cost families: the reweighted cross-entropy classifier of the data-reweighting experiment
+// (App. A listing), its plain cross-entropy upper cost, and the clean-label detector cost of the
+// three-level configuration.  Gradients are hand-written reverse sweeps; Hessian-vector products
+// are R-operator (forward-over-reverse) passes that reuse a cached base forward/backward pass;
+// mixed second derivatives are a directional forward pass followed by the weight net's reverse
+// sweep.  Matrices are bf16 (rounded copies of the fp32 master), accumulation is fp32.
 #include "ops.cuh"
+#include "gemm.cuh"
+
 namespace betty {
-betty_status mlpfam_validate(const betty_level*) { return BETTY_ERR_UNSUPPORTED; }
-size_t mlpfam_workspace(const betty_level*) { return 0; }
-betty_status mlpfam_grad(Ctx&, const betty_level*, const betty_level*, float*) { return BETTY_ERR_UNSUPPORTED; }
-betty_status mlpfam_hvp_begin(Ctx&, const betty_level*, MlpHvpCache**) { return BETTY_ERR_UNSUPPORTED; }
-betty_status mlpfam_hvp(Ctx&, const betty_level*, MlpHvpCache*, const float*, float*) { return BETTY_ERR_UNSUPPORTED; }
-betty_status mlpfam_mixed(Ctx&, const betty_level*, MlpHvpCache*, const betty_level*, const float*, float*) { return BETTY_ERR_UNSUPPORTED; }
-betty_status mlpfam_lower_step(Ctx&, const betty_level*, int) { return BETTY_ERR_UNSUPPORTED; }
-betty_status mlpfam_fd(Ctx&, const betty_level*, const betty_level*, const float*, const float*, float, float, float*, bool) { return BETTY_ERR_UNSUPPORTED; }
+
+static constexpr int MAXL = 16;
+static constexpr int WN_H = 100;
+static constexpr int WN_P = 3 * WN_H + 1;
+
+static inline int64_t ld8(int64_t n) { return (n + 7) & ~int64_t(7); }
+static inline int grid_for(int64_t n, int per_block = 256) {
+  int64_t b = (n + per_block - 1) / per_block;
+  return (int)(b < 1 ? 1 : (b > 148 * 32 ? 148 * 32 : b));
 }
+
+// ------------------------------------------------------------------ activations
+__device__ __forceinline__ float norm_pdf(float a) { return 0.3989422804014327f * expf(-0.5f * a * a); }
+__device__ __forceinline__ float norm_cdf(float a) { return 0.5f * (1.f + erff(a * 0.7071067811865476f)); }
+__device__ __forceinline__ float act_f(int act, float a) { return act == BETTY_ACT_RELU ? fmaxf(a, 0.f) : a * norm_cdf(a); }
+__device__ __forceinline__ float act_d1(int act, float a) {
+  return act == BETTY_ACT_RELU ? (a > 0.f ? 1.f : 0.f) : norm_cdf(a) + a * norm_pdf(a);
+}
+__device__ __forceinline__ float act_d2(int act, float a) {
+  return act == BETTY_ACT_RELU ? 0.f : norm_pdf(a) * (2.f - a * a);
+}
+__device__ __forceinline__ float fd_eps(const float* vnorm2, float eps0) {
+  const float nv2 = *vnorm2;
+  return nv2 > 0.f ? eps0 / sqrtf(nv2) : 0.f;
+}
+
+// ------------------------------------------------------------------ elementwise / row kernels
+// dst[r, c] = bf16(scale * src[r, c]); scale = eps0/|v| when vnorm2 is given, else 1.  Pad columns are zeroed.
+__global__ void k_cast_rows(const float* src, bf16* dst, int64_t rows, int64_t cols, int64_t ld, const float* vnorm2,
+                            float eps0) {
+  const float s = vnorm2 ? fd_eps(vnorm2, eps0) : 1.f;
+  const int64_t total = rows * ld;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / ld, c = i - r * ld;
+    dst[i] = __float2bfloat16_rn(c < cols ? s * src[r * cols + c] : 0.f);
+  }
+}
+// a += bias; h = act(a) as bf16 (hidden layers)
+__global__ void k_bias_act(float* a, const float* bias, bf16* h, int64_t rows, int64_t N, int64_t ldh, int act) {
+  const int64_t total = rows * N;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / N, n = i - r * N;
+    const float v = a[i] + bias[n];
+    a[i] = v;
+    if (h) h[r * ldh + n] = __float2bfloat16_rn(act_f(act, v));
+  }
+}
+// one warp per row: p = softmax(z), ell = -log p[y]
+__global__ void k_softmax_ce(const float* z, const int32_t* y, float* p, float* ell, int64_t B, int64_t C) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+  if (row >= B) return;
+  const float* zr = z + row * C;
+  float mx = -INFINITY;
+  for (int64_t c = lane; c < C; c += 32) mx = fmaxf(mx, zr[c]);
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  float s = 0.f;
+  for (int64_t c = lane; c < C; c += 32) s += expf(zr[c] - mx);
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  const float ls = logf(s);
+  for (int64_t c = lane; c < C; c += 32) p[row * C + c] = expf(zr[c] - mx - ls);
+  if (lane == 0) {
+    int32_t yy = y[row];
+    yy = yy < 0 ? 0 : (yy >= C ? (int32_t)C - 1 : yy);     // class ids are validated on the host side of a dataset; clamp
+    ell[row] = -(zr[yy] - mx - ls);
+  }
+}
+// delta = coef_i * (p - onehot(y))
+__global__ void k_delta_top(const float* p, const int32_t* y, const float* coef, float scale, bf16* delta, int64_t B,
+                            int64_t C, int64_t ld) {
+  const int64_t total = B * ld;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / ld, c = i - r * ld;
+    float v = 0.f;
+    if (c < C) v = (coef ? coef[r] : scale) * (p[r * C + c] - (c == y[r] ? 1.f : 0.f));
+    delta[i] = __float2bfloat16_rn(v);
+  }
+}
+__global__ void k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, float* out) {
+  const int64_t n = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (n >= N) return;
+  float acc = 0.f;
+  for (int64_t i = 0; i < B; ++i) acc += __bfloat162float(d[i * ld + n]);
+  out[n] = acc;
+}
+// delta_prev = dh * act'(a)
+__global__ void k_act_backward(const float* dh, const float* a, bf16* dprev, int64_t B, int64_t N, int64_t ld, int act) {
+  const int64_t total = B * ld;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / ld, n = i - r * ld;
+    dprev[i] = __float2bfloat16_rn(n < N ? dh[r * N + n] * act_d1(act, a[r * N + n]) : 0.f);
+  }
+}
+// Ra += c ; Rh = act'(a) * Ra
+__global__ void k_r_act_forward(float* Ra, const float* cdir, const float* a, bf16* Rh, int64_t B, int64_t N,
+                                int64_t ldh, int act) {
+  const int64_t total = B * N;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / N, n = i - r * N;
+    const float v = Ra[i] + cdir[n];
+    Ra[i] = v;
+    if (Rh) Rh[r * ldh + n] = __float2bfloat16_rn(act_d1(act, a[i]) * v);
+  }
+}
+// one warp per row: Rdelta = coef_i * (p.*Ra - p * (p . Ra))
+__global__ void k_r_delta_top(const float* p, const float* Ra, const float* coef, float scale, bf16* Rd, int64_t B,
+                              int64_t C, int64_t ld) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+  if (row >= B) return;
+  float s = 0.f;
+  for (int64_t c = lane; c < C; c += 32) s += p[row * C + c] * Ra[row * C + c];
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  const float k = coef ? coef[row] : scale;
+  for (int64_t c = lane; c < ld; c += 32) {
+    float v = 0.f;
+    if (c < C) { const float pc = p[row * C + c]; v = k * (pc * Ra[row * C + c] - pc * s); }
+    Rd[row * ld + c] = __float2bfloat16_rn(v);
+  }
+}
+// Rdelta_prev = Rdh * act'(a) + dh * act''(a) * Ra
+__global__ void k_r_act_backward(const float* Rdh, const float* dh, const float* a, const float* Ra, bf16* Rdprev,
+                                 int64_t B, int64_t N, int64_t ld, int act) {
+  const int64_t total = B * ld;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / ld, n = i - r * ld;
+    float v = 0.f;
+    if (n < N) {
+      const int64_t j = r * N + n;
+      v = Rdh[j] * act_d1(act, a[j]);
+      if (act != BETTY_ACT_RELU) v += dh[j] * act_d2(act, a[j]) * Ra[j];
+    }
+    Rdprev[i] = __float2bfloat16_rn(v);
+  }
+}
+// one warp per row: d_i = sum_c (p - onehot) * Ra
+__global__ void k_jvp_rows(const float* p, const int32_t* y, const float* Ra, float* d, int64_t B, int64_t C) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+  if (row >= B) return;
+  float s = 0.f;
+  for (int64_t c = lane; c < C; c += 32) s += (p[row * C + c] - (c == y[row] ? 1.f : 0.f)) * Ra[row * C + c];
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) d[row] = s;
+}
+__global__ void k_sgd(float* x, const float* g, float lr, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    x[i] -= lr * g[i];
+}
+// out[r, c] += exp(lam) * W[r, c]   (out contiguous [rows, cols]; W bf16 with leading dimension ldw)
+__global__ void k_wd_add_bf16(float* out, const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* lam) {
+  const float k = expf(*lam);
+  const int64_t total = rows * cols;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / cols, c = i - r * cols;
+    out[i] += k * __bfloat162float(W[r * ldw + c]);
+  }
+}
+__global__ void k_wd_add_f32(float* out, const float* u, int64_t n, const float* lam) {
+  const float k = expf(*lam);
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    out[i] += k * u[i];
+}
+// one block: out (+)= scale * exp(lam) * <W, q>  (q == nullptr: <W, W>), fixed summation order
+__global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
+                            float scale, float* out, int accumulate) {
+  __shared__ double sh[32];
+  double acc = 0.0;
+  const int64_t total = rows * cols;
+  for (int64_t i = threadIdx.x; i < total; i += blockDim.x) {
+    const int64_t r = i / cols, c = i - r * cols;
+    const float w = __bfloat162float(W[r * ldw + c]);
+    acc += (double)w * (double)(q ? q[i] : w);
+  }
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += sh[i];
+    const float v = scale * expf(*lam) * (float)t;
+    *out = (accumulate ? *out : 0.f) + v;
+  }
+}
+
+// ------------------------------------------------------------------ weight net 1-100-1
+enum WnMode { WN_REWEIGHT_COEF = 0, WN_REWEIGHT_TGRAD, WN_REWEIGHT_TMIXED, WN_DETECT_TGRAD, WN_DETECT_WGRAD,
+              WN_DETECT_THVP, WN_DETECT_WMIXED };
+
+// One thread per sample: s = a2 . relu(a1*l + b1) + b2, r = sigmoid(s), and the per-sample scalar the
+// caller's reverse sweep needs (see WnMode).  dir: a direction in theta space (modes *_THVP, *_WMIXED).
+__global__ void k_wn_sample(int mode, const float* theta, const float* dir, const float* ell, const float* aux,
+                            const float* din, int64_t B, float invB, float* out1, float* out2) {
+  __shared__ float th[WN_P], dr[WN_P];
+  for (int i = threadIdx.x; i < WN_P; i += blockDim.x) { th[i] = theta[i]; dr[i] = dir ? dir[i] : 0.f; }
+  __syncthreads();
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= B) return;
+  const float l = ell[i];
+  float s = th[3 * WN_H], dsdl = 0.f, Jd = dr[3 * WN_H], dJd = 0.f;
+  for (int k = 0; k < WN_H; ++k) {
+    const float a1 = th[k], b1 = th[WN_H + k], a2 = th[2 * WN_H + k];
+    const float pre = a1 * l + b1;
+    if (pre > 0.f) {
+      s += a2 * pre;
+      dsdl += a1 * a2;
+      Jd += a2 * l * dr[k] + a2 * dr[WN_H + k] + pre * dr[2 * WN_H + k];
+      dJd += a2 * dr[k] + a1 * dr[2 * WN_H + k];
+    }
+  }
+  const float r = 1.f / (1.f + expf(-s));
+  const float rp = r * (1.f - r);
+  const float c = aux ? aux[i] : 0.f;
+  const float fp = 2.f * (r - c) * rp;
+  const float fpp = 2.f * rp * rp + 2.f * (r - c) * rp * (1.f - 2.f * r);
+  switch (mode) {
+    case WN_REWEIGHT_COEF: out1[i] = r * invB; break;
+    case WN_REWEIGHT_TGRAD: out1[i] = l * rp * invB; break;
+    case WN_REWEIGHT_TMIXED: out1[i] = din[i] * rp * invB; break;
+    case WN_DETECT_TGRAD: out1[i] = fp * invB; break;
+    case WN_DETECT_WGRAD: out1[i] = fp * dsdl * invB; break;
+    case WN_DETECT_THVP: out1[i] = fpp * Jd * invB; out2[i] = fp * invB; break;
+    case WN_DETECT_WMIXED: out1[i] = (fpp * dsdl * Jd + fp * dJd) * invB; break;
+  }
+}
+// One block, thread k owns hidden unit k:  out = sum_i cA_i * ds_i/dtheta + cB_i * (d2s_i/dtheta2 . dir) + mu*muvec
+__global__ void k_wn_backward(const float* theta, const float* dir, const float* ell, const float* cA, const float* cB,
+                              int64_t B, float mu, const float* muvec, float* out, int accumulate, float out_scale) {
+  const int k = threadIdx.x;
+  double ga1 = 0.0, gb1 = 0.0, ga2 = 0.0, gb2 = 0.0;
+  if (k < WN_H) {
+    const float a1 = theta[k], b1 = theta[WN_H + k], a2 = theta[2 * WN_H + k];
+    const float da1 = dir ? dir[k] : 0.f, db1 = dir ? dir[WN_H + k] : 0.f, da2 = dir ? dir[2 * WN_H + k] : 0.f;
+    for (int64_t i = 0; i < B; ++i) {
+      const float l = ell[i], ca = cA[i], cb = cB ? cB[i] : 0.f;
+      const float pre = a1 * l + b1;
+      if (pre > 0.f) {
+        const float t = ca * a2 + cb * da2;
+        ga1 += (double)(l * t);
+        gb1 += (double)t;
+        ga2 += (double)(ca * pre + cb * (l * da1 + db1));
+      }
+    }
+  } else if (k == WN_H) {
+    for (int64_t i = 0; i < B; ++i) gb2 += (double)cA[i];
+  }
+  auto put = [&](int idx, double g) {
+    float v = out_scale * ((float)g + (muvec ? mu * muvec[idx] : 0.f));
+    out[idx] = (accumulate ? out[idx] : 0.f) + v;
+  };
+  if (k < WN_H) { put(k, ga1); put(WN_H + k, gb1); put(2 * WN_H + k, ga2); }
+  else if (k == WN_H) put(3 * WN_H, gb2);
+}
+
+// ------------------------------------------------------------------ finite-difference pieces
+// da_tot = da + sign*eps*c.  Hidden layer: hp = act(a + da_tot) -> bf16, dh = hp - act(a) -> bf16.
+// Output layer: z = a + da_tot (fp32).
+__global__ void k_fd_act(const float* a, const float* da, const float* cdir, const float* vnorm2, float eps0, float sign,
+                         bf16* hpm, bf16* dhd, float* zpm, int64_t B, int64_t N, int64_t ldh, int act) {
+  const float e = sign * fd_eps(vnorm2, eps0);
+  const int64_t total = B * N;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / N, n = i - r * N;
+    const float d = da[i] + e * cdir[n];
+    if (zpm) { zpm[i] = a[i] + d; continue; }
+    const float h0 = act_f(act, a[i]), hp = act_f(act, a[i] + d);
+    hpm[r * ldh + n] = __float2bfloat16_rn(hp);
+    dhd[r * ldh + n] = __float2bfloat16_rn(hp - h0);
+  }
+}
+__global__ void k_fd_combine(float* out, const float* gp, const float* gm, const float* vnorm2, float eps0, float alpha,
+                             int accumulate, int64_t n) {
+  const float e = fd_eps(vnorm2, eps0);
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const float base = accumulate ? out[i] : 0.f;
+    out[i] = e > 0.f ? base - alpha * (gp[i] - gm[i]) / (2.f * e) : base;
+  }
+}
+
+// ------------------------------------------------------------------ host-side state
+struct Net {
+  int L;
+  int act;
+  int64_t w[MAXL + 1];
+  int64_t woff[MAXL], boff[MAXL], ldw[MAXL];
+  const float* master;
+  bf16* W[MAXL];
+};
+struct Pass {
+  int64_t B;
+  const int32_t* y;
+  const bf16* h[MAXL];   // h[l]: input of layer l
+  int64_t ldh[MAXL];
+  float* a[MAXL];        // pre-activations [B, w[l+1]]
+  float* p;              // softmax [B, C]
+  float* ell;            // per-sample cross-entropy
+  bf16* delta[MAXL];     // dC/da_l, leading dimension ld8(w[l+1])
+  float* dh[MAXL];       // dC/dh_l (input side of layer l), l >= 1, fp32 [B, w[l]]
+};
+struct MlpHvpCache {
+  Net net;
+  Pass pass;
+  const float* coef;     // per-sample top coefficient (r_i/B) or null (1/B)
+  const float* lam;      // device per-layer log weight decay or null
+  const betty_level* theta;
+};
+
+static betty_status net_layout(const betty_level* M, Net& n) {
+  if (M->param_kind != BETTY_PARAM_MLP || M->n_layers < 1 || M->n_layers > MAXL || !M->widths) return BETTY_ERR_INVALID_ARG;
+  n.L = M->n_layers;
+  n.act = M->activation;
+  if (n.act != BETTY_ACT_RELU && n.act != BETTY_ACT_GELU) return BETTY_ERR_INVALID_ARG;
+  int64_t off = 0;
+  for (int l = 0; l <= n.L; ++l) {
+    n.w[l] = M->widths[l];
+    if (n.w[l] <= 0) return BETTY_ERR_SHAPE;
+  }
+  for (int l = 0; l < n.L; ++l) {
+    n.woff[l] = off; off += n.w[l + 1] * n.w[l];
+    n.boff[l] = off; off += n.w[l + 1];
+    n.ldw[l] = ld8(n.w[l]);
+  }
+  if (off != M->n_params) return BETTY_ERR_SHAPE;
+  n.master = M->params;
+  return BETTY_OK;
+}
+
+static betty_status cast_matrix(Ctx& c, const float* src, bf16* dst, int64_t rows, int64_t cols, int64_t ld,
+                                const float* vnorm2 = nullptr, float eps0 = 0.f) {
+  k_cast_rows<<<grid_for(rows * ld), 256, 0, c.stream>>>(src, dst, rows, cols, ld, vnorm2, eps0);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
+// bf16 compute copy of the classifier's matrices (the single quantisation point)
+static betty_status net_setup(Ctx& c, const betty_level* M, Net& n) {
+  BETTY_TRY(net_layout(M, n));
+  for (int l = 0; l < n.L; ++l) {
+    BETTY_ALLOC(Wl, bf16, c, (size_t)(n.w[l + 1] * n.ldw[l]));
+    n.W[l] = Wl;
+    BETTY_TRY(cast_matrix(c, n.master + n.woff[l], Wl, n.w[l + 1], n.w[l], n.ldw[l]));
+  }
+  return BETTY_OK;
+}
+
+static betty_status forward(Ctx& c, const Net& n, const betty_level* D, Pass& ps) {
+  ps.B = D->n;
+  ps.y = (const int32_t*)D->y;
+  const int64_t B = ps.B;
+  ps.h[0] = (const bf16*)D->X;
+  ps.ldh[0] = D->d;
+  for (int l = 0; l < n.L; ++l) {
+    const int64_t N = n.w[l + 1];
+    BETTY_ALLOC(al, float, c, (size_t)(B * N));
+    ps.a[l] = al;
+    GemmDesc g; g.M = (int)B; g.N = (int)N; g.npairs = 1; g.C = al; g.ldc = N; g.beta = 0.f;
+    g.p[0] = gemm_pair(ps.h[l], ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)n.w[l]);
+    BETTY_TRY(gemm(c, g));
+    bf16* hn = nullptr;
+    if (l < n.L - 1) {
+      ps.ldh[l + 1] = ld8(N);
+      hn = c.arena.alloc<bf16>((size_t)(B * ps.ldh[l + 1]));
+      if (!hn) return BETTY_ERR_WORKSPACE;
+      if (ps.ldh[l + 1] != N) cudaMemsetAsync(hn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(bf16), c.stream);
+      ps.h[l + 1] = hn;
+    }
+    k_bias_act<<<grid_for(B * N), 256, 0, c.stream>>>(al, n.master + n.boff[l], hn, B, N, hn ? ps.ldh[l + 1] : 0, n.act);
+    BETTY_LAUNCH_CHECK();
+  }
+  const int64_t C = n.w[n.L];
+  BETTY_ALLOC(p, float, c, (size_t)(B * C));
+  BETTY_ALLOC(ell, float, c, (size_t)B);
+  ps.p = p; ps.ell = ell;
+  k_softmax_ce<<<grid_for(B * 32), 256, 0, c.stream>>>(ps.a[n.L - 1], ps.y, p, ell, B, C);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
+// Reverse sweep from delta_top = coef_i (p - onehot).  gflat (nullable): receives [gW_l, gb_l]; lam
+// (nullable): adds exp(lam_l) W_l.  Always leaves delta[l] and dh[l] in `ps` for an R-operator pass.
+static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, float* gflat, const float* lam) {
+  const int64_t B = ps.B;
+  const int64_t C = n.w[n.L];
+  {
+    const int64_t ld = ld8(C);
+    BETTY_ALLOC(dt, bf16, c, (size_t)(B * ld));
+    ps.delta[n.L - 1] = dt;
+    k_delta_top<<<grid_for(B * ld), 256, 0, c.stream>>>(ps.p, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld);
+    BETTY_LAUNCH_CHECK();
+  }
+  for (int l = n.L - 1; l >= 0; --l) {
+    const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
+    if (gflat) {
+      GemmDesc g; g.M = (int)N; g.N = (int)K; g.npairs = 1; g.C = gflat + n.woff[l]; g.ldc = K; g.beta = 0.f;
+      g.p[0] = gemm_pair(ps.delta[l], ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
+      BETTY_TRY(gemm(c, g));
+      if (lam) {
+        k_wd_add_bf16<<<grid_for(N * K), 256, 0, c.stream>>>(gflat + n.woff[l], n.W[l], N, K, n.ldw[l], lam + l);
+        BETTY_LAUNCH_CHECK();
+      }
+      k_colsum_bf16<<<grid_for(N), 256, 0, c.stream>>>(ps.delta[l], B, N, ldd, gflat + n.boff[l]);
+      BETTY_LAUNCH_CHECK();
+    }
+    if (l > 0) {
+      BETTY_ALLOC(dh, float, c, (size_t)(B * K));
+      ps.dh[l] = dh;
+      GemmDesc g; g.M = (int)B; g.N = (int)K; g.npairs = 1; g.C = dh; g.ldc = K; g.beta = 0.f;
+      g.p[0] = gemm_pair(ps.delta[l], ldd, false, n.W[l], n.ldw[l], false, (int)N);
+      BETTY_TRY(gemm(c, g));
+      const int64_t ldp = ld8(K);
+      BETTY_ALLOC(dp, bf16, c, (size_t)(B * ldp));
+      ps.delta[l - 1] = dp;
+      k_act_backward<<<grid_for(B * ldp), 256, 0, c.stream>>>(dh, ps.a[l - 1], dp, B, K, ldp, n.act);
+      BETTY_LAUNCH_CHECK();
+    }
+  }
+  return BETTY_OK;
+}
+
+// Directional derivative of the forward pass along `dir` (flat, same layout as the parameters).
+struct RPass {
+  bf16* U[MAXL];
+  float* Ra[MAXL];
+  const bf16* Rh[MAXL];   // Rh[0] == nullptr (inputs do not move)
+};
+static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* dir, RPass& rp) {
+  const int64_t B = ps.B;
+  rp.Rh[0] = nullptr;
+  for (int l = 0; l < n.L; ++l) {
+    const int64_t N = n.w[l + 1], K = n.w[l];
+    BETTY_ALLOC(Ul, bf16, c, (size_t)(N * n.ldw[l]));
+    rp.U[l] = Ul;
+    BETTY_TRY(cast_matrix(c, dir + n.woff[l], Ul, N, K, n.ldw[l]));
+    BETTY_ALLOC(Ra, float, c, (size_t)(B * N));
+    rp.Ra[l] = Ra;
+    GemmDesc g; g.M = (int)B; g.N = (int)N; g.C = Ra; g.ldc = N; g.beta = 0.f;
+    g.npairs = 0;
+    g.p[g.npairs++] = gemm_pair(ps.h[l], ps.ldh[l], false, Ul, n.ldw[l], true, (int)K);
+    if (l > 0) g.p[g.npairs++] = gemm_pair(rp.Rh[l], ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)K);
+    BETTY_TRY(gemm(c, g));
+    bf16* Rhn = nullptr;
+    if (l < n.L - 1) {
+      Rhn = c.arena.alloc<bf16>((size_t)(B * ps.ldh[l + 1]));
+      if (!Rhn) return BETTY_ERR_WORKSPACE;
+      if (ps.ldh[l + 1] != N) cudaMemsetAsync(Rhn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(bf16), c.stream);
+      rp.Rh[l + 1] = Rhn;
+    }
+    k_r_act_forward<<<grid_for(B * N), 256, 0, c.stream>>>(Ra, dir + n.boff[l], ps.a[l], Rhn, B, N,
+                                                          Rhn ? ps.ldh[l + 1] : 0, n.act);
+    BETTY_LAUNCH_CHECK();
+  }
+  return BETTY_OK;
+}
+
+// ------------------------------------------------------------------ participants
+struct Parts {
+  const betty_level* mlp;
+  const betty_level* theta;   // weight net or null
+  const betty_level* lam;     // log weight decay or null
+};
+static Parts parts_of(const betty_level* L) {
+  Parts p;
+  p.mlp = find_participant(L, BETTY_PARAM_MLP);
+  if (L->loss == BETTY_LOSS_WEIGHTNET_DETECT) {
+    p.theta = find_participant(L, BETTY_PARAM_WEIGHTNET);
+    p.lam = nullptr;
+  } else if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
+    p.theta = find_constraint(L, BETTY_PARAM_WEIGHTNET);
+    p.lam = find_constraint(L, BETTY_PARAM_LOGWD);
+  } else {
+    p.theta = nullptr; p.lam = nullptr;
+  }
+  return p;
+}
+
+betty_status mlpfam_validate(const betty_level* L) {
+  const Parts P = parts_of(L);
+  if (!P.mlp || !P.mlp->params) return BETTY_ERR_INVALID_ARG;
+  if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT && L->param_kind != BETTY_PARAM_MLP) return BETTY_ERR_INVALID_ARG;
+  Net n;
+  BETTY_TRY(net_layout(P.mlp, n));
+  if (L->n < 0 || L->d != n.w[0]) return BETTY_ERR_SHAPE;
+  if (L->x_dtype != BETTY_BF16) return BETTY_ERR_DTYPE;
+  if (L->n > 0 && (!L->X || !L->y)) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(L->X) || !aligned16(P.mlp->params)) return BETTY_ERR_ALIGNMENT;
+  if (L->d % 8 != 0) return BETTY_ERR_ALIGNMENT;     // bf16 rows must start on 16-byte boundaries
+  if (P.theta && (P.theta->n_params != WN_P || !P.theta->params)) return BETTY_ERR_SHAPE;
+  if (P.lam && (P.lam->n_params != n.L || !P.lam->params)) return BETTY_ERR_SHAPE;
+  if (L->loss == BETTY_LOSS_WEIGHTNET_DETECT) {
+    if (!P.theta) return BETTY_ERR_INVALID_ARG;
+    if (L->n > 0 && !L->aux) return BETTY_ERR_INVALID_ARG;
+  }
+  return BETTY_OK;
+}
+
+size_t mlpfam_workspace(const betty_level* L) {
+  const Parts P = parts_of(L);
+  if (!P.mlp || !P.mlp->widths) return 0;
+  size_t S = 0;
+  for (int l = 0; l <= P.mlp->n_layers; ++l) S += (size_t)ld8(P.mlp->widths[l]) + 8;
+  const size_t B = (size_t)(L->n > 0 ? L->n : 1);
+  return 24 * (size_t)P.mlp->n_params + 96 * B * S + 64 * 256 * (size_t)(P.mlp->n_layers + 4) + (1 << 20);
+}
+
+// per-sample scalar through the weight net
+static betty_status wn_sample(Ctx& c, int mode, const betty_level* theta, const float* dir, const Pass& ps,
+                              const float* aux, const float* din, float* out1, float* out2) {
+  const int64_t B = ps.B;
+  k_wn_sample<<<grid_for(B, 128), 128, 0, c.stream>>>(mode, theta->params, dir, ps.ell, aux, din, B,
+                                                      B > 0 ? 1.f / (float)B : 0.f, out1, out2);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+static betty_status wn_backward(Ctx& c, const betty_level* theta, const float* dir, const Pass& ps, const float* cA,
+                                const float* cB, float mu, const float* muvec, float* out, bool accumulate = false,
+                                float out_scale = 1.f) {
+  k_wn_backward<<<1, 128, 0, c.stream>>>(theta->params, dir, ps.ell, cA, cB, ps.B, mu, muvec, out, accumulate ? 1 : 0,
+                                         out_scale);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
+// top coefficient of the classifier's own cost: r_i/B with a weight net attached, else 1/B (null)
+static betty_status reweight_coef(Ctx& c, const Parts& P, const Pass& ps, const float** coef) {
+  *coef = nullptr;
+  if (!P.theta) return BETTY_OK;
+  BETTY_ALLOC(cf, float, c, (size_t)(ps.B > 0 ? ps.B : 1));
+  BETTY_TRY(wn_sample(c, WN_REWEIGHT_COEF, P.theta, nullptr, ps, nullptr, nullptr, cf, nullptr));
+  *coef = cf;
+  return BETTY_OK;
+}
+
+betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out) {
+  const Parts P = parts_of(L);
+  const size_t mark = c.arena.mark();
+  const bool touches = (wrt == P.mlp) || (P.theta && wrt == P.theta) || (P.lam && wrt == P.lam);
+  if (!touches) return vec_zero(c, out, wrt->n_params);
+  Net n; Pass ps;
+  BETTY_TRY(net_setup(c, P.mlp, n));
+  if (P.lam && wrt == P.lam) {
+    for (int l = 0; l < n.L; ++l) {
+      k_layer_dot<<<1, 1024, 0, c.stream>>>(n.W[l], n.w[l + 1], n.w[l], n.ldw[l], nullptr, P.lam->params + l, 0.5f, out + l, 0);
+      BETTY_LAUNCH_CHECK();
+    }
+    c.arena.release(mark);
+    return BETTY_OK;
+  }
+  BETTY_TRY(forward(c, n, L, ps));
+  BETTY_ALLOC(s1, float, c, (size_t)(ps.B > 0 ? ps.B : 1));
+  if (L->loss == BETTY_LOSS_MLP_CE) {
+    BETTY_TRY(backward(c, n, ps, nullptr, out, nullptr));
+  } else if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
+    if (wrt == P.mlp) {
+      const float* coef;
+      BETTY_TRY(reweight_coef(c, P, ps, &coef));
+      BETTY_TRY(backward(c, n, ps, coef, out, P.lam ? P.lam->params : nullptr));
+    } else {
+      BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, ps, nullptr, nullptr, s1, nullptr));
+      BETTY_TRY(wn_backward(c, P.theta, nullptr, ps, s1, nullptr, 0.f, nullptr, out));
+    }
+  } else {  // WEIGHTNET_DETECT
+    if (wrt == P.theta) {
+      BETTY_TRY(wn_sample(c, WN_DETECT_TGRAD, P.theta, nullptr, ps, L->aux, nullptr, s1, nullptr));
+      BETTY_TRY(wn_backward(c, P.theta, nullptr, ps, s1, nullptr, L->mu, P.theta->params, out));
+    } else {
+      BETTY_TRY(wn_sample(c, WN_DETECT_WGRAD, P.theta, nullptr, ps, L->aux, nullptr, s1, nullptr));
+      BETTY_TRY(backward(c, n, ps, s1, out, nullptr));
+    }
+  }
+  c.arena.release(mark);
+  return BETTY_OK;
+}
+
+betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache) {
+  static thread_local MlpHvpCache store;   // host-side bookkeeping only; device state lives in the workspace
+  MlpHvpCache& h = store;
+  const Parts P = parts_of(L);
+  h.theta = P.theta;
+  h.lam = P.lam ? P.lam->params : nullptr;
+  h.coef = nullptr;
+  BETTY_TRY(net_setup(c, P.mlp, h.net));
+  BETTY_TRY(forward(c, h.net, L, h.pass));
+  if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
+    BETTY_TRY(reweight_coef(c, P, h.pass, &h.coef));
+    BETTY_TRY(backward(c, h.net, h.pass, h.coef, nullptr, nullptr));
+  } else if (!(L->loss == BETTY_LOSS_WEIGHTNET_DETECT && L->param_kind == BETTY_PARAM_WEIGHTNET)) {
+    return BETTY_ERR_UNSUPPORTED;
+  }
+  *cache = &h;
+  return BETTY_OK;
+}
+
+betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* u, float* Hu) {
+  const size_t mark = c.arena.mark();
+  const Net& n = h->net;
+  Pass& ps = h->pass;
+  const int64_t B = ps.B;
+  if (L->loss == BETTY_LOSS_WEIGHTNET_DETECT) {
+    BETTY_ALLOC(cA, float, c, (size_t)(B > 0 ? B : 1));
+    BETTY_ALLOC(cB, float, c, (size_t)(B > 0 ? B : 1));
+    BETTY_TRY(wn_sample(c, WN_DETECT_THVP, L, u, ps, L->aux, nullptr, cA, cB));
+    BETTY_TRY(wn_backward(c, L, u, ps, cA, cB, L->mu, u, Hu));
+    c.arena.release(mark);
+    return BETTY_OK;
+  }
+  RPass rp;
+  BETTY_TRY(rforward(c, n, ps, u, rp));
+  const int64_t C = n.w[n.L];
+  bf16* Rd;
+  {
+    const int64_t ld = ld8(C);
+    Rd = c.arena.alloc<bf16>((size_t)(B * ld));
+    if (!Rd) return BETTY_ERR_WORKSPACE;
+    k_r_delta_top<<<grid_for(B * 32), 256, 0, c.stream>>>(ps.p, rp.Ra[n.L - 1], h->coef, B > 0 ? 1.f / (float)B : 0.f, Rd,
+                                                         B, C, ld);
+    BETTY_LAUNCH_CHECK();
+  }
+  for (int l = n.L - 1; l >= 0; --l) {
+    const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
+    {  // R gW_l = Rdelta^T h_l + delta_l^T Rh_l + exp(lam_l) U_l
+      GemmDesc g; g.M = (int)N; g.N = (int)K; g.C = Hu + n.woff[l]; g.ldc = K; g.beta = 0.f; g.npairs = 0;
+      g.p[g.npairs++] = gemm_pair(Rd, ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
+      if (l > 0) g.p[g.npairs++] = gemm_pair(ps.delta[l], ldd, true, rp.Rh[l], ps.ldh[l], false, (int)B);
+      BETTY_TRY(gemm(c, g));
+      if (h->lam) {
+        k_wd_add_f32<<<grid_for(N * K), 256, 0, c.stream>>>(Hu + n.woff[l], u + n.woff[l], N * K, h->lam + l);
+        BETTY_LAUNCH_CHECK();
+      }
+      k_colsum_bf16<<<grid_for(N), 256, 0, c.stream>>>(Rd, B, N, ldd, Hu + n.boff[l]);
+      BETTY_LAUNCH_CHECK();
+    }
+    if (l > 0) {  // R dh = Rdelta W_l + delta_l U_l ; Rdelta_{l-1} = Rdh*act' + dh*act''*Ra
+      BETTY_ALLOC(Rdh, float, c, (size_t)(B * K));
+      GemmDesc g; g.M = (int)B; g.N = (int)K; g.C = Rdh; g.ldc = K; g.beta = 0.f; g.npairs = 2;
+      g.p[0] = gemm_pair(Rd, ldd, false, n.W[l], n.ldw[l], false, (int)N);
+      g.p[1] = gemm_pair(ps.delta[l], ldd, false, rp.U[l], n.ldw[l], false, (int)N);
+      BETTY_TRY(gemm(c, g));
+      const int64_t ldp = ld8(K);
+      BETTY_ALLOC(Rdp, bf16, c, (size_t)(B * ldp));
+      k_r_act_backward<<<grid_for(B * ldp), 256, 0, c.stream>>>(Rdh, ps.dh[l], ps.a[l - 1], rp.Ra[l - 1], Rdp, B, K, ldp,
+                                                              n.act);
+      BETTY_LAUNCH_CHECK();
+      Rd = Rdp;
+    }
+  }
+  c.arena.release(mark);
+  return BETTY_OK;
+}
+
+betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const betty_level* wrt, const float* q,
+                          float* out) {
+  const size_t mark = c.arena.mark();
+  const Parts P = parts_of(L);
+  const Net& n = h->net;
+  Pass& ps = h->pass;
+  const int64_t B = ps.B;
+  if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
+    if (P.lam && wrt == P.lam) {
+      for (int l = 0; l < n.L; ++l) {
+        k_layer_dot<<<1, 1024, 0, c.stream>>>(n.W[l], n.w[l + 1], n.w[l], n.ldw[l], q + n.woff[l], P.lam->params + l, 1.f,
+                                              out + l, 0);
+        BETTY_LAUNCH_CHECK();
+      }
+    } else if (P.theta && wrt == P.theta) {
+      RPass rp;
+      BETTY_TRY(rforward(c, n, ps, q, rp));
+      BETTY_ALLOC(d, float, c, (size_t)(B > 0 ? B : 1));
+      BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
+      k_jvp_rows<<<grid_for(B * 32), 256, 0, c.stream>>>(ps.p, ps.y, rp.Ra[n.L - 1], d, B, n.w[n.L]);
+      BETTY_LAUNCH_CHECK();
+      BETTY_TRY(wn_sample(c, WN_REWEIGHT_TMIXED, P.theta, nullptr, ps, nullptr, d, s1, nullptr));
+      BETTY_TRY(wn_backward(c, P.theta, nullptr, ps, s1, nullptr, 0.f, nullptr, out));
+    } else {
+      return BETTY_ERR_INVALID_ARG;
+    }
+  } else if (L->loss == BETTY_LOSS_WEIGHTNET_DETECT && L->param_kind == BETTY_PARAM_WEIGHTNET && wrt == P.mlp) {
+    BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
+    BETTY_TRY(wn_sample(c, WN_DETECT_WMIXED, L, q, ps, L->aux, nullptr, s1, nullptr));
+    BETTY_TRY(backward(c, n, ps, s1, out, nullptr));
+  } else {
+    return BETTY_ERR_INVALID_ARG;
+  }
+  c.arena.release(mark);
+  return BETTY_OK;
+}
+
+betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps) {
+  if (L->loss != BETTY_LOSS_MLP_CE_REWEIGHT) return BETTY_ERR_UNSUPPORTED;
+  const size_t mark = c.arena.mark();
+  BETTY_ALLOC(g, float, c, (size_t)L->n_params);
+  for (int s = 0; s < n_steps; ++s) {
+    BETTY_TRY(mlpfam_grad(c, L, L, g));
+    k_sgd<<<grid_for(L->n_params, 1024), 256, 0, c.stream>>>(L->params, g, L->lr, L->n_params);
+    BETTY_LAUNCH_CHECK();
+  }
+  c.arena.release(mark);
+  return BETTY_OK;
+}
+
+// Finite difference of dC/dc at x +- eps v.  For the weight-net constraint the two perturbed forward
+// passes carry the perturbation separately from the base activations (base + delta operands), so that
+// an eps*v far below bf16 resolution of the weights survives the bf16 matrix products.
+betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
+                       float eps0, float alpha, float* out, bool accumulate) {
+  if (L->loss != BETTY_LOSS_MLP_CE_REWEIGHT) return BETTY_ERR_UNSUPPORTED;
+  const Parts P = parts_of(L);
+  const size_t mark = c.arena.mark();
+  Net n; Pass ps;
+  BETTY_TRY(net_setup(c, P.mlp, n));
+  if (P.lam && wrt == P.lam) {
+    // dC/d(lam_l) = 1/2 exp(lam_l)|W_l|^2 is quadratic in W: its central difference is exactly
+    // exp(lam_l) <W_l, V_l> for every eps, which is what is evaluated.
+    for (int l = 0; l < n.L; ++l) {
+      k_layer_dot<<<1, 1024, 0, c.stream>>>(n.W[l], n.w[l + 1], n.w[l], n.ldw[l], v + n.woff[l], P.lam->params + l, -alpha,
+                                            out + l, accumulate ? 1 : 0);
+      BETTY_LAUNCH_CHECK();
+    }
+    c.arena.release(mark);
+    return BETTY_OK;
+  }
+  if (!P.theta || wrt != P.theta) return BETTY_ERR_INVALID_ARG;
+  BETTY_TRY(forward(c, n, L, ps));
+  const int64_t B = ps.B, C = n.w[n.L];
+  bf16* E[MAXL];
+  for (int l = 0; l < n.L; ++l) {
+    E[l] = c.arena.alloc<bf16>((size_t)(n.w[l + 1] * n.ldw[l]));
+    if (!E[l]) return BETTY_ERR_WORKSPACE;
+    BETTY_TRY(cast_matrix(c, v + n.woff[l], E[l], n.w[l + 1], n.w[l], n.ldw[l], vnorm2, eps0));
+  }
+  BETTY_ALLOC(G, float, c, 2 * 512);
+  BETTY_ALLOC(zpm, float, c, (size_t)(B * C));
+  BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
+  Pass pp = ps;   // perturbed pass: reuses y/B, gets its own p/ell
+  BETTY_ALLOC(p2, float, c, (size_t)(B * C));
+  BETTY_ALLOC(ell2, float, c, (size_t)(B > 0 ? B : 1));
+  pp.p = p2; pp.ell = ell2;
+  for (int sgn = 0; sgn < 2; ++sgn) {
+    const float sign = sgn == 0 ? 1.f : -1.f;
+    const size_t m2 = c.arena.mark();
+    const bf16* hp = ps.h[0];      // perturbed input of the layer (layer 0: the data itself)
+    const bf16* dh = nullptr;      // its difference from the base input
+    for (int l = 0; l < n.L; ++l) {
+      const int64_t N = n.w[l + 1], K = n.w[l];
+      BETTY_ALLOC(da, float, c, (size_t)(B * N));
+      GemmDesc g; g.M = (int)B; g.N = (int)N; g.C = da; g.ldc = N; g.beta = 0.f; g.npairs = 0;
+      g.p[g.npairs++] = gemm_pair(hp, ps.ldh[l], false, E[l], n.ldw[l], true, (int)K, sign);
+      if (l > 0) g.p[g.npairs++] = gemm_pair(dh, ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)K);
+      BETTY_TRY(gemm(c, g));
+      if (l < n.L - 1) {
+        const size_t cnt = (size_t)(B * ps.ldh[l + 1]);
+        BETTY_ALLOC(hn, bf16, c, cnt);
+        BETTY_ALLOC(dn, bf16, c, cnt);
+        if (ps.ldh[l + 1] != N) {
+          cudaMemsetAsync(hn, 0, cnt * sizeof(bf16), c.stream);
+          cudaMemsetAsync(dn, 0, cnt * sizeof(bf16), c.stream);
+        }
+        k_fd_act<<<grid_for(B * N), 256, 0, c.stream>>>(ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, hn, dn, nullptr, B, N,
+                                                       ps.ldh[l + 1], n.act);
+        BETTY_LAUNCH_CHECK();
+        hp = hn; dh = dn;
+      } else {
+        k_fd_act<<<grid_for(B * N), 256, 0, c.stream>>>(ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, nullptr, nullptr, zpm,
+                                                       B, N, 0, n.act);
+        BETTY_LAUNCH_CHECK();
+      }
+    }
+    k_softmax_ce<<<grid_for(B * 32), 256, 0, c.stream>>>(zpm, ps.y, pp.p, pp.ell, B, C);
+    BETTY_LAUNCH_CHECK();
+    BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, pp, nullptr, nullptr, s1, nullptr));
+    BETTY_TRY(wn_backward(c, P.theta, nullptr, pp, s1, nullptr, 0.f, nullptr, G + 512 * sgn));
+    c.arena.release(m2);
+  }
+  k_fd_combine<<<grid_for(WN_P), 256, 0, c.stream>>>(out, G, G + 512, vnorm2, eps0, alpha, accumulate ? 1 : 0, WN_P);
+  BETTY_LAUNCH_CHECK();
+  c.arena.release(mark);
+  return BETTY_OK;
+}
+
+}  // namespace betty

@@ -1,0 +1,193 @@
+"""Parity of the CUDA path with the fp64 oracle for the MLP cost families (data reweighting,
+three-level chain), through the C ABI, on the same seeded inputs.  bf16 matrices with fp32
+accumulation: relative L2 error <= 2e-2 (the oracle consumes the same bf16-rounded weights and
+inputs and computes everything else in fp64)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from tests import oracle_build as ob
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def bt():
+    import paper_2207_02849_b200 as bt
+    return bt
+
+
+def _vec(n):
+    return torch.empty(n, dtype=torch.float32, device="cuda")
+
+
+def _perturb(inp, seed):
+    """Move away from the symmetric initialisation: non-zero biases, a livelier weight net."""
+    inp.w = inp.w + si.to_bf16_values(si.normal_f32(seed, 300, inp.w.shape) * np.float32(0.02))
+    inp.theta = (si.weightnet_init(seed, 200) * np.float32(3.0)).astype(np.float32)
+    return inp
+
+
+@pytest.mark.parametrize("act,widths,B", [("relu", (24, 40, 16), 37), ("gelu", (24, 40, 16), 37),
+                                          ("gelu", (16, 72, 64, 10), 130), ("relu", (784, 96, 10), 64)])
+def test_reweight_primitives_match_oracle(bt, act, widths, B):
+    from tests import cuda_build as cb
+    inp = _perturb(si.reweight_bilevel(41, widths, B, 0.4, activation=act), 41)
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    ws = bt.Workspace([w, th])
+    P = inp.w.size
+    out, outt = _vec(P), _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_grad(w, w, out, ws)
+    assert cb.rel_l2(out, oracle.grad(ow, ow)) < TOL
+    bt.betty_grad(w, th, outt, ws)
+    assert cb.rel_l2(outt, oracle.grad(ow, oth)) < TOL
+    bt.betty_grad(th, w, out, ws)
+    assert cb.rel_l2(out, oracle.grad(oth, ow)) < TOL
+    bt.betty_grad(th, th, outt, ws)
+    assert torch.all(outt == 0)
+    u = si.normal_f32(43, 1, (P,))
+    bt.betty_hvp(w, cb.dev(u), out, ws)
+    assert cb.rel_l2(out, oracle.hvp(ow, u)) < TOL
+    bt.betty_mixed_vjp(w, th, cb.dev(u), outt, ws)
+    assert cb.rel_l2(outt, oracle.mixed_vjp(ow, oth, u)) < TOL
+    bt.betty_lower_step(w, 2, ws)
+    oracle.lower_step(ow, 2)
+    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+@pytest.mark.parametrize("act", ["relu", "gelu"])
+def test_reweight_hypergradients_match_oracle(bt, act):
+    from tests import cuda_build as cb
+    inp = _perturb(si.reweight_bilevel(47, (64, 96, 10), 128, 0.4, activation=act), 47)
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    ws = bt.Workspace([w, th])
+    bt.betty_lower_step(w, 1, ws)
+    oracle.lower_step(ow, 1)
+    out = _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_hypergrad_neumann(w, th, th, 5, 0.01, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_neumann(ow, oth, oth, 5, 0.01)) < TOL
+    bt.betty_hypergrad_fd(w, th, th, 0.01, 1.0, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_fd(ow, oth, oth, 0.01, 1.0)) < TOL
+    bt.betty_hypergrad_cg(w, th, th, 3, 0.0, out, ws)
+    info = {}
+    ref = oracle.hypergrad_cg(ow, oth, oth, 3, 0.0, info=info)
+    st, iters = bt.betty_poll_status(ws, raise_on_error=False)
+    if info["status"] == "ok":
+        assert st == bt.BETTY_OK and iters == info["iters"]
+        assert cb.rel_l2(out, ref) < 5e-2          # CG divides by p^T H p: looser in bf16
+    else:
+        assert st == bt.BETTY_ERR_BREAKDOWN
+
+
+def _three(act="relu", widths=(32, 48, 40, 10), B=96, seed=53):
+    inp = si.three_level(seed, widths, B, 0.3, activation=act)
+    inp.w = inp.w + si.to_bf16_values(si.normal_f32(seed, 300, inp.w.shape) * np.float32(0.02))
+    inp.theta = (si.weightnet_init(seed, 200) * np.float32(3.0)).astype(np.float32)
+    return inp
+
+
+@pytest.mark.parametrize("act", ["relu", "gelu"])
+def test_three_level_primitives_and_chain_match_oracle(bt, act):
+    from tests import cuda_build as cb
+    inp = _three(act)
+    P1, P2, P3 = cb.three_levels(inp)
+    O1, O2, O3 = ob.three_levels(inp)
+    ws = bt.Workspace([P1, P2, P3])
+    Pw, Pt, Pl = inp.w.size, si.WEIGHTNET_PARAMS, inp.lam.size
+    gw, gt, gl = _vec(Pw), _vec(Pt), _vec(Pl)
+    # classifier with both constraints attached
+    bt.betty_grad(P1, P1, gw, ws); assert cb.rel_l2(gw, oracle.grad(O1, O1)) < TOL
+    bt.betty_grad(P1, P3, gl, ws); assert cb.rel_l2(gl, oracle.grad(O1, O3)) < 1e-4
+    u = si.normal_f32(55, 1, (Pw,))
+    bt.betty_hvp(P1, cb.dev(u), gw, ws); assert cb.rel_l2(gw, oracle.hvp(O1, u)) < TOL
+    bt.betty_mixed_vjp(P1, P3, cb.dev(u), gl, ws); assert cb.rel_l2(gl, oracle.mixed_vjp(O1, O3, u)) < 1e-4
+    bt.betty_mixed_vjp(P1, P2, cb.dev(u), gt, ws); assert cb.rel_l2(gt, oracle.mixed_vjp(O1, O2, u)) < TOL
+    # detector cost: middle level and top level
+    bt.betty_grad(P2, P2, gt, ws); assert cb.rel_l2(gt, oracle.grad(O2, O2)) < TOL
+    bt.betty_grad(P2, P1, gw, ws); assert cb.rel_l2(gw, oracle.grad(O2, O1)) < TOL
+    bt.betty_grad(P3, P2, gt, ws); assert cb.rel_l2(gt, oracle.grad(O3, O2)) < TOL
+    bt.betty_grad(P3, P1, gw, ws); assert cb.rel_l2(gw, oracle.grad(O3, O1)) < TOL
+    q = si.normal_f32(55, 2, (Pt,))
+    bt.betty_hvp(P2, cb.dev(q), gt, ws); assert cb.rel_l2(gt, oracle.hvp(O2, q)) < TOL
+    bt.betty_mixed_vjp(P2, P1, cb.dev(q), gw, ws); assert cb.rel_l2(gw, oracle.mixed_vjp(O2, O1, q)) < TOL
+    # the level-3 hypergradient: both paths from lambda merged at the w* node
+    nm = dict(method="neumann", K=3, alpha=0.01)
+    cfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=3, alpha=0.01)
+    ref_a = oracle.chain_levels([O1, O2, O3], [2, 0], [nm])
+    ref_b = oracle.chain_levels([O1, O2, O3], [2, 0, 1], [nm, nm])
+    out = _vec(Pl)
+    bt.betty_chain_levels([P1, P2, P3], [2, 0], [cfg], None, out, False, ws)
+    assert cb.rel_l2(out, ref_a) < TOL
+    bt.betty_chain_levels([P1, P2, P3], [2, 0, 1], [cfg, cfg], None, out, False, ws)
+    assert cb.rel_l2(out, ref_b) < TOL
+    v_t = _vec(Pt)
+    bt.betty_grad(P3, P1, gw, ws)                                                   # u <- dC3/dw*
+    bt.betty_grad(P3, P2, v_t, ws)
+    bt.betty_chain_levels([P1, P2, P3], [0, 1], [cfg], v_t, gw, True, ws)           # u += BRJ(P2, w; dC3/dtheta*)
+    bt.betty_chain_levels([P1, P2, P3], [2, 0], [cfg], gw, out, False, ws)          # out = BRJ(P1, lambda; u)
+    assert cb.rel_l2(out, ref_a + ref_b) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+def test_config3_full_size(bt):
+    """3072 -> 1024 -> 10, batch 512: one lower step, then the finite-difference and the Neumann
+    (K = 5) hypergradients of the weight net."""
+    from tests import cuda_build as cb
+    inp = si.config3()
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    ws = bt.Workspace([w, th])
+    bt.betty_lower_step(w, inp.lower_steps, ws)
+    oracle.lower_step(ow, inp.lower_steps)
+    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    out = _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_hypergrad_fd(w, th, th, inp.eps0, inp.fd_alpha, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_fd(ow, oth, oth, inp.eps0, inp.fd_alpha)) < TOL
+    bt.betty_hypergrad_neumann(w, th, th, inp.K, inp.alpha, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+def test_config4_full_size(bt):
+    """784 -> 512 -> 512 -> 10, batch 1024, three levels, two Neumann (K = 3) edges."""
+    from tests import cuda_build as cb
+    inp = si.config4()
+    P1, P2, P3 = cb.three_levels(inp)
+    O1, O2, O3 = ob.three_levels(inp)
+    ws = bt.Workspace([P1, P2, P3])
+    bt.betty_lower_step(P1, 1, ws)
+    oracle.lower_step(O1, 1)
+    cfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=inp.K, alpha=inp.alpha)
+    nm = dict(method="neumann", K=inp.K, alpha=inp.alpha)
+    u, v_t, out = _vec(inp.w.size), _vec(si.WEIGHTNET_PARAMS), _vec(inp.lam.size)
+    bt.betty_grad(P3, P1, u, ws)
+    bt.betty_grad(P3, P2, v_t, ws)
+    bt.betty_chain_levels([P1, P2, P3], [0, 1], [cfg], v_t, u, True, ws)
+    bt.betty_chain_levels([P1, P2, P3], [2, 0], [cfg], u, out, False, ws)
+    ou = oracle.grad(O3, O1) + oracle.chain_levels([O1, O2, O3], [0, 1], [nm], v_in=oracle.grad(O3, O2))
+    ref = oracle.chain_levels([O1, O2, O3], [2, 0], [nm], v_in=ou)
+    assert cb.rel_l2(u, ou) < TOL
+    assert cb.rel_l2(out, ref) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+def test_config5_reduced_width(bt):
+    """Same depth (8 hidden GELU layers + head) and method as configuration 5 at width 256."""
+    from tests import cuda_build as cb
+    inp = si.config5(width=256, depth=8, n_classes=1000, B=192)
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    ws = bt.Workspace([w, th])
+    bt.betty_lower_step(w, inp.lower_steps, ws)
+    oracle.lower_step(ow, inp.lower_steps)
+    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    out = _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_hypergrad_neumann(w, th, th, inp.K, inp.alpha, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK

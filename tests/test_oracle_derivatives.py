@@ -312,15 +312,42 @@ def test_three_level_classifier_cost_with_both_constraints():
     assert rel(oracle.mixed_vjp(P1, P2, q), mth.numpy()) < 1e-11
 
 
-def test_bf16_level_evaluates_cost_at_rounded_matrices():
+def test_bf16_level_quantises_matrices_and_hidden_activations():
+    """A mixed-precision level evaluates its cost with bf16 operands in every matrix product:
+    matrices and hidden activations rounded (torch's conversion is the reference), fp64
+    everywhere else; the full-precision level does not."""
     inp = _tiny_reweight("relu", seed=23)
     inp.w = inp.w + si.normal_f32(23, 400, inp.w.shape) * 1e-3        # not bf16-representable
     w16, th16 = reweight_levels(inp, bf16=True)
+    q = lambda t: t.to(torch.float32).to(torch.bfloat16).to(torch.float64)
     Ws, bs = olv.mlp_unpack(inp.widths, inp.w.astype(np.float64))
-    rounded = olv.mlp_pack([_t(np.asarray(W, np.float32)).to(torch.bfloat16).to(torch.float64)
-                            .numpy() for W in Ws], bs)
+    h = _t(inp.train.X)
+    for l, (W, b) in enumerate(zip(Ws, bs)):
+        a = h @ q(_t(W)).T + _t(b)
+        h = q(torch.relu(a)) if l < len(Ws) - 1 else a
+    ell = torch.nn.functional.cross_entropy(h, torch.from_numpy(inp.train.y.astype(np.int64)),
+                                            reduction="none")
+    ref = (_torch_weightnet(_t(inp.theta), ell) * ell).mean().item()
+    assert abs(olv.cost(w16) - ref) < 1e-13
+    assert abs(olv.cost(reweight_levels(inp, bf16=False)[0]) - ref) > 1e-9
+    # derivatives are straight-through: same formulas, evaluated on the quantised forward pass
     w64, th64 = reweight_levels(inp, bf16=False)
-    w64.params = rounded
-    assert olv.cost(w16) == olv.cost(w64)
-    np.testing.assert_array_equal(oracle.grad(w16, w16), oracle.grad(w64, w64))
-    assert olv.cost(w16) != olv.cost(reweight_levels(inp, bf16=False)[0])
+    assert rel(oracle.grad(w16, w16), oracle.grad(w64, w64)) < 5e-2
+
+
+def test_fd_on_a_bf16_level_keeps_quantisation_offsets_frozen():
+    """The finite difference on a mixed-precision level must see the perturbation, which is far
+    below bf16 resolution: with frozen rounding offsets it agrees with the full-precision
+    level's finite difference to within the quantisation error of the base point."""
+    inp = _tiny_reweight("gelu", seed=29, widths=(8, 12, 10, 5), B=40)
+    w16, th16 = reweight_levels(inp, bf16=True)
+    w64, th64 = reweight_levels(inp, bf16=False)
+    v = np.random.default_rng(3).standard_normal(inp.w.size)
+    f16 = oracle.brj(w16, th16, v, "fd", eps0=1e-3, alpha=1.0)
+    f64 = oracle.brj(w64, th64, v, "fd", eps0=1e-3, alpha=1.0)
+    assert rel(f16, f64) < 5e-2
+    # re-rounding the perturbed weights instead would wipe the perturbation out
+    eps = 1e-3 / np.linalg.norm(v)
+    naive = -(oracle.grad(w16, th16, {id(w16): w16.params + eps * v})
+              - oracle.grad(w16, th16, {id(w16): w16.params - eps * v})) / (2 * eps)
+    assert rel(naive, f64) > 10 * rel(f16, f64)
