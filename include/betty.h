@@ -203,6 +203,25 @@ betty_status betty_hvp_logreg_static(const float* X, int64_t n, int64_t d, const
                                      const float* lam, const float* u, float* Hu,
                                      int32_t* status_dev, void* stream);
 
+/* Building block of the MLP families' forward, backward and R-operator passes (the matrix products
+ * behind the Hessian-vector products of Sec. 3.2), exposed so that it can be checked on its own:
+ *   C[M,N] (fp32, leading dimension ldc) = sum_{i < n_pairs} alpha_i * op(A_i) op(B_i) + beta * C
+ * with bf16 operands and fp32 accumulation, n_pairs in {1, 2}.  Logical A is [M,K]: stored row-major
+ * [M,K] (a_transposed = 0) or [K,M] (a_transposed = 1); logical B is [K,N]: stored [K,N]
+ * (b_transposed = 0) or [N,K] (b_transposed = 1); lda/ldb are leading dimensions in elements.
+ * path: 0 = library's choice, 1 = CUDA-core kernel, 2 = tensor-core (tcgen05) kernel, which needs
+ * 16-byte aligned operands, lda/ldb multiples of 8 and alpha = +-1 (else BETTY_ERR_UNSUPPORTED).
+ * All pointers are device pointers; `pairs` is host memory. */
+typedef struct {
+  const void* A; int64_t lda; int32_t a_transposed;
+  const void* B; int64_t ldb; int32_t b_transposed;
+  int32_t K;
+  float alpha;
+} betty_gemm_operands;
+betty_status betty_gemm_bf16(int32_t M, int32_t N, int32_t n_pairs, const betty_gemm_operands* pairs,
+                             float* C, int64_t ldc, float beta, int32_t path, void* ws, size_t ws_bytes,
+                             void* stream);
+
 const char* betty_status_string(betty_status s);
 
 /* Number of CUDA kernels this library has launched in the calling process since it was loaded

@@ -46,6 +46,11 @@ _Level._fields_ = [
     ("constraints", C.POINTER(C.POINTER(_Level))),
 ]
 
+class _GemmOperands(C.Structure):
+    _fields_ = [("A", C.c_void_p), ("lda", C.c_int64), ("a_transposed", C.c_int32), ("B", C.c_void_p),
+                ("ldb", C.c_int64), ("b_transposed", C.c_int32), ("K", C.c_int32), ("alpha", C.c_float)]
+
+
 _lib = None
 
 
@@ -80,6 +85,7 @@ def lib():
                                VP, SZ, VP],
     }
     sig["betty_hvp_logreg_static"] = [VP, C.c_int64, C.c_int64, VP, VP, VP, VP, VP, VP]
+    sig["betty_gemm_bf16"] = [I32, I32, I32, C.POINTER(_GemmOperands), VP, C.c_int64, F, I32, VP, SZ, VP]
     for name, args in sig.items():
         fn = getattr(L, name)
         fn.argtypes, fn.restype = args, C.c_int
@@ -248,3 +254,13 @@ def betty_hvp_logreg_static(X: torch.Tensor, w: torch.Tensor, lam: torch.Tensor,
     n, d = X.shape
     _check(lib().betty_hvp_logreg_static(_ptr(X) if n else None, n, d, _ptr(w), _ptr(lam), _ptr(u), _ptr(Hu),
                                          _ptr(status_dev), _stream(stream)), "betty_hvp_logreg_static")
+
+
+def betty_gemm_bf16(M: int, N: int, pairs, Cout: torch.Tensor, ldc: int, beta: float, path: int, ws: Workspace,
+                    stream=None) -> None:
+    """pairs: sequence of (A, lda, a_transposed, B, ldb, b_transposed, K, alpha) with bf16 device tensors."""
+    arr = (_GemmOperands * len(pairs))()
+    for i, (A, lda, ta, B, ldb, tb, K, alpha) in enumerate(pairs):
+        arr[i] = _GemmOperands(_ptr(A), int(lda), int(bool(ta)), _ptr(B), int(ldb), int(bool(tb)), int(K), float(alpha))
+    _check(lib().betty_gemm_bf16(int(M), int(N), len(pairs), arr, _ptr(Cout), int(ldc), float(beta), int(path), ws.ptr,
+                                 ws.nbytes, _stream(stream)), "betty_gemm_bf16")

@@ -73,6 +73,32 @@ betty_status gemm_simt(Ctx& c, const GemmDesc& g) {
   return BETTY_OK;
 }
 
-betty_status gemm(Ctx& c, const GemmDesc& g) { return gemm_simt(c, g); }
+int g_gemm_path = 0;   // 0: tensor cores when the operands allow it; 1: CUDA cores always
+
+betty_status gemm(Ctx& c, const GemmDesc& g) {
+  if (g_gemm_path == 0 && gemm_tc_eligible(g)) return gemm_tc(c, g);
+  return gemm_simt(c, g);
+}
 
 }  // namespace betty
+
+using namespace betty;
+
+extern "C" betty_status betty_gemm_bf16(int32_t M, int32_t N, int32_t n_pairs, const betty_gemm_operands* pairs,
+                                        float* C, int64_t ldc, float beta, int32_t path, void* ws, size_t ws_bytes,
+                                        void* stream) {
+  if (M < 0 || N < 0 || n_pairs < 1 || n_pairs > 2 || !pairs || (!C && M > 0 && N > 0)) return BETTY_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < sizeof(StatusBlock) || (((uintptr_t)ws) & 255u)) return BETTY_ERR_WORKSPACE;
+  Ctx c(ws, ws_bytes, stream);
+  GemmDesc g;
+  g.M = M; g.N = N; g.npairs = n_pairs; g.C = C; g.ldc = ldc; g.beta = beta;
+  for (int i = 0; i < n_pairs; ++i) {
+    const betty_gemm_operands& o = pairs[i];
+    if (!o.A || !o.B || o.K < 0) return BETTY_ERR_INVALID_ARG;
+    g.p[i] = gemm_pair((const bf16*)o.A, o.lda, o.a_transposed != 0, (const bf16*)o.B, o.ldb, o.b_transposed != 0, o.K,
+                       o.alpha);
+  }
+  if (path == 1) return gemm_simt(c, g);
+  if (path == 2) return gemm_tc_eligible(g) ? gemm_tc(c, g) : BETTY_ERR_UNSUPPORTED;
+  return gemm(c, g);
+}

@@ -21,6 +21,10 @@ struct GemmDesc {
 };
 
 betty_status gemm(Ctx& c, const GemmDesc& g);
+// tcgen05 / tensor-memory path (gemm_tc.cu): needs 16-byte aligned operands, leading dimensions that
+// are multiples of 8 elements and alpha = +-1
+bool gemm_tc_eligible(const GemmDesc& g);
+betty_status gemm_tc(Ctx& c, const GemmDesc& g);
 // CUDA-core reference path (any shape, any stride); also the fallback for shapes the tensor-core
 // path does not take.
 betty_status gemm_simt(Ctx& c, const GemmDesc& g);

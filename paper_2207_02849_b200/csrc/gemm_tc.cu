@@ -1,0 +1,320 @@
+// Tensor-core matrix products for sm_100a: tcgen05.mma with the accumulator in tensor memory,
+// operands staged in shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), an mbarrier
+// pipeline between one producer thread, one MMA-issuing thread and four epilogue warps.
+//
+//   C[M,N] (fp32) = sum over 1..2 operand pairs of (+/-) op(A) op(B)  (+ beta * C)
+//
+// Each operand may be K-major (K contiguous in memory) or MN-major (M or N contiguous): forward
+// passes are K-major x K-major, backward-data passes K-major x N-major, weight-gradient passes
+// M-major x N-major.  Ragged M, N and K are handled by TMA's zero fill and predicated stores.
+// No cluster multicast is used anywhere.
+#include <cuda.h>
+#include "gemm.cuh"
+
+namespace betty {
+
+static constexpr int TC_BM = 128;
+static constexpr int TC_BN = 128;
+static constexpr int TC_BK = 64;            // 64 bf16 = one 128-byte swizzle row
+static constexpr int TC_STAGES = 6;
+static constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;
+static constexpr int TC_B_BYTES = TC_BN * TC_BK * 2;
+static constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
+static constexpr uint32_t TC_SPIN = 1u << 24;
+static constexpr int TC_SMEM = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct TcPair { int K; int a_mn; int b_mn; int neg; };
+struct TcArgs {
+  int M, N, npairs;
+  TcPair p[2];
+  float* C; int64_t ldc; float beta;
+  StatusBlock* sb;
+};
+
+__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void tc_mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void tc_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool tc_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(s_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Gives up early when another role has already raised the abort flag.
+__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < TC_SPIN; ++i) {
+    if (tc_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(s_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(s_u32(bar)) : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading and stride byte
+// offsets in 16-byte units, descriptor version 1 (bits 46-47), layout type 2 (bits 61-63).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 operands, majors, optional negation of A.
+__device__ __forceinline__ uint32_t instr_desc(int a_mn, int b_mn, int neg_a, int n, int m) {
+  uint32_t d = 0;
+  d |= 1u << 4;                 // D format: F32
+  d |= 1u << 7;                 // A format: BF16
+  d |= 1u << 10;                // B format: BF16
+  d |= (uint32_t)(neg_a & 1) << 13;
+  d |= (uint32_t)(a_mn & 1) << 15;
+  d |= (uint32_t)(b_mn & 1) << 16;
+  d |= (uint32_t)(n >> 3) << 17;
+  d |= (uint32_t)(m >> 4) << 24;
+  return d;
+}
+
+__global__ void __launch_bounds__(128, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+          const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1, TcArgs g) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = (uint64_t*)(smem + TC_STAGES * TC_STAGE_BYTES);
+  uint64_t* empty = full + TC_STAGES;
+  uint64_t* accum = empty + TC_STAGES;
+  uint32_t* tmem_slot = (uint32_t*)(accum + 1);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m0 = blockIdx.y * TC_BM, n0 = blockIdx.x * TC_BN;
+  int iters[2] = {0, 0};
+  for (int p = 0; p < g.npairs; ++p) iters[p] = (g.p[p].K + TC_BK - 1) / TC_BK;
+  const int T = iters[0] + iters[1];
+
+  if (tid == 0) {
+    for (int s = 0; s < TC_STAGES; ++s) { tc_mbar_init(&full[s], 1); tc_mbar_init(&empty[s], 1); }
+    tc_mbar_init(accum, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {   // one warp allocates the accumulator columns in tensor memory
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "r"(TC_BN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0 && lane == 0) {
+    // ---------------- producer: TMA loads into the stage ring
+    int armed = 0;
+    for (int it = 0; it < T; ++it) {
+      const int s = it % TC_STAGES;
+      if (it >= TC_STAGES && !tc_wait(&empty[s], (uint32_t)(((it / TC_STAGES) - 1) & 1), abort_flag)) break;
+      const int p = it < iters[0] ? 0 : 1;
+      const int k0 = (p == 0 ? it : it - iters[0]) * TC_BK;
+      const CUtensorMap* ta = p == 0 ? &tmA0 : &tmA1;
+      const CUtensorMap* tb = p == 0 ? &tmB0 : &tmB1;
+      unsigned char* sa = smem + s * TC_STAGE_BYTES;
+      unsigned char* sb = sa + TC_A_BYTES;
+      tc_expect_tx(&full[s], TC_STAGE_BYTES);
+      if (!g.p[p].a_mn) {
+        tma_load_2d(sa, ta, k0, m0, &full[s]);                                  // box 64(K) x 128(M)
+      } else {
+        for (int j = 0; j < TC_BM / 64; ++j) tma_load_2d(sa + j * 8192, ta, m0 + 64 * j, k0, &full[s]);   // box 64(M) x 64(K)
+      }
+      if (!g.p[p].b_mn) {
+        tma_load_2d(sb, tb, k0, n0, &full[s]);                                  // box 64(K) x 128(N)
+      } else {
+        for (int j = 0; j < TC_BN / 64; ++j) tma_load_2d(sb + j * 8192, tb, n0 + 64 * j, k0, &full[s]);   // box 64(N) x 64(K)
+      }
+      armed = it + 1;
+    }
+    if (*abort_flag) {
+      // let copies that were already issued land before the CTA's shared memory goes away
+      for (int it = (armed > TC_STAGES ? armed - TC_STAGES : 0); it < armed; ++it)
+        for (uint32_t i = 0; i < (1u << 16); ++i)
+          if (tc_try_wait(&full[it % TC_STAGES], (uint32_t)((it / TC_STAGES) & 1))) break;
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer
+    bool ok = true;
+    for (int it = 0; it < T && ok; ++it) {
+      const int s = it % TC_STAGES;
+      if (!tc_wait(&full[s], (uint32_t)((it / TC_STAGES) & 1), abort_flag)) { ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int p = it < iters[0] ? 0 : 1;
+      const uint32_t idesc = instr_desc(g.p[p].a_mn, g.p[p].b_mn, g.p[p].neg, TC_BN, TC_BM);
+      const uint32_t sa = s_u32(smem + s * TC_STAGE_BYTES), sb = sa + TC_A_BYTES;
+#pragma unroll
+      for (int kk = 0; kk < TC_BK / 16; ++kk) {
+        // K-major: 16 elements = 32 bytes further along the swizzled row; groups of 8 rows 1024 B apart.
+        // MN-major: 16 k-rows = 2048 bytes further; 64-element blocks along M/N 8192 B apart.
+        const uint64_t da = g.p[p].a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
+        const uint64_t db = g.p[p].b_mn ? smem_desc(sb + kk * 2048, 8192, 1024) : smem_desc(sb + kk * 32, 16, 1024);
+        const uint32_t acc = (it > 0 || kk > 0) ? 1u : 0u;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem_base), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+      }
+      // the stage may be refilled once these MMAs have read it
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(&empty[s])) : "memory");
+    }
+    if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(accum)) : "memory");
+  }
+  __syncwarp();
+
+  // ---------------- epilogue: all four warps, warp w owns accumulator lanes 32w..32w+31
+  bool have = T > 0 && tc_wait(accum, 0, abort_flag);
+  have = __all_sync(0xffffffffu, have);
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  if (have) {
+    const int m = m0 + warp * 32 + lane;
+#pragma unroll 1
+    for (int c = 0; c < TC_BN / 32; ++c) {
+      uint32_t r[32];
+      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32);
+      asm volatile(
+          "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+          "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+          "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+          : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+            "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+            "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+            "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+          : "r"(taddr) : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (m < g.M) {
+        float* crow = g.C + (int64_t)m * g.ldc;
+        const int nb = n0 + c * 32;
+        const bool vec = ((g.ldc & 3) == 0) && ((((uintptr_t)g.C) & 15) == 0) && (nb + 32 <= g.N);
+        if (vec) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                   __uint_as_float(r[j + 3]));
+            float4* dst = (float4*)(crow + nb + j);
+            if (g.beta != 0.f) { float4 o = *dst; v.x += g.beta * o.x; v.y += g.beta * o.y; v.z += g.beta * o.z; v.w += g.beta * o.w; }
+            *dst = v;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int n = nb + j;
+            if (n < g.N) {
+              float v = __uint_as_float(r[j]);
+              if (g.beta != 0.f) v += g.beta * crow[n];
+              crow[n] = v;
+            }
+          }
+        }
+      }
+    }
+  } else if (T == 0) {
+    // no products: C = beta * C
+    const int m = m0 + warp * 32 + lane;
+    if (m < g.M)
+      for (int n = n0; n < n0 + TC_BN && n < g.N; ++n) {
+        float* cp = g.C + (int64_t)m * g.ldc + n;
+        *cp = g.beta != 0.f ? g.beta * *cp : 0.f;
+      }
+  }
+  if (*abort_flag && tid == 0) record_status(g.sb, BETTY_ERR_TIMEOUT);
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_BN) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+    else
+      (void)cudaGetLastError();
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor map over a row-major matrix [outer, inner] with leading dimension ld (elements)
+static bool make_map(CUtensorMap* tm, const bf16* base, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+                     int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(bf16)};
+  cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool gemm_tc_eligible(const GemmDesc& g) {
+  if (g.M <= 0 || g.N <= 0 || g.npairs < 1 || g.npairs > 2) return false;
+  for (int i = 0; i < g.npairs; ++i) {
+    const GemmPair& p = g.p[i];
+    if (p.K <= 0) return false;
+    if (p.alpha != 1.f && p.alpha != -1.f) return false;
+    if ((((uintptr_t)p.A) & 15) || (((uintptr_t)p.B) & 15)) return false;
+    if ((p.lda & 7) || (p.ldb & 7)) return false;
+  }
+  return encode_fn() != nullptr;
+}
+
+betty_status gemm_tc(Ctx& c, const GemmDesc& g) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM) != cudaSuccess) return BETTY_ERR_CUDA;
+    attr_set = true;
+  }
+  CUtensorMap tm[4];
+  TcArgs a;
+  a.M = g.M; a.N = g.N; a.npairs = g.npairs; a.C = g.C; a.ldc = g.ldc; a.beta = g.beta; a.sb = c.arena.status();
+  for (int i = 0; i < 2; ++i) {
+    const GemmPair& p = g.p[i < g.npairs ? i : 0];
+    a.p[i].K = i < g.npairs ? p.K : 0;
+    a.p[i].a_mn = p.ta ? 1 : 0;
+    a.p[i].b_mn = p.tb ? 0 : 1;
+    a.p[i].neg = p.alpha < 0.f ? 1 : 0;
+    bool ok;
+    // A: K-major = stored [M,K]; M-major = stored [K,M]
+    ok = p.ta ? make_map(&tm[2 * i], p.A, g.M, p.K, p.lda, 64, 64) : make_map(&tm[2 * i], p.A, p.K, g.M, p.lda, TC_BK, TC_BM);
+    if (!ok) return BETTY_ERR_CUDA;
+    // B: K-major = stored [N,K]; N-major = stored [K,N]
+    ok = p.tb ? make_map(&tm[2 * i + 1], p.B, p.K, g.N, p.ldb, TC_BK, TC_BN) : make_map(&tm[2 * i + 1], p.B, g.N, p.K, p.ldb, 64, 64);
+    if (!ok) return BETTY_ERR_CUDA;
+  }
+  dim3 grid((unsigned)((g.N + TC_BN - 1) / TC_BN), (unsigned)((g.M + TC_BM - 1) / TC_BM));
+  k_gemm_tc<<<grid, 128, TC_SMEM, c.stream>>>(tm[0], tm[1], tm[2], tm[3], a);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
+}  // namespace betty
