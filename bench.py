@@ -199,10 +199,171 @@ class LogregWorkload:
         return dt / frac, f"first {n_s} of {self.n} train rows and {nv_s} of {self.nv} validation rows, full step, time scaled by {1/frac:.0f}x"
 
 
+class ReweightWorkload:
+    """Configs 3 and 5: data reweighting (App. A listing): lower MLP classifier, upper 1-100-1 weight net."""
+
+    def __init__(self, cfg: int, method: str):
+        import synth_inputs as si
+        self.cfg = cfg
+        self.inp = si.config3() if cfg == 3 else si.config5()
+        self.method = method or ("fd" if cfg == 3 else "neumann")
+        w = self.inp.widths
+        self.B = self.inp.train.X.shape[0]
+        self.name = (f"config{cfg}: data reweighting, MLP {'x'.join(map(str, w)) if len(w) < 5 else f'{w[0]}->{len(w)-2}x{w[1]}->{w[-1]}'} "
+                     f"{self.inp.activation} bf16/fp32-acc, batch {self.B}, {self.inp.lower_steps} lower SGD step(s), "
+                     f"{self.method}" + (f" K={self.inp.K}" if self.method != "fd" else " eps0=0.01"))
+        self.dtype = "bf16"
+
+    def setup_device(self):
+        import torch
+        import paper_2207_02849_b200 as bt
+        from tests import cuda_build as cb
+        self.bt, self.torch = bt, torch
+        self.w, self.th = cb.reweight_levels(self.inp)
+        self.w0 = self.w.params.clone()
+        self.out = torch.empty(self.th.params.numel(), dtype=torch.float32, device="cuda")
+        self.ws = bt.Workspace([self.w, self.th])
+
+    def step(self):
+        bt = self.bt
+        self.w.params.copy_(self.w0)
+        bt.betty_lower_step(self.w, self.inp.lower_steps, self.ws)
+        if self.method == "fd":
+            bt.betty_hypergrad_fd(self.w, self.th, self.th, self.inp.eps0, self.inp.fd_alpha, self.out, self.ws)
+        elif self.method == "neumann":
+            bt.betty_hypergrad_neumann(self.w, self.th, self.th, self.inp.K, self.inp.alpha, self.out, self.ws)
+        else:
+            bt.betty_hypergrad_cg(self.w, self.th, self.th, self.inp.K, 0.0, self.out, self.ws)
+
+    def setup_host(self):
+        torch = self.torch
+        pin = lambda t: t.detach().cpu().pin_memory()
+        self.d_in = [self.w.X, self.w.y, self.th.X, self.th.y, self.th.params, self.w0]
+        self.h_in = [pin(t) for t in self.d_in]
+        self.h_out = torch.empty(self.out.numel(), dtype=torch.float32).pin_memory()
+        self.h2d = sum(t.numel() * t.element_size() for t in self.h_in)
+        self.d2h = self.h_out.numel() * 4
+
+    def step_e2e(self):
+        for h, d in zip(self.h_in, self.d_in):
+            d.copy_(h, non_blocking=True)
+        self.step()
+        self.h_out.copy_(self.out, non_blocking=True)
+
+    def roofline_probe(self, reps: int):
+        """The dominant kernel is the tensor-core GEMM; its most frequent shape in this workload
+        (batch x width x width, forward layout) is timed alone through the C ABI."""
+        torch, bt = self.torch, self.bt
+        w = self.inp.widths
+        M, N, K = self.B, w[1], (w[1] if len(w) > 3 else w[0])
+        A = torch.randn(M, K, device="cuda").to(torch.bfloat16)
+        Bm = torch.randn(N, K, device="cuda").to(torch.bfloat16)
+        Cm = torch.empty(M, N, dtype=torch.float32, device="cuda")
+        pairs = [(A, K, 0, Bm, K, 1, K, 1.0)]
+        for _ in range(3):
+            bt.betty_gemm_bf16(M, N, pairs, Cm, N, 0.0, 2, self.ws)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in evs:
+            a.record()
+            bt.betty_gemm_bf16(M, N, pairs, Cm, N, 0.0, 2, self.ws)
+            b.record()
+        torch.cuda.synchronize()
+        ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+        return {"kernel": f"k_gemm_tc {M}x{N}x{K}", "ms": ms, "flops": 2.0 * M * N * K, "bound": "tensor"}
+
+    def oracle_sample(self, budget_rows: int):
+        import copy
+        import oracle
+        from tests import oracle_build as ob
+        frac = 1.0 if self.cfg == 3 else 1.0 / 8
+        nb = max(1, int(self.B * frac))
+        inp = copy.copy(self.inp)
+        cut = lambda b: type(b)(X=b.X[:nb], y=b.y[:nb], y_clean=b.y_clean[:nb], clean=b.clean[:nb])
+        inp.train, inp.val = cut(self.inp.train), cut(self.inp.val)
+        ow, oth = ob.reweight_levels(inp)
+        t0 = time.perf_counter()
+        oracle.lower_step(ow, inp.lower_steps)
+        if self.method == "fd":
+            oracle.hypergrad_fd(ow, oth, oth, inp.eps0, inp.fd_alpha)
+        elif self.method == "neumann":
+            oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)
+        else:
+            oracle.hypergrad_cg(ow, oth, oth, inp.K, 0.0)
+        dt = time.perf_counter() - t0
+        return dt / frac, f"first {nb} of {self.B} rows of the train and validation batches, full step, time scaled by {1/frac:.0f}x"
+
+
+class ThreeLevelWorkload:
+    """Config 4: three-level chain; the timed unit is the level-3 hypergradient after one lower step."""
+
+    def __init__(self, method: str):
+        import synth_inputs as si
+        self.inp = si.config4()
+        self.method = "neumann"
+        self.B = self.inp.D1.X.shape[0]
+        self.name = (f"config4: three-level chain, MLP {'x'.join(map(str, self.inp.widths))} relu bf16/fp32-acc, batch "
+                     f"{self.B}, weight net 1-100-1, per-layer log weight decay, two Neumann K={self.inp.K} edges")
+        self.dtype = "bf16"
+
+    def setup_device(self):
+        import torch
+        import paper_2207_02849_b200 as bt
+        from tests import cuda_build as cb
+        self.bt, self.torch = bt, torch
+        self.P = cb.three_levels(self.inp)
+        self.w0 = self.P[0].params.clone()
+        self.u = torch.empty(self.inp.w.size, dtype=torch.float32, device="cuda")
+        self.vt = torch.empty(self.inp.theta.size, dtype=torch.float32, device="cuda")
+        self.out = torch.empty(self.inp.lam.size, dtype=torch.float32, device="cuda")
+        self.ws = bt.Workspace(list(self.P))
+        self.cfgm = bt.MethodCfg(bt.BETTY_NEUMANN, K=self.inp.K, alpha=self.inp.alpha)
+
+    def step(self):
+        bt, (P1, P2, P3) = self.bt, self.P
+        P1.params.copy_(self.w0)
+        bt.betty_lower_step(P1, 1, self.ws)
+        bt.betty_grad(P3, P1, self.u, self.ws)
+        bt.betty_grad(P3, P2, self.vt, self.ws)
+        bt.betty_chain_levels(list(self.P), [0, 1], [self.cfgm], self.vt, self.u, True, self.ws)
+        bt.betty_chain_levels(list(self.P), [2, 0], [self.cfgm], self.u, self.out, False, self.ws)
+
+    def setup_host(self):
+        torch = self.torch
+        P1, P2, P3 = self.P
+        pin = lambda t: t.detach().cpu().pin_memory()
+        self.d_in = [P1.X, P1.y, P2.X, P2.y, P2.aux, P3.X, P3.y, P3.aux, P2.params, P3.params, self.w0]
+        self.h_in = [pin(t) for t in self.d_in]
+        self.h_out = torch.empty(self.out.numel(), dtype=torch.float32).pin_memory()
+        self.h2d = sum(t.numel() * t.element_size() for t in self.h_in)
+        self.d2h = self.h_out.numel() * 4
+
+    step_e2e = ReweightWorkload.step_e2e
+
+    def roofline_probe(self, reps: int):
+        self.inp.widths  # forward-layout GEMM batch x 512 x 784
+        rw = ReweightWorkload.roofline_probe
+        return rw(self, reps)
+
+    def oracle_sample(self, budget_rows: int):
+        import oracle
+        from tests import oracle_build as ob
+        O1, O2, O3 = ob.three_levels(self.inp)
+        nm = dict(method="neumann", K=self.inp.K, alpha=self.inp.alpha)
+        t0 = time.perf_counter()
+        oracle.lower_step(O1, 1)
+        u = oracle.grad(O3, O1) + oracle.chain_levels([O1, O2, O3], [0, 1], [nm], v_in=oracle.grad(O3, O2))
+        oracle.chain_levels([O1, O2, O3], [2, 0], [nm], v_in=u)
+        return time.perf_counter() - t0, "the full workload"
+
+
 def make_workload(cfg: int, method: str, scale: float):
     if cfg in (1, 2):
         return LogregWorkload(cfg, method, scale)
-    raise SystemExit(f"config {cfg} is not wired into the benchmark yet")
+    if cfg in (3, 5):
+        return ReweightWorkload(cfg, method)
+    if cfg == 4:
+        return ThreeLevelWorkload(method)
+    raise SystemExit(f"unknown config {cfg}")
 
 
 def blas_threads() -> int:
@@ -288,25 +449,44 @@ def main():
         if sampler:
             sampler.mark_begin()
         l0 = bt.betty_kernel_launches()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
-            fn()
-        e1.record()
+        if flush is None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                fn()
+            e1.record()
+            pairs = [(e0, e1)]
+        else:
+            pairs = []
+            for _ in range(steps):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn()
+                e1.record()
+                pairs.append((e0, e1))
         barrier()
         if sampler:
             sampler.mark_end()
         launches = bt.betty_kernel_launches() - l0
         clocks = sampler.stop() if sampler else None
-        ms = e0.elapsed_time(e1)
+        ms = sum(a.elapsed_time(b) for a, b in pairs)
         if world > 1:
             t = torch.tensor([ms], dtype=torch.float64, device="cuda")
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             ms = float(t.item())
         return ms, launches, clocks
 
+    # configs whose inputs fit in L2 get a flush (a 512 MiB write) before every step
+    flush = None
+    if args.config != 2:
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    l2_note = ("inputs (train matrix) larger than L2; no flush between steps" if flush is None
+               else "L2 flushed (512 MiB write) before every step; each step timed by its own event pair, flush excluded")
+    step_dev, step_host = wl.step, wl.step_e2e
+
     sampler = ClockSampler(local) if rank == 0 else None
-    ms, launches, clocks = timed(wl.step, args.steps, warm, sampler)
+    ms, launches, clocks = timed(step_dev, args.steps, warm, sampler)
     st, _ = bt.betty_poll_status(wl.ws)
     ms_per_step = ms / args.steps
     value = world * 1e3 / ms_per_step
@@ -314,7 +494,7 @@ def main():
     e2e = None
     if not args.no_e2e:
         wl.setup_host()
-        ms_e, _, _ = timed(wl.step_e2e, max(1, min(args.steps, 5)), 3)
+        ms_e, _, _ = timed(step_host, max(1, min(args.steps, 5)), 3)
         e_steps = max(1, min(args.steps, 5))
         e2e = {"value": world * 1e3 / (ms_e / e_steps), "unit": UNIT, "h2d_bytes_per_step": int(wl.h2d),
                "d2h_bytes_per_step": int(wl.d2h)}
@@ -336,7 +516,8 @@ def main():
             traffic = tj["dram_bytes_per_unit"] * (probe["bytes"] / tj["unit_bytes"])
     roofline = {"bound": probe["bound"], "kernel": probe["kernel"], "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": traffic, "peak_source": f"{peaks['source']} (burst; kernel timed alone)",
-                "kernel_ms": probe["ms"], "algorithmic_bytes_per_launch": probe.get("bytes")}
+                "kernel_ms": probe["ms"], "algorithmic_bytes_per_launch": probe.get("bytes"),
+                "algorithmic_flops_per_launch": probe.get("flops")}
 
     if rank != 0:
         if world > 1:
@@ -351,7 +532,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": wl.dtype, "data": "synthetic",
-            "config": {"workload": wl.name, "l2": "inputs (train matrix) larger than L2; no flush between steps",
+            "config": {"workload": wl.name, "l2": l2_note,
                        "replicas": world, "device_status": bt.betty_status_string(st)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
