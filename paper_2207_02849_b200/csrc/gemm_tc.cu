@@ -14,14 +14,17 @@
 namespace betty {
 
 static constexpr int TC_BM = 128;
-static constexpr int TC_BN = 128;
 static constexpr int TC_BK = 64;            // 64 bf16 = one 128-byte swizzle row
-static constexpr int TC_STAGES = 6;
 static constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;
-static constexpr int TC_B_BYTES = TC_BN * TC_BK * 2;
-static constexpr int TC_STAGE_BYTES = TC_A_BYTES + TC_B_BYTES;
 static constexpr uint32_t TC_SPIN = 1u << 24;
-static constexpr int TC_SMEM = TC_STAGES * TC_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+static constexpr int TC_THREADS = 192;      // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+template <int BN> struct TcCfg {
+  static constexpr int B_BYTES = BN * TC_BK * 2;
+  static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
+  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int TMEM_COLS = 2 * BN;  // two accumulators: the epilogue of one tile overlaps the next tile's MMAs
+};
 
 struct TcPair { int K; int a_mn; int b_mn; int neg; };
 struct TcArgs {
@@ -86,31 +89,41 @@ __device__ __forceinline__ uint32_t instr_desc(int a_mn, int b_mn, int neg_a, in
   return d;
 }
 
-__global__ void __launch_bounds__(128, 1)
+__device__ __forceinline__ void tc_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(bar)) : "memory");
+}
+
+// Persistent kernel: CTA b works on output tiles b, b + gridDim.x, ...
+template <int BN>
+__global__ void __launch_bounds__(TC_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
           const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1, TcArgs g) {
+  using Cfg = TcCfg<BN>;
+  constexpr int S = Cfg::STAGES;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint64_t* full = (uint64_t*)(smem + TC_STAGES * TC_STAGE_BYTES);
-  uint64_t* empty = full + TC_STAGES;
-  uint64_t* accum = empty + TC_STAGES;
-  uint32_t* tmem_slot = (uint32_t*)(accum + 1);
+  uint64_t* full = (uint64_t*)(smem + S * Cfg::STAGE_BYTES);
+  uint64_t* empty = full + S;
+  uint64_t* acc_full = empty + S;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int m0 = blockIdx.y * TC_BM, n0 = blockIdx.x * TC_BN;
   int iters[2] = {0, 0};
   for (int p = 0; p < g.npairs; ++p) iters[p] = (g.p[p].K + TC_BK - 1) / TC_BK;
   const int T = iters[0] + iters[1];
+  const int tiles_n = (g.N + BN - 1) / BN;
+  const int tiles = tiles_n * ((g.M + TC_BM - 1) / TC_BM);
 
   if (tid == 0) {
-    for (int s = 0; s < TC_STAGES; ++s) { tc_mbar_init(&full[s], 1); tc_mbar_init(&empty[s], 1); }
-    tc_mbar_init(accum, 1);
+    for (int s = 0; s < S; ++s) { tc_mbar_init(&full[s], 1); tc_mbar_init(&empty[s], 1); }
+    for (int s = 0; s < 2; ++s) { tc_mbar_init(&acc_full[s], 1); tc_mbar_init(&acc_empty[s], 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {   // one warp allocates the accumulator columns in tensor memory
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "r"(TC_BN) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "r"(Cfg::TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -118,126 +131,147 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0 && lane == 0) {
+  if (warp == 0 && lane == 0 && T > 0) {
     // ---------------- producer: TMA loads into the stage ring
-    int armed = 0;
-    for (int it = 0; it < T; ++it) {
-      const int s = it % TC_STAGES;
-      if (it >= TC_STAGES && !tc_wait(&empty[s], (uint32_t)(((it / TC_STAGES) - 1) & 1), abort_flag)) break;
-      const int p = it < iters[0] ? 0 : 1;
-      const int k0 = (p == 0 ? it : it - iters[0]) * TC_BK;
-      const CUtensorMap* ta = p == 0 ? &tmA0 : &tmA1;
-      const CUtensorMap* tb = p == 0 ? &tmB0 : &tmB1;
-      unsigned char* sa = smem + s * TC_STAGE_BYTES;
-      unsigned char* sb = sa + TC_A_BYTES;
-      tc_expect_tx(&full[s], TC_STAGE_BYTES);
-      if (!g.p[p].a_mn) {
-        tma_load_2d(sa, ta, k0, m0, &full[s]);                                  // box 64(K) x 128(M)
-      } else {
-        for (int j = 0; j < TC_BM / 64; ++j) tma_load_2d(sa + j * 8192, ta, m0 + 64 * j, k0, &full[s]);   // box 64(M) x 64(K)
+    long long git = 0, armed = 0;
+    for (int t = blockIdx.x; t < tiles && !*abort_flag; t += gridDim.x) {
+      const int m0 = (t / tiles_n) * TC_BM, n0 = (t % tiles_n) * BN;
+      for (int it = 0; it < T; ++it, ++git) {
+        const int s = (int)(git % S);
+        if (git >= S && !tc_wait(&empty[s], (uint32_t)(((git / S) - 1) & 1), abort_flag)) break;
+        const int p = it < iters[0] ? 0 : 1;
+        const int k0 = (p == 0 ? it : it - iters[0]) * TC_BK;
+        const CUtensorMap* ta = p == 0 ? &tmA0 : &tmA1;
+        const CUtensorMap* tb = p == 0 ? &tmB0 : &tmB1;
+        unsigned char* sa = smem + s * Cfg::STAGE_BYTES;
+        unsigned char* sb = sa + TC_A_BYTES;
+        tc_expect_tx(&full[s], Cfg::STAGE_BYTES);
+        if (!g.p[p].a_mn) {
+          tma_load_2d(sa, ta, k0, m0, &full[s]);                                  // box 64(K) x 128(M)
+        } else {
+          for (int j = 0; j < TC_BM / 64; ++j) tma_load_2d(sa + j * 8192, ta, m0 + 64 * j, k0, &full[s]);   // box 64(M) x 64(K)
+        }
+        if (!g.p[p].b_mn) {
+          tma_load_2d(sb, tb, k0, n0, &full[s]);                                  // box 64(K) x BN(N)
+        } else {
+          for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, tb, n0 + 64 * j, k0, &full[s]);      // box 64(N) x 64(K)
+        }
+        armed = git + 1;
       }
-      if (!g.p[p].b_mn) {
-        tma_load_2d(sb, tb, k0, n0, &full[s]);                                  // box 64(K) x 128(N)
-      } else {
-        for (int j = 0; j < TC_BN / 64; ++j) tma_load_2d(sb + j * 8192, tb, n0 + 64 * j, k0, &full[s]);   // box 64(N) x 64(K)
-      }
-      armed = it + 1;
     }
     if (*abort_flag) {
       // let copies that were already issued land before the CTA's shared memory goes away
-      for (int it = (armed > TC_STAGES ? armed - TC_STAGES : 0); it < armed; ++it)
+      for (long long i2 = (armed > S ? armed - S : 0); i2 < armed; ++i2)
         for (uint32_t i = 0; i < (1u << 16); ++i)
-          if (tc_try_wait(&full[it % TC_STAGES], (uint32_t)((it / TC_STAGES) & 1))) break;
+          if (tc_try_wait(&full[i2 % S], (uint32_t)((i2 / S) & 1))) break;
     }
-  } else if (warp == 1 && lane == 0) {
+  } else if (warp == 1 && lane == 0 && T > 0) {
     // ---------------- MMA issuer
+    long long git = 0;
+    int j = 0;
     bool ok = true;
-    for (int it = 0; it < T && ok; ++it) {
-      const int s = it % TC_STAGES;
-      if (!tc_wait(&full[s], (uint32_t)((it / TC_STAGES) & 1), abort_flag)) { ok = false; break; }
+    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++j) {
+      const int as = j & 1;
+      if (j >= 2 && !tc_wait(&acc_empty[as], (uint32_t)(((j >> 1) - 1) & 1), abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int p = it < iters[0] ? 0 : 1;
-      const uint32_t idesc = instr_desc(g.p[p].a_mn, g.p[p].b_mn, g.p[p].neg, TC_BN, TC_BM);
-      const uint32_t sa = s_u32(smem + s * TC_STAGE_BYTES), sb = sa + TC_A_BYTES;
+      const uint32_t tmem_acc = tmem_base + (uint32_t)(as * BN);
+      for (int it = 0; it < T; ++it, ++git) {
+        const int s = (int)(git % S);
+        if (!tc_wait(&full[s], (uint32_t)((git / S) & 1), abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int p = it < iters[0] ? 0 : 1;
+        const uint32_t idesc = instr_desc(g.p[p].a_mn, g.p[p].b_mn, g.p[p].neg, BN, TC_BM);
+        const uint32_t sa = s_u32(smem + s * Cfg::STAGE_BYTES), sb = sa + TC_A_BYTES;
 #pragma unroll
-      for (int kk = 0; kk < TC_BK / 16; ++kk) {
-        // K-major: 16 elements = 32 bytes further along the swizzled row; groups of 8 rows 1024 B apart.
-        // MN-major: 16 k-rows = 2048 bytes further; 64-element blocks along M/N 8192 B apart.
-        const uint64_t da = g.p[p].a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
-        const uint64_t db = g.p[p].b_mn ? smem_desc(sb + kk * 2048, 8192, 1024) : smem_desc(sb + kk * 32, 16, 1024);
-        const uint32_t acc = (it > 0 || kk > 0) ? 1u : 0u;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(tmem_base), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+        for (int kk = 0; kk < TC_BK / 16; ++kk) {
+          // K-major: 16 elements = 32 bytes further along the swizzled row; groups of 8 rows 1024 B apart.
+          // MN-major: 16 k-rows = 2048 bytes further; 64-element blocks along M/N 8192 B apart.
+          const uint64_t da = g.p[p].a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
+          const uint64_t db = g.p[p].b_mn ? smem_desc(sb + kk * 2048, 8192, 1024) : smem_desc(sb + kk * 32, 16, 1024);
+          const uint32_t acc = (it > 0 || kk > 0) ? 1u : 0u;
+          asm volatile(
+              "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+              "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+              ::"r"(tmem_acc), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+        }
+        // the stage may be refilled once these MMAs have read it
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(&empty[s])) : "memory");
       }
-      // the stage may be refilled once these MMAs have read it
-      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(&empty[s])) : "memory");
+      if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(&acc_full[as])) : "memory");
     }
-    if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(accum)) : "memory");
-  }
-  __syncwarp();
-
-  // ---------------- epilogue: all four warps, warp w owns accumulator lanes 32w..32w+31
-  bool have = T > 0 && tc_wait(accum, 0, abort_flag);
-  have = __all_sync(0xffffffffu, have);
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  if (have) {
-    const int m = m0 + warp * 32 + lane;
+  } else if (warp >= 2) {
+    // ---------------- epilogue: warp w may touch accumulator lanes 32*(w%4) .. 32*(w%4)+31
+    const int q = warp & 3;
+    int j = 0;
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++j) {
+      const int m0 = (t / tiles_n) * TC_BM, n0 = (t % tiles_n) * BN;
+      const int as = j & 1;
+      const int m = m0 + q * 32 + lane;
+      if (T > 0) {
+        bool have = tc_wait(&acc_full[as], (uint32_t)((j >> 1) & 1), abort_flag);
+        have = __all_sync(0xffffffffu, have);
+        if (!have) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-    for (int c = 0; c < TC_BN / 32; ++c) {
-      uint32_t r[32];
-      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32);
-      asm volatile(
-          "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-          "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-          "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-          : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-            "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-            "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-            "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-          : "r"(taddr) : "memory");
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      if (m < g.M) {
-        float* crow = g.C + (int64_t)m * g.ldc;
-        const int nb = n0 + c * 32;
-        const bool vec = ((g.ldc & 3) == 0) && ((((uintptr_t)g.C) & 15) == 0) && (nb + 32 <= g.N);
-        if (vec) {
+        for (int c = 0; c < BN / 32; ++c) {
+          if (n0 + c * 32 >= g.N) break;            // uniform: nothing to store from these columns
+          uint32_t r[32];
+          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32);
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+              "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+              "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+              : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+              : "r"(taddr) : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          if (m < g.M) {
+            float* crow = g.C + (int64_t)m * g.ldc;
+            const int nb = n0 + c * 32;
+            const bool vec = ((g.ldc & 3) == 0) && ((((uintptr_t)g.C) & 15) == 0) && (nb + 32 <= g.N);
+            if (vec) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                                   __uint_as_float(r[j + 3]));
-            float4* dst = (float4*)(crow + nb + j);
-            if (g.beta != 0.f) { float4 o = *dst; v.x += g.beta * o.x; v.y += g.beta * o.y; v.z += g.beta * o.z; v.w += g.beta * o.w; }
-            *dst = v;
-          }
-        } else {
+              for (int jj = 0; jj < 32; jj += 4) {
+                float4 v = make_float4(__uint_as_float(r[jj]), __uint_as_float(r[jj + 1]), __uint_as_float(r[jj + 2]),
+                                       __uint_as_float(r[jj + 3]));
+                float4* dst = (float4*)(crow + nb + jj);
+                if (g.beta != 0.f) { float4 o = *dst; v.x += g.beta * o.x; v.y += g.beta * o.y; v.z += g.beta * o.z; v.w += g.beta * o.w; }
+                *dst = v;
+              }
+            } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int n = nb + j;
-            if (n < g.N) {
-              float v = __uint_as_float(r[j]);
-              if (g.beta != 0.f) v += g.beta * crow[n];
-              crow[n] = v;
+              for (int jj = 0; jj < 32; ++jj) {
+                const int n = nb + jj;
+                if (n < g.N) {
+                  float v = __uint_as_float(r[jj]);
+                  if (g.beta != 0.f) v += g.beta * crow[n];
+                  crow[n] = v;
+                }
+              }
             }
           }
         }
+        // this warp has drained its quarter of the accumulator: the MMA warp may reuse it
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) tc_arrive(&acc_empty[as]);
+      } else if (m < g.M) {
+        // no products: C = beta * C
+        for (int n = n0; n < n0 + BN && n < g.N; ++n) {
+          float* cp = g.C + (int64_t)m * g.ldc + n;
+          *cp = g.beta != 0.f ? g.beta * *cp : 0.f;
+        }
       }
     }
-  } else if (T == 0) {
-    // no products: C = beta * C
-    const int m = m0 + warp * 32 + lane;
-    if (m < g.M)
-      for (int n = n0; n < n0 + TC_BN && n < g.N; ++n) {
-        float* cp = g.C + (int64_t)m * g.ldc + n;
-        *cp = g.beta != 0.f ? g.beta * *cp : 0.f;
-      }
   }
-  if (*abort_flag && tid == 0) record_status(g.sb, BETTY_ERR_TIMEOUT);
+  __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  if (*abort_flag && tid == 0) record_status(g.sb, BETTY_ERR_TIMEOUT);
   if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg::TMEM_COLS) : "memory");
   }
 }
 
@@ -288,10 +322,12 @@ bool gemm_tc_eligible(const GemmDesc& g) {
   return encode_fn() != nullptr;
 }
 
-betty_status gemm_tc(Ctx& c, const GemmDesc& g) {
+template <int BN>
+static betty_status launch_tc(Ctx& c, const GemmDesc& g) {
+  using Cfg = TcCfg<BN>;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM) != cudaSuccess) return BETTY_ERR_CUDA;
+    if (cudaFuncSetAttribute(k_gemm_tc<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM) != cudaSuccess) return BETTY_ERR_CUDA;
     attr_set = true;
   }
   CUtensorMap tm[4];
@@ -308,13 +344,21 @@ betty_status gemm_tc(Ctx& c, const GemmDesc& g) {
     ok = p.ta ? make_map(&tm[2 * i], p.A, g.M, p.K, p.lda, 64, 64) : make_map(&tm[2 * i], p.A, p.K, g.M, p.lda, TC_BK, TC_BM);
     if (!ok) return BETTY_ERR_CUDA;
     // B: K-major = stored [N,K]; N-major = stored [K,N]
-    ok = p.tb ? make_map(&tm[2 * i + 1], p.B, p.K, g.N, p.ldb, TC_BK, TC_BN) : make_map(&tm[2 * i + 1], p.B, g.N, p.K, p.ldb, 64, 64);
+    ok = p.tb ? make_map(&tm[2 * i + 1], p.B, p.K, g.N, p.ldb, TC_BK, BN) : make_map(&tm[2 * i + 1], p.B, g.N, p.K, p.ldb, 64, 64);
     if (!ok) return BETTY_ERR_CUDA;
   }
-  dim3 grid((unsigned)((g.N + TC_BN - 1) / TC_BN), (unsigned)((g.M + TC_BM - 1) / TC_BM));
-  k_gemm_tc<<<grid, 128, TC_SMEM, c.stream>>>(tm[0], tm[1], tm[2], tm[3], a);
+  const int tiles = ((g.N + BN - 1) / BN) * ((g.M + TC_BM - 1) / TC_BM);
+  const int grid = tiles < c.sm_count ? tiles : c.sm_count;
+  k_gemm_tc<BN><<<grid, TC_THREADS, Cfg::SMEM, c.stream>>>(tm[0], tm[1], tm[2], tm[3], a);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
+}
+
+betty_status gemm_tc(Ctx& c, const GemmDesc& g) {
+  // wide tiles unless the problem is narrow or would leave most SMs without a tile
+  const int tiles256 = ((g.N + 255) / 256) * ((g.M + TC_BM - 1) / TC_BM);
+  if (g.N > 128 && tiles256 >= 96) return launch_tc<256>(c, g);
+  return launch_tc<128>(c, g);
 }
 
 }  // namespace betty
