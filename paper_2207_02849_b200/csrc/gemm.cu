@@ -59,8 +59,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmDesc g) {
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tx * 4 + j;
       if (n >= g.N) continue;
-      float* cp = g.C + (int64_t)m * g.ldc + n;
-      *cp = acc[i][j] + (g.beta != 0.f ? g.beta * *cp : 0.f);
+      gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.N, m, n, acc[i][j]);
     }
   }
 }
@@ -90,7 +89,7 @@ extern "C" betty_status betty_gemm_bf16(int32_t M, int32_t N, int32_t n_pairs, c
   if (M < 0 || N < 0 || n_pairs < 1 || n_pairs > 2 || !pairs || (!C && M > 0 && N > 0)) return BETTY_ERR_INVALID_ARG;
   if (!ws || ws_bytes < sizeof(StatusBlock) || (((uintptr_t)ws) & 255u)) return BETTY_ERR_WORKSPACE;
   Ctx c(ws, ws_bytes, stream);
-  GemmDesc g;
+  GemmDesc g = {};
   g.M = M; g.N = N; g.npairs = n_pairs; g.C = C; g.ldc = ldc; g.beta = beta;
   for (int i = 0; i < n_pairs; ++i) {
     const betty_gemm_operands& o = pairs[i];

@@ -12,13 +12,78 @@ struct GemmPair {
   int K;
   float alpha;
 };
+// What happens to an accumulator element acc[m,n] on its way out.
+enum GemmEpiMode {
+  EPI_STORE = 0,     // C = acc + beta*C
+  EPI_BIAS_ACT = 1,  // v = acc + bias[n];  C = v;  out16 = act(v)                       (forward layer)
+  EPI_ACT_BWD = 2,   // C = acc (if C);     out16 = acc * act'(a[m,n])                   (backward through an activation)
+  EPI_R_FWD = 3,     // v = acc + bias[n];  C = v;  out16 = act'(a[m,n]) * v             (R-operator forward)
+  EPI_R_BWD = 4      // out16 = acc * act'(a) + dh * act''(a) * Ra                       (R-operator backward)
+};
+struct GemmEpilogue {
+  int mode;
+  int act;                 // betty_activation
+  const float* bias;       // [N]
+  const float* a;          // [M,N] pre-activations, leading dimension N
+  const float* dh;         // [M,N]
+  const float* Ra;         // [M,N]
+  bf16* out16;             // [M, ld16] or null
+  int64_t ld16;
+};
 struct GemmDesc {
   int M, N;
   int npairs;
   GemmPair p[2];
-  float* C; int64_t ldc;
+  float* C; int64_t ldc;   // may be null for EPI_ACT_BWD / EPI_R_BWD
   float beta;
+  GemmEpilogue epi;        // zero-initialise for a plain store
 };
+
+// ---- activation functions shared by the matrix-product epilogues and the row kernels ----
+__device__ __forceinline__ float norm_pdf(float a) { return 0.3989422804014327f * expf(-0.5f * a * a); }
+__device__ __forceinline__ float norm_cdf(float a) { return 0.5f * (1.f + erff(a * 0.7071067811865476f)); }
+__device__ __forceinline__ float act_f(int act, float a) { return act == BETTY_ACT_RELU ? fmaxf(a, 0.f) : a * norm_cdf(a); }
+__device__ __forceinline__ float act_d1(int act, float a) {
+  return act == BETTY_ACT_RELU ? (a > 0.f ? 1.f : 0.f) : norm_cdf(a) + a * norm_pdf(a);
+}
+__device__ __forceinline__ float act_d2(int act, float a) {
+  return act == BETTY_ACT_RELU ? 0.f : norm_pdf(a) * (2.f - a * a);
+}
+
+// One output element.  Used as is by the CUDA-core kernel; the tensor-core kernel applies the same
+// formulas to 32 consecutive columns of a row at a time.
+__device__ __forceinline__ void gemm_epilogue_store(const GemmEpilogue& e, float* C, int64_t ldc, float beta, int N,
+                                                    int m, int n, float acc) {
+  const int64_t j = (int64_t)m * N + n;
+  float* cp = C ? C + (int64_t)m * ldc + n : nullptr;
+  switch (e.mode) {
+    case EPI_STORE:
+      *cp = acc + (beta != 0.f ? beta * *cp : 0.f);
+      break;
+    case EPI_BIAS_ACT: {
+      const float v = acc + e.bias[n];
+      *cp = v;
+      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(act_f(e.act, v));
+      break;
+    }
+    case EPI_ACT_BWD:
+      if (cp) *cp = acc;
+      e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(acc * act_d1(e.act, e.a[j]));
+      break;
+    case EPI_R_FWD: {
+      const float v = acc + e.bias[n];
+      *cp = v;
+      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(act_d1(e.act, e.a[j]) * v);
+      break;
+    }
+    case EPI_R_BWD: {
+      float v = acc * act_d1(e.act, e.a[j]);
+      if (e.act != BETTY_ACT_RELU) v += e.dh[j] * act_d2(e.act, e.a[j]) * e.Ra[j];
+      e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(v);
+      break;
+    }
+  }
+}
 
 betty_status gemm(Ctx& c, const GemmDesc& g);
 // tcgen05 / tensor-memory path (gemm_tc.cu): needs 16-byte aligned operands, leading dimensions that

@@ -31,6 +31,8 @@ struct TcArgs {
   int M, N, npairs;
   TcPair p[2];
   float* C; int64_t ldc; float beta;
+  GemmEpilogue epi;
+  int vec_ok;            // every pointer the epilogue touches is 16-byte aligned and N, ldc, ld16 allow vector access
   StatusBlock* sb;
 };
 
@@ -228,28 +230,67 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
               : "r"(taddr) : "memory");
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
           if (m < g.M) {
-            float* crow = g.C + (int64_t)m * g.ldc;
             const int nb = n0 + c * 32;
-            const bool vec = ((g.ldc & 3) == 0) && ((((uintptr_t)g.C) & 15) == 0) && (nb + 32 <= g.N);
-            if (vec) {
+            const GemmEpilogue& e = g.epi;
+            if (g.vec_ok && nb + 32 <= g.N) {
+              float* crow = g.C ? g.C + (int64_t)m * g.ldc + nb : nullptr;
+              const int64_t jb = (int64_t)m * g.N + nb;
+              bf16* orow = e.out16 ? e.out16 + (int64_t)m * e.ld16 + nb : nullptr;
 #pragma unroll
-              for (int jj = 0; jj < 32; jj += 4) {
-                float4 v = make_float4(__uint_as_float(r[jj]), __uint_as_float(r[jj + 1]), __uint_as_float(r[jj + 2]),
-                                       __uint_as_float(r[jj + 3]));
-                float4* dst = (float4*)(crow + nb + jj);
-                if (g.beta != 0.f) { float4 o = *dst; v.x += g.beta * o.x; v.y += g.beta * o.y; v.z += g.beta * o.z; v.w += g.beta * o.w; }
-                *dst = v;
-              }
-            } else {
+              for (int j8 = 0; j8 < 32; j8 += 8) {
+                float v[8], o[8];
 #pragma unroll
-              for (int jj = 0; jj < 32; ++jj) {
-                const int n = nb + jj;
-                if (n < g.N) {
-                  float v = __uint_as_float(r[jj]);
-                  if (g.beta != 0.f) v += g.beta * crow[n];
-                  crow[n] = v;
+                for (int k = 0; k < 8; ++k) v[k] = __uint_as_float(r[j8 + k]);
+                if (e.mode == EPI_STORE) {
+                  if (g.beta != 0.f) {
+                    const float4 c0 = *(const float4*)(crow + j8), c1 = *(const float4*)(crow + j8 + 4);
+                    v[0] += g.beta * c0.x; v[1] += g.beta * c0.y; v[2] += g.beta * c0.z; v[3] += g.beta * c0.w;
+                    v[4] += g.beta * c1.x; v[5] += g.beta * c1.y; v[6] += g.beta * c1.z; v[7] += g.beta * c1.w;
+                  }
+                } else if (e.mode == EPI_BIAS_ACT || e.mode == EPI_R_FWD) {
+                  const float4 b0 = *(const float4*)(e.bias + nb + j8), b1 = *(const float4*)(e.bias + nb + j8 + 4);
+                  v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+                  v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+                  if (orow) {
+                    if (e.mode == EPI_BIAS_ACT) {
+#pragma unroll
+                      for (int k = 0; k < 8; ++k) o[k] = act_f(e.act, v[k]);
+                    } else {
+                      const float4 a0 = *(const float4*)(e.a + jb + j8), a1 = *(const float4*)(e.a + jb + j8 + 4);
+                      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+                      for (int k = 0; k < 8; ++k) o[k] = act_d1(e.act, av[k]) * v[k];
+                    }
+                  }
+                } else {   // EPI_ACT_BWD, EPI_R_BWD
+                  const float4 a0 = *(const float4*)(e.a + jb + j8), a1 = *(const float4*)(e.a + jb + j8 + 4);
+                  const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+                  for (int k = 0; k < 8; ++k) o[k] = v[k] * act_d1(e.act, av[k]);
+                  if (e.mode == EPI_R_BWD && e.act != BETTY_ACT_RELU) {
+                    const float4 d0 = *(const float4*)(e.dh + jb + j8), d1 = *(const float4*)(e.dh + jb + j8 + 4);
+                    const float4 q0 = *(const float4*)(e.Ra + jb + j8), q1 = *(const float4*)(e.Ra + jb + j8 + 4);
+                    const float dv[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                    const float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) o[k] += dv[k] * act_d2(e.act, av[k]) * qv[k];
+                  }
+                }
+                if (crow && e.mode != EPI_R_BWD) {
+                  *(float4*)(crow + j8) = make_float4(v[0], v[1], v[2], v[3]);
+                  *(float4*)(crow + j8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                }
+                if (orow && e.mode != EPI_STORE) {
+                  __nv_bfloat162 ob[4];
+#pragma unroll
+                  for (int k = 0; k < 4; ++k) ob[k] = __floats2bfloat162_rn(o[2 * k], o[2 * k + 1]);
+                  *(uint4*)(orow + j8) = *(uint4*)ob;
                 }
               }
+            } else {
+#pragma unroll 4
+              for (int jj = 0; jj < 32; ++jj)
+                if (nb + jj < g.N) gemm_epilogue_store(e, g.C, g.ldc, g.beta, g.N, m, nb + jj, __uint_as_float(r[jj]));
             }
           }
         }
@@ -258,11 +299,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
         __syncwarp();
         if (lane == 0) tc_arrive(&acc_empty[as]);
       } else if (m < g.M) {
-        // no products: C = beta * C
-        for (int n = n0; n < n0 + BN && n < g.N; ++n) {
-          float* cp = g.C + (int64_t)m * g.ldc + n;
-          *cp = g.beta != 0.f ? g.beta * *cp : 0.f;
-        }
+        // no products: the accumulator is zero
+        for (int n = n0; n < n0 + BN && n < g.N; ++n) gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.N, m, n, 0.f);
       }
     }
   }
@@ -333,6 +371,14 @@ static betty_status launch_tc(Ctx& c, const GemmDesc& g) {
   CUtensorMap tm[4];
   TcArgs a;
   a.M = g.M; a.N = g.N; a.npairs = g.npairs; a.C = g.C; a.ldc = g.ldc; a.beta = g.beta; a.sb = c.arena.status();
+  a.epi = g.epi;
+  {
+    auto al16 = [](const void* p) { return (((uintptr_t)p) & 15) == 0; };
+    const GemmEpilogue& e = g.epi;
+    bool ok = (g.N % 4 == 0) && al16(g.C) && (g.ldc % 4 == 0) && al16(e.bias) && al16(e.a) && al16(e.dh) && al16(e.Ra) &&
+              al16(e.out16) && (e.ld16 % 8 == 0);
+    a.vec_ok = ok ? 1 : 0;
+  }
   for (int i = 0; i < 2; ++i) {
     const GemmPair& p = g.p[i < g.npairs ? i : 0];
     a.p[i].K = i < g.npairs ? p.K : 0;

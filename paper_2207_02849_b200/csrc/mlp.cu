@@ -19,16 +19,7 @@ static inline int grid_for(int64_t n, int per_block = 256) {
   return (int)(b < 1 ? 1 : (b > 148 * 32 ? 148 * 32 : b));
 }
 
-// ------------------------------------------------------------------ activations
-__device__ __forceinline__ float norm_pdf(float a) { return 0.3989422804014327f * expf(-0.5f * a * a); }
-__device__ __forceinline__ float norm_cdf(float a) { return 0.5f * (1.f + erff(a * 0.7071067811865476f)); }
-__device__ __forceinline__ float act_f(int act, float a) { return act == BETTY_ACT_RELU ? fmaxf(a, 0.f) : a * norm_cdf(a); }
-__device__ __forceinline__ float act_d1(int act, float a) {
-  return act == BETTY_ACT_RELU ? (a > 0.f ? 1.f : 0.f) : norm_cdf(a) + a * norm_pdf(a);
-}
-__device__ __forceinline__ float act_d2(int act, float a) {
-  return act == BETTY_ACT_RELU ? 0.f : norm_pdf(a) * (2.f - a * a);
-}
+// ------------------------------------------------------------------ helpers
 __device__ __forceinline__ float fd_eps(const float* vnorm2, float eps0) {
   const float nv2 = *vnorm2;
   return nv2 > 0.f ? eps0 / sqrtf(nv2) : 0.f;
@@ -86,12 +77,22 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
     delta[i] = __float2bfloat16_rn(v);
   }
 }
+// out[n] = sum_i d[i, n].  Block = 32 columns x 8 row groups; fixed summation order.
 __global__ void k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, float* out) {
-  const int64_t n = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  if (n >= N) return;
+  __shared__ float sh[8][33];
+  const int cx = threadIdx.x & 31, rg = threadIdx.x >> 5;
+  const int64_t n = blockIdx.x * 32 + cx;
   float acc = 0.f;
-  for (int64_t i = 0; i < B; ++i) acc += __bfloat162float(d[i * ld + n]);
-  out[n] = acc;
+  if (n < N)
+    for (int64_t i = rg; i < B; i += 8) acc += __bfloat162float(d[i * ld + n]);
+  sh[rg][cx] = acc;
+  __syncthreads();
+  if (rg == 0 && n < N) {
+    float t = 0.f;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) t += sh[r][cx];
+    out[n] = t;
+  }
 }
 // delta_prev = dh * act'(a)
 __global__ void k_act_backward(const float* dh, const float* a, bf16* dprev, int64_t B, int64_t N, int64_t ld, int act) {
@@ -335,9 +336,26 @@ static betty_status net_layout(const betty_level* M, Net& n) {
   return BETTY_OK;
 }
 
+// contiguous case (ld == cols, cols % 8 == 0): 8 elements per thread, 2 x float4 in, 1 x 16 bytes out
+__global__ void k_cast_dense8(const float* src, bf16* dst, int64_t n8, const float* vnorm2, float eps0) {
+  const float s = vnorm2 ? fd_eps(vnorm2, eps0) : 1.f;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
+    const float4 a = ((const float4*)src)[2 * i], b = ((const float4*)src)[2 * i + 1];
+    __nv_bfloat162 o[4];
+    o[0] = __floats2bfloat162_rn(s * a.x, s * a.y); o[1] = __floats2bfloat162_rn(s * a.z, s * a.w);
+    o[2] = __floats2bfloat162_rn(s * b.x, s * b.y); o[3] = __floats2bfloat162_rn(s * b.z, s * b.w);
+    ((uint4*)dst)[i] = *(uint4*)o;
+  }
+}
+
 static betty_status cast_matrix(Ctx& c, const float* src, bf16* dst, int64_t rows, int64_t cols, int64_t ld,
                                 const float* vnorm2 = nullptr, float eps0 = 0.f) {
-  k_cast_rows<<<grid_for(rows * ld), 256, 0, c.stream>>>(src, dst, rows, cols, ld, vnorm2, eps0);
+  if (ld == cols && (cols & 7) == 0 && ((((uintptr_t)src) & 15) == 0)) {
+    const int64_t n8 = rows * cols / 8;
+    k_cast_dense8<<<grid_for(n8), 256, 0, c.stream>>>(src, dst, n8, vnorm2, eps0);
+  } else {
+    k_cast_rows<<<grid_for(rows * ld), 256, 0, c.stream>>>(src, dst, rows, cols, ld, vnorm2, eps0);
+  }
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
@@ -363,9 +381,6 @@ static betty_status forward(Ctx& c, const Net& n, const betty_level* D, Pass& ps
     const int64_t N = n.w[l + 1];
     BETTY_ALLOC(al, float, c, (size_t)(B * N));
     ps.a[l] = al;
-    GemmDesc g; g.M = (int)B; g.N = (int)N; g.npairs = 1; g.C = al; g.ldc = N; g.beta = 0.f;
-    g.p[0] = gemm_pair(ps.h[l], ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)n.w[l]);
-    BETTY_TRY(gemm(c, g));
     bf16* hn = nullptr;
     if (l < n.L - 1) {
       ps.ldh[l + 1] = ld8(N);
@@ -374,8 +389,12 @@ static betty_status forward(Ctx& c, const Net& n, const betty_level* D, Pass& ps
       if (ps.ldh[l + 1] != N) cudaMemsetAsync(hn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(bf16), c.stream);
       ps.h[l + 1] = hn;
     }
-    k_bias_act<<<grid_for(B * N), 256, 0, c.stream>>>(al, n.master + n.boff[l], hn, B, N, hn ? ps.ldh[l + 1] : 0, n.act);
-    BETTY_LAUNCH_CHECK();
+    // a_l = h_l W_l^T + b_l (kept in fp32 for the derivative passes), h_{l+1} = act(a_l) in bf16: one kernel
+    GemmDesc g = {}; g.M = (int)B; g.N = (int)N; g.npairs = 1; g.C = al; g.ldc = N; g.beta = 0.f;
+    g.p[0] = gemm_pair(ps.h[l], ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)n.w[l]);
+    g.epi.mode = EPI_BIAS_ACT; g.epi.act = n.act; g.epi.bias = n.master + n.boff[l];
+    g.epi.out16 = hn; g.epi.ld16 = hn ? ps.ldh[l + 1] : 0;
+    BETTY_TRY(gemm(c, g));
   }
   const int64_t C = n.w[n.L];
   BETTY_ALLOC(p, float, c, (size_t)(B * C));
@@ -401,27 +420,33 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
     if (gflat) {
-      GemmDesc g; g.M = (int)N; g.N = (int)K; g.npairs = 1; g.C = gflat + n.woff[l]; g.ldc = K; g.beta = 0.f;
+      GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.npairs = 1; g.C = gflat + n.woff[l]; g.ldc = K; g.beta = 0.f;
       g.p[0] = gemm_pair(ps.delta[l], ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
       BETTY_TRY(gemm(c, g));
       if (lam) {
         k_wd_add_bf16<<<grid_for(N * K), 256, 0, c.stream>>>(gflat + n.woff[l], n.W[l], N, K, n.ldw[l], lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      k_colsum_bf16<<<grid_for(N), 256, 0, c.stream>>>(ps.delta[l], B, N, ldd, gflat + n.boff[l]);
+      k_colsum_bf16<<<(unsigned)((N + 31) / 32), 256, 0, c.stream>>>(ps.delta[l], B, N, ldd, gflat + n.boff[l]);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {
-      BETTY_ALLOC(dh, float, c, (size_t)(B * K));
+      // dh = delta_l W_l ; delta_{l-1} = dh * act'(a_{l-1}) in bf16: one kernel.  dh itself is kept
+      // only when the activation has a second derivative (the R-operator pass needs it then).
+      float* dh = nullptr;
+      if (n.act != BETTY_ACT_RELU) {
+        dh = c.arena.alloc<float>((size_t)(B * K));
+        if (!dh) return BETTY_ERR_WORKSPACE;
+      }
       ps.dh[l] = dh;
-      GemmDesc g; g.M = (int)B; g.N = (int)K; g.npairs = 1; g.C = dh; g.ldc = K; g.beta = 0.f;
-      g.p[0] = gemm_pair(ps.delta[l], ldd, false, n.W[l], n.ldw[l], false, (int)N);
-      BETTY_TRY(gemm(c, g));
       const int64_t ldp = ld8(K);
       BETTY_ALLOC(dp, bf16, c, (size_t)(B * ldp));
+      if (ldp != K) cudaMemsetAsync(dp, 0, (size_t)(B * ldp) * sizeof(bf16), c.stream);
       ps.delta[l - 1] = dp;
-      k_act_backward<<<grid_for(B * ldp), 256, 0, c.stream>>>(dh, ps.a[l - 1], dp, B, K, ldp, n.act);
-      BETTY_LAUNCH_CHECK();
+      GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.npairs = 1; g.C = dh; g.ldc = K; g.beta = 0.f;
+      g.p[0] = gemm_pair(ps.delta[l], ldd, false, n.W[l], n.ldw[l], false, (int)N);
+      g.epi.mode = EPI_ACT_BWD; g.epi.act = n.act; g.epi.a = ps.a[l - 1]; g.epi.out16 = dp; g.epi.ld16 = ldp;
+      BETTY_TRY(gemm(c, g));
     }
   }
   return BETTY_OK;
@@ -443,11 +468,6 @@ static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* 
     BETTY_TRY(cast_matrix(c, dir + n.woff[l], Ul, N, K, n.ldw[l]));
     BETTY_ALLOC(Ra, float, c, (size_t)(B * N));
     rp.Ra[l] = Ra;
-    GemmDesc g; g.M = (int)B; g.N = (int)N; g.C = Ra; g.ldc = N; g.beta = 0.f;
-    g.npairs = 0;
-    g.p[g.npairs++] = gemm_pair(ps.h[l], ps.ldh[l], false, Ul, n.ldw[l], true, (int)K);
-    if (l > 0) g.p[g.npairs++] = gemm_pair(rp.Rh[l], ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)K);
-    BETTY_TRY(gemm(c, g));
     bf16* Rhn = nullptr;
     if (l < n.L - 1) {
       Rhn = c.arena.alloc<bf16>((size_t)(B * ps.ldh[l + 1]));
@@ -455,9 +475,14 @@ static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* 
       if (ps.ldh[l + 1] != N) cudaMemsetAsync(Rhn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(bf16), c.stream);
       rp.Rh[l + 1] = Rhn;
     }
-    k_r_act_forward<<<grid_for(B * N), 256, 0, c.stream>>>(Ra, dir + n.boff[l], ps.a[l], Rhn, B, N,
-                                                          Rhn ? ps.ldh[l + 1] : 0, n.act);
-    BETTY_LAUNCH_CHECK();
+    // Ra_l = h_l U_l^T + Rh_l W_l^T + c_l ; Rh_{l+1} = act'(a_l) * Ra_l: one kernel
+    GemmDesc g = {}; g.M = (int)B; g.N = (int)N; g.C = Ra; g.ldc = N; g.beta = 0.f;
+    g.npairs = 0;
+    g.p[g.npairs++] = gemm_pair(ps.h[l], ps.ldh[l], false, Ul, n.ldw[l], true, (int)K);
+    if (l > 0) g.p[g.npairs++] = gemm_pair(rp.Rh[l], ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)K);
+    g.epi.mode = EPI_R_FWD; g.epi.act = n.act; g.epi.bias = dir + n.boff[l]; g.epi.a = ps.a[l];
+    g.epi.out16 = Rhn; g.epi.ld16 = Rhn ? ps.ldh[l + 1] : 0;
+    BETTY_TRY(gemm(c, g));
   }
   return BETTY_OK;
 }
@@ -628,7 +653,7 @@ betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const floa
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
     {  // R gW_l = Rdelta^T h_l + delta_l^T Rh_l + exp(lam_l) U_l
-      GemmDesc g; g.M = (int)N; g.N = (int)K; g.C = Hu + n.woff[l]; g.ldc = K; g.beta = 0.f; g.npairs = 0;
+      GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.C = Hu + n.woff[l]; g.ldc = K; g.beta = 0.f; g.npairs = 0;
       g.p[g.npairs++] = gemm_pair(Rd, ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
       if (l > 0) g.p[g.npairs++] = gemm_pair(ps.delta[l], ldd, true, rp.Rh[l], ps.ldh[l], false, (int)B);
       BETTY_TRY(gemm(c, g));
@@ -636,20 +661,19 @@ betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const floa
         k_wd_add_f32<<<grid_for(N * K), 256, 0, c.stream>>>(Hu + n.woff[l], u + n.woff[l], N * K, h->lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      k_colsum_bf16<<<grid_for(N), 256, 0, c.stream>>>(Rd, B, N, ldd, Hu + n.boff[l]);
+      k_colsum_bf16<<<(unsigned)((N + 31) / 32), 256, 0, c.stream>>>(Rd, B, N, ldd, Hu + n.boff[l]);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {  // R dh = Rdelta W_l + delta_l U_l ; Rdelta_{l-1} = Rdh*act' + dh*act''*Ra
-      BETTY_ALLOC(Rdh, float, c, (size_t)(B * K));
-      GemmDesc g; g.M = (int)B; g.N = (int)K; g.C = Rdh; g.ldc = K; g.beta = 0.f; g.npairs = 2;
-      g.p[0] = gemm_pair(Rd, ldd, false, n.W[l], n.ldw[l], false, (int)N);
-      g.p[1] = gemm_pair(ps.delta[l], ldd, false, rp.U[l], n.ldw[l], false, (int)N);
-      BETTY_TRY(gemm(c, g));
       const int64_t ldp = ld8(K);
       BETTY_ALLOC(Rdp, bf16, c, (size_t)(B * ldp));
-      k_r_act_backward<<<grid_for(B * ldp), 256, 0, c.stream>>>(Rdh, ps.dh[l], ps.a[l - 1], rp.Ra[l - 1], Rdp, B, K, ldp,
-                                                              n.act);
-      BETTY_LAUNCH_CHECK();
+      if (ldp != K) cudaMemsetAsync(Rdp, 0, (size_t)(B * ldp) * sizeof(bf16), c.stream);
+      GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.C = nullptr; g.ldc = K; g.beta = 0.f; g.npairs = 2;
+      g.p[0] = gemm_pair(Rd, ldd, false, n.W[l], n.ldw[l], false, (int)N);
+      g.p[1] = gemm_pair(ps.delta[l], ldd, false, rp.U[l], n.ldw[l], false, (int)N);
+      g.epi.mode = EPI_R_BWD; g.epi.act = n.act; g.epi.a = ps.a[l - 1]; g.epi.dh = ps.dh[l]; g.epi.Ra = rp.Ra[l - 1];
+      g.epi.out16 = Rdp; g.epi.ld16 = ldp;
+      BETTY_TRY(gemm(c, g));
       Rd = Rdp;
     }
   }
@@ -752,7 +776,7 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
     for (int l = 0; l < n.L; ++l) {
       const int64_t N = n.w[l + 1], K = n.w[l];
       BETTY_ALLOC(da, float, c, (size_t)(B * N));
-      GemmDesc g; g.M = (int)B; g.N = (int)N; g.C = da; g.ldc = N; g.beta = 0.f; g.npairs = 0;
+      GemmDesc g = {}; g.M = (int)B; g.N = (int)N; g.C = da; g.ldc = N; g.beta = 0.f; g.npairs = 0;
       g.p[g.npairs++] = gemm_pair(hp, ps.ldh[l], false, E[l], n.ldw[l], true, (int)K, sign);
       if (l > 0) g.p[g.npairs++] = gemm_pair(dh, ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)K);
       BETTY_TRY(gemm(c, g));
