@@ -396,6 +396,41 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def gemm_probe(args, torch, bt):
+    """Times `steps` back-to-back launches of one matrix product (queued behind a long memset so
+    that host-side launch cost does not show) and prints achieved TFLOP/s."""
+    f = [int(x) for x in args.gemm.split(",")]
+    M, N, K = f[:3]
+    ta, tb, npairs, path = (f[3:] + [0, 1, 1, 0][len(f) - 3:])[:4]
+    A = torch.randn((K, M) if ta else (M, K), device="cuda").to(torch.bfloat16)
+    B = torch.randn((N, K) if tb else (K, N), device="cuda").to(torch.bfloat16)
+    C = torch.empty(M, N, dtype=torch.float32, device="cuda")
+    pairs = [(A, A.shape[1], ta, B, B.shape[1], tb, K, 1.0)] * npairs
+    lv = bt.Level(bt.LOSS_LOGREG, bt.PARAM_VECTOR, torch.zeros(8, device="cuda"))
+    ws = bt.Workspace.__new__(bt.Workspace)
+    ws.nbytes = 4096
+    ws.buf = torch.zeros(4096 + 256, dtype=torch.uint8, device="cuda")
+    ws.ptr = ws.buf.data_ptr() + (-ws.buf.data_ptr()) % 256
+    for _ in range(max(args.warmup, 3)):
+        bt.betty_gemm_bf16(M, N, pairs, C, N, 0.0, path, ws)
+    big = torch.empty(1 << 28, dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    big.zero_(); big.zero_()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        bt.betty_gemm_bf16(M, N, pairs, C, N, 0.0, path, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    peaks = _peaks()
+    tf = 2.0 * M * N * K * npairs / (ms * 1e-3) / 1e12
+    print(json.dumps({"kernel": "betty_gemm_bf16", "M": M, "N": N, "K": K, "a_transposed": ta, "b_transposed": tb,
+                      "n_pairs": npairs, "path": path, "us_per_launch": ms * 1e3, "tflops": tf,
+                      "frac_of_bf16_peak": tf / peaks["bf16_tflops"], "peak_source": peaks["source"],
+                      "device_status": bt.betty_status_string(bt.betty_poll_status(ws, raise_on_error=False)[0])}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -406,6 +441,12 @@ def main():
     ap.add_argument("--method", default="")
     ap.add_argument("--scale", type=float, default=1.0, help="row-count scale of config 2 (tests/profiling only)")
     ap.add_argument("--oracle-rows", type=int, default=131072)
+    ap.add_argument("--graph", type=int, default=-1,
+                    help="replay the step from a CUDA graph captured from the C-ABI calls (default: on for the "
+                         "launch-bound configs 1, 3, 4)")
+    ap.add_argument("--gemm", default="",
+                    help="M,N,K[,a_transposed,b_transposed,n_pairs,path]: time only the bf16 matrix-product kernel "
+                         "through betty_gemm_bf16 (kernel study; prints its own JSON line)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -431,6 +472,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     import paper_2207_02849_b200 as bt
 
+    if args.gemm:
+        gemm_probe(args, torch, bt)
+        return
     wl = make_workload(args.config, args.method, args.scale)
     wl.setup_device()
     warm = max(args.warmup, 3)
@@ -469,6 +513,8 @@ def main():
         if sampler:
             sampler.mark_end()
         launches = bt.betty_kernel_launches() - l0
+        if launches_per_replay is not None:
+            launches = launches_per_replay * steps
         clocks = sampler.stop() if sampler else None
         ms = sum(a.elapsed_time(b) for a, b in pairs)
         if world > 1:
@@ -483,6 +529,24 @@ def main():
         flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     l2_note = ("inputs (train matrix) larger than L2; no flush between steps" if flush is None
                else "L2 flushed (512 MiB write) before every step; each step timed by its own event pair, flush excluded")
+    use_graph = (args.graph == 1) or (args.graph == -1 and args.config in (1, 3, 4))
+    launches_per_replay = None
+    if use_graph:
+        # The library's calls only enqueue work on the current stream and keep every scalar on the
+        # device, so a whole step can be captured once and replayed without host-side launch cost.
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(2):
+                wl.step()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        l0 = bt.betty_kernel_launches()
+        with torch.cuda.graph(graph):
+            wl.step()
+        launches_per_replay = bt.betty_kernel_launches() - l0
+        wl.step = graph.replay
     step_dev, step_host = wl.step, wl.step_e2e
 
     sampler = ClockSampler(local) if rank == 0 else None
@@ -533,7 +597,7 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": wl.dtype, "data": "synthetic",
             "config": {"workload": wl.name, "l2": l2_note,
-                       "replicas": world, "device_status": bt.betty_status_string(st)},
+                       "replicas": world, "cuda_graph": bool(use_graph), "device_status": bt.betty_status_string(st)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:

@@ -90,6 +90,7 @@ betty_status gemm(Ctx& c, const GemmDesc& g);
 // are multiples of 8 elements and alpha = +-1
 bool gemm_tc_eligible(const GemmDesc& g);
 betty_status gemm_tc(Ctx& c, const GemmDesc& g);
+betty_status gemm_tc_pair(Ctx& c, const GemmDesc& g);   // two-SM (cta_group::2) kernel, 256 x 256 tiles
 // CUDA-core reference path (any shape, any stride); also the fallback for shapes the tensor-core
 // path does not take.
 betty_status gemm_simt(Ctx& c, const GemmDesc& g);

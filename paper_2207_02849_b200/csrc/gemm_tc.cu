@@ -95,6 +95,85 @@ __device__ __forceinline__ void tc_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(bar)) : "memory");
 }
 
+// 32 consecutive accumulator columns of this thread's lane
+__device__ __forceinline__ void tmem_load32(uint32_t (&r)[32], uint32_t taddr) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Epilogue of row m, columns nb .. nb+31 (accumulator bits in r)
+__device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, const uint32_t (&r)[32]) {
+  const GemmEpilogue& e = g.epi;
+  if (g.vec_ok && nb + 32 <= g.N) {
+    float* crow = g.C ? g.C + (int64_t)m * g.ldc + nb : nullptr;
+    const int64_t jb = (int64_t)m * g.N + nb;
+    bf16* orow = e.out16 ? e.out16 + (int64_t)m * e.ld16 + nb : nullptr;
+#pragma unroll
+    for (int j8 = 0; j8 < 32; j8 += 8) {
+      float v[8], o[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) { v[k] = __uint_as_float(r[j8 + k]); o[k] = 0.f; }
+      if (e.mode == EPI_STORE) {
+        if (g.beta != 0.f) {
+          const float4 c0 = *(const float4*)(crow + j8), c1 = *(const float4*)(crow + j8 + 4);
+          v[0] += g.beta * c0.x; v[1] += g.beta * c0.y; v[2] += g.beta * c0.z; v[3] += g.beta * c0.w;
+          v[4] += g.beta * c1.x; v[5] += g.beta * c1.y; v[6] += g.beta * c1.z; v[7] += g.beta * c1.w;
+        }
+      } else if (e.mode == EPI_BIAS_ACT || e.mode == EPI_R_FWD) {
+        const float4 b0 = *(const float4*)(e.bias + nb + j8), b1 = *(const float4*)(e.bias + nb + j8 + 4);
+        v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
+        v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
+        if (orow) {
+          if (e.mode == EPI_BIAS_ACT) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) o[k] = act_f(e.act, v[k]);
+          } else {
+            const float4 a0 = *(const float4*)(e.a + jb + j8), a1 = *(const float4*)(e.a + jb + j8 + 4);
+            const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+            for (int k = 0; k < 8; ++k) o[k] = act_d1(e.act, av[k]) * v[k];
+          }
+        }
+      } else {   // EPI_ACT_BWD, EPI_R_BWD
+        const float4 a0 = *(const float4*)(e.a + jb + j8), a1 = *(const float4*)(e.a + jb + j8 + 4);
+        const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+        for (int k = 0; k < 8; ++k) o[k] = v[k] * act_d1(e.act, av[k]);
+        if (e.mode == EPI_R_BWD && e.act != BETTY_ACT_RELU) {
+          const float4 d0 = *(const float4*)(e.dh + jb + j8), d1 = *(const float4*)(e.dh + jb + j8 + 4);
+          const float4 q0 = *(const float4*)(e.Ra + jb + j8), q1 = *(const float4*)(e.Ra + jb + j8 + 4);
+          const float dv[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+          const float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+          for (int k = 0; k < 8; ++k) o[k] += dv[k] * act_d2(e.act, av[k]) * qv[k];
+        }
+      }
+      if (crow && e.mode != EPI_R_BWD) {
+        *(float4*)(crow + j8) = make_float4(v[0], v[1], v[2], v[3]);
+        *(float4*)(crow + j8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+      }
+      if (orow && e.mode != EPI_STORE) {
+        __nv_bfloat162 ob[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) ob[k] = __floats2bfloat162_rn(o[2 * k], o[2 * k + 1]);
+        *(uint4*)(orow + j8) = *(uint4*)ob;
+      }
+    }
+  } else {
+#pragma unroll 4
+    for (int jj = 0; jj < 32; ++jj)
+      if (nb + jj < g.N) gemm_epilogue_store(e, g.C, g.ldc, g.beta, g.N, m, nb + jj, __uint_as_float(r[jj]));
+  }
+}
+
 // Persistent kernel: CTA b works on output tiles b, b + gridDim.x, ...
 template <int BN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -219,80 +298,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
           if (n0 + c * 32 >= g.N) break;            // uniform: nothing to store from these columns
           uint32_t r[32];
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32);
-          asm volatile(
-              "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-              "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-              "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-              : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-              : "r"(taddr) : "memory");
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          if (m < g.M) {
-            const int nb = n0 + c * 32;
-            const GemmEpilogue& e = g.epi;
-            if (g.vec_ok && nb + 32 <= g.N) {
-              float* crow = g.C ? g.C + (int64_t)m * g.ldc + nb : nullptr;
-              const int64_t jb = (int64_t)m * g.N + nb;
-              bf16* orow = e.out16 ? e.out16 + (int64_t)m * e.ld16 + nb : nullptr;
-#pragma unroll
-              for (int j8 = 0; j8 < 32; j8 += 8) {
-                float v[8], o[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) v[k] = __uint_as_float(r[j8 + k]);
-                if (e.mode == EPI_STORE) {
-                  if (g.beta != 0.f) {
-                    const float4 c0 = *(const float4*)(crow + j8), c1 = *(const float4*)(crow + j8 + 4);
-                    v[0] += g.beta * c0.x; v[1] += g.beta * c0.y; v[2] += g.beta * c0.z; v[3] += g.beta * c0.w;
-                    v[4] += g.beta * c1.x; v[5] += g.beta * c1.y; v[6] += g.beta * c1.z; v[7] += g.beta * c1.w;
-                  }
-                } else if (e.mode == EPI_BIAS_ACT || e.mode == EPI_R_FWD) {
-                  const float4 b0 = *(const float4*)(e.bias + nb + j8), b1 = *(const float4*)(e.bias + nb + j8 + 4);
-                  v[0] += b0.x; v[1] += b0.y; v[2] += b0.z; v[3] += b0.w;
-                  v[4] += b1.x; v[5] += b1.y; v[6] += b1.z; v[7] += b1.w;
-                  if (orow) {
-                    if (e.mode == EPI_BIAS_ACT) {
-#pragma unroll
-                      for (int k = 0; k < 8; ++k) o[k] = act_f(e.act, v[k]);
-                    } else {
-                      const float4 a0 = *(const float4*)(e.a + jb + j8), a1 = *(const float4*)(e.a + jb + j8 + 4);
-                      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-#pragma unroll
-                      for (int k = 0; k < 8; ++k) o[k] = act_d1(e.act, av[k]) * v[k];
-                    }
-                  }
-                } else {   // EPI_ACT_BWD, EPI_R_BWD
-                  const float4 a0 = *(const float4*)(e.a + jb + j8), a1 = *(const float4*)(e.a + jb + j8 + 4);
-                  const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-#pragma unroll
-                  for (int k = 0; k < 8; ++k) o[k] = v[k] * act_d1(e.act, av[k]);
-                  if (e.mode == EPI_R_BWD && e.act != BETTY_ACT_RELU) {
-                    const float4 d0 = *(const float4*)(e.dh + jb + j8), d1 = *(const float4*)(e.dh + jb + j8 + 4);
-                    const float4 q0 = *(const float4*)(e.Ra + jb + j8), q1 = *(const float4*)(e.Ra + jb + j8 + 4);
-                    const float dv[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-                    const float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) o[k] += dv[k] * act_d2(e.act, av[k]) * qv[k];
-                  }
-                }
-                if (crow && e.mode != EPI_R_BWD) {
-                  *(float4*)(crow + j8) = make_float4(v[0], v[1], v[2], v[3]);
-                  *(float4*)(crow + j8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
-                }
-                if (orow && e.mode != EPI_STORE) {
-                  __nv_bfloat162 ob[4];
-#pragma unroll
-                  for (int k = 0; k < 4; ++k) ob[k] = __floats2bfloat162_rn(o[2 * k], o[2 * k + 1]);
-                  *(uint4*)(orow + j8) = *(uint4*)ob;
-                }
-              }
-            } else {
-#pragma unroll 4
-              for (int jj = 0; jj < 32; ++jj)
-                if (nb + jj < g.N) gemm_epilogue_store(e, g.C, g.ldc, g.beta, g.N, m, nb + jj, __uint_as_float(r[jj]));
-            }
-          }
+          tmem_load32(r, taddr);
+          if (m < g.M) epilogue_row32(g, m, n0 + c * 32, r);
         }
         // this warp has drained its quarter of the accumulator: the MMA warp may reuse it
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -310,6 +317,182 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   if (*abort_flag && tid == 0) record_status(g.sb, BETTY_ERR_TIMEOUT);
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg::TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ two-SM variant
+// A pair of CTAs (a cluster of two, on the two SMs of one TPC) works on one 256 x 256 output tile
+// with tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of A and 128 of the 256 columns
+// of B, so every byte of B fetched from L2 feeds twice as many MMA rows as in the one-SM kernel.
+// The even CTA of the pair issues the MMAs; each CTA holds the accumulator rows of its own half in
+// its tensor memory and runs its own epilogue.  Plain TMA loads, no multicast.
+static constexpr int TC2_BN = 256;           // tile width; each CTA stages half of it
+static constexpr int TC2_STAGE_BYTES = TC_A_BYTES + (TC2_BN / 2) * TC_BK * 2;   // 32 KB per CTA
+static constexpr int TC2_STAGES = 6;
+static constexpr int TC2_SMEM = TC2_STAGES * TC2_STAGE_BYTES + 1024 + 256;
+
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* tm, int x, int y, uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(s_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void commit_pair(uint32_t bar_cluster_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+           const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1, TcArgs g) {
+  constexpr int S = TC2_STAGES;
+  constexpr int BN = TC2_BN, HB = TC2_BN / 2;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = (uint64_t*)(smem + S * TC2_STAGE_BYTES);
+  uint64_t* empty = full + S;
+  uint64_t* acc_full = empty + S;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const bool leader = rank == 0;
+  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+  int iters[2] = {0, 0};
+  for (int p = 0; p < g.npairs; ++p) iters[p] = (g.p[p].K + TC_BK - 1) / TC_BK;
+  const int T = iters[0] + iters[1];
+  const int tiles_n = (g.N + BN - 1) / BN;
+  const int tiles = tiles_n * ((g.M + 2 * TC_BM - 1) / (2 * TC_BM));
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { tc_mbar_init(&full[s], 1); tc_mbar_init(&empty[s], 1); }
+    for (int s = 0; s < 2; ++s) { tc_mbar_init(&acc_full[s], 1); tc_mbar_init(&acc_empty[s], 8); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {   // the same warp of both CTAs allocates the pair's accumulator columns
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "r"(2 * BN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();     // the peer's barriers exist before anything is signalled across the pair
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0 && lane == 0 && T > 0) {
+    // ---------------- producer (both CTAs): own half of A and of B; completion counted on the leader's barrier
+    long long git = 0;
+    for (int t = cluster_id; t < tiles && !*abort_flag; t += n_clusters) {
+      const int m0 = (t / tiles_n) * (2 * TC_BM) + (int)rank * TC_BM, n0 = (t % tiles_n) * BN + (int)rank * HB;
+      for (int it = 0; it < T; ++it, ++git) {
+        const int s = (int)(git % S);
+        if (git >= S && !tc_wait(&empty[s], (uint32_t)(((git / S) - 1) & 1), abort_flag)) break;
+        const int p = it < iters[0] ? 0 : 1;
+        const int k0 = (p == 0 ? it : it - iters[0]) * TC_BK;
+        const CUtensorMap* ta = p == 0 ? &tmA0 : &tmA1;
+        const CUtensorMap* tb = p == 0 ? &tmB0 : &tmB1;
+        unsigned char* sa = smem + s * TC2_STAGE_BYTES;
+        unsigned char* sb = sa + TC_A_BYTES;
+        const uint32_t bar = map_to_cta(s_u32(&full[s]), 0);
+        if (leader) tc_expect_tx(&full[s], 2 * TC2_STAGE_BYTES);
+        if (!g.p[p].a_mn) {
+          tma_load_2d_pair(sa, ta, k0, m0, bar);
+        } else {
+          for (int j = 0; j < TC_BM / 64; ++j) tma_load_2d_pair(sa + j * 8192, ta, m0 + 64 * j, k0, bar);
+        }
+        if (!g.p[p].b_mn) {
+          tma_load_2d_pair(sb, tb, k0, n0, bar);
+        } else {
+          for (int j = 0; j < HB / 64; ++j) tma_load_2d_pair(sb + j * 8192, tb, n0 + 64 * j, k0, bar);
+        }
+      }
+    }
+  } else if (warp == 1 && lane == 0 && T > 0 && leader) {
+    // ---------------- MMA issuer (even CTA of the pair only)
+    long long git = 0;
+    int j = 0;
+    bool ok = true;
+    for (int t = cluster_id; t < tiles && ok; t += n_clusters, ++j) {
+      const int as = j & 1;
+      if (j >= 2 && !tc_wait(&acc_empty[as], (uint32_t)(((j >> 1) - 1) & 1), abort_flag)) { ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t tmem_acc = tmem_base + (uint32_t)(as * BN);
+      for (int it = 0; it < T; ++it, ++git) {
+        const int s = (int)(git % S);
+        if (!tc_wait(&full[s], (uint32_t)((git / S) & 1), abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int p = it < iters[0] ? 0 : 1;
+        const uint32_t idesc = instr_desc(g.p[p].a_mn, g.p[p].b_mn, g.p[p].neg, BN, 2 * TC_BM);
+        const uint32_t sa = s_u32(smem + s * TC2_STAGE_BYTES), sb = sa + TC_A_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < TC_BK / 16; ++kk) {
+          const uint64_t da = g.p[p].a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
+          const uint64_t db = g.p[p].b_mn ? smem_desc(sb + kk * 2048, 8192, 1024) : smem_desc(sb + kk * 32, 16, 1024);
+          const uint32_t acc = (it > 0 || kk > 0) ? 1u : 0u;
+          asm volatile(
+              "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+              "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+              ::"r"(tmem_acc), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+        }
+        // both CTAs may refill the stage once these MMAs have read it
+        commit_pair(map_to_cta(s_u32(&empty[s]), 0));
+        commit_pair(map_to_cta(s_u32(&empty[s]), 1));
+      }
+      if (ok) {
+        commit_pair(map_to_cta(s_u32(&acc_full[as]), 0));
+        commit_pair(map_to_cta(s_u32(&acc_full[as]), 1));
+      }
+    }
+  } else if (warp >= 2) {
+    // ---------------- epilogue (both CTAs): own 128 rows of the pair's tile
+    const int q = warp & 3;
+    int j = 0;
+    for (int t = cluster_id; t < tiles; t += n_clusters, ++j) {
+      const int m0 = (t / tiles_n) * (2 * TC_BM) + (int)rank * TC_BM, n0 = (t % tiles_n) * BN;
+      const int as = j & 1;
+      const int m = m0 + q * 32 + lane;
+      if (T > 0) {
+        bool have = tc_wait(&acc_full[as], (uint32_t)((j >> 1) & 1), abort_flag);
+        have = __all_sync(0xffffffffu, have);
+        if (!have) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          if (n0 + c * 32 >= g.N) break;
+          uint32_t r[32];
+          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32);
+          tmem_load32(r, taddr);
+          if (m < g.M) epilogue_row32(g, m, n0 + c * 32, r);
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          const uint32_t bar = map_to_cta(s_u32(&acc_empty[as]), 0);
+          asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+        }
+      } else if (m < g.M) {
+        for (int n = n0; n < n0 + BN && n < g.N; ++n) gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.N, m, n, 0.f);
+      }
+    }
+  }
+  __syncwarp();
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();     // neither CTA leaves while the other may still signal its barriers
+  if (*abort_flag && tid == 0) record_status(g.sb, BETTY_ERR_TIMEOUT);
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
   }
 }
 
@@ -360,6 +543,8 @@ bool gemm_tc_eligible(const GemmDesc& g) {
   return encode_fn() != nullptr;
 }
 
+static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a);
+
 template <int BN>
 static betty_status launch_tc(Ctx& c, const GemmDesc& g) {
   using Cfg = TcCfg<BN>;
@@ -370,24 +555,11 @@ static betty_status launch_tc(Ctx& c, const GemmDesc& g) {
   }
   CUtensorMap tm[4];
   TcArgs a;
-  a.M = g.M; a.N = g.N; a.npairs = g.npairs; a.C = g.C; a.ldc = g.ldc; a.beta = g.beta; a.sb = c.arena.status();
-  a.epi = g.epi;
-  {
-    auto al16 = [](const void* p) { return (((uintptr_t)p) & 15) == 0; };
-    const GemmEpilogue& e = g.epi;
-    bool ok = (g.N % 4 == 0) && al16(g.C) && (g.ldc % 4 == 0) && al16(e.bias) && al16(e.a) && al16(e.dh) && al16(e.Ra) &&
-              al16(e.out16) && (e.ld16 % 8 == 0);
-    a.vec_ok = ok ? 1 : 0;
-  }
+  fill_args(c, g, a);
   for (int i = 0; i < 2; ++i) {
     const GemmPair& p = g.p[i < g.npairs ? i : 0];
-    a.p[i].K = i < g.npairs ? p.K : 0;
-    a.p[i].a_mn = p.ta ? 1 : 0;
-    a.p[i].b_mn = p.tb ? 0 : 1;
-    a.p[i].neg = p.alpha < 0.f ? 1 : 0;
-    bool ok;
     // A: K-major = stored [M,K]; M-major = stored [K,M]
-    ok = p.ta ? make_map(&tm[2 * i], p.A, g.M, p.K, p.lda, 64, 64) : make_map(&tm[2 * i], p.A, p.K, g.M, p.lda, TC_BK, TC_BM);
+    bool ok = p.ta ? make_map(&tm[2 * i], p.A, g.M, p.K, p.lda, 64, 64) : make_map(&tm[2 * i], p.A, p.K, g.M, p.lda, TC_BK, TC_BM);
     if (!ok) return BETTY_ERR_CUDA;
     // B: K-major = stored [N,K]; N-major = stored [K,N]
     ok = p.tb ? make_map(&tm[2 * i + 1], p.B, p.K, g.N, p.ldb, TC_BK, BN) : make_map(&tm[2 * i + 1], p.B, g.N, p.K, p.ldb, 64, 64);
@@ -399,6 +571,49 @@ static betty_status launch_tc(Ctx& c, const GemmDesc& g) {
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
+
+static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a) {
+  a.M = g.M; a.N = g.N; a.npairs = g.npairs; a.C = g.C; a.ldc = g.ldc; a.beta = g.beta; a.sb = c.arena.status();
+  a.epi = g.epi;
+  auto al16 = [](const void* p) { return (((uintptr_t)p) & 15) == 0; };
+  const GemmEpilogue& e = g.epi;
+  const bool ok = (g.N % 4 == 0) && al16(g.C) && (g.ldc % 4 == 0) && al16(e.bias) && al16(e.a) && al16(e.dh) && al16(e.Ra) &&
+                  al16(e.out16) && (e.ld16 % 8 == 0);
+  a.vec_ok = ok ? 1 : 0;
+  for (int i = 0; i < 2; ++i) {
+    const GemmPair& p = g.p[i < g.npairs ? i : 0];
+    a.p[i].K = i < g.npairs ? p.K : 0;
+    a.p[i].a_mn = p.ta ? 1 : 0;
+    a.p[i].b_mn = p.tb ? 0 : 1;
+    a.p[i].neg = p.alpha < 0.f ? 1 : 0;
+  }
+}
+
+static betty_status launch_tc2(Ctx& c, const GemmDesc& g) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k_gemm_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, TC2_SMEM) != cudaSuccess) return BETTY_ERR_CUDA;
+    attr_set = true;
+  }
+  CUtensorMap tm[4];
+  TcArgs a;
+  fill_args(c, g, a);
+  for (int i = 0; i < 2; ++i) {
+    const GemmPair& p = g.p[i < g.npairs ? i : 0];
+    bool ok = p.ta ? make_map(&tm[2 * i], p.A, g.M, p.K, p.lda, 64, 64) : make_map(&tm[2 * i], p.A, p.K, g.M, p.lda, TC_BK, TC_BM);
+    if (!ok) return BETTY_ERR_CUDA;
+    ok = p.tb ? make_map(&tm[2 * i + 1], p.B, p.K, g.N, p.ldb, TC_BK, TC2_BN / 2) : make_map(&tm[2 * i + 1], p.B, g.N, p.K, p.ldb, 64, 64);
+    if (!ok) return BETTY_ERR_CUDA;
+  }
+  const int tiles = ((g.N + TC2_BN - 1) / TC2_BN) * ((g.M + 2 * TC_BM - 1) / (2 * TC_BM));
+  const int max_pairs = c.sm_count / 2;
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  k_gemm_tc2<<<2 * pairs, TC_THREADS, TC2_SMEM, c.stream>>>(tm[0], tm[1], tm[2], tm[3], a);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
+betty_status gemm_tc_pair(Ctx& c, const GemmDesc& g) { return launch_tc2(c, g); }
 
 betty_status gemm_tc(Ctx& c, const GemmDesc& g) {
   // wide tiles unless the problem is narrow or would leave most SMs without a tile

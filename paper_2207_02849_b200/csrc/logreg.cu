@@ -251,7 +251,11 @@ template <int NCH, bool HVP>
 static betty_status launch_stream(Ctx& c, const LrArgs& a, int grid) {
   size_t smem = (size_t)LR_S * LR_R * a.d * sizeof(float) + LR_S * sizeof(uint64_t) + 2 * LR_WARPS * 2 * LR_R * sizeof(float);
   auto kern = k_logreg_stream<NCH, HVP>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BETTY_ERR_CUDA;
+  static size_t attr_bytes = 0;     // raise the dynamic shared memory limit once per instantiation (and again if it grows)
+  if (smem > attr_bytes) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BETTY_ERR_CUDA;
+    attr_bytes = smem;
+  }
   kern<<<grid, LR_THREADS, smem, c.stream>>>(a);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
