@@ -94,8 +94,9 @@ betty_status vec_mul(Ctx& c, float* out, float a, const float* x, const float* y
 // *result = x.y, deterministic two-phase; records NONFINITE
 betty_status vec_dot(Ctx& c, const float* x, const float* y, int64_t n, float* result, float* partials);
 int64_t vec_dot_partials(int64_t n);
-// Neumann: t <- t - alpha*Ht ; s <- s + t
-betty_status neumann_update(Ctx& c, float* t, float* s, const float* Ht, float alpha, int64_t n);
+// Neumann: t_out = t_in - alpha*Ht ; s_out = s_in + t_out  (in-place allowed)
+betty_status neumann_update(Ctx& c, const float* t_in, const float* s_in, const float* Ht, float alpha, float* t_out,
+                            float* s_out, int64_t n);
 // CG pieces driven by a SolveState on the device
 betty_status cg_init(Ctx& c, SolveState* st, const float* v, float* q, float* r, float* p, float tol,
                      int64_t n, float* partials);

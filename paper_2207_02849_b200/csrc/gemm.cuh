@@ -18,7 +18,9 @@ enum GemmEpiMode {
   EPI_BIAS_ACT = 1,  // v = acc + bias[n];  C = v;  out16 = act(v)                       (forward layer)
   EPI_ACT_BWD = 2,   // C = acc (if C);     out16 = acc * act'(a[m,n])                   (backward through an activation)
   EPI_R_FWD = 3,     // v = acc + bias[n];  C = v;  out16 = act'(a[m,n]) * v             (R-operator forward)
-  EPI_R_BWD = 4      // out16 = acc * act'(a) + dh * act''(a) * Ra                       (R-operator backward)
+  EPI_R_BWD = 4,     // out16 = acc * act'(a) + dh * act''(a) * Ra                       (R-operator backward)
+  EPI_SGD = 5,       // g = acc + exp(lam) * w16;  C = C - lr * g;  out16 = bf16(new C)  (weight gradient -> gradient step)
+  EPI_NEUMANN = 6    // Hu = acc + exp(lam) * t_in;  t = t_in - alpha * Hu -> C;  s_out = s_in + t   (weight HVP -> series update)
 };
 struct GemmEpilogue {
   int mode;
@@ -29,6 +31,14 @@ struct GemmEpilogue {
   const float* Ra;         // [M,N]
   bf16* out16;             // [M, ld16] or null
   int64_t ld16;
+  // EPI_SGD / EPI_NEUMANN (all [M,N] with the leading dimension of C unless noted)
+  const float* lam;        // device scalar: log weight decay of this layer, or null
+  const bf16* w16;         // EPI_SGD: bf16 weights the gradient was taken at, leading dimension ldw16
+  int64_t ldw16;
+  float step;              // EPI_SGD: learning rate; EPI_NEUMANN: alpha
+  const float* t_in;       // EPI_NEUMANN: current series term (the HVP direction)
+  const float* s_in;       // EPI_NEUMANN: running sum in
+  float* s_out;            // EPI_NEUMANN: running sum out
 };
 struct GemmDesc {
   int M, N;
@@ -80,6 +90,24 @@ __device__ __forceinline__ void gemm_epilogue_store(const GemmEpilogue& e, float
       float v = acc * act_d1(e.act, e.a[j]);
       if (e.act != BETTY_ACT_RELU) v += e.dh[j] * act_d2(e.act, e.a[j]) * e.Ra[j];
       e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(v);
+      break;
+    }
+    case EPI_SGD: {
+      float gval = acc;
+      if (e.lam) gval += expf(*e.lam) * __bfloat162float(e.w16[(int64_t)m * e.ldw16 + n]);
+      const float w = *cp - e.step * gval;
+      *cp = w;
+      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(w);
+      break;
+    }
+    case EPI_NEUMANN: {
+      const int64_t jc = (int64_t)m * ldc + n;
+      const float ti = e.t_in[jc];
+      float hu = acc;
+      if (e.lam) hu += expf(*e.lam) * ti;
+      const float tn = ti - e.step * hu;
+      *cp = tn;
+      e.s_out[jc] = e.s_in[jc] + tn;
       break;
     }
   }

@@ -17,7 +17,8 @@ static constexpr int TC_BM = 128;
 static constexpr int TC_BK = 64;            // 64 bf16 = one 128-byte swizzle row
 static constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;
 static constexpr uint32_t TC_SPIN = 1u << 24;
-static constexpr int TC_THREADS = 192;      // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
+static constexpr int TC_THREADS = 320;      // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
+static constexpr int TC_EPI_WARPS = 8;      // two warps per accumulator lane quarter, each takes half of the columns
 template <int BN> struct TcCfg {
   static constexpr int B_BYTES = BN * TC_BK * 2;
   static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
@@ -142,6 +143,31 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
             for (int k = 0; k < 8; ++k) o[k] = act_d1(e.act, av[k]) * v[k];
           }
         }
+      } else if (e.mode == EPI_SGD) {
+        const float kap = e.lam ? expf(*e.lam) : 0.f;
+        const float4 c0 = *(const float4*)(crow + j8), c1 = *(const float4*)(crow + j8 + 4);
+        const float cv[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        float wv[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (e.lam) {
+          const uint4 wq = *(const uint4*)(e.w16 + (int64_t)m * e.ldw16 + nb + j8);
+          const __nv_bfloat162* wp = (const __nv_bfloat162*)&wq;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) { const float2 f = __bfloat1622float2(wp[k]); wv[2 * k] = f.x; wv[2 * k + 1] = f.y; }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { v[k] = cv[k] - e.step * (v[k] + kap * wv[k]); o[k] = v[k]; }
+      } else if (e.mode == EPI_NEUMANN) {
+        const float kap = e.lam ? expf(*e.lam) : 0.f;
+        const int64_t jc = (int64_t)m * g.ldc + nb + j8;
+        const float4 t0 = *(const float4*)(e.t_in + jc), t1 = *(const float4*)(e.t_in + jc + 4);
+        const float4 s0 = *(const float4*)(e.s_in + jc), s1 = *(const float4*)(e.s_in + jc + 4);
+        const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+        const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+        float so[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { v[k] = tv[k] - e.step * (v[k] + kap * tv[k]); so[k] = sv[k] + v[k]; }
+        *(float4*)(e.s_out + jc) = make_float4(so[0], so[1], so[2], so[3]);
+        *(float4*)(e.s_out + jc + 4) = make_float4(so[4], so[5], so[6], so[7]);
       } else {   // EPI_ACT_BWD, EPI_R_BWD
         const float4 a0 = *(const float4*)(e.a + jb + j8), a1 = *(const float4*)(e.a + jb + j8 + 4);
         const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
@@ -199,7 +225,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { tc_mbar_init(&full[s], 1); tc_mbar_init(&empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { tc_mbar_init(&acc_full[s], 1); tc_mbar_init(&acc_empty[s], 4); }
+    for (int s = 0; s < 2; ++s) { tc_mbar_init(&acc_full[s], 1); tc_mbar_init(&acc_empty[s], TC_EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -293,8 +319,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
         have = __all_sync(0xffffffffu, have);
         if (!have) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int half = (warp - 2) >> 2;           // which half of the tile's columns this warp drains
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
           if (n0 + c * 32 >= g.N) break;            // uniform: nothing to store from these columns
           uint32_t r[32];
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32);
@@ -376,7 +403,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUt
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { tc_mbar_init(&full[s], 1); tc_mbar_init(&empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { tc_mbar_init(&acc_full[s], 1); tc_mbar_init(&acc_empty[s], 8); }
+    for (int s = 0; s < 2; ++s) { tc_mbar_init(&acc_full[s], 1); tc_mbar_init(&acc_empty[s], 2 * TC_EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -467,8 +494,9 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUt
         have = __all_sync(0xffffffffu, have);
         if (!have) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int half = (warp - 2) >> 2;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
           if (n0 + c * 32 >= g.N) break;
           uint32_t r[32];
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32);
@@ -578,7 +606,8 @@ static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a) {
   auto al16 = [](const void* p) { return (((uintptr_t)p) & 15) == 0; };
   const GemmEpilogue& e = g.epi;
   const bool ok = (g.N % 4 == 0) && al16(g.C) && (g.ldc % 4 == 0) && al16(e.bias) && al16(e.a) && al16(e.dh) && al16(e.Ra) &&
-                  al16(e.out16) && (e.ld16 % 8 == 0);
+                  al16(e.out16) && (e.ld16 % 8 == 0) && al16(e.w16) && (e.ldw16 % 8 == 0) && al16(e.t_in) && al16(e.s_in) &&
+                  al16(e.s_out);
   a.vec_ok = ok ? 1 : 0;
   for (int i = 0; i < 2; ++i) {
     const GemmPair& p = g.p[i < g.npairs ? i : 0];

@@ -77,8 +77,12 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
     delta[i] = __float2bfloat16_rn(v);
   }
 }
-// out[n] = sum_i d[i, n].  Block = 32 columns x 8 row groups; fixed summation order.
-__global__ void k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, float* out) {
+// Column sums sum_i d[i, n] (bias gradients), with the consumer fused in.  Block = 32 columns x 8 row
+// groups; fixed summation order.
+//   mode 0: out[n] = sum            mode 1: out[n] -= step * sum   (gradient step on a bias)
+//   mode 2: t = t_in[n] - step * sum; out[n] = t; s_out[n] = s_in[n] + t   (Neumann-series update)
+struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; float* s_out; };
+__global__ void k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
   __shared__ float sh[8][33];
   const int cx = threadIdx.x & 31, rg = threadIdx.x >> 5;
   const int64_t n = blockIdx.x * 32 + cx;
@@ -91,7 +95,9 @@ __global__ void k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, f
     float t = 0.f;
 #pragma unroll
     for (int r = 0; r < 8; ++r) t += sh[r][cx];
-    out[n] = t;
+    if (k.mode == 0) k.out[n] = t;
+    else if (k.mode == 1) k.out[n] -= k.step * t;
+    else { const float tn = k.t_in[n] - k.step * t; k.out[n] = tn; k.s_out[n] = k.s_in[n] + tn; }
   }
 }
 // delta_prev = dh * act'(a)
@@ -153,10 +159,6 @@ __global__ void k_jvp_rows(const float* p, const int32_t* y, const float* Ra, fl
   for (int64_t c = lane; c < C; c += 32) s += (p[row * C + c] - (c == y[row] ? 1.f : 0.f)) * Ra[row * C + c];
   for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
   if (lane == 0) d[row] = s;
-}
-__global__ void k_sgd(float* x, const float* g, float lr, int64_t n) {
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
-    x[i] -= lr * g[i];
 }
 // out[r, c] += exp(lam) * W[r, c]   (out contiguous [rows, cols]; W bf16 with leading dimension ldw)
 __global__ void k_wd_add_bf16(float* out, const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* lam) {
@@ -405,9 +407,19 @@ static betty_status forward(Ctx& c, const Net& n, const betty_level* D, Pass& ps
   return BETTY_OK;
 }
 
-// Reverse sweep from delta_top = coef_i (p - onehot).  gflat (nullable): receives [gW_l, gb_l]; lam
-// (nullable): adds exp(lam_l) W_l.  Always leaves delta[l] and dh[l] in `ps` for an R-operator pass.
-static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, float* gflat, const float* lam) {
+// Where the parameter gradient of a reverse sweep goes.
+struct GradSink {
+  float* gflat;            // plain gradient [gW_l, gb_l] (null: no parameter gradient wanted)
+  const float* lam;        // device per-layer log weight decay: adds exp(lam_l) W_l (null: none)
+  bool sgd;                // instead of storing the gradient, take the step  master -= lr * grad  in the epilogue
+  float lr;
+  float* master;           // sgd: parameters to update in place
+  bf16* const* Wnext;      // sgd: per-layer bf16 copies of the updated matrices (for the next step), or null
+};
+
+// Reverse sweep from delta_top = coef_i (p - onehot).  Always leaves delta[l] (and dh[l] for smooth
+// activations) in `ps` for an R-operator pass.
+static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, const GradSink& sink) {
   const int64_t B = ps.B;
   const int64_t C = n.w[n.L];
   {
@@ -419,15 +431,25 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
   }
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
-    if (gflat) {
-      GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.npairs = 1; g.C = gflat + n.woff[l]; g.ldc = K; g.beta = 0.f;
+    if (sink.gflat || sink.sgd) {
+      GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.npairs = 1; g.ldc = K; g.beta = 0.f;
       g.p[0] = gemm_pair(ps.delta[l], ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
+      ColsumSink cs = {};
+      if (sink.sgd) {
+        g.C = sink.master + n.woff[l];
+        g.epi.mode = EPI_SGD; g.epi.lam = sink.lam ? sink.lam + l : nullptr; g.epi.w16 = n.W[l]; g.epi.ldw16 = n.ldw[l];
+        g.epi.step = sink.lr; g.epi.out16 = sink.Wnext ? sink.Wnext[l] : nullptr; g.epi.ld16 = n.ldw[l];
+        cs.mode = 1; cs.step = sink.lr; cs.out = sink.master + n.boff[l];
+      } else {
+        g.C = sink.gflat + n.woff[l];
+        cs.mode = 0; cs.out = sink.gflat + n.boff[l];
+      }
       BETTY_TRY(gemm(c, g));
-      if (lam) {
-        k_wd_add_bf16<<<grid_for(N * K), 256, 0, c.stream>>>(gflat + n.woff[l], n.W[l], N, K, n.ldw[l], lam + l);
+      if (!sink.sgd && sink.lam) {
+        k_wd_add_bf16<<<grid_for(N * K), 256, 0, c.stream>>>(sink.gflat + n.woff[l], n.W[l], N, K, n.ldw[l], sink.lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      k_colsum_bf16<<<(unsigned)((N + 31) / 32), 256, 0, c.stream>>>(ps.delta[l], B, N, ldd, gflat + n.boff[l]);
+      k_colsum_bf16<<<(unsigned)((N + 31) / 32), 256, 0, c.stream>>>(ps.delta[l], B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {
@@ -450,6 +472,9 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
     }
   }
   return BETTY_OK;
+}
+static inline GradSink grad_into(float* gflat, const float* lam) {
+  GradSink s = {}; s.gflat = gflat; s.lam = lam; return s;
 }
 
 // Directional derivative of the forward pass along `dir` (flat, same layout as the parameters).
@@ -583,12 +608,12 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
   BETTY_TRY(forward(c, n, L, ps));
   BETTY_ALLOC(s1, float, c, (size_t)(ps.B > 0 ? ps.B : 1));
   if (L->loss == BETTY_LOSS_MLP_CE) {
-    BETTY_TRY(backward(c, n, ps, nullptr, out, nullptr));
+    BETTY_TRY(backward(c, n, ps, nullptr, grad_into(out, nullptr)));
   } else if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
     if (wrt == P.mlp) {
       const float* coef;
       BETTY_TRY(reweight_coef(c, P, ps, &coef));
-      BETTY_TRY(backward(c, n, ps, coef, out, P.lam ? P.lam->params : nullptr));
+      BETTY_TRY(backward(c, n, ps, coef, grad_into(out, P.lam ? P.lam->params : nullptr)));
     } else {
       BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, ps, nullptr, nullptr, s1, nullptr));
       BETTY_TRY(wn_backward(c, P.theta, nullptr, ps, s1, nullptr, 0.f, nullptr, out));
@@ -599,7 +624,7 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
       BETTY_TRY(wn_backward(c, P.theta, nullptr, ps, s1, nullptr, L->mu, P.theta->params, out));
     } else {
       BETTY_TRY(wn_sample(c, WN_DETECT_WGRAD, P.theta, nullptr, ps, L->aux, nullptr, s1, nullptr));
-      BETTY_TRY(backward(c, n, ps, s1, out, nullptr));
+      BETTY_TRY(backward(c, n, ps, s1, grad_into(out, nullptr)));
     }
   }
   c.arena.release(mark);
@@ -617,7 +642,7 @@ betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache)
   BETTY_TRY(forward(c, h.net, L, h.pass));
   if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
     BETTY_TRY(reweight_coef(c, P, h.pass, &h.coef));
-    BETTY_TRY(backward(c, h.net, h.pass, h.coef, nullptr, nullptr));
+    BETTY_TRY(backward(c, h.net, h.pass, h.coef, grad_into(nullptr, nullptr)));
   } else if (!(L->loss == BETTY_LOSS_WEIGHTNET_DETECT && L->param_kind == BETTY_PARAM_WEIGHTNET)) {
     return BETTY_ERR_UNSUPPORTED;
   }
@@ -625,7 +650,13 @@ betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache)
   return BETTY_OK;
 }
 
-betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* u, float* Hu) {
+// Neumann-series consumer of an HVP: t_out = t_in - alpha * H t_in ; s_out = s_in + t_out
+struct SeriesSink { const float* s_in; float alpha; float* t_out; float* s_out; };
+
+// H u.  Without a sink the product is written to Hu; with one, u is the current series term t_in and
+// the update is applied inside the weight-gradient products and bias column sums (Hu is not used).
+static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* u, float* Hu,
+                             const SeriesSink* sink) {
   const size_t mark = c.arena.mark();
   const Net& n = h->net;
   Pass& ps = h->pass;
@@ -634,7 +665,10 @@ betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const floa
     BETTY_ALLOC(cA, float, c, (size_t)(B > 0 ? B : 1));
     BETTY_ALLOC(cB, float, c, (size_t)(B > 0 ? B : 1));
     BETTY_TRY(wn_sample(c, WN_DETECT_THVP, L, u, ps, L->aux, nullptr, cA, cB));
-    BETTY_TRY(wn_backward(c, L, u, ps, cA, cB, L->mu, u, Hu));
+    float* dst = Hu;
+    if (sink) { dst = c.arena.alloc<float>(512); if (!dst) return BETTY_ERR_WORKSPACE; }
+    BETTY_TRY(wn_backward(c, L, u, ps, cA, cB, L->mu, u, dst));
+    if (sink) BETTY_TRY(neumann_update(c, u, sink->s_in, dst, sink->alpha, sink->t_out, sink->s_out, WN_P));
     c.arena.release(mark);
     return BETTY_OK;
   }
@@ -653,15 +687,26 @@ betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const floa
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
     {  // R gW_l = Rdelta^T h_l + delta_l^T Rh_l + exp(lam_l) U_l
-      GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.C = Hu + n.woff[l]; g.ldc = K; g.beta = 0.f; g.npairs = 0;
+      GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.ldc = K; g.beta = 0.f; g.npairs = 0;
       g.p[g.npairs++] = gemm_pair(Rd, ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
       if (l > 0) g.p[g.npairs++] = gemm_pair(ps.delta[l], ldd, true, rp.Rh[l], ps.ldh[l], false, (int)B);
+      ColsumSink cs = {};
+      if (sink) {
+        g.C = sink->t_out + n.woff[l];
+        g.epi.mode = EPI_NEUMANN; g.epi.lam = h->lam ? h->lam + l : nullptr; g.epi.step = sink->alpha;
+        g.epi.t_in = u + n.woff[l]; g.epi.s_in = sink->s_in + n.woff[l]; g.epi.s_out = sink->s_out + n.woff[l];
+        cs.mode = 2; cs.step = sink->alpha; cs.out = sink->t_out + n.boff[l]; cs.t_in = u + n.boff[l];
+        cs.s_in = sink->s_in + n.boff[l]; cs.s_out = sink->s_out + n.boff[l];
+      } else {
+        g.C = Hu + n.woff[l];
+        cs.mode = 0; cs.out = Hu + n.boff[l];
+      }
       BETTY_TRY(gemm(c, g));
-      if (h->lam) {
+      if (!sink && h->lam) {
         k_wd_add_f32<<<grid_for(N * K), 256, 0, c.stream>>>(Hu + n.woff[l], u + n.woff[l], N * K, h->lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      k_colsum_bf16<<<(unsigned)((N + 31) / 32), 256, 0, c.stream>>>(Rd, B, N, ldd, Hu + n.boff[l]);
+      k_colsum_bf16<<<(unsigned)((N + 31) / 32), 256, 0, c.stream>>>(Rd, B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {  // R dh = Rdelta W_l + delta_l U_l ; Rdelta_{l-1} = Rdh*act' + dh*act''*Ra
@@ -679,6 +724,16 @@ betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const floa
   }
   c.arena.release(mark);
   return BETTY_OK;
+}
+
+betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* u, float* Hu) {
+  return hvp_impl(c, L, h, u, Hu, nullptr);
+}
+
+betty_status mlpfam_hvp_neumann(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* t_in, const float* s_in,
+                                float alpha, float* t_out, float* s_out) {
+  SeriesSink sink = {s_in, alpha, t_out, s_out};
+  return hvp_impl(c, L, h, t_in, nullptr, &sink);
 }
 
 betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const betty_level* wrt, const float* q,
@@ -710,7 +765,7 @@ betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const be
   } else if (L->loss == BETTY_LOSS_WEIGHTNET_DETECT && L->param_kind == BETTY_PARAM_WEIGHTNET && wrt == P.mlp) {
     BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
     BETTY_TRY(wn_sample(c, WN_DETECT_WMIXED, L, q, ps, L->aux, nullptr, s1, nullptr));
-    BETTY_TRY(backward(c, n, ps, s1, out, nullptr));
+    BETTY_TRY(backward(c, n, ps, s1, grad_into(out, nullptr)));
   } else {
     return BETTY_ERR_INVALID_ARG;
   }
@@ -720,12 +775,32 @@ betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const be
 
 betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps) {
   if (L->loss != BETTY_LOSS_MLP_CE_REWEIGHT) return BETTY_ERR_UNSUPPORTED;
+  if (n_steps <= 0) return BETTY_OK;
   const size_t mark = c.arena.mark();
-  BETTY_ALLOC(g, float, c, (size_t)L->n_params);
+  const Parts P = parts_of(L);
+  // The gradient step is taken inside the weight-gradient products' epilogues, which also write the
+  // bf16 copy of the updated matrices for the next step: one cast at the start, none afterwards.
+  Net n;
+  BETTY_TRY(net_setup(c, P.mlp, n));
+  bf16* alt[MAXL];
+  for (int l = 0; l < n.L; ++l) {
+    const size_t cnt = (size_t)(n.w[l + 1] * n.ldw[l]);
+    alt[l] = c.arena.alloc<bf16>(cnt);
+    if (!alt[l]) return BETTY_ERR_WORKSPACE;
+    if (n.ldw[l] != n.w[l]) cudaMemsetAsync(alt[l], 0, cnt * sizeof(bf16), c.stream);
+  }
   for (int s = 0; s < n_steps; ++s) {
-    BETTY_TRY(mlpfam_grad(c, L, L, g));
-    k_sgd<<<grid_for(L->n_params, 1024), 256, 0, c.stream>>>(L->params, g, L->lr, L->n_params);
-    BETTY_LAUNCH_CHECK();
+    const size_t m2 = c.arena.mark();
+    Pass ps;
+    BETTY_TRY(forward(c, n, L, ps));
+    const float* coef;
+    BETTY_TRY(reweight_coef(c, P, ps, &coef));
+    GradSink sink = {};
+    sink.lam = P.lam ? P.lam->params : nullptr;
+    sink.sgd = true; sink.lr = L->lr; sink.master = L->params; sink.Wnext = alt;
+    BETTY_TRY(backward(c, n, ps, coef, sink));
+    for (int l = 0; l < n.L; ++l) { bf16* t = n.W[l]; n.W[l] = alt[l]; alt[l] = t; }
+    c.arena.release(m2);
   }
   c.arena.release(mark);
   return BETTY_OK;

@@ -43,6 +43,10 @@ size_t mlpfam_workspace(const betty_level* L);
 betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);
 betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache);
 betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* u, float* Hu);
+// One Neumann-series iteration with the update fused into the HVP's weight-gradient products:
+// t_out = t_in - alpha * H t_in ; s_out = s_in + t_out  (t_in == t_out and s_in == s_out allowed)
+betty_status mlpfam_hvp_neumann(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* t_in, const float* s_in,
+                                float alpha, float* t_out, float* s_out);
 betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* cache, const betty_level* wrt, const float* q,
                           float* out);
 betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps);

@@ -29,11 +29,12 @@ __global__ void k_mul(float* out, float a, const float* x, const float* y, int64
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     out[i] = a * x[i] * y[i];
 }
-__global__ void k_neumann(float* t, float* s, const float* Ht, float alpha, int64_t n) {
+__global__ void k_neumann(const float* t_in, const float* s_in, const float* Ht, float alpha, float* t_out, float* s_out,
+                          int64_t n) {
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-    float tn = t[i] - alpha * Ht[i];
-    t[i] = tn;
-    s[i] += tn;
+    float tn = t_in[i] - alpha * Ht[i];
+    t_out[i] = tn;
+    s_out[i] = s_in[i] + tn;
   }
 }
 
@@ -61,9 +62,10 @@ betty_status vec_mul(Ctx& c, float* out, float a, const float* x, const float* y
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
-betty_status neumann_update(Ctx& c, float* t, float* s, const float* Ht, float alpha, int64_t n) {
+betty_status neumann_update(Ctx& c, const float* t_in, const float* s_in, const float* Ht, float alpha, float* t_out,
+                            float* s_out, int64_t n) {
   if (n <= 0) return BETTY_OK;
-  k_neumann<<<ew_blocks(n), VT, 0, c.stream>>>(t, s, Ht, alpha, n);
+  k_neumann<<<ew_blocks(n), VT, 0, c.stream>>>(t_in, s_in, Ht, alpha, t_out, s_out, n);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
