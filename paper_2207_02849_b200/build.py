@@ -11,7 +11,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libbetty.so")
-SOURCES = ["api.cu", "vec.cu", "logreg.cu", "mlp.cu", "gemm.cu", "gemm_tc.cu"]
+SOURCES = ["api.cu", "vec.cu", "logreg.cu", "logreg_small.cu", "mlp.cu", "gemm.cu", "gemm_tc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--use_fast_math", "-Xcompiler", "-fPIC",

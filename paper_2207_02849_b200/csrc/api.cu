@@ -90,6 +90,9 @@ betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, 
 betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps) {
   if (!vec_has_wd(L)) return BETTY_ERR_UNSUPPORTED;
   const float* lam = find_constraint(L, BETTY_PARAM_VECTOR)->params;
+  if (n_steps > 1 && logreg_small_eligible(L->n, 0, L->d))   // all steps in one launch, data resident on chip
+    return logreg_small_lower_step(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, lam,
+                                   n_steps, L->lr);
   for (int s = 0; s < n_steps; ++s)
     BETTY_TRY(logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, nullptr, lam,
                           nullptr, L->params, L->lr));
@@ -202,6 +205,13 @@ static betty_status hypergrad(const betty_level* lower, const betty_level* upper
   if (!is_participant(upper, lower) || !is_participant(upper, wrt) || !is_participant(lower, wrt) || wrt == lower)
     return BETTY_ERR_INVALID_ARG;
   Ctx c(ws, ws_bytes, stream);
+  // Small logistic / least-squares bilevel pair: the whole hypergradient in one launch.
+  if (vec_has_wd(lower) && (upper->loss == BETTY_LOSS_LOGREG || upper->loss == BETTY_LOSS_QUADRATIC) &&
+      find_constraint(upper, BETTY_PARAM_VECTOR) == lower && wrt == find_constraint(lower, BETTY_PARAM_VECTOR) &&
+      cfg.K >= 0 && logreg_small_eligible(lower->n, upper->n, lower->d))
+    return logreg_small_hypergrad(c, vec_family(lower), (const float*)lower->X, (const float*)lower->y, lower->n,
+                                  vec_family(upper), (const float*)upper->X, (const float*)upper->y, upper->n, lower->d,
+                                  lower->params, wrt->params, cfg, out);
   BETTY_ALLOC(v, float, c, (size_t)lower->n_params);
   BETTY_TRY(level_grad(c, upper, lower, v));     // dC_u / d theta_lower
   BETTY_TRY(level_grad(c, upper, wrt, out));     // direct gradient

@@ -1,0 +1,297 @@
+// Small-problem variant of the logistic / least-squares family (App. D.1 problem at a size where the
+// whole data set fits on chip): one launch runs a complete loop -- all unrolled lower-level gradient
+// steps, or a complete hypergradient (validation gradient, Neumann / CG / finite-difference solve,
+// mixed product).  A cluster of 8 CTAs keeps the rows of X (and of the validation matrix) resident
+// in shared memory for the whole launch; in every pass each CTA pushes its column sums into all
+// eight CTAs through distributed shared memory, one cluster barrier follows, and every CTA then repeats the same O(d)
+// vector arithmetic on its own copy of the solver state, in the same order, so all copies stay
+// bit-identical.  At this size the path is bound by the latency of ~100 dependent passes, not by
+// bandwidth: the point of the kernel is to pay one launch instead of hundreds.
+#include "ops.cuh"
+
+namespace betty {
+
+static constexpr int SM_CL = 8;          // CTAs per cluster
+static constexpr int SM_T = 256;         // threads per CTA
+static constexpr int SM_MAXD = 256;
+static constexpr int SM_NVEC = 10;       // vectors of length d kept per CTA
+
+struct SmallArgs {
+  const float* X; const float* y; int64_t n;       // lower problem data
+  const float* Xv; const float* yv; int64_t nv;    // upper problem data (hypergradient mode)
+  int d;
+  int family, family_up;                            // 0 logistic, 1 least squares
+  float* w;                                         // lower parameters (updated in lower-step mode)
+  const float* lam;
+  int mode;                                         // 0: lower steps; 1: hypergradient
+  int n_steps; float lr;
+  int method, K; float alpha, eps0, tol;            // betty_method and its parameters
+  float* out;                                       // hypergradient [d] (added to nothing: direct gradient is zero)
+  int rows_per_cta, rows_per_cta_v;
+  StatusBlock* sb;
+};
+
+__device__ __forceinline__ uint32_t sm_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void st_remote(float* local_ptr, uint32_t rank, float v) {
+  uint32_t a;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(sm_u32(local_ptr)), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float sigm(float t) { return 1.f / (1.f + expf(-t)); }
+
+// block-wide sum of one value per thread (fixed order)
+__device__ __forceinline__ float block_sum_f(float v, float* sh) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int i = 0; i < SM_T / 32; ++i) t += sh[i];
+  __syncthreads();
+  return t;
+}
+__device__ __forceinline__ float vdot(const float* a, const float* b, int d, float* sh) {
+  float v = 0.f;
+  for (int j = threadIdx.x; j < d; j += SM_T) v += a[j] * b[j];
+  return block_sum_f(v, sh);
+}
+
+// One pass over this CTA's resident rows: coef_i from the row dot products, then the column sums
+// sum_i coef_i x_ij, reduced over the cluster into res[0..d) (identical in every CTA).
+//   kind 0: gradient coefficients at `wv`;  kind 1: HVP coefficients curv_i * (x_i . dir)
+__device__ void pass(const float* Xs, const float* ys, const float* curv, int rows, int d, int family, float inv_n,
+                     int kind, const float* wv, const float* dir, float* coef, float* part, float* cpart, float* res,
+                     uint32_t rank) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // A: one warp per row, four rows in flight per warp so that the shuffle chains overlap
+  const float* vv = kind == 0 ? wv : dir;
+  for (int i0 = warp * 4; i0 < rows; i0 += (SM_T / 32) * 4) {
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u;
+      if (i < rows) {
+        const float* xr = Xs + (size_t)i * d;
+        for (int j = lane; j < d; j += 32) s[u] += xr[j] * vv[j];
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
+    }
+    if (lane < 4 && i0 + lane < rows) {
+      const int i = i0 + lane;
+      const float sv = lane == 0 ? s[0] : (lane == 1 ? s[1] : (lane == 2 ? s[2] : s[3]));
+      float cf;
+      if (kind == 0) cf = family == 0 ? -ys[i] * sigm(-ys[i] * sv) * inv_n : (sv - ys[i]);
+      else cf = curv[i] * sv;
+      coef[i] = cf;
+    }
+  }
+  __syncthreads();
+  // B: thread per column (x row groups), then fold the row groups
+  const int ct = d <= 32 ? 32 : (d <= 64 ? 64 : (d <= 128 ? 128 : 256));
+  const int groups = SM_T / ct, c0 = tid % ct, rg = tid / ct;
+  for (int j = c0; j < d; j += ct) {
+    float a = 0.f;
+    for (int i = rg; i < rows; i += groups) a += coef[i] * Xs[(size_t)i * d + j];
+    part[rg * SM_MAXD + j] = a;
+  }
+  __syncthreads();
+  // fold the row groups and push this CTA's column sums into slot `rank` of every CTA of the cluster
+  for (int j = tid; j < d; j += SM_T) {
+    float a = 0.f;
+    for (int g2 = 0; g2 < groups; ++g2) a += part[g2 * SM_MAXD + j];
+#pragma unroll
+    for (uint32_t r = 0; r < SM_CL; ++r) st_remote(cpart + rank * SM_MAXD + j, r, a);
+  }
+  cluster_barrier();                       // all pushes have landed everywhere
+  for (int j = tid; j < d; j += SM_T) {
+    float a = 0.f;
+#pragma unroll
+    for (int r = 0; r < SM_CL; ++r) a += cpart[r * SM_MAXD + j];
+    res[j] = a;
+  }
+  __syncthreads();
+  (void)rank;
+}
+
+__global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logreg_small(SmallArgs a) {
+  extern __shared__ __align__(16) float sm[];
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const int d = a.d, tid = threadIdx.x;
+  const int R = a.rows_per_cta, Rv = a.rows_per_cta_v;
+  float* Xs = sm;                                  // [R, d]
+  float* Xvs = Xs + (size_t)R * d;                 // [Rv, d]
+  float* ys = Xvs + (size_t)Rv * d;                // [R]
+  float* yvs = ys + R;                             // [Rv]
+  float* curv = yvs + Rv;                          // [R]  sigmoid(z) sigmoid(-z) / n at the current w
+  float* coef = curv + R;                          // [max(R, Rv)]
+  float* vec = coef + (R > Rv ? R : Rv);           // SM_NVEC vectors of SM_MAXD
+  float* part = vec + SM_NVEC * SM_MAXD;           // [8][SM_MAXD] row-group partials
+  float* cpart = part + 8 * SM_MAXD;               // [2][SM_CL][SM_MAXD] column sums of every CTA (double-buffered)
+  float* red = cpart + 2 * SM_CL * SM_MAXD;                // [8] block reduction scratch
+  float *w = vec, *lam = vec + SM_MAXD, *g = vec + 2 * SM_MAXD, *v = vec + 3 * SM_MAXD, *q = vec + 4 * SM_MAXD,
+        *r = vec + 5 * SM_MAXD, *p = vec + 6 * SM_MAXD, *h = vec + 7 * SM_MAXD, *t = vec + 8 * SM_MAXD;
+
+  // resident rows of this CTA
+  const int64_t r0 = (int64_t)rank * R, r0v = (int64_t)rank * Rv;
+  int rows = (int)(a.n - r0 < R ? a.n - r0 : R); if (rows < 0) rows = 0;
+  int rowsv = (int)(a.nv - r0v < Rv ? a.nv - r0v : Rv); if (rowsv < 0) rowsv = 0;
+  for (int64_t i = tid; i < (int64_t)rows * d; i += SM_T) Xs[i] = a.X[r0 * d + i];
+  for (int i = tid; i < rows; i += SM_T) ys[i] = a.y[r0 + i];
+  if (a.mode == 1) {
+    for (int64_t i = tid; i < (int64_t)rowsv * d; i += SM_T) Xvs[i] = a.Xv[r0v * d + i];
+    for (int i = tid; i < rowsv; i += SM_T) yvs[i] = a.yv[r0v + i];
+  }
+  for (int j = tid; j < d; j += SM_T) { w[j] = a.w[j]; lam[j] = a.lam[j]; }
+  cluster_barrier();    // every CTA of the cluster is running before anyone touches a neighbour's shared memory
+  const float inv_n = a.n > 0 ? 1.f / (float)a.n : 0.f, inv_nv = a.nv > 0 ? 1.f / (float)a.nv : 0.f;
+  int pb = 0;   // which half of cpart this pass writes
+
+  if (a.mode == 0) {
+    for (int s = 0; s < a.n_steps; ++s) {
+      pass(Xs, ys, nullptr, rows, d, a.family, inv_n, 0, w, nullptr, coef, part, cpart + pb * SM_CL * SM_MAXD, g, rank);
+      pb ^= 1;
+      for (int j = tid; j < d; j += SM_T) w[j] -= a.lr * (g[j] + lam[j] * w[j]);
+      __syncthreads();
+    }
+    if (rank == 0)
+      for (int j = tid; j < d; j += SM_T) a.w[j] = w[j];
+  } else {
+    // v = dC_upper/dw on the validation rows
+    pass(Xvs, yvs, nullptr, rowsv, d, a.family_up, inv_nv, 0, w, nullptr, coef, part, cpart + pb * SM_CL * SM_MAXD, v, rank);
+    pb ^= 1;
+    if (a.method == BETTY_FD) {
+      // dC/d(lambda) = 1/2 w^2: the central difference at w +- eps v, evaluated as written
+      const float nv2 = vdot(v, v, d, red);
+      for (int j = tid; j < d; j += SM_T) {
+        float o = 0.f;
+        if (nv2 > 0.f) {
+          const double eps = (double)a.eps0 / sqrt((double)nv2);
+          const double wp = (double)w[j] + eps * (double)v[j], wm = (double)w[j] - eps * (double)v[j];
+          o = (float)(-(double)a.alpha * (0.5 * wp * wp - 0.5 * wm * wm) / (2.0 * eps));
+        }
+        if (rank == 0) a.out[j] = o;
+      }
+    } else {
+      // curvature weights at the current w (constant over the solve)
+      for (int i = tid >> 5; i < rows; i += SM_T / 32) {
+        const float* xr = Xs + (size_t)i * d;
+        float s = 0.f;
+        for (int j = tid & 31; j < d; j += 32) s += xr[j] * w[j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if ((tid & 31) == 0) { const float sg = sigm(s); curv[i] = a.family == 0 ? sg * (1.f - sg) * inv_n : 1.f; }
+      }
+      __syncthreads();
+      float qscale = 1.f;
+      if (a.method == BETTY_NEUMANN) {
+        for (int j = tid; j < d; j += SM_T) { t[j] = v[j]; q[j] = v[j]; }
+        __syncthreads();
+        for (int k = 0; k < a.K; ++k) {
+          pass(Xs, ys, curv, rows, d, a.family, inv_n, 1, w, t, coef, part, cpart + pb * SM_CL * SM_MAXD, h, rank);
+          pb ^= 1;
+          for (int j = tid; j < d; j += SM_T) {
+            const float tn = t[j] - a.alpha * (h[j] + lam[j] * t[j]);
+            t[j] = tn; q[j] += tn;
+          }
+          __syncthreads();
+        }
+        qscale = a.alpha;
+      } else {
+        // conjugate gradient on H q = v, same recurrences and stopping rules as the large-problem path
+        for (int j = tid; j < d; j += SM_T) { q[j] = 0.f; r[j] = v[j]; p[j] = v[j]; }
+        __syncthreads();
+        float rho = vdot(r, r, d, red);
+        const float stop = a.tol * a.tol * rho;
+        int iters = 0, status = 0;
+        bool active = rho > stop;
+        if (!isfinite(rho)) { status = BETTY_ERR_NONFINITE; active = false; }
+        for (int k = 0; k < a.K && active; ++k) {
+          pass(Xs, ys, curv, rows, d, a.family, inv_n, 1, w, p, coef, part, cpart + pb * SM_CL * SM_MAXD, h, rank);
+          pb ^= 1;
+          for (int j = tid; j < d; j += SM_T) h[j] += lam[j] * p[j];
+          __syncthreads();
+          const float gamma = vdot(p, h, d, red);
+          if (!isfinite(gamma)) { status = BETTY_ERR_NONFINITE; break; }
+          if (!(gamma > 0.f)) { status = BETTY_ERR_BREAKDOWN; break; }
+          const float al = rho / gamma;
+          for (int j = tid; j < d; j += SM_T) { q[j] += al * p[j]; r[j] -= al * h[j]; }
+          __syncthreads();
+          const float rho_new = vdot(r, r, d, red);
+          const float beta = rho_new / rho;
+          for (int j = tid; j < d; j += SM_T) p[j] = r[j] + beta * p[j];
+          __syncthreads();
+          rho = rho_new;
+          ++iters;
+          if (!isfinite(rho)) { status = BETTY_ERR_NONFINITE; break; }
+          if (rho <= stop) break;
+        }
+        if (rank == 0 && tid == 0) {
+          a.sb->cg_iters = iters;
+          if (status) record_status(a.sb, status);
+        }
+      }
+      // out = -(w .* q) * qscale   (mixed second derivative of the weight-decay term)
+      if (rank == 0)
+        for (int j = tid; j < d; j += SM_T) a.out[j] = -qscale * w[j] * q[j];
+    }
+  }
+  // no CTA may leave while a neighbour can still read its column sums
+  cluster_barrier();
+}
+
+static size_t small_smem_bytes(int R, int Rv, int d) {
+  size_t floats = (size_t)R * d + (size_t)Rv * d + R + Rv + R + (R > Rv ? R : Rv) + (size_t)SM_NVEC * SM_MAXD + 8 * SM_MAXD +
+                  2 * SM_CL * SM_MAXD + 8;
+  return floats * sizeof(float) + 16;
+}
+
+// True when the whole problem fits the cluster's shared memory.
+bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d) {
+  if (d <= 0 || d > SM_MAXD || n <= 0 || n > (1 << 20) || nv < 0 || nv > (1 << 20)) return false;
+  const int R = (int)((n + SM_CL - 1) / SM_CL), Rv = (int)((nv + SM_CL - 1) / SM_CL);
+  return small_smem_bytes(R, Rv, (int)d) <= 200 * 1024;
+}
+
+static betty_status launch_small(Ctx& c, SmallArgs& a) {
+  a.rows_per_cta = (int)((a.n + SM_CL - 1) / SM_CL);
+  a.rows_per_cta_v = a.mode == 1 ? (int)((a.nv + SM_CL - 1) / SM_CL) : 0;
+  a.sb = c.arena.status();
+  const size_t smem = small_smem_bytes(a.rows_per_cta, a.rows_per_cta_v, a.d);
+  static size_t attr_bytes = 0;
+  if (smem > attr_bytes) {
+    if (cudaFuncSetAttribute(k_logreg_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BETTY_ERR_CUDA;
+    attr_bytes = smem;
+  }
+  k_logreg_small<<<SM_CL, SM_T, smem, c.stream>>>(a);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
+betty_status logreg_small_lower_step(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, float* w,
+                                     const float* lam, int n_steps, float lr) {
+  SmallArgs a = {};
+  a.X = X; a.y = y; a.n = n; a.d = (int)d; a.family = family; a.w = w; a.lam = lam; a.mode = 0; a.n_steps = n_steps; a.lr = lr;
+  return launch_small(c, a);
+}
+
+betty_status logreg_small_hypergrad(Ctx& c, int family, const float* X, const float* y, int64_t n, int family_up,
+                                    const float* Xv, const float* yv, int64_t nv, int64_t d, float* w, const float* lam,
+                                    const betty_method_cfg& cfg, float* out) {
+  SmallArgs a = {};
+  a.X = X; a.y = y; a.n = n; a.Xv = Xv; a.yv = yv; a.nv = nv; a.d = (int)d; a.family = family; a.family_up = family_up;
+  a.w = w; a.lam = lam; a.mode = 1; a.method = cfg.method; a.K = cfg.K; a.alpha = cfg.alpha; a.eps0 = cfg.eps0; a.tol = cfg.tol;
+  a.out = out;
+  return launch_small(c, a);
+}
+
+}  // namespace betty

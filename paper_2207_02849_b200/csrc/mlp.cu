@@ -82,22 +82,31 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
 //   mode 0: out[n] = sum            mode 1: out[n] -= step * sum   (gradient step on a bias)
 //   mode 2: t = t_in[n] - step * sum; out[n] = t; s_out[n] = s_in[n] + t   (Neumann-series update)
 struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; float* s_out; };
-__global__ void k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
-  __shared__ float sh[8][33];
+__global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
+  // 1024 threads: 32 lanes x 2 adjacent columns, 32 row groups; ld is even, so a column pair is one 4-byte load
+  __shared__ float sh[32][65];
   const int cx = threadIdx.x & 31, rg = threadIdx.x >> 5;
-  const int64_t n = blockIdx.x * 32 + cx;
-  float acc = 0.f;
-  if (n < N)
-    for (int64_t i = rg; i < B; i += 8) acc += __bfloat162float(d[i * ld + n]);
-  sh[rg][cx] = acc;
+  const int64_t n = blockIdx.x * 64 + 2 * cx;
+  float a0 = 0.f, a1 = 0.f;
+  if (n < N) {
+#pragma unroll 4
+    for (int64_t i = rg; i < B; i += 32) {
+      const float2 f = __bfloat1622float2(*(const __nv_bfloat162*)(d + i * ld + n));
+      a0 += f.x; a1 += f.y;
+    }
+  }
+  sh[rg][2 * cx] = a0; sh[rg][2 * cx + 1] = a1;
   __syncthreads();
-  if (rg == 0 && n < N) {
-    float t = 0.f;
+  if (threadIdx.x < 64) {
+    const int64_t nn = blockIdx.x * 64 + threadIdx.x;
+    if (nn < N) {
+      float t = 0.f;
 #pragma unroll
-    for (int r = 0; r < 8; ++r) t += sh[r][cx];
-    if (k.mode == 0) k.out[n] = t;
-    else if (k.mode == 1) k.out[n] -= k.step * t;
-    else { const float tn = k.t_in[n] - k.step * t; k.out[n] = tn; k.s_out[n] = k.s_in[n] + tn; }
+      for (int r = 0; r < 32; ++r) t += sh[r][threadIdx.x];
+      if (k.mode == 0) k.out[nn] = t;
+      else if (k.mode == 1) k.out[nn] -= k.step * t;
+      else { const float tn = k.t_in[nn] - k.step * t; k.out[nn] = tn; k.s_out[nn] = k.s_in[nn] + tn; }
+    }
   }
 }
 // delta_prev = dh * act'(a)
@@ -449,7 +458,7 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
         k_wd_add_bf16<<<grid_for(N * K), 256, 0, c.stream>>>(sink.gflat + n.woff[l], n.W[l], N, K, n.ldw[l], sink.lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      k_colsum_bf16<<<(unsigned)((N + 31) / 32), 256, 0, c.stream>>>(ps.delta[l], B, N, ldd, cs);
+      k_colsum_bf16<<<(unsigned)((N + 63) / 64), 1024, 0, c.stream>>>(ps.delta[l], B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {
@@ -706,7 +715,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
         k_wd_add_f32<<<grid_for(N * K), 256, 0, c.stream>>>(Hu + n.woff[l], u + n.woff[l], N * K, h->lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      k_colsum_bf16<<<(unsigned)((N + 31) / 32), 256, 0, c.stream>>>(Rd, B, N, ldd, cs);
+      k_colsum_bf16<<<(unsigned)((N + 63) / 64), 1024, 0, c.stream>>>(Rd, B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {  // R dh = Rdelta W_l + delta_l U_l ; Rdelta_{l-1} = Rdh*act' + dh*act''*Ra

@@ -26,6 +26,14 @@ static inline bool is_mlp_family(int loss) {
 betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
                          const float* u, const float* lam, float* out, float* w_update, float lr);
 
+// logreg_small.cu: whole-loop kernels for problems that fit a cluster's shared memory
+bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d);
+betty_status logreg_small_lower_step(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, float* w,
+                                     const float* lam, int n_steps, float lr);
+betty_status logreg_small_hypergrad(Ctx& c, int family, const float* X, const float* y, int64_t n, int family_up,
+                                    const float* Xv, const float* yv, int64_t nv, int64_t d, float* w, const float* lam,
+                                    const betty_method_cfg& cfg, float* out);
+
 // ---- vector families (api.cu) ----
 betty_status vecfam_validate(const betty_level* L);
 betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);

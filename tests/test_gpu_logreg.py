@@ -93,6 +93,36 @@ def test_hypergradients_match_oracle(bt, n, d, nv, steps, K):
     assert cb.rel_l2(out, ref) < TOL
 
 
+@pytest.mark.parametrize("n,d,nv", [(5, 8, 3), (1000, 50, 77), (777, 256, 100), (64, 33, 9), (2048, 128, 512)])
+def test_on_chip_whole_loop_kernel_matches_oracle(bt, n, d, nv):
+    """Problems that fit a cluster's shared memory run each loop (all lower steps; a whole
+    hypergradient) in one launch; ragged row counts, CTAs without rows and odd widths included."""
+    from tests import cuda_build as cb
+    inp = si.logreg_bilevel(900 + n + d, n, d, nv)
+    inp.lam = (np.abs(si.normal_f32(11, 2, (d,))) * 0.05 + 0.01).astype(np.float32)
+    (w, lam), (ow, olam) = _pair(inp)
+    ws = bt.Workspace([w, lam])
+    l0 = bt.betty_kernel_launches()
+    bt.betty_lower_step(w, 30, ws)
+    assert bt.betty_kernel_launches() - l0 == 1
+    oracle.lower_step(ow, 30)
+    assert cb.rel_l2(w.params, ow.params) < TOL
+    out = _vec(d)
+    for name, call, ref in [
+        ("neumann", lambda: bt.betty_hypergrad_neumann(w, lam, lam, 7, 0.05, out, ws),
+         lambda: oracle.hypergrad_neumann(ow, olam, olam, 7, 0.05)),
+        ("cg", lambda: bt.betty_hypergrad_cg(w, lam, lam, min(d, 6), 0.0, out, ws),
+         lambda: oracle.hypergrad_cg(ow, olam, olam, min(d, 6), 0.0)),
+        ("fd", lambda: bt.betty_hypergrad_fd(w, lam, lam, 0.01, 0.5, out, ws),
+         lambda: oracle.hypergrad_fd(ow, olam, olam, 0.01, 0.5)),
+    ]:
+        l0 = bt.betty_kernel_launches()
+        call()
+        assert bt.betty_kernel_launches() - l0 == 1, name
+        assert cb.rel_l2(out, ref()) < TOL, name
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
 def test_cg_early_stop_counts_iterations_like_the_oracle(bt):
     from tests import cuda_build as cb
     inp = si.logreg_bilevel(5, 400, 16, 100)
