@@ -12,7 +12,7 @@
 namespace betty {
 
 static constexpr int SM_CL = 8;          // CTAs per cluster
-static constexpr int SM_T = 256;         // threads per CTA
+static constexpr int SM_T = 1024;        // threads per CTA: the passes are latency chains, many warps hide them
 static constexpr int SM_MAXD = 256;
 static constexpr int SM_NVEC = 10;       // vectors of length d kept per CTA
 
@@ -96,7 +96,7 @@ __device__ void pass(const float* Xs, const float* ys, const float* curv, int ro
   }
   __syncthreads();
   // B: thread per column (x row groups), then fold the row groups
-  const int ct = d <= 32 ? 32 : (d <= 64 ? 64 : (d <= 128 ? 128 : 256));
+  const int ct = d <= 32 ? 32 : (d <= 64 ? 64 : (d <= 128 ? 128 : 256));   // SM_T / ct row groups, at most 32
   const int groups = SM_T / ct, c0 = tid % ct, rg = tid / ct;
   for (int j = c0; j < d; j += ct) {
     float a = 0.f;
@@ -135,9 +135,9 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   float* curv = yvs + Rv;                          // [R]  sigmoid(z) sigmoid(-z) / n at the current w
   float* coef = curv + R;                          // [max(R, Rv)]
   float* vec = coef + (R > Rv ? R : Rv);           // SM_NVEC vectors of SM_MAXD
-  float* part = vec + SM_NVEC * SM_MAXD;           // [8][SM_MAXD] row-group partials
-  float* cpart = part + 8 * SM_MAXD;               // [2][SM_CL][SM_MAXD] column sums of every CTA (double-buffered)
-  float* red = cpart + 2 * SM_CL * SM_MAXD;                // [8] block reduction scratch
+  float* part = vec + SM_NVEC * SM_MAXD;           // [32][SM_MAXD] row-group partials
+  float* cpart = part + 32 * SM_MAXD;              // [2][SM_CL][SM_MAXD] column sums of every CTA (double-buffered)
+  float* red = cpart + 2 * SM_CL * SM_MAXD;                // [32] block reduction scratch
   float *w = vec, *lam = vec + SM_MAXD, *g = vec + 2 * SM_MAXD, *v = vec + 3 * SM_MAXD, *q = vec + 4 * SM_MAXD,
         *r = vec + 5 * SM_MAXD, *p = vec + 6 * SM_MAXD, *h = vec + 7 * SM_MAXD, *t = vec + 8 * SM_MAXD;
 
@@ -250,8 +250,8 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
 }
 
 static size_t small_smem_bytes(int R, int Rv, int d) {
-  size_t floats = (size_t)R * d + (size_t)Rv * d + R + Rv + R + (R > Rv ? R : Rv) + (size_t)SM_NVEC * SM_MAXD + 8 * SM_MAXD +
-                  2 * SM_CL * SM_MAXD + 8;
+  size_t floats = (size_t)R * d + (size_t)Rv * d + R + Rv + R + (R > Rv ? R : Rv) + (size_t)SM_NVEC * SM_MAXD + 32 * SM_MAXD +
+                  2 * SM_CL * SM_MAXD + 32;
   return floats * sizeof(float) + 16;
 }
 
@@ -259,7 +259,7 @@ static size_t small_smem_bytes(int R, int Rv, int d) {
 bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d) {
   if (d <= 0 || d > SM_MAXD || n <= 0 || n > (1 << 20) || nv < 0 || nv > (1 << 20)) return false;
   const int R = (int)((n + SM_CL - 1) / SM_CL), Rv = (int)((nv + SM_CL - 1) / SM_CL);
-  return small_smem_bytes(R, Rv, (int)d) <= 200 * 1024;
+  return small_smem_bytes(R, Rv, (int)d) <= 225 * 1024;
 }
 
 static betty_status launch_small(Ctx& c, SmallArgs& a) {
