@@ -646,6 +646,9 @@ betty_status gemm_tc_pair(Ctx& c, const GemmDesc& g) { return launch_tc2(c, g); 
 
 betty_status gemm_tc(Ctx& c, const GemmDesc& g) {
   // wide tiles unless the problem is narrow or would leave most SMs without a tile
+  // many tiles per SM (weight-gradient shapes): the two-SM kernel halves the B traffic per SM and measured faster
+  const int pair_tiles = ((g.N + TC2_BN - 1) / TC2_BN) * ((g.M + 2 * TC_BM - 1) / (2 * TC_BM));
+  if (pair_tiles >= 2 * (c.sm_count / 2)) return launch_tc2(c, g);
   const int tiles256 = ((g.N + 255) / 256) * ((g.M + TC_BM - 1) / TC_BM);
   if (g.N > 128 && tiles256 >= 96) return launch_tc<256>(c, g);
   return launch_tc<128>(c, g);
