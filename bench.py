@@ -127,11 +127,15 @@ class LogregWorkload:
         self.w, self.lam = cb.logreg_levels(self.inp)
         self.w0 = self.w.params.clone()
         self.out = torch.empty(self.d, dtype=torch.float32, device="cuda")
-        self.ws = bt.Workspace([self.w, self.lam])
+        extra = (self.inp.lower_steps + 1) * (self.d + 64) * 4 if self.method == "itd" else 0
+        self.ws = bt.Workspace([self.w, self.lam], extra_bytes=extra)
 
     def step(self):
         bt = self.bt
         self.w.params.copy_(self.w0)
+        if self.method == "itd":      # the unrolled steps are part of the call
+            bt.betty_hypergrad_itd(self.w, self.lam, self.lam, self.inp.lower_steps, self.out, self.ws)
+            return
         bt.betty_lower_step(self.w, self.inp.lower_steps, self.ws)
         if self.method == "cg":
             bt.betty_hypergrad_cg(self.w, self.lam, self.lam, self.inp.K, 0.0, self.out, self.ws)
@@ -187,8 +191,13 @@ class LogregWorkload:
         inp.X, inp.y, inp.Xv, inp.yv = self.inp.X[:n_s], self.inp.y[:n_s], self.inp.Xv[:nv_s], self.inp.yv[:nv_s]
         ow, olam = ob.logreg_levels(inp)
         t0 = time.perf_counter()
-        oracle.lower_step(ow, inp.lower_steps)
-        if self.method == "cg":
+        if self.method == "itd":
+            oracle.hypergrad_itd(ow, olam, olam, inp.lower_steps)
+        else:
+            oracle.lower_step(ow, inp.lower_steps)
+        if self.method == "itd":
+            pass
+        elif self.method == "cg":
             oracle.hypergrad_cg(ow, olam, olam, inp.K, 0.0)
         elif self.method == "neumann":
             oracle.hypergrad_neumann(ow, olam, olam, inp.K, inp.alpha)
@@ -211,7 +220,7 @@ class ReweightWorkload:
         self.B = self.inp.train.X.shape[0]
         self.name = (f"config{cfg}: data reweighting, MLP {'x'.join(map(str, w)) if len(w) < 5 else f'{w[0]}->{len(w)-2}x{w[1]}->{w[-1]}'} "
                      f"{self.inp.activation} bf16/fp32-acc, batch {self.B}, {self.inp.lower_steps} lower SGD step(s), "
-                     f"{self.method}" + (f" K={self.inp.K}" if self.method != "fd" else " eps0=0.01"))
+                     f"{self.method}" + (f" K={self.inp.K}" if self.method in ("neumann", "cg") else (" eps0=0.01" if self.method == "fd" else "")))
         self.dtype = "bf16"
 
     def setup_device(self):
@@ -222,11 +231,15 @@ class ReweightWorkload:
         self.w, self.th = cb.reweight_levels(self.inp)
         self.w0 = self.w.params.clone()
         self.out = torch.empty(self.th.params.numel(), dtype=torch.float32, device="cuda")
-        self.ws = bt.Workspace([self.w, self.th])
+        extra = (self.inp.lower_steps + 1) * (self.inp.w.size + 64) * 4 if self.method == "itd" else 0
+        self.ws = bt.Workspace([self.w, self.th], extra_bytes=extra)
 
     def step(self):
         bt = self.bt
         self.w.params.copy_(self.w0)
+        if self.method == "itd":
+            bt.betty_hypergrad_itd(self.w, self.th, self.th, self.inp.lower_steps, self.out, self.ws)
+            return
         bt.betty_lower_step(self.w, self.inp.lower_steps, self.ws)
         if self.method == "fd":
             bt.betty_hypergrad_fd(self.w, self.th, self.th, self.inp.eps0, self.inp.fd_alpha, self.out, self.ws)
@@ -282,8 +295,13 @@ class ReweightWorkload:
         inp.train, inp.val = cut(self.inp.train), cut(self.inp.val)
         ow, oth = ob.reweight_levels(inp)
         t0 = time.perf_counter()
-        oracle.lower_step(ow, inp.lower_steps)
-        if self.method == "fd":
+        if self.method == "itd":
+            oracle.hypergrad_itd(ow, oth, oth, inp.lower_steps)
+        else:
+            oracle.lower_step(ow, inp.lower_steps)
+        if self.method == "itd":
+            pass
+        elif self.method == "fd":
             oracle.hypergrad_fd(ow, oth, oth, inp.eps0, inp.fd_alpha)
         elif self.method == "neumann":
             oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)
@@ -438,7 +456,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--config", type=int, default=2)
-    ap.add_argument("--method", default="")
+    ap.add_argument("--method", default="", choices=["", "cg", "neumann", "fd", "itd"])
     ap.add_argument("--scale", type=float, default=1.0, help="row-count scale of config 2 (tests/profiling only)")
     ap.add_argument("--oracle-rows", type=int, default=131072)
     ap.add_argument("--graph", type=int, default=-1,

@@ -172,6 +172,16 @@ betty_status betty_hypergrad_fd(const betty_level* lower, const betty_level* upp
                                 const betty_level* wrt, float eps0, float alpha, float* out,
                                 void* ws, size_t ws_bytes, void* stream);
 
+/* Iterative differentiation with reverse-mode autodiff (ITD-RMAD, Sec. 3.2; the method of the original
+ * Meta-Weight-Net in Sec. 5.1): takes n_steps unrolled lower steps from the current lower parameters
+ * (they are left at the last iterate, the earlier ones are kept in ws), then differentiates the
+ * upper cost through those steps in reverse:  a = dC_upper/d(lower) at the last iterate; for
+ * t = T-1..0: out -= lr * M_t^T a, a -= lr * H_t a.  out[wrt->n_params] also receives the direct
+ * gradient.  ws must hold n_steps parameter vectors in addition to betty_workspace_size(). */
+betty_status betty_hypergrad_itd(const betty_level* lower, const betty_level* upper,
+                                 const betty_level* wrt, int32_t n_steps, float* out, void* ws,
+                                 size_t ws_bytes, void* stream);
+
 /* One path term of Eq. 2, evaluated right to left (Sec. 3.2).  path = [k, q(1), ..., q(m)] indexes
  * `levels`; q(1) is reached from k by the upper-to-lower edge, q(i+1) from q(i) by lower-to-upper
  * edges; per_edge[i] configures the edge into q(i+1) (per_edge[0]: the upper-to-lower edge).

@@ -26,6 +26,6 @@ parity is "parity unpinned" by the paper and pinned only by their mathematical d
 """
 from .levels import Level  # noqa: F401
 from .solvers import (  # noqa: F401
-    brj, cg_solve, chain_levels, grad, hvp, hypergrad_cg, hypergrad_fd, hypergrad_neumann,
+    brj, cg_solve, chain_levels, grad, hvp, hypergrad_cg, hypergrad_fd, hypergrad_itd, hypergrad_neumann,
     lower_step, mixed_vjp, neumann_solve,
 )

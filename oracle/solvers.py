@@ -120,6 +120,29 @@ def hypergrad_fd(lower: Level, upper: Level, wrt: Level, eps0: float = 0.01, alp
     return _hypergrad(lower, upper, wrt, method="fd", eps0=eps0, alpha=alpha)
 
 
+def hypergrad_itd(lower: Level, upper: Level, wrt: Level, n_steps: int) -> np.ndarray:
+    """Iterative differentiation with reverse-mode autodiff (ITD-RMAD, Sec. 3.2): take n_steps
+    unrolled gradient steps x_{t+1} = x_t - lr * g(x_t, c) from the current lower parameters
+    (which are left at x_T), then differentiate C_upper(x_T(c), c) through the stored steps:
+
+        a <- dC_u/dx at x_T;   out <- dC_u/dc
+        for t = T-1 .. 0:   out <- out - lr * M_t^T a ;   a <- a - lr * H_t a
+
+    with H_t, M_t the second derivatives of the lower cost at x_t (same stop-gradient and
+    quantisation conventions as `hvp` / `mixed_vjp`)."""
+    xs = []
+    for _ in range(int(n_steps)):
+        xs.append(lower.params.copy())
+        lower.params = lower.params - lower.lr * grad(lower, lower)
+    a = grad(upper, lower)
+    out = grad(upper, wrt).copy()
+    for x_t in reversed(xs):
+        over = {id(lower): x_t}
+        out = out - lower.lr * mixed_vjp(lower, wrt, a, over)
+        a = a - lower.lr * hvp(lower, a, over)
+    return out
+
+
 def chain_levels(levels, path, cfgs, v_in=None) -> np.ndarray:
     """One path term of Eq. 2, evaluated right to left (Sec. 3.2).
 

@@ -81,6 +81,7 @@ def lib():
         "betty_hypergrad_neumann": [LP, LP, LP, I32, F, VP, VP, SZ, VP],
         "betty_hypergrad_cg": [LP, LP, LP, I32, F, VP, VP, SZ, VP],
         "betty_hypergrad_fd": [LP, LP, LP, F, F, VP, VP, SZ, VP],
+        "betty_hypergrad_itd": [LP, LP, LP, I32, VP, VP, SZ, VP],
         "betty_chain_levels": [C.POINTER(LP), I32, C.POINTER(I32), I32, C.POINTER(_MethodCfg), VP, VP, I32,
                                VP, SZ, VP],
     }
@@ -235,6 +236,12 @@ def betty_hypergrad_fd(lower: Level, upper: Level, wrt: Level, eps0: float, alph
                        ws: Workspace, stream=None) -> None:
     _check(lib().betty_hypergrad_fd(lower.ref, upper.ref, wrt.ref, float(eps0), float(alpha), _ptr(out), ws.ptr,
                                     ws.nbytes, _stream(stream)), "betty_hypergrad_fd")
+
+
+def betty_hypergrad_itd(lower: Level, upper: Level, wrt: Level, n_steps: int, out: torch.Tensor, ws: Workspace,
+                        stream=None) -> None:
+    _check(lib().betty_hypergrad_itd(lower.ref, upper.ref, wrt.ref, int(n_steps), _ptr(out), ws.ptr, ws.nbytes,
+                                     _stream(stream)), "betty_hypergrad_itd")
 
 
 def betty_chain_levels(levels: Sequence[Level], path: Sequence[int], per_edge: Sequence[MethodCfg],

@@ -218,11 +218,61 @@ static betty_status hypergrad(const betty_level* lower, const betty_level* upper
   return brj(c, lower, wrt, v, cfg, out, true);
 }
 
+// ITD-RMAD: n_steps unrolled lower steps with the iterates kept in the workspace, then the reverse
+// sweep  a <- a - lr H_t a,  out <- out - lr M_t^T a  from t = T-1 down to 0.
+static betty_status hypergrad_itd(const betty_level* lower, const betty_level* upper, const betty_level* wrt,
+                                  int n_steps, float* out, void* ws, size_t ws_bytes, void* stream) {
+  BETTY_TRY(validate_level(lower));
+  BETTY_TRY(validate_level(upper));
+  if (!wrt || !out || n_steps < 0) return BETTY_ERR_INVALID_ARG;
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  if (!is_participant(upper, lower) || !is_participant(upper, wrt) || !is_participant(lower, wrt) || wrt == lower)
+    return BETTY_ERR_INVALID_ARG;
+  Ctx c(ws, ws_bytes, stream);
+  const int64_t n = lower->n_params, nc = wrt->n_params;
+  const bool vecfam = is_vector_family(lower->loss);
+  const size_t stride = ((size_t)n + 63) & ~size_t(63);
+  BETTY_ALLOC(iter, float, c, stride * (size_t)(n_steps > 0 ? n_steps : 1));
+  BETTY_ALLOC(a, float, c, (size_t)n);
+  BETTY_ALLOC(h, float, c, (size_t)n);
+  BETTY_ALLOC(m, float, c, (size_t)nc);
+  for (int t = 0; t < n_steps; ++t) {
+    BETTY_TRY(vec_copy(c, iter + stride * t, lower->params, n));
+    BETTY_TRY(vecfam ? vecfam_lower_step(c, lower, 1) : mlpfam_lower_step(c, lower, 1));
+  }
+  BETTY_TRY(level_grad(c, upper, lower, a));
+  BETTY_TRY(level_grad(c, upper, wrt, out));
+  betty_level at = *lower;            // the lower problem seen at a stored iterate
+  for (int t = n_steps - 1; t >= 0; --t) {
+    at.params = iter + stride * t;
+    const size_t mark = c.arena.mark();
+    if (vecfam) {
+      BETTY_TRY(vecfam_mixed(c, &at, wrt, a, m));
+      BETTY_TRY(vecfam_hvp(c, &at, a, h));
+    } else {
+      MlpHvpCache* cache = nullptr;
+      BETTY_TRY(mlpfam_hvp_begin(c, &at, &cache));
+      BETTY_TRY(mlpfam_mixed(c, &at, cache, wrt, a, m));
+      BETTY_TRY(mlpfam_hvp(c, &at, cache, a, h));
+    }
+    k_scale_into<<<ew_grid(nc), 256, 0, c.stream>>>(out, m, -lower->lr, 1, nc);
+    BETTY_LAUNCH_CHECK();
+    BETTY_TRY(vec_axpby(c, a, 1.f, a, -lower->lr, h, n));
+    c.arena.release(mark);
+  }
+  return BETTY_OK;
+}
+
 }  // namespace betty
 
 using namespace betty;
 
 extern "C" {
+
+betty_status betty_hypergrad_itd(const betty_level* lower, const betty_level* upper, const betty_level* wrt,
+                                 int32_t n_steps, float* out, void* ws, size_t ws_bytes, void* stream) {
+  return hypergrad_itd(lower, upper, wrt, n_steps, out, ws, ws_bytes, stream);
+}
 
 const char* betty_status_string(betty_status s) {
   switch (s) {

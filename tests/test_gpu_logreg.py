@@ -204,3 +204,18 @@ def test_repeated_calls_are_bitwise_identical(bt):
     bt.betty_hvp(w, u, a, ws)
     bt.betty_hvp(w, u, b, ws)
     assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("n,d,nv,T", [(1024, 64, 256, 100), (700, 1028, 90, 12)])
+def test_itd_hypergradient_matches_oracle(bt, n, d, nv, T):
+    """ITD-RMAD: reverse sweep through the stored unrolled steps."""
+    from tests import cuda_build as cb
+    inp = si.config1() if (n, d) == (1024, 64) else si.logreg_bilevel(77, n, d, nv)
+    (w, lam), (ow, olam) = _pair(inp)
+    ws = bt.Workspace([w, lam], extra_bytes=(T + 1) * (d + 64) * 4)
+    out = _vec(d)
+    bt.betty_hypergrad_itd(w, lam, lam, T, out, ws)
+    ref = oracle.hypergrad_itd(ow, olam, olam, T)
+    assert cb.rel_l2(w.params, ow.params) < TOL
+    assert cb.rel_l2(out, ref) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK

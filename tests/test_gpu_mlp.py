@@ -195,3 +195,19 @@ def test_config5_reduced_width(bt):
     bt.betty_hypergrad_neumann(w, th, th, inp.K, inp.alpha, out, ws)
     assert cb.rel_l2(out, oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)) < TOL
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+@pytest.mark.parametrize("act", ["relu", "gelu"])
+def test_itd_on_reweighting_matches_oracle(bt, act):
+    from tests import cuda_build as cb
+    inp = _perturb(si.reweight_bilevel(71, (64, 96, 10), 128, 0.4, activation=act), 71)
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    T = 3
+    ws = bt.Workspace([w, th], extra_bytes=(T + 1) * (inp.w.size + 64) * 4)
+    out = _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_hypergrad_itd(w, th, th, T, out, ws)
+    ref = oracle.hypergrad_itd(ow, oth, oth, T)
+    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    assert cb.rel_l2(out, ref) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK

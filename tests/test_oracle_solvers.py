@@ -198,6 +198,45 @@ def test_lower_step_is_plain_gradient_descent():
     assert rel(lo.params, w) < 1e-8
 
 
+def test_itd_equals_autodiff_through_the_unrolled_steps():
+    """ITD-RMAD against reverse-mode autodiff (torch, fp64) of the upper cost through T explicit
+    gradient-descent steps of the lower cost, for the logistic problem and for the reweighted MLP."""
+    # logistic weight decay
+    inp = si.logreg_bilevel(23, 50, 6, 20)
+    inp.lam = (np.abs(si.normal_f32(23, 7, (6,))) * 0.1 + 0.02).astype(np.float32)
+    lo, up = logreg_levels(inp)
+    X, y, Xv, yv = _t(inp.X), _t(inp.y), _t(inp.Xv), _t(inp.yv)
+    lam = _t(inp.lam).requires_grad_(True)
+    w = _t(inp.w0)
+    sp = torch.nn.functional.softplus
+    for _ in range(7):
+        wg = w.detach().requires_grad_(True) if not w.requires_grad else w
+        c = sp(-y * (X @ wg)).mean() + 0.5 * (lam * wg * wg).sum()
+        g, = torch.autograd.grad(c, [wg], create_graph=True)
+        w = wg - inp.lr * g
+    cu = sp(-yv * (Xv @ w)).mean()
+    ref, = torch.autograd.grad(cu, [lam])
+    got = oracle.hypergrad_itd(lo, up, up, 7)
+    assert rel(got, ref.numpy()) < 1e-10
+    assert rel(lo.params, w.detach().numpy()) < 1e-12
+    # reweighted MLP (stop-gradient on the weight net's input), gelu
+    from tests.test_oracle_derivatives import _tiny_reweight, _torch_mlp_logits
+    from tests.oracle_build import reweight_levels
+    inp = _tiny_reweight("gelu", seed=43)
+    w_lv, th_lv = reweight_levels(inp, bf16=False)
+    th = _t(inp.theta).requires_grad_(True)
+    w = _t(inp.w).requires_grad_(True)
+    for _ in range(3):
+        c = _torch_reweight_cost(inp, w, th, None)
+        g, = torch.autograd.grad(c, [w], create_graph=True)
+        w = w - inp.lr * g
+    zv = _torch_mlp_logits(inp.widths, "gelu", w, _t(inp.val.X))
+    cu = torch.nn.functional.cross_entropy(zv, torch.from_numpy(inp.val.y.astype(np.int64)))
+    ref, = torch.autograd.grad(cu, [th])
+    got = oracle.hypergrad_itd(w_lv, th_lv, th_lv, 3)
+    assert rel(got, ref.numpy()) < 1e-9
+
+
 # ------------------------------------------------------------------ chain (Eq. 2)
 def _dense_three_level(inp):
     """Hessians and mixed second derivatives of a tiny three-level program by autodiff."""
