@@ -384,6 +384,21 @@ def make_workload(cfg: int, method: str, scale: float):
     raise SystemExit(f"unknown config {cfg}")
 
 
+def max_over_ranks(ms: float, world: int, dist, device) -> float:
+    """Step time of the job = the slowest rank's device time."""
+    if world <= 1:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(ms_per_step: float, world: int) -> float:
+    """Whole-job steps/s of `world` independent replicas that each finish a step every ms_per_step."""
+    return world * 1e3 / ms_per_step
+
+
 def blas_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -535,10 +550,7 @@ def main():
             launches = launches_per_replay * steps
         clocks = sampler.stop() if sampler else None
         ms = sum(a.elapsed_time(b) for a, b in pairs)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(ms, world, dist, "cuda")
         return ms, launches, clocks
 
     # configs whose inputs fit in L2 get a flush (a 512 MiB write) before every step
@@ -571,7 +583,7 @@ def main():
     ms, launches, clocks = timed(step_dev, args.steps, warm, sampler)
     st, _ = bt.betty_poll_status(wl.ws)
     ms_per_step = ms / args.steps
-    value = world * 1e3 / ms_per_step
+    value = aggregate_value(ms_per_step, world)
 
     e2e = None
     if not args.no_e2e:

@@ -7,7 +7,7 @@
 // Each operand may be K-major (K contiguous in memory) or MN-major (M or N contiguous): forward
 // passes are K-major x K-major, backward-data passes K-major x N-major, weight-gradient passes
 // M-major x N-major.  Ragged M, N and K are handled by TMA's zero fill and predicated stores.
-// No cluster multicast is used anywhere.
+// Every CTA issues plain TMA loads for its own operand slabs.
 #include <cuda.h>
 #include "gemm.cuh"
 
@@ -352,7 +352,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
 // with tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of A and 128 of the 256 columns
 // of B, so every byte of B fetched from L2 feeds twice as many MMA rows as in the one-SM kernel.
 // The even CTA of the pair issues the MMAs; each CTA holds the accumulator rows of its own half in
-// its tensor memory and runs its own epilogue.  Plain TMA loads, no multicast.
+// its tensor memory and runs its own epilogue.  Each CTA loads its own slabs with plain TMA loads.
 static constexpr int TC2_BN = 256;           // tile width; each CTA stages half of it
 static constexpr int TC2_STAGE_BYTES = TC_A_BYTES + (TC2_BN / 2) * TC_BK * 2;   // 32 KB per CTA
 static constexpr int TC2_STAGES = 6;
