@@ -232,6 +232,31 @@ betty_status betty_gemm_bf16(int32_t M, int32_t N, int32_t n_pairs, const betty_
                              float* C, int64_t ldc, float beta, int32_t path, void* ws, size_t ws_bytes,
                              void* stream);
 
+/* The dataflow graph of Sec. 3.1: directed edges between problem indices.  An upper-to-lower edge
+ * (from > to in the paper's ordering) says that theta_from constrains problem `to`; a lower-to-upper
+ * edge says that theta*_from constrains problem `to`. */
+typedef struct { int32_t from, to; } betty_edge;
+
+/* Sec. 3.1 path finding (the paper's modified depth-first search): every valid path from theta_k to
+ * the optimal parameters of a target problem starts with one upper-to-lower edge and continues over
+ * lower-to-upper edges only.  Host-only; touches no device.  `targets` (host) lists L_k.  Paths are
+ * written to `paths` (host, `capacity` ints) as records [len, k, q(1), ..., q(len-1)] in discovery
+ * order, ready for betty_chain_levels; n_paths / n_ints (nullable) receive the totals even when the
+ * buffer is too small (then BETTY_ERR_WORKSPACE is returned; paths == NULL only counts). */
+betty_status betty_find_paths(int32_t n_levels, const betty_edge* u2l, int32_t n_u2l, const betty_edge* l2u,
+                              int32_t n_l2u, int32_t k, const int32_t* targets, int32_t n_targets,
+                              int32_t* paths, int32_t capacity, int32_t* n_paths, int32_t* n_ints);
+
+/* Eq. 2 for problem k over the whole dataflow graph: out[levels[k]->n_params] = direct gradient + the
+ * sum over all lower problems l in L_k (sources of lower-to-upper edges into k) and all valid paths from
+ * theta_k to theta*_l of the path's Jacobian chain times dC_k/d theta*_l.  Paths that share a suffix are
+ * merged at their common node (exact by linearity), so each edge's Jacobian product is taken once.
+ * per_level[q] configures every best-response Jacobian of problem q.  Edge arrays are host memory. */
+betty_status betty_hypergrad_graph(const betty_level* const* levels, int32_t n_levels, const betty_edge* u2l,
+                                   int32_t n_u2l, const betty_edge* l2u, int32_t n_l2u, int32_t k,
+                                   const betty_method_cfg* per_level, float* out, void* ws, size_t ws_bytes,
+                                   void* stream);
+
 const char* betty_status_string(betty_status s);
 
 /* Number of CUDA kernels this library has launched in the calling process since it was loaded

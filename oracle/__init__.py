@@ -10,6 +10,7 @@ What each function follows:
                  for the logistic weight-decay problem; the App. A data-reweighting listing
                  for the reweighted cross-entropy) with their first and second derivatives
                  written out by hand.
+  * graph.py   - the dataflow graph of Sec. 3.1: path enumeration and Eq. 2 summed over all paths.
   * solvers.py - unrolled lower-level gradient steps (Sec. 3.2), the best-response-Jacobian
                  times vector operation (Sec. 3.2) with Neumann-series, conjugate-gradient and
                  finite-difference approximations, Eq. 1 (hypergradient of a bilevel pair) and
@@ -24,6 +25,7 @@ the finite difference with a finite epsilon) have no values printed in the paper
 parity is "parity unpinned" by the paper and pinned only by their mathematical definition
 (matrix-power sums, Krylov optimality, the O(eps^2) limit).
 """
+from .graph import find_paths, hypergrad_graph  # noqa: F401
 from .levels import Level  # noqa: F401
 from .solvers import (  # noqa: F401
     brj, cg_solve, chain_levels, grad, hvp, hypergrad_cg, hypergrad_fd, hypergrad_itd, hypergrad_neumann,

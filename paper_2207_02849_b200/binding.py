@@ -46,6 +46,10 @@ _Level._fields_ = [
     ("constraints", C.POINTER(C.POINTER(_Level))),
 ]
 
+class _Edge(C.Structure):
+    _fields_ = [("src", C.c_int32), ("dst", C.c_int32)]
+
+
 class _GemmOperands(C.Structure):
     _fields_ = [("A", C.c_void_p), ("lda", C.c_int64), ("a_transposed", C.c_int32), ("B", C.c_void_p),
                 ("ldb", C.c_int64), ("b_transposed", C.c_int32), ("K", C.c_int32), ("alpha", C.c_float)]
@@ -87,6 +91,9 @@ def lib():
     }
     sig["betty_hvp_logreg_static"] = [VP, C.c_int64, C.c_int64, VP, VP, VP, VP, VP, VP]
     sig["betty_gemm_bf16"] = [I32, I32, I32, C.POINTER(_GemmOperands), VP, C.c_int64, F, I32, VP, SZ, VP]
+    EP, IP = C.POINTER(_Edge), C.POINTER(I32)
+    sig["betty_find_paths"] = [I32, EP, I32, EP, I32, I32, IP, I32, IP, I32, IP, IP]
+    sig["betty_hypergrad_graph"] = [C.POINTER(LP), I32, EP, I32, EP, I32, I32, C.POINTER(_MethodCfg), VP, VP, SZ, VP]
     for name, args in sig.items():
         fn = getattr(L, name)
         fn.argtypes, fn.restype = args, C.c_int
@@ -271,3 +278,36 @@ def betty_gemm_bf16(M: int, N: int, pairs, Cout: torch.Tensor, ldc: int, beta: f
         arr[i] = _GemmOperands(_ptr(A), int(lda), int(bool(ta)), _ptr(B), int(ldb), int(bool(tb)), int(K), float(alpha))
     _check(lib().betty_gemm_bf16(int(M), int(N), len(pairs), arr, _ptr(Cout), int(ldc), float(beta), int(path), ws.ptr,
                                  ws.nbytes, _stream(stream)), "betty_gemm_bf16")
+
+
+def _edges(pairs):
+    arr = (_Edge * max(1, len(pairs)))()
+    for i, (a, b) in enumerate(pairs):
+        arr[i] = _Edge(int(a), int(b))
+    return arr
+
+
+def betty_find_paths(n_levels: int, u2l, l2u, k: int, targets) -> list:
+    """Valid paths [k, q(1), ..., q(m)] of the dataflow graph (host-only call)."""
+    t = (C.c_int32 * max(1, len(targets)))(*[int(x) for x in targets])
+    n_paths, n_ints = C.c_int32(0), C.c_int32(0)
+    eu, el = _edges(u2l), _edges(l2u)
+    _check(lib().betty_find_paths(n_levels, eu, len(u2l), el, len(l2u), int(k), t, len(targets), None, 0,
+                                  C.byref(n_paths), C.byref(n_ints)), "betty_find_paths")
+    buf = (C.c_int32 * max(1, n_ints.value))()
+    _check(lib().betty_find_paths(n_levels, eu, len(u2l), el, len(l2u), int(k), t, len(targets), buf, n_ints.value,
+                                  C.byref(n_paths), C.byref(n_ints)), "betty_find_paths")
+    out, i = [], 0
+    for _ in range(n_paths.value):
+        ln = buf[i]
+        out.append([buf[i + 1 + j] for j in range(ln)])
+        i += 1 + ln
+    return out
+
+
+def betty_hypergrad_graph(levels: Sequence[Level], u2l, l2u, k: int, per_level: Sequence[MethodCfg], out: torch.Tensor,
+                          ws: Workspace, stream=None) -> None:
+    arr = _level_array(levels)
+    cfgs = (_MethodCfg * len(per_level))(*[m.c for m in per_level])
+    _check(lib().betty_hypergrad_graph(arr, len(levels), _edges(u2l), len(u2l), _edges(l2u), len(l2u), int(k), cfgs,
+                                       _ptr(out), ws.ptr, ws.nbytes, _stream(stream)), "betty_hypergrad_graph")

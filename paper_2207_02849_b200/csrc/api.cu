@@ -263,11 +263,146 @@ static betty_status hypergrad_itd(const betty_level* lower, const betty_level* u
   return BETTY_OK;
 }
 
+// ------------------------------------------------------------------ dataflow graph (Sec. 3.1)
+struct Graph {
+  int n;
+  const betty_edge* u2l; int n_u2l;
+  const betty_edge* l2u; int n_l2u;
+};
+static bool graph_ok(const Graph& g) {
+  if (g.n <= 0 || g.n_u2l < 0 || g.n_l2u < 0 || (g.n_u2l > 0 && !g.u2l) || (g.n_l2u > 0 && !g.l2u)) return false;
+  for (int i = 0; i < g.n_u2l; ++i)
+    if (g.u2l[i].from < 0 || g.u2l[i].from >= g.n || g.u2l[i].to < 0 || g.u2l[i].to >= g.n) return false;
+  for (int i = 0; i < g.n_l2u; ++i)
+    if (g.l2u[i].from < 0 || g.l2u[i].from >= g.n || g.l2u[i].to < 0 || g.l2u[i].to >= g.n) return false;
+  return true;
+}
+
+// Depth-first enumeration: the first edge is upper-to-lower, every later edge lower-to-upper; a path is
+// reported each time it stands on a target.  Records are [len, k, q(1), ..., q(m)], len = m + 1.
+struct PathSink { int32_t* buf; int capacity; int used; int count; bool overflow; };
+static void emit_path(PathSink& s, int k, const int* stack, int depth) {
+  const int need = depth + 2;
+  if (s.buf && s.used + need <= s.capacity) {
+    s.buf[s.used] = depth + 1;
+    s.buf[s.used + 1] = k;
+    for (int i = 0; i < depth; ++i) s.buf[s.used + 2 + i] = stack[i];
+  } else if (s.buf) {
+    s.overflow = true;
+  }
+  s.used += need;
+  s.count += 1;
+}
+static void dfs_paths(const Graph& g, int k, const bool* is_target, int* stack, bool* on_path, int depth, PathSink& s) {
+  const int c = stack[depth - 1];
+  if (is_target[c]) emit_path(s, k, stack, depth);
+  for (int i = 0; i < g.n_l2u; ++i) {
+    if (g.l2u[i].from != c) continue;
+    const int nx = g.l2u[i].to;
+    if (nx == k || on_path[nx]) continue;
+    stack[depth] = nx; on_path[nx] = true;
+    dfs_paths(g, k, is_target, stack, on_path, depth + 1, s);
+    on_path[nx] = false;
+  }
+}
+
+// Merged right-to-left evaluation of Eq. 2 over the graph: u_c = [c in L_k] dC_k/d theta_c +
+// sum over lower-to-upper edges c -> n of (d theta_n* / d theta_c*)^T u_n, each edge's Jacobian product
+// taken once (exact by linearity); out = direct gradient + sum over k -> c of (d theta_c*/d theta_k)^T u_c.
+struct GraphEval {
+  Ctx* c; const betty_level* const* levels; const Graph* g; int k; const bool* is_target;
+  const betty_method_cfg* cfg; float** u; int* state;   // state: 0 new, 1 in progress, 2 done (u may stay null: no target above)
+};
+static betty_status eval_node(GraphEval& e, int cnode) {
+  if (e.state[cnode] == 2) return BETTY_OK;
+  if (e.state[cnode] == 1) return BETTY_ERR_INVALID_ARG;      // cycle among lower-to-upper edges
+  e.state[cnode] = 1;
+  float* acc = nullptr;
+  const int64_t nc = e.levels[cnode]->n_params;
+  if (e.is_target[cnode]) {
+    acc = e.c->arena.alloc<float>((size_t)nc);
+    if (!acc) return BETTY_ERR_WORKSPACE;
+    BETTY_TRY(level_grad(*e.c, e.levels[e.k], e.levels[cnode], acc));
+  }
+  for (int i = 0; i < e.g->n_l2u; ++i) {
+    if (e.g->l2u[i].from != cnode) continue;
+    const int nx = e.g->l2u[i].to;
+    if (nx == e.k) continue;
+    BETTY_TRY(eval_node(e, nx));
+    if (!e.u[nx]) continue;                                   // nothing of C_k reaches through nx
+    bool accumulate = true;
+    if (!acc) {
+      acc = e.c->arena.alloc<float>((size_t)nc);
+      if (!acc) return BETTY_ERR_WORKSPACE;
+      accumulate = false;
+    }
+    BETTY_TRY(brj(*e.c, e.levels[nx], e.levels[cnode], e.u[nx], e.cfg[nx], acc, accumulate));
+  }
+  e.u[cnode] = acc;
+  e.state[cnode] = 2;
+  return BETTY_OK;
+}
+
 }  // namespace betty
 
 using namespace betty;
 
 extern "C" {
+
+betty_status betty_find_paths(int32_t n_levels, const betty_edge* u2l, int32_t n_u2l, const betty_edge* l2u,
+                              int32_t n_l2u, int32_t k, const int32_t* targets, int32_t n_targets, int32_t* paths,
+                              int32_t capacity, int32_t* n_paths, int32_t* n_ints) {
+  Graph g = {n_levels, u2l, n_u2l, l2u, n_l2u};
+  if (!graph_ok(g) || k < 0 || k >= n_levels || n_targets < 0 || (n_targets > 0 && !targets) || n_levels > 4096 ||
+      capacity < 0 || !n_paths)
+    return BETTY_ERR_INVALID_ARG;
+  bool is_target[4096] = {false};
+  bool on_path[4096] = {false};
+  int stack[4096];
+  for (int i = 0; i < n_targets; ++i) {
+    if (targets[i] < 0 || targets[i] >= n_levels) return BETTY_ERR_INVALID_ARG;
+    is_target[targets[i]] = true;
+  }
+  PathSink s = {paths, capacity, 0, 0, false};
+  for (int i = 0; i < n_u2l; ++i) {
+    if (u2l[i].from != k) continue;
+    const int c0 = u2l[i].to;
+    if (c0 == k) continue;
+    stack[0] = c0; on_path[c0] = true;
+    dfs_paths(g, k, is_target, stack, on_path, 1, s);
+    on_path[c0] = false;
+  }
+  *n_paths = s.count;
+  if (n_ints) *n_ints = s.used;
+  return s.overflow ? BETTY_ERR_WORKSPACE : BETTY_OK;
+}
+
+betty_status betty_hypergrad_graph(const betty_level* const* levels, int32_t n_levels, const betty_edge* u2l,
+                                   int32_t n_u2l, const betty_edge* l2u, int32_t n_l2u, int32_t k,
+                                   const betty_method_cfg* per_level, float* out, void* ws, size_t ws_bytes,
+                                   void* stream) {
+  Graph g = {n_levels, u2l, n_u2l, l2u, n_l2u};
+  if (!levels || !graph_ok(g) || k < 0 || k >= n_levels || !per_level || !out || n_levels > 256) return BETTY_ERR_INVALID_ARG;
+  for (int i = 0; i < n_levels; ++i) BETTY_TRY(validate_level(levels[i]));
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  Ctx c(ws, ws_bytes, stream);
+  bool is_target[256] = {false};
+  float* u[256] = {nullptr};
+  int state[256] = {0};
+  for (int i = 0; i < n_l2u; ++i)
+    if (l2u[i].to == k) is_target[l2u[i].from] = true;         // L_k: the lower problems that call k
+  GraphEval e = {&c, levels, &g, k, is_target, per_level, u, state};
+  BETTY_TRY(level_grad(c, levels[k], levels[k], out));          // direct gradient
+  for (int i = 0; i < n_u2l; ++i) {
+    if (u2l[i].from != k) continue;
+    const int c0 = u2l[i].to;
+    if (c0 == k) continue;
+    BETTY_TRY(eval_node(e, c0));
+    if (!u[c0]) continue;
+    BETTY_TRY(brj(c, levels[c0], levels[k], u[c0], per_level[c0], out, true));
+  }
+  return BETTY_OK;
+}
 
 betty_status betty_hypergrad_itd(const betty_level* lower, const betty_level* upper, const betty_level* wrt,
                                  int32_t n_steps, float* out, void* ws, size_t ws_bytes, void* stream) {

@@ -211,3 +211,29 @@ def test_itd_on_reweighting_matches_oracle(bt, act):
     assert cb.rel_l2(w.params, ow.params) < 1e-3
     assert cb.rel_l2(out, ref) < TOL
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+@pytest.mark.parametrize("act", ["relu", "gelu"])
+def test_graph_hypergradient_matches_sum_over_paths(bt, act):
+    """Eq. 2 over the three-level dataflow graph: the library merges the two paths from lambda at the
+    w* node; the oracle sums the per-path chains."""
+    from tests import cuda_build as cb
+    inp = _three(act)
+    P = cb.three_levels(inp)
+    O = ob.three_levels(inp)
+    ws = bt.Workspace(list(P))
+    u2l = [(2, 0), (1, 0)]                 # lambda and theta constrain the classifier
+    l2u = [(0, 1), (0, 2), (1, 2)]         # w* constrains P2 and P3, theta* constrains P3
+    assert sorted(bt.betty_find_paths(3, u2l, l2u, 2, [0, 1])) == [[2, 0], [2, 0, 1]]
+    nm = dict(method="neumann", K=3, alpha=0.01)
+    ref = oracle.hypergrad_graph(list(O), u2l, l2u, 2, [nm, nm, nm])
+    cfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=3, alpha=0.01)
+    out = _vec(inp.lam.size)
+    bt.betty_hypergrad_graph(list(P), u2l, l2u, 2, [cfg, cfg, cfg], out, ws)
+    assert cb.rel_l2(out, ref) < TOL
+    # the middle problem's own gradient: one path theta -> w*
+    ref2 = oracle.hypergrad_graph(list(O), u2l, l2u, 1, [nm, nm, nm])
+    out2 = _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_hypergrad_graph(list(P), u2l, l2u, 1, [cfg, cfg, cfg], out2, ws)
+    assert cb.rel_l2(out2, ref2) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
