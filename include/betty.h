@@ -257,6 +257,19 @@ betty_status betty_hypergrad_graph(const betty_level* const* levels, int32_t n_l
                                    const betty_method_cfg* per_level, float* out, void* ws, size_t ws_bytes,
                                    void* stream);
 
+/* Execution of the whole program (Sec. 3.3).  n_iterations times, every lowermost problem (one that no
+ * lower-to-upper edge enters) takes one gradient step; a problem that has taken unroll_steps[j] steps
+ * since its last call-out calls every problem it constrains through a lower-to-upper edge, and a called
+ * problem takes its own step once all problems of its L set have called.  A step of problem j is
+ * params_j -= lr_j * dC_j/d theta_j with the gradient of Eq. 2 (betty_hypergrad_graph); problems without
+ * lower problems use the fused betty_lower_step.  step_log (host, nullable, log_capacity ints) receives the
+ * indices of the problems in the order they stepped; n_steps_taken (nullable) the total count.
+ * Everything is enqueued on `stream`; parameters are updated in place. */
+betty_status betty_engine_run(const betty_level* const* levels, int32_t n_levels, const betty_edge* u2l, int32_t n_u2l,
+                              const betty_edge* l2u, int32_t n_l2u, const betty_method_cfg* per_level,
+                              const int32_t* unroll_steps, int32_t n_iterations, int32_t* step_log,
+                              int32_t log_capacity, int32_t* n_steps_taken, void* ws, size_t ws_bytes, void* stream);
+
 const char* betty_status_string(betty_status s);
 
 /* Number of CUDA kernels this library has launched in the calling process since it was loaded

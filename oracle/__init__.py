@@ -25,7 +25,7 @@ the finite difference with a finite epsilon) have no values printed in the paper
 parity is "parity unpinned" by the paper and pinned only by their mathematical definition
 (matrix-power sums, Krylov optimality, the O(eps^2) limit).
 """
-from .graph import find_paths, hypergrad_graph  # noqa: F401
+from .graph import engine_run, find_paths, hypergrad_graph  # noqa: F401
 from .levels import Level  # noqa: F401
 from .solvers import (  # noqa: F401
     brj, cg_solve, chain_levels, grad, hvp, hypergrad_cg, hypergrad_fd, hypergrad_itd, hypergrad_neumann,

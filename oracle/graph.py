@@ -40,3 +40,33 @@ def hypergrad_graph(levels, u2l, l2u, k, cfgs) -> np.ndarray:
         edge_cfgs = [cfgs[q] for q in path[1:]]
         total = total + chain_levels(levels, path, edge_cfgs)
     return total
+
+
+def engine_run(levels, u2l, l2u, cfgs, unroll, n_iterations):
+    """Execution of the whole program (Sec. 3.3).  Only the lowermost problems are stepped directly;
+    a problem that has completed `unroll[j]` steps calls the problems it constrains through
+    lower-to-upper edges; a called problem steps once every problem of its L set has called.  One
+    step of problem j is theta_j <- theta_j - lr_j * dC_j/d theta_j with the gradient of Eq. 2.
+    Returns the list of problem indices in the order they stepped."""
+    n = len(levels)
+    n_lower = [sum(1 for a, b in l2u if b == j) for j in range(n)]
+    count, ready, log = [0] * n, [0] * n, []
+
+    def step(j):
+        log.append(j)
+        g = hypergrad_graph(levels, u2l, l2u, j, cfgs)
+        levels[j].params = levels[j].params - levels[j].lr * g
+        count[j] += 1
+        if count[j] % unroll[j] == 0:
+            for a, b in l2u:
+                if a == j:
+                    ready[b] += 1
+                    if ready[b] >= n_lower[b]:
+                        ready[b] = 0
+                        step(b)
+
+    for _ in range(int(n_iterations)):
+        for j in range(n):
+            if n_lower[j] == 0:
+                step(j)
+    return log

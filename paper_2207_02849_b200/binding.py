@@ -93,6 +93,7 @@ def lib():
     sig["betty_gemm_bf16"] = [I32, I32, I32, C.POINTER(_GemmOperands), VP, C.c_int64, F, I32, VP, SZ, VP]
     EP, IP = C.POINTER(_Edge), C.POINTER(I32)
     sig["betty_find_paths"] = [I32, EP, I32, EP, I32, I32, IP, I32, IP, I32, IP, IP]
+    sig["betty_engine_run"] = [C.POINTER(LP), I32, EP, I32, EP, I32, C.POINTER(_MethodCfg), IP, I32, IP, I32, IP, VP, SZ, VP]
     sig["betty_hypergrad_graph"] = [C.POINTER(LP), I32, EP, I32, EP, I32, I32, C.POINTER(_MethodCfg), VP, VP, SZ, VP]
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -311,3 +312,17 @@ def betty_hypergrad_graph(levels: Sequence[Level], u2l, l2u, k: int, per_level: 
     cfgs = (_MethodCfg * len(per_level))(*[m.c for m in per_level])
     _check(lib().betty_hypergrad_graph(arr, len(levels), _edges(u2l), len(u2l), _edges(l2u), len(l2u), int(k), cfgs,
                                        _ptr(out), ws.ptr, ws.nbytes, _stream(stream)), "betty_hypergrad_graph")
+
+
+def betty_engine_run(levels: Sequence[Level], u2l, l2u, per_level: Sequence[MethodCfg], unroll_steps: Sequence[int],
+                     n_iterations: int, ws: Workspace, stream=None, log_capacity: int = 65536) -> list:
+    """Runs the program's execution schedule (Sec. 3.3); returns the order in which problems stepped."""
+    arr = _level_array(levels)
+    cfgs = (_MethodCfg * len(per_level))(*[m.c for m in per_level])
+    un = (C.c_int32 * len(unroll_steps))(*[int(x) for x in unroll_steps])
+    log = (C.c_int32 * log_capacity)()
+    n = C.c_int32(0)
+    _check(lib().betty_engine_run(arr, len(levels), _edges(u2l), len(u2l), _edges(l2u), len(l2u), cfgs, un,
+                                  int(n_iterations), log, log_capacity, C.byref(n), ws.ptr, ws.nbytes, _stream(stream)),
+           "betty_engine_run")
+    return [log[i] for i in range(min(n.value, log_capacity))]

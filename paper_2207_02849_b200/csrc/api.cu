@@ -343,6 +343,71 @@ static betty_status eval_node(GraphEval& e, int cnode) {
   return BETTY_OK;
 }
 
+static betty_status graph_hypergrad(Ctx& c, const betty_level* const* levels, const Graph& g, int k,
+                                    const betty_method_cfg* per_level, float* out) {
+  bool is_target[256] = {false};
+  float* u[256] = {nullptr};
+  int state[256] = {0};
+  for (int i = 0; i < g.n_l2u; ++i)
+    if (g.l2u[i].to == k) is_target[g.l2u[i].from] = true;     // L_k: the lower problems that call k
+  GraphEval e = {&c, levels, &g, k, is_target, per_level, u, state};
+  BETTY_TRY(level_grad(c, levels[k], levels[k], out));          // direct gradient
+  for (int i = 0; i < g.n_u2l; ++i) {
+    if (g.u2l[i].from != k) continue;
+    const int c0 = g.u2l[i].to;
+    if (c0 == k) continue;
+    BETTY_TRY(eval_node(e, c0));
+    if (!u[c0]) continue;
+    BETTY_TRY(brj(c, levels[c0], levels[k], u[c0], per_level[c0], out, true));
+  }
+  return BETTY_OK;
+}
+
+// Execution of Sec. 3.3: a problem takes one gradient step when called; after every unroll_steps of
+// its steps it calls the problems it constrains through lower-to-upper edges; a called problem steps
+// once all problems of its L set have called.
+struct Engine {
+  Ctx* c; const betty_level* const* levels; const Graph* g; const betty_method_cfg* cfg; const int32_t* unroll;
+  int32_t* log; int log_capacity; int n_logged;
+  int n_lower[256]; bool has_child[256]; int count[256]; int ready[256];
+};
+__global__ void k_descent(float* x, const float* gvec, float lr, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    x[i] -= lr * gvec[i];
+}
+static betty_status engine_step(Engine& e, int j, int depth) {
+  if (depth > 256) return BETTY_ERR_INVALID_ARG;
+  const betty_level* L = e.levels[j];
+  if (e.log && e.n_logged < e.log_capacity) e.log[e.n_logged] = j;
+  e.n_logged += 1;
+  const size_t mark = e.c->arena.mark();
+  const bool fused = !e.has_child[j] && (L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_QUADRATIC_WD ||
+                                         L->loss == BETTY_LOSS_MLP_CE_REWEIGHT);
+  if (fused) {
+    BETTY_TRY(is_vector_family(L->loss) ? vecfam_lower_step(*e.c, L, 1) : mlpfam_lower_step(*e.c, L, 1));
+  } else {
+    float* gvec = e.c->arena.alloc<float>((size_t)L->n_params);
+    if (!gvec) return BETTY_ERR_WORKSPACE;
+    BETTY_TRY(graph_hypergrad(*e.c, e.levels, *e.g, j, e.cfg, gvec));
+    k_descent<<<ew_grid(L->n_params), 256, 0, e.c->stream>>>(L->params, gvec, L->lr, L->n_params);
+    BETTY_LAUNCH_CHECK();
+  }
+  e.c->arena.release(mark);
+  e.count[j] += 1;
+  if (e.count[j] % e.unroll[j] == 0) {
+    for (int i = 0; i < e.g->n_l2u; ++i) {
+      if (e.g->l2u[i].from != j) continue;
+      const int m = e.g->l2u[i].to;
+      e.ready[m] += 1;
+      if (e.ready[m] >= e.n_lower[m]) {
+        e.ready[m] = 0;
+        BETTY_TRY(engine_step(e, m, depth + 1));
+      }
+    }
+  }
+  return BETTY_OK;
+}
+
 }  // namespace betty
 
 using namespace betty;
@@ -386,22 +451,33 @@ betty_status betty_hypergrad_graph(const betty_level* const* levels, int32_t n_l
   for (int i = 0; i < n_levels; ++i) BETTY_TRY(validate_level(levels[i]));
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
-  bool is_target[256] = {false};
-  float* u[256] = {nullptr};
-  int state[256] = {0};
-  for (int i = 0; i < n_l2u; ++i)
-    if (l2u[i].to == k) is_target[l2u[i].from] = true;         // L_k: the lower problems that call k
-  GraphEval e = {&c, levels, &g, k, is_target, per_level, u, state};
-  BETTY_TRY(level_grad(c, levels[k], levels[k], out));          // direct gradient
-  for (int i = 0; i < n_u2l; ++i) {
-    if (u2l[i].from != k) continue;
-    const int c0 = u2l[i].to;
-    if (c0 == k) continue;
-    BETTY_TRY(eval_node(e, c0));
-    if (!u[c0]) continue;
-    BETTY_TRY(brj(c, levels[c0], levels[k], u[c0], per_level[c0], out, true));
+  return graph_hypergrad(c, levels, g, k, per_level, out);
+}
+
+betty_status betty_engine_run(const betty_level* const* levels, int32_t n_levels, const betty_edge* u2l, int32_t n_u2l,
+                              const betty_edge* l2u, int32_t n_l2u, const betty_method_cfg* per_level,
+                              const int32_t* unroll_steps, int32_t n_iterations, int32_t* step_log,
+                              int32_t log_capacity, int32_t* n_steps_taken, void* ws, size_t ws_bytes, void* stream) {
+  Graph g = {n_levels, u2l, n_u2l, l2u, n_l2u};
+  if (!levels || !graph_ok(g) || !per_level || !unroll_steps || n_iterations < 0 || n_levels > 256 || log_capacity < 0)
+    return BETTY_ERR_INVALID_ARG;
+  for (int i = 0; i < n_levels; ++i) {
+    BETTY_TRY(validate_level(levels[i]));
+    if (unroll_steps[i] < 1) return BETTY_ERR_INVALID_ARG;
   }
-  return BETTY_OK;
+  BETTY_TRY(check_ws(ws, ws_bytes));
+  Ctx c(ws, ws_bytes, stream);
+  Engine e = {};
+  e.c = &c; e.levels = levels; e.g = &g; e.cfg = per_level; e.unroll = unroll_steps;
+  e.log = step_log; e.log_capacity = log_capacity;
+  for (int i = 0; i < n_l2u; ++i) e.n_lower[l2u[i].to] += 1;
+  for (int i = 0; i < n_u2l; ++i) e.has_child[u2l[i].from] = true;
+  betty_status st = BETTY_OK;
+  for (int it = 0; it < n_iterations && st == BETTY_OK; ++it)
+    for (int j = 0; j < n_levels && st == BETTY_OK; ++j)
+      if (e.n_lower[j] == 0) st = engine_step(e, j, 0);       // only the lowermost problems are called directly
+  if (n_steps_taken) *n_steps_taken = e.n_logged;
+  return st;
 }
 
 betty_status betty_hypergrad_itd(const betty_level* lower, const betty_level* upper, const betty_level* wrt,
