@@ -270,6 +270,12 @@ betty_status betty_engine_run(const betty_level* const* levels, int32_t n_levels
                               const int32_t* unroll_steps, int32_t n_iterations, int32_t* step_log,
                               int32_t log_capacity, int32_t* n_steps_taken, void* ws, size_t ws_bytes, void* stream);
 
+/* Self test of the failure path: enqueues a one-warp kernel whose bounded mbarrier wait can never be
+ * satisfied.  The wait gives up after its poll limit (a fraction of a second), the kernel records
+ * BETTY_ERR_TIMEOUT in the status block of ws and returns; the context stays usable.  betty_poll_status
+ * then reports the condition.  Every wait in the library's kernels uses the same bounded form. */
+betty_status betty_selftest_wait_timeout(void* ws, size_t ws_bytes, void* stream);
+
 const char* betty_status_string(betty_status s);
 
 /* Number of CUDA kernels this library has launched in the calling process since it was loaded

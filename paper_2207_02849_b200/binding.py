@@ -93,6 +93,7 @@ def lib():
     sig["betty_gemm_bf16"] = [I32, I32, I32, C.POINTER(_GemmOperands), VP, C.c_int64, F, I32, VP, SZ, VP]
     EP, IP = C.POINTER(_Edge), C.POINTER(I32)
     sig["betty_find_paths"] = [I32, EP, I32, EP, I32, I32, IP, I32, IP, I32, IP, IP]
+    sig["betty_selftest_wait_timeout"] = [VP, SZ, VP]
     sig["betty_engine_run"] = [C.POINTER(LP), I32, EP, I32, EP, I32, C.POINTER(_MethodCfg), IP, I32, IP, I32, IP, VP, SZ, VP]
     sig["betty_hypergrad_graph"] = [C.POINTER(LP), I32, EP, I32, EP, I32, I32, C.POINTER(_MethodCfg), VP, VP, SZ, VP]
     for name, args in sig.items():
@@ -326,3 +327,7 @@ def betty_engine_run(levels: Sequence[Level], u2l, l2u, per_level: Sequence[Meth
                                   int(n_iterations), log, log_capacity, C.byref(n), ws.ptr, ws.nbytes, _stream(stream)),
            "betty_engine_run")
     return [log[i] for i in range(min(n.value, log_capacity))]
+
+
+def betty_selftest_wait_timeout(ws: Workspace, stream=None) -> None:
+    _check(lib().betty_selftest_wait_timeout(ws.ptr, ws.nbytes, _stream(stream)), "betty_selftest_wait_timeout")

@@ -44,8 +44,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false if the phase did not complete within SPIN_LIMIT polls.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit = SPIN_LIMIT) {
+  for (uint32_t i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
@@ -307,6 +307,28 @@ betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int
 }
 
 }  // namespace betty
+
+// ------------------------------------------------------------------ bounded-wait self test
+// A wait that nothing will ever satisfy: the same bounded mbarrier wait the streaming kernel uses must
+// give up, record BETTY_ERR_TIMEOUT in the status block and let the kernel return normally.
+namespace betty {
+__global__ void k_wait_that_expires(StatusBlock* sb) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait_bounded(&bar, 0, 1u << 15)) record_status(sb, BETTY_ERR_TIMEOUT);   // short limit: well under a second
+  }
+}
+}  // namespace betty
+
+extern "C" betty_status betty_selftest_wait_timeout(void* ws, size_t ws_bytes, void* stream) {
+  using namespace betty;
+  if (!ws || ws_bytes < sizeof(StatusBlock) || (((uintptr_t)ws) & 255u)) return BETTY_ERR_WORKSPACE;
+  k_wait_that_expires<<<1, 32, 0, (cudaStream_t)stream>>>((StatusBlock*)ws);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
 
 // ------------------------------------------------------------------ allocation-free HVP
 // Scratch that belongs to the library image itself: every GPU that loads the library holds

@@ -237,3 +237,26 @@ def test_graph_hypergradient_matches_sum_over_paths(bt, act):
     bt.betty_hypergrad_graph(list(P), u2l, l2u, 1, [cfg, cfg, cfg], out2, ws)
     assert cb.rel_l2(out2, ref2) < TOL
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+@pytest.mark.parametrize("widths,B", [((24, 50, 7), 1), ((24, 50, 7), 129), ((8, 9, 3), 5), ((40, 130, 66, 12), 200)])
+def test_odd_widths_and_ragged_batches(bt, widths, B):
+    """Hidden widths and class counts that are not multiples of the tile or vector sizes, batches of
+    one and of one more than a tile: padded leading dimensions, zero fill and scalar epilogues."""
+    from tests import cuda_build as cb
+    inp = _perturb(si.reweight_bilevel(83, widths, B, 0.3, activation="gelu"), 83)
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    ws = bt.Workspace([w, th])
+    P = inp.w.size
+    out, outt = _vec(P), _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_grad(w, w, out, ws)
+    assert cb.rel_l2(out, oracle.grad(ow, ow)) < TOL
+    bt.betty_lower_step(w, 2, ws)
+    oracle.lower_step(ow, 2)
+    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    bt.betty_hypergrad_neumann(w, th, th, 2, 0.01, outt, ws)
+    assert cb.rel_l2(outt, oracle.hypergrad_neumann(ow, oth, oth, 2, 0.01)) < TOL_RANDOM_DIR
+    bt.betty_hypergrad_fd(w, th, th, 0.01, 1.0, outt, ws)
+    assert cb.rel_l2(outt, oracle.hypergrad_fd(ow, oth, oth, 0.01, 1.0)) < TOL_RANDOM_DIR
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
