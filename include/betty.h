@@ -94,6 +94,16 @@ typedef enum { BETTY_NEUMANN = 0, BETTY_CG = 1, BETTY_FD = 2 } betty_method;
 typedef enum { BETTY_ACT_RELU = 0, BETTY_ACT_GELU = 1 } betty_activation; /* GELU: erf form */
 typedef enum { BETTY_F32 = 0, BETTY_BF16 = 1, BETTY_I32 = 2 } betty_dtype;
 
+/* How a problem's gradient step is taken (the paper lets each problem bring its own optimiser: SGD with
+ * momentum and weight decay for the classifiers, Adam for the weight net, App. C).
+ *  GD      : x -= lr * g
+ *  MOMENTUM: g' = g + weight_decay * x;  buf = momentum * buf + g';  x -= lr * buf      (buf starts at 0)
+ *  ADAM    : g' = g + weight_decay * x;  m = b1 m + (1-b1) g';  v = b2 v + (1-b2) g'^2;  t += 1;
+ *            x -= lr * (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps)
+ * State lives in opt_state (device fp32, caller-owned, zero-initialised by the caller): MOMENTUM needs
+ * n_params floats, ADAM 2 * n_params + 1 (the last one counts steps). */
+typedef enum { BETTY_OPT_GD = 0, BETTY_OPT_MOMENTUM = 1, BETTY_OPT_ADAM = 2 } betty_optimizer;
+
 /* Approximation of one best-response Jacobian (Sec. 3.2).
  *  NEUMANN: q = alpha * sum_{j=0..K} (I - alpha H)^j v   (K Hessian-vector products)
  *  CG     : K iterations of conjugate gradient on H q = v from q = 0; stops early once
@@ -123,6 +133,11 @@ typedef struct betty_level {
   int32_t activation;   /* betty_activation (hidden layers) */
   float lr;             /* step size of betty_lower_step */
   float mu;             /* WEIGHTNET_DETECT ridge term */
+  int32_t optimizer;    /* betty_optimizer used by betty_lower_step and betty_engine_run */
+  float momentum;       /* MOMENTUM */
+  float beta1, beta2, adam_eps; /* ADAM */
+  float weight_decay;   /* MOMENTUM / ADAM: L2 term added to the gradient */
+  float* opt_state;     /* device fp32 state, see betty_optimizer; NULL for GD */
   int32_t n_constraints;
   const struct betty_level* const* constraints; /* host array: U_k and L_k providers */
 } betty_level;

@@ -7,7 +7,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from .solvers import chain_levels, grad
+from .solvers import apply_optimizer, chain_levels, grad
 
 
 def find_paths(u2l, l2u, k, targets):
@@ -46,7 +46,7 @@ def engine_run(levels, u2l, l2u, cfgs, unroll, n_iterations):
     """Execution of the whole program (Sec. 3.3).  Only the lowermost problems are stepped directly;
     a problem that has completed `unroll[j]` steps calls the problems it constrains through
     lower-to-upper edges; a called problem steps once every problem of its L set has called.  One
-    step of problem j is theta_j <- theta_j - lr_j * dC_j/d theta_j with the gradient of Eq. 2.
+    step of problem j is one step of its optimiser along the gradient of Eq. 2.
     Returns the list of problem indices in the order they stepped."""
     n = len(levels)
     n_lower = [sum(1 for a, b in l2u if b == j) for j in range(n)]
@@ -55,7 +55,7 @@ def engine_run(levels, u2l, l2u, cfgs, unroll, n_iterations):
     def step(j):
         log.append(j)
         g = hypergrad_graph(levels, u2l, l2u, j, cfgs)
-        levels[j].params = levels[j].params - levels[j].lr * g
+        apply_optimizer(levels[j], g)
         count[j] += 1
         if count[j] % unroll[j] == 0:
             for a, b in l2u:

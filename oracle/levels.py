@@ -50,6 +50,13 @@ class Level:
     mu: float = 0.0
     bf16: bool = False                 # MLP matrices are used through a bf16-rounded copy
     constraints: list = field(default_factory=list)
+    optimizer: str = "gd"              # 'gd' | 'momentum' | 'adam' (App. C: SGD with momentum / Adam per problem)
+    momentum: float = 0.0
+    beta1: float = 0.9
+    beta2: float = 0.999
+    adam_eps: float = 1e-8
+    weight_decay: float = 0.0
+    opt_state: dict = field(default_factory=dict)
 
     def __post_init__(self):
         self.params = np.array(self.params, dtype=np.float64).reshape(-1)

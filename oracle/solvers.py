@@ -29,13 +29,36 @@ hvp = _lv.hvp
 mixed_vjp = _lv.mixed_vjp
 
 
+def apply_optimizer(L: Level, g: np.ndarray) -> None:
+    """One step of the problem's optimiser along gradient g (App. C names SGD with momentum and weight
+    decay for the classifiers and Adam for the weight net; the update rules are the standard ones)."""
+    x = L.params
+    if L.optimizer == "gd":
+        L.params = x - L.lr * g
+        return
+    gg = g + L.weight_decay * x
+    st = L.opt_state
+    if L.optimizer == "momentum":
+        st["buf"] = L.momentum * st.get("buf", np.zeros_like(x)) + gg
+        L.params = x - L.lr * st["buf"]
+    elif L.optimizer == "adam":
+        st["t"] = st.get("t", 0) + 1
+        st["m"] = L.beta1 * st.get("m", np.zeros_like(x)) + (1.0 - L.beta1) * gg
+        st["v"] = L.beta2 * st.get("v", np.zeros_like(x)) + (1.0 - L.beta2) * gg * gg
+        mhat = st["m"] / (1.0 - L.beta1 ** st["t"])
+        vhat = st["v"] / (1.0 - L.beta2 ** st["t"])
+        L.params = x - L.lr * mhat / (np.sqrt(vhat) + L.adam_eps)
+    else:
+        raise ValueError(L.optimizer)
+
+
 def lower_step(L: Level, n_steps: int) -> None:
     """x <- x - lr * dC/dx, n_steps times on the level's fixed batch (Sec. 3.2: w* is
     approximated by a small number of unrolled gradient steps).  Updates L.params in place.
     For mixed-precision levels the gradient is taken at the bf16-rounded copy of the
     current master, which is re-derived at every step."""
     for _ in range(int(n_steps)):
-        L.params = L.params - L.lr * grad(L, L)
+        apply_optimizer(L, grad(L, L))
 
 
 def neumann_solve(hv, v, K: int, alpha: float) -> np.ndarray:
@@ -130,6 +153,8 @@ def hypergrad_itd(lower: Level, upper: Level, wrt: Level, n_steps: int) -> np.nd
 
     with H_t, M_t the second derivatives of the lower cost at x_t (same stop-gradient and
     quantisation conventions as `hvp` / `mixed_vjp`)."""
+    if lower.optimizer != "gd":
+        raise ValueError("ITD-RMAD differentiates plain gradient-descent steps")
     xs = []
     for _ in range(int(n_steps)):
         xs.append(lower.params.copy())

@@ -21,6 +21,7 @@ PARAM_VECTOR, PARAM_MLP, PARAM_WEIGHTNET, PARAM_LOGWD = range(4)
 BETTY_NEUMANN, BETTY_CG, BETTY_FD = range(3)
 ACT_RELU, ACT_GELU = range(2)
 BETTY_F32, BETTY_BF16, BETTY_I32 = range(3)
+BETTY_OPT_GD, BETTY_OPT_MOMENTUM, BETTY_OPT_ADAM = range(3)
 
 
 class BettyError(RuntimeError):
@@ -42,7 +43,9 @@ _Level._fields_ = [
     ("loss", C.c_int32), ("param_kind", C.c_int32), ("params", C.c_void_p), ("n_params", C.c_int64),
     ("X", C.c_void_p), ("x_dtype", C.c_int32), ("n", C.c_int64), ("d", C.c_int64),
     ("y", C.c_void_p), ("aux", C.c_void_p), ("n_layers", C.c_int32), ("widths", C.POINTER(C.c_int64)),
-    ("activation", C.c_int32), ("lr", C.c_float), ("mu", C.c_float), ("n_constraints", C.c_int32),
+    ("activation", C.c_int32), ("lr", C.c_float), ("mu", C.c_float), ("optimizer", C.c_int32),
+    ("momentum", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("adam_eps", C.c_float),
+    ("weight_decay", C.c_float), ("opt_state", C.c_void_p), ("n_constraints", C.c_int32),
     ("constraints", C.POINTER(C.POINTER(_Level))),
 ]
 
@@ -158,6 +161,8 @@ class Level:
         else:
             s.n_layers, s.widths = 0, None
         s.activation, s.lr, s.mu = int(activation), float(lr), float(mu)
+        s.optimizer, s.opt_state = BETTY_OPT_GD, None
+        self.opt_state = None
         s.n_constraints, s.constraints = 0, None
         self.c = s
 
@@ -166,6 +171,18 @@ class Level:
         self._carr = (C.POINTER(_Level) * max(1, len(levels)))(*[C.pointer(l.c) for l in levels])
         self.c.n_constraints = len(levels)
         self.c.constraints = self._carr if levels else None
+        return self
+
+    def set_optimizer(self, kind: int, momentum: float = 0.0, beta1: float = 0.9, beta2: float = 0.999,
+                      eps: float = 1e-8, weight_decay: float = 0.0) -> "Level":
+        """Chooses the optimiser of this problem's steps and allocates its zero-initialised state."""
+        n = self.params.numel()
+        size = {BETTY_OPT_GD: 0, BETTY_OPT_MOMENTUM: n, BETTY_OPT_ADAM: 2 * n + 1}[int(kind)]
+        self.opt_state = torch.zeros(max(size, 1), dtype=torch.float32, device=self.params.device) if size else None
+        self.c.optimizer, self.c.momentum = int(kind), float(momentum)
+        self.c.beta1, self.c.beta2, self.c.adam_eps = float(beta1), float(beta2), float(eps)
+        self.c.weight_decay = float(weight_decay)
+        self.c.opt_state = _ptr(self.opt_state)
         return self
 
     @property

@@ -29,6 +29,32 @@ __global__ void k_fd_weight_decay(float* out, const float* w, const float* v, co
     out[i] = base;
   }
 }
+// optimiser steps (see betty_optimizer); the step counter of Adam is the float behind the two moments
+__global__ void k_opt_momentum(float* x, const float* g, float* buf, float lr, float mom, float wd, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const float gg = g[i] + wd * x[i];
+    const float b = mom * buf[i] + gg;
+    buf[i] = b;
+    x[i] -= lr * b;
+  }
+}
+__global__ void k_opt_adam(float* x, const float* g, float* m, float* v, const float* tcount, float lr, float b1, float b2,
+                           float eps, float wd, int64_t n) {
+  const float t = *tcount + 1.f;                       // this step's index; the counter is advanced afterwards
+  const float c1 = 1.f - powf(b1, t), c2 = 1.f - powf(b2, t);
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const float gg = g[i] + wd * x[i];
+    const float mi = b1 * m[i] + (1.f - b1) * gg;
+    const float vi = b2 * v[i] + (1.f - b2) * gg * gg;
+    m[i] = mi; v[i] = vi;
+    x[i] -= lr * (mi / c1) / (sqrtf(vi / c2) + eps);
+  }
+}
+__global__ void k_opt_tick(float* tcount) { *tcount += 1.f; }
+__global__ void k_opt_gd(float* x, const float* g, float lr, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    x[i] -= lr * g[i];
+}
 static inline int ew_grid(int64_t n) {
   int64_t b = (n + 1023) / 1024;
   return (int)(b < 1 ? 1 : (b > 2368 ? 2368 : b));
@@ -107,6 +133,25 @@ betty_status vecfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
   return BETTY_OK;
 }
 
+// params of L <- one optimiser step along gradient g
+static betty_status apply_optimizer(Ctx& c, const betty_level* L, const float* g) {
+  const int64_t n = L->n_params;
+  if (n <= 0) return BETTY_OK;
+  const int grid = (int)((n + 1023) / 1024 < 1 ? 1 : ((n + 1023) / 1024 > 2368 ? 2368 : (n + 1023) / 1024));
+  if (L->optimizer == BETTY_OPT_GD) {
+    k_opt_gd<<<grid, 256, 0, c.stream>>>(L->params, g, L->lr, n);
+  } else if (L->optimizer == BETTY_OPT_MOMENTUM) {
+    k_opt_momentum<<<grid, 256, 0, c.stream>>>(L->params, g, L->opt_state, L->lr, L->momentum, L->weight_decay, n);
+  } else {
+    float* m = L->opt_state; float* v = m + n; float* t = v + n;
+    k_opt_adam<<<grid, 256, 0, c.stream>>>(L->params, g, m, v, t, L->lr, L->beta1, L->beta2, L->adam_eps, L->weight_decay, n);
+    BETTY_LAUNCH_CHECK();
+    k_opt_tick<<<1, 1, 0, c.stream>>>(t);
+  }
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
 // ------------------------------------------------------------------ dispatch
 static betty_status validate_level(const betty_level* L) {
   if (!L) return BETTY_ERR_INVALID_ARG;
@@ -115,6 +160,8 @@ static betty_status validate_level(const betty_level* L) {
     if (!L->constraints[i]) return BETTY_ERR_INVALID_ARG;
   if (L->n_params < 0 || (L->n_params > 0 && !L->params)) return BETTY_ERR_INVALID_ARG;
   if (L->param_kind < BETTY_PARAM_VECTOR || L->param_kind > BETTY_PARAM_LOGWD) return BETTY_ERR_INVALID_ARG;
+  if (L->optimizer < BETTY_OPT_GD || L->optimizer > BETTY_OPT_ADAM) return BETTY_ERR_INVALID_ARG;
+  if (L->optimizer != BETTY_OPT_GD && !L->opt_state) return BETTY_ERR_INVALID_ARG;
   if (is_vector_family(L->loss)) return vecfam_validate(L);
   if (is_mlp_family(L->loss)) return mlpfam_validate(L);
   return BETTY_ERR_INVALID_ARG;
@@ -225,6 +272,7 @@ static betty_status hypergrad_itd(const betty_level* lower, const betty_level* u
   BETTY_TRY(validate_level(lower));
   BETTY_TRY(validate_level(upper));
   if (!wrt || !out || n_steps < 0) return BETTY_ERR_INVALID_ARG;
+  if (lower->optimizer != BETTY_OPT_GD) return BETTY_ERR_UNSUPPORTED;   // the reverse sweep differentiates plain GD steps
   BETTY_TRY(check_ws(ws, ws_bytes));
   if (!is_participant(upper, lower) || !is_participant(upper, wrt) || !is_participant(lower, wrt) || wrt == lower)
     return BETTY_ERR_INVALID_ARG;
@@ -371,17 +419,13 @@ struct Engine {
   int32_t* log; int log_capacity; int n_logged;
   int n_lower[256]; bool has_child[256]; int count[256]; int ready[256];
 };
-__global__ void k_descent(float* x, const float* gvec, float lr, int64_t n) {
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
-    x[i] -= lr * gvec[i];
-}
 static betty_status engine_step(Engine& e, int j, int depth) {
   if (depth > 256) return BETTY_ERR_INVALID_ARG;
   const betty_level* L = e.levels[j];
   if (e.log && e.n_logged < e.log_capacity) e.log[e.n_logged] = j;
   e.n_logged += 1;
   const size_t mark = e.c->arena.mark();
-  const bool fused = !e.has_child[j] && (L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_QUADRATIC_WD ||
+  const bool fused = L->optimizer == BETTY_OPT_GD && !e.has_child[j] && (L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_QUADRATIC_WD ||
                                          L->loss == BETTY_LOSS_MLP_CE_REWEIGHT);
   if (fused) {
     BETTY_TRY(is_vector_family(L->loss) ? vecfam_lower_step(*e.c, L, 1) : mlpfam_lower_step(*e.c, L, 1));
@@ -389,8 +433,7 @@ static betty_status engine_step(Engine& e, int j, int depth) {
     float* gvec = e.c->arena.alloc<float>((size_t)L->n_params);
     if (!gvec) return BETTY_ERR_WORKSPACE;
     BETTY_TRY(graph_hypergrad(*e.c, e.levels, *e.g, j, e.cfg, gvec));
-    k_descent<<<ew_grid(L->n_params), 256, 0, e.c->stream>>>(L->params, gvec, L->lr, L->n_params);
-    BETTY_LAUNCH_CHECK();
+    BETTY_TRY(apply_optimizer(*e.c, L, gvec));
   }
   e.c->arena.release(mark);
   e.count[j] += 1;
@@ -551,6 +594,14 @@ betty_status betty_lower_step(const betty_level* L, int32_t n_steps, void* ws, s
   if (n_steps < 0) return BETTY_ERR_INVALID_ARG;
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
+  if (L->optimizer != BETTY_OPT_GD) {
+    BETTY_ALLOC(g, float, c, (size_t)L->n_params);
+    for (int s = 0; s < n_steps; ++s) {
+      BETTY_TRY(level_grad(c, L, L, g));
+      BETTY_TRY(apply_optimizer(c, L, g));
+    }
+    return BETTY_OK;
+  }
   if (is_vector_family(L->loss)) return vecfam_lower_step(c, L, n_steps);
   return mlpfam_lower_step(c, L, n_steps);
 }

@@ -1,0 +1,65 @@
+"""Optimiser variants of a problem's step (SGD with momentum and weight decay, Adam) on the GPU
+against the oracle, in betty_lower_step and inside the execution schedule."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from tests import oracle_build as ob
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bt():
+    import paper_2207_02849_b200 as bt
+    return bt
+
+
+KINDS = {"momentum": 1, "adam": 2}
+
+
+@pytest.mark.parametrize("kind", ["momentum", "adam"])
+def test_lower_steps_logistic(bt, kind):
+    from tests import cuda_build as cb
+    inp = si.logreg_bilevel(37, 500, 48, 60)
+    w, lam = cb.logreg_levels(inp)
+    ow, olam = ob.logreg_levels(inp)
+    w.c.lr = ow.lr = 0.05
+    w.set_optimizer(KINDS[kind], momentum=0.9, weight_decay=0.01)
+    ow.optimizer, ow.momentum, ow.weight_decay = kind, 0.9, 0.01
+    ws = bt.Workspace([w, lam])
+    bt.betty_lower_step(w, 12, ws)
+    oracle.lower_step(ow, 12)
+    assert cb.rel_l2(w.params, ow.params) < 1e-4
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+    out = torch.empty(48, dtype=torch.float32, device="cuda")
+    with pytest.raises(bt.BettyError) as e:          # the reverse sweep of ITD assumes plain gradient steps
+        bt.betty_hypergrad_itd(w, lam, lam, 2, out, ws)
+    assert e.value.status == bt.BETTY_ERR_UNSUPPORTED
+
+
+def test_reweighting_run_with_momentum_classifier_and_adam_weight_net(bt):
+    """The optimiser pairing of the data-reweighting experiment (App. C): SGD with momentum and weight
+    decay for the classifier, Adam for the weight net, run through the execution schedule."""
+    from tests import cuda_build as cb
+    from tests.test_gpu_mlp import _perturb
+    inp = _perturb(si.reweight_bilevel(91, (64, 96, 10), 128, 0.4, activation="relu"), 91)
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    w.c.lr = ow.lr = 0.1
+    th.c.lr = oth.lr = 1e-3
+    w.set_optimizer(bt.BETTY_OPT_MOMENTUM, momentum=0.9, weight_decay=5e-4)
+    ow.optimizer, ow.momentum, ow.weight_decay = "momentum", 0.9, 5e-4
+    th.set_optimizer(bt.BETTY_OPT_ADAM)
+    oth.optimizer = "adam"
+    ws = bt.Workspace([w, th])
+    u2l, l2u = [(1, 0)], [(0, 1)]
+    cfg, ocfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=3, alpha=0.01), dict(method="neumann", K=3, alpha=0.01)
+    log = bt.betty_engine_run([w, th], u2l, l2u, [cfg, cfg], [2, 1], 4, ws)
+    assert log == oracle.engine_run([ow, oth], u2l, l2u, [ocfg, ocfg], [2, 1], 4) == [0, 0, 1, 0, 0, 1]
+    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    # Adam's first steps have magnitude lr whatever the gradient scale, so theta's displacement is well resolved
+    assert cb.rel_l2(th.params - cb.dev(inp.theta), oth.params - inp.theta.astype(np.float64)) < 3e-2
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK

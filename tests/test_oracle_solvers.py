@@ -301,3 +301,26 @@ def test_three_level_chain_equals_product_of_materialised_jacobians():
     assert rel(out_nm, (-T1 @ M1lam).T @ ((-T2 @ M2w).T @ v_th)) < 1e-9
     # a wrong order of the factors or a missing transpose would not even have this shape
     assert out_nm.shape == (2,)
+
+
+# ------------------------------------------------------------------ optimiser variants
+@pytest.mark.parametrize("kind", ["momentum", "adam"])
+def test_optimizer_steps_match_torch_optim(kind):
+    """lower_step with SGD-momentum / Adam against torch.optim on autodiff gradients of the same cost."""
+    inp = si.logreg_bilevel(29, 40, 5, 10)
+    inp.w0 = si.normal_f32(29, 9, (5,)) * 0.3
+    inp.lam = (np.abs(si.normal_f32(29, 7, (5,))) * 0.1 + 0.02).astype(np.float32)
+    lo, up = logreg_levels(inp)
+    lo.optimizer, lo.lr, lo.weight_decay = kind, 0.05, 0.01
+    lo.momentum = 0.9
+    w = _t(inp.w0).requires_grad_(True)
+    opt = (torch.optim.SGD([w], lr=0.05, momentum=0.9, weight_decay=0.01) if kind == "momentum"
+           else torch.optim.Adam([w], lr=0.05, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.01))
+    X, y, lam = _t(inp.X), _t(inp.y), _t(inp.lam)
+    for _ in range(6):
+        opt.zero_grad()
+        c = torch.nn.functional.softplus(-y * (X @ w)).mean() + 0.5 * (lam * w * w).sum()
+        c.backward()
+        opt.step()
+    oracle.lower_step(lo, 6)
+    assert rel(lo.params, w.detach().numpy()) < 1e-10
