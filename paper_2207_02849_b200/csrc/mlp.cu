@@ -245,15 +245,22 @@ __global__ void k_wn_sample(int mode, const float* theta, const float* dir, cons
     case WN_DETECT_WMIXED: out1[i] = (fpp * dsdl * Jd + fp * dJd) * invB; break;
   }
 }
-// One block, thread k owns hidden unit k:  out = sum_i cA_i * ds_i/dtheta + cB_i * (d2s_i/dtheta2 . dir) + mu*muvec
+// out = sum_i cA_i * ds_i/dtheta + cB_i * (d2s_i/dtheta2 . dir) + mu*muvec.  Thread k owns hidden unit k;
+// block b sums its slice of the samples (fp64), the block that draws the last ticket adds the per-block
+// partial sums in block order: the result does not depend on scheduling.
+static constexpr int WN_MAX_BLOCKS = 64;
+static constexpr int WN_STRIDE = 304;    // doubles per block in the partial buffer
 __global__ void k_wn_backward(const float* theta, const float* dir, const float* ell, const float* cA, const float* cB,
-                              int64_t B, float mu, const float* muvec, float* out, int accumulate, float out_scale) {
+                              int64_t B, float mu, const float* muvec, float* out, int accumulate, float out_scale,
+                              double* partial, unsigned* counter) {
   const int k = threadIdx.x;
+  const int64_t per = (B + gridDim.x - 1) / gridDim.x;
+  const int64_t i0 = blockIdx.x * per, i1 = (i0 + per < B) ? i0 + per : B;
   double ga1 = 0.0, gb1 = 0.0, ga2 = 0.0, gb2 = 0.0;
   if (k < WN_H) {
     const float a1 = theta[k], b1 = theta[WN_H + k], a2 = theta[2 * WN_H + k];
     const float da1 = dir ? dir[k] : 0.f, db1 = dir ? dir[WN_H + k] : 0.f, da2 = dir ? dir[2 * WN_H + k] : 0.f;
-    for (int64_t i = 0; i < B; ++i) {
+    for (int64_t i = i0; i < i1; ++i) {
       const float l = ell[i], ca = cA[i], cb = cB ? cB[i] : 0.f;
       const float pre = a1 * l + b1;
       if (pre > 0.f) {
@@ -264,14 +271,30 @@ __global__ void k_wn_backward(const float* theta, const float* dir, const float*
       }
     }
   } else if (k == WN_H) {
-    for (int64_t i = 0; i < B; ++i) gb2 += (double)cA[i];
+    for (int64_t i = i0; i < i1; ++i) gb2 += (double)cA[i];
   }
-  auto put = [&](int idx, double g) {
-    float v = out_scale * ((float)g + (muvec ? mu * muvec[idx] : 0.f));
+  double* mine = partial + (size_t)blockIdx.x * WN_STRIDE;
+  if (k < WN_H) { mine[k] = ga1; mine[WN_H + k] = gb1; mine[2 * WN_H + k] = ga2; }
+  else if (k == WN_H) mine[3 * WN_H] = gb2;
+  __shared__ bool is_last;
+  __threadfence();
+  __syncthreads();
+  if (k == 0) is_last = atomicAdd(counter, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  auto total = [&](int idx) {
+    double t = 0.0;
+    for (unsigned bb = 0; bb < gridDim.x; ++bb) t += ((volatile double*)partial)[(size_t)bb * WN_STRIDE + idx];
+    return t;
+  };
+  auto put = [&](int idx) {
+    float v = out_scale * ((float)total(idx) + (muvec ? mu * muvec[idx] : 0.f));
     out[idx] = (accumulate ? out[idx] : 0.f) + v;
   };
-  if (k < WN_H) { put(k, ga1); put(WN_H + k, gb1); put(2 * WN_H + k, ga2); }
-  else if (k == WN_H) put(3 * WN_H, gb2);
+  if (k < WN_H) { put(k); put(WN_H + k); put(2 * WN_H + k); }
+  else if (k == WN_H) put(3 * WN_H);
+  if (k == 0) *counter = 0u;
 }
 
 // ------------------------------------------------------------------ finite-difference pieces
@@ -583,9 +606,16 @@ static betty_status wn_sample(Ctx& c, int mode, const betty_level* theta, const 
 static betty_status wn_backward(Ctx& c, const betty_level* theta, const float* dir, const Pass& ps, const float* cA,
                                 const float* cB, float mu, const float* muvec, float* out, bool accumulate = false,
                                 float out_scale = 1.f) {
-  k_wn_backward<<<1, 128, 0, c.stream>>>(theta->params, dir, ps.ell, cA, cB, ps.B, mu, muvec, out, accumulate ? 1 : 0,
-                                         out_scale);
+  int nb = (int)((ps.B + 15) / 16);
+  nb = nb < 1 ? 1 : (nb > WN_MAX_BLOCKS ? WN_MAX_BLOCKS : nb);
+  const size_t mark = c.arena.mark();
+  BETTY_ALLOC(partial, double, c, (size_t)nb * WN_STRIDE);
+  BETTY_ALLOC(counter, unsigned, c, 8);
+  if (cudaMemsetAsync(counter, 0, 32, c.stream) != cudaSuccess) return BETTY_ERR_CUDA;
+  k_wn_backward<<<nb, 128, 0, c.stream>>>(theta->params, dir, ps.ell, cA, cB, ps.B, mu, muvec, out, accumulate ? 1 : 0,
+                                          out_scale, partial, counter);
   BETTY_LAUNCH_CHECK();
+  c.arena.release(mark);
   return BETTY_OK;
 }
 
