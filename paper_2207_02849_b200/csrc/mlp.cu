@@ -183,13 +183,16 @@ __global__ void k_wd_add_f32(float* out, const float* u, int64_t n, const float*
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     out[i] += k * u[i];
 }
-// one block: out (+)= scale * exp(lam) * <W, q>  (q == nullptr: <W, W>), fixed summation order
+// out (+)= scale * exp(lam) * <W, q>  (q == nullptr: <W, W>).  Each block sums a slice in fp64; the block
+// that draws the last ticket adds the per-block sums in block order (fixed summation order).
+static constexpr int LD_MAX_BLOCKS = 128;
 __global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
-                            float scale, float* out, int accumulate) {
+                            float scale, float* out, int accumulate, double* partial, unsigned* counter) {
   __shared__ double sh[32];
+  __shared__ bool is_last;
   double acc = 0.0;
   const int64_t total = rows * cols;
-  for (int64_t i = threadIdx.x; i < total; i += blockDim.x) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / cols, c = i - r * cols;
     const float w = __bfloat162float(W[r * ldw + c]);
     acc += (double)w * (double)(q ? q[i] : w);
@@ -200,9 +203,31 @@ __global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t l
   if (threadIdx.x == 0) {
     double t = 0.0;
     for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += sh[i];
-    const float v = scale * expf(*lam) * (float)t;
-    *out = (accumulate ? *out : 0.f) + v;
+    partial[blockIdx.x] = t;
+    __threadfence();
+    is_last = atomicAdd(counter, 1u) == gridDim.x - 1;
+    if (is_last) {
+      __threadfence();
+      double tot = 0.0;
+      for (unsigned bb = 0; bb < gridDim.x; ++bb) tot += ((volatile double*)partial)[bb];
+      const float v = scale * expf(*lam) * (float)tot;
+      *out = (accumulate ? *out : 0.f) + v;
+      *counter = 0u;
+    }
   }
+}
+static betty_status layer_dot(Ctx& c, const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
+                              float scale, float* out, bool accumulate) {
+  int64_t nb = (rows * cols + 256 * 16 - 1) / (256 * 16);
+  nb = nb < 1 ? 1 : (nb > LD_MAX_BLOCKS ? LD_MAX_BLOCKS : nb);
+  const size_t mark = c.arena.mark();
+  BETTY_ALLOC(partial, double, c, (size_t)nb);
+  BETTY_ALLOC(counter, unsigned, c, 8);
+  if (cudaMemsetAsync(counter, 0, 32, c.stream) != cudaSuccess) return BETTY_ERR_CUDA;
+  k_layer_dot<<<(unsigned)nb, 256, 0, c.stream>>>(W, rows, cols, ldw, q, lam, scale, out, accumulate ? 1 : 0, partial, counter);
+  BETTY_LAUNCH_CHECK();
+  c.arena.release(mark);
+  return BETTY_OK;
 }
 
 // ------------------------------------------------------------------ weight net 1-100-1
@@ -638,8 +663,7 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
   BETTY_TRY(net_setup(c, P.mlp, n));
   if (P.lam && wrt == P.lam) {
     for (int l = 0; l < n.L; ++l) {
-      k_layer_dot<<<1, 1024, 0, c.stream>>>(n.W[l], n.w[l + 1], n.w[l], n.ldw[l], nullptr, P.lam->params + l, 0.5f, out + l, 0);
-      BETTY_LAUNCH_CHECK();
+      BETTY_TRY(layer_dot(c, n.W[l], n.w[l + 1], n.w[l], n.ldw[l], nullptr, P.lam->params + l, 0.5f, out + l, false));
     }
     c.arena.release(mark);
     return BETTY_OK;
@@ -785,9 +809,7 @@ betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const be
   if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
     if (P.lam && wrt == P.lam) {
       for (int l = 0; l < n.L; ++l) {
-        k_layer_dot<<<1, 1024, 0, c.stream>>>(n.W[l], n.w[l + 1], n.w[l], n.ldw[l], q + n.woff[l], P.lam->params + l, 1.f,
-                                              out + l, 0);
-        BETTY_LAUNCH_CHECK();
+        BETTY_TRY(layer_dot(c, n.W[l], n.w[l + 1], n.w[l], n.ldw[l], q + n.woff[l], P.lam->params + l, 1.f, out + l, false));
       }
     } else if (P.theta && wrt == P.theta) {
       RPass rp;
@@ -859,9 +881,7 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
     // dC/d(lam_l) = 1/2 exp(lam_l)|W_l|^2 is quadratic in W: its central difference is exactly
     // exp(lam_l) <W_l, V_l> for every eps, which is what is evaluated.
     for (int l = 0; l < n.L; ++l) {
-      k_layer_dot<<<1, 1024, 0, c.stream>>>(n.W[l], n.w[l + 1], n.w[l], n.ldw[l], v + n.woff[l], P.lam->params + l, -alpha,
-                                            out + l, accumulate ? 1 : 0);
-      BETTY_LAUNCH_CHECK();
+      BETTY_TRY(layer_dot(c, n.W[l], n.w[l + 1], n.w[l], n.ldw[l], v + n.woff[l], P.lam->params + l, -alpha, out + l, accumulate));
     }
     c.arena.release(mark);
     return BETTY_OK;
