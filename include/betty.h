@@ -235,7 +235,8 @@ betty_status betty_hvp_logreg_static(const float* X, int64_t n, int64_t d, const
  * [M,K] (a_transposed = 0) or [K,M] (a_transposed = 1); logical B is [K,N]: stored [K,N]
  * (b_transposed = 0) or [N,K] (b_transposed = 1); lda/ldb are leading dimensions in elements.
  * path: 0 = library's choice, 1 = CUDA-core kernel, 2 = tensor-core (tcgen05) kernel, 3 = its two-SM
- * (cta_group::2) form; the tensor-core kernels need 16-byte aligned operands, lda/ldb multiples of 8 and alpha = +-1 (else BETTY_ERR_UNSUPPORTED).
+ * (cta_group::2) form, both holding C transposed in tensor memory so that the epilogue's accesses
+ * coalesce; 4 and 5 = the same two kernels with one accumulator row per thread; the tensor-core kernels need 16-byte aligned operands, lda/ldb multiples of 8 and alpha = +-1 (else BETTY_ERR_UNSUPPORTED).
  * All pointers are device pointers; `pairs` is host memory. */
 typedef struct {
   const void* A; int64_t lda; int32_t a_transposed;

@@ -100,5 +100,7 @@ extern "C" betty_status betty_gemm_bf16(int32_t M, int32_t N, int32_t n_pairs, c
   if (path == 1) return gemm_simt(c, g);
   if (path == 2) return gemm_tc_eligible(g) ? gemm_tc(c, g) : BETTY_ERR_UNSUPPORTED;
   if (path == 3) return gemm_tc_eligible(g) ? gemm_tc_pair(c, g) : BETTY_ERR_UNSUPPORTED;
+  if (path == 4) return gemm_tc_eligible(g) ? gemm_tc(c, g, false) : BETTY_ERR_UNSUPPORTED;
+  if (path == 5) return gemm_tc_eligible(g) ? gemm_tc_pair(c, g, false) : BETTY_ERR_UNSUPPORTED;
   return gemm(c, g);
 }

@@ -19,7 +19,7 @@ enum GemmEpiMode {
   EPI_ACT_BWD = 2,   // C = acc (if C);     out16 = acc * act'(a[m,n])                   (backward through an activation)
   EPI_R_FWD = 3,     // v = acc + bias[n];  C = v;  out16 = act'(a[m,n]) * v             (R-operator forward)
   EPI_R_BWD = 4,     // out16 = acc * act'(a) + dh * act''(a) * Ra                       (R-operator backward)
-  EPI_SGD = 5,       // g = acc + exp(lam) * w16;  C = C - lr * g;  out16 = bf16(new C)  (weight gradient -> gradient step)
+  EPI_SGD = 5,       // g = acc + exp(lam) * w16;  C = C - lr * g;  out16 = bf16(new C)  (weight gradient -> gradient step; w16 == bf16(C))
   EPI_NEUMANN = 6    // Hu = acc + exp(lam) * t_in;  t = t_in - alpha * Hu -> C;  s_out = s_in + t   (weight HVP -> series update)
 };
 struct GemmEpilogue {
@@ -117,8 +117,10 @@ betty_status gemm(Ctx& c, const GemmDesc& g);
 // tcgen05 / tensor-memory path (gemm_tc.cu): needs 16-byte aligned operands, leading dimensions that
 // are multiples of 8 elements and alpha = +-1
 bool gemm_tc_eligible(const GemmDesc& g);
-betty_status gemm_tc(Ctx& c, const GemmDesc& g);
-betty_status gemm_tc_pair(Ctx& c, const GemmDesc& g);   // two-SM (cta_group::2) kernel, 256 x 256 tiles
+// tr: keep C transposed in tensor memory (operand roles exchanged) so that the epilogue's global accesses
+// coalesce; false: one accumulator row per thread.
+betty_status gemm_tc(Ctx& c, const GemmDesc& g, bool tr = true);
+betty_status gemm_tc_pair(Ctx& c, const GemmDesc& g, bool tr = true);   // two-SM (cta_group::2) kernel, 256 x 256 tiles
 // CUDA-core reference path (any shape, any stride); also the fallback for shapes the tensor-core
 // path does not take.
 betty_status gemm_simt(Ctx& c, const GemmDesc& g);

@@ -34,6 +34,7 @@ struct TcArgs {
   float* C; int64_t ldc; float beta;
   GemmEpilogue epi;
   int vec_ok;            // every pointer the epilogue touches is 16-byte aligned and N, ldc, ld16 allow vector access
+  int tr;                // the accumulator holds C transposed: lane = column of C, accumulator column = row of C
   StatusBlock* sb;
 };
 
@@ -194,9 +195,108 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
       }
     }
   } else {
-#pragma unroll 4
+#pragma unroll   // constant indices keep r in registers
     for (int jj = 0; jj < 32; ++jj)
       if (nb + jj < g.N) gemm_epilogue_store(e, g.C, g.ldc, g.beta, g.N, m, nb + jj, __uint_as_float(r[jj]));
+  }
+}
+
+// Transposed accumulator (tr): the host swapped the operand roles, so this thread's accumulator lane is
+// column n of C and r holds rows mb .. mb+31 of that column.  For a fixed row the 32 lanes of a warp
+// touch 32 consecutive elements of C and of every epilogue input: each access is one full 128-byte
+// line per warp (64 bytes for the bf16 outputs) instead of 32 separate lines.
+// C is [MC, NC] = [g.N, g.M] here.  Loads of a batch of rows are issued before its stores.  Mode and
+// activation are compile-time parameters: one compact loop per case.
+template <int MODE, int ACT>
+__device__ __forceinline__ void epilogue_t32_impl(const TcArgs& g, int n, int mb, const uint32_t (&r)[32]) {
+  const GemmEpilogue& e = g.epi;
+  const int MC = g.N, NC = g.M;
+  constexpr int U = 8;
+  const float bias = (MODE == EPI_BIAS_ACT || MODE == EPI_R_FWD) ? e.bias[n] : 0.f;
+  const float kap = ((MODE == EPI_SGD || MODE == EPI_NEUMANN) && e.lam) ? expf(*e.lam) : 0.f;
+  float* cp = g.C ? g.C + (int64_t)mb * g.ldc + n : nullptr;
+  const float* ap = e.a ? e.a + (int64_t)mb * NC + n : nullptr;
+  const float* dp = e.dh ? e.dh + (int64_t)mb * NC + n : nullptr;
+  const float* qp = e.Ra ? e.Ra + (int64_t)mb * NC + n : nullptr;
+  const float* tp = e.t_in ? e.t_in + (int64_t)mb * g.ldc + n : nullptr;
+  const float* sp = e.s_in ? e.s_in + (int64_t)mb * g.ldc + n : nullptr;
+  float* so = e.s_out ? e.s_out + (int64_t)mb * g.ldc + n : nullptr;
+  bf16* op = e.out16 ? e.out16 + (int64_t)mb * e.ld16 + n : nullptr;
+  const int rows = MC - mb;     // > 0
+  const bool second = MODE == EPI_R_BWD && ACT != BETTY_ACT_RELU;
+#pragma unroll
+  for (int j0 = 0; j0 < 32; j0 += U) {
+    float x0[U], x1[U], x2[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+      const int j = j0 + k;
+      x0[k] = 0.f; x1[k] = 0.f; x2[k] = 0.f;
+      if (j < rows) {
+        if (MODE == EPI_STORE) { if (g.beta != 0.f) x0[k] = cp[(int64_t)j * g.ldc]; }
+        if (MODE == EPI_R_FWD) { if (op) x0[k] = ap[(int64_t)j * NC]; }
+        if (MODE == EPI_ACT_BWD || MODE == EPI_R_BWD) x0[k] = ap[(int64_t)j * NC];
+        if (second) { x1[k] = dp[(int64_t)j * NC]; x2[k] = qp[(int64_t)j * NC]; }
+        if (MODE == EPI_SGD) x0[k] = cp[(int64_t)j * g.ldc];
+        if (MODE == EPI_NEUMANN) { x0[k] = tp[(int64_t)j * g.ldc]; x1[k] = sp[(int64_t)j * g.ldc]; }
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+      const int j = j0 + k;
+      if (j < rows) {
+        const float acc = __uint_as_float(r[j]);
+        float* c1 = cp + (int64_t)j * g.ldc;
+        bf16* o1 = op + (int64_t)j * e.ld16;
+        if (MODE == EPI_STORE) *c1 = acc + g.beta * x0[k];
+        if (MODE == EPI_BIAS_ACT) {
+          const float v = acc + bias;
+          *c1 = v;
+          if (op) *o1 = __float2bfloat16_rn(act_f(ACT, v));
+        }
+        if (MODE == EPI_R_FWD) {
+          const float v = acc + bias;
+          *c1 = v;
+          if (op) *o1 = __float2bfloat16_rn(act_d1(ACT, x0[k]) * v);
+        }
+        if (MODE == EPI_ACT_BWD) {
+          if (cp) *c1 = acc;
+          *o1 = __float2bfloat16_rn(acc * act_d1(ACT, x0[k]));
+        }
+        if (MODE == EPI_R_BWD) {
+          float v = acc * act_d1(ACT, x0[k]);
+          if (second) v += x1[k] * act_d2(ACT, x0[k]) * x2[k];
+          *o1 = __float2bfloat16_rn(v);
+        }
+        if (MODE == EPI_SGD) {
+          // the bf16 weights the gradient was taken at (w16) are the rounded master weights: no second read
+          const float wq = __bfloat162float(__float2bfloat16_rn(x0[k]));
+          const float w = x0[k] - e.step * (acc + kap * wq);
+          *c1 = w;
+          if (op) *o1 = __float2bfloat16_rn(w);
+        }
+        if (MODE == EPI_NEUMANN) {
+          const float tn = x0[k] - e.step * (acc + kap * x0[k]);
+          *c1 = tn;
+          so[(int64_t)j * g.ldc] = x1[k] + tn;
+        }
+      }
+    }
+  }
+}
+template <int MODE>
+__device__ __forceinline__ void epilogue_t32_act(const TcArgs& g, int n, int mb, const uint32_t (&r)[32]) {
+  if (g.epi.act == BETTY_ACT_RELU) epilogue_t32_impl<MODE, BETTY_ACT_RELU>(g, n, mb, r);
+  else epilogue_t32_impl<MODE, BETTY_ACT_GELU>(g, n, mb, r);
+}
+__device__ __forceinline__ void epilogue_t32(const TcArgs& g, int n, int mb, const uint32_t (&r)[32]) {
+  switch (g.epi.mode) {
+    case EPI_STORE: epilogue_t32_impl<EPI_STORE, BETTY_ACT_RELU>(g, n, mb, r); break;
+    case EPI_BIAS_ACT: epilogue_t32_act<EPI_BIAS_ACT>(g, n, mb, r); break;
+    case EPI_ACT_BWD: epilogue_t32_act<EPI_ACT_BWD>(g, n, mb, r); break;
+    case EPI_R_FWD: epilogue_t32_act<EPI_R_FWD>(g, n, mb, r); break;
+    case EPI_R_BWD: epilogue_t32_act<EPI_R_BWD>(g, n, mb, r); break;
+    case EPI_SGD: epilogue_t32_impl<EPI_SGD, BETTY_ACT_RELU>(g, n, mb, r); break;
+    case EPI_NEUMANN: epilogue_t32_impl<EPI_NEUMANN, BETTY_ACT_RELU>(g, n, mb, r); break;
   }
 }
 
@@ -326,7 +426,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
           uint32_t r[32];
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32);
           tmem_load32(r, taddr);
-          if (m < g.M) epilogue_row32(g, m, n0 + c * 32, r);
+          if (m < g.M) {
+            if (g.tr) epilogue_t32(g, m, n0 + c * 32, r);
+            else epilogue_row32(g, m, n0 + c * 32, r);
+          }
         }
         // this warp has drained its quarter of the accumulator: the MMA warp may reuse it
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -334,7 +437,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
         if (lane == 0) tc_arrive(&acc_empty[as]);
       } else if (m < g.M) {
         // no products: the accumulator is zero
-        for (int n = n0; n < n0 + BN && n < g.N; ++n) gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.N, m, n, 0.f);
+        for (int n = n0; n < n0 + BN && n < g.N; ++n) {
+          if (g.tr) gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.M, n, m, 0.f);
+          else gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.N, m, n, 0.f);
+        }
       }
     }
   }
@@ -501,7 +607,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUt
           uint32_t r[32];
           const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * BN + c * 32);
           tmem_load32(r, taddr);
-          if (m < g.M) epilogue_row32(g, m, n0 + c * 32, r);
+          if (m < g.M) {
+            if (g.tr) epilogue_t32(g, m, n0 + c * 32, r);
+            else epilogue_row32(g, m, n0 + c * 32, r);
+          }
         }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
@@ -510,7 +619,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUt
           asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
         }
       } else if (m < g.M) {
-        for (int n = n0; n < n0 + BN && n < g.N; ++n) gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.N, m, n, 0.f);
+        for (int n = n0; n < n0 + BN && n < g.N; ++n) {
+          if (g.tr) gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.M, n, m, 0.f);
+          else gemm_epilogue_store(g.epi, g.C, g.ldc, g.beta, g.N, m, n, 0.f);
+        }
       }
     }
   }
@@ -571,11 +683,24 @@ bool gemm_tc_eligible(const GemmDesc& g) {
   return encode_fn() != nullptr;
 }
 
-static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a);
+static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a, bool tr);
+
+// C^T = B^T A^T: the same products with the operand roles exchanged.  The kernels then hold C transposed
+// in tensor memory (lane = column of C), which is what the coalesced epilogue wants.
+static GemmDesc swapped(const GemmDesc& g) {
+  GemmDesc s = g;
+  s.M = g.N; s.N = g.M;
+  for (int i = 0; i < g.npairs; ++i) {
+    const GemmPair& p = g.p[i];
+    s.p[i] = gemm_pair(p.B, p.ldb, !p.tb, p.A, p.lda, !p.ta, p.K, p.alpha);
+  }
+  return s;
+}
 
 template <int BN>
-static betty_status launch_tc(Ctx& c, const GemmDesc& g) {
+static betty_status launch_tc(Ctx& c, const GemmDesc& g0, bool tr) {
   using Cfg = TcCfg<BN>;
+  const GemmDesc g = tr ? swapped(g0) : g0;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k_gemm_tc<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM) != cudaSuccess) return BETTY_ERR_CUDA;
@@ -583,7 +708,7 @@ static betty_status launch_tc(Ctx& c, const GemmDesc& g) {
   }
   CUtensorMap tm[4];
   TcArgs a;
-  fill_args(c, g, a);
+  fill_args(c, g, a, tr);
   for (int i = 0; i < 2; ++i) {
     const GemmPair& p = g.p[i < g.npairs ? i : 0];
     // A: K-major = stored [M,K]; M-major = stored [K,M]
@@ -600,7 +725,8 @@ static betty_status launch_tc(Ctx& c, const GemmDesc& g) {
   return BETTY_OK;
 }
 
-static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a) {
+static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a, bool tr) {
+  a.tr = tr ? 1 : 0;
   a.M = g.M; a.N = g.N; a.npairs = g.npairs; a.C = g.C; a.ldc = g.ldc; a.beta = g.beta; a.sb = c.arena.status();
   a.epi = g.epi;
   auto al16 = [](const void* p) { return (((uintptr_t)p) & 15) == 0; };
@@ -618,7 +744,8 @@ static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a) {
   }
 }
 
-static betty_status launch_tc2(Ctx& c, const GemmDesc& g) {
+static betty_status launch_tc2(Ctx& c, const GemmDesc& g0, bool tr) {
+  const GemmDesc g = tr ? swapped(g0) : g0;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k_gemm_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, TC2_SMEM) != cudaSuccess) return BETTY_ERR_CUDA;
@@ -626,7 +753,7 @@ static betty_status launch_tc2(Ctx& c, const GemmDesc& g) {
   }
   CUtensorMap tm[4];
   TcArgs a;
-  fill_args(c, g, a);
+  fill_args(c, g, a, tr);
   for (int i = 0; i < 2; ++i) {
     const GemmPair& p = g.p[i < g.npairs ? i : 0];
     bool ok = p.ta ? make_map(&tm[2 * i], p.A, g.M, p.K, p.lda, 64, 64) : make_map(&tm[2 * i], p.A, p.K, g.M, p.lda, TC_BK, TC_BM);
@@ -642,16 +769,17 @@ static betty_status launch_tc2(Ctx& c, const GemmDesc& g) {
   return BETTY_OK;
 }
 
-betty_status gemm_tc_pair(Ctx& c, const GemmDesc& g) { return launch_tc2(c, g); }
+betty_status gemm_tc_pair(Ctx& c, const GemmDesc& g, bool tr) { return launch_tc2(c, g, tr); }
 
-betty_status gemm_tc(Ctx& c, const GemmDesc& g) {
-  // wide tiles unless the problem is narrow or would leave most SMs without a tile
+betty_status gemm_tc(Ctx& c, const GemmDesc& g0, bool tr) {
+  const GemmDesc g = tr ? swapped(g0) : g0;    // tile counts are taken in the kernel's own orientation
   // many tiles per SM (weight-gradient shapes): the two-SM kernel halves the B traffic per SM and measured faster
   const int pair_tiles = ((g.N + TC2_BN - 1) / TC2_BN) * ((g.M + 2 * TC_BM - 1) / (2 * TC_BM));
-  if (pair_tiles >= 2 * (c.sm_count / 2)) return launch_tc2(c, g);
+  if (pair_tiles >= 2 * (c.sm_count / 2)) return launch_tc2(c, g0, tr);
+  // wide tiles unless the problem is narrow or would leave most SMs without a tile
   const int tiles256 = ((g.N + 255) / 256) * ((g.M + TC_BM - 1) / TC_BM);
-  if (g.N > 128 && tiles256 >= 96) return launch_tc<256>(c, g);
-  return launch_tc<128>(c, g);
+  if (g.N > 128 && tiles256 >= 96) return launch_tc<256>(c, g0, tr);
+  return launch_tc<128>(c, g0, tr);
 }
 
 }  // namespace betty

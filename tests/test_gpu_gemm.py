@@ -34,7 +34,7 @@ SHAPES = [(128, 128, 64), (256, 384, 192), (200, 136, 104), (512, 10, 1024), (10
           (300, 1000, 72), (64, 4096, 8), (130, 70, 1000)]
 
 
-@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("path", [1, 2, 3, 4, 5])
 @pytest.mark.parametrize("ta,tb", [(0, 1), (0, 0), (1, 0), (1, 1)])
 @pytest.mark.parametrize("M,N,K", SHAPES)
 def test_single_product(path, ta, tb, M, N, K):
@@ -56,7 +56,7 @@ def test_single_product(path, ta, tb, M, N, K):
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 1e-5
 
 
-@pytest.mark.parametrize("path", [1, 2, 3])
+@pytest.mark.parametrize("path", [1, 2, 3, 4, 5])
 def test_two_products_negation_and_beta(path):
     import paper_2207_02849_b200 as bt
     M, N, K1, K2 = 200, 264, 136, 72
