@@ -35,6 +35,7 @@ struct TcArgs {
   GemmEpilogue epi;
   int vec_ok;            // every pointer the epilogue touches is 16-byte aligned and N, ldc, ld16 allow vector access
   int tr;                // the accumulator holds C transposed: lane = column of C, accumulator column = row of C
+  int pf_ok;             // transposed mode: the epilogue's fp32 inputs are pulled into L2 one tile ahead
   StatusBlock* sb;
 };
 
@@ -205,13 +206,15 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
 // column n of C and r holds rows mb .. mb+31 of that column.  For a fixed row the 32 lanes of a warp
 // touch 32 consecutive elements of C and of every epilogue input: each access is one full 128-byte
 // line per warp (64 bytes for the bf16 outputs) instead of 32 separate lines.
-// C is [MC, NC] = [g.N, g.M] here.  Loads of a batch of rows are issued before its stores.  Mode and
-// activation are compile-time parameters: one compact loop per case.
-template <int MODE, int ACT>
-__device__ __forceinline__ void epilogue_t32_impl(const TcArgs& g, int n, int mb, const uint32_t (&r)[32]) {
+// C is [MC, NC] = [g.N, g.M] here.  Every load of a batch of rows is issued before the first use: the
+// epilogue is bound by bytes in flight per SM (eight warps), so a batch is as deep as the registers
+// allow (all 32 rows; 16 when three inputs are read).  Mode and activation are compile-time
+// parameters: one compact loop per case.
+template <int MODE, int ACT, bool FULL>
+__device__ __forceinline__ void epilogue_t32_rows(const TcArgs& g, int n, int mb, const uint32_t (&r)[32]) {
   const GemmEpilogue& e = g.epi;
   const int MC = g.N, NC = g.M;
-  constexpr int U = 8;
+  constexpr int U = (MODE == EPI_R_BWD && ACT != BETTY_ACT_RELU) ? 16 : 32;
   const float bias = (MODE == EPI_BIAS_ACT || MODE == EPI_R_FWD) ? e.bias[n] : 0.f;
   const float kap = ((MODE == EPI_SGD || MODE == EPI_NEUMANN) && e.lam) ? expf(*e.lam) : 0.f;
   float* cp = g.C ? g.C + (int64_t)mb * g.ldc + n : nullptr;
@@ -222,7 +225,7 @@ __device__ __forceinline__ void epilogue_t32_impl(const TcArgs& g, int n, int mb
   const float* sp = e.s_in ? e.s_in + (int64_t)mb * g.ldc + n : nullptr;
   float* so = e.s_out ? e.s_out + (int64_t)mb * g.ldc + n : nullptr;
   bf16* op = e.out16 ? e.out16 + (int64_t)mb * e.ld16 + n : nullptr;
-  const int rows = MC - mb;     // > 0
+  const int rows = MC - mb;     // > 0; FULL: >= 32, and no per-row guards, so that the rows' dependency chains interleave
   const bool second = MODE == EPI_R_BWD && ACT != BETTY_ACT_RELU;
 #pragma unroll
   for (int j0 = 0; j0 < 32; j0 += U) {
@@ -231,7 +234,7 @@ __device__ __forceinline__ void epilogue_t32_impl(const TcArgs& g, int n, int mb
     for (int k = 0; k < U; ++k) {
       const int j = j0 + k;
       x0[k] = 0.f; x1[k] = 0.f; x2[k] = 0.f;
-      if (j < rows) {
+      if (FULL || j < rows) {
         if (MODE == EPI_STORE) { if (g.beta != 0.f) x0[k] = cp[(int64_t)j * g.ldc]; }
         if (MODE == EPI_R_FWD) { if (op) x0[k] = ap[(int64_t)j * NC]; }
         if (MODE == EPI_ACT_BWD || MODE == EPI_R_BWD) x0[k] = ap[(int64_t)j * NC];
@@ -243,7 +246,7 @@ __device__ __forceinline__ void epilogue_t32_impl(const TcArgs& g, int n, int mb
 #pragma unroll
     for (int k = 0; k < U; ++k) {
       const int j = j0 + k;
-      if (j < rows) {
+      if (FULL || j < rows) {
         const float acc = __uint_as_float(r[j]);
         float* c1 = cp + (int64_t)j * g.ldc;
         bf16* o1 = op + (int64_t)j * e.ld16;
@@ -283,6 +286,11 @@ __device__ __forceinline__ void epilogue_t32_impl(const TcArgs& g, int n, int mb
     }
   }
 }
+template <int MODE, int ACT>
+__device__ __forceinline__ void epilogue_t32_impl(const TcArgs& g, int n, int mb, const uint32_t (&r)[32]) {
+  if (g.N - mb >= 32) epilogue_t32_rows<MODE, ACT, true>(g, n, mb, r);
+  else epilogue_t32_rows<MODE, ACT, false>(g, n, mb, r);
+}
 template <int MODE>
 __device__ __forceinline__ void epilogue_t32_act(const TcArgs& g, int n, int mb, const uint32_t (&r)[32]) {
   if (g.epi.act == BETTY_ACT_RELU) epilogue_t32_impl<MODE, BETTY_ACT_RELU>(g, n, mb, r);
@@ -298,6 +306,49 @@ __device__ __forceinline__ void epilogue_t32(const TcArgs& g, int n, int mb, con
     case EPI_SGD: epilogue_t32_impl<EPI_SGD, BETTY_ACT_RELU>(g, n, mb, r); break;
     case EPI_NEUMANN: epilogue_t32_impl<EPI_NEUMANN, BETTY_ACT_RELU>(g, n, mb, r); break;
   }
+}
+
+// Warms L2 with the fp32 arrays that the epilogue of the tile at kernel coordinates (m0, n0) will read
+// (transposed mode: rows n0 .. n0+BN-1 of C, up to 128 columns from m0).  Issued by the 256 epilogue
+// threads (e = 0 .. 255, one row each) a whole tile ahead, so that the epilogue's loads find their
+// lines in L2 instead of waiting on HBM.  Plain loads of one word per 256 bytes with the 256-byte L2
+// prefetch size: measured on this part, prefetch instructions proper (prefetch.global.L2 and the bulk L2
+// prefetch) left most later loads at HBM latency, loads with the size hint did not.
+__device__ __forceinline__ void l2_touch(const float* p) {
+  float v;
+  asm volatile("ld.global.L2::256B.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void prefetch_epilogue_inputs(const TcArgs& g, int m0, int n0, int BN, int e) {
+  if (!g.pf_ok || m0 >= g.M) return;
+  const GemmEpilogue& ep = g.epi;
+  const float* pc[2] = {nullptr, nullptr};   // arrays with the leading dimension of C
+  const float* pa[3] = {nullptr, nullptr, nullptr};   // arrays stored [MC, NC] densely
+  switch (ep.mode) {
+    case EPI_STORE: if (g.beta != 0.f) pc[0] = g.C; break;
+    case EPI_SGD: pc[0] = g.C; break;
+    case EPI_NEUMANN: pc[0] = ep.t_in; pc[1] = ep.s_in; break;
+    case EPI_R_FWD: if (ep.out16) pa[0] = ep.a; break;
+    case EPI_ACT_BWD: pa[0] = ep.a; break;
+    case EPI_R_BWD: pa[0] = ep.a; if (ep.act != BETTY_ACT_RELU) { pa[1] = ep.dh; pa[2] = ep.Ra; } break;
+    default: break;
+  }
+  const int R = n0 + e;
+  if (e >= BN || R >= g.N) return;
+  const bool two = g.M - m0 > 64;       // the row segment spans a second 256-byte block
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+    if (pc[i]) {
+      const float* p = pc[i] + (int64_t)R * g.ldc + m0;
+      l2_touch(p);
+      if (two) l2_touch(p + 64);
+    }
+#pragma unroll
+  for (int i = 0; i < 3; ++i)
+    if (pa[i]) {
+      const float* p = pa[i] + (int64_t)R * g.M + m0;
+      l2_touch(p);
+      if (two) l2_touch(p + 64);
+    }
 }
 
 // Persistent kernel: CTA b works on output tiles b, b + gridDim.x, ...
@@ -410,11 +461,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
     // ---------------- epilogue: warp w may touch accumulator lanes 32*(w%4) .. 32*(w%4)+31
     const int q = warp & 3;
     int j = 0;
+    if ((int)blockIdx.x < tiles)
+      prefetch_epilogue_inputs(g, ((int)blockIdx.x / tiles_n) * TC_BM, ((int)blockIdx.x % tiles_n) * BN, BN, tid - 64);
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++j) {
       const int m0 = (t / tiles_n) * TC_BM, n0 = (t % tiles_n) * BN;
       const int as = j & 1;
       const int m = m0 + q * 32 + lane;
       if (T > 0) {
+        const int tn = t + (int)gridDim.x;    // this CTA's next tile: ask for its inputs one epilogue ahead
+        if (tn < tiles) prefetch_epilogue_inputs(g, (tn / tiles_n) * TC_BM, (tn % tiles_n) * BN, BN, tid - 64);
         bool have = tc_wait(&acc_full[as], (uint32_t)((j >> 1) & 1), abort_flag);
         have = __all_sync(0xffffffffu, have);
         if (!have) break;
@@ -591,11 +646,16 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUt
     // ---------------- epilogue (both CTAs): own 128 rows of the pair's tile
     const int q = warp & 3;
     int j = 0;
+    if (cluster_id < tiles)
+      prefetch_epilogue_inputs(g, (cluster_id / tiles_n) * (2 * TC_BM) + (int)rank * TC_BM, (cluster_id % tiles_n) * BN, BN, tid - 64);
     for (int t = cluster_id; t < tiles; t += n_clusters, ++j) {
       const int m0 = (t / tiles_n) * (2 * TC_BM) + (int)rank * TC_BM, n0 = (t % tiles_n) * BN;
       const int as = j & 1;
       const int m = m0 + q * 32 + lane;
       if (T > 0) {
+        const int tn = t + n_clusters;
+        if (tn < tiles)
+          prefetch_epilogue_inputs(g, (tn / tiles_n) * (2 * TC_BM) + (int)rank * TC_BM, (tn % tiles_n) * BN, BN, tid - 64);
         bool have = tc_wait(&acc_full[as], (uint32_t)((j >> 1) & 1), abort_flag);
         have = __all_sync(0xffffffffu, have);
         if (!have) break;
@@ -735,6 +795,7 @@ static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a, bool tr) {
                   al16(e.out16) && (e.ld16 % 8 == 0) && al16(e.w16) && (e.ldw16 % 8 == 0) && al16(e.t_in) && al16(e.s_in) &&
                   al16(e.s_out);
   a.vec_ok = ok ? 1 : 0;
+  a.pf_ok = tr ? 1 : 0;
   for (int i = 0; i < 2; ++i) {
     const GemmPair& p = g.p[i < g.npairs ? i : 0];
     a.p[i].K = i < g.npairs ? p.K : 0;
