@@ -11,6 +11,7 @@ unsigned long long g_kernel_launches = 0;
 // ------------------------------------------------------------------ small kernels
 // out (+)= scale * x
 __global__ void k_scale_into(float* out, const float* x, float scale, int accumulate, int64_t n) {
+  pdl_enter();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     out[i] = (accumulate ? out[i] : 0.f) + scale * x[i];
 }
@@ -18,6 +19,7 @@ __global__ void k_scale_into(float* out, const float* x, float scale, int accumu
 // in double to keep the cancellation exact:  out (+)= -alpha*[(w+ev)^2 - (w-ev)^2]/(4e)
 __global__ void k_fd_weight_decay(float* out, const float* w, const float* v, const float* vnorm2, float eps0,
                                   float alpha, int accumulate, int64_t n) {
+  pdl_enter();
   const double nv = sqrt((double)*vnorm2);
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     float base = accumulate ? out[i] : 0.f;
@@ -31,6 +33,7 @@ __global__ void k_fd_weight_decay(float* out, const float* w, const float* v, co
 }
 // optimiser steps (see betty_optimizer); the step counter of Adam is the float behind the two moments
 __global__ void k_opt_momentum(float* x, const float* g, float* buf, float lr, float mom, float wd, int64_t n) {
+  pdl_enter();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     const float gg = g[i] + wd * x[i];
     const float b = mom * buf[i] + gg;
@@ -40,6 +43,7 @@ __global__ void k_opt_momentum(float* x, const float* g, float* buf, float lr, f
 }
 __global__ void k_opt_adam(float* x, const float* g, float* m, float* v, const float* tcount, float lr, float b1, float b2,
                            float eps, float wd, int64_t n) {
+  pdl_enter();
   const float t = *tcount + 1.f;                       // this step's index; the counter is advanced afterwards
   const float c1 = 1.f - powf(b1, t), c2 = 1.f - powf(b2, t);
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
@@ -50,8 +54,12 @@ __global__ void k_opt_adam(float* x, const float* g, float* m, float* v, const f
     x[i] -= lr * (mi / c1) / (sqrtf(vi / c2) + eps);
   }
 }
-__global__ void k_opt_tick(float* tcount) { *tcount += 1.f; }
+__global__ void k_opt_tick(float* tcount) {
+  pdl_enter();
+  *tcount += 1.f;
+}
 __global__ void k_opt_gd(float* x, const float* g, float lr, int64_t n) {
+  pdl_enter();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     x[i] -= lr * g[i];
 }
@@ -128,7 +136,7 @@ betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps) {
 betty_status vecfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
                        float eps0, float alpha, float* out, bool accumulate) {
   if (!vec_has_wd(L) || wrt != find_constraint(L, BETTY_PARAM_VECTOR)) return BETTY_ERR_INVALID_ARG;
-  k_fd_weight_decay<<<ew_grid(L->d), 256, 0, c.stream>>>(out, L->params, v, vnorm2, eps0, alpha, accumulate ? 1 : 0, L->d);
+  launch_pdl(k_fd_weight_decay, dim3(ew_grid(L->d)), dim3(256), 0, c.stream, out, L->params, v, vnorm2, eps0, alpha, accumulate ? 1 : 0, L->d);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
@@ -139,14 +147,14 @@ static betty_status apply_optimizer(Ctx& c, const betty_level* L, const float* g
   if (n <= 0) return BETTY_OK;
   const int grid = (int)((n + 1023) / 1024 < 1 ? 1 : ((n + 1023) / 1024 > 2368 ? 2368 : (n + 1023) / 1024));
   if (L->optimizer == BETTY_OPT_GD) {
-    k_opt_gd<<<grid, 256, 0, c.stream>>>(L->params, g, L->lr, n);
+    launch_pdl(k_opt_gd, dim3(grid), dim3(256), 0, c.stream, L->params, g, L->lr, n);
   } else if (L->optimizer == BETTY_OPT_MOMENTUM) {
-    k_opt_momentum<<<grid, 256, 0, c.stream>>>(L->params, g, L->opt_state, L->lr, L->momentum, L->weight_decay, n);
+    launch_pdl(k_opt_momentum, dim3(grid), dim3(256), 0, c.stream, L->params, g, L->opt_state, L->lr, L->momentum, L->weight_decay, n);
   } else {
     float* m = L->opt_state; float* v = m + n; float* t = v + n;
-    k_opt_adam<<<grid, 256, 0, c.stream>>>(L->params, g, m, v, t, L->lr, L->beta1, L->beta2, L->adam_eps, L->weight_decay, n);
+    launch_pdl(k_opt_adam, dim3(grid), dim3(256), 0, c.stream, L->params, g, m, v, t, L->lr, L->beta1, L->beta2, L->adam_eps, L->weight_decay, n);
     BETTY_LAUNCH_CHECK();
-    k_opt_tick<<<1, 1, 0, c.stream>>>(t);
+    launch_pdl(k_opt_tick, dim3(1), dim3(1), 0, c.stream, t);
   }
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
@@ -237,7 +245,7 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
     }
   }
   BETTY_TRY(vecfam ? vecfam_mixed(c, L, wrt, q, m) : mlpfam_mixed(c, L, cache, wrt, q, m));
-  k_scale_into<<<ew_grid(nc), 256, 0, c.stream>>>(out, m, -qscale, accumulate ? 1 : 0, nc);
+  launch_pdl(k_scale_into, dim3(ew_grid(nc)), dim3(256), 0, c.stream, out, m, -qscale, accumulate ? 1 : 0, nc);
   BETTY_LAUNCH_CHECK();
   c.arena.release(mark);
   return BETTY_OK;
@@ -303,7 +311,7 @@ static betty_status hypergrad_itd(const betty_level* lower, const betty_level* u
       BETTY_TRY(mlpfam_mixed(c, &at, cache, wrt, a, m));
       BETTY_TRY(mlpfam_hvp(c, &at, cache, a, h));
     }
-    k_scale_into<<<ew_grid(nc), 256, 0, c.stream>>>(out, m, -lower->lr, 1, nc);
+    launch_pdl(k_scale_into, dim3(ew_grid(nc)), dim3(256), 0, c.stream, out, m, -lower->lr, 1, nc);
     BETTY_LAUNCH_CHECK();
     BETTY_TRY(vec_axpby(c, a, 1.f, a, -lower->lr, h, n));
     c.arena.release(mark);

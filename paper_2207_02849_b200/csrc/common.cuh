@@ -84,6 +84,32 @@ extern unsigned long long g_kernel_launches;
 
 static inline bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
 
+// ---- programmatic dependent launch ----
+// Consecutive kernels of a call are launched with programmatic stream serialisation: the next grid
+// may be scheduled while the current one is still running, and blocks in griddepcontrol.wait until
+// the current grid has completed and its memory operations are visible.  What this hides is launch
+// latency and per-kernel set-up (barrier initialisation, tensor-memory allocation).  The rules that
+// keep it correct: every kernel launched through launch_pdl executes pdl_wait() before its first
+// global-memory access (reads and writes: the predecessor may still be reading what this kernel
+// overwrites), and no kernel depends on anything older than its stream predecessor without that
+// predecessor having waited too (completion is transitive only because every kernel waits).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// wait for the predecessor, then let the successor start its own set-up
+__device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_trigger(); }
+
+template <typename... KArgs, typename... Args>
+static inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // errors surface in BETTY_LAUNCH_CHECK
+}
+
 // ---- vector kernels (vec.cu); all vectors fp32, scalars stay on the device ----
 betty_status vec_zero(Ctx& c, float* x, int64_t n);
 betty_status vec_copy(Ctx& c, float* dst, const float* src, int64_t n);

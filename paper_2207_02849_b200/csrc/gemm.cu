@@ -7,6 +7,7 @@ static constexpr int GT = 64;   // C tile edge
 static constexpr int GK = 16;   // K slab
 
 __global__ void __launch_bounds__(256) k_gemm_simt(GemmDesc g) {
+  pdl_enter();
   __shared__ float As[GK][GT + 1];
   __shared__ float Bs[GK][GT + 1];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmDesc g) {
 betty_status gemm_simt(Ctx& c, const GemmDesc& g) {
   if (g.M <= 0 || g.N <= 0) return BETTY_OK;
   dim3 grid((unsigned)((g.N + GT - 1) / GT), (unsigned)((g.M + GT - 1) / GT));
-  k_gemm_simt<<<grid, 256, 0, c.stream>>>(g);
+  launch_pdl(k_gemm_simt, dim3(grid), dim3(256), 0, c.stream, g);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }

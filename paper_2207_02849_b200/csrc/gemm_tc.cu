@@ -388,6 +388,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above touched only this CTA's shared and tensor memory and may overlap the previous
+  // kernel's tail; global memory (operands, epilogue inputs and outputs) is touched from here on.
+  pdl_enter();
 
   if (warp == 0 && lane == 0 && T > 0) {
     // ---------------- producer: TMA loads into the stage ring
@@ -577,6 +580,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUt
   cluster_sync_all();     // the peer's barriers exist before anything is signalled across the pair
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  pdl_enter();            // set-up done; global memory is touched from here on
 
   if (warp == 0 && lane == 0 && T > 0) {
     // ---------------- producer (both CTAs): own half of A and of B; completion counted on the leader's barrier
@@ -780,7 +784,7 @@ static betty_status launch_tc(Ctx& c, const GemmDesc& g0, bool tr) {
   }
   const int tiles = ((g.N + BN - 1) / BN) * ((g.M + TC_BM - 1) / TC_BM);
   const int grid = tiles < c.sm_count ? tiles : c.sm_count;
-  k_gemm_tc<BN><<<grid, TC_THREADS, Cfg::SMEM, c.stream>>>(tm[0], tm[1], tm[2], tm[3], a);
+  launch_pdl(k_gemm_tc<BN>, dim3(grid), dim3(TC_THREADS), Cfg::SMEM, c.stream, tm[0], tm[1], tm[2], tm[3], a);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
@@ -825,7 +829,7 @@ static betty_status launch_tc2(Ctx& c, const GemmDesc& g0, bool tr) {
   const int tiles = ((g.N + TC2_BN - 1) / TC2_BN) * ((g.M + 2 * TC_BM - 1) / (2 * TC_BM));
   const int max_pairs = c.sm_count / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  k_gemm_tc2<<<2 * pairs, TC_THREADS, TC2_SMEM, c.stream>>>(tm[0], tm[1], tm[2], tm[3], a);
+  launch_pdl(k_gemm_tc2, dim3(2 * pairs), dim3(TC_THREADS), TC2_SMEM, c.stream, tm[0], tm[1], tm[2], tm[3], a);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }

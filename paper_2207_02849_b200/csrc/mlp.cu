@@ -29,6 +29,7 @@ __device__ __forceinline__ float fd_eps(const float* vnorm2, float eps0) {
 // dst[r, c] = bf16(scale * src[r, c]); scale = eps0/|v| when vnorm2 is given, else 1.  Pad columns are zeroed.
 __global__ void k_cast_rows(const float* src, bf16* dst, int64_t rows, int64_t cols, int64_t ld, const float* vnorm2,
                             float eps0) {
+  pdl_enter();
   const float s = vnorm2 ? fd_eps(vnorm2, eps0) : 1.f;
   const int64_t total = rows * ld;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -38,6 +39,7 @@ __global__ void k_cast_rows(const float* src, bf16* dst, int64_t rows, int64_t c
 }
 // a += bias; h = act(a) as bf16 (hidden layers)
 __global__ void k_bias_act(float* a, const float* bias, bf16* h, int64_t rows, int64_t N, int64_t ldh, int act) {
+  pdl_enter();
   const int64_t total = rows * N;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / N, n = i - r * N;
@@ -48,6 +50,7 @@ __global__ void k_bias_act(float* a, const float* bias, bf16* h, int64_t rows, i
 }
 // one warp per row: p = softmax(z), ell = -log p[y]
 __global__ void k_softmax_ce(const float* z, const int32_t* y, float* p, float* ell, int64_t B, int64_t C) {
+  pdl_enter();
   const int lane = threadIdx.x & 31;
   const int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
   if (row >= B) return;
@@ -69,6 +72,7 @@ __global__ void k_softmax_ce(const float* z, const int32_t* y, float* p, float* 
 // delta = coef_i * (p - onehot(y))
 __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef, float scale, bf16* delta, int64_t B,
                             int64_t C, int64_t ld) {
+  pdl_enter();
   const int64_t total = B * ld;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / ld, c = i - r * ld;
@@ -83,6 +87,7 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
 //   mode 2: t = t_in[n] - step * sum; out[n] = t; s_out[n] = s_in[n] + t   (Neumann-series update)
 struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; float* s_out; };
 __global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
+  pdl_enter();
   // 1024 threads: 32 lanes x 2 adjacent columns, 32 row groups; ld is even, so a column pair is one 4-byte load
   __shared__ float sh[32][65];
   const int cx = threadIdx.x & 31, rg = threadIdx.x >> 5;
@@ -111,6 +116,7 @@ __global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, 
 }
 // delta_prev = dh * act'(a)
 __global__ void k_act_backward(const float* dh, const float* a, bf16* dprev, int64_t B, int64_t N, int64_t ld, int act) {
+  pdl_enter();
   const int64_t total = B * ld;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / ld, n = i - r * ld;
@@ -120,6 +126,7 @@ __global__ void k_act_backward(const float* dh, const float* a, bf16* dprev, int
 // Ra += c ; Rh = act'(a) * Ra
 __global__ void k_r_act_forward(float* Ra, const float* cdir, const float* a, bf16* Rh, int64_t B, int64_t N,
                                 int64_t ldh, int act) {
+  pdl_enter();
   const int64_t total = B * N;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / N, n = i - r * N;
@@ -131,6 +138,7 @@ __global__ void k_r_act_forward(float* Ra, const float* cdir, const float* a, bf
 // one warp per row: Rdelta = coef_i * (p.*Ra - p * (p . Ra))
 __global__ void k_r_delta_top(const float* p, const float* Ra, const float* coef, float scale, bf16* Rd, int64_t B,
                               int64_t C, int64_t ld) {
+  pdl_enter();
   const int lane = threadIdx.x & 31;
   const int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
   if (row >= B) return;
@@ -147,6 +155,7 @@ __global__ void k_r_delta_top(const float* p, const float* Ra, const float* coef
 // Rdelta_prev = Rdh * act'(a) + dh * act''(a) * Ra
 __global__ void k_r_act_backward(const float* Rdh, const float* dh, const float* a, const float* Ra, bf16* Rdprev,
                                  int64_t B, int64_t N, int64_t ld, int act) {
+  pdl_enter();
   const int64_t total = B * ld;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / ld, n = i - r * ld;
@@ -161,6 +170,7 @@ __global__ void k_r_act_backward(const float* Rdh, const float* dh, const float*
 }
 // one warp per row: d_i = sum_c (p - onehot) * Ra
 __global__ void k_jvp_rows(const float* p, const int32_t* y, const float* Ra, float* d, int64_t B, int64_t C) {
+  pdl_enter();
   const int lane = threadIdx.x & 31;
   const int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
   if (row >= B) return;
@@ -171,6 +181,7 @@ __global__ void k_jvp_rows(const float* p, const int32_t* y, const float* Ra, fl
 }
 // out[r, c] += exp(lam) * W[r, c]   (out contiguous [rows, cols]; W bf16 with leading dimension ldw)
 __global__ void k_wd_add_bf16(float* out, const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* lam) {
+  pdl_enter();
   const float k = expf(*lam);
   const int64_t total = rows * cols;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -179,6 +190,7 @@ __global__ void k_wd_add_bf16(float* out, const bf16* W, int64_t rows, int64_t c
   }
 }
 __global__ void k_wd_add_f32(float* out, const float* u, int64_t n, const float* lam) {
+  pdl_enter();
   const float k = expf(*lam);
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     out[i] += k * u[i];
@@ -188,6 +200,7 @@ __global__ void k_wd_add_f32(float* out, const float* u, int64_t n, const float*
 static constexpr int LD_MAX_BLOCKS = 128;
 __global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
                             float scale, float* out, int accumulate, double* partial, unsigned* counter) {
+  pdl_enter();
   __shared__ double sh[32];
   __shared__ bool is_last;
   double acc = 0.0;
@@ -224,7 +237,7 @@ static betty_status layer_dot(Ctx& c, const bf16* W, int64_t rows, int64_t cols,
   BETTY_ALLOC(partial, double, c, (size_t)nb);
   BETTY_ALLOC(counter, unsigned, c, 8);
   if (cudaMemsetAsync(counter, 0, 32, c.stream) != cudaSuccess) return BETTY_ERR_CUDA;
-  k_layer_dot<<<(unsigned)nb, 256, 0, c.stream>>>(W, rows, cols, ldw, q, lam, scale, out, accumulate ? 1 : 0, partial, counter);
+  launch_pdl(k_layer_dot, dim3((unsigned)nb), dim3(256), 0, c.stream, W, rows, cols, ldw, q, lam, scale, out, accumulate ? 1 : 0, partial, counter);
   BETTY_LAUNCH_CHECK();
   c.arena.release(mark);
   return BETTY_OK;
@@ -238,6 +251,7 @@ enum WnMode { WN_REWEIGHT_COEF = 0, WN_REWEIGHT_TGRAD, WN_REWEIGHT_TMIXED, WN_DE
 // caller's reverse sweep needs (see WnMode).  dir: a direction in theta space (modes *_THVP, *_WMIXED).
 __global__ void k_wn_sample(int mode, const float* theta, const float* dir, const float* ell, const float* aux,
                             const float* din, int64_t B, float invB, float* out1, float* out2) {
+  pdl_enter();
   __shared__ float th[WN_P], dr[WN_P];
   for (int i = threadIdx.x; i < WN_P; i += blockDim.x) { th[i] = theta[i]; dr[i] = dir ? dir[i] : 0.f; }
   __syncthreads();
@@ -278,6 +292,7 @@ static constexpr int WN_STRIDE = 304;    // doubles per block in the partial buf
 __global__ void k_wn_backward(const float* theta, const float* dir, const float* ell, const float* cA, const float* cB,
                               int64_t B, float mu, const float* muvec, float* out, int accumulate, float out_scale,
                               double* partial, unsigned* counter) {
+  pdl_enter();
   const int k = threadIdx.x;
   const int64_t per = (B + gridDim.x - 1) / gridDim.x;
   const int64_t i0 = blockIdx.x * per, i1 = (i0 + per < B) ? i0 + per : B;
@@ -327,6 +342,7 @@ __global__ void k_wn_backward(const float* theta, const float* dir, const float*
 // Output layer: z = a + da_tot (fp32).
 __global__ void k_fd_act(const float* a, const float* da, const float* cdir, const float* vnorm2, float eps0, float sign,
                          bf16* hpm, bf16* dhd, float* zpm, int64_t B, int64_t N, int64_t ldh, int act) {
+  pdl_enter();
   const float e = sign * fd_eps(vnorm2, eps0);
   const int64_t total = B * N;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -340,6 +356,7 @@ __global__ void k_fd_act(const float* a, const float* da, const float* cdir, con
 }
 __global__ void k_fd_combine(float* out, const float* gp, const float* gm, const float* vnorm2, float eps0, float alpha,
                              int accumulate, int64_t n) {
+  pdl_enter();
   const float e = fd_eps(vnorm2, eps0);
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     const float base = accumulate ? out[i] : 0.f;
@@ -397,6 +414,7 @@ static betty_status net_layout(const betty_level* M, Net& n) {
 
 // contiguous case (ld == cols, cols % 8 == 0): 8 elements per thread, 2 x float4 in, 1 x 16 bytes out
 __global__ void k_cast_dense8(const float* src, bf16* dst, int64_t n8, const float* vnorm2, float eps0) {
+  pdl_enter();
   const float s = vnorm2 ? fd_eps(vnorm2, eps0) : 1.f;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
     const float4 a = ((const float4*)src)[2 * i], b = ((const float4*)src)[2 * i + 1];
@@ -411,9 +429,9 @@ static betty_status cast_matrix(Ctx& c, const float* src, bf16* dst, int64_t row
                                 const float* vnorm2 = nullptr, float eps0 = 0.f) {
   if (ld == cols && (cols & 7) == 0 && ((((uintptr_t)src) & 15) == 0)) {
     const int64_t n8 = rows * cols / 8;
-    k_cast_dense8<<<grid_for(n8), 256, 0, c.stream>>>(src, dst, n8, vnorm2, eps0);
+    launch_pdl(k_cast_dense8, dim3(grid_for(n8)), dim3(256), 0, c.stream, src, dst, n8, vnorm2, eps0);
   } else {
-    k_cast_rows<<<grid_for(rows * ld), 256, 0, c.stream>>>(src, dst, rows, cols, ld, vnorm2, eps0);
+    launch_pdl(k_cast_rows, dim3(grid_for(rows * ld)), dim3(256), 0, c.stream, src, dst, rows, cols, ld, vnorm2, eps0);
   }
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
@@ -459,7 +477,7 @@ static betty_status forward(Ctx& c, const Net& n, const betty_level* D, Pass& ps
   BETTY_ALLOC(p, float, c, (size_t)(B * C));
   BETTY_ALLOC(ell, float, c, (size_t)B);
   ps.p = p; ps.ell = ell;
-  k_softmax_ce<<<grid_for(B * 32), 256, 0, c.stream>>>(ps.a[n.L - 1], ps.y, p, ell, B, C);
+  launch_pdl(k_softmax_ce, dim3(grid_for(B * 32)), dim3(256), 0, c.stream, ps.a[n.L - 1], ps.y, p, ell, B, C);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
@@ -483,7 +501,7 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
     const int64_t ld = ld8(C);
     BETTY_ALLOC(dt, bf16, c, (size_t)(B * ld));
     ps.delta[n.L - 1] = dt;
-    k_delta_top<<<grid_for(B * ld), 256, 0, c.stream>>>(ps.p, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld);
+    launch_pdl(k_delta_top, dim3(grid_for(B * ld)), dim3(256), 0, c.stream, ps.p, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld);
     BETTY_LAUNCH_CHECK();
   }
   for (int l = n.L - 1; l >= 0; --l) {
@@ -503,10 +521,10 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       }
       BETTY_TRY(gemm(c, g));
       if (!sink.sgd && sink.lam) {
-        k_wd_add_bf16<<<grid_for(N * K), 256, 0, c.stream>>>(sink.gflat + n.woff[l], n.W[l], N, K, n.ldw[l], sink.lam + l);
+        launch_pdl(k_wd_add_bf16, dim3(grid_for(N * K)), dim3(256), 0, c.stream, sink.gflat + n.woff[l], n.W[l], N, K, n.ldw[l], sink.lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      k_colsum_bf16<<<(unsigned)((N + 63) / 64), 1024, 0, c.stream>>>(ps.delta[l], B, N, ldd, cs);
+      launch_pdl(k_colsum_bf16, dim3((unsigned)((N + 63) / 64)), dim3(1024), 0, c.stream, ps.delta[l], B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {
@@ -623,7 +641,7 @@ size_t mlpfam_workspace(const betty_level* L) {
 static betty_status wn_sample(Ctx& c, int mode, const betty_level* theta, const float* dir, const Pass& ps,
                               const float* aux, const float* din, float* out1, float* out2) {
   const int64_t B = ps.B;
-  k_wn_sample<<<grid_for(B, 128), 128, 0, c.stream>>>(mode, theta->params, dir, ps.ell, aux, din, B,
+  launch_pdl(k_wn_sample, dim3(grid_for(B, 128)), dim3(128), 0, c.stream, mode, theta->params, dir, ps.ell, aux, din, B,
                                                       B > 0 ? 1.f / (float)B : 0.f, out1, out2);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
@@ -637,7 +655,7 @@ static betty_status wn_backward(Ctx& c, const betty_level* theta, const float* d
   BETTY_ALLOC(partial, double, c, (size_t)nb * WN_STRIDE);
   BETTY_ALLOC(counter, unsigned, c, 8);
   if (cudaMemsetAsync(counter, 0, 32, c.stream) != cudaSuccess) return BETTY_ERR_CUDA;
-  k_wn_backward<<<nb, 128, 0, c.stream>>>(theta->params, dir, ps.ell, cA, cB, ps.B, mu, muvec, out, accumulate ? 1 : 0,
+  launch_pdl(k_wn_backward, dim3(nb), dim3(128), 0, c.stream, theta->params, dir, ps.ell, cA, cB, ps.B, mu, muvec, out, accumulate ? 1 : 0,
                                           out_scale, partial, counter);
   BETTY_LAUNCH_CHECK();
   c.arena.release(mark);
@@ -743,7 +761,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
     const int64_t ld = ld8(C);
     Rd = c.arena.alloc<bf16>((size_t)(B * ld));
     if (!Rd) return BETTY_ERR_WORKSPACE;
-    k_r_delta_top<<<grid_for(B * 32), 256, 0, c.stream>>>(ps.p, rp.Ra[n.L - 1], h->coef, B > 0 ? 1.f / (float)B : 0.f, Rd,
+    launch_pdl(k_r_delta_top, dim3(grid_for(B * 32)), dim3(256), 0, c.stream, ps.p, rp.Ra[n.L - 1], h->coef, B > 0 ? 1.f / (float)B : 0.f, Rd,
                                                          B, C, ld);
     BETTY_LAUNCH_CHECK();
   }
@@ -766,10 +784,10 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
       }
       BETTY_TRY(gemm(c, g));
       if (!sink && h->lam) {
-        k_wd_add_f32<<<grid_for(N * K), 256, 0, c.stream>>>(Hu + n.woff[l], u + n.woff[l], N * K, h->lam + l);
+        launch_pdl(k_wd_add_f32, dim3(grid_for(N * K)), dim3(256), 0, c.stream, Hu + n.woff[l], u + n.woff[l], N * K, h->lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      k_colsum_bf16<<<(unsigned)((N + 63) / 64), 1024, 0, c.stream>>>(Rd, B, N, ldd, cs);
+      launch_pdl(k_colsum_bf16, dim3((unsigned)((N + 63) / 64)), dim3(1024), 0, c.stream, Rd, B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {  // R dh = Rdelta W_l + delta_l U_l ; Rdelta_{l-1} = Rdh*act' + dh*act''*Ra
@@ -816,7 +834,7 @@ betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const be
       BETTY_TRY(rforward(c, n, ps, q, rp));
       BETTY_ALLOC(d, float, c, (size_t)(B > 0 ? B : 1));
       BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
-      k_jvp_rows<<<grid_for(B * 32), 256, 0, c.stream>>>(ps.p, ps.y, rp.Ra[n.L - 1], d, B, n.w[n.L]);
+      launch_pdl(k_jvp_rows, dim3(grid_for(B * 32)), dim3(256), 0, c.stream, ps.p, ps.y, rp.Ra[n.L - 1], d, B, n.w[n.L]);
       BETTY_LAUNCH_CHECK();
       BETTY_TRY(wn_sample(c, WN_REWEIGHT_TMIXED, P.theta, nullptr, ps, nullptr, d, s1, nullptr));
       BETTY_TRY(wn_backward(c, P.theta, nullptr, ps, s1, nullptr, 0.f, nullptr, out));
@@ -922,23 +940,23 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
           cudaMemsetAsync(hn, 0, cnt * sizeof(bf16), c.stream);
           cudaMemsetAsync(dn, 0, cnt * sizeof(bf16), c.stream);
         }
-        k_fd_act<<<grid_for(B * N), 256, 0, c.stream>>>(ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, hn, dn, nullptr, B, N,
+        launch_pdl(k_fd_act, dim3(grid_for(B * N)), dim3(256), 0, c.stream, ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, hn, dn, nullptr, B, N,
                                                        ps.ldh[l + 1], n.act);
         BETTY_LAUNCH_CHECK();
         hp = hn; dh = dn;
       } else {
-        k_fd_act<<<grid_for(B * N), 256, 0, c.stream>>>(ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, nullptr, nullptr, zpm,
+        launch_pdl(k_fd_act, dim3(grid_for(B * N)), dim3(256), 0, c.stream, ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, nullptr, nullptr, zpm,
                                                        B, N, 0, n.act);
         BETTY_LAUNCH_CHECK();
       }
     }
-    k_softmax_ce<<<grid_for(B * 32), 256, 0, c.stream>>>(zpm, ps.y, pp.p, pp.ell, B, C);
+    launch_pdl(k_softmax_ce, dim3(grid_for(B * 32)), dim3(256), 0, c.stream, zpm, ps.y, pp.p, pp.ell, B, C);
     BETTY_LAUNCH_CHECK();
     BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, pp, nullptr, nullptr, s1, nullptr));
     BETTY_TRY(wn_backward(c, P.theta, nullptr, pp, s1, nullptr, 0.f, nullptr, G + 512 * sgn));
     c.arena.release(m2);
   }
-  k_fd_combine<<<grid_for(WN_P), 256, 0, c.stream>>>(out, G, G + 512, vnorm2, eps0, alpha, accumulate ? 1 : 0, WN_P);
+  launch_pdl(k_fd_combine, dim3(grid_for(WN_P)), dim3(256), 0, c.stream, out, G, G + 512, vnorm2, eps0, alpha, accumulate ? 1 : 0, WN_P);
   BETTY_LAUNCH_CHECK();
   c.arena.release(mark);
   return BETTY_OK;

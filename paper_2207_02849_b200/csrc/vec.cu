@@ -16,21 +16,26 @@ static inline int ew_blocks(int64_t n, int per_thread = 4) {
 }
 
 __global__ void k_zero(float* x, int64_t n) {
+  pdl_enter();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) x[i] = 0.f;
 }
 __global__ void k_copy(float* d, const float* s, int64_t n) {
+  pdl_enter();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) d[i] = s[i];
 }
 __global__ void k_axpby(float* out, float a, const float* x, float b, const float* y, int64_t n) {
+  pdl_enter();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     out[i] = y ? a * x[i] + b * y[i] : a * x[i];
 }
 __global__ void k_mul(float* out, float a, const float* x, const float* y, int64_t n) {
+  pdl_enter();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     out[i] = a * x[i] * y[i];
 }
 __global__ void k_neumann(const float* t_in, const float* s_in, const float* Ht, float alpha, float* t_out, float* s_out,
                           int64_t n) {
+  pdl_enter();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     float tn = t_in[i] - alpha * Ht[i];
     t_out[i] = tn;
@@ -40,32 +45,32 @@ __global__ void k_neumann(const float* t_in, const float* s_in, const float* Ht,
 
 betty_status vec_zero(Ctx& c, float* x, int64_t n) {
   if (n <= 0) return BETTY_OK;
-  k_zero<<<ew_blocks(n), VT, 0, c.stream>>>(x, n);
+  launch_pdl(k_zero, dim3(ew_blocks(n)), dim3(VT), 0, c.stream, x, n);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
 betty_status vec_copy(Ctx& c, float* d, const float* s, int64_t n) {
   if (n <= 0) return BETTY_OK;
-  k_copy<<<ew_blocks(n), VT, 0, c.stream>>>(d, s, n);
+  launch_pdl(k_copy, dim3(ew_blocks(n)), dim3(VT), 0, c.stream, d, s, n);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
 betty_status vec_axpby(Ctx& c, float* out, float a, const float* x, float b, const float* y, int64_t n) {
   if (n <= 0) return BETTY_OK;
-  k_axpby<<<ew_blocks(n), VT, 0, c.stream>>>(out, a, x, b, y, n);
+  launch_pdl(k_axpby, dim3(ew_blocks(n)), dim3(VT), 0, c.stream, out, a, x, b, y, n);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
 betty_status vec_mul(Ctx& c, float* out, float a, const float* x, const float* y, int64_t n) {
   if (n <= 0) return BETTY_OK;
-  k_mul<<<ew_blocks(n), VT, 0, c.stream>>>(out, a, x, y, n);
+  launch_pdl(k_mul, dim3(ew_blocks(n)), dim3(VT), 0, c.stream, out, a, x, y, n);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
 betty_status neumann_update(Ctx& c, const float* t_in, const float* s_in, const float* Ht, float alpha, float* t_out,
                             float* s_out, int64_t n) {
   if (n <= 0) return BETTY_OK;
-  k_neumann<<<ew_blocks(n), VT, 0, c.stream>>>(t_in, s_in, Ht, alpha, t_out, s_out, n);
+  launch_pdl(k_neumann, dim3(ew_blocks(n)), dim3(VT), 0, c.stream, t_in, s_in, Ht, alpha, t_out, s_out, n);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
@@ -118,6 +123,7 @@ static inline int dot_blocks(int64_t n) {
 
 __global__ void k_dot(const float* x, const float* y, int64_t n, float* result, double* partials,
                       unsigned* counter, StatusBlock* sb) {
+  pdl_enter();
   __shared__ double sh[VT / 32];
   double acc = 0.0;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
@@ -138,7 +144,7 @@ betty_status vec_reduce_init(Ctx& c, float* partials) {
 betty_status vec_dot(Ctx& c, const float* x, const float* y, int64_t n, float* result, float* partials) {
   double* pd = (double*)partials;
   unsigned* counter = (unsigned*)(pd + DOT_MAX_BLOCKS);
-  k_dot<<<dot_blocks(n), VT, 0, c.stream>>>(x, y, n, result, pd, counter, c.arena.status());
+  launch_pdl(k_dot, dim3(dot_blocks(n)), dim3(VT), 0, c.stream, x, y, n, result, pd, counter, c.arena.status());
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
@@ -147,6 +153,7 @@ betty_status vec_dot(Ctx& c, const float* x, const float* y, int64_t n, float* r
 // q <- 0, r <- v, p <- v, rho <- v.v, stop <- tol^2 * v.v
 __global__ void k_cg_init(SolveState* st, const float* v, float* q, float* r, float* p, float tol, int64_t n,
                           double* partials, unsigned* counter, StatusBlock* sb) {
+  pdl_enter();
   __shared__ double sh[VT / 32];
   double acc = 0.0;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
@@ -169,6 +176,7 @@ __global__ void k_cg_init(SolveState* st, const float* v, float* q, float* r, fl
 // gamma <- p.h
 __global__ void k_cg_gamma(SolveState* st, const float* p, const float* h, int64_t n, double* partials,
                            unsigned* counter, StatusBlock* sb) {
+  pdl_enter();
   __shared__ double sh[VT / 32];
   double acc = 0.0;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
@@ -186,6 +194,7 @@ __global__ void k_cg_gamma(SolveState* st, const float* p, const float* h, int64
 // a = rho/gamma; q += a p; r -= a h; rho_new <- r.r   (no-op when the solve has stopped)
 __global__ void k_cg_update(SolveState* st, float* q, float* r, const float* p, const float* h, int64_t n,
                             double* partials, unsigned* counter) {
+  pdl_enter();
   __shared__ double sh[VT / 32];
   if (!st->active) return;
   const float a = st->rho / st->gamma;
@@ -204,6 +213,7 @@ __global__ void k_cg_update(SolveState* st, float* q, float* r, const float* p, 
 // and deactivates the solve once rho <= stop.
 __global__ void k_cg_direction(SolveState* st, float* p, const float* r, int64_t n, unsigned* counter,
                                StatusBlock* sb) {
+  pdl_enter();
   if (!st->active) return;
   const float beta = st->rho_new / st->rho;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
@@ -227,7 +237,7 @@ betty_status cg_init(Ctx& c, SolveState* st, const float* v, float* q, float* r,
                      float* partials) {
   double* pd = (double*)partials;
   unsigned* counter = (unsigned*)(pd + DOT_MAX_BLOCKS);
-  k_cg_init<<<dot_blocks(n), VT, 0, c.stream>>>(st, v, q, r, p, tol, n, pd, counter, c.arena.status());
+  launch_pdl(k_cg_init, dim3(dot_blocks(n)), dim3(VT), 0, c.stream, st, v, q, r, p, tol, n, pd, counter, c.arena.status());
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
@@ -237,11 +247,11 @@ betty_status cg_step(Ctx& c, SolveState* st, float* q, float* r, float* p, const
   double* pd = (double*)partials;
   unsigned* counter = (unsigned*)(pd + DOT_MAX_BLOCKS);
   const int nb = dot_blocks(n);
-  k_cg_gamma<<<nb, VT, 0, c.stream>>>(st, p, h, n, pd, counter, c.arena.status());
+  launch_pdl(k_cg_gamma, dim3(nb), dim3(VT), 0, c.stream, st, p, h, n, pd, counter, c.arena.status());
   BETTY_LAUNCH_CHECK();
-  k_cg_update<<<nb, VT, 0, c.stream>>>(st, q, r, p, h, n, pd, counter);
+  launch_pdl(k_cg_update, dim3(nb), dim3(VT), 0, c.stream, st, q, r, p, h, n, pd, counter);
   BETTY_LAUNCH_CHECK();
-  k_cg_direction<<<nb, VT, 0, c.stream>>>(st, p, r, n, counter + 1, c.arena.status());
+  launch_pdl(k_cg_direction, dim3(nb), dim3(VT), 0, c.stream, st, p, r, n, counter + 1, c.arena.status());
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
