@@ -222,6 +222,7 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
   if (cfg.method == BETTY_NEUMANN) {
     // t_0 = s_0 = v are read straight from v in the first iteration: no copies
     BETTY_ALLOC(t, float, c, (size_t)n);
+    if (!vecfam && cfg.K > 1 && L->param_kind == BETTY_PARAM_MLP) BETTY_TRY(mlpfam_hvp_keep_direction(c, cache));
     if (cfg.K == 0) BETTY_TRY(vec_copy(c, q, v, n));
     for (int k = 0; k < cfg.K; ++k) {
       const float* t_in = k == 0 ? v : t;
@@ -268,9 +269,13 @@ static betty_status hypergrad(const betty_level* lower, const betty_level* upper
                                   vec_family(upper), (const float*)upper->X, (const float*)upper->y, upper->n, lower->d,
                                   lower->params, wrt->params, cfg, out);
   BETTY_ALLOC(v, float, c, (size_t)lower->n_params);
+  // the upper gradient and the Jacobian product both evaluate costs at the lower level's present parameters
+  BETTY_TRY(mlpfam_share_weights(c, lower));
   BETTY_TRY(level_grad(c, upper, lower, v));     // dC_u / d theta_lower
   BETTY_TRY(level_grad(c, upper, wrt, out));     // direct gradient
-  return brj(c, lower, wrt, v, cfg, out, true);
+  const betty_status rc = brj(c, lower, wrt, v, cfg, out, true);
+  mlpfam_unshare_weights(c);
+  return rc;
 }
 
 // ITD-RMAD: n_steps unrolled lower steps with the iterates kept in the workspace, then the reverse

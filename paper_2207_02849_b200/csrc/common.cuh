@@ -54,11 +54,20 @@ struct Arena {
   __host__ StatusBlock* status() const { return (StatusBlock*)base; }
 };
 
+// bf16 copies of an MLP's matrices that several passes of one call share (see mlpfam_share_weights)
+struct SharedWeights {
+  const float* master;   // the fp32 parameters the copies were rounded from; null: none
+  bf16* W[16];
+};
+
 struct Ctx {
   cudaStream_t stream;
   Arena arena;
   int sm_count;
-  __host__ Ctx(void* ws, size_t ws_bytes, void* s) : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(148) {}
+  SharedWeights shared;
+  __host__ Ctx(void* ws, size_t ws_bytes, void* s) : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(148) {
+    shared.master = nullptr;
+  }
 };
 
 #define BETTY_TRY(expr)                       \

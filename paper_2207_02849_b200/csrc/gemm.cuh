@@ -20,7 +20,7 @@ enum GemmEpiMode {
   EPI_R_FWD = 3,     // v = acc + bias[n];  C = v;  out16 = act'(a[m,n]) * v             (R-operator forward)
   EPI_R_BWD = 4,     // out16 = acc * act'(a) + dh * act''(a) * Ra                       (R-operator backward)
   EPI_SGD = 5,       // g = acc + exp(lam) * w16;  C = C - lr * g;  out16 = bf16(new C)  (weight gradient -> gradient step; w16 == bf16(C))
-  EPI_NEUMANN = 6    // Hu = acc + exp(lam) * t_in;  t = t_in - alpha * Hu -> C;  s_out = s_in + t   (weight HVP -> series update)
+  EPI_NEUMANN = 6    // Hu = acc + exp(lam) * t_in;  t = t_in - alpha * Hu -> C;  s_out = s_in + t;  out16 = bf16(t) if given   (weight HVP -> series update)
 };
 struct GemmEpilogue {
   int mode;
@@ -121,6 +121,7 @@ __device__ __forceinline__ void gemm_epilogue_store(const GemmEpilogue& e, float
       const float tn = ti - e.step * hu;
       *cp = tn;
       e.s_out[jc] = e.s_in[jc] + tn;
+      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(tn);
       break;
     }
   }

@@ -167,7 +167,7 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
         const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
         float so[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { v[k] = tv[k] - e.step * (v[k] + kap * tv[k]); so[k] = sv[k] + v[k]; }
+        for (int k = 0; k < 8; ++k) { v[k] = tv[k] - e.step * (v[k] + kap * tv[k]); so[k] = sv[k] + v[k]; o[k] = v[k]; }
         *(float4*)(e.s_out + jc) = make_float4(so[0], so[1], so[2], so[3]);
         *(float4*)(e.s_out + jc + 4) = make_float4(so[4], so[5], so[6], so[7]);
       } else {   // EPI_ACT_BWD, EPI_R_BWD
@@ -281,6 +281,7 @@ __device__ __forceinline__ void epilogue_t32_rows(const TcArgs& g, int n, int mb
           const float tn = x0[k] - e.step * (acc + kap * x0[k]);
           *c1 = tn;
           so[(int64_t)j * g.ldc] = x1[k] + tn;
+          if (op) *o1 = __float2bfloat16_rn(tn);
         }
       }
     }
@@ -308,6 +309,49 @@ __device__ __forceinline__ void epilogue_t32(const TcArgs& g, int n, int mb, con
   }
 }
 
+// What the MMA-issuing thread needs per operand pair, worked out once per kernel: the issuing thread is a
+// single lane, and every instruction it spends between two MMAs is paid in full (measured: with the
+// descriptors rebuilt per k-step and the ring position taken by division, one 64-wide slab cost the
+// issuer ~800 clocks against the 512 its four MMAs run for).
+struct IssuePlan {
+  uint64_t a0, b0;            // shared-memory descriptors of stage 0, k-step 0
+  uint32_t a_step, b_step;    // descriptor increment per 16-element k-step, in 16-byte units
+  uint32_t idesc;
+};
+__device__ __forceinline__ IssuePlan issue_plan(const TcPair& p, uint32_t sa0, uint32_t sb0, int n, int m) {
+  IssuePlan q;
+  // K-major: 16 elements = 32 bytes further along the swizzled row; groups of 8 rows 1024 B apart.
+  // MN-major: 16 k-rows = 2048 bytes further; 64-element blocks along M/N 8192 B apart.
+  q.a0 = p.a_mn ? smem_desc(sa0, 8192, 1024) : smem_desc(sa0, 16, 1024);
+  q.b0 = p.b_mn ? smem_desc(sb0, 8192, 1024) : smem_desc(sb0, 16, 1024);
+  q.a_step = p.a_mn ? (2048u >> 4) : (32u >> 4);
+  q.b_step = p.b_mn ? (2048u >> 4) : (32u >> 4);
+  q.idesc = instr_desc(p.a_mn, p.b_mn, p.neg, n, m);
+  return q;
+}
+// Position in the stage ring: stage, how many times the ring has wrapped, and the stage's offset in
+// 16-byte units (what is added to a stage-0 descriptor; the address field holds 14 bits and shared
+// memory ends below 2^18 bytes, so the sum never carries out of the field).
+struct RingPos {
+  int s; uint32_t round; uint32_t off16;
+  __device__ __forceinline__ void advance(int S, uint32_t stage16) {
+    if (++s == S) { s = 0; ++round; off16 = 0; } else off16 += stage16;
+  }
+};
+template <int CG>
+__device__ __forceinline__ void mma_f16(uint32_t tmem_acc, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  if (CG == 1)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_acc), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_acc), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 // Warms L2 with the fp32 arrays that the epilogue of the tile at kernel coordinates (m0, n0) will read
 // (transposed mode: rows n0 .. n0+BN-1 of C, up to 128 columns from m0).  Issued by the 256 epilogue
 // threads (e = 0 .. 255, one row each) a whole tile ahead, so that the epilogue's loads find their
@@ -317,6 +361,7 @@ __device__ __forceinline__ void epilogue_t32(const TcArgs& g, int n, int mb, con
 __device__ __forceinline__ void l2_touch(const float* p) {
   float v;
   asm volatile("ld.global.L2::256B.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+  (void)v;
 }
 __device__ __forceinline__ void prefetch_epilogue_inputs(const TcArgs& g, int m0, int n0, int BN, int e) {
   if (!g.pf_ok || m0 >= g.M) return;
@@ -394,31 +439,35 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
 
   if (warp == 0 && lane == 0 && T > 0) {
     // ---------------- producer: TMA loads into the stage ring
-    long long git = 0, armed = 0;
+    RingPos r = {0, 0u, 0u};
+    long long armed = 0;
     for (int t = blockIdx.x; t < tiles && !*abort_flag; t += gridDim.x) {
       const int m0 = (t / tiles_n) * TC_BM, n0 = (t % tiles_n) * BN;
-      for (int it = 0; it < T; ++it, ++git) {
-        const int s = (int)(git % S);
-        if (git >= S && !tc_wait(&empty[s], (uint32_t)(((git / S) - 1) & 1), abort_flag)) break;
-        const int p = it < iters[0] ? 0 : 1;
-        const int k0 = (p == 0 ? it : it - iters[0]) * TC_BK;
-        const CUtensorMap* ta = p == 0 ? &tmA0 : &tmA1;
-        const CUtensorMap* tb = p == 0 ? &tmB0 : &tmB1;
-        unsigned char* sa = smem + s * Cfg::STAGE_BYTES;
+      int p = 0, k0 = 0;
+      const CUtensorMap* ta = &tmA0;
+      const CUtensorMap* tb = &tmB0;
+      bool a_mn = g.p[0].a_mn, b_mn = g.p[0].b_mn;
+      bool ok = true;
+      for (int it = 0; it < T; ++it, k0 += TC_BK) {
+        if (p == 0 && it == iters[0]) { p = 1; k0 = 0; ta = &tmA1; tb = &tmB1; a_mn = g.p[1].a_mn; b_mn = g.p[1].b_mn; }
+        if (r.round && !tc_wait(&empty[r.s], (r.round - 1) & 1u, abort_flag)) { ok = false; break; }
+        unsigned char* sa = smem + r.s * Cfg::STAGE_BYTES;
         unsigned char* sb = sa + TC_A_BYTES;
-        tc_expect_tx(&full[s], Cfg::STAGE_BYTES);
-        if (!g.p[p].a_mn) {
-          tma_load_2d(sa, ta, k0, m0, &full[s]);                                  // box 64(K) x 128(M)
+        tc_expect_tx(&full[r.s], Cfg::STAGE_BYTES);
+        if (!a_mn) {
+          tma_load_2d(sa, ta, k0, m0, &full[r.s]);                                  // box 64(K) x 128(M)
         } else {
-          for (int j = 0; j < TC_BM / 64; ++j) tma_load_2d(sa + j * 8192, ta, m0 + 64 * j, k0, &full[s]);   // box 64(M) x 64(K)
+          for (int j = 0; j < TC_BM / 64; ++j) tma_load_2d(sa + j * 8192, ta, m0 + 64 * j, k0, &full[r.s]);   // box 64(M) x 64(K)
         }
-        if (!g.p[p].b_mn) {
-          tma_load_2d(sb, tb, k0, n0, &full[s]);                                  // box 64(K) x BN(N)
+        if (!b_mn) {
+          tma_load_2d(sb, tb, k0, n0, &full[r.s]);                                  // box 64(K) x BN(N)
         } else {
-          for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, tb, n0 + 64 * j, k0, &full[s]);      // box 64(N) x 64(K)
+          for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, tb, n0 + 64 * j, k0, &full[r.s]);      // box 64(N) x 64(K)
         }
-        armed = git + 1;
+        ++armed;
+        r.advance(S, Cfg::STAGE_BYTES >> 4);
       }
+      if (!ok) break;
     }
     if (*abort_flag) {
       // let copies that were already issued land before the CTA's shared memory goes away
@@ -428,7 +477,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
     }
   } else if (warp == 1 && lane == 0 && T > 0) {
     // ---------------- MMA issuer
-    long long git = 0;
+    const uint32_t sa0 = s_u32(smem), sb0 = sa0 + TC_A_BYTES;
+    const IssuePlan plan0 = issue_plan(g.p[0], sa0, sb0, BN, TC_BM);
+    const IssuePlan plan1 = issue_plan(g.p[1], sa0, sb0, BN, TC_BM);
+    RingPos r = {0, 0u, 0u};
     int j = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++j) {
@@ -436,27 +488,20 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUte
       if (j >= 2 && !tc_wait(&acc_empty[as], (uint32_t)(((j >> 1) - 1) & 1), abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t tmem_acc = tmem_base + (uint32_t)(as * BN);
-      for (int it = 0; it < T; ++it, ++git) {
-        const int s = (int)(git % S);
-        if (!tc_wait(&full[s], (uint32_t)((git / S) & 1), abort_flag)) { ok = false; break; }
+      for (int it = 0; it < T; ++it) {
+        if (!tc_wait(&full[r.s], r.round & 1u, abort_flag)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int p = it < iters[0] ? 0 : 1;
-        const uint32_t idesc = instr_desc(g.p[p].a_mn, g.p[p].b_mn, g.p[p].neg, BN, TC_BM);
-        const uint32_t sa = s_u32(smem + s * Cfg::STAGE_BYTES), sb = sa + TC_A_BYTES;
+        const IssuePlan& pl = it < iters[0] ? plan0 : plan1;
+        uint64_t da = pl.a0 + r.off16, db = pl.b0 + r.off16;
+        mma_f16<1>(tmem_acc, da, db, pl.idesc, it > 0 ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < TC_BK / 16; ++kk) {
-          // K-major: 16 elements = 32 bytes further along the swizzled row; groups of 8 rows 1024 B apart.
-          // MN-major: 16 k-rows = 2048 bytes further; 64-element blocks along M/N 8192 B apart.
-          const uint64_t da = g.p[p].a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
-          const uint64_t db = g.p[p].b_mn ? smem_desc(sb + kk * 2048, 8192, 1024) : smem_desc(sb + kk * 32, 16, 1024);
-          const uint32_t acc = (it > 0 || kk > 0) ? 1u : 0u;
-          asm volatile(
-              "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-              "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-              ::"r"(tmem_acc), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+        for (int kk = 1; kk < TC_BK / 16; ++kk) {
+          da += pl.a_step; db += pl.b_step;
+          mma_f16<1>(tmem_acc, da, db, pl.idesc, 1u);
         }
         // the stage may be refilled once these MMAs have read it
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(&empty[s])) : "memory");
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(&empty[r.s])) : "memory");
+        r.advance(S, Cfg::STAGE_BYTES >> 4);
       }
       if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s_u32(&acc_full[as])) : "memory");
     }
@@ -536,8 +581,11 @@ __device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* t
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(s_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
 }
-__device__ __forceinline__ void commit_pair(uint32_t bar_cluster_addr) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
+// Arrival, once the MMAs issued so far have completed, on the barrier at this shared-memory offset in
+// both CTAs of the pair (multicast over the cluster; the mask names CTA ranks 0 and 1).
+__device__ __forceinline__ void commit_both(uint32_t bar_local_addr) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar_local_addr), "h"((uint16_t)3) : "memory");
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
@@ -584,35 +632,42 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUt
 
   if (warp == 0 && lane == 0 && T > 0) {
     // ---------------- producer (both CTAs): own half of A and of B; completion counted on the leader's barrier
-    long long git = 0;
+    RingPos r = {0, 0u, 0u};
+    const uint32_t full0 = map_to_cta(s_u32(&full[0]), 0);      // the leader's full[0]; barriers are 8 bytes apart
     for (int t = cluster_id; t < tiles && !*abort_flag; t += n_clusters) {
       const int m0 = (t / tiles_n) * (2 * TC_BM) + (int)rank * TC_BM, n0 = (t % tiles_n) * BN + (int)rank * HB;
-      for (int it = 0; it < T; ++it, ++git) {
-        const int s = (int)(git % S);
-        if (git >= S && !tc_wait(&empty[s], (uint32_t)(((git / S) - 1) & 1), abort_flag)) break;
-        const int p = it < iters[0] ? 0 : 1;
-        const int k0 = (p == 0 ? it : it - iters[0]) * TC_BK;
-        const CUtensorMap* ta = p == 0 ? &tmA0 : &tmA1;
-        const CUtensorMap* tb = p == 0 ? &tmB0 : &tmB1;
-        unsigned char* sa = smem + s * TC2_STAGE_BYTES;
+      int p = 0, k0 = 0;
+      const CUtensorMap* ta = &tmA0;
+      const CUtensorMap* tb = &tmB0;
+      bool a_mn = g.p[0].a_mn, b_mn = g.p[0].b_mn;
+      bool ok = true;
+      for (int it = 0; it < T; ++it, k0 += TC_BK) {
+        if (p == 0 && it == iters[0]) { p = 1; k0 = 0; ta = &tmA1; tb = &tmB1; a_mn = g.p[1].a_mn; b_mn = g.p[1].b_mn; }
+        if (r.round && !tc_wait(&empty[r.s], (r.round - 1) & 1u, abort_flag)) { ok = false; break; }
+        unsigned char* sa = smem + r.s * TC2_STAGE_BYTES;
         unsigned char* sb = sa + TC_A_BYTES;
-        const uint32_t bar = map_to_cta(s_u32(&full[s]), 0);
-        if (leader) tc_expect_tx(&full[s], 2 * TC2_STAGE_BYTES);
-        if (!g.p[p].a_mn) {
+        const uint32_t bar = full0 + 8u * (uint32_t)r.s;
+        if (leader) tc_expect_tx(&full[r.s], 2 * TC2_STAGE_BYTES);
+        if (!a_mn) {
           tma_load_2d_pair(sa, ta, k0, m0, bar);
         } else {
           for (int j = 0; j < TC_BM / 64; ++j) tma_load_2d_pair(sa + j * 8192, ta, m0 + 64 * j, k0, bar);
         }
-        if (!g.p[p].b_mn) {
+        if (!b_mn) {
           tma_load_2d_pair(sb, tb, k0, n0, bar);
         } else {
           for (int j = 0; j < HB / 64; ++j) tma_load_2d_pair(sb + j * 8192, tb, n0 + 64 * j, k0, bar);
         }
+        r.advance(S, TC2_STAGE_BYTES >> 4);
       }
+      if (!ok) break;
     }
   } else if (warp == 1 && lane == 0 && T > 0 && leader) {
     // ---------------- MMA issuer (even CTA of the pair only)
-    long long git = 0;
+    const uint32_t sa0 = s_u32(smem), sb0 = sa0 + TC_A_BYTES;
+    const IssuePlan plan0 = issue_plan(g.p[0], sa0, sb0, BN, 2 * TC_BM);
+    const IssuePlan plan1 = issue_plan(g.p[1], sa0, sb0, BN, 2 * TC_BM);
+    RingPos r = {0, 0u, 0u};
     int j = 0;
     bool ok = true;
     for (int t = cluster_id; t < tiles && ok; t += n_clusters, ++j) {
@@ -620,31 +675,22 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUt
       if (j >= 2 && !tc_wait(&acc_empty[as], (uint32_t)(((j >> 1) - 1) & 1), abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t tmem_acc = tmem_base + (uint32_t)(as * BN);
-      for (int it = 0; it < T; ++it, ++git) {
-        const int s = (int)(git % S);
-        if (!tc_wait(&full[s], (uint32_t)((git / S) & 1), abort_flag)) { ok = false; break; }
+      for (int it = 0; it < T; ++it) {
+        if (!tc_wait(&full[r.s], r.round & 1u, abort_flag)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int p = it < iters[0] ? 0 : 1;
-        const uint32_t idesc = instr_desc(g.p[p].a_mn, g.p[p].b_mn, g.p[p].neg, BN, 2 * TC_BM);
-        const uint32_t sa = s_u32(smem + s * TC2_STAGE_BYTES), sb = sa + TC_A_BYTES;
+        const IssuePlan& pl = it < iters[0] ? plan0 : plan1;
+        uint64_t da = pl.a0 + r.off16, db = pl.b0 + r.off16;
+        mma_f16<2>(tmem_acc, da, db, pl.idesc, it > 0 ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < TC_BK / 16; ++kk) {
-          const uint64_t da = g.p[p].a_mn ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
-          const uint64_t db = g.p[p].b_mn ? smem_desc(sb + kk * 2048, 8192, 1024) : smem_desc(sb + kk * 32, 16, 1024);
-          const uint32_t acc = (it > 0 || kk > 0) ? 1u : 0u;
-          asm volatile(
-              "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-              "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-              ::"r"(tmem_acc), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+        for (int kk = 1; kk < TC_BK / 16; ++kk) {
+          da += pl.a_step; db += pl.b_step;
+          mma_f16<2>(tmem_acc, da, db, pl.idesc, 1u);
         }
-        // both CTAs may refill the stage once these MMAs have read it
-        commit_pair(map_to_cta(s_u32(&empty[s]), 0));
-        commit_pair(map_to_cta(s_u32(&empty[s]), 1));
+        // both CTAs may refill the stage once these MMAs have read it: one arrival on empty[s] of each CTA
+        commit_both(s_u32(&empty[r.s]));
+        r.advance(S, TC2_STAGE_BYTES >> 4);
       }
-      if (ok) {
-        commit_pair(map_to_cta(s_u32(&acc_full[as]), 0));
-        commit_pair(map_to_cta(s_u32(&acc_full[as]), 1));
-      }
+      if (ok) commit_both(s_u32(&acc_full[as]));
     }
   } else if (warp >= 2) {
     // ---------------- epilogue (both CTAs): own 128 rows of the pair's tile

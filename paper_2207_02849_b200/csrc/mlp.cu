@@ -88,16 +88,26 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
 struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; float* s_out; };
 __global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
   pdl_enter();
-  // 1024 threads: 32 lanes x 2 adjacent columns, 32 row groups; ld is even, so a column pair is one 4-byte load
+  // 1024 threads: 32 lanes x 2 adjacent columns, 32 row groups; ld is even, so a column pair is one 4-byte load.
+  // A thread's loads are issued 16 at a time (the kernel is bound by latency, not by bytes).
   __shared__ float sh[32][65];
   const int cx = threadIdx.x & 31, rg = threadIdx.x >> 5;
   const int64_t n = blockIdx.x * 64 + 2 * cx;
   float a0 = 0.f, a1 = 0.f;
   if (n < N) {
-#pragma unroll 4
-    for (int64_t i = rg; i < B; i += 32) {
-      const float2 f = __bfloat1622float2(*(const __nv_bfloat162*)(d + i * ld + n));
-      a0 += f.x; a1 += f.y;
+    constexpr int U = 16;
+    for (int64_t i0 = rg; i0 < B; i0 += 32 * U) {
+      __nv_bfloat162 v[U];
+#pragma unroll
+      for (int k = 0; k < U; ++k) {
+        const int64_t i = i0 + 32 * k;
+        v[k] = i < B ? *(const __nv_bfloat162*)(d + i * ld + n) : __floats2bfloat162_rn(0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < U; ++k) {   // same order as a plain loop over the rows
+        const float2 f = __bfloat1622float2(v[k]);
+        a0 += f.x; a1 += f.y;
+      }
     }
   }
   sh[rg][2 * cx] = a0; sh[rg][2 * cx + 1] = a1;
@@ -390,6 +400,10 @@ struct MlpHvpCache {
   const float* coef;     // per-sample top coefficient (r_i/B) or null (1/B)
   const float* lam;      // device per-layer log weight decay or null
   const betty_level* theta;
+  // bf16 copies of a direction's matrices that outlive one HVP (series solves): the weight-HVP epilogues
+  // of iteration k leave the rounded next term here, so that iteration k+1 starts without a cast pass
+  bf16* dir16[MAXL];     // null: every R-forward pass rounds its direction into scratch of its own
+  const float* dir16_of; // the fp32 vector that dir16 currently mirrors, or null
 };
 
 static betty_status net_layout(const betty_level* M, Net& n) {
@@ -440,6 +454,10 @@ static betty_status cast_matrix(Ctx& c, const float* src, bf16* dst, int64_t row
 // bf16 compute copy of the classifier's matrices (the single quantisation point)
 static betty_status net_setup(Ctx& c, const betty_level* M, Net& n) {
   BETTY_TRY(net_layout(M, n));
+  if (c.shared.master == M->params) {
+    for (int l = 0; l < n.L; ++l) n.W[l] = c.shared.W[l];
+    return BETTY_OK;
+  }
   for (int l = 0; l < n.L; ++l) {
     BETTY_ALLOC(Wl, bf16, c, (size_t)(n.w[l + 1] * n.ldw[l]));
     n.W[l] = Wl;
@@ -447,6 +465,21 @@ static betty_status net_setup(Ctx& c, const betty_level* M, Net& n) {
   }
   return BETTY_OK;
 }
+
+// Rounds the matrices of MLP level M once, at the arena's current top, for every pass of this call that
+// evaluates a cost at M's present parameters.  The caller guarantees that the parameters do not change
+// and that the arena is not released below this point while the copies are shared, and ends the sharing
+// with mlpfam_unshare_weights.
+betty_status mlpfam_share_weights(Ctx& c, const betty_level* M) {
+  c.shared.master = nullptr;
+  if (!M || M->param_kind != BETTY_PARAM_MLP) return BETTY_OK;
+  Net n;
+  BETTY_TRY(net_setup(c, M, n));
+  for (int l = 0; l < n.L; ++l) c.shared.W[l] = n.W[l];
+  c.shared.master = M->params;
+  return BETTY_OK;
+}
+void mlpfam_unshare_weights(Ctx& c) { c.shared.master = nullptr; }
 
 static betty_status forward(Ctx& c, const Net& n, const betty_level* D, Pass& ps) {
   ps.B = D->n;
@@ -494,7 +527,7 @@ struct GradSink {
 
 // Reverse sweep from delta_top = coef_i (p - onehot).  Always leaves delta[l] (and dh[l] for smooth
 // activations) in `ps` for an R-operator pass.
-static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, const GradSink& sink) {
+static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, const GradSink& sink, bool keep_dh = false) {
   const int64_t B = ps.B;
   const int64_t C = n.w[n.L];
   {
@@ -529,9 +562,9 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
     }
     if (l > 0) {
       // dh = delta_l W_l ; delta_{l-1} = dh * act'(a_{l-1}) in bf16: one kernel.  dh itself is kept
-      // only when the activation has a second derivative (the R-operator pass needs it then).
+      // only for an R-operator pass over an activation with a second derivative.
       float* dh = nullptr;
-      if (n.act != BETTY_ACT_RELU) {
+      if (keep_dh && n.act != BETTY_ACT_RELU) {
         dh = c.arena.alloc<float>((size_t)(B * K));
         if (!dh) return BETTY_ERR_WORKSPACE;
       }
@@ -558,14 +591,17 @@ struct RPass {
   float* Ra[MAXL];
   const bf16* Rh[MAXL];   // Rh[0] == nullptr (inputs do not move)
 };
-static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* dir, RPass& rp) {
+static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* dir, RPass& rp, MlpHvpCache* keep) {
   const int64_t B = ps.B;
   rp.Rh[0] = nullptr;
+  const bool kept = keep && keep->dir16[0];
+  const bool fresh = kept && keep->dir16_of == dir;      // the kept copies already mirror this direction
   for (int l = 0; l < n.L; ++l) {
     const int64_t N = n.w[l + 1], K = n.w[l];
-    BETTY_ALLOC(Ul, bf16, c, (size_t)(N * n.ldw[l]));
+    bf16* Ul = kept ? keep->dir16[l] : c.arena.alloc<bf16>((size_t)(N * n.ldw[l]));
+    if (!Ul) return BETTY_ERR_WORKSPACE;
     rp.U[l] = Ul;
-    BETTY_TRY(cast_matrix(c, dir + n.woff[l], Ul, N, K, n.ldw[l]));
+    if (!fresh) BETTY_TRY(cast_matrix(c, dir + n.woff[l], Ul, N, K, n.ldw[l]));
     BETTY_ALLOC(Ra, float, c, (size_t)(B * N));
     rp.Ra[l] = Ra;
     bf16* Rhn = nullptr;
@@ -584,6 +620,7 @@ static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* 
     g.epi.out16 = Rhn; g.epi.ld16 = Rhn ? ps.ldh[l + 1] : 0;
     BETTY_TRY(gemm(c, g));
   }
+  if (kept) keep->dir16_of = dir;
   return BETTY_OK;
 }
 
@@ -719,11 +756,13 @@ betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache)
   h.theta = P.theta;
   h.lam = P.lam ? P.lam->params : nullptr;
   h.coef = nullptr;
+  for (int l = 0; l < MAXL; ++l) h.dir16[l] = nullptr;
+  h.dir16_of = nullptr;
   BETTY_TRY(net_setup(c, P.mlp, h.net));
   BETTY_TRY(forward(c, h.net, L, h.pass));
   if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
     BETTY_TRY(reweight_coef(c, P, h.pass, &h.coef));
-    BETTY_TRY(backward(c, h.net, h.pass, h.coef, grad_into(nullptr, nullptr)));
+    BETTY_TRY(backward(c, h.net, h.pass, h.coef, grad_into(nullptr, nullptr), true));
   } else if (!(L->loss == BETTY_LOSS_WEIGHTNET_DETECT && L->param_kind == BETTY_PARAM_WEIGHTNET)) {
     return BETTY_ERR_UNSUPPORTED;
   }
@@ -754,7 +793,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
     return BETTY_OK;
   }
   RPass rp;
-  BETTY_TRY(rforward(c, n, ps, u, rp));
+  BETTY_TRY(rforward(c, n, ps, u, rp, h));
   const int64_t C = n.w[n.L];
   bf16* Rd;
   {
@@ -765,8 +804,23 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
                                                          B, C, ld);
     BETTY_LAUNCH_CHECK();
   }
+  const bool leave16 = sink && h->dir16[0];     // the weight-HVP epilogues also leave bf16(t_out) in dir16
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
+    bf16* Rdp = nullptr;
+    if (l > 0) {  // R dh = Rdelta W_l + delta_l U_l ; Rdelta_{l-1} = Rdh*act' + dh*act''*Ra
+      // (before this layer's weight product, whose epilogue may overwrite U_l with the next term)
+      const int64_t ldp = ld8(K);
+      Rdp = c.arena.alloc<bf16>((size_t)(B * ldp));
+      if (!Rdp) return BETTY_ERR_WORKSPACE;
+      if (ldp != K) cudaMemsetAsync(Rdp, 0, (size_t)(B * ldp) * sizeof(bf16), c.stream);
+      GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.C = nullptr; g.ldc = K; g.beta = 0.f; g.npairs = 2;
+      g.p[0] = gemm_pair(Rd, ldd, false, n.W[l], n.ldw[l], false, (int)N);
+      g.p[1] = gemm_pair(ps.delta[l], ldd, false, rp.U[l], n.ldw[l], false, (int)N);
+      g.epi.mode = EPI_R_BWD; g.epi.act = n.act; g.epi.a = ps.a[l - 1]; g.epi.dh = ps.dh[l]; g.epi.Ra = rp.Ra[l - 1];
+      g.epi.out16 = Rdp; g.epi.ld16 = ldp;
+      BETTY_TRY(gemm(c, g));
+    }
     {  // R gW_l = Rdelta^T h_l + delta_l^T Rh_l + exp(lam_l) U_l
       GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.ldc = K; g.beta = 0.f; g.npairs = 0;
       g.p[g.npairs++] = gemm_pair(Rd, ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
@@ -776,6 +830,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
         g.C = sink->t_out + n.woff[l];
         g.epi.mode = EPI_NEUMANN; g.epi.lam = h->lam ? h->lam + l : nullptr; g.epi.step = sink->alpha;
         g.epi.t_in = u + n.woff[l]; g.epi.s_in = sink->s_in + n.woff[l]; g.epi.s_out = sink->s_out + n.woff[l];
+        if (leave16) { g.epi.out16 = h->dir16[l]; g.epi.ld16 = n.ldw[l]; }
         cs.mode = 2; cs.step = sink->alpha; cs.out = sink->t_out + n.boff[l]; cs.t_in = u + n.boff[l];
         cs.s_in = sink->s_in + n.boff[l]; cs.s_out = sink->s_out + n.boff[l];
       } else {
@@ -790,20 +845,23 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
       launch_pdl(k_colsum_bf16, dim3((unsigned)((N + 63) / 64)), dim3(1024), 0, c.stream, Rd, B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
-    if (l > 0) {  // R dh = Rdelta W_l + delta_l U_l ; Rdelta_{l-1} = Rdh*act' + dh*act''*Ra
-      const int64_t ldp = ld8(K);
-      BETTY_ALLOC(Rdp, bf16, c, (size_t)(B * ldp));
-      if (ldp != K) cudaMemsetAsync(Rdp, 0, (size_t)(B * ldp) * sizeof(bf16), c.stream);
-      GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.C = nullptr; g.ldc = K; g.beta = 0.f; g.npairs = 2;
-      g.p[0] = gemm_pair(Rd, ldd, false, n.W[l], n.ldw[l], false, (int)N);
-      g.p[1] = gemm_pair(ps.delta[l], ldd, false, rp.U[l], n.ldw[l], false, (int)N);
-      g.epi.mode = EPI_R_BWD; g.epi.act = n.act; g.epi.a = ps.a[l - 1]; g.epi.dh = ps.dh[l]; g.epi.Ra = rp.Ra[l - 1];
-      g.epi.out16 = Rdp; g.epi.ld16 = ldp;
-      BETTY_TRY(gemm(c, g));
-      Rd = Rdp;
-    }
+    if (l > 0) Rd = Rdp;
   }
+  if (leave16) h->dir16_of = sink->t_out;
   c.arena.release(mark);
+  return BETTY_OK;
+}
+
+// Gives the HVPs of a series solve persistent storage for the bf16 copy of the current term (allocated
+// at the arena's current top: call it after mlpfam_hvp_begin and before the first HVP of the solve).
+betty_status mlpfam_hvp_keep_direction(Ctx& c, MlpHvpCache* h) {
+  if (!h || h->dir16[0]) return BETTY_OK;
+  const Net& n = h->net;
+  for (int l = 0; l < n.L; ++l) {
+    h->dir16[l] = c.arena.alloc<bf16>((size_t)(n.w[l + 1] * n.ldw[l]));
+    if (!h->dir16[l]) { h->dir16[0] = nullptr; return BETTY_ERR_WORKSPACE; }
+  }
+  h->dir16_of = nullptr;
   return BETTY_OK;
 }
 
@@ -831,7 +889,7 @@ betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const be
       }
     } else if (P.theta && wrt == P.theta) {
       RPass rp;
-      BETTY_TRY(rforward(c, n, ps, q, rp));
+      BETTY_TRY(rforward(c, n, ps, q, rp, h));
       BETTY_ALLOC(d, float, c, (size_t)(B > 0 ? B : 1));
       BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
       launch_pdl(k_jvp_rows, dim3(grid_for(B * 32)), dim3(256), 0, c.stream, ps.p, ps.y, rp.Ra[n.L - 1], d, B, n.w[n.L]);

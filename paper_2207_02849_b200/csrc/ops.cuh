@@ -49,7 +49,10 @@ struct MlpHvpCache;  // base forward/backward state shared by the HVPs of one so
 betty_status mlpfam_validate(const betty_level* L);
 size_t mlpfam_workspace(const betty_level* L);
 betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);
+betty_status mlpfam_share_weights(Ctx& c, const betty_level* M);
+void mlpfam_unshare_weights(Ctx& c);
 betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache);
+betty_status mlpfam_hvp_keep_direction(Ctx& c, MlpHvpCache* cache);
 betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* u, float* Hu);
 // One Neumann-series iteration with the update fused into the HVP's weight-gradient products:
 // t_out = t_in - alpha * H t_in ; s_out = s_in + t_out  (t_in == t_out and s_in == s_out allowed)
