@@ -220,19 +220,20 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
   BETTY_ALLOC(m, float, c, (size_t)nc);
   float qscale = 1.f;
   if (cfg.method == BETTY_NEUMANN) {
-    // t_0 = s_0 = v are read straight from v in the first iteration: no copies
-    BETTY_ALLOC(t, float, c, (size_t)n);
-    if (!vecfam && cfg.K > 1 && L->param_kind == BETTY_PARAM_MLP) BETTY_TRY(mlpfam_hvp_keep_direction(c, cache));
     if (cfg.K == 0) BETTY_TRY(vec_copy(c, q, v, n));
-    for (int k = 0; k < cfg.K; ++k) {
-      const float* t_in = k == 0 ? v : t;
-      const float* s_in = k == 0 ? v : q;
-      if (vecfam) {
+    if (vecfam) {
+      // term / sum recurrence; t_0 = s_0 = v are read straight from v in the first iteration: no copies
+      BETTY_ALLOC(t, float, c, (size_t)n);
+      for (int k = 0; k < cfg.K; ++k) {
+        const float* t_in = k == 0 ? v : t;
+        const float* s_in = k == 0 ? v : q;
         BETTY_TRY(vecfam_hvp(c, L, t_in, h));
         BETTY_TRY(neumann_update(c, t_in, s_in, h, cfg.alpha, t, q, n));
-      } else {
-        BETTY_TRY(mlpfam_hvp_neumann(c, L, cache, t_in, s_in, cfg.alpha, t, q));
       }
+    } else {
+      // the same sum by Horner's rule, q <- v + (I - alpha H) q from q = v, fused into the HVP's epilogues
+      if (cfg.K > 0 && L->param_kind == BETTY_PARAM_MLP) BETTY_TRY(mlpfam_hvp_keep_direction(c, cache));
+      for (int k = 0; k < cfg.K; ++k) BETTY_TRY(mlpfam_hvp_series(c, L, cache, k == 0 ? v : q, v, cfg.alpha, q));
     }
     qscale = cfg.alpha;   // q holds the plain sum; alpha is applied with the sign below
   } else {

@@ -20,7 +20,7 @@ enum GemmEpiMode {
   EPI_R_FWD = 3,     // v = acc + bias[n];  C = v;  out16 = act'(a[m,n]) * v             (R-operator forward)
   EPI_R_BWD = 4,     // out16 = acc * act'(a) + dh * act''(a) * Ra                       (R-operator backward)
   EPI_SGD = 5,       // g = acc + exp(lam) * w16;  C = C - lr * g;  out16 = bf16(new C)  (weight gradient -> gradient step; w16 == bf16(C))
-  EPI_NEUMANN = 6    // Hu = acc + exp(lam) * t_in;  t = t_in - alpha * Hu -> C;  s_out = s_in + t;  out16 = bf16(t) if given   (weight HVP -> series update)
+  EPI_NEUMANN = 6    // Hu = acc + exp(lam) * t_in;  C = s_in + t_in - alpha * Hu;  out16 = bf16(C) if given   (weight HVP -> one Horner step of the Neumann series)
 };
 struct GemmEpilogue {
   int mode;
@@ -36,9 +36,8 @@ struct GemmEpilogue {
   const bf16* w16;         // EPI_SGD: bf16 weights the gradient was taken at, leading dimension ldw16
   int64_t ldw16;
   float step;              // EPI_SGD: learning rate; EPI_NEUMANN: alpha
-  const float* t_in;       // EPI_NEUMANN: current series term (the HVP direction)
-  const float* s_in;       // EPI_NEUMANN: running sum in
-  float* s_out;            // EPI_NEUMANN: running sum out
+  const float* t_in;       // EPI_NEUMANN: the HVP direction = the partial sum so far (may alias C)
+  const float* s_in;       // EPI_NEUMANN: the series' constant term v
 };
 struct GemmDesc {
   int M, N;
@@ -118,9 +117,8 @@ __device__ __forceinline__ void gemm_epilogue_store(const GemmEpilogue& e, float
       const float ti = e.t_in[jc];
       float hu = acc;
       if (e.lam) hu += expf(*e.lam) * ti;
-      const float tn = ti - e.step * hu;
+      const float tn = e.s_in[jc] + (ti - e.step * hu);
       *cp = tn;
-      e.s_out[jc] = e.s_in[jc] + tn;
       if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(tn);
       break;
     }

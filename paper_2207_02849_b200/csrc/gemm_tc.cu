@@ -165,11 +165,8 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
         const float4 s0 = *(const float4*)(e.s_in + jc), s1 = *(const float4*)(e.s_in + jc + 4);
         const float tv[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
         const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-        float so[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { v[k] = tv[k] - e.step * (v[k] + kap * tv[k]); so[k] = sv[k] + v[k]; o[k] = v[k]; }
-        *(float4*)(e.s_out + jc) = make_float4(so[0], so[1], so[2], so[3]);
-        *(float4*)(e.s_out + jc + 4) = make_float4(so[4], so[5], so[6], so[7]);
+        for (int k = 0; k < 8; ++k) { v[k] = sv[k] + (tv[k] - e.step * (v[k] + kap * tv[k])); o[k] = v[k]; }
       } else {   // EPI_ACT_BWD, EPI_R_BWD
         const float4 a0 = *(const float4*)(e.a + jb + j8), a1 = *(const float4*)(e.a + jb + j8 + 4);
         const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
@@ -223,7 +220,6 @@ __device__ __forceinline__ void epilogue_t32_rows(const TcArgs& g, int n, int mb
   const float* qp = e.Ra ? e.Ra + (int64_t)mb * NC + n : nullptr;
   const float* tp = e.t_in ? e.t_in + (int64_t)mb * g.ldc + n : nullptr;
   const float* sp = e.s_in ? e.s_in + (int64_t)mb * g.ldc + n : nullptr;
-  float* so = e.s_out ? e.s_out + (int64_t)mb * g.ldc + n : nullptr;
   bf16* op = e.out16 ? e.out16 + (int64_t)mb * e.ld16 + n : nullptr;
   const int rows = MC - mb;     // > 0; FULL: >= 32, and no per-row guards, so that the rows' dependency chains interleave
   const bool second = MODE == EPI_R_BWD && ACT != BETTY_ACT_RELU;
@@ -278,9 +274,8 @@ __device__ __forceinline__ void epilogue_t32_rows(const TcArgs& g, int n, int mb
           if (op) *o1 = __float2bfloat16_rn(w);
         }
         if (MODE == EPI_NEUMANN) {
-          const float tn = x0[k] - e.step * (acc + kap * x0[k]);
+          const float tn = x1[k] + (x0[k] - e.step * (acc + kap * x0[k]));
           *c1 = tn;
-          so[(int64_t)j * g.ldc] = x1[k] + tn;
           if (op) *o1 = __float2bfloat16_rn(tn);
         }
       }
@@ -842,8 +837,7 @@ static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a, bool tr) {
   auto al16 = [](const void* p) { return (((uintptr_t)p) & 15) == 0; };
   const GemmEpilogue& e = g.epi;
   const bool ok = (g.N % 4 == 0) && al16(g.C) && (g.ldc % 4 == 0) && al16(e.bias) && al16(e.a) && al16(e.dh) && al16(e.Ra) &&
-                  al16(e.out16) && (e.ld16 % 8 == 0) && al16(e.w16) && (e.ldw16 % 8 == 0) && al16(e.t_in) && al16(e.s_in) &&
-                  al16(e.s_out);
+                  al16(e.out16) && (e.ld16 % 8 == 0) && al16(e.w16) && (e.ldw16 % 8 == 0) && al16(e.t_in) && al16(e.s_in);
   a.vec_ok = ok ? 1 : 0;
   a.pf_ok = tr ? 1 : 0;
   for (int i = 0; i < 2; ++i) {

@@ -84,8 +84,8 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
 // Column sums sum_i d[i, n] (bias gradients), with the consumer fused in.  Block = 32 columns x 8 row
 // groups; fixed summation order.
 //   mode 0: out[n] = sum            mode 1: out[n] -= step * sum   (gradient step on a bias)
-//   mode 2: t = t_in[n] - step * sum; out[n] = t; s_out[n] = s_in[n] + t   (Neumann-series update)
-struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; float* s_out; };
+//   mode 2: out[n] = s_in[n] + t_in[n] - step * sum   (one Horner step of the Neumann series; out may alias t_in)
+struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; };
 __global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
   pdl_enter();
   // 1024 threads: 32 lanes x 2 adjacent columns, 32 row groups; ld is even, so a column pair is one 4-byte load.
@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, 
       for (int r = 0; r < 32; ++r) t += sh[r][threadIdx.x];
       if (k.mode == 0) k.out[nn] = t;
       else if (k.mode == 1) k.out[nn] -= k.step * t;
-      else { const float tn = k.t_in[nn] - k.step * t; k.out[nn] = tn; k.s_out[nn] = k.s_in[nn] + tn; }
+      else k.out[nn] = k.s_in[nn] + (k.t_in[nn] - k.step * t);
     }
   }
 }
@@ -770,11 +770,14 @@ betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache)
   return BETTY_OK;
 }
 
-// Neumann-series consumer of an HVP: t_out = t_in - alpha * H t_in ; s_out = s_in + t_out
-struct SeriesSink { const float* s_in; float alpha; float* t_out; float* s_out; };
+// Neumann-series consumer of an HVP.  The truncated series alpha * sum_{j<=K} (I - alpha H)^j v is
+// evaluated by Horner's rule, s <- v + (I - alpha H) s starting from s = v: per step one vector is read
+// as the HVP direction, v is read and the new partial sum written (the term/sum recurrence reads and
+// writes two vectors per step; at 138M parameters that is 1.1 GB less traffic per step).
+struct SeriesSink { const float* v; float alpha; float* out; };
 
-// H u.  Without a sink the product is written to Hu; with one, u is the current series term t_in and
-// the update is applied inside the weight-gradient products and bias column sums (Hu is not used).
+// H u.  Without a sink the product is written to Hu; with one, u is the partial sum so far and the
+// Horner step is applied inside the weight-gradient products and bias column sums (Hu is not used).
 static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* u, float* Hu,
                              const SeriesSink* sink) {
   const size_t mark = c.arena.mark();
@@ -788,7 +791,10 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
     float* dst = Hu;
     if (sink) { dst = c.arena.alloc<float>(512); if (!dst) return BETTY_ERR_WORKSPACE; }
     BETTY_TRY(wn_backward(c, L, u, ps, cA, cB, L->mu, u, dst));
-    if (sink) BETTY_TRY(neumann_update(c, u, sink->s_in, dst, sink->alpha, sink->t_out, sink->s_out, WN_P));
+    if (sink) {   // out = v + (u - alpha H u)
+      BETTY_ALLOC(tmp, float, c, 512);
+      BETTY_TRY(neumann_update(c, u, sink->v, dst, sink->alpha, tmp, sink->out, WN_P));
+    }
     c.arena.release(mark);
     return BETTY_OK;
   }
@@ -804,7 +810,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
                                                          B, C, ld);
     BETTY_LAUNCH_CHECK();
   }
-  const bool leave16 = sink && h->dir16[0];     // the weight-HVP epilogues also leave bf16(t_out) in dir16
+  const bool leave16 = sink && h->dir16[0];     // the weight-HVP epilogues also leave the bf16 copy of the new partial sum in dir16
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
     bf16* Rdp = nullptr;
@@ -827,12 +833,12 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
       if (l > 0) g.p[g.npairs++] = gemm_pair(ps.delta[l], ldd, true, rp.Rh[l], ps.ldh[l], false, (int)B);
       ColsumSink cs = {};
       if (sink) {
-        g.C = sink->t_out + n.woff[l];
+        g.C = sink->out + n.woff[l];
         g.epi.mode = EPI_NEUMANN; g.epi.lam = h->lam ? h->lam + l : nullptr; g.epi.step = sink->alpha;
-        g.epi.t_in = u + n.woff[l]; g.epi.s_in = sink->s_in + n.woff[l]; g.epi.s_out = sink->s_out + n.woff[l];
+        g.epi.t_in = u + n.woff[l]; g.epi.s_in = sink->v + n.woff[l];
         if (leave16) { g.epi.out16 = h->dir16[l]; g.epi.ld16 = n.ldw[l]; }
-        cs.mode = 2; cs.step = sink->alpha; cs.out = sink->t_out + n.boff[l]; cs.t_in = u + n.boff[l];
-        cs.s_in = sink->s_in + n.boff[l]; cs.s_out = sink->s_out + n.boff[l];
+        cs.mode = 2; cs.step = sink->alpha; cs.out = sink->out + n.boff[l]; cs.t_in = u + n.boff[l];
+        cs.s_in = sink->v + n.boff[l];
       } else {
         g.C = Hu + n.woff[l];
         cs.mode = 0; cs.out = Hu + n.boff[l];
@@ -847,7 +853,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
     }
     if (l > 0) Rd = Rdp;
   }
-  if (leave16) h->dir16_of = sink->t_out;
+  if (leave16) h->dir16_of = sink->out;
   c.arena.release(mark);
   return BETTY_OK;
 }
@@ -869,10 +875,10 @@ betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const floa
   return hvp_impl(c, L, h, u, Hu, nullptr);
 }
 
-betty_status mlpfam_hvp_neumann(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* t_in, const float* s_in,
-                                float alpha, float* t_out, float* s_out) {
-  SeriesSink sink = {s_in, alpha, t_out, s_out};
-  return hvp_impl(c, L, h, t_in, nullptr, &sink);
+betty_status mlpfam_hvp_series(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* s, const float* v, float alpha,
+                               float* s_out) {
+  SeriesSink sink = {v, alpha, s_out};
+  return hvp_impl(c, L, h, s, nullptr, &sink);
 }
 
 betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const betty_level* wrt, const float* q,

@@ -55,9 +55,9 @@ betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache)
 betty_status mlpfam_hvp_keep_direction(Ctx& c, MlpHvpCache* cache);
 betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* u, float* Hu);
 // One Neumann-series iteration with the update fused into the HVP's weight-gradient products:
-// t_out = t_in - alpha * H t_in ; s_out = s_in + t_out  (t_in == t_out and s_in == s_out allowed)
-betty_status mlpfam_hvp_neumann(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* t_in, const float* s_in,
-                                float alpha, float* t_out, float* s_out);
+// One Horner step of the Neumann series: s_out = v + (s - alpha * H s)   (s_out == s allowed)
+betty_status mlpfam_hvp_series(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* s, const float* v, float alpha,
+                               float* s_out);
 betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* cache, const betty_level* wrt, const float* q,
                           float* out);
 betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps);
