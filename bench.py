@@ -75,6 +75,9 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        t_wait = time.time()
+        while not self.lines and time.time() - t_wait < 3.0:    # nvidia-smi needs about a second for its first line
+            time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -83,7 +86,8 @@ class ClockSampler:
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         inside = [ln for (t, ln) in self.lines if self.t0 is not None and self.t0 <= t <= (self.t1 or t) + 0.05]
-        if not inside:      # region shorter than one sampling period: fall back to every sample taken under load
+        short = not inside
+        if short:           # region shorter than one sampling period: fall back to every sample taken
             inside = [ln for (_, ln) in self.lines]
         for ln in inside:
             f = [x.strip() for x in ln.split(",")]
@@ -96,8 +100,11 @@ class ClockSampler:
             for nm, v in zip(names, f[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(nm)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        out = {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+               "samples": len(sm), "reasons": sorted(reasons)}
+        if short:
+            out["note"] = "timed region shorter than one sampling period: samples taken next to it"
+        return out
 
 
 # ------------------------------------------------------------------------------ workloads

@@ -104,6 +104,16 @@ typedef enum { BETTY_F32 = 0, BETTY_BF16 = 1, BETTY_I32 = 2 } betty_dtype;
  * n_params floats, ADAM 2 * n_params + 1 (the last one counts steps). */
 typedef enum { BETTY_OPT_GD = 0, BETTY_OPT_MOMENTUM = 1, BETTY_OPT_ADAM = 2 } betty_optimizer;
 
+/* Step size as a function of the number t of steps the problem has already taken (App. C trains the
+ * classifiers with a step size "decayed by a factor of 10" at two given iterations, or "decayed with the
+ * cosine annealing schedule" to a minimum by the end of training).
+ *  CONSTANT : lr
+ *  MULTISTEP: lr * lr_gamma^(number of lr_milestones[i] > 0 with lr_milestones[i] <= t)
+ *  COSINE   : lr_min + (lr - lr_min) * (1 + cos(pi * min(t, lr_t_max) / lr_t_max)) / 2
+ * t = lr_step0 + the steps taken so far inside the call (betty_lower_step, betty_hypergrad_itd,
+ * betty_engine_run); the caller advances lr_step0 between calls.  The value is worked out on the host. */
+typedef enum { BETTY_LR_CONSTANT = 0, BETTY_LR_MULTISTEP = 1, BETTY_LR_COSINE = 2 } betty_lr_schedule;
+
 /* Approximation of one best-response Jacobian (Sec. 3.2).
  *  NEUMANN: q = alpha * sum_{j=0..K} (I - alpha H)^j v   (K Hessian-vector products)
  *  CG     : K iterations of conjugate gradient on H q = v from q = 0; stops early once
@@ -140,6 +150,12 @@ typedef struct betty_level {
   float* opt_state;     /* device fp32 state, see betty_optimizer; NULL for GD */
   int32_t n_constraints;
   const struct betty_level* const* constraints; /* host array: U_k and L_k providers */
+  int32_t lr_schedule;  /* betty_lr_schedule; the fields below are read only when it is not CONSTANT */
+  int32_t lr_step0;     /* steps this problem had taken before this call */
+  int32_t lr_t_max;     /* COSINE: length of the schedule in steps (> 0) */
+  int32_t lr_milestones[4]; /* MULTISTEP: step counts at which the step size drops; unused entries 0 */
+  float lr_gamma;       /* MULTISTEP: factor per milestone passed */
+  float lr_min;         /* COSINE: step size reached at lr_t_max */
 } betty_level;
 
 /* Scratch bytes sufficient for any call below on these levels (Sec. 2: the whole program). */
@@ -155,7 +171,7 @@ betty_status betty_reset_status(void* ws, size_t ws_bytes, void* stream);
 betty_status betty_poll_status(const void* ws, void* stream, int32_t* cg_iters);
 
 /* Sec. 3.2 (approximating w* by unrolled gradient steps): n_steps times
- * params <- params - lr * dC/d(params) on the level's batch.  MLP blocks: the gradient is taken
+ * params <- params - lr_t * dC/d(params) on the level's batch (lr_t: betty_lr_schedule).  MLP blocks: the gradient is taken
  * at the bf16-rounded copy of the fp32 master, re-derived every step. */
 betty_status betty_lower_step(const betty_level* L, int32_t n_steps, void* ws, size_t ws_bytes,
                               void* stream);

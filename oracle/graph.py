@@ -55,7 +55,7 @@ def engine_run(levels, u2l, l2u, cfgs, unroll, n_iterations):
     def step(j):
         log.append(j)
         g = hypergrad_graph(levels, u2l, l2u, j, cfgs)
-        apply_optimizer(levels[j], g)
+        apply_optimizer(levels[j], g, count[j])
         count[j] += 1
         if count[j] % unroll[j] == 0:
             for a, b in l2u:

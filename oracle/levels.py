@@ -57,6 +57,12 @@ class Level:
     adam_eps: float = 1e-8
     weight_decay: float = 0.0
     opt_state: dict = field(default_factory=dict)
+    lr_schedule: str = "constant"      # 'constant' | 'multistep' | 'cosine' (App. C: decay by 10 at given iterations / cosine annealing)
+    lr_step0: int = 0                  # steps taken before the present call
+    lr_milestones: tuple = ()
+    lr_gamma: float = 0.1
+    lr_t_max: int = 1
+    lr_min: float = 0.0
 
     def __post_init__(self):
         self.params = np.array(self.params, dtype=np.float64).reshape(-1)

@@ -29,25 +29,43 @@ hvp = _lv.hvp
 mixed_vjp = _lv.mixed_vjp
 
 
-def apply_optimizer(L: Level, g: np.ndarray) -> None:
+def lr_at(L: Level, step_in_call: int) -> float:
+    """Step size of the problem's step number t = lr_step0 + step_in_call (App. C: the classifiers' step
+    size is "decayed by a factor of 10" at stated iterations, or follows "the cosine annealing schedule"
+    down to a minimum at the end of training; the weight net's is constant)."""
+    t = int(L.lr_step0) + int(step_in_call)
+    if L.lr_schedule == "constant":
+        return float(L.lr)
+    if L.lr_schedule == "multistep":
+        passed = sum(1 for m in L.lr_milestones if m > 0 and t >= m)
+        return float(L.lr) * float(L.lr_gamma) ** passed
+    if L.lr_schedule == "cosine":
+        u = min(t, L.lr_t_max) / float(L.lr_t_max)
+        return float(L.lr_min) + (float(L.lr) - float(L.lr_min)) * 0.5 * (1.0 + np.cos(np.pi * u))
+    raise ValueError(L.lr_schedule)
+
+
+def apply_optimizer(L: Level, g: np.ndarray, step_in_call: int = 0) -> None:
     """One step of the problem's optimiser along gradient g (App. C names SGD with momentum and weight
-    decay for the classifiers and Adam for the weight net; the update rules are the standard ones)."""
+    decay for the classifiers and Adam for the weight net; the update rules are the standard ones),
+    with the step size of the schedule at this step."""
     x = L.params
+    lr = lr_at(L, step_in_call)
     if L.optimizer == "gd":
-        L.params = x - L.lr * g
+        L.params = x - lr * g
         return
     gg = g + L.weight_decay * x
     st = L.opt_state
     if L.optimizer == "momentum":
         st["buf"] = L.momentum * st.get("buf", np.zeros_like(x)) + gg
-        L.params = x - L.lr * st["buf"]
+        L.params = x - lr * st["buf"]
     elif L.optimizer == "adam":
         st["t"] = st.get("t", 0) + 1
         st["m"] = L.beta1 * st.get("m", np.zeros_like(x)) + (1.0 - L.beta1) * gg
         st["v"] = L.beta2 * st.get("v", np.zeros_like(x)) + (1.0 - L.beta2) * gg * gg
         mhat = st["m"] / (1.0 - L.beta1 ** st["t"])
         vhat = st["v"] / (1.0 - L.beta2 ** st["t"])
-        L.params = x - L.lr * mhat / (np.sqrt(vhat) + L.adam_eps)
+        L.params = x - lr * mhat / (np.sqrt(vhat) + L.adam_eps)
     else:
         raise ValueError(L.optimizer)
 
@@ -57,8 +75,8 @@ def lower_step(L: Level, n_steps: int) -> None:
     approximated by a small number of unrolled gradient steps).  Updates L.params in place.
     For mixed-precision levels the gradient is taken at the bf16-rounded copy of the
     current master, which is re-derived at every step."""
-    for _ in range(int(n_steps)):
-        apply_optimizer(L, grad(L, L))
+    for s in range(int(n_steps)):
+        apply_optimizer(L, grad(L, L), s)
 
 
 def neumann_solve(hv, v, K: int, alpha: float) -> np.ndarray:
@@ -156,15 +174,16 @@ def hypergrad_itd(lower: Level, upper: Level, wrt: Level, n_steps: int) -> np.nd
     if lower.optimizer != "gd":
         raise ValueError("ITD-RMAD differentiates plain gradient-descent steps")
     xs = []
-    for _ in range(int(n_steps)):
+    for t in range(int(n_steps)):
         xs.append(lower.params.copy())
-        lower.params = lower.params - lower.lr * grad(lower, lower)
+        lower.params = lower.params - lr_at(lower, t) * grad(lower, lower)
     a = grad(upper, lower)
     out = grad(upper, wrt).copy()
-    for x_t in reversed(xs):
-        over = {id(lower): x_t}
-        out = out - lower.lr * mixed_vjp(lower, wrt, a, over)
-        a = a - lower.lr * hvp(lower, a, over)
+    for t in reversed(range(len(xs))):
+        over = {id(lower): xs[t]}
+        lr_t = lr_at(lower, t)
+        out = out - lr_t * mixed_vjp(lower, wrt, a, over)
+        a = a - lr_t * hvp(lower, a, over)
     return out
 
 

@@ -22,6 +22,7 @@ BETTY_NEUMANN, BETTY_CG, BETTY_FD = range(3)
 ACT_RELU, ACT_GELU = range(2)
 BETTY_F32, BETTY_BF16, BETTY_I32 = range(3)
 BETTY_OPT_GD, BETTY_OPT_MOMENTUM, BETTY_OPT_ADAM = range(3)
+BETTY_LR_CONSTANT, BETTY_LR_MULTISTEP, BETTY_LR_COSINE = range(3)
 
 
 class BettyError(RuntimeError):
@@ -47,6 +48,8 @@ _Level._fields_ = [
     ("momentum", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("adam_eps", C.c_float),
     ("weight_decay", C.c_float), ("opt_state", C.c_void_p), ("n_constraints", C.c_int32),
     ("constraints", C.POINTER(C.POINTER(_Level))),
+    ("lr_schedule", C.c_int32), ("lr_step0", C.c_int32), ("lr_t_max", C.c_int32), ("lr_milestones", C.c_int32 * 4),
+    ("lr_gamma", C.c_float), ("lr_min", C.c_float),
 ]
 
 class _Edge(C.Structure):
@@ -183,6 +186,18 @@ class Level:
         self.c.beta1, self.c.beta2, self.c.adam_eps = float(beta1), float(beta2), float(eps)
         self.c.weight_decay = float(weight_decay)
         self.c.opt_state = _ptr(self.opt_state)
+        return self
+
+    def set_lr_schedule(self, kind: int, step0: int = 0, milestones: Sequence[int] = (), gamma: float = 0.1,
+                        t_max: int = 1, lr_min: float = 0.0) -> "Level":
+        """Step size as a function of the steps taken (betty_lr_schedule); step0 = steps taken before the
+        next call."""
+        if len(milestones) > 4:
+            raise ValueError("at most 4 milestones")
+        self.c.lr_schedule, self.c.lr_step0, self.c.lr_t_max = int(kind), int(step0), int(t_max)
+        for i in range(4):
+            self.c.lr_milestones[i] = int(milestones[i]) if i < len(milestones) else 0
+        self.c.lr_gamma, self.c.lr_min = float(gamma), float(lr_min)
         return self
 
     @property

@@ -121,15 +121,16 @@ betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, 
   return vec_mul(c, out, 1.0f, L->params, q, L->d);
 }
 
-betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps) {
+betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step) {
   if (!vec_has_wd(L)) return BETTY_ERR_UNSUPPORTED;
   const float* lam = find_constraint(L, BETTY_PARAM_VECTOR)->params;
-  if (n_steps > 1 && logreg_small_eligible(L->n, 0, L->d))   // all steps in one launch, data resident on chip
+  // all steps in one launch, data resident on chip (one step size for the whole launch)
+  if (n_steps > 1 && L->lr_schedule == BETTY_LR_CONSTANT && logreg_small_eligible(L->n, 0, L->d))
     return logreg_small_lower_step(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, lam,
                                    n_steps, L->lr);
   for (int s = 0; s < n_steps; ++s)
     BETTY_TRY(logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, nullptr, lam,
-                          nullptr, L->params, L->lr));
+                          nullptr, L->params, lr_at(L, first_step + s)));
   return BETTY_OK;
 }
 
@@ -142,17 +143,18 @@ betty_status vecfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
 }
 
 // params of L <- one optimiser step along gradient g
-static betty_status apply_optimizer(Ctx& c, const betty_level* L, const float* g) {
+static betty_status apply_optimizer(Ctx& c, const betty_level* L, const float* g, int step_in_call) {
+  const float lr = lr_at(L, step_in_call);
   const int64_t n = L->n_params;
   if (n <= 0) return BETTY_OK;
   const int grid = (int)((n + 1023) / 1024 < 1 ? 1 : ((n + 1023) / 1024 > 2368 ? 2368 : (n + 1023) / 1024));
   if (L->optimizer == BETTY_OPT_GD) {
-    launch_pdl(k_opt_gd, dim3(grid), dim3(256), 0, c.stream, L->params, g, L->lr, n);
+    launch_pdl(k_opt_gd, dim3(grid), dim3(256), 0, c.stream, L->params, g, lr, n);
   } else if (L->optimizer == BETTY_OPT_MOMENTUM) {
-    launch_pdl(k_opt_momentum, dim3(grid), dim3(256), 0, c.stream, L->params, g, L->opt_state, L->lr, L->momentum, L->weight_decay, n);
+    launch_pdl(k_opt_momentum, dim3(grid), dim3(256), 0, c.stream, L->params, g, L->opt_state, lr, L->momentum, L->weight_decay, n);
   } else {
     float* m = L->opt_state; float* v = m + n; float* t = v + n;
-    launch_pdl(k_opt_adam, dim3(grid), dim3(256), 0, c.stream, L->params, g, m, v, t, L->lr, L->beta1, L->beta2, L->adam_eps, L->weight_decay, n);
+    launch_pdl(k_opt_adam, dim3(grid), dim3(256), 0, c.stream, L->params, g, m, v, t, lr, L->beta1, L->beta2, L->adam_eps, L->weight_decay, n);
     BETTY_LAUNCH_CHECK();
     launch_pdl(k_opt_tick, dim3(1), dim3(1), 0, c.stream, t);
   }
@@ -300,7 +302,7 @@ static betty_status hypergrad_itd(const betty_level* lower, const betty_level* u
   BETTY_ALLOC(m, float, c, (size_t)nc);
   for (int t = 0; t < n_steps; ++t) {
     BETTY_TRY(vec_copy(c, iter + stride * t, lower->params, n));
-    BETTY_TRY(vecfam ? vecfam_lower_step(c, lower, 1) : mlpfam_lower_step(c, lower, 1));
+    BETTY_TRY(vecfam ? vecfam_lower_step(c, lower, 1, t) : mlpfam_lower_step(c, lower, 1, t));
   }
   BETTY_TRY(level_grad(c, upper, lower, a));
   BETTY_TRY(level_grad(c, upper, wrt, out));
@@ -317,9 +319,10 @@ static betty_status hypergrad_itd(const betty_level* lower, const betty_level* u
       BETTY_TRY(mlpfam_mixed(c, &at, cache, wrt, a, m));
       BETTY_TRY(mlpfam_hvp(c, &at, cache, a, h));
     }
-    launch_pdl(k_scale_into, dim3(ew_grid(nc)), dim3(256), 0, c.stream, out, m, -lower->lr, 1, nc);
+    const float lr_t = lr_at(lower, t);     // the step size step t was taken with
+    launch_pdl(k_scale_into, dim3(ew_grid(nc)), dim3(256), 0, c.stream, out, m, -lr_t, 1, nc);
     BETTY_LAUNCH_CHECK();
-    BETTY_TRY(vec_axpby(c, a, 1.f, a, -lower->lr, h, n));
+    BETTY_TRY(vec_axpby(c, a, 1.f, a, -lr_t, h, n));
     c.arena.release(mark);
   }
   return BETTY_OK;
@@ -442,12 +445,12 @@ static betty_status engine_step(Engine& e, int j, int depth) {
   const bool fused = L->optimizer == BETTY_OPT_GD && !e.has_child[j] && (L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_QUADRATIC_WD ||
                                          L->loss == BETTY_LOSS_MLP_CE_REWEIGHT);
   if (fused) {
-    BETTY_TRY(is_vector_family(L->loss) ? vecfam_lower_step(*e.c, L, 1) : mlpfam_lower_step(*e.c, L, 1));
+    BETTY_TRY(is_vector_family(L->loss) ? vecfam_lower_step(*e.c, L, 1, e.count[j]) : mlpfam_lower_step(*e.c, L, 1, e.count[j]));
   } else {
     float* gvec = e.c->arena.alloc<float>((size_t)L->n_params);
     if (!gvec) return BETTY_ERR_WORKSPACE;
     BETTY_TRY(graph_hypergrad(*e.c, e.levels, *e.g, j, e.cfg, gvec));
-    BETTY_TRY(apply_optimizer(*e.c, L, gvec));
+    BETTY_TRY(apply_optimizer(*e.c, L, gvec, e.count[j]));
   }
   e.c->arena.release(mark);
   e.count[j] += 1;
@@ -612,7 +615,7 @@ betty_status betty_lower_step(const betty_level* L, int32_t n_steps, void* ws, s
     BETTY_ALLOC(g, float, c, (size_t)L->n_params);
     for (int s = 0; s < n_steps; ++s) {
       BETTY_TRY(level_grad(c, L, L, g));
-      BETTY_TRY(apply_optimizer(c, L, g));
+      BETTY_TRY(apply_optimizer(c, L, g, s));
     }
     return BETTY_OK;
   }

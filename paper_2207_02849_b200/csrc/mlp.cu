@@ -916,7 +916,7 @@ betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const be
   return BETTY_OK;
 }
 
-betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps) {
+betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step) {
   if (L->loss != BETTY_LOSS_MLP_CE_REWEIGHT) return BETTY_ERR_UNSUPPORTED;
   if (n_steps <= 0) return BETTY_OK;
   const size_t mark = c.arena.mark();
@@ -940,7 +940,7 @@ betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps) {
     BETTY_TRY(reweight_coef(c, P, ps, &coef));
     GradSink sink = {};
     sink.lam = P.lam ? P.lam->params : nullptr;
-    sink.sgd = true; sink.lr = L->lr; sink.master = L->params; sink.Wnext = alt;
+    sink.sgd = true; sink.lr = lr_at(L, first_step + s); sink.master = L->params; sink.Wnext = alt;
     BETTY_TRY(backward(c, n, ps, coef, sink));
     for (int l = 0; l < n.L; ++l) { bf16* t = n.W[l]; n.W[l] = alt[l]; alt[l] = t; }
     c.arena.release(m2);

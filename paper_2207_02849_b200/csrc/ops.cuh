@@ -1,6 +1,7 @@
 // Per-cost-family operations behind the C ABI.  Each function enqueues kernels on ctx.stream
 // and allocates its scratch from ctx.arena.
 #pragma once
+#include <math.h>
 #include "common.cuh"
 
 namespace betty {
@@ -39,12 +40,28 @@ betty_status vecfam_validate(const betty_level* L);
 betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);
 betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu);
 betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, const float* q, float* out);
-betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps);
+betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step = 0);
 // out (+)= -alpha*[dC/dc(x+eps v) - dC/dc(x-eps v)]/(2 eps), eps = eps0/sqrt(*vnorm2) on the device
 betty_status vecfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
                        float eps0, float alpha, float* out, bool accumulate);
 
 // ---- MLP families (mlp.cu) ----
+// Step size of problem L for its step number `step_in_call` of the present call (betty_lr_schedule)
+static inline float lr_at(const betty_level* L, int step_in_call) {
+  const long long t = (long long)L->lr_step0 + step_in_call;
+  if (L->lr_schedule == BETTY_LR_MULTISTEP) {
+    double lr = L->lr;
+    for (int i = 0; i < 4; ++i)
+      if (L->lr_milestones[i] > 0 && t >= L->lr_milestones[i]) lr *= (double)L->lr_gamma;
+    return (float)lr;
+  }
+  if (L->lr_schedule == BETTY_LR_COSINE && L->lr_t_max > 0) {
+    const double u = (double)(t < L->lr_t_max ? t : L->lr_t_max) / (double)L->lr_t_max;
+    return (float)((double)L->lr_min + ((double)L->lr - (double)L->lr_min) * 0.5 * (1.0 + cos(3.14159265358979323846 * u)));
+  }
+  return L->lr;
+}
+
 struct MlpHvpCache;  // base forward/backward state shared by the HVPs of one solve
 betty_status mlpfam_validate(const betty_level* L);
 size_t mlpfam_workspace(const betty_level* L);
@@ -60,7 +77,7 @@ betty_status mlpfam_hvp_series(Ctx& c, const betty_level* L, MlpHvpCache* cache,
                                float* s_out);
 betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* cache, const betty_level* wrt, const float* q,
                           float* out);
-betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps);
+betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step = 0);
 betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
                        float eps0, float alpha, float* out, bool accumulate);
 

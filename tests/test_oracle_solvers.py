@@ -324,3 +324,63 @@ def test_optimizer_steps_match_torch_optim(kind):
         opt.step()
     oracle.lower_step(lo, 6)
     assert rel(lo.params, w.detach().numpy()) < 1e-10
+
+
+# ------------------------------------------------------------------ step-size schedules
+@pytest.mark.parametrize("sched", ["multistep", "cosine"])
+def test_scheduled_steps_match_torch_lr_schedulers(sched):
+    """The step size as a function of the step count against torch.optim.lr_scheduler (MultiStepLR: decay
+    by a factor at given iterations; CosineAnnealingLR down to a minimum at T_max), value by value and
+    through a momentum-SGD trajectory on autodiff gradients of the same cost."""
+    from oracle.solvers import lr_at
+    inp = si.logreg_bilevel(31, 40, 5, 10)
+    inp.w0 = si.normal_f32(31, 9, (5,)) * 0.3
+    lo, up = logreg_levels(inp)
+    lo.optimizer, lo.lr, lo.momentum, lo.weight_decay = "momentum", 0.1, 0.9, 0.01
+    lo.lr_schedule = sched
+    lo.lr_milestones, lo.lr_gamma, lo.lr_t_max, lo.lr_min = (3, 7), 0.1, 10, 0.004
+    w = _t(inp.w0).requires_grad_(True)
+    opt = torch.optim.SGD([w], lr=0.1, momentum=0.9, weight_decay=0.01)
+    sch = (torch.optim.lr_scheduler.MultiStepLR(opt, milestones=[3, 7], gamma=0.1) if sched == "multistep"
+           else torch.optim.lr_scheduler.CosineAnnealingLR(opt, T_max=10, eta_min=0.004))
+    X, y, lam = _t(inp.X), _t(inp.y), _t(inp.lam)
+    for t in range(10):
+        assert abs(lr_at(lo, t) - opt.param_groups[0]["lr"]) < 1e-12 * 0.1 + 1e-15, t
+        opt.zero_grad()
+        c = torch.nn.functional.softplus(-y * (X @ w)).mean() + 0.5 * (lam * w * w).sum()
+        c.backward()
+        opt.step()
+        sch.step()
+    oracle.lower_step(lo, 10)
+    assert rel(lo.params, w.detach().numpy()) < 1e-10
+    # a second call continues on the schedule when the caller advances lr_step0
+    lo.lr_step0 = 10
+    assert abs(lr_at(lo, 0) - (0.1 * 0.01 if sched == "multistep" else 0.004)) < 1e-15
+    # beyond T_max the cosine schedule stays at its minimum; a constant schedule ignores every field
+    assert sched != "cosine" or lr_at(lo, 25) == 0.004
+    lo.lr_schedule = "constant"
+    assert lr_at(lo, 3) == 0.1
+
+
+def test_itd_with_a_schedule_matches_autodiff_through_the_unrolled_steps():
+    """ITD-RMAD with a different step size per unrolled step against reverse-mode autodiff (torch, fp64)
+    through the same steps."""
+    inp = si.logreg_bilevel(33, 30, 4, 12)
+    inp.w0 = si.normal_f32(33, 9, (4,)) * 0.2
+    inp.lam = (np.abs(si.normal_f32(33, 7, (4,))) * 0.1 + 0.05).astype(np.float32)
+    lo, up = logreg_levels(inp)
+    lamL = lo.constraints[0]
+    lo.lr, lo.lr_schedule, lo.lr_milestones, lo.lr_gamma = 0.5, "multistep", (2, 4), 0.5
+    X, y, Xv, yv = _t(inp.X), _t(inp.y), _t(inp.Xv), _t(inp.yv)
+    lam = _t(inp.lam).requires_grad_(True)
+    w = _t(inp.w0)
+    for t in range(5):
+        lr = 0.5 * 0.5 ** sum(1 for m in (2, 4) if t >= m)
+        wd = w.detach().requires_grad_(True) if t == 0 else w
+        c = torch.nn.functional.softplus(-y * (X @ wd)).mean() + 0.5 * (lam * wd * wd).sum()
+        (g,) = torch.autograd.grad(c, wd, create_graph=True)
+        w = wd - lr * g
+    cu = torch.nn.functional.softplus(-yv * (Xv @ w)).mean()
+    (ref,) = torch.autograd.grad(cu, lam)
+    out = oracle.hypergrad_itd(lo, up, lamL, 5)
+    assert rel(out, ref.numpy()) < 1e-9
