@@ -77,3 +77,41 @@ def test_three_level_mlp_run(bt):
     assert np.linalg.norm(O[2].params - inp.lam) > 1e-4   # the step is well above fp32 resolution of lambda
     assert cb.rel_l2(P[2].params - cb.dev(inp.lam), O[2].params - inp.lam.astype(np.float64)) < 5e-2
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+def test_two_upper_problems_share_one_lower_problem(bt):
+    """The extended bilevel structure of the paper's noisy-label program (Sec. 5.1: a reweighting and a
+    label-correcting problem above one classifier): two upper problems, each with an upper-to-lower edge
+    into the classifier and a lower-to-upper edge out of it.  Built from the cost families at hand: the
+    classifier's reweighted cross-entropy with per-layer decay, a weight net and a log-weight-decay vector
+    above it, each with the plain cross-entropy of the classifier on a batch of its own."""
+    from tests import cuda_build as cb
+    from tests.test_gpu_mlp import _three
+    inp = _three("gelu")
+    inp.lam = np.full(3, np.log(0.05), dtype=np.float32)
+    bf = torch.bfloat16
+    P1 = bt.Level(bt.LOSS_MLP_CE_REWEIGHT, bt.PARAM_MLP, cb.dev(inp.w), X=cb.dev(inp.D1.X, bf), y=cb.dev(inp.D1.y),
+                  widths=inp.widths, activation=bt.ACT_GELU, lr=0.1)
+    P2 = bt.Level(bt.LOSS_MLP_CE, bt.PARAM_WEIGHTNET, cb.dev(inp.theta), X=cb.dev(inp.D2.X, bf), y=cb.dev(inp.D2.y_clean), lr=0.05)
+    P3 = bt.Level(bt.LOSS_MLP_CE, bt.PARAM_LOGWD, cb.dev(inp.lam), X=cb.dev(inp.D3.X, bf), y=cb.dev(inp.D3.y_clean), lr=200.0)
+    P1.set_constraints([P2, P3]); P2.set_constraints([P1]); P3.set_constraints([P1])
+    O1 = oracle.Level(loss="mlp_ce_reweight", param_kind="mlp", params=inp.w, X=inp.D1.X, y=inp.D1.y, widths=inp.widths,
+                      activation="gelu", lr=0.1, bf16=True)
+    O2 = oracle.Level(loss="mlp_ce", param_kind="weightnet", params=inp.theta, X=inp.D2.X, y=inp.D2.y_clean, lr=0.05,
+                      constraints=[O1])
+    O3 = oracle.Level(loss="mlp_ce", param_kind="logwd", params=inp.lam, X=inp.D3.X, y=inp.D3.y_clean, lr=200.0,
+                      constraints=[O1])
+    O1.constraints = [O2, O3]
+    u2l, l2u = [(1, 0), (2, 0)], [(0, 1), (0, 2)]
+    # each upper parameter reaches the classifier's optimum along exactly one path
+    assert bt.betty_find_paths(3, u2l, l2u, 1, [0]) == oracle.find_paths(u2l, l2u, 1, [0]) == [[1, 0]]
+    assert bt.betty_find_paths(3, u2l, l2u, 2, [0]) == oracle.find_paths(u2l, l2u, 2, [0]) == [[2, 0]]
+    cfg, ocfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=3, alpha=0.01), dict(method="neumann", K=3, alpha=0.01)
+    ws = bt.Workspace([P1, P2, P3])
+    log = bt.betty_engine_run([P1, P2, P3], u2l, l2u, [cfg] * 3, [2, 1, 1], 4, ws)
+    assert log == oracle.engine_run([O1, O2, O3], u2l, l2u, [ocfg] * 3, [2, 1, 1], 4) == [0, 0, 1, 2, 0, 0, 1, 2]
+    assert cb.rel_l2(P1.params, O1.params) < 1e-3
+    assert cb.rel_l2(P2.params - cb.dev(inp.theta), O2.params - inp.theta.astype(np.float64)) < 3e-2
+    assert np.linalg.norm(O3.params - inp.lam) > 1e-4
+    assert cb.rel_l2(P3.params - cb.dev(inp.lam), O3.params - inp.lam.astype(np.float64)) < 5e-2
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
