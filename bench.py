@@ -614,7 +614,10 @@ def main():
         with open(tpath) as f:
             tj = json.load(f).get(probe["kernel"])
         if tj and tj.get("valid"):
-            traffic = tj["dram_bytes_per_unit"] * (probe["bytes"] / tj["unit_bytes"])
+            if "dram_bytes_per_launch" in tj:       # captured at the probe's own shape
+                traffic = float(tj["dram_bytes_per_launch"])
+            else:                                   # captured on a smaller case; grows with the units streamed
+                traffic = tj["dram_bytes_per_unit"] * (probe["bytes"] / tj["unit_bytes"])
     roofline = {"bound": probe["bound"], "kernel": probe["kernel"], "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": traffic, "peak_source": f"{peaks['source']} (burst; kernel timed alone)",
                 "kernel_ms": probe["ms"], "algorithmic_bytes_per_launch": probe.get("bytes"),
