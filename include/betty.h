@@ -156,6 +156,11 @@ typedef struct betty_level {
   int32_t lr_milestones[4]; /* MULTISTEP: step counts at which the step size drops; unused entries 0 */
   float lr_gamma;       /* MULTISTEP: factor per milestone passed */
   float lr_min;         /* COSINE: step size reached at lr_t_max */
+  int32_t grad_accum;   /* gradient accumulation (Sec. 4, systems support): a step of a problem without lower
+                         * problems takes its batch as grad_accum equal micro-batches of n / grad_accum rows, one
+                         * after the other, and averages their gradients before the optimiser step: the
+                         * activations of one micro-batch are alive at a time.  0 or 1: off.  n must be a
+                         * multiple of it (else BETTY_ERR_SHAPE).  Used by betty_lower_step and betty_engine_run. */
 } betty_level;
 
 /* Scratch bytes sufficient for any call below on these levels (Sec. 2: the whole program). */

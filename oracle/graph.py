@@ -7,7 +7,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from .solvers import apply_optimizer, chain_levels, grad
+from .solvers import apply_optimizer, chain_levels, grad, step_gradient
 
 
 def find_paths(u2l, l2u, k, targets):
@@ -54,7 +54,10 @@ def engine_run(levels, u2l, l2u, cfgs, unroll, n_iterations):
 
     def step(j):
         log.append(j)
-        g = hypergrad_graph(levels, u2l, l2u, j, cfgs)
+        if n_lower[j] == 0 and levels[j].grad_accum > 1:
+            g = step_gradient(levels[j])
+        else:
+            g = hypergrad_graph(levels, u2l, l2u, j, cfgs)
         apply_optimizer(levels[j], g, count[j])
         count[j] += 1
         if count[j] % unroll[j] == 0:

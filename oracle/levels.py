@@ -63,6 +63,7 @@ class Level:
     lr_gamma: float = 0.1
     lr_t_max: int = 1
     lr_min: float = 0.0
+    grad_accum: int = 1                # micro-batches whose gradients are averaged into one step (Sec. 4)
 
     def __post_init__(self):
         self.params = np.array(self.params, dtype=np.float64).reshape(-1)

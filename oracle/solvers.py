@@ -19,6 +19,8 @@ weights).  Readings where the paper is silent:
 """
 from __future__ import annotations
 
+import copy
+
 import numpy as np
 
 from . import levels as _lv
@@ -70,13 +72,34 @@ def apply_optimizer(L: Level, g: np.ndarray, step_in_call: int = 0) -> None:
         raise ValueError(L.optimizer)
 
 
+def step_gradient(L: Level) -> np.ndarray:
+    """Gradient that a step of a problem without lower problems follows.  With gradient accumulation (one
+    of the systems features Sec. 4 lists) the batch is taken as L.grad_accum equal micro-batches, one
+    after the other, and their gradients are averaged before the optimiser step."""
+    A = int(L.grad_accum)
+    if A <= 1:
+        return grad(L, L)
+    n = L.X.shape[0]
+    if n % A:
+        raise ValueError("batch size must be a multiple of grad_accum")
+    nb = n // A
+    total = 0.0
+    for a in range(A):
+        Ls = copy.copy(L)
+        Ls.X, Ls.y = L.X[a * nb:(a + 1) * nb], L.y[a * nb:(a + 1) * nb]
+        if L.aux is not None:
+            Ls.aux = L.aux[a * nb:(a + 1) * nb]
+        total = total + grad(Ls, Ls)
+    return total / A
+
+
 def lower_step(L: Level, n_steps: int) -> None:
     """x <- x - lr * dC/dx, n_steps times on the level's fixed batch (Sec. 3.2: w* is
     approximated by a small number of unrolled gradient steps).  Updates L.params in place.
     For mixed-precision levels the gradient is taken at the bf16-rounded copy of the
     current master, which is re-derived at every step."""
     for s in range(int(n_steps)):
-        apply_optimizer(L, grad(L, L), s)
+        apply_optimizer(L, step_gradient(L), s)
 
 
 def neumann_solve(hv, v, K: int, alpha: float) -> np.ndarray:

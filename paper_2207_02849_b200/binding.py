@@ -49,7 +49,7 @@ _Level._fields_ = [
     ("weight_decay", C.c_float), ("opt_state", C.c_void_p), ("n_constraints", C.c_int32),
     ("constraints", C.POINTER(C.POINTER(_Level))),
     ("lr_schedule", C.c_int32), ("lr_step0", C.c_int32), ("lr_t_max", C.c_int32), ("lr_milestones", C.c_int32 * 4),
-    ("lr_gamma", C.c_float), ("lr_min", C.c_float),
+    ("lr_gamma", C.c_float), ("lr_min", C.c_float), ("grad_accum", C.c_int32),
 ]
 
 class _Edge(C.Structure):
@@ -198,6 +198,11 @@ class Level:
         for i in range(4):
             self.c.lr_milestones[i] = int(milestones[i]) if i < len(milestones) else 0
         self.c.lr_gamma, self.c.lr_min = float(gamma), float(lr_min)
+        return self
+
+    def set_grad_accum(self, n_micro: int) -> "Level":
+        """Steps of this problem average the gradients of n_micro equal micro-batches of its batch."""
+        self.c.grad_accum = int(n_micro)
         return self
 
     @property

@@ -195,6 +195,30 @@ static betty_status level_grad(Ctx& c, const betty_level* L, const betty_level* 
   return mlpfam_grad(c, L, wrt, out);
 }
 
+// Gradient of a step of a problem without lower problems: dC_L/d(own), taken over the whole batch at once
+// or, with gradient accumulation, as the average over L->grad_accum equal micro-batches processed one
+// after the other (each micro-batch's activations are released before the next one starts).
+static betty_status step_grad(Ctx& c, const betty_level* L, float* out) {
+  const int A = L->grad_accum;
+  if (A <= 1) return level_grad(c, L, L, out);
+  if (L->n <= 0 || L->n % A != 0) return BETTY_ERR_SHAPE;
+  const int64_t nb = L->n / A;
+  const size_t xsz = L->x_dtype == BETTY_BF16 ? 2 : 4;
+  const size_t mark = c.arena.mark();
+  BETTY_ALLOC(ga, float, c, (size_t)L->n_params);
+  for (int a = 0; a < A; ++a) {
+    betty_level Ls = *L;                 // the same problem on rows a*nb .. (a+1)*nb - 1 of its batch
+    Ls.n = nb;
+    Ls.X = (const char*)L->X + (size_t)a * nb * L->d * xsz;
+    Ls.y = (const char*)L->y + (size_t)a * nb * 4;          // labels are fp32 or int32
+    if (L->aux) Ls.aux = L->aux + (size_t)a * nb;
+    BETTY_TRY(level_grad(c, &Ls, &Ls, ga));
+    BETTY_TRY(vec_axpby(c, out, 1.f / (float)A, ga, a > 0 ? 1.f : 0.f, a > 0 ? out : nullptr, L->n_params));
+  }
+  c.arena.release(mark);
+  return BETTY_OK;
+}
+
 // (d x*/d c)^T v by the configured approximation; out (+)= result.
 static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v,
                         const betty_method_cfg& cfg, float* out, bool accumulate) {
@@ -442,14 +466,15 @@ static betty_status engine_step(Engine& e, int j, int depth) {
   if (e.log && e.n_logged < e.log_capacity) e.log[e.n_logged] = j;
   e.n_logged += 1;
   const size_t mark = e.c->arena.mark();
-  const bool fused = L->optimizer == BETTY_OPT_GD && !e.has_child[j] && (L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_QUADRATIC_WD ||
+  const bool fused = L->optimizer == BETTY_OPT_GD && L->grad_accum <= 1 && !e.has_child[j] && (L->loss == BETTY_LOSS_LOGREG_WD || L->loss == BETTY_LOSS_QUADRATIC_WD ||
                                          L->loss == BETTY_LOSS_MLP_CE_REWEIGHT);
   if (fused) {
     BETTY_TRY(is_vector_family(L->loss) ? vecfam_lower_step(*e.c, L, 1, e.count[j]) : mlpfam_lower_step(*e.c, L, 1, e.count[j]));
   } else {
     float* gvec = e.c->arena.alloc<float>((size_t)L->n_params);
     if (!gvec) return BETTY_ERR_WORKSPACE;
-    BETTY_TRY(graph_hypergrad(*e.c, e.levels, *e.g, j, e.cfg, gvec));
+    if (e.n_lower[j] == 0 && L->grad_accum > 1) BETTY_TRY(step_grad(*e.c, L, gvec));
+    else BETTY_TRY(graph_hypergrad(*e.c, e.levels, *e.g, j, e.cfg, gvec));
     BETTY_TRY(apply_optimizer(*e.c, L, gvec, e.count[j]));
   }
   e.c->arena.release(mark);
@@ -611,10 +636,10 @@ betty_status betty_lower_step(const betty_level* L, int32_t n_steps, void* ws, s
   if (n_steps < 0) return BETTY_ERR_INVALID_ARG;
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
-  if (L->optimizer != BETTY_OPT_GD) {
+  if (L->optimizer != BETTY_OPT_GD || L->grad_accum > 1) {
     BETTY_ALLOC(g, float, c, (size_t)L->n_params);
     for (int s = 0; s < n_steps; ++s) {
-      BETTY_TRY(level_grad(c, L, L, g));
+      BETTY_TRY(step_grad(c, L, g));
       BETTY_TRY(apply_optimizer(c, L, g, s));
     }
     return BETTY_OK;

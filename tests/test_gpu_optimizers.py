@@ -156,3 +156,51 @@ def test_scheduled_run_through_the_execution_schedule(bt):
     assert cb.rel_l2(w.params, ow.params) < 1e-4
     assert cb.rel_l2(lam.params - cb.dev(inp.lam), olam.params - inp.lam.astype(np.float64)) < 1e-3
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+# ------------------------------------------------------------------ gradient accumulation
+@pytest.mark.parametrize("opt", ["gd", "momentum"])
+def test_accumulated_steps_mlp(bt, opt):
+    from tests import cuda_build as cb
+    from tests.test_gpu_mlp import _perturb
+    inp = _perturb(si.reweight_bilevel(95, (64, 96, 10), 128, 0.4, activation="gelu"), 95)
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    w.c.lr = ow.lr = 0.2
+    if opt == "momentum":
+        w.set_optimizer(bt.BETTY_OPT_MOMENTUM, momentum=0.9, weight_decay=5e-4)
+        ow.optimizer, ow.momentum, ow.weight_decay = "momentum", 0.9, 5e-4
+    w.set_grad_accum(4)
+    ow.grad_accum = 4
+    ws = bt.Workspace([w, th])
+    bt.betty_lower_step(w, 5, ws)
+    oracle.lower_step(ow, 5)
+    w0 = cb.dev(inp.w)
+    assert cb.rel_l2(w.params - w0, ow.params - inp.w.astype(np.float64)) < 2e-2
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+    w.set_grad_accum(3)                                    # 128 rows do not split into 3 equal micro-batches
+    with pytest.raises(bt.BettyError) as e:
+        bt.betty_lower_step(w, 1, ws)
+    assert e.value.status == bt.BETTY_ERR_SHAPE
+
+
+def test_accumulated_steps_logistic_and_schedule_run(bt):
+    from tests import cuda_build as cb
+    inp = si.logreg_bilevel(47, 512, 32, 64)
+    w, lam = cb.logreg_levels(inp)
+    ow, olam = ob.logreg_levels(inp)
+    w.c.lr = ow.lr = 0.5
+    w.set_grad_accum(4)
+    ow.grad_accum = 4
+    ws = bt.Workspace([w, lam])
+    bt.betty_lower_step(w, 6, ws)
+    oracle.lower_step(ow, 6)
+    assert cb.rel_l2(w.params, ow.params) < 1e-4
+    lam.c.lr = olam.lr = 0.2
+    u2l, l2u = [(1, 0)], [(0, 1)]
+    cfg, ocfg = bt.MethodCfg(bt.BETTY_CG, K=8), dict(method="cg", K=8, tol=0.0)
+    log = bt.betty_engine_run([w, lam], u2l, l2u, [cfg, cfg], [3, 1], 6, ws)
+    assert log == oracle.engine_run([ow, olam], u2l, l2u, [ocfg, ocfg], [3, 1], 6)
+    assert cb.rel_l2(w.params, ow.params) < 1e-4
+    assert cb.rel_l2(lam.params - cb.dev(inp.lam), olam.params - inp.lam.astype(np.float64)) < 1e-3
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK

@@ -384,3 +384,35 @@ def test_itd_with_a_schedule_matches_autodiff_through_the_unrolled_steps():
     (ref,) = torch.autograd.grad(cu, lam)
     out = oracle.hypergrad_itd(lo, up, lamL, 5)
     assert rel(out, ref.numpy()) < 1e-9
+
+
+# ------------------------------------------------------------------ gradient accumulation
+def test_accumulated_step_gradient_equals_full_batch_and_torch_accumulation():
+    """Averaging the gradients of equal micro-batches is the full-batch gradient of a mean cost; the step
+    it drives equals PyTorch's accumulation idiom (backward of cost/A per micro-batch, one optimiser step)."""
+    from oracle.solvers import step_gradient
+    inp = si.logreg_bilevel(35, 48, 5, 10)
+    inp.w0 = si.normal_f32(35, 9, (5,)) * 0.3
+    lo, up = logreg_levels(inp)
+    full = oracle.grad(lo, lo)
+    lo.grad_accum = 4
+    assert rel(step_gradient(lo), full) < 1e-13
+    lam = lo.constraints[0].params
+    # weight decay is part of every micro-batch's cost: counted once in the average, not A times
+    assert rel(step_gradient(lo) - lam * lo.params, full - lam * lo.params) < 1e-12
+    w = _t(inp.w0).requires_grad_(True)
+    opt = torch.optim.SGD([w], lr=0.1, momentum=0.9)
+    lo.optimizer, lo.momentum, lo.lr = "momentum", 0.9, 0.1
+    X, y, lamt = _t(inp.X), _t(inp.y), _t(inp.lam)
+    for _ in range(3):
+        opt.zero_grad()
+        for a in range(4):
+            Xa, ya = X[a * 12:(a + 1) * 12], y[a * 12:(a + 1) * 12]
+            c = torch.nn.functional.softplus(-ya * (Xa @ w)).mean() + 0.5 * (lamt * w * w).sum()
+            (c / 4).backward()
+        opt.step()
+    oracle.lower_step(lo, 3)
+    assert rel(lo.params, w.detach().numpy()) < 1e-10
+    lo.grad_accum = 5
+    with pytest.raises(ValueError):
+        step_gradient(lo)
