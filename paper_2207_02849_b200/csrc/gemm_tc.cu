@@ -22,7 +22,7 @@ static constexpr int TC_EPI_WARPS = 8;      // two warps per accumulator lane qu
 template <int BN> struct TcCfg {
   static constexpr int B_BYTES = BN * TC_BK * 2;
   static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
-  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);     // 192 KB of stages in every case
   static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
   static constexpr int TMEM_COLS = 2 * BN;  // two accumulators: the epilogue of one tile overlaps the next tile's MMAs
 };
@@ -884,6 +884,10 @@ betty_status gemm_tc(Ctx& c, const GemmDesc& g0, bool tr) {
   // wide tiles unless the problem is narrow or would leave most SMs without a tile
   const int tiles256 = ((g.N + 255) / 256) * ((g.M + TC_BM - 1) / TC_BM);
   if (g.N > 128 && tiles256 >= 96) return launch_tc<256>(c, g0, tr);
+  // 128-wide tiles would fill under half of the SMs: halve the tile width again (twice the CTAs, each
+  // staging and reading a quarter less per k-slab)
+  const int tiles128 = ((g.N + 127) / 128) * ((g.M + TC_BM - 1) / TC_BM);
+  if (g.N > 64 && tiles128 * 2 <= c.sm_count) return launch_tc<64>(c, g0, tr);
   return launch_tc<128>(c, g0, tr);
 }
 
