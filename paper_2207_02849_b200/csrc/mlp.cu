@@ -81,43 +81,43 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
     delta[i] = __float2bfloat16_rn(v);
   }
 }
-// Column sums sum_i d[i, n] (bias gradients), with the consumer fused in.  Block = 32 columns x 8 row
-// groups; fixed summation order.
+// Column sums sum_i d[i, n] (bias gradients), with the consumer fused in.  Block = 32 columns (16 lanes x 2
+// adjacent columns; ld is even, so a column pair is one 4-byte load) x 64 row groups; a thread's loads are
+// issued 16 at a time (the kernel is bound by latency, not by bytes); fixed summation order.
 //   mode 0: out[n] = sum            mode 1: out[n] -= step * sum   (gradient step on a bias)
 //   mode 2: out[n] = s_in[n] + t_in[n] - step * sum   (one Horner step of the Neumann series; out may alias t_in)
 struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; };
+static constexpr int CS_COLS = 32, CS_GROUPS = 64;
 __global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
   pdl_enter();
-  // 1024 threads: 32 lanes x 2 adjacent columns, 32 row groups; ld is even, so a column pair is one 4-byte load.
-  // A thread's loads are issued 16 at a time (the kernel is bound by latency, not by bytes).
-  __shared__ float sh[32][65];
-  const int cx = threadIdx.x & 31, rg = threadIdx.x >> 5;
-  const int64_t n = blockIdx.x * 64 + 2 * cx;
+  __shared__ float sh[CS_GROUPS][CS_COLS + 1];
+  const int cx = threadIdx.x & 15, rg = threadIdx.x >> 4;
+  const int64_t n = blockIdx.x * CS_COLS + 2 * cx;
   float a0 = 0.f, a1 = 0.f;
   if (n < N) {
     constexpr int U = 16;
-    for (int64_t i0 = rg; i0 < B; i0 += 32 * U) {
+    for (int64_t i0 = rg; i0 < B; i0 += CS_GROUPS * U) {
       __nv_bfloat162 v[U];
 #pragma unroll
-      for (int k = 0; k < U; ++k) {
-        const int64_t i = i0 + 32 * k;
-        v[k] = i < B ? *(const __nv_bfloat162*)(d + i * ld + n) : __floats2bfloat162_rn(0.f, 0.f);
+      for (int k2 = 0; k2 < U; ++k2) {
+        const int64_t i = i0 + CS_GROUPS * k2;
+        v[k2] = i < B ? *(const __nv_bfloat162*)(d + i * ld + n) : __floats2bfloat162_rn(0.f, 0.f);
       }
 #pragma unroll
-      for (int k = 0; k < U; ++k) {   // same order as a plain loop over the rows
-        const float2 f = __bfloat1622float2(v[k]);
+      for (int k2 = 0; k2 < U; ++k2) {   // same order as a plain loop over the rows
+        const float2 f = __bfloat1622float2(v[k2]);
         a0 += f.x; a1 += f.y;
       }
     }
   }
   sh[rg][2 * cx] = a0; sh[rg][2 * cx + 1] = a1;
   __syncthreads();
-  if (threadIdx.x < 64) {
-    const int64_t nn = blockIdx.x * 64 + threadIdx.x;
+  if (threadIdx.x < CS_COLS) {
+    const int64_t nn = blockIdx.x * CS_COLS + threadIdx.x;
     if (nn < N) {
       float t = 0.f;
 #pragma unroll
-      for (int r = 0; r < 32; ++r) t += sh[r][threadIdx.x];
+      for (int r = 0; r < CS_GROUPS; ++r) t += sh[r][threadIdx.x];
       if (k.mode == 0) k.out[nn] = t;
       else if (k.mode == 1) k.out[nn] -= k.step * t;
       else k.out[nn] = k.s_in[nn] + (k.t_in[nn] - k.step * t);
@@ -557,7 +557,7 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
         launch_pdl(k_wd_add_bf16, dim3(grid_for(N * K)), dim3(256), 0, c.stream, sink.gflat + n.woff[l], n.W[l], N, K, n.ldw[l], sink.lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      launch_pdl(k_colsum_bf16, dim3((unsigned)((N + 63) / 64)), dim3(1024), 0, c.stream, ps.delta[l], B, N, ldd, cs);
+      launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, ps.delta[l], B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {
@@ -848,7 +848,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
         launch_pdl(k_wd_add_f32, dim3(grid_for(N * K)), dim3(256), 0, c.stream, Hu + n.woff[l], u + n.woff[l], N * K, h->lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      launch_pdl(k_colsum_bf16, dim3((unsigned)((N + 63) / 64)), dim3(1024), 0, c.stream, Rd, B, N, ldd, cs);
+      launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, Rd, B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) Rd = Rdp;
