@@ -206,7 +206,8 @@ __global__ void k_wd_add_f32(float* out, const float* u, int64_t n, const float*
     out[i] += k * u[i];
 }
 // out (+)= scale * exp(lam) * <W, q>  (q == nullptr: <W, W>).  Each block sums a slice in fp64; the block
-// that draws the last ticket adds the per-block sums in block order (fixed summation order).
+// that draws the last ticket adds the per-block sums in a fixed order (one warp: strided partial sums, then a
+// shuffle tree), so the result does not depend on scheduling.
 static constexpr int LD_MAX_BLOCKS = 128;
 __global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
                             float scale, float* out, int accumulate, double* partial, unsigned* counter) {
@@ -229,10 +230,15 @@ __global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t l
     partial[blockIdx.x] = t;
     __threadfence();
     is_last = atomicAdd(counter, 1u) == gridDim.x - 1;
-    if (is_last) {
-      __threadfence();
-      double tot = 0.0;
-      for (unsigned bb = 0; bb < gridDim.x; ++bb) tot += ((volatile double*)partial)[bb];
+  }
+  __syncthreads();
+  if (is_last && threadIdx.x < 32) {
+    // second phase by one warp: lane l adds blocks l, l+32, ... in order, then a fixed shuffle tree
+    __threadfence();
+    double tot = 0.0;
+    for (unsigned bb = threadIdx.x; bb < gridDim.x; bb += 32) tot += ((volatile double*)partial)[bb];
+    for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+    if (threadIdx.x == 0) {
       const float v = scale * expf(*lam) * (float)tot;
       *out = (accumulate ? *out : 0.f) + v;
       *counter = 0u;
@@ -686,7 +692,9 @@ static betty_status wn_sample(Ctx& c, int mode, const betty_level* theta, const 
 static betty_status wn_backward(Ctx& c, const betty_level* theta, const float* dir, const Pass& ps, const float* cA,
                                 const float* cB, float mu, const float* muvec, float* out, bool accumulate = false,
                                 float out_scale = 1.f) {
-  int nb = (int)((ps.B + 15) / 16);
+  // 64 samples per block: the block that comes last reads every block's 301 partial sums, so few blocks
+  // keep that second phase short (batch 1024: 16 blocks)
+  int nb = (int)((ps.B + 63) / 64);
   nb = nb < 1 ? 1 : (nb > WN_MAX_BLOCKS ? WN_MAX_BLOCKS : nb);
   const size_t mark = c.arena.mark();
   BETTY_ALLOC(partial, double, c, (size_t)nb * WN_STRIDE);
