@@ -89,6 +89,23 @@ def test_reweight_hypergradients_match_oracle(bt, act):
         assert st == bt.BETTY_ERR_BREAKDOWN
 
 
+@pytest.mark.parametrize("K", [0, 1, 2])
+@pytest.mark.parametrize("B", [8, 128])
+def test_short_series_and_tiny_batches(bt, K, B):
+    """Degenerate ends of the series solve: no term beyond v (K = 0), a single Horner step whose epilogue
+    also feeds the mixed product (K = 1), two steps (the second reads the first one's bf16 copy); on a batch
+    of eight rows and on a regular one.  A larger alpha than the configurations' makes the terms differ."""
+    from tests import cuda_build as cb
+    inp = _perturb(si.reweight_bilevel(49, (64, 96, 10), B, 0.4, activation="gelu"), 49)
+    w, th = cb.reweight_levels(inp)
+    ow, oth = ob.reweight_levels(inp)
+    ws = bt.Workspace([w, th])
+    out = _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_hypergrad_neumann(w, th, th, K, 0.5, out, ws)
+    assert cb.rel_l2(out, oracle.hypergrad_neumann(ow, oth, oth, K, 0.5)) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
 def _three(act="relu", widths=(32, 48, 40, 10), B=96, seed=53):
     inp = si.three_level(seed, widths, B, 0.3, activation=act)
     inp.w = inp.w + si.to_bf16_values(si.normal_f32(seed, 300, inp.w.shape) * np.float32(0.02))
