@@ -110,10 +110,13 @@ betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
   return vec_zero(c, out, wrt->n_params);
 }
 
-betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu) {
+betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu, VecHvpCache* cache) {
   if (!vec_has_wd(L)) return BETTY_ERR_UNSUPPORTED;
-  return logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, u,
-                     find_constraint(L, BETTY_PARAM_VECTOR)->params, Hu, nullptr, 0.f);
+  const betty_status s = logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, u,
+                                     find_constraint(L, BETTY_PARAM_VECTOR)->params, Hu, nullptr, 0.f,
+                                     cache ? cache->curv : nullptr, cache ? cache->valid : false);
+  if (cache && cache->curv && s == BETTY_OK) cache->valid = true;
+  return s;
 }
 
 betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, const float* q, float* out) {
@@ -241,6 +244,10 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
   if (cfg.K < 0) return BETTY_ERR_INVALID_ARG;
   MlpHvpCache* cache = nullptr;
   if (!vecfam) BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
+  // logistic levels: the per-row curvature at the (fixed) lower parameters is shared by the solve's HVPs
+  VecHvpCache vcache = {nullptr, false};
+  if (vecfam && L->n > 0 && cfg.K > 1) vcache.curv = c.arena.alloc<float>((size_t)L->n);
+  if (c.arena.overflow) { c.arena.overflow = false; vcache.curv = nullptr; }
   BETTY_ALLOC(q, float, c, (size_t)n);
   BETTY_ALLOC(h, float, c, (size_t)n);
   BETTY_ALLOC(m, float, c, (size_t)nc);
@@ -253,7 +260,7 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
       for (int k = 0; k < cfg.K; ++k) {
         const float* t_in = k == 0 ? v : t;
         const float* s_in = k == 0 ? v : q;
-        BETTY_TRY(vecfam_hvp(c, L, t_in, h));
+        BETTY_TRY(vecfam_hvp(c, L, t_in, h, &vcache));
         BETTY_TRY(neumann_update(c, t_in, s_in, h, cfg.alpha, t, q, n));
       }
     } else {
@@ -268,7 +275,7 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
     BETTY_ALLOC(p, float, c, (size_t)n);
     BETTY_TRY(cg_init(c, st, v, q, r, p, cfg.tol, n, partials));
     for (int k = 0; k < cfg.K; ++k) {
-      BETTY_TRY(vecfam ? vecfam_hvp(c, L, p, h) : mlpfam_hvp(c, L, cache, p, h));
+      BETTY_TRY(vecfam ? vecfam_hvp(c, L, p, h, &vcache) : mlpfam_hvp(c, L, cache, p, h));
       BETTY_TRY(cg_step(c, st, q, r, p, h, n, partials));
     }
   }
@@ -601,7 +608,8 @@ betty_status betty_workspace_size(const betty_level* const* levels, int32_t n_le
     if (is_vector_family(L->loss)) {
       // per-CTA column partials of the streaming pass (2 CTAs per SM) or the fallback's row scratch
       size_t d = (size_t)(L->d > 0 ? L->d : 1), n = (size_t)(L->n > 0 ? L->n : 1);
-      size_t need = (2 * 148 + 64) * d * sizeof(float) + n * sizeof(float) + 4096;
+      // (+ n floats: the per-row curvature shared by the HVPs of one solve)
+      size_t need = (2 * 148 + 64) * d * sizeof(float) + 2 * n * sizeof(float) + 8192;
       if (need > total) total = need + (1 << 20);
     } else if (is_mlp_family(L->loss)) {
       total += mlpfam_workspace(L);

@@ -21,6 +21,8 @@ struct LrArgs {
   const float* X; const float* y; int64_t n; int64_t d;
   const float* w; const float* u;
   float* partials;       // [gridDim.x][d]
+  float* curv;           // [n] per-row curvature s_i = sigmoid(z_i) sigmoid(-z_i) / n at w: written by an HVP pass
+                         // of form LR_HVP (if non-null), read by one of form LR_HVP_CACHED
   int family;            // 0 logistic, 1 least squares
   float inv_n;
   StatusBlock* sb;
@@ -57,19 +59,26 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
 
 __device__ __forceinline__ float sigmoidf_(float t) { return 1.f / (1.f + __expf(-t)); }
 
+// Forms of the pass.  During one inverse-Hessian solve w does not move, so z = X w and with it the per-row
+// curvature are the same in every HVP: the first HVP of a solve leaves the curvature in `curv`, the others read
+// it and take one dot product per row instead of two (the cost of a gradient pass).
+enum { LR_GRAD = 0, LR_HVP = 1, LR_HVP_CACHED = 2 };
+
 // coefficient multiplying row i in the accumulation
 template <bool HVP>
 __device__ __forceinline__ float row_coef(int family, float z, float t, float y, float inv_n) {
   if (family == 0) {
-    if (HVP) { float s = sigmoidf_(z); return s * (1.f - s) * t * inv_n; }
+    if (HVP) { float s = sigmoidf_(z); return (s * (1.f - s) * inv_n) * t; }     // curvature first: see LR_HVP_CACHED
     return -y * sigmoidf_(-y * z) * inv_n;
   }
   return HVP ? t : (z - y);
 }
 
 // NCH: float4 column chunks per thread (d <= 1024*NCH, d % 4 == 0)
-template <int NCH, bool HVP>
+template <int NCH, int FORM>
 __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
+  constexpr bool HVP = FORM != LR_GRAD;            // a direction u is read
+  constexpr bool NEEDZ = FORM != LR_HVP_CACHED;    // z = x . w is formed
   extern __shared__ __align__(128) unsigned char smem[];
   const int64_t d = a.d;
   const int d4 = (int)(d >> 2);
@@ -83,7 +92,7 @@ __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
 #pragma unroll
   for (int k = 0; k < NCH; ++k) {
     int c4 = tid + k * LR_THREADS;
-    wv[k] = (c4 < d4) ? __ldg((const float4*)a.w + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    wv[k] = (NEEDZ && c4 < d4) ? __ldg((const float4*)a.w + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
     uv[k] = (HVP && c4 < d4) ? __ldg((const float4*)a.u + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
     acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
@@ -130,7 +139,7 @@ __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (c4 < d4 && r < rows) v = tile4[(size_t)r * d4 + c4];
         x[r][k] = v;
-        pz[r] += v.x * wv[k].x + v.y * wv[k].y + v.z * wv[k].z + v.w * wv[k].w;
+        if (NEEDZ) pz[r] += v.x * wv[k].x + v.y * wv[k].y + v.z * wv[k].z + v.w * wv[k].w;
         if (HVP) pt[r] += v.x * uv[k].x + v.y * uv[k].y + v.z * uv[k].z + v.w * uv[k].w;
       }
     }
@@ -138,7 +147,7 @@ __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
     for (int r = 0; r < LR_R; ++r) {
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
-        pz[r] += __shfl_xor_sync(0xffffffffu, pz[r], o);
+        if (NEEDZ) pz[r] += __shfl_xor_sync(0xffffffffu, pz[r], o);
         if (HVP) pt[r] += __shfl_xor_sync(0xffffffffu, pt[r], o);
       }
     }
@@ -163,7 +172,17 @@ __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
 #pragma unroll
       for (int wi = 0; wi < LR_WARPS; ++wi) { z += rb[wi * 2 * LR_R + 2 * r]; tt += rb[wi * 2 * LR_R + 2 * r + 1]; }
       float c = 0.f;
-      if (r < rows) c = row_coef<HVP>(a.family, z, tt, a.family == 0 && HVP ? 0.f : __ldg(a.y + t * LR_R + r), a.inv_n);
+      if (r < rows) {
+        if (FORM == LR_HVP_CACHED) {
+          c = (a.family == 0 ? __ldg(a.curv + t * LR_R + r) : 1.f) * tt;
+        } else {
+          c = row_coef<HVP>(a.family, z, tt, a.family == 0 && HVP ? 0.f : __ldg(a.y + t * LR_R + r), a.inv_n);
+          if (FORM == LR_HVP && a.curv && a.family == 0 && tid == r) {
+            const float sg = sigmoidf_(z);
+            a.curv[t * LR_R + r] = sg * (1.f - sg) * a.inv_n;
+          }
+        }
+      }
 #pragma unroll
       for (int k = 0; k < NCH; ++k) {
         acc[k].x += c * x[r][k].x; acc[k].y += c * x[r][k].y; acc[k].z += c * x[r][k].z; acc[k].w += c * x[r][k].w;
@@ -247,10 +266,10 @@ __global__ void k_logreg_finalize(const float* partials, int nparts, int64_t d, 
   }
 }
 
-template <int NCH, bool HVP>
+template <int NCH, int FORM>
 static betty_status launch_stream(Ctx& c, const LrArgs& a, int grid) {
   size_t smem = (size_t)LR_S * LR_R * a.d * sizeof(float) + LR_S * sizeof(uint64_t) + 2 * LR_WARPS * 2 * LR_R * sizeof(float);
-  auto kern = k_logreg_stream<NCH, HVP>;
+  auto kern = k_logreg_stream<NCH, FORM>;
   static size_t attr_bytes = 0;     // raise the dynamic shared memory limit once per instantiation (and again if it grows)
   if (smem > attr_bytes) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BETTY_ERR_CUDA;
@@ -265,12 +284,14 @@ static betty_status launch_stream(Ctx& c, const LrArgs& a, int grid) {
 // (gradient) or lam.*u (HVP).  out (nullable) receives the vector; w_update (nullable) is
 // decremented by lr times it.
 betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
-                         const float* u, const float* lam, float* out, float* w_update, float lr) {
+                         const float* u, const float* lam, float* out, float* w_update, float lr, float* curv,
+                         bool curv_valid) {
   if (d <= 0) return BETTY_OK;
   LrArgs a;
   a.X = X; a.y = y; a.n = n; a.d = d; a.w = w; a.u = u; a.family = family;
   a.inv_n = n > 0 ? 1.0f / (float)n : 0.f;
   a.sb = c.arena.status();
+  a.curv = u ? curv : nullptr;
   const size_t mark = c.arena.mark();
   int nparts;
   const bool fast = (d % 4 == 0) && d <= 4096 && aligned16(X) && aligned16(w) && (!u || aligned16(u));
@@ -282,10 +303,10 @@ betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int
     BETTY_ALLOC(partials, float, c, (size_t)grid * d);
     a.partials = partials;
     betty_status s;
-    const bool hv = u != nullptr;
-    if (d <= 1024) s = hv ? launch_stream<1, true>(c, a, grid) : launch_stream<1, false>(c, a, grid);
-    else if (d <= 2048) s = hv ? launch_stream<2, true>(c, a, grid) : launch_stream<2, false>(c, a, grid);
-    else s = hv ? launch_stream<4, true>(c, a, grid) : launch_stream<4, false>(c, a, grid);
+    const int form = !u ? LR_GRAD : (a.curv && curv_valid) ? LR_HVP_CACHED : LR_HVP;
+    if (d <= 1024) s = form == LR_GRAD ? launch_stream<1, LR_GRAD>(c, a, grid) : form == LR_HVP ? launch_stream<1, LR_HVP>(c, a, grid) : launch_stream<1, LR_HVP_CACHED>(c, a, grid);
+    else if (d <= 2048) s = form == LR_GRAD ? launch_stream<2, LR_GRAD>(c, a, grid) : form == LR_HVP ? launch_stream<2, LR_HVP>(c, a, grid) : launch_stream<2, LR_HVP_CACHED>(c, a, grid);
+    else s = form == LR_GRAD ? launch_stream<4, LR_GRAD>(c, a, grid) : form == LR_HVP ? launch_stream<4, LR_HVP>(c, a, grid) : launch_stream<4, LR_HVP_CACHED>(c, a, grid);
     BETTY_TRY(s);
   } else {
     int64_t want = (n + 255) / 256; if (want < 1) want = 1; if (want > 64) want = 64;
@@ -382,9 +403,10 @@ extern "C" betty_status betty_hvp_logreg_static(const float* X, int64_t n, int64
   int grid = NOALLOC_MAX_CTAS;
   if (ntiles < grid) grid = ntiles > 0 ? (int)ntiles : 1;
   betty_status st;
-  if (d <= 1024) st = launch_stream<1, true>(c, a, grid);
-  else if (d <= 2048) st = launch_stream<2, true>(c, a, grid);
-  else st = launch_stream<4, true>(c, a, grid);
+  a.curv = nullptr;
+  if (d <= 1024) st = launch_stream<1, LR_HVP>(c, a, grid);
+  else if (d <= 2048) st = launch_stream<2, LR_HVP>(c, a, grid);
+  else st = launch_stream<4, LR_HVP>(c, a, grid);
   if (st != BETTY_OK) return st;
   k_logreg_finalize<<<(unsigned)((d + 31) / 32), 256, 0, s>>>(a.partials, grid, d, lam, u, Hu, nullptr, 0.f);
   BETTY_LAUNCH_CHECK();

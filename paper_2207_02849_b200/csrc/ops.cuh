@@ -25,7 +25,8 @@ static inline bool is_mlp_family(int loss) {
 
 // logreg.cu
 betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
-                         const float* u, const float* lam, float* out, float* w_update, float lr);
+                         const float* u, const float* lam, float* out, float* w_update, float lr, float* curv = nullptr,
+                         bool curv_valid = false);
 
 // logreg_small.cu: whole-loop kernels for problems that fit a cluster's shared memory
 bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d);
@@ -38,7 +39,10 @@ betty_status logreg_small_hypergrad(Ctx& c, int family, const float* X, const fl
 // ---- vector families (api.cu) ----
 betty_status vecfam_validate(const betty_level* L);
 betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);
-betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu);
+// Per-row curvature of a logistic level at its present parameters, shared by the HVPs of one solve: the first
+// HVP fills it, the later ones read it (n floats in the caller's workspace; null: every HVP recomputes z = X w).
+struct VecHvpCache { float* curv; bool valid; };
+betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu, VecHvpCache* cache = nullptr);
 betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, const float* q, float* out);
 betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step = 0);
 // out (+)= -alpha*[dC/dc(x+eps v) - dC/dc(x-eps v)]/(2 eps), eps = eps0/sqrt(*vnorm2) on the device
