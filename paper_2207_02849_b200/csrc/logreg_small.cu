@@ -28,6 +28,7 @@ struct SmallArgs {
   int method, K; float alpha, eps0, tol;            // betty_method and its parameters
   float* out;                                       // hypergradient [d] (added to nothing: direct gradient is zero)
   int rows_per_cta, rows_per_cta_v;
+  int in_regs;                                      // rows live in registers (see pass_reg); else in shared memory
   StatusBlock* sb;
 };
 
@@ -122,6 +123,54 @@ __device__ void pass(const float* Xs, const float* ys, const float* curv, int ro
   (void)rank;
 }
 
+// The same pass with the CTA's rows held in registers for the whole launch: d / 8 adjacent threads own one
+// row, eight columns each (d a power of two between 8 and 256, at most SM_T / (d / 8) rows per CTA: the
+// 1024 x 64 problem gives every CTA 128 rows of 8 threads).  A pass is then 8 multiply-adds, a shuffle
+// reduction over the row's threads, the coefficient, 8 more multiply-adds and a shuffle reduction over the
+// warp's rows; shared memory is touched only for the 32 per-warp column sums.  (The shared-memory pass above
+// spends ~3400 clocks per 128 rows on its two sweeps over X.)
+//   x8: this thread's eight columns of its row; yv: the row's label (kind 0) or curvature (kind 1); has: row exists
+__device__ void pass_reg(const float (&x8)[8], float yv, bool has, int d, int family, float inv_n, int kind,
+                         const float* vv, float* part, float* cpart, float* res, uint32_t rank) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tpr = d >> 3, c8 = tid & (tpr - 1);
+  const float4 v0 = *(const float4*)(vv + 8 * c8), v1 = *(const float4*)(vv + 8 * c8 + 4);
+  float sdot = x8[0] * v0.x + x8[1] * v0.y + x8[2] * v0.z + x8[3] * v0.w + x8[4] * v1.x + x8[5] * v1.y + x8[6] * v1.z + x8[7] * v1.w;
+  for (int o = tpr >> 1; o > 0; o >>= 1) sdot += __shfl_xor_sync(0xffffffffu, sdot, o);
+  float cf = 0.f;
+  if (has) {
+    if (kind == 0) cf = family == 0 ? -yv * sigm(-yv * sdot) * inv_n : (sdot - yv);
+    else cf = yv * sdot;
+  }
+  float col[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) col[k] = cf * x8[k];
+  for (int o = tpr; o < 32; o <<= 1) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) col[k] += __shfl_xor_sync(0xffffffffu, col[k], o);
+  }
+  if (lane < tpr) {
+    *(float4*)(part + warp * SM_MAXD + 8 * c8) = make_float4(col[0], col[1], col[2], col[3]);
+    *(float4*)(part + warp * SM_MAXD + 8 * c8 + 4) = make_float4(col[4], col[5], col[6], col[7]);
+  }
+  __syncthreads();
+  for (int j = tid; j < d; j += SM_T) {
+    float acc = 0.f;
+#pragma unroll
+    for (int w2 = 0; w2 < SM_T / 32; ++w2) acc += part[w2 * SM_MAXD + j];
+#pragma unroll
+    for (uint32_t r = 0; r < SM_CL; ++r) st_remote(cpart + rank * SM_MAXD + j, r, acc);
+  }
+  cluster_barrier();                       // all pushes have landed everywhere
+  for (int j = tid; j < d; j += SM_T) {
+    float acc = 0.f;
+#pragma unroll
+    for (int r = 0; r < SM_CL; ++r) acc += cpart[r * SM_MAXD + j];
+    res[j] = acc;
+  }
+  __syncthreads();
+}
+
 __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logreg_small(SmallArgs a) {
   extern __shared__ __align__(16) float sm[];
   uint32_t rank;
@@ -134,7 +183,8 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   float* yvs = ys + R;                             // [Rv]
   float* curv = yvs + Rv;                          // [R]  sigmoid(z) sigmoid(-z) / n at the current w
   float* coef = curv + R;                          // [max(R, Rv)]
-  float* vec = coef + (R > Rv ? R : Rv);           // SM_NVEC vectors of SM_MAXD
+  float* vec = coef + (R > Rv ? R : Rv);           // SM_NVEC vectors of SM_MAXD, 16-byte aligned for float4 access
+  vec += (4 - ((vec - sm) & 3)) & 3;
   float* part = vec + SM_NVEC * SM_MAXD;           // [32][SM_MAXD] row-group partials
   float* cpart = part + 32 * SM_MAXD;              // [2][SM_CL][SM_MAXD] column sums of every CTA (double-buffered)
   float* red = cpart + 2 * SM_CL * SM_MAXD;                // [32] block reduction scratch
@@ -145,21 +195,54 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   const int64_t r0 = (int64_t)rank * R, r0v = (int64_t)rank * Rv;
   int rows = (int)(a.n - r0 < R ? a.n - r0 : R); if (rows < 0) rows = 0;
   int rowsv = (int)(a.nv - r0v < Rv ? a.nv - r0v : Rv); if (rowsv < 0) rowsv = 0;
-  for (int64_t i = tid; i < (int64_t)rows * d; i += SM_T) Xs[i] = a.X[r0 * d + i];
-  for (int i = tid; i < rows; i += SM_T) ys[i] = a.y[r0 + i];
-  if (a.mode == 1) {
-    for (int64_t i = tid; i < (int64_t)rowsv * d; i += SM_T) Xvs[i] = a.Xv[r0v * d + i];
-    for (int i = tid; i < rowsv; i += SM_T) yvs[i] = a.yv[r0v + i];
+  // register form: thread tid owns columns [8 c8, 8 c8 + 8) of row tid / (d / 8) of each matrix
+  const bool regs = a.in_regs != 0;
+  float x8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, xv8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float yreg = 0.f, yvreg = 0.f, curvreg = 0.f;
+  bool has = false, hasv = false;
+  if (regs) {
+    const int tpr = d >> 3, row = tid / tpr, c8 = tid & (tpr - 1);
+    has = row < rows; hasv = a.mode == 1 && row < rowsv;
+    if (has) {
+      const float4 lo = *(const float4*)(a.X + (r0 + row) * d + 8 * c8), hi = *(const float4*)(a.X + (r0 + row) * d + 8 * c8 + 4);
+      x8[0] = lo.x; x8[1] = lo.y; x8[2] = lo.z; x8[3] = lo.w; x8[4] = hi.x; x8[5] = hi.y; x8[6] = hi.z; x8[7] = hi.w;
+      yreg = a.y[r0 + row];
+    }
+    if (hasv) {
+      const float4 lo = *(const float4*)(a.Xv + (r0v + row) * d + 8 * c8), hi = *(const float4*)(a.Xv + (r0v + row) * d + 8 * c8 + 4);
+      xv8[0] = lo.x; xv8[1] = lo.y; xv8[2] = lo.z; xv8[3] = lo.w; xv8[4] = hi.x; xv8[5] = hi.y; xv8[6] = hi.z; xv8[7] = hi.w;
+      yvreg = a.yv[r0v + row];
+    }
+  } else {
+    for (int64_t i = tid; i < (int64_t)rows * d; i += SM_T) Xs[i] = a.X[r0 * d + i];
+    for (int i = tid; i < rows; i += SM_T) ys[i] = a.y[r0 + i];
+    if (a.mode == 1) {
+      for (int64_t i = tid; i < (int64_t)rowsv * d; i += SM_T) Xvs[i] = a.Xv[r0v * d + i];
+      for (int i = tid; i < rowsv; i += SM_T) yvs[i] = a.yv[r0v + i];
+    }
   }
   for (int j = tid; j < d; j += SM_T) { w[j] = a.w[j]; lam[j] = a.lam[j]; }
   cluster_barrier();    // every CTA of the cluster is running before anyone touches a neighbour's shared memory
   const float inv_n = a.n > 0 ? 1.f / (float)a.n : 0.f, inv_nv = a.nv > 0 ? 1.f / (float)a.nv : 0.f;
   int pb = 0;   // which half of cpart this pass writes
+  // one pass over the training rows (kind 0: gradient at vv; kind 1: curvature-weighted product with vv)
+  // or over the validation rows (gradient of the upper loss at vv)
+  auto train_pass = [&](int kind, const float* vv, float* res) {
+    float* cp = cpart + pb * SM_CL * SM_MAXD;
+    if (regs) pass_reg(x8, kind == 0 ? yreg : curvreg, has, d, a.family, inv_n, kind, vv, part, cp, res, rank);
+    else pass(Xs, ys, curv, rows, d, a.family, inv_n, kind, vv, vv, coef, part, cp, res, rank);
+    pb ^= 1;
+  };
+  auto valid_pass = [&](const float* vv, float* res) {
+    float* cp = cpart + pb * SM_CL * SM_MAXD;
+    if (regs) pass_reg(xv8, yvreg, hasv, d, a.family_up, inv_nv, 0, vv, part, cp, res, rank);
+    else pass(Xvs, yvs, nullptr, rowsv, d, a.family_up, inv_nv, 0, vv, nullptr, coef, part, cp, res, rank);
+    pb ^= 1;
+  };
 
   if (a.mode == 0) {
     for (int s = 0; s < a.n_steps; ++s) {
-      pass(Xs, ys, nullptr, rows, d, a.family, inv_n, 0, w, nullptr, coef, part, cpart + pb * SM_CL * SM_MAXD, g, rank);
-      pb ^= 1;
+      train_pass(0, w, g);
       for (int j = tid; j < d; j += SM_T) w[j] -= a.lr * (g[j] + lam[j] * w[j]);
       __syncthreads();
     }
@@ -167,8 +250,7 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
       for (int j = tid; j < d; j += SM_T) a.w[j] = w[j];
   } else {
     // v = dC_upper/dw on the validation rows
-    pass(Xvs, yvs, nullptr, rowsv, d, a.family_up, inv_nv, 0, w, nullptr, coef, part, cpart + pb * SM_CL * SM_MAXD, v, rank);
-    pb ^= 1;
+    valid_pass(w, v);
     if (a.method == BETTY_FD) {
       // dC/d(lambda) = 1/2 w^2: the central difference at w +- eps v, evaluated as written
       const float nv2 = vdot(v, v, d, red);
@@ -183,13 +265,22 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
       }
     } else {
       // curvature weights at the current w (constant over the solve)
-      for (int i = tid >> 5; i < rows; i += SM_T / 32) {
-        const float* xr = Xs + (size_t)i * d;
-        float s = 0.f;
-        for (int j = tid & 31; j < d; j += 32) s += xr[j] * w[j];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if ((tid & 31) == 0) { const float sg = sigm(s); curv[i] = a.family == 0 ? sg * (1.f - sg) * inv_n : 1.f; }
+      if (regs) {
+        const int tpr = d >> 3, c8 = tid & (tpr - 1);
+        const float4 w0 = *(const float4*)(w + 8 * c8), w1 = *(const float4*)(w + 8 * c8 + 4);
+        float s = x8[0] * w0.x + x8[1] * w0.y + x8[2] * w0.z + x8[3] * w0.w + x8[4] * w1.x + x8[5] * w1.y + x8[6] * w1.z + x8[7] * w1.w;
+        for (int o = tpr >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const float sg = sigm(s);
+        curvreg = a.family == 0 ? sg * (1.f - sg) * inv_n : 1.f;
+      } else {
+        for (int i = tid >> 5; i < rows; i += SM_T / 32) {
+          const float* xr = Xs + (size_t)i * d;
+          float s = 0.f;
+          for (int j = tid & 31; j < d; j += 32) s += xr[j] * w[j];
+  #pragma unroll
+          for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+          if ((tid & 31) == 0) { const float sg = sigm(s); curv[i] = a.family == 0 ? sg * (1.f - sg) * inv_n : 1.f; }
+        }
       }
       __syncthreads();
       float qscale = 1.f;
@@ -197,8 +288,7 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
         for (int j = tid; j < d; j += SM_T) { t[j] = v[j]; q[j] = v[j]; }
         __syncthreads();
         for (int k = 0; k < a.K; ++k) {
-          pass(Xs, ys, curv, rows, d, a.family, inv_n, 1, w, t, coef, part, cpart + pb * SM_CL * SM_MAXD, h, rank);
-          pb ^= 1;
+          train_pass(1, t, h);
           for (int j = tid; j < d; j += SM_T) {
             const float tn = t[j] - a.alpha * (h[j] + lam[j] * t[j]);
             t[j] = tn; q[j] += tn;
@@ -216,8 +306,7 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
         bool active = rho > stop;
         if (!isfinite(rho)) { status = BETTY_ERR_NONFINITE; active = false; }
         for (int k = 0; k < a.K && active; ++k) {
-          pass(Xs, ys, curv, rows, d, a.family, inv_n, 1, w, p, coef, part, cpart + pb * SM_CL * SM_MAXD, h, rank);
-          pb ^= 1;
+          train_pass(1, p, h);
           for (int j = tid; j < d; j += SM_T) h[j] += lam[j] * p[j];
           __syncthreads();
           const float gamma = vdot(p, h, d, red);
@@ -266,6 +355,12 @@ static betty_status launch_small(Ctx& c, SmallArgs& a) {
   a.rows_per_cta = (int)((a.n + SM_CL - 1) / SM_CL);
   a.rows_per_cta_v = a.mode == 1 ? (int)((a.nv + SM_CL - 1) / SM_CL) : 0;
   a.sb = c.arena.status();
+  {
+    const int d = a.d, tpr = d >> 3;
+    const bool pow2 = d >= 8 && d <= SM_MAXD && (d & (d - 1)) == 0;
+    a.in_regs = pow2 && a.rows_per_cta <= SM_T / tpr && a.rows_per_cta_v <= SM_T / tpr &&
+                (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && (a.mode == 0 || (reinterpret_cast<uintptr_t>(a.Xv) & 15) == 0);
+  }
   const size_t smem = small_smem_bytes(a.rows_per_cta, a.rows_per_cta_v, a.d);
   static size_t attr_bytes = 0;
   if (smem > attr_bytes) {
