@@ -2,10 +2,11 @@
 // whole data set fits on chip): one launch runs a complete loop -- all unrolled lower-level gradient
 // steps, or a complete hypergradient (validation gradient, Neumann / CG / finite-difference solve,
 // mixed product).  A cluster of 8 CTAs keeps the rows of X (and of the validation matrix) resident
-// in shared memory for the whole launch; in every pass each CTA pushes its column sums into all
-// eight CTAs through distributed shared memory, one cluster barrier follows, and every CTA then repeats the same O(d)
-// vector arithmetic on its own copy of the solver state, in the same order, so all copies stay
-// bit-identical.  At this size the path is bound by the latency of ~100 dependent passes, not by
+// for the whole launch -- in registers where the shape allows (pass_reg), else in shared memory (pass).
+// In every pass each CTA sends its column sums to all eight CTAs through distributed shared memory with
+// stores that are counted on the receiver's barrier, waits for the sums addressed to it, and then repeats
+// the same O(d) vector arithmetic on its own copy of the solver state, in the same order, so all copies
+// stay bit-identical.  At this size the path is bound by the latency of ~100 dependent passes, not by
 // bandwidth: the point of the kernel is to pay one launch instead of hundreds.
 #include "ops.cuh"
 
@@ -14,6 +15,7 @@ namespace betty {
 static constexpr int SM_CL = 8;          // CTAs per cluster
 static constexpr int SM_T = 1024;        // threads per CTA: the passes are latency chains, many warps hide them
 static constexpr int SM_MAXD = 256;
+static constexpr int SM_PS = SM_MAXD + 4;   // row stride of the per-group partial sums
 static constexpr int SM_NVEC = 10;       // vectors of length d kept per CTA
 
 struct SmallArgs {
@@ -33,15 +35,54 @@ struct SmallArgs {
 };
 
 __device__ __forceinline__ uint32_t sm_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void st_remote(float* local_ptr, uint32_t rank, float v) {
-  uint32_t a;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(sm_u32(local_ptr)), "r"(rank));
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory");
-}
 __device__ __forceinline__ void cluster_barrier() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// One column sum sent to CTA `rank` of the cluster; its arrival is counted (4 bytes) on that CTA's barrier.
+__device__ __forceinline__ void st_remote_counted(float* local_ptr, uint64_t* local_bar, uint32_t rank, float v) {
+  uint32_t a, b;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(sm_u32(local_ptr)), "r"(rank));
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(b) : "r"(sm_u32(local_bar)), "r"(rank));
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(a), "f"(v), "r"(b) : "memory");
+}
+static constexpr uint32_t SM_WAIT_POLLS = 1u << 22;   // bound on every wait for the neighbours' column sums
+
+// Fold the per-group partial column sums of this CTA, send them to slot `rank` of every CTA of the cluster
+// (each send counted on the receiver's barrier), wait until all SM_CL x d sums addressed to this CTA have
+// landed, and add them up in rank order into res[0..d) -- the same order everywhere, so every CTA holds the
+// same bits.  No cluster-wide barrier: a CTA waits only for data, one way.  The two halves of cpart
+// alternate between passes; a neighbour can be at most one pass ahead (it needs this CTA's sums of the
+// pass before), so what it sends lands in the half this CTA is not reading.  Returns false when the wait
+// ran out (uniform over the CTA).
+__device__ bool exchange_cols(const float* part, int groups, int d, float* cpart, uint64_t* bar, uint32_t parity,
+                              float* res, uint32_t rank) {
+  const int tid = threadIdx.x;
+  if (tid == 0)
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_u32(bar)), "r"((uint32_t)(SM_CL * d * 4)) : "memory");
+  for (int j = tid; j < d; j += SM_T) {
+    float acc = 0.f;
+    for (int g2 = 0; g2 < groups; ++g2) acc += part[g2 * SM_PS + j];   // unrolled where `groups` is a constant: independent loads
+#pragma unroll
+    for (uint32_t r = 0; r < SM_CL; ++r) st_remote_counted(cpart + rank * SM_MAXD + j, bar, r, acc);
+  }
+  // only the warps that read the sums poll the barrier; the others go on to the block barrier below
+  uint32_t done = (tid & ~31) < d ? 0u : 1u, polls = 0;
+  while (!done && polls < SM_WAIT_POLLS) {
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(done) : "r"(sm_u32(bar)), "r"(parity) : "memory");
+    ++polls;
+  }
+  if (done)
+    for (int j = tid; j < d; j += SM_T) {
+      float acc = 0.f;
+#pragma unroll
+      for (int r = 0; r < SM_CL; ++r) acc += cpart[r * SM_MAXD + j];
+      res[j] = acc;
+    }
+  return __syncthreads_or(!done) == 0;
+}
+
 __device__ __forceinline__ float sigm(float t) { return 1.f / (1.f + expf(-t)); }
 
 // block-wide sum of one value per thread (fixed order)
@@ -65,9 +106,9 @@ __device__ __forceinline__ float vdot(const float* a, const float* b, int d, flo
 // One pass over this CTA's resident rows: coef_i from the row dot products, then the column sums
 // sum_i coef_i x_ij, reduced over the cluster into res[0..d) (identical in every CTA).
 //   kind 0: gradient coefficients at `wv`;  kind 1: HVP coefficients curv_i * (x_i . dir)
-__device__ void pass(const float* Xs, const float* ys, const float* curv, int rows, int d, int family, float inv_n,
-                     int kind, const float* wv, const float* dir, float* coef, float* part, float* cpart, float* res,
-                     uint32_t rank) {
+__device__ bool pass(const float* Xs, const float* ys, const float* curv, int rows, int d, int family, float inv_n,
+                     int kind, const float* wv, const float* dir, float* coef, float* part, float* cpart, uint64_t* bar,
+                     uint32_t parity, float* res, uint32_t rank) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // A: one warp per row, four rows in flight per warp so that the shuffle chains overlap
   const float* vv = kind == 0 ? wv : dir;
@@ -102,41 +143,61 @@ __device__ void pass(const float* Xs, const float* ys, const float* curv, int ro
   for (int j = c0; j < d; j += ct) {
     float a = 0.f;
     for (int i = rg; i < rows; i += groups) a += coef[i] * Xs[(size_t)i * d + j];
-    part[rg * SM_MAXD + j] = a;
+    part[rg * SM_PS + j] = a;
   }
   __syncthreads();
-  // fold the row groups and push this CTA's column sums into slot `rank` of every CTA of the cluster
-  for (int j = tid; j < d; j += SM_T) {
-    float a = 0.f;
-    for (int g2 = 0; g2 < groups; ++g2) a += part[g2 * SM_MAXD + j];
-#pragma unroll
-    for (uint32_t r = 0; r < SM_CL; ++r) st_remote(cpart + rank * SM_MAXD + j, r, a);
-  }
-  cluster_barrier();                       // all pushes have landed everywhere
-  for (int j = tid; j < d; j += SM_T) {
-    float a = 0.f;
-#pragma unroll
-    for (int r = 0; r < SM_CL; ++r) a += cpart[r * SM_MAXD + j];
-    res[j] = a;
-  }
-  __syncthreads();
-  (void)rank;
+  return exchange_cols(part, groups, d, cpart, bar, parity, res, rank);
 }
 
-// The same pass with the CTA's rows held in registers for the whole launch: d / 8 adjacent threads own one
-// row, eight columns each (d a power of two between 8 and 256, at most SM_T / (d / 8) rows per CTA: the
+// Column sums over the rows of one warp (TPR threads per row, so 32 / TPR rows; lane bits >= TPR select the
+// row).  A butterfly that halves what a lane keeps at every round -- the lane with the round's bit clear keeps
+// the lower half of its values and receives the partner's contribution to them, the other lane the upper
+// half -- costs 4 + 2 + 1 shuffles for eight values where a plain butterfly costs 8 per round; shuffle issue
+// (one warp-wide shuffle per clock per SM, 32 warps) is what the pass spends most of its time on.
+// On return col[0 .. NF) are the sums of columns 8 c8 + off + i; `writer` is false in lanes holding duplicates.
+template <int O, int N>
+struct WarpColumnSum {
+  static __device__ __forceinline__ void run(float (&col)[8], int lane, int& off, bool& writer) {
+    if constexpr (O < 32) {
+      const bool up = (lane & O) != 0;
+      if constexpr (N > 1) {
+        constexpr int H = N / 2;
+#pragma unroll
+        for (int i = 0; i < H; ++i) {
+          const float send = up ? col[i] : col[i + H];
+          const float keep = up ? col[i + H] : col[i];
+          col[i] = keep + __shfl_xor_sync(0xffffffffu, send, O);
+        }
+        if (up) off += H;
+        WarpColumnSum<O * 2, H>::run(col, lane, off, writer);
+      } else {
+        col[0] += __shfl_xor_sync(0xffffffffu, col[0], O);
+        if (up) writer = false;
+        WarpColumnSum<O * 2, 1>::run(col, lane, off, writer);
+      }
+    }
+  }
+};
+template <int TPR> struct RowsPerWarp { static constexpr int value = 32 / TPR; };
+template <int TPR> struct ColsLeft { static constexpr int value = 8 / RowsPerWarp<TPR>::value > 0 ? 8 / RowsPerWarp<TPR>::value : 1; };
+
+// The same pass with the CTA's rows held in registers for the whole launch: TPR = d / 8 adjacent threads own
+// one row, eight columns each (d a power of two between 8 and 256, at most SM_T / TPR rows per CTA: the
 // 1024 x 64 problem gives every CTA 128 rows of 8 threads).  A pass is then 8 multiply-adds, a shuffle
-// reduction over the row's threads, the coefficient, 8 more multiply-adds and a shuffle reduction over the
-// warp's rows; shared memory is touched only for the 32 per-warp column sums.  (The shared-memory pass above
-// spends ~3400 clocks per 128 rows on its two sweeps over X.)
+// reduction over the row's threads, the coefficient, 8 more multiplies and the column sums over the warp's
+// rows; shared memory is touched only for the 32 per-warp column sums.
 //   x8: this thread's eight columns of its row; yv: the row's label (kind 0) or curvature (kind 1); has: row exists
-__device__ void pass_reg(const float (&x8)[8], float yv, bool has, int d, int family, float inv_n, int kind,
-                         const float* vv, float* part, float* cpart, float* res, uint32_t rank) {
+template <int TPR>
+__device__ __forceinline__ bool pass_reg(const float (&x8)[8], float yv, bool has, int family, float inv_n, int kind,
+                                         const float* vv, float* part, float* cpart, uint64_t* bar, uint32_t parity,
+                                         float* res, uint32_t rank) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int tpr = d >> 3, c8 = tid & (tpr - 1);
+  constexpr int d = 8 * TPR;
+  const int c8 = tid & (TPR - 1);
   const float4 v0 = *(const float4*)(vv + 8 * c8), v1 = *(const float4*)(vv + 8 * c8 + 4);
   float sdot = x8[0] * v0.x + x8[1] * v0.y + x8[2] * v0.z + x8[3] * v0.w + x8[4] * v1.x + x8[5] * v1.y + x8[6] * v1.z + x8[7] * v1.w;
-  for (int o = tpr >> 1; o > 0; o >>= 1) sdot += __shfl_xor_sync(0xffffffffu, sdot, o);
+#pragma unroll
+  for (int o = TPR >> 1; o > 0; o >>= 1) sdot += __shfl_xor_sync(0xffffffffu, sdot, o);
   float cf = 0.f;
   if (has) {
     if (kind == 0) cf = family == 0 ? -yv * sigm(-yv * sdot) * inv_n : (sdot - yv);
@@ -145,30 +206,28 @@ __device__ void pass_reg(const float (&x8)[8], float yv, bool has, int d, int fa
   float col[8];
 #pragma unroll
   for (int k = 0; k < 8; ++k) col[k] = cf * x8[k];
-  for (int o = tpr; o < 32; o <<= 1) {
+  int off = 0;
+  bool writer = true;
+  WarpColumnSum<TPR, 8>::run(col, lane, off, writer);
+  if (writer) {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) col[k] += __shfl_xor_sync(0xffffffffu, col[k], o);
-  }
-  if (lane < tpr) {
-    *(float4*)(part + warp * SM_MAXD + 8 * c8) = make_float4(col[0], col[1], col[2], col[3]);
-    *(float4*)(part + warp * SM_MAXD + 8 * c8 + 4) = make_float4(col[4], col[5], col[6], col[7]);
-  }
-  __syncthreads();
-  for (int j = tid; j < d; j += SM_T) {
-    float acc = 0.f;
-#pragma unroll
-    for (int w2 = 0; w2 < SM_T / 32; ++w2) acc += part[w2 * SM_MAXD + j];
-#pragma unroll
-    for (uint32_t r = 0; r < SM_CL; ++r) st_remote(cpart + rank * SM_MAXD + j, r, acc);
-  }
-  cluster_barrier();                       // all pushes have landed everywhere
-  for (int j = tid; j < d; j += SM_T) {
-    float acc = 0.f;
-#pragma unroll
-    for (int r = 0; r < SM_CL; ++r) acc += cpart[r * SM_MAXD + j];
-    res[j] = acc;
+    for (int i = 0; i < ColsLeft<TPR>::value; ++i) part[warp * SM_PS + 8 * c8 + off + i] = col[i];
   }
   __syncthreads();
+  return exchange_cols(part, SM_T / 32, d, cpart, bar, parity, res, rank);
+}
+// dispatch on the threads per row
+__device__ __forceinline__ bool pass_reg_any(int tpr, const float (&x8)[8], float yv, bool has, int family, float inv_n, int kind,
+                                             const float* vv, float* part, float* cpart, uint64_t* bar, uint32_t parity,
+                                             float* res, uint32_t rank) {
+  switch (tpr) {
+    case 1: return pass_reg<1>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
+    case 2: return pass_reg<2>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
+    case 4: return pass_reg<4>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
+    case 8: return pass_reg<8>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
+    case 16: return pass_reg<16>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
+    default: return pass_reg<32>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
+  }
 }
 
 __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logreg_small(SmallArgs a) {
@@ -185,8 +244,8 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   float* coef = curv + R;                          // [max(R, Rv)]
   float* vec = coef + (R > Rv ? R : Rv);           // SM_NVEC vectors of SM_MAXD, 16-byte aligned for float4 access
   vec += (4 - ((vec - sm) & 3)) & 3;
-  float* part = vec + SM_NVEC * SM_MAXD;           // [32][SM_MAXD] row-group partials
-  float* cpart = part + 32 * SM_MAXD;              // [2][SM_CL][SM_MAXD] column sums of every CTA (double-buffered)
+  float* part = vec + SM_NVEC * SM_MAXD;           // [32][SM_PS] row-group partials
+  float* cpart = part + 32 * SM_PS;               // [2][SM_CL][SM_MAXD] column sums of every CTA (double-buffered)
   float* red = cpart + 2 * SM_CL * SM_MAXD;                // [32] block reduction scratch
   float *w = vec, *lam = vec + SM_MAXD, *g = vec + 2 * SM_MAXD, *v = vec + 3 * SM_MAXD, *q = vec + 4 * SM_MAXD,
         *r = vec + 5 * SM_MAXD, *p = vec + 6 * SM_MAXD, *h = vec + 7 * SM_MAXD, *t = vec + 8 * SM_MAXD;
@@ -222,26 +281,38 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
     }
   }
   for (int j = tid; j < d; j += SM_T) { w[j] = a.w[j]; lam[j] = a.lam[j]; }
-  cluster_barrier();    // every CTA of the cluster is running before anyone touches a neighbour's shared memory
+  __shared__ __align__(8) uint64_t xbar[2];   // one per half of cpart: counts the bytes of column sums that have landed
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_u32(&xbar[0])));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_u32(&xbar[1])));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  cluster_barrier();    // every CTA of the cluster is running, its barriers set up, before anyone sends to it
   const float inv_n = a.n > 0 ? 1.f / (float)a.n : 0.f, inv_nv = a.nv > 0 ? 1.f / (float)a.nv : 0.f;
   int pb = 0;   // which half of cpart this pass writes
   // one pass over the training rows (kind 0: gradient at vv; kind 1: curvature-weighted product with vv)
   // or over the validation rows (gradient of the upper loss at vv)
+  uint32_t ph = 0;   // bit b: parity of the phase half b waits for next
+  bool alive = true; // false once a wait for the neighbours ran out: the loops stop and the status is recorded
   auto train_pass = [&](int kind, const float* vv, float* res) {
     float* cp = cpart + pb * SM_CL * SM_MAXD;
-    if (regs) pass_reg(x8, kind == 0 ? yreg : curvreg, has, d, a.family, inv_n, kind, vv, part, cp, res, rank);
-    else pass(Xs, ys, curv, rows, d, a.family, inv_n, kind, vv, vv, coef, part, cp, res, rank);
-    pb ^= 1;
+    const uint32_t par = (ph >> pb) & 1u;
+    bool ok;
+    if (regs) ok = pass_reg_any(d >> 3, x8, kind == 0 ? yreg : curvreg, has, a.family, inv_n, kind, vv, part, cp, &xbar[pb], par, res, rank);
+    else ok = pass(Xs, ys, curv, rows, d, a.family, inv_n, kind, vv, vv, coef, part, cp, &xbar[pb], par, res, rank);
+    alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
   };
   auto valid_pass = [&](const float* vv, float* res) {
     float* cp = cpart + pb * SM_CL * SM_MAXD;
-    if (regs) pass_reg(xv8, yvreg, hasv, d, a.family_up, inv_nv, 0, vv, part, cp, res, rank);
-    else pass(Xvs, yvs, nullptr, rowsv, d, a.family_up, inv_nv, 0, vv, nullptr, coef, part, cp, res, rank);
-    pb ^= 1;
+    const uint32_t par = (ph >> pb) & 1u;
+    bool ok;
+    if (regs) ok = pass_reg_any(d >> 3, xv8, yvreg, hasv, a.family_up, inv_nv, 0, vv, part, cp, &xbar[pb], par, res, rank);
+    else ok = pass(Xvs, yvs, nullptr, rowsv, d, a.family_up, inv_nv, 0, vv, nullptr, coef, part, cp, &xbar[pb], par, res, rank);
+    alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
   };
 
   if (a.mode == 0) {
-    for (int s = 0; s < a.n_steps; ++s) {
+    for (int s = 0; s < a.n_steps && alive; ++s) {
       train_pass(0, w, g);
       for (int j = tid; j < d; j += SM_T) w[j] -= a.lr * (g[j] + lam[j] * w[j]);
       __syncthreads();
@@ -287,7 +358,7 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
       if (a.method == BETTY_NEUMANN) {
         for (int j = tid; j < d; j += SM_T) { t[j] = v[j]; q[j] = v[j]; }
         __syncthreads();
-        for (int k = 0; k < a.K; ++k) {
+        for (int k = 0; k < a.K && alive; ++k) {
           train_pass(1, t, h);
           for (int j = tid; j < d; j += SM_T) {
             const float tn = t[j] - a.alpha * (h[j] + lam[j] * t[j]);
@@ -307,6 +378,7 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
         if (!isfinite(rho)) { status = BETTY_ERR_NONFINITE; active = false; }
         for (int k = 0; k < a.K && active; ++k) {
           train_pass(1, p, h);
+          if (!alive) break;
           for (int j = tid; j < d; j += SM_T) h[j] += lam[j] * p[j];
           __syncthreads();
           const float gamma = vdot(p, h, d, red);
@@ -334,12 +406,13 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
         for (int j = tid; j < d; j += SM_T) a.out[j] = -qscale * w[j] * q[j];
     }
   }
-  // no CTA may leave while a neighbour can still read its column sums
+  if (!alive && tid == 0) record_status(a.sb, BETTY_ERR_TIMEOUT);
+  // no CTA may leave while a neighbour can still send to it
   cluster_barrier();
 }
 
 static size_t small_smem_bytes(int R, int Rv, int d) {
-  size_t floats = (size_t)R * d + (size_t)Rv * d + R + Rv + R + (R > Rv ? R : Rv) + (size_t)SM_NVEC * SM_MAXD + 32 * SM_MAXD +
+  size_t floats = (size_t)R * d + (size_t)Rv * d + R + Rv + R + (R > Rv ? R : Rv) + (size_t)SM_NVEC * SM_MAXD + 32 * SM_PS +
                   2 * SM_CL * SM_MAXD + 32;
   return floats * sizeof(float) + 16;
 }
