@@ -324,6 +324,14 @@ static betty_status hypergrad_itd(const betty_level* lower, const betty_level* u
   if (!is_participant(upper, lower) || !is_participant(upper, wrt) || !is_participant(lower, wrt) || wrt == lower)
     return BETTY_ERR_INVALID_ARG;
   Ctx c(ws, ws_bytes, stream);
+  // Small logistic / least-squares bilevel pair with one step size: unrolled steps and reverse sweep in one launch.
+  if (n_steps > 0 && vec_has_wd(lower) && lower->lr_schedule == BETTY_LR_CONSTANT &&
+      (upper->loss == BETTY_LOSS_LOGREG || upper->loss == BETTY_LOSS_QUADRATIC) &&
+      find_constraint(upper, BETTY_PARAM_VECTOR) == lower && wrt == find_constraint(lower, BETTY_PARAM_VECTOR) &&
+      logreg_small_eligible(lower->n, upper->n, lower->d, n_steps))
+    return logreg_small_itd(c, vec_family(lower), (const float*)lower->X, (const float*)lower->y, lower->n, vec_family(upper),
+                            (const float*)upper->X, (const float*)upper->y, upper->n, lower->d, lower->params, wrt->params,
+                            n_steps, lower->lr, out);
   const int64_t n = lower->n_params, nc = wrt->n_params;
   const bool vecfam = is_vector_family(lower->loss);
   const size_t stride = ((size_t)n + 63) & ~size_t(63);

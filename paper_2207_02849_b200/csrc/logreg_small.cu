@@ -25,7 +25,7 @@ struct SmallArgs {
   int family, family_up;                            // 0 logistic, 1 least squares
   float* w;                                         // lower parameters (updated in lower-step mode)
   const float* lam;
-  int mode;                                         // 0: lower steps; 1: hypergradient
+  int mode;                                         // 0: lower steps; 1: hypergradient; 2: ITD-RMAD hypergradient over n_steps unrolled steps
   int n_steps; float lr;
   int method, K; float alpha, eps0, tol;            // betty_method and its parameters
   float* out;                                       // hypergradient [d] (added to nothing: direct gradient is zero)
@@ -105,7 +105,8 @@ __device__ __forceinline__ float vdot(const float* a, const float* b, int d, flo
 
 // One pass over this CTA's resident rows: coef_i from the row dot products, then the column sums
 // sum_i coef_i x_ij, reduced over the cluster into res[0..d) (identical in every CTA).
-//   kind 0: gradient coefficients at `wv`;  kind 1: HVP coefficients curv_i * (x_i . dir)
+//   kind 0: gradient coefficients at `wv`;  kind 1: HVP coefficients curv_i * (x_i . dir);
+//   kind 2: HVP coefficients with the curvature taken at `wv` on the fly (a stored iterate of the unrolled loop)
 __device__ bool pass(const float* Xs, const float* ys, const float* curv, int rows, int d, int family, float inv_n,
                      int kind, const float* wv, const float* dir, float* coef, float* part, float* cpart, uint64_t* bar,
                      uint32_t parity, float* res, uint32_t rank) {
@@ -113,13 +114,15 @@ __device__ bool pass(const float* Xs, const float* ys, const float* curv, int ro
   // A: one warp per row, four rows in flight per warp so that the shuffle chains overlap
   const float* vv = kind == 0 ? wv : dir;
   for (int i0 = warp * 4; i0 < rows; i0 += (SM_T / 32) * 4) {
-    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    float s[4] = {0.f, 0.f, 0.f, 0.f}, z[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int i = i0 + u;
       if (i < rows) {
         const float* xr = Xs + (size_t)i * d;
         for (int j = lane; j < d; j += 32) s[u] += xr[j] * vv[j];
+        if (kind == 2)
+          for (int j = lane; j < d; j += 32) z[u] += xr[j] * wv[j];
       }
     }
 #pragma unroll
@@ -127,12 +130,21 @@ __device__ bool pass(const float* Xs, const float* ys, const float* curv, int ro
 #pragma unroll
       for (int u = 0; u < 4; ++u) s[u] += __shfl_xor_sync(0xffffffffu, s[u], o);
     }
+    if (kind == 2) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) z[u] += __shfl_xor_sync(0xffffffffu, z[u], o);
+      }
+    }
     if (lane < 4 && i0 + lane < rows) {
       const int i = i0 + lane;
       const float sv = lane == 0 ? s[0] : (lane == 1 ? s[1] : (lane == 2 ? s[2] : s[3]));
+      const float zv = lane == 0 ? z[0] : (lane == 1 ? z[1] : (lane == 2 ? z[2] : z[3]));
       float cf;
       if (kind == 0) cf = family == 0 ? -ys[i] * sigm(-ys[i] * sv) * inv_n : (sv - ys[i]);
-      else cf = curv[i] * sv;
+      else if (kind == 1) cf = curv[i] * sv;
+      else { const float sg = sigm(zv); cf = (family == 0 ? sg * (1.f - sg) * inv_n : 1.f) * sv; }
       coef[i] = cf;
     }
   }
@@ -186,22 +198,32 @@ template <int TPR> struct ColsLeft { static constexpr int value = 8 / RowsPerWar
 // 1024 x 64 problem gives every CTA 128 rows of 8 threads).  A pass is then 8 multiply-adds, a shuffle
 // reduction over the row's threads, the coefficient, 8 more multiplies and the column sums over the warp's
 // rows; shared memory is touched only for the 32 per-warp column sums.
-//   x8: this thread's eight columns of its row; yv: the row's label (kind 0) or curvature (kind 1); has: row exists
+//   x8: this thread's eight columns of its row; yv: the row's label (kind 0) or curvature (kind 1); has: row exists;
+//   wt: the iterate the curvature is taken at (kind 2)
 template <int TPR>
 __device__ __forceinline__ bool pass_reg(const float (&x8)[8], float yv, bool has, int family, float inv_n, int kind,
-                                         const float* vv, float* part, float* cpart, uint64_t* bar, uint32_t parity,
-                                         float* res, uint32_t rank) {
+                                         const float* vv, const float* wt, float* part, float* cpart, uint64_t* bar,
+                                         uint32_t parity, float* res, uint32_t rank) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int d = 8 * TPR;
   const int c8 = tid & (TPR - 1);
   const float4 v0 = *(const float4*)(vv + 8 * c8), v1 = *(const float4*)(vv + 8 * c8 + 4);
   float sdot = x8[0] * v0.x + x8[1] * v0.y + x8[2] * v0.z + x8[3] * v0.w + x8[4] * v1.x + x8[5] * v1.y + x8[6] * v1.z + x8[7] * v1.w;
+  float zdot = 0.f;
+  if (kind == 2) {
+    const float4 w0 = *(const float4*)(wt + 8 * c8), w1 = *(const float4*)(wt + 8 * c8 + 4);
+    zdot = x8[0] * w0.x + x8[1] * w0.y + x8[2] * w0.z + x8[3] * w0.w + x8[4] * w1.x + x8[5] * w1.y + x8[6] * w1.z + x8[7] * w1.w;
+  }
 #pragma unroll
-  for (int o = TPR >> 1; o > 0; o >>= 1) sdot += __shfl_xor_sync(0xffffffffu, sdot, o);
+  for (int o = TPR >> 1; o > 0; o >>= 1) {
+    sdot += __shfl_xor_sync(0xffffffffu, sdot, o);
+    if (kind == 2) zdot += __shfl_xor_sync(0xffffffffu, zdot, o);
+  }
   float cf = 0.f;
   if (has) {
     if (kind == 0) cf = family == 0 ? -yv * sigm(-yv * sdot) * inv_n : (sdot - yv);
-    else cf = yv * sdot;
+    else if (kind == 1) cf = yv * sdot;
+    else { const float sg = sigm(zdot); cf = (family == 0 ? sg * (1.f - sg) * inv_n : 1.f) * sdot; }
   }
   float col[8];
 #pragma unroll
@@ -218,15 +240,15 @@ __device__ __forceinline__ bool pass_reg(const float (&x8)[8], float yv, bool ha
 }
 // dispatch on the threads per row
 __device__ __forceinline__ bool pass_reg_any(int tpr, const float (&x8)[8], float yv, bool has, int family, float inv_n, int kind,
-                                             const float* vv, float* part, float* cpart, uint64_t* bar, uint32_t parity,
-                                             float* res, uint32_t rank) {
+                                             const float* vv, const float* wt, float* part, float* cpart, uint64_t* bar,
+                                             uint32_t parity, float* res, uint32_t rank) {
   switch (tpr) {
-    case 1: return pass_reg<1>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
-    case 2: return pass_reg<2>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
-    case 4: return pass_reg<4>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
-    case 8: return pass_reg<8>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
-    case 16: return pass_reg<16>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
-    default: return pass_reg<32>(x8, yv, has, family, inv_n, kind, vv, part, cpart, bar, parity, res, rank);
+    case 1: return pass_reg<1>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
+    case 2: return pass_reg<2>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
+    case 4: return pass_reg<4>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
+    case 8: return pass_reg<8>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
+    case 16: return pass_reg<16>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
+    default: return pass_reg<32>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
   }
 }
 
@@ -247,6 +269,8 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   float* part = vec + SM_NVEC * SM_MAXD;           // [32][SM_PS] row-group partials
   float* cpart = part + 32 * SM_PS;               // [2][SM_CL][SM_MAXD] column sums of every CTA (double-buffered)
   float* red = cpart + 2 * SM_CL * SM_MAXD;                // [32] block reduction scratch
+  float* traj = red + 32;                                  // [n_steps][d] stored iterates (ITD-RMAD), 16-byte aligned
+  traj += (4 - ((traj - sm) & 3)) & 3;
   float *w = vec, *lam = vec + SM_MAXD, *g = vec + 2 * SM_MAXD, *v = vec + 3 * SM_MAXD, *q = vec + 4 * SM_MAXD,
         *r = vec + 5 * SM_MAXD, *p = vec + 6 * SM_MAXD, *h = vec + 7 * SM_MAXD, *t = vec + 8 * SM_MAXD;
 
@@ -261,7 +285,7 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   bool has = false, hasv = false;
   if (regs) {
     const int tpr = d >> 3, row = tid / tpr, c8 = tid & (tpr - 1);
-    has = row < rows; hasv = a.mode == 1 && row < rowsv;
+    has = row < rows; hasv = a.mode != 0 && row < rowsv;
     if (has) {
       const float4 lo = *(const float4*)(a.X + (r0 + row) * d + 8 * c8), hi = *(const float4*)(a.X + (r0 + row) * d + 8 * c8 + 4);
       x8[0] = lo.x; x8[1] = lo.y; x8[2] = lo.z; x8[3] = lo.w; x8[4] = hi.x; x8[5] = hi.y; x8[6] = hi.z; x8[7] = hi.w;
@@ -275,7 +299,7 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   } else {
     for (int64_t i = tid; i < (int64_t)rows * d; i += SM_T) Xs[i] = a.X[r0 * d + i];
     for (int i = tid; i < rows; i += SM_T) ys[i] = a.y[r0 + i];
-    if (a.mode == 1) {
+    if (a.mode != 0) {
       for (int64_t i = tid; i < (int64_t)rowsv * d; i += SM_T) Xvs[i] = a.Xv[r0v * d + i];
       for (int i = tid; i < rowsv; i += SM_T) yvs[i] = a.yv[r0v + i];
     }
@@ -294,19 +318,19 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   // or over the validation rows (gradient of the upper loss at vv)
   uint32_t ph = 0;   // bit b: parity of the phase half b waits for next
   bool alive = true; // false once a wait for the neighbours ran out: the loops stop and the status is recorded
-  auto train_pass = [&](int kind, const float* vv, float* res) {
+  auto train_pass = [&](int kind, const float* vv, float* res, const float* wt = nullptr) {
     float* cp = cpart + pb * SM_CL * SM_MAXD;
     const uint32_t par = (ph >> pb) & 1u;
     bool ok;
-    if (regs) ok = pass_reg_any(d >> 3, x8, kind == 0 ? yreg : curvreg, has, a.family, inv_n, kind, vv, part, cp, &xbar[pb], par, res, rank);
-    else ok = pass(Xs, ys, curv, rows, d, a.family, inv_n, kind, vv, vv, coef, part, cp, &xbar[pb], par, res, rank);
+    if (regs) ok = pass_reg_any(d >> 3, x8, kind == 0 ? yreg : curvreg, has, a.family, inv_n, kind, vv, wt, part, cp, &xbar[pb], par, res, rank);
+    else ok = pass(Xs, ys, curv, rows, d, a.family, inv_n, kind, kind == 2 ? wt : vv, vv, coef, part, cp, &xbar[pb], par, res, rank);
     alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
   };
   auto valid_pass = [&](const float* vv, float* res) {
     float* cp = cpart + pb * SM_CL * SM_MAXD;
     const uint32_t par = (ph >> pb) & 1u;
     bool ok;
-    if (regs) ok = pass_reg_any(d >> 3, xv8, yvreg, hasv, a.family_up, inv_nv, 0, vv, part, cp, &xbar[pb], par, res, rank);
+    if (regs) ok = pass_reg_any(d >> 3, xv8, yvreg, hasv, a.family_up, inv_nv, 0, vv, nullptr, part, cp, &xbar[pb], par, res, rank);
     else ok = pass(Xvs, yvs, nullptr, rowsv, d, a.family_up, inv_nv, 0, vv, nullptr, coef, part, cp, &xbar[pb], par, res, rank);
     alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
   };
@@ -319,6 +343,30 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
     }
     if (rank == 0)
       for (int j = tid; j < d; j += SM_T) a.w[j] = w[j];
+  } else if (a.mode == 2) {
+    // ITD-RMAD (Sec. 3.2, iterative differentiation): the unrolled steps with every iterate kept on chip,
+    // then the reverse sweep  out <- out - lr w_t .* a,  a <- a - lr (H(w_t) a + lam .* a)  for t = T-1 ... 0,
+    // one pass per reverse step (both row dot products, x.w_t for the curvature and x.a, in the same pass)
+    for (int s = 0; s < a.n_steps && alive; ++s) {
+      for (int j = tid; j < d; j += SM_T) traj[(size_t)s * d + j] = w[j];
+      train_pass(0, w, g);
+      for (int j = tid; j < d; j += SM_T) w[j] -= a.lr * (g[j] + lam[j] * w[j]);
+      __syncthreads();
+    }
+    valid_pass(w, v);                                  // a = dC_upper/dw at w_T
+    for (int j = tid; j < d; j += SM_T) q[j] = 0.f;    // the upper cost has no direct dependence on lam
+    __syncthreads();
+    for (int s = a.n_steps - 1; s >= 0 && alive; --s) {
+      const float* wt = traj + (size_t)s * d;
+      train_pass(2, v, h, wt);
+      for (int j = tid; j < d; j += SM_T) {
+        q[j] -= a.lr * (wt[j] * v[j]);
+        v[j] -= a.lr * (h[j] + lam[j] * v[j]);
+      }
+      __syncthreads();
+    }
+    if (rank == 0)
+      for (int j = tid; j < d; j += SM_T) { a.out[j] = q[j]; a.w[j] = w[j]; }
   } else {
     // v = dC_upper/dw on the validation rows
     valid_pass(w, v);
@@ -411,22 +459,23 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   cluster_barrier();
 }
 
-static size_t small_smem_bytes(int R, int Rv, int d) {
+static size_t small_smem_bytes(int R, int Rv, int d, int64_t traj_floats) {
   size_t floats = (size_t)R * d + (size_t)Rv * d + R + Rv + R + (R > Rv ? R : Rv) + (size_t)SM_NVEC * SM_MAXD + 32 * SM_PS +
-                  2 * SM_CL * SM_MAXD + 32;
-  return floats * sizeof(float) + 16;
+                  2 * SM_CL * SM_MAXD + 32 + (size_t)traj_floats;
+  return floats * sizeof(float) + 32;
 }
 
-// True when the whole problem fits the cluster's shared memory.
-bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d) {
-  if (d <= 0 || d > SM_MAXD || n <= 0 || n > (1 << 20) || nv < 0 || nv > (1 << 20)) return false;
+// True when the whole problem (and `unrolled_steps` stored iterates, for ITD-RMAD) fits the cluster's shared memory.
+bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d, int64_t unrolled_steps) {
+  if (d <= 0 || d > SM_MAXD || n <= 0 || n > (1 << 20) || nv < 0 || nv > (1 << 20) || unrolled_steps < 0 || unrolled_steps > (1 << 16))
+    return false;
   const int R = (int)((n + SM_CL - 1) / SM_CL), Rv = (int)((nv + SM_CL - 1) / SM_CL);
-  return small_smem_bytes(R, Rv, (int)d) <= 225 * 1024;
+  return small_smem_bytes(R, Rv, (int)d, unrolled_steps * d) <= 225 * 1024;
 }
 
 static betty_status launch_small(Ctx& c, SmallArgs& a) {
   a.rows_per_cta = (int)((a.n + SM_CL - 1) / SM_CL);
-  a.rows_per_cta_v = a.mode == 1 ? (int)((a.nv + SM_CL - 1) / SM_CL) : 0;
+  a.rows_per_cta_v = a.mode != 0 ? (int)((a.nv + SM_CL - 1) / SM_CL) : 0;
   a.sb = c.arena.status();
   {
     const int d = a.d, tpr = d >> 3;
@@ -434,7 +483,7 @@ static betty_status launch_small(Ctx& c, SmallArgs& a) {
     a.in_regs = pow2 && a.rows_per_cta <= SM_T / tpr && a.rows_per_cta_v <= SM_T / tpr &&
                 (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && (a.mode == 0 || (reinterpret_cast<uintptr_t>(a.Xv) & 15) == 0);
   }
-  const size_t smem = small_smem_bytes(a.rows_per_cta, a.rows_per_cta_v, a.d);
+  const size_t smem = small_smem_bytes(a.rows_per_cta, a.rows_per_cta_v, a.d, a.mode == 2 ? (int64_t)a.n_steps * a.d : 0);
   static size_t attr_bytes = 0;
   if (smem > attr_bytes) {
     if (cudaFuncSetAttribute(k_logreg_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BETTY_ERR_CUDA;
@@ -459,6 +508,15 @@ betty_status logreg_small_hypergrad(Ctx& c, int family, const float* X, const fl
   a.X = X; a.y = y; a.n = n; a.Xv = Xv; a.yv = yv; a.nv = nv; a.d = (int)d; a.family = family; a.family_up = family_up;
   a.w = w; a.lam = lam; a.mode = 1; a.method = cfg.method; a.K = cfg.K; a.alpha = cfg.alpha; a.eps0 = cfg.eps0; a.tol = cfg.tol;
   a.out = out;
+  return launch_small(c, a);
+}
+
+betty_status logreg_small_itd(Ctx& c, int family, const float* X, const float* y, int64_t n, int family_up, const float* Xv,
+                              const float* yv, int64_t nv, int64_t d, float* w, const float* lam, int n_steps, float lr,
+                              float* out) {
+  SmallArgs a = {};
+  a.X = X; a.y = y; a.n = n; a.Xv = Xv; a.yv = yv; a.nv = nv; a.d = (int)d; a.family = family; a.family_up = family_up;
+  a.w = w; a.lam = lam; a.mode = 2; a.n_steps = n_steps; a.lr = lr; a.out = out;
   return launch_small(c, a);
 }
 

@@ -29,7 +29,10 @@ betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int
                          bool curv_valid = false);
 
 // logreg_small.cu: whole-loop kernels for problems that fit a cluster's shared memory
-bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d);
+bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d, int64_t unrolled_steps = 0);
+betty_status logreg_small_itd(Ctx& c, int family, const float* X, const float* y, int64_t n, int family_up, const float* Xv,
+                              const float* yv, int64_t nv, int64_t d, float* w, const float* lam, int n_steps, float lr,
+                              float* out);
 betty_status logreg_small_lower_step(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, float* w,
                                      const float* lam, int n_steps, float lr);
 betty_status logreg_small_hypergrad(Ctx& c, int family, const float* X, const float* y, int64_t n, int family_up,

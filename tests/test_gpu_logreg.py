@@ -209,15 +209,25 @@ def test_repeated_calls_are_bitwise_identical(bt):
     assert torch.equal(a, b)
 
 
-@pytest.mark.parametrize("n,d,nv,T", [(1024, 64, 256, 100), (700, 1028, 90, 12)])
-def test_itd_hypergradient_matches_oracle(bt, n, d, nv, T):
-    """ITD-RMAD: reverse sweep through the stored unrolled steps."""
+@pytest.mark.parametrize("n,d,nv,T,on_chip", [
+    (1024, 64, 256, 100, True),      # the small configuration: rows in registers, iterates in shared memory
+    (999, 50, 77, 20, True),         # odd width: rows in shared memory
+    (2048, 128, 256, 10, True),      # 256 rows per CTA: shared memory
+    (300, 16, 10, 1, True),          # a single unrolled step
+    (1024, 64, 256, 500, False),     # 500 stored iterates do not fit beside the rows: general path
+    (700, 1028, 90, 12, False),      # too wide for the on-chip kernel
+])
+def test_itd_hypergradient_matches_oracle(bt, n, d, nv, T, on_chip):
+    """ITD-RMAD: reverse sweep through the stored unrolled steps -- in one launch where the rows and
+    the iterates fit on chip, else step by step with the iterates in the workspace."""
     from tests import cuda_build as cb
     inp = si.config1() if (n, d) == (1024, 64) else si.logreg_bilevel(77, n, d, nv)
     (w, lam), (ow, olam) = _pair(inp)
     ws = bt.Workspace([w, lam], extra_bytes=(T + 1) * (d + 64) * 4)
     out = _vec(d)
+    l0 = bt.betty_kernel_launches()
     bt.betty_hypergrad_itd(w, lam, lam, T, out, ws)
+    assert (bt.betty_kernel_launches() - l0 == 1) == on_chip
     ref = oracle.hypergrad_itd(ow, olam, olam, T)
     assert cb.rel_l2(w.params, ow.params) < TOL
     assert cb.rel_l2(out, ref) < TOL
