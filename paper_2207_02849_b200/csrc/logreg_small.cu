@@ -46,7 +46,7 @@ __device__ __forceinline__ void st_remote_counted(float* local_ptr, uint64_t* lo
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(b) : "r"(sm_u32(local_bar)), "r"(rank));
   asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(a), "f"(v), "r"(b) : "memory");
 }
-static constexpr uint32_t SM_WAIT_POLLS = 1u << 22;   // bound on every wait for the neighbours' column sums
+static constexpr uint32_t SM_WAIT_POLLS = 1u << 20;   // bound on every wait for the neighbours' column sums
 
 // Fold the per-group partial column sums of this CTA, send them to slot `rank` of every CTA of the cluster
 // (each send counted on the receiver's barrier), wait until all SM_CL x d sums addressed to this CTA have
