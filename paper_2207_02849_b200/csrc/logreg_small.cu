@@ -50,13 +50,14 @@ static constexpr uint32_t SM_WAIT_POLLS = 1u << 20;   // bound on every wait for
 
 // Fold the per-group partial column sums of this CTA, send them to slot `rank` of every CTA of the cluster
 // (each send counted on the receiver's barrier), wait until all SM_CL x d sums addressed to this CTA have
-// landed, and add them up in rank order into res[0..d) -- the same order everywhere, so every CTA holds the
-// same bits.  No cluster-wide barrier: a CTA waits only for data, one way.  The two halves of cpart
+// landed, and add them up in rank order -- the same order everywhere, so every CTA holds the
+// same bits and hands each sum to `post(j, sum)`.  No cluster-wide barrier: a CTA waits only for data, one way.  The two halves of cpart
 // alternate between passes; a neighbour can be at most one pass ahead (it needs this CTA's sums of the
 // pass before), so what it sends lands in the half this CTA is not reading.  Returns false when the wait
 // ran out (uniform over the CTA).
-__device__ bool exchange_cols(const float* part, int groups, int d, float* cpart, uint64_t* bar, uint32_t parity,
-                              float* res, uint32_t rank) {
+template <class Post>
+__device__ __forceinline__ bool exchange_cols(const float* part, int groups, int d, float* cpart, uint64_t* bar, uint32_t parity,
+                                              Post post, uint32_t rank) {
   const int tid = threadIdx.x;
   if (tid == 0)
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_u32(bar)), "r"((uint32_t)(SM_CL * d * 4)) : "memory");
@@ -78,7 +79,7 @@ __device__ bool exchange_cols(const float* part, int groups, int d, float* cpart
       float acc = 0.f;
 #pragma unroll
       for (int r = 0; r < SM_CL; ++r) acc += cpart[r * SM_MAXD + j];
-      res[j] = acc;
+      post(j, acc);     // what the caller does with column j's sum (it owns index j of every vector until the barrier)
     }
   return __syncthreads_or(!done) == 0;
 }
@@ -107,9 +108,10 @@ __device__ __forceinline__ float vdot(const float* a, const float* b, int d, flo
 // sum_i coef_i x_ij, reduced over the cluster into res[0..d) (identical in every CTA).
 //   kind 0: gradient coefficients at `wv`;  kind 1: HVP coefficients curv_i * (x_i . dir);
 //   kind 2: HVP coefficients with the curvature taken at `wv` on the fly (a stored iterate of the unrolled loop)
-__device__ bool pass(const float* Xs, const float* ys, const float* curv, int rows, int d, int family, float inv_n,
-                     int kind, const float* wv, const float* dir, float* coef, float* part, float* cpart, uint64_t* bar,
-                     uint32_t parity, float* res, uint32_t rank) {
+template <class Post>
+__device__ __forceinline__ bool pass(const float* Xs, const float* ys, const float* curv, int rows, int d, int family, float inv_n,
+                                     int kind, const float* wv, const float* dir, float* coef, float* part, float* cpart,
+                                     uint64_t* bar, uint32_t parity, Post post, uint32_t rank) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // A: one warp per row, four rows in flight per warp so that the shuffle chains overlap
   const float* vv = kind == 0 ? wv : dir;
@@ -158,7 +160,7 @@ __device__ bool pass(const float* Xs, const float* ys, const float* curv, int ro
     part[rg * SM_PS + j] = a;
   }
   __syncthreads();
-  return exchange_cols(part, groups, d, cpart, bar, parity, res, rank);
+  return exchange_cols(part, groups, d, cpart, bar, parity, post, rank);
 }
 
 // Column sums over the rows of one warp (TPR threads per row, so 32 / TPR rows; lane bits >= TPR select the
@@ -200,10 +202,10 @@ template <int TPR> struct ColsLeft { static constexpr int value = 8 / RowsPerWar
 // rows; shared memory is touched only for the 32 per-warp column sums.
 //   x8: this thread's eight columns of its row; yv: the row's label (kind 0) or curvature (kind 1); has: row exists;
 //   wt: the iterate the curvature is taken at (kind 2)
-template <int TPR>
+template <int TPR, class Post>
 __device__ __forceinline__ bool pass_reg(const float (&x8)[8], float yv, bool has, int family, float inv_n, int kind,
                                          const float* vv, const float* wt, float* part, float* cpart, uint64_t* bar,
-                                         uint32_t parity, float* res, uint32_t rank) {
+                                         uint32_t parity, Post post, uint32_t rank) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int d = 8 * TPR;
   const int c8 = tid & (TPR - 1);
@@ -236,19 +238,20 @@ __device__ __forceinline__ bool pass_reg(const float (&x8)[8], float yv, bool ha
     for (int i = 0; i < ColsLeft<TPR>::value; ++i) part[warp * SM_PS + 8 * c8 + off + i] = col[i];
   }
   __syncthreads();
-  return exchange_cols(part, SM_T / 32, d, cpart, bar, parity, res, rank);
+  return exchange_cols(part, SM_T / 32, d, cpart, bar, parity, post, rank);
 }
 // dispatch on the threads per row
+template <class Post>
 __device__ __forceinline__ bool pass_reg_any(int tpr, const float (&x8)[8], float yv, bool has, int family, float inv_n, int kind,
                                              const float* vv, const float* wt, float* part, float* cpart, uint64_t* bar,
-                                             uint32_t parity, float* res, uint32_t rank) {
+                                             uint32_t parity, Post post, uint32_t rank) {
   switch (tpr) {
-    case 1: return pass_reg<1>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
-    case 2: return pass_reg<2>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
-    case 4: return pass_reg<4>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
-    case 8: return pass_reg<8>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
-    case 16: return pass_reg<16>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
-    default: return pass_reg<32>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, res, rank);
+    case 1: return pass_reg<1>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, post, rank);
+    case 2: return pass_reg<2>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, post, rank);
+    case 4: return pass_reg<4>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, post, rank);
+    case 8: return pass_reg<8>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, post, rank);
+    case 16: return pass_reg<16>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, post, rank);
+    default: return pass_reg<32>(x8, yv, has, family, inv_n, kind, vv, wt, part, cpart, bar, parity, post, rank);
   }
 }
 
@@ -318,52 +321,50 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   // or over the validation rows (gradient of the upper loss at vv)
   uint32_t ph = 0;   // bit b: parity of the phase half b waits for next
   bool alive = true; // false once a wait for the neighbours ran out: the loops stop and the status is recorded
-  auto train_pass = [&](int kind, const float* vv, float* res, const float* wt = nullptr) {
+  // `post(j, sum)` receives column j's sum in the thread that owns index j of every vector until the pass's last barrier
+  auto train_pass = [&](int kind, const float* vv, const float* wt, auto post) {
     float* cp = cpart + pb * SM_CL * SM_MAXD;
     const uint32_t par = (ph >> pb) & 1u;
     bool ok;
-    if (regs) ok = pass_reg_any(d >> 3, x8, kind == 0 ? yreg : curvreg, has, a.family, inv_n, kind, vv, wt, part, cp, &xbar[pb], par, res, rank);
-    else ok = pass(Xs, ys, curv, rows, d, a.family, inv_n, kind, kind == 2 ? wt : vv, vv, coef, part, cp, &xbar[pb], par, res, rank);
+    if (regs) ok = pass_reg_any(d >> 3, x8, kind == 0 ? yreg : curvreg, has, a.family, inv_n, kind, vv, wt, part, cp, &xbar[pb], par, post, rank);
+    else ok = pass(Xs, ys, curv, rows, d, a.family, inv_n, kind, kind == 2 ? wt : vv, vv, coef, part, cp, &xbar[pb], par, post, rank);
     alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
   };
   auto valid_pass = [&](const float* vv, float* res) {
     float* cp = cpart + pb * SM_CL * SM_MAXD;
     const uint32_t par = (ph >> pb) & 1u;
+    auto post = [res](int j, float sum) { res[j] = sum; };
     bool ok;
-    if (regs) ok = pass_reg_any(d >> 3, xv8, yvreg, hasv, a.family_up, inv_nv, 0, vv, nullptr, part, cp, &xbar[pb], par, res, rank);
-    else ok = pass(Xvs, yvs, nullptr, rowsv, d, a.family_up, inv_nv, 0, vv, nullptr, coef, part, cp, &xbar[pb], par, res, rank);
+    if (regs) ok = pass_reg_any(d >> 3, xv8, yvreg, hasv, a.family_up, inv_nv, 0, vv, nullptr, part, cp, &xbar[pb], par, post, rank);
+    else ok = pass(Xvs, yvs, nullptr, rowsv, d, a.family_up, inv_nv, 0, vv, nullptr, coef, part, cp, &xbar[pb], par, post, rank);
     alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
   };
 
   if (a.mode == 0) {
-    for (int s = 0; s < a.n_steps && alive; ++s) {
-      train_pass(0, w, g);
-      for (int j = tid; j < d; j += SM_T) w[j] -= a.lr * (g[j] + lam[j] * w[j]);
-      __syncthreads();
-    }
+    const float lr = a.lr;
+    for (int s = 0; s < a.n_steps && alive; ++s)
+      train_pass(0, w, nullptr, [=](int j, float gsum) { w[j] -= lr * (gsum + lam[j] * w[j]); });
     if (rank == 0)
       for (int j = tid; j < d; j += SM_T) a.w[j] = w[j];
   } else if (a.mode == 2) {
     // ITD-RMAD (Sec. 3.2, iterative differentiation): the unrolled steps with every iterate kept on chip,
     // then the reverse sweep  out <- out - lr w_t .* a,  a <- a - lr (H(w_t) a + lam .* a)  for t = T-1 ... 0,
     // one pass per reverse step (both row dot products, x.w_t for the curvature and x.a, in the same pass)
+    const float lr = a.lr;
     for (int s = 0; s < a.n_steps && alive; ++s) {
-      for (int j = tid; j < d; j += SM_T) traj[(size_t)s * d + j] = w[j];
-      train_pass(0, w, g);
-      for (int j = tid; j < d; j += SM_T) w[j] -= a.lr * (g[j] + lam[j] * w[j]);
-      __syncthreads();
+      float* ws = traj + (size_t)s * d;
+      train_pass(0, w, nullptr, [=](int j, float gsum) { const float wj = w[j]; ws[j] = wj; w[j] = wj - lr * (gsum + lam[j] * wj); });
     }
     valid_pass(w, v);                                  // a = dC_upper/dw at w_T
     for (int j = tid; j < d; j += SM_T) q[j] = 0.f;    // the upper cost has no direct dependence on lam
     __syncthreads();
     for (int s = a.n_steps - 1; s >= 0 && alive; --s) {
       const float* wt = traj + (size_t)s * d;
-      train_pass(2, v, h, wt);
-      for (int j = tid; j < d; j += SM_T) {
-        q[j] -= a.lr * (wt[j] * v[j]);
-        v[j] -= a.lr * (h[j] + lam[j] * v[j]);
-      }
-      __syncthreads();
+      train_pass(2, v, wt, [=](int j, float hsum) {
+        const float aj = v[j];
+        q[j] -= lr * (wt[j] * aj);
+        v[j] = aj - lr * (hsum + lam[j] * aj);
+      });
     }
     if (rank == 0)
       for (int j = tid; j < d; j += SM_T) { a.out[j] = q[j]; a.w[j] = w[j]; }
@@ -407,12 +408,11 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
         for (int j = tid; j < d; j += SM_T) { t[j] = v[j]; q[j] = v[j]; }
         __syncthreads();
         for (int k = 0; k < a.K && alive; ++k) {
-          train_pass(1, t, h);
-          for (int j = tid; j < d; j += SM_T) {
-            const float tn = t[j] - a.alpha * (h[j] + lam[j] * t[j]);
+          const float alpha = a.alpha;
+          train_pass(1, t, nullptr, [=](int j, float hsum) {
+            const float tn = t[j] - alpha * (hsum + lam[j] * t[j]);
             t[j] = tn; q[j] += tn;
-          }
-          __syncthreads();
+          });
         }
         qscale = a.alpha;
       } else {
@@ -425,10 +425,8 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
         bool active = rho > stop;
         if (!isfinite(rho)) { status = BETTY_ERR_NONFINITE; active = false; }
         for (int k = 0; k < a.K && active; ++k) {
-          train_pass(1, p, h);
+          train_pass(1, p, nullptr, [=](int j, float hsum) { h[j] = hsum + lam[j] * p[j]; });
           if (!alive) break;
-          for (int j = tid; j < d; j += SM_T) h[j] += lam[j] * p[j];
-          __syncthreads();
           const float gamma = vdot(p, h, d, red);
           if (!isfinite(gamma)) { status = BETTY_ERR_NONFINITE; break; }
           if (!(gamma > 0.f)) { status = BETTY_ERR_BREAKDOWN; break; }
