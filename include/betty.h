@@ -210,7 +210,8 @@ betty_status betty_hypergrad_fd(const betty_level* lower, const betty_level* upp
 
 /* Iterative differentiation with reverse-mode autodiff (ITD-RMAD, Sec. 3.2; the method of the original
  * Meta-Weight-Net in Sec. 5.1): takes n_steps unrolled lower steps from the current lower parameters
- * (they are left at the last iterate, the earlier ones are kept in ws), then differentiates the
+ * (they are left at the last iterate; the earlier ones are kept in ws, or on chip where a small
+ * logistic / least-squares problem and its iterates fit there), then differentiates the
  * upper cost through those steps in reverse:  a = dC_upper/d(lower) at the last iterate; for
  * t = T-1..0: out -= lr * M_t^T a, a -= lr * H_t a.  out[wrt->n_params] also receives the direct
  * gradient.  ws must hold n_steps parameter vectors in addition to betty_workspace_size(). */
