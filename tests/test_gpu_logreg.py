@@ -126,6 +126,25 @@ def test_on_chip_whole_loop_kernel_matches_oracle(bt, n, d, nv):
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
 
+@pytest.mark.parametrize("n,d,nv", [(1024, 64, 256), (999, 50, 77)])
+def test_on_chip_kernel_is_bitwise_repeatable(bt, n, d, nv):
+    """Every CTA of the cluster adds the same column sums in the same order, so two runs from the
+    same state give the same bits (register form and shared-memory form)."""
+    inp = si.logreg_bilevel(4242, n, d, nv)
+    outs = []
+    for _ in range(2):
+        (w, lam), _o = _pair(inp)
+        ws = bt.Workspace([w, lam], extra_bytes=41 * (d + 64) * 4)
+        bt.betty_lower_step(w, 25, ws)
+        a, b, c = _vec(d), _vec(d), _vec(d)
+        bt.betty_hypergrad_cg(w, lam, lam, 5, 0.0, a, ws)
+        bt.betty_hypergrad_neumann(w, lam, lam, 5, 0.05, b, ws)
+        bt.betty_hypergrad_itd(w, lam, lam, 40, c, ws)
+        outs.append((w.params.clone(), a, b, c))
+    for x, y in zip(*outs):
+        assert torch.equal(x, y)
+
+
 def test_cg_early_stop_counts_iterations_like_the_oracle(bt):
     from tests import cuda_build as cb
     inp = si.logreg_bilevel(5, 400, 16, 100)
