@@ -86,22 +86,24 @@ __device__ __forceinline__ bool exchange_cols(const float* part, int groups, int
 
 __device__ __forceinline__ float sigm(float t) { return 1.f / (1.f + expf(-t)); }
 
-// block-wide sum of one value per thread (fixed order)
-__device__ __forceinline__ float block_sum_f(float v, float* sh) {
+// Sum over j < d <= SM_MAXD of one term per thread (thread j holds term j), the same value in every thread
+// (fixed order): only the first ceil(d / 32) warps hold terms, so only their partial sums are formed and added
+__device__ __forceinline__ float vsum(float term, int d, float* sh) {
+  const int tid = threadIdx.x, nw = (d + 31) >> 5;
+  if ((tid >> 5) < nw) {
+    float v = tid < d ? term : 0.f;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((tid & 31) == 0) sh[tid >> 5] = v;
+  }
   __syncthreads();
   float t = 0.f;
-#pragma unroll
-  for (int i = 0; i < SM_T / 32; ++i) t += sh[i];
+  for (int i = 0; i < nw; ++i) t += sh[i];
   __syncthreads();
   return t;
 }
 __device__ __forceinline__ float vdot(const float* a, const float* b, int d, float* sh) {
-  float v = 0.f;
-  for (int j = threadIdx.x; j < d; j += SM_T) v += a[j] * b[j];
-  return block_sum_f(v, sh);
+  return vsum(threadIdx.x < d ? a[threadIdx.x] * b[threadIdx.x] : 0.f, d, sh);
 }
 
 // One pass over this CTA's resident rows: coef_i from the row dot products, then the column sums
@@ -431,9 +433,13 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
           if (!isfinite(gamma)) { status = BETTY_ERR_NONFINITE; break; }
           if (!(gamma > 0.f)) { status = BETTY_ERR_BREAKDOWN; break; }
           const float al = rho / gamma;
-          for (int j = tid; j < d; j += SM_T) { q[j] += al * p[j]; r[j] -= al * h[j]; }
-          __syncthreads();
-          const float rho_new = vdot(r, r, d, red);
+          float rr = 0.f;
+          if (tid < d) {
+            q[tid] += al * p[tid];
+            const float rn = r[tid] - al * h[tid];
+            r[tid] = rn; rr = rn * rn;
+          }
+          const float rho_new = vsum(rr, d, red);
           const float beta = rho_new / rho;
           for (int j = tid; j < d; j += SM_T) p[j] = r[j] + beta * p[j];
           __syncthreads();
