@@ -171,9 +171,9 @@ __device__ __forceinline__ bool pass(const float* Xs, const float* ys, const flo
 // half -- costs 4 + 2 + 1 shuffles for eight values where a plain butterfly costs 8 per round; shuffle issue
 // (one warp-wide shuffle per clock per SM, 32 warps) is what the pass spends most of its time on.
 // On return col[0 .. NF) are the sums of columns 8 c8 + off + i; `writer` is false in lanes holding duplicates.
-template <int O, int N>
+template <int O, int N, int NV = 8>
 struct WarpColumnSum {
-  static __device__ __forceinline__ void run(float (&col)[8], int lane, int& off, bool& writer) {
+  static __device__ __forceinline__ void run(float (&col)[NV], int lane, int& off, bool& writer) {
     if constexpr (O < 32) {
       const bool up = (lane & O) != 0;
       if constexpr (N > 1) {
@@ -185,11 +185,11 @@ struct WarpColumnSum {
           col[i] = keep + __shfl_xor_sync(0xffffffffu, send, O);
         }
         if (up) off += H;
-        WarpColumnSum<O * 2, H>::run(col, lane, off, writer);
+        WarpColumnSum<O * 2, H, NV>::run(col, lane, off, writer);
       } else {
         col[0] += __shfl_xor_sync(0xffffffffu, col[0], O);
         if (up) writer = false;
-        WarpColumnSum<O * 2, 1>::run(col, lane, off, writer);
+        WarpColumnSum<O * 2, 1, NV>::run(col, lane, off, writer);
       }
     }
   }
@@ -463,6 +463,82 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   cluster_barrier();
 }
 
+// The unrolled lower steps alone, rows in registers with sixteen columns per thread: TPR = d / 16 threads per
+// row on 512 threads (the 1024 x 64 problem: 128 rows of 4 threads per CTA).  Against the 1024-thread form
+// above this halves the warps per scheduler and the warp instructions per pass, which is what a pass is
+// bound by; the other modes keep the 8-column form (they hold the validation rows as well).
+static constexpr int SW_T = 512;
+template <int TPR>
+__global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SW_T, 1) k_logreg_small_steps(SmallArgs a) {
+  __shared__ __align__(16) float w[SM_MAXD];
+  __shared__ __align__(16) float lam[SM_MAXD];
+  __shared__ __align__(16) float part[(SW_T / 32) * SM_PS];
+  __shared__ float cpart[2 * SM_CL * SM_MAXD];
+  __shared__ __align__(8) uint64_t xbar[2];
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  constexpr int d = 16 * TPR;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int R = a.rows_per_cta, row = tid / TPR, c16 = tid & (TPR - 1);
+  const int64_t r0 = (int64_t)rank * R;
+  int rows = (int)(a.n - r0 < R ? a.n - r0 : R); if (rows < 0) rows = 0;
+  const bool has = row < rows;
+  float x[16];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) x[k] = 0.f;
+  float yv = 0.f;
+  if (has) {
+    const float4* src = (const float4*)(a.X + (r0 + row) * d + 16 * c16);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { const float4 t = src[k]; x[4 * k] = t.x; x[4 * k + 1] = t.y; x[4 * k + 2] = t.z; x[4 * k + 3] = t.w; }
+    yv = a.y[r0 + row];
+  }
+  for (int j = tid; j < d; j += SW_T) { w[j] = a.w[j]; lam[j] = a.lam[j]; }
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_u32(&xbar[0])));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_u32(&xbar[1])));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  cluster_barrier();    // every CTA of the cluster is running, its barriers set up, before anyone sends to it
+  const float inv_n = a.n > 0 ? 1.f / (float)a.n : 0.f, lr = a.lr;
+  const int family = a.family;
+  float* wp = w; float* lp = lam;
+  int pb = 0; uint32_t ph = 0; bool alive = true;
+  for (int s = 0; s < a.n_steps && alive; ++s) {
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float4 v = *(const float4*)(w + 16 * c16 + 4 * k);
+      s0 += x[4 * k] * v.x + x[4 * k + 1] * v.y;
+      s1 += x[4 * k + 2] * v.z + x[4 * k + 3] * v.w;
+    }
+    float sdot = s0 + s1;
+#pragma unroll
+    for (int o = TPR >> 1; o > 0; o >>= 1) sdot += __shfl_xor_sync(0xffffffffu, sdot, o);
+    float cf = 0.f;
+    if (has) cf = family == 0 ? -yv * sigm(-yv * sdot) * inv_n : (sdot - yv);
+    float col[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) col[k] = cf * x[k];
+    int off = 0;
+    bool writer = true;
+    WarpColumnSum<TPR, 16, 16>::run(col, lane, off, writer);
+    constexpr int NF = 16 / (32 / TPR) > 0 ? 16 / (32 / TPR) : 1;
+    if (writer) {
+#pragma unroll
+      for (int i = 0; i < NF; ++i) part[warp * SM_PS + 16 * c16 + off + i] = col[i];
+    }
+    __syncthreads();
+    const bool ok = exchange_cols(part, SW_T / 32, d, cpart + pb * SM_CL * SM_MAXD, &xbar[pb], (ph >> pb) & 1u,
+                                  [=](int j, float gsum) { wp[j] -= lr * (gsum + lp[j] * wp[j]); }, rank);
+    alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
+  }
+  if (rank == 0)
+    for (int j = tid; j < d; j += SW_T) a.w[j] = w[j];
+  if (!alive && tid == 0) record_status(a.sb, BETTY_ERR_TIMEOUT);
+  cluster_barrier();    // no CTA may leave while a neighbour can still send to it
+}
+
 static size_t small_smem_bytes(int R, int Rv, int d, int64_t traj_floats) {
   size_t floats = (size_t)R * d + (size_t)Rv * d + R + Rv + R + (R > Rv ? R : Rv) + (size_t)SM_NVEC * SM_MAXD + 32 * SM_PS +
                   2 * SM_CL * SM_MAXD + 32 + (size_t)traj_floats;
@@ -486,6 +562,17 @@ static betty_status launch_small(Ctx& c, SmallArgs& a) {
     const bool pow2 = d >= 8 && d <= SM_MAXD && (d & (d - 1)) == 0;
     a.in_regs = pow2 && a.rows_per_cta <= SM_T / tpr && a.rows_per_cta_v <= SM_T / tpr &&
                 (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && (a.mode == 0 || (reinterpret_cast<uintptr_t>(a.Xv) & 15) == 0);
+  }
+  if (a.mode == 0 && a.in_regs && a.d >= 16 && a.rows_per_cta <= SW_T / (a.d >> 4)) {
+    switch (a.d >> 4) {
+      case 1: k_logreg_small_steps<1><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
+      case 2: k_logreg_small_steps<2><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
+      case 4: k_logreg_small_steps<4><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
+      case 8: k_logreg_small_steps<8><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
+      default: k_logreg_small_steps<16><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
+    }
+    BETTY_LAUNCH_CHECK();
+    return BETTY_OK;
   }
   const size_t smem = small_smem_bytes(a.rows_per_cta, a.rows_per_cta_v, a.d, a.mode == 2 ? (int64_t)a.n_steps * a.d : 0);
   static size_t attr_bytes = 0;
