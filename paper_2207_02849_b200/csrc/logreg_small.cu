@@ -463,13 +463,14 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   cluster_barrier();
 }
 
-// The unrolled lower steps alone, rows in registers with sixteen columns per thread: TPR = d / 16 threads per
-// row on 512 threads (the 1024 x 64 problem: 128 rows of 4 threads per CTA).  Against the 1024-thread form
-// above this halves the warps per scheduler and the warp instructions per pass, which is what a pass is
-// bound by; the other modes keep the 8-column form (they hold the validation rows as well).
-static constexpr int SW_T = 512;
-template <int TPR>
-__global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SW_T, 1) k_logreg_small_steps(SmallArgs a) {
+// The unrolled lower steps alone, rows in registers with CPT = 16 or 32 columns per thread: TPR = d / CPT threads
+// per row on 8192 / CPT threads (the 1024 x 64 problem: 128 rows of 2 threads per CTA at CPT = 32).  Against
+// the 1024-thread, 8-column form above this leaves a half or a quarter of the warps per scheduler and 60% or
+// half of the warp instructions per pass, which is what a pass is bound by (1.235 -> 0.943 -> 0.785 us per
+// pass); the other modes keep the 8-column form (they hold the validation rows as well).
+template <int TPR, int CPT>
+__global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(8192 / CPT, 1) k_logreg_small_steps(SmallArgs a) {
+  constexpr int SW_T = 8192 / CPT;   // 512 threads at 16 columns per thread, 256 at 32
   __shared__ __align__(16) float w[SM_MAXD];
   __shared__ __align__(16) float lam[SM_MAXD];
   __shared__ __align__(16) float part[(SW_T / 32) * SM_PS];
@@ -477,20 +478,20 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SW_T, 1) k_logre
   __shared__ __align__(8) uint64_t xbar[2];
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
-  constexpr int d = 16 * TPR;
+  constexpr int d = CPT * TPR;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int R = a.rows_per_cta, row = tid / TPR, c16 = tid & (TPR - 1);
   const int64_t r0 = (int64_t)rank * R;
   int rows = (int)(a.n - r0 < R ? a.n - r0 : R); if (rows < 0) rows = 0;
   const bool has = row < rows;
-  float x[16];
+  float x[CPT];
 #pragma unroll
-  for (int k = 0; k < 16; ++k) x[k] = 0.f;
+  for (int k = 0; k < CPT; ++k) x[k] = 0.f;
   float yv = 0.f;
   if (has) {
-    const float4* src = (const float4*)(a.X + (r0 + row) * d + 16 * c16);
+    const float4* src = (const float4*)(a.X + (r0 + row) * d + CPT * c16);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) { const float4 t = src[k]; x[4 * k] = t.x; x[4 * k + 1] = t.y; x[4 * k + 2] = t.z; x[4 * k + 3] = t.w; }
+    for (int k = 0; k < CPT / 4; ++k) { const float4 t = src[k]; x[4 * k] = t.x; x[4 * k + 1] = t.y; x[4 * k + 2] = t.z; x[4 * k + 3] = t.w; }
     yv = a.y[r0 + row];
   }
   for (int j = tid; j < d; j += SW_T) { w[j] = a.w[j]; lam[j] = a.lam[j]; }
@@ -507,8 +508,8 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SW_T, 1) k_logre
   for (int s = 0; s < a.n_steps && alive; ++s) {
     float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float4 v = *(const float4*)(w + 16 * c16 + 4 * k);
+    for (int k = 0; k < CPT / 4; ++k) {
+      const float4 v = *(const float4*)(w + CPT * c16 + 4 * k);
       s0 += x[4 * k] * v.x + x[4 * k + 1] * v.y;
       s1 += x[4 * k + 2] * v.z + x[4 * k + 3] * v.w;
     }
@@ -517,16 +518,16 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SW_T, 1) k_logre
     for (int o = TPR >> 1; o > 0; o >>= 1) sdot += __shfl_xor_sync(0xffffffffu, sdot, o);
     float cf = 0.f;
     if (has) cf = family == 0 ? -yv * sigm(-yv * sdot) * inv_n : (sdot - yv);
-    float col[16];
+    float col[CPT];
 #pragma unroll
-    for (int k = 0; k < 16; ++k) col[k] = cf * x[k];
+    for (int k = 0; k < CPT; ++k) col[k] = cf * x[k];
     int off = 0;
     bool writer = true;
-    WarpColumnSum<TPR, 16, 16>::run(col, lane, off, writer);
-    constexpr int NF = 16 / (32 / TPR) > 0 ? 16 / (32 / TPR) : 1;
+    WarpColumnSum<TPR, CPT, CPT>::run(col, lane, off, writer);
+    constexpr int NF = CPT / (32 / TPR) > 0 ? CPT / (32 / TPR) : 1;
     if (writer) {
 #pragma unroll
-      for (int i = 0; i < NF; ++i) part[warp * SM_PS + 16 * c16 + off + i] = col[i];
+      for (int i = 0; i < NF; ++i) part[warp * SM_PS + CPT * c16 + off + i] = col[i];
     }
     __syncthreads();
     const bool ok = exchange_cols(part, SW_T / 32, d, cpart + pb * SM_CL * SM_MAXD, &xbar[pb], (ph >> pb) & 1u,
@@ -563,13 +564,23 @@ static betty_status launch_small(Ctx& c, SmallArgs& a) {
     a.in_regs = pow2 && a.rows_per_cta <= SM_T / tpr && a.rows_per_cta_v <= SM_T / tpr &&
                 (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && (a.mode == 0 || (reinterpret_cast<uintptr_t>(a.Xv) & 15) == 0);
   }
-  if (a.mode == 0 && a.in_regs && a.d >= 16 && a.rows_per_cta <= SW_T / (a.d >> 4)) {
+  if (a.mode == 0 && a.in_regs && a.d >= 32 && a.rows_per_cta <= 256 / (a.d >> 5)) {
+    switch (a.d >> 5) {
+      case 1: k_logreg_small_steps<1, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
+      case 2: k_logreg_small_steps<2, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
+      case 4: k_logreg_small_steps<4, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
+      default: k_logreg_small_steps<8, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
+    }
+    BETTY_LAUNCH_CHECK();
+    return BETTY_OK;
+  }
+  if (a.mode == 0 && a.in_regs && a.d >= 16 && a.rows_per_cta <= 512 / (a.d >> 4)) {
     switch (a.d >> 4) {
-      case 1: k_logreg_small_steps<1><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
-      case 2: k_logreg_small_steps<2><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
-      case 4: k_logreg_small_steps<4><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
-      case 8: k_logreg_small_steps<8><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
-      default: k_logreg_small_steps<16><<<SM_CL, SW_T, 0, c.stream>>>(a); break;
+      case 1: k_logreg_small_steps<1, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
+      case 2: k_logreg_small_steps<2, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
+      case 4: k_logreg_small_steps<4, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
+      case 8: k_logreg_small_steps<8, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
+      default: k_logreg_small_steps<16, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
     }
     BETTY_LAUNCH_CHECK();
     return BETTY_OK;
