@@ -463,11 +463,12 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(SM_T, 1) k_logre
   cluster_barrier();
 }
 
-// The unrolled lower steps alone, rows in registers with CPT = 16 or 32 columns per thread: TPR = d / CPT threads
-// per row on 8192 / CPT threads (the 1024 x 64 problem: 128 rows of 2 threads per CTA at CPT = 32).  Against
-// the 1024-thread, 8-column form above this leaves a half or a quarter of the warps per scheduler and 60% or
-// half of the warp instructions per pass, which is what a pass is bound by (1.235 -> 0.943 -> 0.785 us per
-// pass); the other modes keep the 8-column form (they hold the validation rows as well).
+// The unrolled lower steps alone, rows in registers with CPT = 16, 32 or 64 columns per thread: TPR = d / CPT
+// threads per row on 8192 / CPT threads (the 1024 x 64 problem: one thread per row, 128 threads per CTA).
+// Against the 1024-thread, 8-column form above this leaves 4, 2 or 1 warps per scheduler instead of 8 and
+// 60% to half of the warp instructions per pass, which is what a pass is bound by (1.235 -> 0.943 -> 0.785 ->
+// 0.749 us per pass on that problem); the other modes keep the 8-column form (they hold the validation rows
+// as well).  The block must have at least d threads: the fold and the gather take one column per thread.
 template <int TPR, int CPT>
 __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(8192 / CPT, 1) k_logreg_small_steps(SmallArgs a) {
   constexpr int SW_T = 8192 / CPT;   // 512 threads at 16 columns per thread, 256 at 32
@@ -564,23 +565,15 @@ static betty_status launch_small(Ctx& c, SmallArgs& a) {
     a.in_regs = pow2 && a.rows_per_cta <= SM_T / tpr && a.rows_per_cta_v <= SM_T / tpr &&
                 (reinterpret_cast<uintptr_t>(a.X) & 15) == 0 && (a.mode == 0 || (reinterpret_cast<uintptr_t>(a.Xv) & 15) == 0);
   }
-  if (a.mode == 0 && a.in_regs && a.d >= 32 && a.rows_per_cta <= 256 / (a.d >> 5)) {
-    switch (a.d >> 5) {
-      case 1: k_logreg_small_steps<1, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
-      case 2: k_logreg_small_steps<2, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
-      case 4: k_logreg_small_steps<4, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
-      default: k_logreg_small_steps<8, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
-    }
-    BETTY_LAUNCH_CHECK();
-    return BETTY_OK;
-  }
-  if (a.mode == 0 && a.in_regs && a.d >= 16 && a.rows_per_cta <= 512 / (a.d >> 4)) {
-    switch (a.d >> 4) {
-      case 1: k_logreg_small_steps<1, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
-      case 2: k_logreg_small_steps<2, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
-      case 4: k_logreg_small_steps<4, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
-      case 8: k_logreg_small_steps<8, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
-      default: k_logreg_small_steps<16, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
+  if (a.mode == 0 && a.in_regs && a.d >= 16) {
+    // the widest form whose threads still cover the d columns in the fold and the gather (in_regs: at most
+    // 8192 / d rows per CTA, which is the row capacity of every form)
+    switch (a.d) {
+      case 16: k_logreg_small_steps<1, 16><<<SM_CL, 512, 0, c.stream>>>(a); break;
+      case 32: k_logreg_small_steps<1, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;
+      case 64: k_logreg_small_steps<1, 64><<<SM_CL, 128, 0, c.stream>>>(a); break;
+      case 128: k_logreg_small_steps<2, 64><<<SM_CL, 128, 0, c.stream>>>(a); break;
+      default: k_logreg_small_steps<8, 32><<<SM_CL, 256, 0, c.stream>>>(a); break;   // d = 256
     }
     BETTY_LAUNCH_CHECK();
     return BETTY_OK;

@@ -94,12 +94,15 @@ def test_hypergradients_match_oracle(bt, n, d, nv, steps, K):
 
 
 @pytest.mark.parametrize("n,d,nv", [(5, 8, 3), (1000, 50, 77), (777, 256, 100), (64, 33, 9), (2048, 128, 512),
-                                    (999, 64, 77), (200, 256, 40), (300, 16, 10), (40, 32, 3), (1025, 64, 256)])
+                                    (999, 64, 77), (200, 256, 40), (300, 16, 10), (40, 32, 3), (1025, 64, 256),
+                                    (500, 128, 40), (1000, 128, 64), (3000, 32, 100)])
 def test_on_chip_whole_loop_kernel_matches_oracle(bt, n, d, nv):
     """Problems that fit a cluster's shared memory run each loop (all lower steps; a whole
     hypergradient) in one launch; ragged row counts, CTAs without rows and odd widths included.
     Power-of-two widths with few enough rows per CTA keep the rows in registers (the second line of
-    cases, and the first one); the others, and 1025 x 64 with its 129 rows per CTA, in shared memory."""
+    cases, and the first one); the others, and 1025 x 64 with its 129 rows per CTA, in shared memory.
+    The lower steps hold 64, 32 or 16 columns of a row per thread (widths 64 and 128; 32 and 256; 16), the
+    hypergradient modes 8."""
     from tests import cuda_build as cb
     inp = si.logreg_bilevel(900 + n + d, n, d, nv)
     inp.lam = (np.abs(si.normal_f32(11, 2, (d,))) * 0.05 + 0.01).astype(np.float32)
