@@ -49,6 +49,7 @@ class Level:
     lr: float = 0.1
     mu: float = 0.0
     bf16: bool = False                 # MLP matrices are used through a bf16-rounded copy
+    quant: str = "operands"            # what a bf16 level rounds: "operands" | "weights" (see _mlp_ce_state)
     constraints: list = field(default_factory=list)
     optimizer: str = "gd"              # 'gd' | 'momentum' | 'adam' (App. C: SGD with momentum / Adam per problem)
     momentum: float = 0.0
@@ -259,13 +260,30 @@ def _logreg_parts(L, over):
 def _mlp_ce_state(L: Level, over):
     """Forward pass of the classifier that takes part in cost L and the per-sample CE.
 
-    over["frozen"] (a set of level ids) marks the classifier's override as a perturbed
-    evaluation: its parameters are the base compute copy plus the given displacement, and
-    the activations keep the base pass's rounding offsets."""
+    A mixed-precision classifier (Sec. 4 lists mixed precision among the systems features; the
+    paper does not say what is rounded) is evaluated under one of two stated readings:
+
+    quant = "weights"   the plain reading.  The matrices are rounded to bf16 once per evaluation
+                        of the cost; nothing else is rounded.  A finite-difference evaluation
+                        (Sec. 3.2, AID-FD) displaces the fp64 master copy, x +- eps v, and uses
+                        it as it is, with no rounding at all.
+    quant = "operands"  every matrix product takes bf16 operands: the matrices and each hidden
+                        activation are rounded.  A finite-difference evaluation displaces the
+                        rounded matrices and keeps the base pass's rounding offsets of the hidden
+                        activations (rounding is treated as the identity under differentiation).
+
+    over["frozen"] (a set of level ids) marks the classifier's override as such a perturbed
+    evaluation."""
     M = _find(L, "mlp")
     flat = _p(M, over)
     frozen = over is not None and id(M) in over.get("frozen", ())
-    if frozen and M.bf16:
+    if M.bf16 and M.quant not in ("operands", "weights"):
+        raise ValueError(M.quant)
+    plain = M.bf16 and M.quant == "weights"
+    if frozen and plain:
+        Ws, bs = mlp_unpack(M.widths, flat)
+        h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation)
+    elif frozen and M.bf16:
         Wb, bb = _mlp_weights(M, M.params)
         _, _, offs = _mlp_forward(Wb, bb, L.X, M.activation, quant=True)
         Wd, bd = mlp_unpack(M.widths, flat - M.params)
@@ -274,7 +292,7 @@ def _mlp_ce_state(L: Level, over):
         h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation, offsets=offs)
     else:
         Ws, bs = _mlp_weights(M, flat)
-        h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation, quant=M.bf16)
+        h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation, quant=M.bf16 and not plain)
     p, ell = _softmax_ce(a[-1], np.asarray(L.y, dtype=np.int64))
     return M, Ws, bs, h, a, p, ell
 

@@ -14,8 +14,10 @@ weights).  Readings where the paper is silent:
     norm has fallen to tol*|v|, or (status "breakdown") when a search direction has p^T H p <= 0.
   * FD(eps0, alpha): eps = eps0/|v|_2; result -alpha*[dC/dc(x+eps v) - dC/dc(x-eps v)]/(2 eps),
     i.e. H^{-1} replaced by alpha*I; alpha defaults to 1.  On mixed-precision levels the two
-    perturbed evaluations are not re-quantised: x +- eps v displaces the bf16 compute copy, and
-    the rounding offsets of weights and hidden activations stay at their base-point values.
+    perturbed evaluations are not re-quantised.  Under the plain reading (Level.quant = "weights")
+    x +- eps v is the displaced fp64 master, used unrounded; under the bf16-operand reading
+    (Level.quant = "operands") it displaces the bf16 compute copy, and the rounding offsets of
+    the hidden activations stay at their base-point values.
 """
 from __future__ import annotations
 
@@ -157,8 +159,8 @@ def brj(L: Level, wrt: Level, v, method: str, K: int = 0, alpha: float = 1.0,
         if nv == 0.0:
             return np.zeros(wrt.params.size)
         eps = eps0 / nv
-        # perturbed evaluations keep the base point's bf16 rounding offsets (weights and hidden
-        # activations) frozen; for full-precision levels "frozen" has no effect
+        # "frozen" marks a perturbed evaluation that is not re-quantised (either reading of a
+        # mixed-precision level); for full-precision levels it has no effect
         gp = grad(L, wrt, over={id(L): L.params + eps * v, "frozen": {id(L)}})
         gm = grad(L, wrt, over={id(L): L.params - eps * v, "frozen": {id(L)}})
         return -alpha * (gp - gm) / (2.0 * eps)

@@ -21,21 +21,21 @@ def quadratic_levels(A, b, lam, Av, bv, w0=None):
     return lo, up
 
 
-def reweight_levels(inp, bf16=True):
+def reweight_levels(inp, bf16=True, quant="operands"):
     theta = Level(loss="mlp_ce", param_kind="weightnet", params=inp.theta, X=inp.val.X,
                   y=inp.val.y)
     w = Level(loss="mlp_ce_reweight", param_kind="mlp", params=inp.w, X=inp.train.X,
               y=inp.train.y, widths=inp.widths, activation=inp.activation, lr=inp.lr,
-              bf16=bf16, constraints=[theta])
+              bf16=bf16, quant=quant, constraints=[theta])
     theta.constraints = [w]
     return w, theta
 
 
-def three_levels(inp, bf16=True):
+def three_levels(inp, bf16=True, quant="operands"):
     """P1 classifier, P2 weight net (detector loss on D2), P3 log weight decay (detector
     loss on D3, no mu term)."""
     P1 = Level(loss="mlp_ce_reweight", param_kind="mlp", params=inp.w, X=inp.D1.X, y=inp.D1.y,
-               widths=inp.widths, activation=inp.activation, lr=inp.lr, bf16=bf16)
+               widths=inp.widths, activation=inp.activation, lr=inp.lr, bf16=bf16, quant=quant)
     P2 = Level(loss="weightnet_detect", param_kind="weightnet", params=inp.theta, X=inp.D2.X,
                y=inp.D2.y, aux=inp.D2.clean.astype(np.float64), mu=inp.mu, constraints=[P1])
     P3 = Level(loss="weightnet_detect", param_kind="logwd", params=inp.lam, X=inp.D3.X,

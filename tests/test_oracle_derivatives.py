@@ -351,3 +351,104 @@ def test_fd_on_a_bf16_level_keeps_quantisation_offsets_frozen():
     naive = -(oracle.grad(w16, th16, {id(w16): w16.params + eps * v})
               - oracle.grad(w16, th16, {id(w16): w16.params - eps * v})) / (2 * eps)
     assert rel(naive, f64) > 10 * rel(f16, f64)
+
+
+# ------------------------------------------------------------------ the two readings of a mixed-precision level
+def _q(t):
+    return t.to(torch.float32).to(torch.bfloat16).to(torch.float64)
+
+
+def _theta_gradient_of_reweighted_mean(theta_np, ell):
+    """d/dtheta mean_i sigmoid(net(ell_i)) * ell_i with the per-sample losses as data (autodiff)."""
+    th = _t(theta_np).requires_grad_(True)
+    c = (_torch_weightnet(th, ell.detach()) * ell.detach()).mean()
+    (g,) = torch.autograd.grad(c, [th])
+    return g.numpy()
+
+
+@pytest.mark.parametrize("act", ["relu", "gelu"])
+def test_plain_reading_rounds_the_matrices_only(act):
+    """quant = "weights": the cost sees bf16-rounded matrices and nothing else rounded, and a
+    finite-difference evaluation sees the displaced master with no rounding at all.  Expected values
+    come from a forward-only restatement in torch and reverse-mode autodiff of it."""
+    inp = _tiny_reweight(act, seed=37, widths=(8, 12, 10, 5), B=40)
+    inp.w = inp.w + si.normal_f32(37, 400, inp.w.shape) * 1e-3        # master not bf16-representable
+    w16, th16 = reweight_levels(inp, bf16=True, quant="weights")
+    yt = torch.from_numpy(inp.train.y.astype(np.int64))
+
+    def ell_at(flat, round_matrices):
+        Ws, bs = olv.mlp_unpack(inp.widths, flat)
+        h = _t(inp.train.X)
+        for l, (W, b) in enumerate(zip(Ws, bs)):
+            Wt = _q(_t(W)) if round_matrices else _t(W)
+            a = h @ Wt.T + _t(b)
+            h = _torch_act(act, a) if l < len(Ws) - 1 else a
+        return torch.nn.functional.cross_entropy(h, yt, reduction="none")
+
+    master = inp.w.astype(np.float64)
+    ell = ell_at(master, True)
+    ref = (_torch_weightnet(_t(inp.theta), ell) * ell).mean().item()
+    assert abs(olv.cost(w16) - ref) < 1e-13
+    # it differs from both the unrounded level and the bf16-operand reading
+    assert abs(olv.cost(reweight_levels(inp, bf16=False)[0]) - ref) > 1e-9
+    assert abs(olv.cost(reweight_levels(inp, bf16=True)[0]) - ref) > 1e-9
+    # finite difference: master +- eps v, unrounded
+    v = np.random.default_rng(5).standard_normal(inp.w.size)
+    eps0 = 1e-3
+    eps = eps0 / np.linalg.norm(v)
+    gp = _theta_gradient_of_reweighted_mean(inp.theta, ell_at(master + eps * v, False))
+    gm = _theta_gradient_of_reweighted_mean(inp.theta, ell_at(master - eps * v, False))
+    got = oracle.brj(w16, th16, v, "fd", eps0=eps0, alpha=1.0)
+    assert rel(got, -(gp - gm) / (2 * eps)) < 1e-9
+
+
+@pytest.mark.parametrize("act", ["relu", "gelu"])
+def test_operand_reading_displaces_layer_by_layer_with_frozen_offsets(act):
+    """quant = "operands": in a finite-difference evaluation every hidden activation moves by exactly
+    act(a+) - act(a) from its rounded base value, layer by layer, and the matrices by exactly eps V from
+    their rounded values.  The restatement below carries base and displaced passes side by side and
+    never forms a rounding offset; a wrong sign or a wrong layer index of one offset fails it."""
+    inp = _tiny_reweight(act, seed=41, widths=(8, 12, 10, 9, 5), B=40)
+    inp.w = inp.w + si.normal_f32(41, 400, inp.w.shape) * 1e-3
+    w16, th16 = reweight_levels(inp, bf16=True)
+    yt = torch.from_numpy(inp.train.y.astype(np.int64))
+    master = inp.w.astype(np.float64)
+    v = np.random.default_rng(6).standard_normal(inp.w.size)
+    eps0 = 1e-3
+    eps = eps0 / np.linalg.norm(v)
+    Ws, bs = olv.mlp_unpack(inp.widths, master)
+    Vs, cs = olv.mlp_unpack(inp.widths, v)
+    nl = len(Ws)
+
+    def displaced(sign):
+        hb = hd = _t(inp.train.X)          # base (rounded) and displaced activations
+        acts_b, acts_d = [], []
+        for l in range(nl):
+            Wq = _q(_t(Ws[l]))
+            ab = hb @ Wq.T + _t(bs[l])
+            ad = hd @ (Wq + sign * eps * _t(Vs[l])).T + _t(bs[l]) + sign * eps * _t(cs[l])
+            acts_b.append(ab); acts_d.append(ad)
+            if l < nl - 1:
+                hb_next = _q(_torch_act(act, ab))
+                hd = hb_next + (_torch_act(act, ad) - _torch_act(act, ab))
+                hb = hb_next
+        return acts_b, acts_d
+
+    got_states = {}
+    for sign in (+1.0, -1.0):
+        acts_b, acts_d = displaced(sign)
+        over = {id(w16): master + sign * eps * v, "frozen": {id(w16)}}
+        M, _, _, h, a, p, ell = olv._mlp_ce_state(w16, over)
+        _, _, _, hb, ab, _, _ = olv._mlp_ce_state(w16, None)
+        for l in range(nl):
+            np.testing.assert_allclose(a[l], acts_d[l].numpy(), rtol=0, atol=1e-13)
+            np.testing.assert_allclose(ab[l], acts_b[l].numpy(), rtol=0, atol=1e-13)
+            if l < nl - 1:       # h+- - h_base == act(a+-) - act(a_base), exactly this layer's
+                lhs = h[l + 1] - hb[l + 1]
+                rhs = (_torch_act(act, acts_d[l]) - _torch_act(act, acts_b[l])).numpy()
+                np.testing.assert_allclose(lhs, rhs, rtol=0, atol=1e-15)
+        got_states[sign] = torch.nn.functional.cross_entropy(acts_d[-1], yt, reduction="none")
+    gp = _theta_gradient_of_reweighted_mean(inp.theta, got_states[+1.0])
+    gm = _theta_gradient_of_reweighted_mean(inp.theta, got_states[-1.0])
+    got = oracle.brj(w16, th16, v, "fd", eps0=eps0, alpha=1.0)
+    assert rel(got, -(gp - gm) / (2 * eps)) < 1e-8
