@@ -129,7 +129,7 @@ class LogregWorkload:
     def setup_device(self):
         import torch
         import paper_2207_02849_b200 as bt
-        from tests import cuda_build as cb
+        from paper_2207_02849_b200 import problems as cb
         self.bt, self.torch = bt, torch
         self.w, self.lam = cb.logreg_levels(self.inp)
         self.w0 = self.w.params.clone()
@@ -203,7 +203,7 @@ class LogregWorkload:
     # -- oracle on a bounded sample of the same workload
     def oracle_sample(self, budget_rows: int):
         import oracle
-        from tests import oracle_build as ob
+        from oracle import problems as ob
         import synth_inputs as si
         import copy
         n_s = min(self.n, budget_rows)
@@ -247,7 +247,7 @@ class ReweightWorkload:
     def setup_device(self):
         import torch
         import paper_2207_02849_b200 as bt
-        from tests import cuda_build as cb
+        from paper_2207_02849_b200 import problems as cb
         self.bt, self.torch = bt, torch
         self.w, self.th = cb.reweight_levels(self.inp)
         self.w0 = self.w.params.clone()
@@ -308,7 +308,7 @@ class ReweightWorkload:
     def oracle_sample(self, budget_rows: int):
         import copy
         import oracle
-        from tests import oracle_build as ob
+        from oracle import problems as ob
         frac = 1.0 if self.cfg == 3 else 1.0 / 8
         nb = max(1, int(self.B * frac))
         inp = copy.copy(self.inp)
@@ -347,7 +347,7 @@ class ThreeLevelWorkload:
     def setup_device(self):
         import torch
         import paper_2207_02849_b200 as bt
-        from tests import cuda_build as cb
+        from paper_2207_02849_b200 import problems as cb
         self.bt, self.torch = bt, torch
         self.P = cb.three_levels(self.inp)
         self.w0 = self.P[0].params.clone()
@@ -385,7 +385,7 @@ class ThreeLevelWorkload:
 
     def oracle_sample(self, budget_rows: int):
         import oracle
-        from tests import oracle_build as ob
+        from oracle import problems as ob
         O1, O2, O3 = ob.three_levels(self.inp)
         nm = dict(method="neumann", K=self.inp.K, alpha=self.inp.alpha)
         t0 = time.perf_counter()

@@ -314,6 +314,14 @@ betty_status betty_engine_run(const betty_level* const* levels, int32_t n_levels
  * then reports the condition.  Every wait in the library's kernels uses the same bounded form. */
 betty_status betty_selftest_wait_timeout(void* ws, size_t ws_bytes, void* stream);
 
+/* Self test of a piece of host logic; touches no device.  Kernels that need more than the default
+ * dynamic shared memory have their limit raised once per kernel and per device ordinal (the setting
+ * belongs to a device, and one process may drive several).  This call drives one private instance of
+ * that bookkeeping: reset != 0 forgets everything first; the return value is 1 when a launch that
+ * needs `bytes` on device ordinal `device` would have to set the limit, 0 when an earlier call already
+ * covered it on that device.  Ordinals outside the table (negative or >= 64) always return 1. */
+int32_t betty_selftest_smem_limit(int32_t reset, int32_t device, uint64_t bytes);
+
 const char* betty_status_string(betty_status s);
 
 /* Number of CUDA kernels this library has launched in the calling process since it was loaded

@@ -6,7 +6,8 @@ from .binding import (  # noqa: F401
     BettyError, Level, betty_gemm_bf16, MethodCfg, Workspace, betty_chain_levels, betty_grad, betty_hvp,
     betty_hvp_logreg_static, betty_hypergrad_cg, betty_engine_run, betty_find_paths, betty_hypergrad_fd, betty_hypergrad_graph, betty_hypergrad_itd, betty_hypergrad_neumann, betty_kernel_launches,
     betty_lower_step,
-    betty_mixed_vjp, betty_poll_status, betty_reset_status, betty_selftest_wait_timeout, betty_status_string,
+    betty_mixed_vjp, betty_poll_status, betty_reset_status, betty_selftest_smem_limit, betty_selftest_wait_timeout,
+    betty_status_string,
     betty_workspace_size, lib, lib_path,
 )
 from . import binding as _b

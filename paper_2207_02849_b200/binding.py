@@ -107,6 +107,8 @@ def lib():
         fn.argtypes, fn.restype = args, C.c_int
     L.betty_status_string.argtypes, L.betty_status_string.restype = [C.c_int], C.c_char_p
     L.betty_kernel_launches.argtypes, L.betty_kernel_launches.restype = [], C.c_uint64
+    L.betty_selftest_smem_limit.argtypes = [I32, I32, C.c_uint64]
+    L.betty_selftest_smem_limit.restype = I32
     _lib = L
     return L
 
@@ -368,3 +370,8 @@ def betty_engine_run(levels: Sequence[Level], u2l, l2u, per_level: Sequence[Meth
 
 def betty_selftest_wait_timeout(ws: Workspace, stream=None) -> None:
     _check(lib().betty_selftest_wait_timeout(ws.ptr, ws.nbytes, _stream(stream)), "betty_selftest_wait_timeout")
+
+
+def betty_selftest_smem_limit(reset: bool, device: int, nbytes: int) -> bool:
+    """Host-only: would a launch needing `nbytes` of dynamic shared memory on `device` set the limit?"""
+    return bool(lib().betty_selftest_smem_limit(1 if reset else 0, int(device), int(nbytes)))

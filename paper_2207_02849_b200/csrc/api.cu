@@ -6,7 +6,26 @@
 
 namespace betty {
 
-unsigned long long g_kernel_launches = 0;
+std::atomic<unsigned long long> g_kernel_launches{0};
+
+int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return -1; }
+  return (dev >= 0 && dev < MAX_DEVICES) ? dev : -1;
+}
+int current_sm_count() {
+  static std::atomic<int> cached[MAX_DEVICES];          // 0: not asked yet
+  const int dev = current_device();
+  if (dev < 0) return DEFAULT_SM_COUNT;
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    return DEFAULT_SM_COUNT;
+  }
+  cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
 
 // ------------------------------------------------------------------ small kernels
 // out (+)= scale * x
@@ -112,11 +131,9 @@ betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
 
 betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu, VecHvpCache* cache) {
   if (!vec_has_wd(L)) return BETTY_ERR_UNSUPPORTED;
-  const betty_status s = logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, u,
-                                     find_constraint(L, BETTY_PARAM_VECTOR)->params, Hu, nullptr, 0.f,
-                                     cache ? cache->curv : nullptr, cache ? cache->valid : false);
-  if (cache && cache->curv && s == BETTY_OK) cache->valid = true;
-  return s;
+  return logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, u,
+                     find_constraint(L, BETTY_PARAM_VECTOR)->params, Hu, nullptr, 0.f, cache ? cache->curv : nullptr,
+                     cache ? &cache->valid : nullptr);
 }
 
 betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, const float* q, float* out) {
@@ -291,6 +308,7 @@ static betty_status hypergrad(const betty_level* lower, const betty_level* upper
   BETTY_TRY(validate_level(lower));
   BETTY_TRY(validate_level(upper));
   if (!wrt || !out) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(out)) return BETTY_ERR_ALIGNMENT;
   BETTY_TRY(check_ws(ws, ws_bytes));
   if (!is_participant(upper, lower) || !is_participant(upper, wrt) || !is_participant(lower, wrt) || wrt == lower)
     return BETTY_ERR_INVALID_ARG;
@@ -319,6 +337,7 @@ static betty_status hypergrad_itd(const betty_level* lower, const betty_level* u
   BETTY_TRY(validate_level(lower));
   BETTY_TRY(validate_level(upper));
   if (!wrt || !out || n_steps < 0) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(out)) return BETTY_ERR_ALIGNMENT;
   if (lower->optimizer != BETTY_OPT_GD) return BETTY_ERR_UNSUPPORTED;   // the reverse sweep differentiates plain GD steps
   BETTY_TRY(check_ws(ws, ws_bytes));
   if (!is_participant(upper, lower) || !is_participant(upper, wrt) || !is_participant(lower, wrt) || wrt == lower)
@@ -548,6 +567,7 @@ betty_status betty_hypergrad_graph(const betty_level* const* levels, int32_t n_l
                                    void* stream) {
   Graph g = {n_levels, u2l, n_u2l, l2u, n_l2u};
   if (!levels || !graph_ok(g) || k < 0 || k >= n_levels || !per_level || !out || n_levels > 256) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(out)) return BETTY_ERR_ALIGNMENT;
   for (int i = 0; i < n_levels; ++i) BETTY_TRY(validate_level(levels[i]));
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
@@ -603,7 +623,13 @@ const char* betty_status_string(betty_status s) {
   return "unknown status";
 }
 
-uint64_t betty_kernel_launches(void) { return (uint64_t)g_kernel_launches; }
+uint64_t betty_kernel_launches(void) { return (uint64_t)g_kernel_launches.load(std::memory_order_relaxed); }
+
+int32_t betty_selftest_smem_limit(int32_t reset, int32_t device, uint64_t bytes) {
+  static SmemLimit lim = {};
+  if (reset) lim = SmemLimit{};
+  return lim.raise(device, (size_t)bytes) ? 1 : 0;
+}
 
 betty_status betty_workspace_size(const betty_level* const* levels, int32_t n_levels, size_t* bytes) {
   if (!levels || n_levels <= 0 || !bytes) return BETTY_ERR_INVALID_ARG;
@@ -617,7 +643,7 @@ betty_status betty_workspace_size(const betty_level* const* levels, int32_t n_le
       // per-CTA column partials of the streaming pass (2 CTAs per SM) or the fallback's row scratch
       size_t d = (size_t)(L->d > 0 ? L->d : 1), n = (size_t)(L->n > 0 ? L->n : 1);
       // (+ n floats: the per-row curvature shared by the HVPs of one solve)
-      size_t need = (2 * 148 + 64) * d * sizeof(float) + 2 * n * sizeof(float) + 8192;
+      size_t need = (size_t)(2 * current_sm_count() + 64) * d * sizeof(float) + 2 * n * sizeof(float) + 8192;
       if (need > total) total = need + (1 << 20);
     } else if (is_mlp_family(L->loss)) {
       total += mlpfam_workspace(L);
@@ -643,7 +669,7 @@ betty_status betty_poll_status(const void* ws, void* stream, int32_t* cg_iters) 
   if (cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess) return BETTY_ERR_CUDA;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BETTY_ERR_CUDA;
   if (cg_iters) *cg_iters = h.cg_iters;
-  if (h.code < 0 || h.code > BETTY_ERR_UNSUPPORTED) return BETTY_ERR_CUDA;
+  if (h.code < 0 || h.code > BETTY_ERR_CAPACITY) return BETTY_ERR_CUDA;   // not a status this library writes
   return (betty_status)h.code;
 }
 
@@ -668,6 +694,7 @@ betty_status betty_grad(const betty_level* L, const betty_level* wrt, float* out
                         void* stream) {
   BETTY_TRY(validate_level(L));
   if (!wrt || !out || !is_participant(L, wrt)) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(out)) return BETTY_ERR_ALIGNMENT;
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
   return level_grad(c, L, wrt, out);
@@ -689,6 +716,7 @@ betty_status betty_mixed_vjp(const betty_level* L, const betty_level* wrt, const
                              size_t ws_bytes, void* stream) {
   BETTY_TRY(validate_level(L));
   if (!wrt || !q || !out || !is_participant(L, wrt) || wrt == L) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return BETTY_ERR_ALIGNMENT;
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
   if (is_vector_family(L->loss)) return vecfam_mixed(c, L, wrt, q, out);
@@ -720,6 +748,7 @@ betty_status betty_chain_levels(const betty_level* const* levels, int32_t n_leve
                                 int32_t path_len, const betty_method_cfg* per_edge, const float* v_in, float* out,
                                 int32_t accumulate, void* ws, size_t ws_bytes, void* stream) {
   if (!levels || n_levels <= 0 || !path || path_len < 2 || !per_edge || !out) return BETTY_ERR_INVALID_ARG;
+  if (!aligned16(out) || !aligned16(v_in)) return BETTY_ERR_ALIGNMENT;     // a null v_in counts as aligned
   for (int i = 0; i < path_len; ++i)
     if (path[i] < 0 || path[i] >= n_levels || !levels[path[i]]) return BETTY_ERR_INVALID_ARG;
   for (int i = 0; i < path_len; ++i) BETTY_TRY(validate_level(levels[path[i]]));

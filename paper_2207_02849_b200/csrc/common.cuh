@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <atomic>
 #include "betty.h"
 
 namespace betty {
@@ -60,12 +61,45 @@ struct SharedWeights {
   bf16* W[16];
 };
 
+// ---- per-device facts and settings ----
+// A process may drive several GPUs.  The SM count and every cudaFuncSetAttribute belong to one device, so both
+// are remembered per device ordinal, never process-wide.
+static constexpr int MAX_DEVICES = 64;
+static constexpr int DEFAULT_SM_COUNT = 148;
+// ordinal of the current device, or -1 (no device, or an ordinal beyond MAX_DEVICES)
+int current_device();
+// SM count of the current device, asked once per device; DEFAULT_SM_COUNT when it cannot be asked
+int current_sm_count();
+// Largest dynamic-shared-memory limit already set for one kernel, per device.  One instance per kernel
+// instantiation (a function-local static).
+struct SmemLimit {
+  size_t bytes[MAX_DEVICES];
+  // true when `want` bytes on device `dev` need the attribute to be (re)set; records the new limit
+  bool raise(int dev, size_t want) {
+    if (dev < 0 || dev >= MAX_DEVICES) return true;        // unknown device: set it every time
+    if (want <= bytes[dev]) return false;
+    bytes[dev] = want;
+    return true;
+  }
+};
+// Make `bytes` of dynamic shared memory launchable for `kernel` on the current device.
+template <typename K>
+static inline betty_status ensure_dynamic_smem(K kernel, SmemLimit& lim, size_t bytes) {
+  if (!lim.raise(current_device(), bytes)) return BETTY_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return BETTY_ERR_CUDA;
+  }
+  return BETTY_OK;
+}
+
 struct Ctx {
   cudaStream_t stream;
   Arena arena;
   int sm_count;
   SharedWeights shared;
-  __host__ Ctx(void* ws, size_t ws_bytes, void* s) : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(148) {
+  __host__ Ctx(void* ws, size_t ws_bytes, void* s)
+      : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(current_sm_count()) {
     shared.master = nullptr;
   }
 };
@@ -77,10 +111,10 @@ struct Ctx {
   } while (0)
 
 // Every kernel launch of the library passes through this check, which also counts it.
-extern unsigned long long g_kernel_launches;
+extern std::atomic<unsigned long long> g_kernel_launches;
 #define BETTY_LAUNCH_CHECK()                                   \
   do {                                                         \
-    ++betty::g_kernel_launches;                                \
+    betty::g_kernel_launches.fetch_add(1, std::memory_order_relaxed); \
     if (cudaPeekAtLastError() != cudaSuccess) {                \
       (void)cudaGetLastError();                                \
       return BETTY_ERR_CUDA;                                   \

@@ -806,11 +806,8 @@ template <int BN>
 static betty_status launch_tc(Ctx& c, const GemmDesc& g0, bool tr) {
   using Cfg = TcCfg<BN>;
   const GemmDesc g = tr ? swapped(g0) : g0;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM) != cudaSuccess) return BETTY_ERR_CUDA;
-    attr_set = true;
-  }
+  static SmemLimit limit = {};      // per tile width and per device
+  BETTY_TRY(ensure_dynamic_smem(k_gemm_tc<BN>, limit, (size_t)Cfg::SMEM));
   CUtensorMap tm[4];
   TcArgs a;
   fill_args(c, g, a, tr);
@@ -851,11 +848,8 @@ static void fill_args(Ctx& c, const GemmDesc& g, TcArgs& a, bool tr) {
 
 static betty_status launch_tc2(Ctx& c, const GemmDesc& g0, bool tr) {
   const GemmDesc g = tr ? swapped(g0) : g0;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, TC2_SMEM) != cudaSuccess) return BETTY_ERR_CUDA;
-    attr_set = true;
-  }
+  static SmemLimit limit = {};      // per device
+  BETTY_TRY(ensure_dynamic_smem(k_gemm_tc2, limit, (size_t)TC2_SMEM));
   CUtensorMap tm[4];
   TcArgs a;
   fill_args(c, g, a, tr);

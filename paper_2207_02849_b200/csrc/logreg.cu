@@ -270,11 +270,8 @@ template <int NCH, int FORM>
 static betty_status launch_stream(Ctx& c, const LrArgs& a, int grid) {
   size_t smem = (size_t)LR_S * LR_R * a.d * sizeof(float) + LR_S * sizeof(uint64_t) + 2 * LR_WARPS * 2 * LR_R * sizeof(float);
   auto kern = k_logreg_stream<NCH, FORM>;
-  static size_t attr_bytes = 0;     // raise the dynamic shared memory limit once per instantiation (and again if it grows)
-  if (smem > attr_bytes) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BETTY_ERR_CUDA;
-    attr_bytes = smem;
-  }
+  static SmemLimit limit = {};      // per instantiation and per device; raised again if a wider problem comes
+  BETTY_TRY(ensure_dynamic_smem(kern, limit, smem));
   kern<<<grid, LR_THREADS, smem, c.stream>>>(a);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
@@ -285,13 +282,13 @@ static betty_status launch_stream(Ctx& c, const LrArgs& a, int grid) {
 // decremented by lr times it.
 betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
                          const float* u, const float* lam, float* out, float* w_update, float lr, float* curv,
-                         bool curv_valid) {
+                         bool* curv_valid) {
   if (d <= 0) return BETTY_OK;
   LrArgs a;
   a.X = X; a.y = y; a.n = n; a.d = d; a.w = w; a.u = u; a.family = family;
   a.inv_n = n > 0 ? 1.0f / (float)n : 0.f;
   a.sb = c.arena.status();
-  a.curv = u ? curv : nullptr;
+  a.curv = (u && curv_valid) ? curv : nullptr;
   const size_t mark = c.arena.mark();
   int nparts;
   const bool fast = (d % 4 == 0) && d <= 4096 && aligned16(X) && aligned16(w) && (!u || aligned16(u));
@@ -303,11 +300,12 @@ betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int
     BETTY_ALLOC(partials, float, c, (size_t)grid * d);
     a.partials = partials;
     betty_status s;
-    const int form = !u ? LR_GRAD : (a.curv && curv_valid) ? LR_HVP_CACHED : LR_HVP;
+    const int form = !u ? LR_GRAD : (a.curv && *curv_valid) ? LR_HVP_CACHED : LR_HVP;
     if (d <= 1024) s = form == LR_GRAD ? launch_stream<1, LR_GRAD>(c, a, grid) : form == LR_HVP ? launch_stream<1, LR_HVP>(c, a, grid) : launch_stream<1, LR_HVP_CACHED>(c, a, grid);
     else if (d <= 2048) s = form == LR_GRAD ? launch_stream<2, LR_GRAD>(c, a, grid) : form == LR_HVP ? launch_stream<2, LR_HVP>(c, a, grid) : launch_stream<2, LR_HVP_CACHED>(c, a, grid);
     else s = form == LR_GRAD ? launch_stream<4, LR_GRAD>(c, a, grid) : form == LR_HVP ? launch_stream<4, LR_HVP>(c, a, grid) : launch_stream<4, LR_HVP_CACHED>(c, a, grid);
     BETTY_TRY(s);
+    if (form == LR_HVP && a.curv && family == 0) *curv_valid = true;     // this launch wrote the curvature
   } else {
     int64_t want = (n + 255) / 256; if (want < 1) want = 1; if (want > 64) want = 64;
     nparts = (int)want;
@@ -400,7 +398,8 @@ extern "C" betty_status betty_hvp_logreg_static(const float* X, int64_t n, int64
   a.sb = c.arena.status();
   a.partials = base + sizeof(StatusBlock) / sizeof(float);
   const int64_t ntiles = (n + LR_R - 1) / LR_R;
-  int grid = NOALLOC_MAX_CTAS;
+  int grid = 2 * c.sm_count;
+  if (grid > NOALLOC_MAX_CTAS) grid = NOALLOC_MAX_CTAS;
   if (ntiles < grid) grid = ntiles > 0 ? (int)ntiles : 1;
   betty_status st;
   a.curv = nullptr;

@@ -579,11 +579,8 @@ static betty_status launch_small(Ctx& c, SmallArgs& a) {
     return BETTY_OK;
   }
   const size_t smem = small_smem_bytes(a.rows_per_cta, a.rows_per_cta_v, a.d, a.mode == 2 ? (int64_t)a.n_steps * a.d : 0);
-  static size_t attr_bytes = 0;
-  if (smem > attr_bytes) {
-    if (cudaFuncSetAttribute(k_logreg_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BETTY_ERR_CUDA;
-    attr_bytes = smem;
-  }
+  static SmemLimit limit = {};      // per device
+  BETTY_TRY(ensure_dynamic_smem(k_logreg_small, limit, smem));
   k_logreg_small<<<SM_CL, SM_T, smem, c.stream>>>(a);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;

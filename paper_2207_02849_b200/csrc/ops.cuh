@@ -24,9 +24,12 @@ static inline bool is_mlp_family(int loss) {
 }
 
 // logreg.cu
+// curv / curv_valid: the per-row curvature buffer of one solve and whether it holds the curvature at w.  A pass
+// reads it only when *curv_valid is set and sets *curv_valid only when it has itself written the buffer (the
+// single-pass kernel in its full HVP form); the two-pass fallback neither reads nor writes it.
 betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
                          const float* u, const float* lam, float* out, float* w_update, float lr, float* curv = nullptr,
-                         bool curv_valid = false);
+                         bool* curv_valid = nullptr);
 
 // logreg_small.cu: whole-loop kernels for problems that fit a cluster's shared memory
 bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d, int64_t unrolled_steps = 0);

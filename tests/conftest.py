@@ -1,3 +1,4 @@
+import json
 import os
 import sys
 
@@ -24,3 +25,34 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+_PARITY = {}
+
+
+@pytest.fixture
+def parity_record():
+    """record(name, value): keeps a measured parity error; the session writes all of them to
+    gpurun_out/parity_errors.json (the figures quoted in the documentation come from that file)."""
+    def record(name, value):
+        _PARITY[name] = float(value)
+        return float(value)
+    return record
+
+
+def pytest_sessionfinish(session, exitstatus):
+    if not _PARITY:
+        return
+    out = os.path.join(ROOT, "gpurun_out")
+    try:
+        os.makedirs(out, exist_ok=True)
+        path = os.path.join(out, "parity_errors.json")
+        old = {}
+        if os.path.exists(path):
+            with open(path) as f:
+                old = json.load(f)
+        old.update(_PARITY)
+        with open(path, "w") as f:
+            json.dump(old, f, indent=1, sort_keys=True)
+    except OSError:
+        pass

@@ -1,63 +1,23 @@
-"""Builds CUDA-library `Level` descriptors (device tensors) from the seeded synthetic inputs."""
+"""Test-side names for the library's level builders, plus the error measures the parity tests use."""
 import numpy as np
 import torch
 
-import paper_2207_02849_b200 as bt
+from paper_2207_02849_b200.problems import (  # noqa: F401
+    dev, logreg_levels, quadratic_levels, reweight_levels, three_levels,
+)
 
 
-def dev(a, dtype=None):
-    t = torch.from_numpy(np.ascontiguousarray(a))
-    if dtype is not None:
-        t = t.to(dtype)
-    return t.cuda()
-
-
-def logreg_levels(inp):
-    lam = bt.Level(bt.LOSS_LOGREG, bt.PARAM_VECTOR, dev(inp.lam), X=dev(inp.Xv), y=dev(inp.yv))
-    w = bt.Level(bt.LOSS_LOGREG_WD, bt.PARAM_VECTOR, dev(inp.w0), X=dev(inp.X), y=dev(inp.y), lr=inp.lr)
-    w.set_constraints([lam])
-    lam.set_constraints([w])
-    return w, lam
-
-
-def quadratic_levels(A, b, lam, Av, bv, w0=None):
-    f = lambda a: dev(np.asarray(a, dtype=np.float32))
-    up = bt.Level(bt.LOSS_QUADRATIC, bt.PARAM_VECTOR, f(lam), X=f(Av), y=f(bv))
-    lo = bt.Level(bt.LOSS_QUADRATIC_WD, bt.PARAM_VECTOR, f(np.zeros(A.shape[1]) if w0 is None else w0),
-                  X=f(A), y=f(b))
-    lo.set_constraints([up])
-    up.set_constraints([lo])
-    return lo, up
-
-
-def _act(name):
-    return bt.ACT_RELU if name == "relu" else bt.ACT_GELU
-
-
-def reweight_levels(inp):
-    theta = bt.Level(bt.LOSS_MLP_CE, bt.PARAM_WEIGHTNET, dev(inp.theta), X=dev(inp.val.X, torch.bfloat16),
-                     y=dev(inp.val.y))
-    w = bt.Level(bt.LOSS_MLP_CE_REWEIGHT, bt.PARAM_MLP, dev(inp.w), X=dev(inp.train.X, torch.bfloat16),
-                 y=dev(inp.train.y), widths=inp.widths, activation=_act(inp.activation), lr=inp.lr)
-    w.set_constraints([theta])
-    theta.set_constraints([w])
-    return w, theta
-
-
-def three_levels(inp):
-    P1 = bt.Level(bt.LOSS_MLP_CE_REWEIGHT, bt.PARAM_MLP, dev(inp.w), X=dev(inp.D1.X, torch.bfloat16),
-                  y=dev(inp.D1.y), widths=inp.widths, activation=_act(inp.activation), lr=inp.lr)
-    P2 = bt.Level(bt.LOSS_WEIGHTNET_DETECT, bt.PARAM_WEIGHTNET, dev(inp.theta), X=dev(inp.D2.X, torch.bfloat16),
-                  y=dev(inp.D2.y), aux=dev(inp.D2.clean), mu=inp.mu)
-    P3 = bt.Level(bt.LOSS_WEIGHTNET_DETECT, bt.PARAM_LOGWD, dev(inp.lam), X=dev(inp.D3.X, torch.bfloat16),
-                  y=dev(inp.D3.y), aux=dev(inp.D3.clean), mu=0.0)
-    P1.set_constraints([P2, P3])
-    P2.set_constraints([P1])
-    P3.set_constraints([P2, P1])
-    return P1, P2, P3
+def _np(a):
+    return a.detach().double().cpu().numpy() if isinstance(a, torch.Tensor) else np.asarray(a, np.float64)
 
 
 def rel_l2(got, ref):
-    got = got.detach().double().cpu().numpy() if isinstance(got, torch.Tensor) else np.asarray(got, np.float64)
-    ref = np.asarray(ref, dtype=np.float64)
+    got, ref = _np(got), _np(ref)
     return float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+def rel_max(got, ref):
+    """Largest element error over the largest reference magnitude: catches one wrong component of a short
+    vector that a whole-vector norm would let through."""
+    got, ref = _np(got), _np(ref)
+    return float(np.max(np.abs(got - ref)) / max(np.max(np.abs(ref)), 1e-300)) if ref.size else 0.0

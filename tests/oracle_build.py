@@ -1,44 +1,2 @@
-"""Builds oracle `Level` objects from the seeded synthetic inputs (test helper)."""
-import numpy as np
-
-from oracle import Level
-
-
-def logreg_levels(inp):
-    lam = Level(loss="logreg", param_kind="vector", params=inp.lam, X=inp.Xv, y=inp.yv)
-    w = Level(loss="logreg_wd", param_kind="vector", params=inp.w0, X=inp.X, y=inp.y,
-              lr=inp.lr, constraints=[lam])
-    lam.constraints = [w]
-    return w, lam
-
-
-def quadratic_levels(A, b, lam, Av, bv, w0=None):
-    up = Level(loss="quadratic", param_kind="vector", params=lam, X=Av, y=np.asarray(bv, float))
-    lo = Level(loss="quadratic_wd", param_kind="vector",
-               params=np.zeros(A.shape[1]) if w0 is None else w0, X=A,
-               y=np.asarray(b, float), constraints=[up])
-    up.constraints = [lo]
-    return lo, up
-
-
-def reweight_levels(inp, bf16=True, quant="operands"):
-    theta = Level(loss="mlp_ce", param_kind="weightnet", params=inp.theta, X=inp.val.X,
-                  y=inp.val.y)
-    w = Level(loss="mlp_ce_reweight", param_kind="mlp", params=inp.w, X=inp.train.X,
-              y=inp.train.y, widths=inp.widths, activation=inp.activation, lr=inp.lr,
-              bf16=bf16, quant=quant, constraints=[theta])
-    theta.constraints = [w]
-    return w, theta
-
-
-def three_levels(inp, bf16=True, quant="operands"):
-    """P1 classifier, P2 weight net (detector loss on D2), P3 log weight decay (detector
-    loss on D3, no mu term)."""
-    P1 = Level(loss="mlp_ce_reweight", param_kind="mlp", params=inp.w, X=inp.D1.X, y=inp.D1.y,
-               widths=inp.widths, activation=inp.activation, lr=inp.lr, bf16=bf16, quant=quant)
-    P2 = Level(loss="weightnet_detect", param_kind="weightnet", params=inp.theta, X=inp.D2.X,
-               y=inp.D2.y, aux=inp.D2.clean.astype(np.float64), mu=inp.mu, constraints=[P1])
-    P3 = Level(loss="weightnet_detect", param_kind="logwd", params=inp.lam, X=inp.D3.X,
-               y=inp.D3.y, aux=inp.D3.clean.astype(np.float64), mu=0.0, constraints=[P2, P1])
-    P1.constraints = [P2, P3]
-    return P1, P2, P3
+"""Test-side names for the oracle's level builders."""
+from oracle.problems import logreg_levels, quadratic_levels, reweight_levels, three_levels  # noqa: F401

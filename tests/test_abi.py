@@ -50,3 +50,20 @@ def test_binding_struct_layout_matches_header():
         for part in decl.split(","):
             names.append(re.findall(r"[A-Za-z_][A-Za-z_0-9]*", part)[-1])
     assert names == [f[0] for f in binding._Level._fields_]
+
+
+def test_shared_memory_limits_are_remembered_per_device(libpath):
+    """A kernel's raised shared-memory limit belongs to one device: what device 0 has set says nothing
+    about device 1, a smaller request on the same device needs no new setting, a larger one does."""
+    import paper_2207_02849_b200 as bt
+    f = bt.betty_selftest_smem_limit
+    assert f(True, 0, 98_000) is True
+    assert f(False, 0, 98_000) is False
+    assert f(False, 0, 64_000) is False
+    assert f(False, 1, 64_000) is True          # another device starts from nothing
+    assert f(False, 1, 98_000) is True
+    assert f(False, 0, 200_000) is True         # grows on device 0
+    assert f(False, 0, 98_000) is False
+    assert f(False, -1, 1) is True and f(False, -1, 1) is True      # unknown ordinal: never cached
+    assert f(False, 64, 1) is True
+    assert f(True, 0, 10) is True               # reset forgets

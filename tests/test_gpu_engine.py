@@ -72,10 +72,10 @@ def test_three_level_mlp_run(bt):
     cfg, ocfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=3, alpha=0.01), dict(method="neumann", K=3, alpha=0.01)
     log = bt.betty_engine_run(list(P), u2l, l2u, [cfg] * 3, [2, 1, 1], 4, ws)
     assert log == oracle.engine_run(list(O), u2l, l2u, [ocfg] * 3, [2, 1, 1], 4) == [0, 0, 1, 2, 0, 0, 1, 2]
-    assert cb.rel_l2(P[0].params, O[0].params) < 1e-3
-    assert cb.rel_l2(P[1].params - cb.dev(inp.theta), O[1].params - inp.theta.astype(np.float64)) < 3e-2   # the update itself
+    assert cb.rel_l2(P[0].params - cb.dev(inp.w), O[0].params - inp.w.astype(np.float64)) < 2e-2       # the updates themselves
+    assert cb.rel_l2(P[1].params - cb.dev(inp.theta), O[1].params - inp.theta.astype(np.float64)) < 2e-2
     assert np.linalg.norm(O[2].params - inp.lam) > 1e-4   # the step is well above fp32 resolution of lambda
-    assert cb.rel_l2(P[2].params - cb.dev(inp.lam), O[2].params - inp.lam.astype(np.float64)) < 5e-2
+    assert cb.rel_l2(P[2].params - cb.dev(inp.lam), O[2].params - inp.lam.astype(np.float64)) < 2e-2
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
 
@@ -110,8 +110,8 @@ def test_two_upper_problems_share_one_lower_problem(bt):
     ws = bt.Workspace([P1, P2, P3])
     log = bt.betty_engine_run([P1, P2, P3], u2l, l2u, [cfg] * 3, [2, 1, 1], 4, ws)
     assert log == oracle.engine_run([O1, O2, O3], u2l, l2u, [ocfg] * 3, [2, 1, 1], 4) == [0, 0, 1, 2, 0, 0, 1, 2]
-    assert cb.rel_l2(P1.params, O1.params) < 1e-3
-    assert cb.rel_l2(P2.params - cb.dev(inp.theta), O2.params - inp.theta.astype(np.float64)) < 3e-2
+    assert cb.rel_l2(P1.params - cb.dev(inp.w), O1.params - inp.w.astype(np.float64)) < 2e-2
+    assert cb.rel_l2(P2.params - cb.dev(inp.theta), O2.params - inp.theta.astype(np.float64)) < 2e-2
     assert np.linalg.norm(O3.params - inp.lam) > 1e-4
-    assert cb.rel_l2(P3.params - cb.dev(inp.lam), O3.params - inp.lam.astype(np.float64)) < 5e-2
+    assert cb.rel_l2(P3.params - cb.dev(inp.lam), O3.params - inp.lam.astype(np.float64)) < 2e-2
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK

@@ -32,7 +32,10 @@ def test_config2_full_size_hypergradient():
     assert cb.rel_l2(out, ref) < 1e-4
 
 
-def test_config5_full_size_hypergradient():
+def test_config5_full_size_hypergradient(parity_record):
+    """Held to 2e-2 against the oracle under both readings of a mixed-precision level (bf16 operands in
+    every product; matrices rounded only), for the parameter update of the four lower steps and for the
+    hypergradient (whole vector and largest single component)."""
     import paper_2207_02849_b200 as bt
     from tests import cuda_build as cb
     inp = si.config5()
@@ -42,8 +45,12 @@ def test_config5_full_size_hypergradient():
     out = torch.empty(si.WEIGHTNET_PARAMS, dtype=torch.float32, device="cuda")
     bt.betty_hypergrad_neumann(w, th, th, inp.K, inp.alpha, out, ws)
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
-    ow, oth = ob.reweight_levels(inp)
-    oracle.lower_step(ow, inp.lower_steps)
-    ref = oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)
-    assert cb.rel_l2(w.params, ow.params) < 1e-3
-    assert cb.rel_l2(out, ref) < 2e-2
+    got_w = w.params.double().cpu().numpy()
+    w0 = inp.w.astype(np.float64)
+    for quant in ("operands", "weights"):
+        ow, oth = ob.reweight_levels(inp, quant=quant)
+        oracle.lower_step(ow, inp.lower_steps)
+        ref = oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)
+        assert parity_record(f"config5/{quant}/lower_update", cb.rel_l2(got_w - w0, ow.params - w0)) < 2e-2
+        assert parity_record(f"config5/{quant}/neumann", cb.rel_l2(out, ref)) < 2e-2
+        assert parity_record(f"config5/{quant}/neumann_max", cb.rel_max(out, ref)) < 2e-2

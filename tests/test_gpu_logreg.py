@@ -220,6 +220,43 @@ def test_empty_batch_and_argument_errors(bt):
     assert e.value.status == bt.BETTY_ERR_WORKSPACE
 
 
+def test_misaligned_vectors_are_rejected_and_chain_start_vectors_match_oracle(bt):
+    """Flat vector arguments must start on a 16-byte boundary: a start vector, a direction or an output
+    one float off is refused with BETTY_ERR_ALIGNMENT by every entry point (the single-pass kernel and
+    the curvature it leaves for the later HVPs of a solve rely on it).  With an aligned caller-supplied
+    start vector the chain call agrees with the oracle for both solvers, on a full-width level (single
+    pass, cached curvature) and on a width that takes the two-pass kernels (nothing cached)."""
+    from tests import cuda_build as cb
+    for n, d in [(1500, 4096), (400, 130)]:
+        inp = si.logreg_bilevel(21, n, d, 32)
+        (w, lam), (ow, olam) = _pair(inp)
+        ws = bt.Workspace([w, lam])
+        bt.betty_lower_step(w, 3, ws)
+        oracle.lower_step(ow, 3)
+        v = si.normal_f32(23, 5, (d,))
+        buf = torch.zeros(d + 4, dtype=torch.float32, device="cuda")
+        buf[1:d + 1] = cb.dev(v)
+        out = _vec(d)
+        for cfg, ocfg in [(bt.MethodCfg(bt.BETTY_NEUMANN, K=4, alpha=0.05), dict(method="neumann", K=4, alpha=0.05)),
+                          (bt.MethodCfg(bt.BETTY_CG, K=4), dict(method="cg", K=4, tol=0.0))]:
+            with pytest.raises(bt.BettyError) as e:
+                bt.betty_chain_levels([w, lam], [1, 0], [cfg], buf[1:d + 1], out, False, ws)
+            assert e.value.status == bt.BETTY_ERR_ALIGNMENT
+            with pytest.raises(bt.BettyError) as e:
+                bt.betty_chain_levels([w, lam], [1, 0], [cfg], cb.dev(v), buf[1:d + 1], False, ws)
+            assert e.value.status == bt.BETTY_ERR_ALIGNMENT
+            bt.betty_chain_levels([w, lam], [1, 0], [cfg], cb.dev(v), out, False, ws)
+            assert cb.rel_l2(out, oracle.chain_levels([ow, olam], [1, 0], [ocfg], v_in=v)) < TOL
+        for call in (lambda: bt.betty_grad(w, w, buf[1:d + 1], ws),
+                     lambda: bt.betty_mixed_vjp(w, lam, buf[1:d + 1], out, ws),
+                     lambda: bt.betty_hvp(w, buf[1:d + 1], out, ws),
+                     lambda: bt.betty_hypergrad_cg(w, lam, lam, 2, 0.0, buf[1:d + 1], ws)):
+            with pytest.raises(bt.BettyError) as e:
+                call()
+            assert e.value.status == bt.BETTY_ERR_ALIGNMENT
+        assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
 def test_repeated_calls_are_bitwise_identical(bt):
     inp = si.logreg_bilevel(8, 3000, 4096, 64)
     (w, lam), _ = _pair(inp)

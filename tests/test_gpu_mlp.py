@@ -12,10 +12,22 @@ from tests import oracle_build as ob
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
-# Products with an arbitrary N(0,1) direction on a small batch: the per-sample directional
-# derivative sum_c (p - onehot)_c * Ra_c cancels the common part of Ra, which amplifies the bf16
-# rounding of the direction; hypergradients (gradient-like directions) are held to TOL.
-TOL_RANDOM_DIR = 4e-2
+# Not a hypergradient: the mixed product with an arbitrary N(0,1) direction on a batch of a few dozen rows.
+# Its per-sample terms d_i * grad r_i cancel in the sum over the batch, which magnifies the bf16 rounding of
+# the direction (2^-9 per element); measured 2.6e-2 at worst over the shapes below.  With the direction the
+# solvers actually feed it (a gradient) the same product is held to TOL.
+TOL_RANDOM_DIR_MIXED = 4e-2
+# Not a hypergradient either: the classifier-sized intermediate vector of the three-level chain under the
+# plain reading (hidden activations unrounded in the oracle, bf16 on the GPU); the detector cost's
+# per-sample factors change sign, so its gradient cancels about ten-fold.  The chain's result is held to TOL.
+TOL_INTERMEDIATE_PLAIN = 5e-2
+
+
+def _update_err(cb, level, olevel, start):
+    """Relative L2 error of the parameter *update* (x_T - x_0): the parameters themselves move by a
+    fraction of a percent per step, so comparing them would hide a badly wrong step."""
+    x0 = np.asarray(start, dtype=np.float64)
+    return cb.rel_l2(level.params.double().cpu().numpy() - x0, olevel.params - x0)
 
 
 @pytest.fixture(scope="module")
@@ -37,7 +49,7 @@ def _perturb(inp, seed):
 
 @pytest.mark.parametrize("act,widths,B", [("relu", (24, 40, 16), 37), ("gelu", (24, 40, 16), 37),
                                           ("gelu", (16, 72, 64, 10), 130), ("relu", (784, 96, 10), 64)])
-def test_reweight_primitives_match_oracle(bt, act, widths, B):
+def test_reweight_primitives_match_oracle(bt, act, widths, B, parity_record):
     from tests import cuda_build as cb
     inp = _perturb(si.reweight_bilevel(41, widths, B, 0.4, activation=act), 41)
     w, th = cb.reweight_levels(inp)
@@ -55,12 +67,17 @@ def test_reweight_primitives_match_oracle(bt, act, widths, B):
     assert torch.all(outt == 0)
     u = si.normal_f32(43, 1, (P,))
     bt.betty_hvp(w, cb.dev(u), out, ws)
-    assert cb.rel_l2(out, oracle.hvp(ow, u)) < TOL_RANDOM_DIR
+    assert cb.rel_l2(out, oracle.hvp(ow, u)) < TOL
     bt.betty_mixed_vjp(w, th, cb.dev(u), outt, ws)
-    assert cb.rel_l2(outt, oracle.mixed_vjp(ow, oth, u)) < TOL_RANDOM_DIR
+    tag = f"primitives/{act}-{'x'.join(map(str, widths))}-B{B}"
+    assert parity_record(f"{tag}/mixed_random_direction", cb.rel_l2(outt, oracle.mixed_vjp(ow, oth, u))) < TOL_RANDOM_DIR_MIXED
+    g = oracle.grad(oth, ow)                                  # the direction Eq. 1 starts a solve from
+    bt.betty_mixed_vjp(w, th, cb.dev(g.astype(np.float32)), outt, ws)
+    assert parity_record(f"{tag}/mixed_gradient_direction",
+                         cb.rel_l2(outt, oracle.mixed_vjp(ow, oth, g.astype(np.float32)))) < TOL
     bt.betty_lower_step(w, 2, ws)
     oracle.lower_step(ow, 2)
-    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    assert _update_err(cb, w, ow, inp.w) < TOL
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
 
@@ -84,7 +101,7 @@ def test_reweight_hypergradients_match_oracle(bt, act):
     st, iters = bt.betty_poll_status(ws, raise_on_error=False)
     if info["status"] == "ok":
         assert st == bt.BETTY_OK and iters == info["iters"]
-        assert cb.rel_l2(out, ref) < 5e-2          # CG divides by p^T H p: looser in bf16
+        assert cb.rel_l2(out, ref) < TOL
     else:
         assert st == bt.BETTY_ERR_BREAKDOWN
 
@@ -156,34 +173,39 @@ def test_three_level_primitives_and_chain_match_oracle(bt, act):
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
 
-def test_config3_full_size(bt):
+def test_config3_full_size(bt, parity_record):
     """3072 -> 1024 -> 10, batch 512: one lower step, then the finite-difference and the Neumann
-    (K = 5) hypergradients of the weight net."""
+    (K = 5) hypergradients of the weight net.  Held to 2e-2 against the oracle under both readings of a
+    mixed-precision level: bf16 operands in every product (what the kernels do) and the plain reading
+    (matrices rounded, nothing else; finite difference at the unrounded displaced master)."""
     from tests import cuda_build as cb
     inp = si.config3()
     w, th = cb.reweight_levels(inp)
-    ow, oth = ob.reweight_levels(inp)
     ws = bt.Workspace([w, th])
     bt.betty_lower_step(w, inp.lower_steps, ws)
-    oracle.lower_step(ow, inp.lower_steps)
-    assert cb.rel_l2(w.params, ow.params) < 1e-3
-    out = _vec(si.WEIGHTNET_PARAMS)
-    bt.betty_hypergrad_fd(w, th, th, inp.eps0, inp.fd_alpha, out, ws)
-    assert cb.rel_l2(out, oracle.hypergrad_fd(ow, oth, oth, inp.eps0, inp.fd_alpha)) < TOL
-    bt.betty_hypergrad_neumann(w, th, th, inp.K, inp.alpha, out, ws)
-    assert cb.rel_l2(out, oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)) < TOL
+    fd, nm = _vec(si.WEIGHTNET_PARAMS), _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_hypergrad_fd(w, th, th, inp.eps0, inp.fd_alpha, fd, ws)
+    bt.betty_hypergrad_neumann(w, th, th, inp.K, inp.alpha, nm, ws)
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+    for quant in ("operands", "weights"):
+        ow, oth = ob.reweight_levels(inp, quant=quant)
+        oracle.lower_step(ow, inp.lower_steps)
+        assert parity_record(f"config3/{quant}/lower_update", _update_err(cb, w, ow, inp.w)) < TOL
+        ref_fd = oracle.hypergrad_fd(ow, oth, oth, inp.eps0, inp.fd_alpha)
+        ref_nm = oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)
+        assert parity_record(f"config3/{quant}/fd", cb.rel_l2(fd, ref_fd)) < TOL
+        assert parity_record(f"config3/{quant}/neumann", cb.rel_l2(nm, ref_nm)) < TOL
+        assert parity_record(f"config3/{quant}/fd_max", cb.rel_max(fd, ref_fd)) < TOL
+        assert parity_record(f"config3/{quant}/neumann_max", cb.rel_max(nm, ref_nm)) < TOL
 
 
-def test_config4_full_size(bt):
-    """784 -> 512 -> 512 -> 10, batch 1024, three levels, two Neumann (K = 3) edges."""
+def test_config4_full_size(bt, parity_record):
+    """784 -> 512 -> 512 -> 10, batch 1024, three levels, two Neumann (K = 3) edges; both readings."""
     from tests import cuda_build as cb
     inp = si.config4()
     P1, P2, P3 = cb.three_levels(inp)
-    O1, O2, O3 = ob.three_levels(inp)
     ws = bt.Workspace([P1, P2, P3])
     bt.betty_lower_step(P1, 1, ws)
-    oracle.lower_step(O1, 1)
     cfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=inp.K, alpha=inp.alpha)
     nm = dict(method="neumann", K=inp.K, alpha=inp.alpha)
     u, v_t, out = _vec(inp.w.size), _vec(si.WEIGHTNET_PARAMS), _vec(inp.lam.size)
@@ -191,11 +213,16 @@ def test_config4_full_size(bt):
     bt.betty_grad(P3, P2, v_t, ws)
     bt.betty_chain_levels([P1, P2, P3], [0, 1], [cfg], v_t, u, True, ws)
     bt.betty_chain_levels([P1, P2, P3], [2, 0], [cfg], u, out, False, ws)
-    ou = oracle.grad(O3, O1) + oracle.chain_levels([O1, O2, O3], [0, 1], [nm], v_in=oracle.grad(O3, O2))
-    ref = oracle.chain_levels([O1, O2, O3], [2, 0], [nm], v_in=ou)
-    assert cb.rel_l2(u, ou) < TOL
-    assert cb.rel_l2(out, ref) < TOL
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+    for quant in ("operands", "weights"):
+        O1, O2, O3 = ob.three_levels(inp, quant=quant)
+        oracle.lower_step(O1, 1)
+        assert parity_record(f"config4/{quant}/lower_update", _update_err(cb, P1, O1, inp.w)) < TOL
+        ou = oracle.grad(O3, O1) + oracle.chain_levels([O1, O2, O3], [0, 1], [nm], v_in=oracle.grad(O3, O2))
+        ref = oracle.chain_levels([O1, O2, O3], [2, 0], [nm], v_in=ou)
+        assert parity_record(f"config4/{quant}/u", cb.rel_l2(u, ou)) < (TOL if quant == "operands" else TOL_INTERMEDIATE_PLAIN)
+        assert parity_record(f"config4/{quant}/chain", cb.rel_l2(out, ref)) < TOL
+        assert parity_record(f"config4/{quant}/chain_max", cb.rel_max(out, ref)) < TOL     # each of the three components
 
 
 def test_config5_reduced_width(bt):
@@ -210,7 +237,7 @@ def test_config5_reduced_width(bt):
     ws = bt.Workspace([w, th])
     bt.betty_lower_step(w, inp.lower_steps, ws)
     oracle.lower_step(ow, inp.lower_steps)
-    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    assert _update_err(cb, w, ow, inp.w) < TOL
     out = _vec(si.WEIGHTNET_PARAMS)
     bt.betty_hypergrad_neumann(w, th, th, inp.K, inp.alpha, out, ws)
     assert cb.rel_l2(out, oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha)) < TOL
@@ -228,7 +255,7 @@ def test_itd_on_reweighting_matches_oracle(bt, act):
     out = _vec(si.WEIGHTNET_PARAMS)
     bt.betty_hypergrad_itd(w, th, th, T, out, ws)
     ref = oracle.hypergrad_itd(ow, oth, oth, T)
-    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    assert _update_err(cb, w, ow, inp.w) < TOL
     assert cb.rel_l2(out, ref) < TOL
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
@@ -274,9 +301,9 @@ def test_odd_widths_and_ragged_batches(bt, widths, B):
     assert cb.rel_l2(out, oracle.grad(ow, ow)) < TOL
     bt.betty_lower_step(w, 2, ws)
     oracle.lower_step(ow, 2)
-    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    assert _update_err(cb, w, ow, inp.w) < TOL
     bt.betty_hypergrad_neumann(w, th, th, 2, 0.01, outt, ws)
-    assert cb.rel_l2(outt, oracle.hypergrad_neumann(ow, oth, oth, 2, 0.01)) < TOL_RANDOM_DIR
+    assert cb.rel_l2(outt, oracle.hypergrad_neumann(ow, oth, oth, 2, 0.01)) < TOL
     bt.betty_hypergrad_fd(w, th, th, 0.01, 1.0, outt, ws)
-    assert cb.rel_l2(outt, oracle.hypergrad_fd(ow, oth, oth, 0.01, 1.0)) < TOL_RANDOM_DIR
+    assert cb.rel_l2(outt, oracle.hypergrad_fd(ow, oth, oth, 0.01, 1.0)) < TOL
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK

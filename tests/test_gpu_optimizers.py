@@ -59,9 +59,9 @@ def test_reweighting_run_with_momentum_classifier_and_adam_weight_net(bt):
     cfg, ocfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=3, alpha=0.01), dict(method="neumann", K=3, alpha=0.01)
     log = bt.betty_engine_run([w, th], u2l, l2u, [cfg, cfg], [2, 1], 4, ws)
     assert log == oracle.engine_run([ow, oth], u2l, l2u, [ocfg, ocfg], [2, 1], 4) == [0, 0, 1, 0, 0, 1]
-    assert cb.rel_l2(w.params, ow.params) < 1e-3
+    assert cb.rel_l2(w.params - cb.dev(inp.w), ow.params - inp.w.astype(np.float64)) < 2e-2
     # Adam's first steps have magnitude lr whatever the gradient scale, so theta's displacement is well resolved
-    assert cb.rel_l2(th.params - cb.dev(inp.theta), oth.params - inp.theta.astype(np.float64)) < 3e-2
+    assert cb.rel_l2(th.params - cb.dev(inp.theta), oth.params - inp.theta.astype(np.float64)) < 2e-2
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
 
