@@ -29,6 +29,20 @@ import numpy as np  # noqa: E402
 
 METRIC = "hypergradient_steps_per_sec"
 UNIT = "steps/s"
+# datasheet figures of the part (HGX B200: HBM3e bandwidth, dense bf16), reported beside the measured peaks
+NOMINAL_HBM_GBS = 7700.0
+NOMINAL_BF16_TFLOPS = 2250.0
+# (key, configuration, method, timed steps) of the short runs added to the default line
+PER_CONFIG_RUNS = [("config1_cg", 1, "cg", 50), ("config1_neumann", 1, "neumann", 50), ("config3_fd", 3, "fd", 30),
+                   ("config3_neumann", 3, "neumann", 30), ("config4", 4, "", 30), ("config5", 5, "neumann", 10)]
+
+
+def _release(w):
+    """Drop a workload's device tensors (its captured graph first)."""
+    for k in list(w.__dict__):
+        if k not in ("inp", "name", "dtype"):
+            w.__dict__.pop(k, None)
+    return None
 
 
 def _peaks():
@@ -200,6 +214,23 @@ class LogregWorkload:
         return {"kernel": "k_logreg_stream<HVP>", "ms": ms, "bytes": self.pass_bytes(), "bound": "hbm",
                 "also": {"kernel": "k_logreg_stream<gradient> (betty_lower_step, one step)", "ms": ms_g}}
 
+    def parity(self):
+        """Relative L2 error of one step's hypergradient against the fp64 oracle on the whole workload
+        (small configurations only)."""
+        import oracle
+        from oracle import problems as ob
+        self.step()
+        got = self.out.double().cpu().numpy()
+        ow, olam = ob.logreg_levels(self.inp)
+        oracle.lower_step(ow, self.inp.lower_steps)
+        if self.method == "cg":
+            ref = oracle.hypergrad_cg(ow, olam, olam, self.inp.K, 0.0)
+        elif self.method == "neumann":
+            ref = oracle.hypergrad_neumann(ow, olam, olam, self.inp.K, self.inp.alpha)
+        else:
+            return None
+        return float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
+
     # -- oracle on a bounded sample of the same workload
     def oracle_sample(self, budget_rows: int):
         import oracle
@@ -305,6 +336,34 @@ class ReweightWorkload:
         ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
         return {"kernel": f"k_gemm_tc {M}x{N}x{K}", "ms": ms, "flops": 2.0 * M * N * K, "bound": "tensor"}
 
+    def whole_step_flops(self):
+        """Matrix-product FLOPs of one step with the Neumann method: per layer U_l = 2 B in_l out_l; a
+        gradient is forward + backward-data + weight-gradient products (3 sum U - U_1), a Hessian-vector
+        product with the base pass cached is the R-forward, R-backward-data and two weight-gradient
+        products per layer (6 sum U - 4 U_1: the input has no tangent), the mixed product one R-forward."""
+        if self.method != "neumann":
+            return None
+        w = self.inp.widths
+        U = [2.0 * self.B * w[l] * w[l + 1] for l in range(len(w) - 1)]
+        grad, hvp, jvp = 3 * sum(U) - U[0], 6 * sum(U) - 4 * U[0], 2 * sum(U) - U[0]
+        return (self.inp.lower_steps + 2) * grad + self.inp.K * hvp + jvp
+
+    def parity(self):
+        """Relative L2 error of one step's hypergradient against the fp64 oracle on the whole workload."""
+        import oracle
+        from oracle import problems as ob
+        self.step()
+        got = self.out.double().cpu().numpy()
+        ow, oth = ob.reweight_levels(self.inp)
+        oracle.lower_step(ow, self.inp.lower_steps)
+        if self.method == "fd":
+            ref = oracle.hypergrad_fd(ow, oth, oth, self.inp.eps0, self.inp.fd_alpha)
+        elif self.method == "neumann":
+            ref = oracle.hypergrad_neumann(ow, oth, oth, self.inp.K, self.inp.alpha)
+        else:
+            return None
+        return float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
+
     def oracle_sample(self, budget_rows: int):
         import copy
         import oracle
@@ -382,6 +441,18 @@ class ThreeLevelWorkload:
         self.inp.widths  # forward-layout GEMM batch x 512 x 784
         rw = ReweightWorkload.roofline_probe
         return rw(self, reps)
+
+    def parity(self):
+        import oracle
+        from oracle import problems as ob
+        self.step()
+        got = self.out.double().cpu().numpy()
+        O1, O2, O3 = ob.three_levels(self.inp)
+        nm = dict(method="neumann", K=self.inp.K, alpha=self.inp.alpha)
+        oracle.lower_step(O1, 1)
+        u = oracle.grad(O3, O1) + oracle.chain_levels([O1, O2, O3], [0, 1], [nm], v_in=oracle.grad(O3, O2))
+        ref = oracle.chain_levels([O1, O2, O3], [2, 0], [nm], v_in=u)
+        return float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
 
     def oracle_sample(self, budget_rows: int):
         import oracle
@@ -501,6 +572,9 @@ def main():
     ap.add_argument("--gemm", default="",
                     help="M,N,K[,a_transposed,b_transposed,n_pairs,path]: time only the bf16 matrix-product kernel "
                          "through betty_gemm_bf16 (kernel study; prints its own JSON line)")
+    ap.add_argument("--per-config", type=int, default=-1,
+                    help="add short runs of the other configurations to the line (default: on for the plain "
+                         "single-GPU configuration-2 run)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -529,16 +603,25 @@ def main():
     if args.gemm:
         gemm_probe(args, torch, bt)
         return
-    wl = make_workload(args.config, args.method, args.scale)
-    wl.setup_device()
     warm = max(args.warmup, 3)
+    peaks = _peaks()
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps, warmup, sampler=None):
+    flush_buf = []
+
+    def flush_for(cfg):
+        """Configurations whose inputs fit in L2 get a flush (a 512 MiB write) before every step."""
+        if cfg == 2:
+            return None
+        if not flush_buf:
+            flush_buf.append(torch.empty(512 << 20, dtype=torch.uint8, device="cuda"))
+        return flush_buf[0]
+
+    def timed(fn, steps, warmup, flush, sampler=None, launches_per_replay=None):
         if sampler:
             sampler.start()     # the sampler starts during warm-up; only samples inside the timed region count
         for _ in range(warmup):
@@ -574,15 +657,6 @@ def main():
         ms = max_over_ranks(ms, world, dist, "cuda")
         return ms, launches, clocks
 
-    # configs whose inputs fit in L2 get a flush (a 512 MiB write) before every step
-    flush = None
-    if args.config != 2:
-        flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
-    l2_note = ("inputs (train matrix) larger than L2; no flush between steps" if flush is None
-               else "L2 flushed (512 MiB write) before every step; each step timed by its own event pair, flush excluded")
-    use_graph = (args.graph == 1) or (args.graph == -1 and args.config != 2)
-    launches_per_replay = None
-
     def capture(w):
         """The library's calls only enqueue work on the current stream and keep every scalar on the
         device, so a whole step can be captured once and replayed without host-side launch cost."""
@@ -602,17 +676,55 @@ def main():
         w._graph = graph
         return n
 
-    if use_graph:
-        launches_per_replay = capture(wl)
+    def roofline_of(w, reps=20):
+        probe = w.roofline_probe(reps)
+        if probe["bound"] == "hbm":
+            achieved = probe["bytes"] / (probe["ms"] * 1e-3) / 1e9
+            peak, unit, nominal = peaks["hbm_gbs"], "GB/s", NOMINAL_HBM_GBS
+        else:
+            achieved = probe["flops"] / (probe["ms"] * 1e-3) / 1e12
+            peak, unit, nominal = peaks["bf16_tflops"], "TFLOP/s", NOMINAL_BF16_TFLOPS
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "traffic.json")
+        if os.path.exists(tpath):
+            with open(tpath) as f:
+                tj = json.load(f).get(probe["kernel"])
+            if tj and tj.get("valid"):
+                if "dram_bytes_per_launch" in tj:       # captured at the probe's own shape
+                    traffic = float(tj["dram_bytes_per_launch"])
+                else:                                   # captured on a smaller case; grows with the units streamed
+                    traffic = tj["dram_bytes_per_unit"] * (probe["bytes"] / tj["unit_bytes"])
+        r = {"bound": probe["bound"], "kernel": probe["kernel"], "achieved": achieved, "peak": peak, "unit": unit,
+             "frac": achieved / peak, "traffic": traffic, "peak_source": f"{peaks['source']} (burst; kernel timed alone)",
+             "nominal_peak": nominal, "frac_of_nominal": achieved / nominal,
+             "kernel_ms": probe["ms"], "algorithmic_bytes_per_launch": probe.get("bytes"),
+             "algorithmic_flops_per_launch": probe.get("flops")}
+        if probe.get("also") and probe["bound"] == "hbm":
+            a2 = probe["bytes"] / (probe["also"]["ms"] * 1e-3) / 1e9
+            r["other_forms"] = [{"kernel": probe["also"]["kernel"], "kernel_ms": probe["also"]["ms"], "achieved": a2,
+                                 "frac": a2 / peak, "frac_of_nominal": a2 / nominal}]
+        return r
+
+    def graph_default(cfg):
+        return (args.graph == 1) or (args.graph == -1 and cfg != 2)
+
+    wl = make_workload(args.config, args.method, args.scale)
+    wl.setup_device()
+    flush = flush_for(args.config)
+    l2_note = ("inputs (train matrix) larger than L2; no flush between steps" if flush is None
+               else "L2 flushed (512 MiB write) before every step; each step timed by its own event pair, flush excluded")
+    use_graph = graph_default(args.config)
+    launches_per_replay = capture(wl) if use_graph else None
     step_dev, step_host = wl.step, wl.step_e2e
 
     sampler = ClockSampler(local) if rank == 0 else None
-    ms, launches, clocks = timed(step_dev, args.steps, warm, sampler)
+    ms, launches, clocks = timed(step_dev, args.steps, warm, flush, sampler, launches_per_replay)
     st, _ = bt.betty_poll_status(wl.ws)
     ms_per_step = ms / args.steps
     value = aggregate_value(ms_per_step, world)
 
     e2e = None
+    wl2 = sets = None
     if not args.no_e2e:
         wl.setup_host()
         e_steps = max(1, min(args.steps, 5))
@@ -665,54 +777,71 @@ def main():
             ms_e = max_over_ranks(e0.elapsed_time(e1), world, dist, "cuda")
             how = "two device input sets: step i+1's host-to-device copy overlaps step i's kernels"
         else:
-            ms_e, _, _ = timed(step_host, e_steps, 3)
+            ms_e, _, _ = timed(step_host, e_steps, 3, flush)
             how = "copy, compute and read-back in sequence on one stream"
         e2e = {"value": world * 1e3 / (ms_e / e_steps), "unit": UNIT, "h2d_bytes_per_step": int(wl.h2d),
                "d2h_bytes_per_step": int(wl.d2h), "how": how}
 
-    peaks = _peaks()
-    probe = wl.roofline_probe(20)
-    if probe["bound"] == "hbm":
-        achieved = probe["bytes"] / (probe["ms"] * 1e-3) / 1e9
-        peak, unit = peaks["hbm_gbs"], "GB/s"
+    roofline = roofline_of(wl)
+    wl_name, wl_dtype = wl.name, wl.dtype
+
+    # The other configurations, each as a short run of its own (the metric is quoted per configuration):
+    # only on the default single-GPU run, after the headline workload has released its device memory.
+    per_config = None
+    if args.per_config == 1 or (args.per_config == -1 and world == 1 and args.config == 2 and not args.method
+                                and args.scale == 1.0):
+        cpu_early = None
+        if not args.no_cpu_baseline and world == 1 and rank == 0:
+            sec, sample = wl.oracle_sample(args.oracle_rows)
+            cpu_early = {"value": 1.0 / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample}
+        del step_dev, step_host
+        if wl2 is not None:
+            _release(wl2)
+        wl2 = sets = None
+        wl = _release(wl)
+        torch.cuda.empty_cache()
+        per_config = {}
+        for key, cfg, method, steps_c in PER_CONFIG_RUNS:
+            w = make_workload(cfg, method, 1.0)
+            w.setup_device()
+            lpr = capture(w) if graph_default(cfg) else None
+            smp = ClockSampler(local)
+            ms_c, launches_c, clocks_c = timed(w.step, steps_c, 3, flush_for(cfg), smp, lpr)
+            st_c, _ = bt.betty_poll_status(w.ws)
+            entry = {"workload": w.name, "steps": steps_c, "ms_per_step": ms_c / steps_c,
+                     "steps_per_s": 1e3 * steps_c / ms_c, "gpu_launches_per_step": int(launches_c // steps_c),
+                     "cuda_graph": lpr is not None, "device_status": bt.betty_status_string(st_c), "clocks": clocks_c,
+                     "roofline": roofline_of(w, 10)}
+            if hasattr(w, "whole_step_flops") and w.whole_step_flops():
+                tf = w.whole_step_flops() / (ms_c / steps_c * 1e-3) / 1e12
+                entry["whole_step"] = {"tflops": tf, "frac_of_burst_peak": tf / peaks["bf16_tflops"],
+                                       "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"]}
+            if cfg in (1, 3, 4):
+                entry["rel_l2_vs_oracle"] = w.parity()
+            per_config[key] = entry
+            w = _release(w)
+            torch.cuda.empty_cache()
     else:
-        achieved = probe["flops"] / (probe["ms"] * 1e-3) / 1e12
-        peak, unit = peaks["bf16_tflops"], "TFLOP/s"
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            tj = json.load(f).get(probe["kernel"])
-        if tj and tj.get("valid"):
-            if "dram_bytes_per_launch" in tj:       # captured at the probe's own shape
-                traffic = float(tj["dram_bytes_per_launch"])
-            else:                                   # captured on a smaller case; grows with the units streamed
-                traffic = tj["dram_bytes_per_unit"] * (probe["bytes"] / tj["unit_bytes"])
-    roofline = {"bound": probe["bound"], "kernel": probe["kernel"], "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": traffic, "peak_source": f"{peaks['source']} (burst; kernel timed alone)",
-                "kernel_ms": probe["ms"], "algorithmic_bytes_per_launch": probe.get("bytes"),
-                "algorithmic_flops_per_launch": probe.get("flops")}
-    if probe.get("also") and probe["bound"] == "hbm":
-        a2 = probe["bytes"] / (probe["also"]["ms"] * 1e-3) / 1e9
-        roofline["other_forms"] = [{"kernel": probe["also"]["kernel"], "kernel_ms": probe["also"]["ms"], "achieved": a2,
-                                    "frac": a2 / peak}]
+        cpu_early = None
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    cpu = None
-    if not args.no_cpu_baseline and world == 1:
+    cpu = cpu_early
+    if cpu is None and not args.no_cpu_baseline and world == 1:
         sec, sample = wl.oracle_sample(args.oracle_rows)
         cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": wl.dtype, "data": "synthetic",
-            "config": {"workload": wl.name, "l2": l2_note,
+            "dtype": wl_dtype, "data": "synthetic",
+            "config": {"workload": wl_name, "l2": l2_note,
                        "replicas": world, "cuda_graph": bool(use_graph), "device_status": bt.betty_status_string(st)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
+    if per_config is not None:
+        line["per_config"] = per_config
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
