@@ -125,15 +125,28 @@ class ClockSampler:
 class LogregWorkload:
     """Configs 1 and 2: bilevel weight decay for logistic regression (App. D.1 problem)."""
 
-    def __init__(self, cfg: int, method: str, scale: float = 1.0):
+    def __init__(self, cfg: int, method: str, scale: float = 1.0, shard=None):
         import synth_inputs as si
         self.cfg = cfg
         self.inp = si.config1() if cfg == 1 else si.config2(scale)
         self.method = method or ("cg" if cfg == 2 else "cg")
         self.n, self.d = self.inp.X.shape
         self.nv = self.inp.Xv.shape[0]
-        self.name = (f"config{cfg}: logistic weight-decay bilevel, X fp32 {self.n}x{self.d} train / "
-                     f"{self.nv}x{self.d} val, {self.inp.lower_steps} lower GD steps, {self.method} K={self.inp.K}")
+        self.shard = shard
+        if shard is not None:       # strong scaling: this rank keeps its share of the rows of both matrices
+            from paper_2207_02849_b200 import data_parallel as dp
+            import copy
+            rank, world = shard
+            self.n_global, self.nv_global = self.n, self.nv
+            lo, hi = dp.shard_rows(self.n, rank, world)
+            lov, hiv = dp.shard_rows(self.nv, rank, world)
+            inp = copy.copy(self.inp)
+            inp.X, inp.y, inp.Xv, inp.yv = self.inp.X[lo:hi], self.inp.y[lo:hi], self.inp.Xv[lov:hiv], self.inp.yv[lov:hiv]
+            self.inp = inp
+            self.n, self.nv = hi - lo, hiv - lov
+        ng, nvg = (self.n_global, self.nv_global) if shard is not None else (self.n, self.nv)
+        self.name = (f"config{cfg}: logistic weight-decay bilevel, X fp32 {ng}x{self.d} train / "
+                     f"{nvg}x{self.d} val, {self.inp.lower_steps} lower GD steps, {self.method} K={self.inp.K}")
         self.dtype = "f32"
 
     # algorithmic bytes of one streaming pass over the train matrix (the dominant kernel)
@@ -146,6 +159,11 @@ class LogregWorkload:
         from paper_2207_02849_b200 import problems as cb
         self.bt, self.torch = bt, torch
         self.w, self.lam = cb.logreg_levels(self.inp)
+        if self.shard is not None:
+            from paper_2207_02849_b200 import data_parallel as dp
+            self.allreduce = dp.DeviceAllReduce()
+            dp.shard_level(self.w, self.n_global, self.shard[0], self.shard[1], self.allreduce)
+            dp.shard_level(self.lam, self.nv_global, self.shard[0], self.shard[1], self.allreduce)
         self.w0 = self.w.params.clone()
         self.out = torch.empty(self.d, dtype=torch.float32, device="cuda")
         extra = (self.inp.lower_steps + 1) * (self.d + 64) * 4 if self.method == "itd" else 0
@@ -263,13 +281,23 @@ class LogregWorkload:
 class ReweightWorkload:
     """Configs 3 and 5: data reweighting (App. A listing): lower MLP classifier, upper 1-100-1 weight net."""
 
-    def __init__(self, cfg: int, method: str):
+    def __init__(self, cfg: int, method: str, shard=None):
         import synth_inputs as si
         self.cfg = cfg
         self.inp = si.config3() if cfg == 3 else si.config5()
         self.method = method or ("fd" if cfg == 3 else "neumann")
         w = self.inp.widths
         self.B = self.inp.train.X.shape[0]
+        self.shard = shard
+        if shard is not None:       # strong scaling: this rank keeps its share of the rows of both batches
+            from paper_2207_02849_b200 import data_parallel as dp
+            import copy
+            self.B_global = self.B
+            lo, hi = dp.shard_rows(self.B, shard[0], shard[1])
+            cut = lambda b: type(b)(X=b.X[lo:hi], y=b.y[lo:hi], y_clean=b.y_clean[lo:hi], clean=b.clean[lo:hi])
+            inp = copy.copy(self.inp)
+            inp.train, inp.val = cut(self.inp.train), cut(self.inp.val)
+            self.inp = inp
         self.name = (f"config{cfg}: data reweighting, MLP {'x'.join(map(str, w)) if len(w) < 5 else f'{w[0]}->{len(w)-2}x{w[1]}->{w[-1]}'} "
                      f"{self.inp.activation} bf16/fp32-acc, batch {self.B}, {self.inp.lower_steps} lower SGD step(s), "
                      f"{self.method}" + (f" K={self.inp.K}" if self.method in ("neumann", "cg") else (" eps0=0.01" if self.method == "fd" else "")))
@@ -281,6 +309,11 @@ class ReweightWorkload:
         from paper_2207_02849_b200 import problems as cb
         self.bt, self.torch = bt, torch
         self.w, self.th = cb.reweight_levels(self.inp)
+        if self.shard is not None:
+            from paper_2207_02849_b200 import data_parallel as dp
+            self.allreduce = dp.DeviceAllReduce()
+            dp.shard_level(self.w, self.B_global, self.shard[0], self.shard[1], self.allreduce)
+            dp.shard_level(self.th, self.B_global, self.shard[0], self.shard[1], self.allreduce)
         self.w0 = self.w.params.clone()
         self.out = torch.empty(self.th.params.numel(), dtype=torch.float32, device="cuda")
         extra = (self.inp.lower_steps + 1) * (self.inp.w.size + 64) * 4 if self.method == "itd" else 0
@@ -466,12 +499,14 @@ class ThreeLevelWorkload:
         return time.perf_counter() - t0, "the full workload"
 
 
-def make_workload(cfg: int, method: str, scale: float):
+def make_workload(cfg: int, method: str, scale: float, shard=None):
     if cfg in (1, 2):
-        return LogregWorkload(cfg, method, scale)
+        return LogregWorkload(cfg, method, scale, shard)
     if cfg in (3, 5):
-        return ReweightWorkload(cfg, method)
+        return ReweightWorkload(cfg, method, shard)
     if cfg == 4:
+        if shard is not None:
+            raise SystemExit("strong scaling is offered for configurations 1, 2, 3 and 5")
         return ThreeLevelWorkload(method)
     raise SystemExit(f"unknown config {cfg}")
 
@@ -567,11 +602,14 @@ def main():
     ap.add_argument("--scale", type=float, default=1.0, help="row-count scale of config 2 (tests/profiling only)")
     ap.add_argument("--oracle-rows", type=int, default=131072)
     ap.add_argument("--graph", type=int, default=-1,
-                    help="replay the step from a CUDA graph captured from the C-ABI calls (default: on, except for "
-                         "configuration 2 whose step is 26 ms of large kernels)")
+                    help="replay the step from a CUDA graph captured from the C-ABI calls (default: on; 0 = plain calls)")
     ap.add_argument("--gemm", default="",
                     help="M,N,K[,a_transposed,b_transposed,n_pairs,path]: time only the bf16 matrix-product kernel "
                          "through betty_gemm_bf16 (kernel study; prints its own JSON line)")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: weak = N independent replicas of the workload (default); strong = ONE workload "
+                         "whose rows are sharded over the N ranks, one all-reduce of a parameter-sized vector per "
+                         "gradient / Hessian-vector product / mixed product")
     ap.add_argument("--per-config", type=int, default=-1,
                     help="add short runs of the other configurations to the line (default: on for the plain "
                          "single-GPU configuration-2 run)")
@@ -706,14 +744,15 @@ def main():
         return r
 
     def graph_default(cfg):
-        return (args.graph == 1) or (args.graph == -1 and cfg != 2)
+        return args.graph != 0
 
-    wl = make_workload(args.config, args.method, args.scale)
+    strong = args.scaling == "strong"
+    wl = make_workload(args.config, args.method, args.scale, (rank, world) if strong else None)
     wl.setup_device()
     flush = flush_for(args.config)
     l2_note = ("inputs (train matrix) larger than L2; no flush between steps" if flush is None
                else "L2 flushed (512 MiB write) before every step; each step timed by its own event pair, flush excluded")
-    use_graph = graph_default(args.config)
+    use_graph = graph_default(args.config) and not strong      # the all-reduce between kernels is not captured
     launches_per_replay = capture(wl) if use_graph else None
     step_dev, step_host = wl.step, wl.step_e2e
 
@@ -721,7 +760,7 @@ def main():
     ms, launches, clocks = timed(step_dev, args.steps, warm, flush, sampler, launches_per_replay)
     st, _ = bt.betty_poll_status(wl.ws)
     ms_per_step = ms / args.steps
-    value = aggregate_value(ms_per_step, world)
+    value = 1e3 / ms_per_step if strong else aggregate_value(ms_per_step, world)
 
     e2e = None
     wl2 = sets = None
@@ -779,7 +818,7 @@ def main():
         else:
             ms_e, _, _ = timed(step_host, e_steps, 3, flush)
             how = "copy, compute and read-back in sequence on one stream"
-        e2e = {"value": world * 1e3 / (ms_e / e_steps), "unit": UNIT, "h2d_bytes_per_step": int(wl.h2d),
+        e2e = {"value": (1 if strong else world) * 1e3 / (ms_e / e_steps), "unit": UNIT, "h2d_bytes_per_step": int(wl.h2d),
                "d2h_bytes_per_step": int(wl.d2h), "how": how}
 
     roofline = roofline_of(wl)
@@ -835,10 +874,15 @@ def main():
         cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": args.scaling, "vs_baseline": None,
             "dtype": wl_dtype, "data": "synthetic",
             "config": {"workload": wl_name, "l2": l2_note,
-                       "replicas": world, "cuda_graph": bool(use_graph), "device_status": bt.betty_status_string(st)},
+                       "replicas": 1 if strong else world,
+                       "parallelism": (f"rows of every batch sharded over {world} rank(s); parameters and solver state "
+                                       "replicated; one all-reduce (sum) of a parameter-sized vector per gradient, "
+                                       "Hessian-vector product and mixed product") if strong
+                       else f"{world} independent replica(s), no exchange in the data path",
+                       "cuda_graph": bool(use_graph), "device_status": bt.betty_status_string(st)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
     if per_config is not None:
         line["per_config"] = per_config

@@ -127,6 +127,29 @@ typedef struct {
   float tol;
 } betty_method_cfg;
 
+/* Data-parallel evaluation (Sec. 4 lists data-parallel training among the systems features; App. E reports
+ * its memory on 2 GPUs).  The rows of a problem's batch are partitioned over the ranks of a job, one GPU
+ * and one process per rank; parameters and all solver state are replicated.  Every cost here is a mean
+ * over the rows plus terms that do not depend on the data, so with row_weight_r = n_r / n (they sum to 1)
+ *     C = sum_r row_weight_r * C_r ,   C_r = the same cost evaluated on rank r's rows,
+ * and the same holds for every derivative of C.  A level whose `comm` is set is one rank's share of its
+ * problem: whenever the library has formed a gradient, a Hessian-vector product, a mixed product or the
+ * finite difference of gradients of that level's cost on the local rows, it multiplies the vector by
+ * row_weight and calls `allreduce`, which must replace the count floats at buf (DEVICE memory on the
+ * current device) by their sum over all ranks, ordered after the work already enqueued on `stream` and
+ * before work enqueued later (enqueue it on that stream, or synchronise around it), and return 0 on success
+ * (anything else makes the library call return BETTY_ERR_CUDA).  All ranks then hold the same bits and take
+ * the same solver steps.  The library never touches another GPU's memory: the exchange is entirely the
+ * caller's (torch.distributed / NCCL in the Python binding).  With `comm` set the fused forms (update in
+ * the reduction kernel or in a matrix product's epilogue, whole loops on chip) are replaced by their
+ * unfused equivalents; betty_hypergrad_itd and betty_engine_run return BETTY_ERR_UNSUPPORTED. */
+typedef int32_t (*betty_allreduce_fn)(void* user, float* buf, int64_t count, void* stream);
+typedef struct {
+  betty_allreduce_fn allreduce;
+  void* user;          /* passed back to allreduce */
+  float row_weight;    /* this rank's rows / all rows of the problem's batch */
+} betty_comm;
+
 /* One problem P_k. */
 typedef struct betty_level {
   int32_t loss;         /* betty_loss */
@@ -161,6 +184,7 @@ typedef struct betty_level {
                          * after the other, and averages their gradients before the optimiser step: the
                          * activations of one micro-batch are alive at a time.  0 or 1: off.  n must be a
                          * multiple of it (else BETTY_ERR_SHAPE).  Used by betty_lower_step and betty_engine_run. */
+  const betty_comm* comm; /* host; NULL: the level holds its problem's whole batch (see betty_comm) */
 } betty_level;
 
 /* Scratch bytes sufficient for any call below on these levels (Sec. 2: the whole program). */

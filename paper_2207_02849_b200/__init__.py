@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     betty_workspace_size, lib, lib_path,
 )
 from . import binding as _b
+from . import data_parallel  # noqa: F401
 
 for _k, _v in vars(_b).items():
     if _k.startswith(("BETTY_", "LOSS_", "PARAM_", "ACT_")):

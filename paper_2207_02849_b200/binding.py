@@ -36,6 +36,13 @@ class _MethodCfg(C.Structure):
                 ("tol", C.c_float)]
 
 
+_ALLREDUCE = C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p)
+
+
+class _Comm(C.Structure):
+    _fields_ = [("allreduce", _ALLREDUCE), ("user", C.c_void_p), ("row_weight", C.c_float)]
+
+
 class _Level(C.Structure):
     pass
 
@@ -49,7 +56,7 @@ _Level._fields_ = [
     ("weight_decay", C.c_float), ("opt_state", C.c_void_p), ("n_constraints", C.c_int32),
     ("constraints", C.POINTER(C.POINTER(_Level))),
     ("lr_schedule", C.c_int32), ("lr_step0", C.c_int32), ("lr_t_max", C.c_int32), ("lr_milestones", C.c_int32 * 4),
-    ("lr_gamma", C.c_float), ("lr_min", C.c_float), ("grad_accum", C.c_int32),
+    ("lr_gamma", C.c_float), ("lr_min", C.c_float), ("grad_accum", C.c_int32), ("comm", C.POINTER(_Comm)),
 ]
 
 class _Edge(C.Structure):
@@ -121,8 +128,14 @@ def betty_kernel_launches() -> int:
     return int(lib().betty_kernel_launches())
 
 
+_comm_error = [None]      # exception raised inside a data-parallel all-reduce callback, if any
+
+
 def _check(status: int, where: str):
     if status != BETTY_OK:
+        cause, _comm_error[0] = _comm_error[0], None
+        if cause is not None:
+            raise BettyError(status, where) from cause
         raise BettyError(status, where)
 
 
@@ -200,6 +213,29 @@ class Level:
         for i in range(4):
             self.c.lr_milestones[i] = int(milestones[i]) if i < len(milestones) else 0
         self.c.lr_gamma, self.c.lr_min = float(gamma), float(lr_min)
+        return self
+
+    def set_comm(self, allreduce, row_weight: float) -> "Level":
+        """Marks this level as one rank's share of its problem's batch (betty_comm).  `allreduce(ptr, count,
+        stream)` must sum `count` floats at device address `ptr` over all ranks, in place, ordered on the
+        CUDA stream handle `stream`; an exception it raises surfaces as BETTY_ERR_CUDA from the library call
+        (and is re-raised by the binding).  row_weight = this rank's rows / all rows.  None removes it."""
+        if allreduce is None:
+            self._comm = self._comm_cb = None
+            self.c.comm = None
+            return self
+        self.comm_error = None
+
+        def _cb(user, buf, count, stream):
+            try:
+                allreduce(int(buf), int(count), int(stream or 0))
+                return 0
+            except BaseException as e:           # never let an exception cross the C frames
+                self.comm_error = _comm_error[0] = e
+                return 1
+        self._comm_cb = _ALLREDUCE(_cb)
+        self._comm = _Comm(self._comm_cb, None, float(row_weight))
+        self.c.comm = C.pointer(self._comm)
         return self
 
     def set_grad_accum(self, n_micro: int) -> "Level":

@@ -8,6 +8,11 @@ namespace betty {
 
 std::atomic<unsigned long long> g_kernel_launches{0};
 
+std::mutex& smem_limit_mutex() {
+  static std::mutex m;
+  return m;
+}
+
 int current_device() {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return -1; }
@@ -129,11 +134,11 @@ betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
   return vec_zero(c, out, wrt->n_params);
 }
 
-betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu, VecHvpCache* cache) {
+betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu, VecHvpCache* cache, const LrTail* tail) {
   if (!vec_has_wd(L)) return BETTY_ERR_UNSUPPORTED;
   return logreg_pass(c, vec_family(L), (const float*)L->X, (const float*)L->y, L->n, L->d, L->params, u,
                      find_constraint(L, BETTY_PARAM_VECTOR)->params, Hu, nullptr, 0.f, cache ? cache->curv : nullptr,
-                     cache ? &cache->valid : nullptr);
+                     cache ? &cache->valid : nullptr, tail);
 }
 
 betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, const float* q, float* out) {
@@ -210,9 +215,19 @@ static betty_status check_ws(void* ws, size_t ws_bytes) {
   return BETTY_OK;
 }
 
+// Data-parallel levels (betty_comm): a vector formed from this rank's rows becomes the whole batch's by
+// weighting it with the rank's share of the rows and summing over the ranks.  The exchange is the caller's.
+static betty_status dp_reduce(Ctx& c, const betty_level* L, float* vec, int64_t n) {
+  if (!L->comm || n <= 0) return BETTY_OK;
+  if (!L->comm->allreduce) return BETTY_ERR_INVALID_ARG;
+  launch_pdl(k_scale_into, dim3(ew_grid(n)), dim3(256), 0, c.stream, vec, (const float*)vec, L->comm->row_weight, 0, n);
+  BETTY_LAUNCH_CHECK();
+  return L->comm->allreduce(L->comm->user, vec, n, (void*)c.stream) == 0 ? BETTY_OK : BETTY_ERR_CUDA;
+}
+
 static betty_status level_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out) {
-  if (is_vector_family(L->loss)) return vecfam_grad(c, L, wrt, out);
-  return mlpfam_grad(c, L, wrt, out);
+  BETTY_TRY(is_vector_family(L->loss) ? vecfam_grad(c, L, wrt, out) : mlpfam_grad(c, L, wrt, out));
+  return dp_reduce(c, L, out, wrt->n_params);
 }
 
 // Gradient of a step of a problem without lower problems: dC_L/d(own), taken over the whole batch at once
@@ -252,8 +267,19 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
   if (cfg.method == BETTY_FD) {
     BETTY_ALLOC(st, SolveState, c, 1);
     BETTY_TRY(vec_dot(c, v, v, n, &st->vnorm2, partials));
-    rc = vecfam ? vecfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, out, accumulate)
-                : mlpfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, out, accumulate);
+    float* dst = out;
+    if (L->comm) {           // local rows first, then the sum over ranks, then into out
+      dst = c.arena.alloc<float>((size_t)nc);
+      if (!dst) return BETTY_ERR_WORKSPACE;
+    }
+    const bool acc_local = accumulate && !L->comm;
+    rc = vecfam ? vecfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, dst, acc_local)
+                : mlpfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, dst, acc_local);
+    if (rc == BETTY_OK && L->comm) {
+      BETTY_TRY(dp_reduce(c, L, dst, nc));
+      launch_pdl(k_scale_into, dim3(ew_grid(nc)), dim3(256), 0, c.stream, out, (const float*)dst, 1.f, accumulate ? 1 : 0, nc);
+      BETTY_LAUNCH_CHECK();
+    }
     c.arena.release(mark);
     return rc;
   }
@@ -274,10 +300,29 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
     if (vecfam) {
       // term / sum recurrence; t_0 = s_0 = v are read straight from v in the first iteration: no copies
       BETTY_ALLOC(t, float, c, (size_t)n);
+      // the update t <- t - alpha H t, s <- s + t rides in the pass's reduction kernel (one rank: nothing
+      // comes between the product and its use)
       for (int k = 0; k < cfg.K; ++k) {
         const float* t_in = k == 0 ? v : t;
         const float* s_in = k == 0 ? v : q;
-        BETTY_TRY(vecfam_hvp(c, L, t_in, h, &vcache));
+        if (L->comm) {
+          BETTY_TRY(vecfam_hvp(c, L, t_in, h, &vcache));
+          BETTY_TRY(dp_reduce(c, L, h, n));
+          BETTY_TRY(neumann_update(c, t_in, s_in, h, cfg.alpha, t, q, n));
+          continue;
+        }
+        LrTail tail = {};
+        tail.kind = LR_TAIL_NEUMANN; tail.s_in = s_in; tail.t_out = t; tail.s_out = q; tail.alpha = cfg.alpha;
+        BETTY_TRY(vecfam_hvp(c, L, t_in, h, &vcache, &tail));
+      }
+    } else if (L->comm) {
+      // data-parallel MLP level: plain products, summed over ranks, then the term / sum recurrence
+      BETTY_ALLOC(t, float, c, (size_t)n);
+      for (int k = 0; k < cfg.K; ++k) {
+        const float* t_in = k == 0 ? v : t;
+        const float* s_in = k == 0 ? v : q;
+        BETTY_TRY(mlpfam_hvp(c, L, cache, t_in, h));
+        BETTY_TRY(dp_reduce(c, L, h, n));
         BETTY_TRY(neumann_update(c, t_in, s_in, h, cfg.alpha, t, q, n));
       }
     } else {
@@ -291,12 +336,23 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
     BETTY_ALLOC(r, float, c, (size_t)n);
     BETTY_ALLOC(p, float, c, (size_t)n);
     BETTY_TRY(cg_init(c, st, v, q, r, p, cfg.tol, n, partials));
+    // vector families of moderate width: the whole iteration after H p rides in the pass's reduction kernel
+    const bool fused = vecfam && !L->comm && n <= logreg_tail_max_d();
+    LrTail tail = {};
+    tail.kind = LR_TAIL_CG; tail.st = st; tail.q = q; tail.r = r; tail.p = p;
+    tail.partials = (double*)partials; tail.counter = (unsigned*)((double*)partials + 592) + 2;
     for (int k = 0; k < cfg.K; ++k) {
+      if (fused) {
+        BETTY_TRY(vecfam_hvp(c, L, p, h, &vcache, &tail));
+        continue;
+      }
       BETTY_TRY(vecfam ? vecfam_hvp(c, L, p, h, &vcache) : mlpfam_hvp(c, L, cache, p, h));
+      BETTY_TRY(dp_reduce(c, L, h, n));
       BETTY_TRY(cg_step(c, st, q, r, p, h, n, partials));
     }
   }
   BETTY_TRY(vecfam ? vecfam_mixed(c, L, wrt, q, m) : mlpfam_mixed(c, L, cache, wrt, q, m));
+  BETTY_TRY(dp_reduce(c, L, m, nc));
   launch_pdl(k_scale_into, dim3(ew_grid(nc)), dim3(256), 0, c.stream, out, m, -qscale, accumulate ? 1 : 0, nc);
   BETTY_LAUNCH_CHECK();
   c.arena.release(mark);
@@ -316,7 +372,7 @@ static betty_status hypergrad(const betty_level* lower, const betty_level* upper
   // Small logistic / least-squares bilevel pair: the whole hypergradient in one launch.
   if (vec_has_wd(lower) && (upper->loss == BETTY_LOSS_LOGREG || upper->loss == BETTY_LOSS_QUADRATIC) &&
       find_constraint(upper, BETTY_PARAM_VECTOR) == lower && wrt == find_constraint(lower, BETTY_PARAM_VECTOR) &&
-      cfg.K >= 0 && logreg_small_eligible(lower->n, upper->n, lower->d))
+      cfg.K >= 0 && !lower->comm && !upper->comm && logreg_small_eligible(lower->n, upper->n, lower->d))
     return logreg_small_hypergrad(c, vec_family(lower), (const float*)lower->X, (const float*)lower->y, lower->n,
                                   vec_family(upper), (const float*)upper->X, (const float*)upper->y, upper->n, lower->d,
                                   lower->params, wrt->params, cfg, out);
@@ -339,6 +395,7 @@ static betty_status hypergrad_itd(const betty_level* lower, const betty_level* u
   if (!wrt || !out || n_steps < 0) return BETTY_ERR_INVALID_ARG;
   if (!aligned16(out)) return BETTY_ERR_ALIGNMENT;
   if (lower->optimizer != BETTY_OPT_GD) return BETTY_ERR_UNSUPPORTED;   // the reverse sweep differentiates plain GD steps
+  if (lower->comm || upper->comm) return BETTY_ERR_UNSUPPORTED;          // not offered for data-parallel levels
   BETTY_TRY(check_ws(ws, ws_bytes));
   if (!is_participant(upper, lower) || !is_participant(upper, wrt) || !is_participant(lower, wrt) || wrt == lower)
     return BETTY_ERR_INVALID_ARG;
@@ -584,6 +641,7 @@ betty_status betty_engine_run(const betty_level* const* levels, int32_t n_levels
   for (int i = 0; i < n_levels; ++i) {
     BETTY_TRY(validate_level(levels[i]));
     if (unroll_steps[i] < 1) return BETTY_ERR_INVALID_ARG;
+    if (levels[i]->comm) return BETTY_ERR_UNSUPPORTED;                 // not offered for data-parallel levels
   }
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
@@ -678,7 +736,7 @@ betty_status betty_lower_step(const betty_level* L, int32_t n_steps, void* ws, s
   if (n_steps < 0) return BETTY_ERR_INVALID_ARG;
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
-  if (L->optimizer != BETTY_OPT_GD || L->grad_accum > 1) {
+  if (L->optimizer != BETTY_OPT_GD || L->grad_accum > 1 || L->comm) {
     BETTY_ALLOC(g, float, c, (size_t)L->n_params);
     for (int s = 0; s < n_steps; ++s) {
       BETTY_TRY(step_grad(c, L, g));
@@ -706,10 +764,14 @@ betty_status betty_hvp(const betty_level* L, const float* u, float* Hu, void* ws
   if (!aligned16(u) || !aligned16(Hu)) return BETTY_ERR_ALIGNMENT;
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
-  if (is_vector_family(L->loss)) return vecfam_hvp(c, L, u, Hu);
-  MlpHvpCache* cache = nullptr;
-  BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
-  return mlpfam_hvp(c, L, cache, u, Hu);
+  if (is_vector_family(L->loss)) {
+    BETTY_TRY(vecfam_hvp(c, L, u, Hu));
+  } else {
+    MlpHvpCache* cache = nullptr;
+    BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
+    BETTY_TRY(mlpfam_hvp(c, L, cache, u, Hu));
+  }
+  return dp_reduce(c, L, Hu, L->n_params);
 }
 
 betty_status betty_mixed_vjp(const betty_level* L, const betty_level* wrt, const float* q, float* out, void* ws,
@@ -719,10 +781,14 @@ betty_status betty_mixed_vjp(const betty_level* L, const betty_level* wrt, const
   if (!aligned16(q) || !aligned16(out)) return BETTY_ERR_ALIGNMENT;
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
-  if (is_vector_family(L->loss)) return vecfam_mixed(c, L, wrt, q, out);
-  MlpHvpCache* cache = nullptr;
-  BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
-  return mlpfam_mixed(c, L, cache, wrt, q, out);
+  if (is_vector_family(L->loss)) {
+    BETTY_TRY(vecfam_mixed(c, L, wrt, q, out));
+  } else {
+    MlpHvpCache* cache = nullptr;
+    BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
+    BETTY_TRY(mlpfam_mixed(c, L, cache, wrt, q, out));
+  }
+  return dp_reduce(c, L, out, wrt->n_params);
 }
 
 betty_status betty_hypergrad_neumann(const betty_level* lower, const betty_level* upper, const betty_level* wrt,

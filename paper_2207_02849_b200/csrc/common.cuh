@@ -5,6 +5,7 @@
 #include <stdint.h>
 #include <stddef.h>
 #include <atomic>
+#include <mutex>
 #include "betty.h"
 
 namespace betty {
@@ -83,8 +84,13 @@ struct SmemLimit {
   }
 };
 // Make `bytes` of dynamic shared memory launchable for `kernel` on the current device.
+// Several host threads may call the library at once (each on its own stream and workspace): the check and the
+// setting happen under one lock, so that no thread launches on the strength of a limit another thread has
+// recorded but not yet set.
+std::mutex& smem_limit_mutex();
 template <typename K>
 static inline betty_status ensure_dynamic_smem(K kernel, SmemLimit& lim, size_t bytes) {
+  std::lock_guard<std::mutex> guard(smem_limit_mutex());
   if (!lim.raise(current_device(), bytes)) return BETTY_OK;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
     (void)cudaGetLastError();

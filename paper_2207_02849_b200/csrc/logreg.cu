@@ -7,7 +7,7 @@
 // products and the scaled accumulation, and per-CTA column sums are reduced in a fixed order by a
 // small second kernel that also applies the weight-decay term and, for a lower-level step, the
 // gradient-descent update.
-#include "common.cuh"
+#include "ops.cuh"
 
 namespace betty {
 
@@ -88,21 +88,25 @@ __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
   float* red = (float*)(full + LR_S);     // [2][LR_WARPS][2*LR_R]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  float4 wv[NCH], uv[NCH], acc[NCH];
-#pragma unroll
-  for (int k = 0; k < NCH; ++k) {
-    int c4 = tid + k * LR_THREADS;
-    wv[k] = (NEEDZ && c4 < d4) ? __ldg((const float4*)a.w + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
-    uv[k] = (HVP && c4 < d4) ? __ldg((const float4*)a.u + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
-    acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-
   const int64_t ntiles = (a.n + LR_R - 1) / LR_R;
   if (tid == 0) {
     for (int s = 0; s < LR_S; ++s) mbar_init(&full[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // the barriers exist; everything below reads or writes global memory, which the previous kernel of the
+  // stream (the reduction that produced w or u) must have finished with
+  pdl_enter();
+
+  // w and u were written by an earlier kernel of the same stream: plain (coherent) loads, not the read-only path
+  float4 wv[NCH], uv[NCH], acc[NCH];
+#pragma unroll
+  for (int k = 0; k < NCH; ++k) {
+    int c4 = tid + k * LR_THREADS;
+    wv[k] = (NEEDZ && c4 < d4) ? *((const float4*)a.w + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    uv[k] = (HVP && c4 < d4) ? *((const float4*)a.u + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
 
   auto issue = [&](int s, int64_t t) {
     int64_t rows = a.n - t * LR_R; if (rows > LR_R) rows = LR_R;
@@ -242,10 +246,18 @@ __global__ void k_colacc(LrArgs a, const float* coef) {
   a.partials[(size_t)blockIdx.y * a.d + j] = acc;
 }
 
-// out_j = sum_c partials[c][j] + lam_j * vec_j ; optionally w_j <- w_j - lr * (that)
+// out_j = sum_c partials[c][j] + lam_j * vec_j ; optionally w_j <- w_j - lr * (that).
+// TAIL selects what else happens to the finished vector h (see LrTail): nothing; one term/sum update of the
+// Neumann series, elementwise, by the thread that owns the column; or one whole conjugate-gradient iteration,
+// done by the block that draws the last ticket once every block has stored its part of h.  The iteration's
+// arithmetic and its order of additions depend only on d, so results repeat bit for bit.
+template <int TAIL>
 __global__ void k_logreg_finalize(const float* partials, int nparts, int64_t d, const float* lam, const float* vec,
-                                  float* out, float* w_update, float lr) {
+                                  float* out, float* w_update, float lr, LrTail tl, StatusBlock* sb) {
+  pdl_enter();
   __shared__ float sh[8][32];
+  __shared__ double shd[8];
+  __shared__ int last_block;
   const int cx = threadIdx.x & 31, sl = threadIdx.x >> 5;
   const int64_t j = blockIdx.x * 32 + cx;
   float acc = 0.f;
@@ -256,14 +268,98 @@ __global__ void k_logreg_finalize(const float* partials, int nparts, int64_t d, 
   }
   sh[sl][cx] = acc;
   __syncthreads();
+  double ph = 0.0;          // CG: this column's term of p . h
   if (sl == 0 && j < d) {
     float g = 0.f;
 #pragma unroll
     for (int s = 0; s < 8; ++s) g += sh[s][cx];
-    if (lam) g += lam[j] * vec[j];
+    const float vj = (lam || TAIL != LR_TAIL_NONE) ? vec[j] : 0.f;
+    if (lam) g += lam[j] * vj;
     if (out) out[j] = g;
     if (w_update) w_update[j] = w_update[j] - lr * g;
+    if (TAIL == LR_TAIL_NEUMANN) {
+      const float tn = vj - tl.alpha * g;
+      const float sn = tl.s_in[j] + tn;
+      tl.t_out[j] = tn;
+      tl.s_out[j] = sn;
+    }
+    if (TAIL == LR_TAIL_CG) ph = (double)vj * (double)g;
   }
+  if (TAIL != LR_TAIL_CG) return;
+  // ---- conjugate gradient: gamma = p . h in fixed order, then the update by the last block
+  if (sl == 0) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ph += __shfl_xor_sync(0xffffffffu, ph, o);
+    if (cx == 0) {
+      tl.partials[blockIdx.x] = ph;
+      __threadfence();
+      last_block = atomicAdd(tl.counter, 1u) == gridDim.x - 1 ? 1 : 0;
+    }
+  }
+  __syncthreads();
+  if (!last_block) return;
+  __threadfence();
+  SolveState* st = tl.st;
+  __shared__ int s_active;
+  __shared__ float s_rho;
+  if (threadIdx.x == 0) { *tl.counter = 0u; s_active = st->active; s_rho = st->rho; }
+  __syncthreads();
+  if (!s_active) return;                         // the solve has stopped: h was stored, nothing else moves
+  double gsum = 0.0;
+  for (unsigned i = 0; i < gridDim.x; ++i) gsum += ((volatile double*)tl.partials)[i];   // same order in every thread
+  const float gamma = (float)gsum;
+  if (!isfinite(gsum) || !(gsum > 0.0)) {
+    if (threadIdx.x == 0) {
+      st->gamma = gamma;
+      record_status(sb, !isfinite(gsum) ? BETTY_ERR_NONFINITE : BETTY_ERR_BREAKDOWN);
+      st->active = 0;
+    }
+    return;
+  }
+  const float rho = s_rho;
+  const float a = rho / gamma;
+  const float* h = out;
+  double rr = 0.0;
+  for (int64_t i = threadIdx.x; i < d; i += blockDim.x) {
+    const float pi = tl.p[i];
+    tl.q[i] += a * pi;
+    const float ri = tl.r[i] - a * __ldcg(h + i);
+    tl.r[i] = ri;
+    rr += (double)ri * (double)ri;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) rr += __shfl_xor_sync(0xffffffffu, rr, o);
+  if (cx == 0) shd[sl] = rr;
+  __syncthreads();
+  double rsum = 0.0;
+  for (int i = 0; i < 8; ++i) rsum += shd[i];
+  const float rho_new = (float)rsum;
+  const float beta = rho_new / rho;
+  for (int64_t i = threadIdx.x; i < d; i += blockDim.x) tl.p[i] = tl.r[i] + beta * tl.p[i];
+  if (threadIdx.x == 0) {
+    st->gamma = gamma;
+    st->rho_new = rho_new;
+    st->rho = rho_new;
+    st->iters += 1;
+    sb->cg_iters = st->iters;
+    if (!isfinite(rho_new)) { record_status(sb, BETTY_ERR_NONFINITE); st->active = 0; }
+    else if (rho_new <= st->stop) st->active = 0;
+  }
+}
+
+int64_t logreg_tail_max_d() { return 32 * 592; }     // one double per 32 columns in a 592-entry reduction buffer
+
+static betty_status launch_finalize(Ctx& c, const float* partials, int nparts, int64_t d, const float* lam, const float* vec,
+                                    float* out, float* w_update, float lr, const LrTail* tail) {
+  LrTail tl = {};
+  if (tail) tl = *tail;
+  const dim3 grid((unsigned)((d + 31) / 32)), block(256);
+  StatusBlock* sb = c.arena.status();
+  if (tl.kind == LR_TAIL_CG) launch_pdl(k_logreg_finalize<LR_TAIL_CG>, grid, block, 0, c.stream, partials, nparts, d, lam, vec, out, w_update, lr, tl, sb);
+  else if (tl.kind == LR_TAIL_NEUMANN) launch_pdl(k_logreg_finalize<LR_TAIL_NEUMANN>, grid, block, 0, c.stream, partials, nparts, d, lam, vec, out, w_update, lr, tl, sb);
+  else launch_pdl(k_logreg_finalize<LR_TAIL_NONE>, grid, block, 0, c.stream, partials, nparts, d, lam, vec, out, w_update, lr, tl, sb);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
 }
 
 template <int NCH, int FORM>
@@ -272,7 +368,7 @@ static betty_status launch_stream(Ctx& c, const LrArgs& a, int grid) {
   auto kern = k_logreg_stream<NCH, FORM>;
   static SmemLimit limit = {};      // per instantiation and per device; raised again if a wider problem comes
   BETTY_TRY(ensure_dynamic_smem(kern, limit, smem));
-  kern<<<grid, LR_THREADS, smem, c.stream>>>(a);
+  launch_pdl(kern, dim3(grid), dim3(LR_THREADS), smem, c.stream, a);
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
@@ -282,7 +378,7 @@ static betty_status launch_stream(Ctx& c, const LrArgs& a, int grid) {
 // decremented by lr times it.
 betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
                          const float* u, const float* lam, float* out, float* w_update, float lr, float* curv,
-                         bool* curv_valid) {
+                         bool* curv_valid, const LrTail* tail) {
   if (d <= 0) return BETTY_OK;
   LrArgs a;
   a.X = X; a.y = y; a.n = n; a.d = d; a.w = w; a.u = u; a.family = family;
@@ -319,8 +415,8 @@ betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int
     k_colacc<<<g, 256, 0, c.stream>>>(a, coef);
     BETTY_LAUNCH_CHECK();
   }
-  k_logreg_finalize<<<(unsigned)((d + 31) / 32), 256, 0, c.stream>>>(a.partials, nparts, d, lam, u ? u : w, out, w_update, lr);
-  BETTY_LAUNCH_CHECK();
+  if (tail && tail->kind != LR_TAIL_NONE && (!u || !out)) return BETTY_ERR_INVALID_ARG;   // tails act on an HVP's result
+  BETTY_TRY(launch_finalize(c, a.partials, nparts, d, lam, u ? u : w, out, w_update, lr, tail));
   c.arena.release(mark);
   return BETTY_OK;
 }
@@ -407,8 +503,7 @@ extern "C" betty_status betty_hvp_logreg_static(const float* X, int64_t n, int64
   else if (d <= 2048) st = launch_stream<2, LR_HVP>(c, a, grid);
   else st = launch_stream<4, LR_HVP>(c, a, grid);
   if (st != BETTY_OK) return st;
-  k_logreg_finalize<<<(unsigned)((d + 31) / 32), 256, 0, s>>>(a.partials, grid, d, lam, u, Hu, nullptr, 0.f);
-  BETTY_LAUNCH_CHECK();
+  if ((st = launch_finalize(c, a.partials, grid, d, lam, u, Hu, nullptr, 0.f, nullptr)) != BETTY_OK) return st;
   if (status_dev) {
     k_noalloc_report<<<1, 32, 0, s>>>(a.sb, status_dev);
     BETTY_LAUNCH_CHECK();

@@ -24,12 +24,26 @@ static inline bool is_mlp_family(int loss) {
 }
 
 // logreg.cu
+// What the pass's reduction kernel does with the finished product h = H u besides storing it: the solver update
+// that would otherwise be one to three more small kernels between two passes over the matrix.
+enum { LR_TAIL_NONE = 0, LR_TAIL_NEUMANN = 1, LR_TAIL_CG = 2 };
+struct LrTail {
+  int kind;
+  // LR_TAIL_NEUMANN (the pass's direction u is the current term t):  t_out = u - alpha*h,  s_out = s_in + t_out
+  const float* s_in; float* t_out; float* s_out; float alpha;
+  // LR_TAIL_CG (the pass's direction u is p): gamma = p.h; a = rho/gamma; q += a p; r -= a h; rho' = r.r;
+  // p = r + (rho'/rho) p; the state advances as in cg_step.  partials holds one double per 32 columns,
+  // counter is a zeroed ticket (both from the solve's reduction buffer).
+  SolveState* st; float* q; float* r; float* p; double* partials; unsigned* counter;
+};
+// number of 32-column blocks the fused CG iteration can take (size of a reduction buffer)
+int64_t logreg_tail_max_d();
 // curv / curv_valid: the per-row curvature buffer of one solve and whether it holds the curvature at w.  A pass
 // reads it only when *curv_valid is set and sets *curv_valid only when it has itself written the buffer (the
 // single-pass kernel in its full HVP form); the two-pass fallback neither reads nor writes it.
 betty_status logreg_pass(Ctx& c, int family, const float* X, const float* y, int64_t n, int64_t d, const float* w,
                          const float* u, const float* lam, float* out, float* w_update, float lr, float* curv = nullptr,
-                         bool* curv_valid = nullptr);
+                         bool* curv_valid = nullptr, const LrTail* tail = nullptr);
 
 // logreg_small.cu: whole-loop kernels for problems that fit a cluster's shared memory
 bool logreg_small_eligible(int64_t n, int64_t nv, int64_t d, int64_t unrolled_steps = 0);
@@ -48,7 +62,8 @@ betty_status vecfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
 // Per-row curvature of a logistic level at its present parameters, shared by the HVPs of one solve: the first
 // HVP fills it, the later ones read it (n floats in the caller's workspace; null: every HVP recomputes z = X w).
 struct VecHvpCache { float* curv; bool valid; };
-betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu, VecHvpCache* cache = nullptr);
+betty_status vecfam_hvp(Ctx& c, const betty_level* L, const float* u, float* Hu, VecHvpCache* cache = nullptr,
+                        const LrTail* tail = nullptr);
 betty_status vecfam_mixed(Ctx& c, const betty_level* L, const betty_level* wrt, const float* q, float* out);
 betty_status vecfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step = 0);
 // out (+)= -alpha*[dC/dc(x+eps v) - dC/dc(x-eps v)]/(2 eps), eps = eps0/sqrt(*vnorm2) on the device
