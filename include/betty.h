@@ -92,7 +92,7 @@ typedef enum {
 
 typedef enum { BETTY_NEUMANN = 0, BETTY_CG = 1, BETTY_FD = 2 } betty_method;
 typedef enum { BETTY_ACT_RELU = 0, BETTY_ACT_GELU = 1 } betty_activation; /* GELU: erf form */
-typedef enum { BETTY_F32 = 0, BETTY_BF16 = 1, BETTY_I32 = 2 } betty_dtype;
+typedef enum { BETTY_F32 = 0, BETTY_BF16 = 1, BETTY_I32 = 2, BETTY_F16 = 3 } betty_dtype;
 
 /* How a problem's gradient step is taken (the paper lets each problem bring its own optimiser: SGD with
  * momentum and weight decay for the classifiers, Adam for the weight net, App. C).
@@ -185,6 +185,18 @@ typedef struct betty_level {
                          * activations of one micro-batch are alive at a time.  0 or 1: off.  n must be a
                          * multiple of it (else BETTY_ERR_SHAPE).  Used by betty_lower_step and betty_engine_run. */
   const betty_comm* comm; /* host; NULL: the level holds its problem's whole batch (see betty_comm) */
+  int32_t precision;    /* MLP own block: operand type of its matrix products (Sec. 4, mixed precision): BETTY_BF16
+                         * (0 means the same) or BETTY_F16, fp32 accumulation and fp32 master parameters either way.
+                         * Every cost the block takes part in must bring its batch X in that type (x_dtype). */
+  float* loss_scale;    /* device fp32[4], caller-owned, or NULL: loss scaling for the steps betty_lower_step takes on
+                         * a BETTY_F16 block (the paper's fp16 option; a half-precision backward pass loses small
+                         * gradients to underflow unless the loss is scaled up).  [0] scale S > 0, [1] steps taken in a
+                         * row without overflow, [2] growth interval G (0: the scale is static), [3] steps skipped so far.
+                         * Each step: the top-layer deltas are multiplied by S, the gradient divided by S; if it holds a
+                         * non-finite value (a 16-bit delta overflowed) the update is skipped, S is halved, [1] returns
+                         * to 0 and [3] counts up; otherwise the optimiser step is taken, [1] counts up, and when it
+                         * reaches G > 0 the scale doubles and [1] returns to 0.  All of it stays on the device.
+                         * Other calls on the block run unscaled.  Not offered by betty_engine_run. */
 } betty_level;
 
 /* Scratch bytes sufficient for any call below on these levels (Sec. 2: the whole program). */

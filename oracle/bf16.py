@@ -1,5 +1,6 @@
-"""Round-to-nearest-even conversion to bfloat16 precision, written from the format's
-definition (1 sign, 8 exponent, 7 mantissa bits = the upper half of an IEEE binary32)."""
+"""Round-to-nearest-even conversion to the two 16-bit operand formats: bfloat16, written from the format's
+definition (1 sign, 8 exponent, 7 mantissa bits = the upper half of an IEEE binary32), and IEEE binary16
+(1 sign, 5 exponent, 10 mantissa bits), for which numpy's own conversion is the library step."""
 import numpy as np
 
 
@@ -16,3 +17,13 @@ def round_to_bf16(a: np.ndarray) -> np.ndarray:
     finite = np.isfinite(f)
     out = np.where(finite, out, f)
     return out.astype(np.float64).reshape(np.shape(a))
+
+
+FP16_MAX = 65504.0          # largest finite binary16 value; magnitudes from 65520 up round to infinity
+
+
+def round_to_fp16(a: np.ndarray) -> np.ndarray:
+    """Return `a` rounded to binary32 and then to the nearest IEEE binary16 value (ties to even, overflow
+    to infinity, gradual underflow), as fp64."""
+    with np.errstate(over="ignore"):
+        return np.asarray(a, dtype=np.float32).astype(np.float16).astype(np.float64).reshape(np.shape(a))

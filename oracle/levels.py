@@ -31,7 +31,7 @@ from typing import Optional
 import numpy as np
 from scipy.special import erf, expit
 
-from .bf16 import round_to_bf16
+from .bf16 import round_to_bf16, round_to_fp16
 
 WN_H = 100  # hidden width of the 1-100-1 weight net (App. C, "Meta-Weight-Network")
 
@@ -50,6 +50,8 @@ class Level:
     mu: float = 0.0
     bf16: bool = False                 # MLP matrices are used through a bf16-rounded copy
     quant: str = "operands"            # what a bf16 level rounds: "operands" | "weights" (see _mlp_ce_state)
+    operand_dtype: str = "bf16"        # 16-bit format of a mixed-precision level: "bf16" | "fp16"
+    loss_scale: Optional[list] = None  # fp16 levels: [scale, good steps, growth interval, skipped steps] (solvers.lower_step)
     constraints: list = field(default_factory=list)
     optimizer: str = "gd"              # 'gd' | 'momentum' | 'adam' (App. C: SGD with momentum / Adam per problem)
     momentum: float = 0.0
@@ -143,16 +145,26 @@ def mlp_pack(Ws, bs):
     return np.concatenate([np.concatenate([W.reshape(-1), b.reshape(-1)]) for W, b in zip(Ws, bs)])
 
 
+def _round16(level: Level):
+    """Rounding to the level's 16-bit operand format."""
+    if level.operand_dtype == "bf16":
+        return round_to_bf16
+    if level.operand_dtype == "fp16":
+        return round_to_fp16
+    raise ValueError(level.operand_dtype)
+
+
 def _mlp_weights(level: Level, flat):
-    """The copy of the parameters the cost is evaluated at: matrices rounded to bf16 for
-    mixed-precision levels, biases as they are."""
+    """The copy of the parameters the cost is evaluated at: matrices rounded to the 16-bit operand
+    format for mixed-precision levels, biases as they are."""
     Ws, bs = mlp_unpack(level.widths, flat)
     if level.bf16:
-        Ws = [round_to_bf16(W) for W in Ws]
+        rnd = _round16(level)
+        Ws = [rnd(W) for W in Ws]
     return Ws, bs
 
 
-def _mlp_forward(Ws, bs, X, act, quant=False, offsets=None):
+def _mlp_forward(Ws, bs, X, act, quant=False, offsets=None, rnd=round_to_bf16):
     """h[l] is the input of layer l (h[0] = X), a[l] its pre-activation; logits = a[-1].
 
     Mixed-precision levels (quant=True) feed every matrix product bf16 operands, so each hidden
@@ -168,7 +180,7 @@ def _mlp_forward(Ws, bs, X, act, quant=False, offsets=None):
             if offsets is not None:
                 hn = hn + offsets[l]
             elif quant:
-                hq = round_to_bf16(hn)
+                hq = rnd(hn)
                 offs.append(hq - hn)
                 hn = hq
             h.append(hn)
@@ -285,14 +297,14 @@ def _mlp_ce_state(L: Level, over):
         h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation)
     elif frozen and M.bf16:
         Wb, bb = _mlp_weights(M, M.params)
-        _, _, offs = _mlp_forward(Wb, bb, L.X, M.activation, quant=True)
+        _, _, offs = _mlp_forward(Wb, bb, L.X, M.activation, quant=True, rnd=_round16(M))
         Wd, bd = mlp_unpack(M.widths, flat - M.params)
         Ws = [W0 + dW for W0, dW in zip(Wb, Wd)]
         bs = [b0 + db for b0, db in zip(bb, bd)]
         h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation, offsets=offs)
     else:
         Ws, bs = _mlp_weights(M, flat)
-        h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation, quant=M.bf16 and not plain)
+        h, a, _ = _mlp_forward(Ws, bs, L.X, M.activation, quant=M.bf16 and not plain, rnd=_round16(M))
     p, ell = _softmax_ce(a[-1], np.asarray(L.y, dtype=np.int64))
     return M, Ws, bs, h, a, p, ell
 
@@ -421,6 +433,20 @@ def grad(L: Level, wrt: Level, over=None) -> np.ndarray:
             return mlp_pack(gW, gb)
         return np.zeros(n_out)
     raise ValueError(L.loss)
+
+
+def largest_backward_operand(L: Level, over=None) -> float:
+    """max over layers and entries of |delta_l| = |dC_L/da_l| in the gradient of the reweighted cross-entropy
+    with respect to its own classifier: the quantities a mixed-precision backward pass holds in 16 bits.
+    With fp16 operands and loss scale S, a step overflows when S times this reaches the format's range."""
+    if L.loss != "mlp_ce_reweight":
+        raise ValueError("loss scaling is defined for the classifier's own reweighted cross-entropy")
+    M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+    B = L.X.shape[0]
+    r, _ = _reweight_r(L, ell, over)
+    delta_top = (r / B)[:, None] * (p - _onehot(np.asarray(L.y, np.int64), p.shape[1]))
+    _, _, deltas, _ = _mlp_backward(Ws, h, a, delta_top, M.activation)
+    return float(max(np.max(np.abs(d)) for d in deltas))
 
 
 def hvp(L: Level, u: np.ndarray, over=None) -> np.ndarray:

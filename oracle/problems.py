@@ -23,12 +23,12 @@ def quadratic_levels(A, b, lam, Av, bv, w0=None):
     return lo, up
 
 
-def reweight_levels(inp, bf16=True, quant="operands"):
+def reweight_levels(inp, bf16=True, quant="operands", operand_dtype="bf16"):
     theta = Level(loss="mlp_ce", param_kind="weightnet", params=inp.theta, X=inp.val.X,
                   y=inp.val.y)
     w = Level(loss="mlp_ce_reweight", param_kind="mlp", params=inp.w, X=inp.train.X,
               y=inp.train.y, widths=inp.widths, activation=inp.activation, lr=inp.lr,
-              bf16=bf16, quant=quant, constraints=[theta])
+              bf16=bf16, quant=quant, operand_dtype=operand_dtype, constraints=[theta])
     theta.constraints = [w]
     return w, theta
 

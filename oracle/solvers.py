@@ -101,7 +101,34 @@ def lower_step(L: Level, n_steps: int) -> None:
     For mixed-precision levels the gradient is taken at the bf16-rounded copy of the
     current master, which is re-derived at every step."""
     for s in range(int(n_steps)):
-        apply_optimizer(L, step_gradient(L), s)
+        g = step_gradient(L)
+        if L.loss_scale is not None and not _loss_scaled_step_is_taken(L):
+            continue
+        apply_optimizer(L, g, s)
+
+
+FP16_OVERFLOW = 65520.0      # magnitudes from here up round to infinity in IEEE binary16
+
+
+def _loss_scaled_step_is_taken(L: Level) -> bool:
+    """Loss scaling of a half-precision level (Sec. 4 lists mixed precision; the paper's listings switch it on
+    with an fp16 flag and leave the scaling rule to the framework; the rule here is the usual dynamic one).
+    State L.loss_scale = [S, good, G, skipped].  The backward pass multiplies its top-layer deltas by S and the
+    gradient is divided by S again, which changes nothing in exact arithmetic, so only the overflow decision
+    is modelled: the step overflows when S times the largest 16-bit backward operand rounds to infinity.  Then
+    the update is skipped, S halves, `good` returns to 0 and `skipped` counts up.  Otherwise the step is
+    taken, `good` counts up and, when it reaches G > 0, S doubles and `good` returns to 0."""
+    st = L.loss_scale
+    if st[0] * _lv.largest_backward_operand(L) >= FP16_OVERFLOW:
+        st[0] *= 0.5
+        st[1] = 0
+        st[3] += 1
+        return False
+    st[1] += 1
+    if st[2] > 0 and st[1] >= st[2]:
+        st[0] *= 2.0
+        st[1] = 0
+    return True
 
 
 def neumann_solve(hv, v, K: int, alpha: float) -> np.ndarray:

@@ -20,7 +20,7 @@ BETTY_OK = 0
 PARAM_VECTOR, PARAM_MLP, PARAM_WEIGHTNET, PARAM_LOGWD = range(4)
 BETTY_NEUMANN, BETTY_CG, BETTY_FD = range(3)
 ACT_RELU, ACT_GELU = range(2)
-BETTY_F32, BETTY_BF16, BETTY_I32 = range(3)
+BETTY_F32, BETTY_BF16, BETTY_I32, BETTY_F16 = range(4)
 BETTY_OPT_GD, BETTY_OPT_MOMENTUM, BETTY_OPT_ADAM = range(3)
 BETTY_LR_CONSTANT, BETTY_LR_MULTISTEP, BETTY_LR_COSINE = range(3)
 
@@ -57,6 +57,7 @@ _Level._fields_ = [
     ("constraints", C.POINTER(C.POINTER(_Level))),
     ("lr_schedule", C.c_int32), ("lr_step0", C.c_int32), ("lr_t_max", C.c_int32), ("lr_milestones", C.c_int32 * 4),
     ("lr_gamma", C.c_float), ("lr_min", C.c_float), ("grad_accum", C.c_int32), ("comm", C.POINTER(_Comm)),
+    ("precision", C.c_int32), ("loss_scale", C.c_void_p),
 ]
 
 class _Edge(C.Structure):
@@ -153,7 +154,7 @@ def _stream(stream) -> int:
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 
-_DT = {torch.float32: BETTY_F32, torch.bfloat16: BETTY_BF16, torch.int32: BETTY_I32}
+_DT = {torch.float32: BETTY_F32, torch.bfloat16: BETTY_BF16, torch.int32: BETTY_I32, torch.float16: BETTY_F16}
 
 
 class Level:
@@ -236,6 +237,23 @@ class Level:
         self._comm_cb = _ALLREDUCE(_cb)
         self._comm = _Comm(self._comm_cb, None, float(row_weight))
         self.c.comm = C.pointer(self._comm)
+        return self
+
+    def set_precision(self, dtype: int) -> "Level":
+        """Operand type of an MLP block's matrix products: BETTY_BF16 (default) or BETTY_F16."""
+        self.c.precision = int(dtype)
+        return self
+
+    def set_loss_scale(self, scale: Optional[float], growth_interval: int = 0) -> "Level":
+        """Loss scaling of the lower steps of a BETTY_F16 block: allocates the four-float device state
+        [scale, good steps, growth interval, skipped steps] (see betty.h); None switches it off."""
+        if scale is None:
+            self.loss_scale_state = None
+            self.c.loss_scale = None
+            return self
+        self.loss_scale_state = torch.tensor([float(scale), 0.0, float(growth_interval), 0.0], dtype=torch.float32,
+                                             device=self.params.device)
+        self.c.loss_scale = _ptr(self.loss_scale_state)
         return self
 
     def set_grad_accum(self, n_micro: int) -> "Level":

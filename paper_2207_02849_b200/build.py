@@ -12,6 +12,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libbetty.so")
 SOURCES = ["api.cu", "vec.cu", "logreg.cu", "logreg_small.cu", "mlp.cu", "gemm.cu", "gemm_tc.cu"]
+FAMILY_SOURCES = ["mlp.cu", "gemm.cu", "gemm_tc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--use_fast_math", "-Xcompiler", "-fPIC",
@@ -43,12 +44,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
     build_dir = os.path.join(PKG_DIR, "_build")
     os.makedirs(build_dir, exist_ok=True)
     procs = []
-    for src in SOURCES:
-        obj = os.path.join(build_dir, src.replace(".cu", ".o"))
-        cmd = [nvcc, "-c", os.path.join(CSRC, src), "-o", obj] + NVCC_FLAGS
+    # the MLP family sources are compiled twice: bfloat16 operands (default) and IEEE half operands
+    units = [(src, "", []) for src in SOURCES] + [(src, "_f16", ["-DBETTY_FP16_OPERANDS"]) for src in FAMILY_SOURCES]
+    for src, suffix, extra in units:
+        obj = os.path.join(build_dir, src.replace(".cu", suffix + ".o"))
+        cmd = [nvcc, "-c", os.path.join(CSRC, src), "-o", obj] + NVCC_FLAGS + extra
         if verbose:
             cmd += ["-Xptxas", "-v"]
-        procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+        procs.append((src + suffix, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     for src, p in procs:
         out, _ = p.communicate()

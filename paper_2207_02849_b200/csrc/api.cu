@@ -8,6 +8,47 @@ namespace betty {
 
 std::atomic<unsigned long long> g_kernel_launches{0};
 
+// ------------------------------------------------------------------ MLP families: one per 16-bit operand type
+// The classifier block that takes part in a cost decides which build of the family serves the call.
+static inline bool mlp_f16(const betty_level* L) {
+  const betty_level* M = find_participant(L, BETTY_PARAM_MLP);
+  return M && M->precision == BETTY_F16;
+}
+#define BETTY_MLP_DISPATCH(L, call) (mlp_f16(L) ? fam_f16::call : fam_bf16::call)
+static betty_status mlpfam_validate(const betty_level* L) { return BETTY_MLP_DISPATCH(L, mlpfam_validate(L)); }
+static size_t mlpfam_workspace(const betty_level* L) { return BETTY_MLP_DISPATCH(L, mlpfam_workspace(L)); }
+static betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_grad(c, L, wrt, out));
+}
+static betty_status mlpfam_share_weights(Ctx& c, const betty_level* M) {
+  return (M && M->precision == BETTY_F16) ? fam_f16::mlpfam_share_weights(c, M) : fam_bf16::mlpfam_share_weights(c, M);
+}
+static void mlpfam_unshare_weights(Ctx& c) { c.shared.master = nullptr; }
+static betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_hvp_begin(c, L, cache));
+}
+static betty_status mlpfam_hvp_keep_direction(Ctx& c, const betty_level* L, MlpHvpCache* cache) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_hvp_keep_direction(c, cache));
+}
+static betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* u, float* Hu) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_hvp(c, L, cache, u, Hu));
+}
+static betty_status mlpfam_hvp_series(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* sv, const float* v,
+                                      float alpha, float* s_out) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_hvp_series(c, L, cache, sv, v, alpha, s_out));
+}
+static betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* cache, const betty_level* wrt, const float* q,
+                                 float* out) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_mixed(c, L, cache, wrt, q, out));
+}
+static betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step = 0) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_lower_step(c, L, n_steps, first_step));
+}
+static betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
+                              float eps0, float alpha, float* out, bool accumulate) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_fd(c, L, wrt, v, vnorm2, eps0, alpha, out, accumulate));
+}
+
 std::mutex& smem_limit_mutex() {
   static std::mutex m;
   return m;
@@ -56,8 +97,10 @@ __global__ void k_fd_weight_decay(float* out, const float* w, const float* v, co
   }
 }
 // optimiser steps (see betty_optimizer); the step counter of Adam is the float behind the two moments
-__global__ void k_opt_momentum(float* x, const float* g, float* buf, float lr, float mom, float wd, int64_t n) {
+// `skip` (nullable, device): a step whose gradient overflowed under loss scaling is not taken
+__global__ void k_opt_momentum(float* x, const float* g, float* buf, float lr, float mom, float wd, int64_t n, const int* skip) {
   pdl_enter();
+  if (skip && *skip) return;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     const float gg = g[i] + wd * x[i];
     const float b = mom * buf[i] + gg;
@@ -66,8 +109,9 @@ __global__ void k_opt_momentum(float* x, const float* g, float* buf, float lr, f
   }
 }
 __global__ void k_opt_adam(float* x, const float* g, float* m, float* v, const float* tcount, float lr, float b1, float b2,
-                           float eps, float wd, int64_t n) {
+                           float eps, float wd, int64_t n, const int* skip) {
   pdl_enter();
+  if (skip && *skip) return;
   const float t = *tcount + 1.f;                       // this step's index; the counter is advanced afterwards
   const float c1 = 1.f - powf(b1, t), c2 = 1.f - powf(b2, t);
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
@@ -78,14 +122,36 @@ __global__ void k_opt_adam(float* x, const float* g, float* m, float* v, const f
     x[i] -= lr * (mi / c1) / (sqrtf(vi / c2) + eps);
   }
 }
-__global__ void k_opt_tick(float* tcount) {
+__global__ void k_opt_tick(float* tcount, const int* skip) {
   pdl_enter();
+  if (skip && *skip) return;
   *tcount += 1.f;
 }
-__global__ void k_opt_gd(float* x, const float* g, float lr, int64_t n) {
+__global__ void k_opt_gd(float* x, const float* g, float lr, int64_t n, const int* skip) {
   pdl_enter();
+  if (skip && *skip) return;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     x[i] -= lr * g[i];
+}
+// Loss scaling (betty_level.loss_scale = [S, good steps, growth interval, skipped steps]).
+// g <- g / S; *flag |= any element non-finite (the flag is zeroed by the caller before the launch)
+__global__ void k_unscale_check(float* g, int64_t n, const float* state, int* flag) {
+  pdl_enter();
+  const float inv = 1.f / state[0];
+  int bad = 0;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const float v = g[i] * inv;
+    g[i] = v;
+    if (!isfinite(v)) bad = 1;
+  }
+  if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(flag, 1);
+}
+// overflow: halve the scale, count the skipped step; else count the good step and double the scale every G of them
+__global__ void k_loss_scale_update(float* state, const int* flag) {
+  pdl_enter();
+  if (*flag) { state[0] *= 0.5f; state[1] = 0.f; state[3] += 1.f; return; }
+  state[1] += 1.f;
+  if (state[2] > 0.f && state[1] >= state[2]) { state[0] *= 2.f; state[1] = 0.f; }
 }
 static inline int ew_grid(int64_t n) {
   int64_t b = (n + 1023) / 1024;
@@ -168,20 +234,20 @@ betty_status vecfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
 }
 
 // params of L <- one optimiser step along gradient g
-static betty_status apply_optimizer(Ctx& c, const betty_level* L, const float* g, int step_in_call) {
+static betty_status apply_optimizer(Ctx& c, const betty_level* L, const float* g, int step_in_call, const int* skip = nullptr) {
   const float lr = lr_at(L, step_in_call);
   const int64_t n = L->n_params;
   if (n <= 0) return BETTY_OK;
   const int grid = (int)((n + 1023) / 1024 < 1 ? 1 : ((n + 1023) / 1024 > 2368 ? 2368 : (n + 1023) / 1024));
   if (L->optimizer == BETTY_OPT_GD) {
-    launch_pdl(k_opt_gd, dim3(grid), dim3(256), 0, c.stream, L->params, g, lr, n);
+    launch_pdl(k_opt_gd, dim3(grid), dim3(256), 0, c.stream, L->params, g, lr, n, skip);
   } else if (L->optimizer == BETTY_OPT_MOMENTUM) {
-    launch_pdl(k_opt_momentum, dim3(grid), dim3(256), 0, c.stream, L->params, g, L->opt_state, lr, L->momentum, L->weight_decay, n);
+    launch_pdl(k_opt_momentum, dim3(grid), dim3(256), 0, c.stream, L->params, g, L->opt_state, lr, L->momentum, L->weight_decay, n, skip);
   } else {
     float* m = L->opt_state; float* v = m + n; float* t = v + n;
-    launch_pdl(k_opt_adam, dim3(grid), dim3(256), 0, c.stream, L->params, g, m, v, t, lr, L->beta1, L->beta2, L->adam_eps, L->weight_decay, n);
+    launch_pdl(k_opt_adam, dim3(grid), dim3(256), 0, c.stream, L->params, g, m, v, t, lr, L->beta1, L->beta2, L->adam_eps, L->weight_decay, n, skip);
     BETTY_LAUNCH_CHECK();
-    launch_pdl(k_opt_tick, dim3(1), dim3(1), 0, c.stream, t);
+    launch_pdl(k_opt_tick, dim3(1), dim3(1), 0, c.stream, t, skip);
   }
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
@@ -197,6 +263,9 @@ static betty_status validate_level(const betty_level* L) {
   if (L->param_kind < BETTY_PARAM_VECTOR || L->param_kind > BETTY_PARAM_LOGWD) return BETTY_ERR_INVALID_ARG;
   if (L->optimizer < BETTY_OPT_GD || L->optimizer > BETTY_OPT_ADAM) return BETTY_ERR_INVALID_ARG;
   if (L->optimizer != BETTY_OPT_GD && !L->opt_state) return BETTY_ERR_INVALID_ARG;
+  if (L->precision != 0 && L->precision != BETTY_BF16 && L->precision != BETTY_F16) return BETTY_ERR_DTYPE;
+  if (L->precision == BETTY_F16 && L->param_kind != BETTY_PARAM_MLP) return BETTY_ERR_DTYPE;
+  if (L->loss_scale && !(L->precision == BETTY_F16 && L->param_kind == BETTY_PARAM_MLP)) return BETTY_ERR_INVALID_ARG;
   if (is_vector_family(L->loss)) return vecfam_validate(L);
   if (is_mlp_family(L->loss)) return mlpfam_validate(L);
   return BETTY_ERR_INVALID_ARG;
@@ -327,7 +396,7 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
       }
     } else {
       // the same sum by Horner's rule, q <- v + (I - alpha H) q from q = v, fused into the HVP's epilogues
-      if (cfg.K > 0 && L->param_kind == BETTY_PARAM_MLP) BETTY_TRY(mlpfam_hvp_keep_direction(c, cache));
+      if (cfg.K > 0 && L->param_kind == BETTY_PARAM_MLP) BETTY_TRY(mlpfam_hvp_keep_direction(c, L, cache));
       for (int k = 0; k < cfg.K; ++k) BETTY_TRY(mlpfam_hvp_series(c, L, cache, k == 0 ? v : q, v, cfg.alpha, q));
     }
     qscale = cfg.alpha;   // q holds the plain sum; alpha is applied with the sign below
@@ -641,7 +710,7 @@ betty_status betty_engine_run(const betty_level* const* levels, int32_t n_levels
   for (int i = 0; i < n_levels; ++i) {
     BETTY_TRY(validate_level(levels[i]));
     if (unroll_steps[i] < 1) return BETTY_ERR_INVALID_ARG;
-    if (levels[i]->comm) return BETTY_ERR_UNSUPPORTED;                 // not offered for data-parallel levels
+    if (levels[i]->comm || levels[i]->loss_scale) return BETTY_ERR_UNSUPPORTED;   // not offered for data-parallel or loss-scaled levels
   }
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
@@ -736,12 +805,28 @@ betty_status betty_lower_step(const betty_level* L, int32_t n_steps, void* ws, s
   if (n_steps < 0) return BETTY_ERR_INVALID_ARG;
   BETTY_TRY(check_ws(ws, ws_bytes));
   Ctx c(ws, ws_bytes, stream);
-  if (L->optimizer != BETTY_OPT_GD || L->grad_accum > 1 || L->comm) {
+  if (L->optimizer != BETTY_OPT_GD || L->grad_accum > 1 || L->comm || L->loss_scale) {
     BETTY_ALLOC(g, float, c, (size_t)L->n_params);
+    int* overflow = nullptr;
+    if (L->loss_scale) {
+      overflow = c.arena.alloc<int>(8);
+      if (!overflow) return BETTY_ERR_WORKSPACE;
+      c.loss_scale = L->loss_scale;       // the gradient pass multiplies its top deltas by the scale
+    }
     for (int s = 0; s < n_steps; ++s) {
       BETTY_TRY(step_grad(c, L, g));
-      BETTY_TRY(apply_optimizer(c, L, g, s));
+      if (overflow) {
+        if (cudaMemsetAsync(overflow, 0, sizeof(int), c.stream) != cudaSuccess) return BETTY_ERR_CUDA;
+        launch_pdl(k_unscale_check, dim3(ew_grid(L->n_params)), dim3(256), 0, c.stream, g, L->n_params, (const float*)L->loss_scale, overflow);
+        BETTY_LAUNCH_CHECK();
+      }
+      BETTY_TRY(apply_optimizer(c, L, g, s, overflow));
+      if (overflow) {
+        launch_pdl(k_loss_scale_update, dim3(1), dim3(1), 0, c.stream, L->loss_scale, (const int*)overflow);
+        BETTY_LAUNCH_CHECK();
+      }
     }
+    c.loss_scale = nullptr;
     return BETTY_OK;
   }
   if (is_vector_family(L->loss)) return vecfam_lower_step(c, L, n_steps);

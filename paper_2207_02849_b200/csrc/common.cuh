@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 #include <stddef.h>
 #include <atomic>
@@ -10,7 +11,27 @@
 
 namespace betty {
 
-typedef __nv_bfloat16 bf16;
+// 16-bit operand type of the MLP families' matrix products.  The family sources (mlp.cu, gemm.cu, gemm_tc.cu)
+// are compiled twice into two namespaces: with bfloat16 operands (fam_bf16, the default) and, with
+// BETTY_FP16_OPERANDS defined, with IEEE binary16 operands (fam_f16; Sec. 4 lists mixed precision, and the
+// paper's listings switch it on with an fp16 flag).  Accumulation is fp32 in both.
+#ifdef BETTY_FP16_OPERANDS
+#define BETTY_FAM fam_f16
+typedef __half op16;
+typedef __half2 op16x2;
+__device__ __forceinline__ op16 to_op16(float v) { return __float2half_rn(v); }
+__device__ __forceinline__ float from_op16(op16 v) { return __half2float(v); }
+__device__ __forceinline__ op16x2 to_op16x2(float a, float b) { return __floats2half2_rn(a, b); }
+__device__ __forceinline__ float2 from_op16x2(op16x2 v) { return __half22float2(v); }
+#else
+#define BETTY_FAM fam_bf16
+typedef __nv_bfloat16 op16;
+typedef __nv_bfloat162 op16x2;
+__device__ __forceinline__ op16 to_op16(float v) { return __float2bfloat16_rn(v); }
+__device__ __forceinline__ float from_op16(op16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ op16x2 to_op16x2(float a, float b) { return __floats2bfloat162_rn(a, b); }
+__device__ __forceinline__ float2 from_op16x2(op16x2 v) { return __bfloat1622float2(v); }
+#endif
 
 // Device status block: the first 256 bytes of the caller's workspace.
 struct StatusBlock {
@@ -59,7 +80,7 @@ struct Arena {
 // bf16 copies of an MLP's matrices that several passes of one call share (see mlpfam_share_weights)
 struct SharedWeights {
   const float* master;   // the fp32 parameters the copies were rounded from; null: none
-  bf16* W[16];
+  void* W[16];           // 16-bit copies, of the operand type of the family that made them
 };
 
 // ---- per-device facts and settings ----
@@ -104,8 +125,9 @@ struct Ctx {
   Arena arena;
   int sm_count;
   SharedWeights shared;
+  const float* loss_scale;   // device loss scale of the lower step in progress (betty_level.loss_scale), else null
   __host__ Ctx(void* ws, size_t ws_bytes, void* s)
-      : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(current_sm_count()) {
+      : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(current_sm_count()), loss_scale(nullptr) {
     shared.master = nullptr;
   }
 };

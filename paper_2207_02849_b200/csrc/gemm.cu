@@ -2,6 +2,7 @@
 #include "gemm.cuh"
 
 namespace betty {
+namespace BETTY_FAM {
 
 static constexpr int GT = 64;   // C tile edge
 static constexpr int GK = 16;   // K slab
@@ -28,14 +29,14 @@ __global__ void __launch_bounds__(256) k_gemm_simt(GemmDesc g) {
         else { int idx = tid + j * 256; m = idx & 63; k = idx >> 6; }
         float v = 0.f;
         if (m0 + m < g.M && k0 + k < p.K)
-          v = __bfloat162float(p.ta ? p.A[(int64_t)(k0 + k) * p.lda + m0 + m] : p.A[(int64_t)(m0 + m) * p.lda + k0 + k]);
+          v = from_op16(p.ta ? p.A[(int64_t)(k0 + k) * p.lda + m0 + m] : p.A[(int64_t)(m0 + m) * p.lda + k0 + k]);
         As[k][m] = v * p.alpha;
         int n;
         if (p.tb) { int idx = tid * 4 + j; n = idx >> 4; k = idx & 15; }
         else { int idx = tid + j * 256; n = idx & 63; k = idx >> 6; }
         v = 0.f;
         if (n0 + n < g.N && k0 + k < p.K)
-          v = __bfloat162float(p.tb ? p.B[(int64_t)(n0 + n) * p.ldb + k0 + k] : p.B[(int64_t)(k0 + k) * p.ldb + n0 + n]);
+          v = from_op16(p.tb ? p.B[(int64_t)(n0 + n) * p.ldb + k0 + k] : p.B[(int64_t)(k0 + k) * p.ldb + n0 + n]);
         Bs[k][n] = v;
       }
       __syncthreads();
@@ -80,9 +81,12 @@ betty_status gemm(Ctx& c, const GemmDesc& g) {
   return gemm_simt(c, g);
 }
 
+}  // namespace BETTY_FAM
 }  // namespace betty
 
+#ifndef BETTY_FP16_OPERANDS      // the kernel-level check is offered for the default operand type
 using namespace betty;
+using namespace betty::BETTY_FAM;
 
 extern "C" betty_status betty_gemm_bf16(int32_t M, int32_t N, int32_t n_pairs, const betty_gemm_operands* pairs,
                                         float* C, int64_t ldc, float beta, int32_t path, void* ws, size_t ws_bytes,
@@ -95,7 +99,7 @@ extern "C" betty_status betty_gemm_bf16(int32_t M, int32_t N, int32_t n_pairs, c
   for (int i = 0; i < n_pairs; ++i) {
     const betty_gemm_operands& o = pairs[i];
     if (!o.A || !o.B || o.K < 0) return BETTY_ERR_INVALID_ARG;
-    g.p[i] = gemm_pair((const bf16*)o.A, o.lda, o.a_transposed != 0, (const bf16*)o.B, o.ldb, o.b_transposed != 0, o.K,
+    g.p[i] = gemm_pair((const op16*)o.A, o.lda, o.a_transposed != 0, (const op16*)o.B, o.ldb, o.b_transposed != 0, o.K,
                        o.alpha);
   }
   if (path == 1) return gemm_simt(c, g);
@@ -105,3 +109,4 @@ extern "C" betty_status betty_gemm_bf16(int32_t M, int32_t N, int32_t n_pairs, c
   if (path == 5) return gemm_tc_eligible(g) ? gemm_tc_pair(c, g, false) : BETTY_ERR_UNSUPPORTED;
   return gemm(c, g);
 }
+#endif

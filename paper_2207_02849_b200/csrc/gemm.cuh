@@ -1,14 +1,15 @@
-// bf16 x bf16 -> fp32 matrix products used by the MLP families (forward, backward and
+// op16 x op16 -> fp32 matrix products used by the MLP families (forward, backward and
 // R-operator passes).  One call computes  C = sum_p alpha_p * op(A_p) op(B_p) + beta * C  over
 // one or two operand pairs: the R-operator needs sums such as Rh W^T + h U^T in one accumulator.
 #pragma once
 #include "common.cuh"
 
 namespace betty {
+namespace BETTY_FAM {
 
 struct GemmPair {
-  const bf16* A; int64_t lda; bool ta;   // logical A is [M,K]; ta: stored [K,M] (M contiguous)
-  const bf16* B; int64_t ldb; bool tb;   // logical B is [K,N]; tb: stored [N,K] (K contiguous)
+  const op16* A; int64_t lda; bool ta;   // logical A is [M,K]; ta: stored [K,M] (M contiguous)
+  const op16* B; int64_t ldb; bool tb;   // logical B is [K,N]; tb: stored [N,K] (K contiguous)
   int K;
   float alpha;
 };
@@ -19,8 +20,8 @@ enum GemmEpiMode {
   EPI_ACT_BWD = 2,   // C = acc (if C);     out16 = acc * act'(a[m,n])                   (backward through an activation)
   EPI_R_FWD = 3,     // v = acc + bias[n];  C = v;  out16 = act'(a[m,n]) * v             (R-operator forward)
   EPI_R_BWD = 4,     // out16 = acc * act'(a) + dh * act''(a) * Ra                       (R-operator backward)
-  EPI_SGD = 5,       // g = acc + exp(lam) * w16;  C = C - lr * g;  out16 = bf16(new C)  (weight gradient -> gradient step; w16 == bf16(C))
-  EPI_NEUMANN = 6    // Hu = acc + exp(lam) * t_in;  C = s_in + t_in - alpha * Hu;  out16 = bf16(C) if given   (weight HVP -> one Horner step of the Neumann series)
+  EPI_SGD = 5,       // g = acc + exp(lam) * w16;  C = C - lr * g;  out16 = op16(new C)  (weight gradient -> gradient step; w16 == op16(C))
+  EPI_NEUMANN = 6    // Hu = acc + exp(lam) * t_in;  C = s_in + t_in - alpha * Hu;  out16 = op16(C) if given   (weight HVP -> one Horner step of the Neumann series)
 };
 struct GemmEpilogue {
   int mode;
@@ -29,11 +30,11 @@ struct GemmEpilogue {
   const float* a;          // [M,N] pre-activations, leading dimension N
   const float* dh;         // [M,N]
   const float* Ra;         // [M,N]
-  bf16* out16;             // [M, ld16] or null
+  op16* out16;             // [M, ld16] or null
   int64_t ld16;
   // EPI_SGD / EPI_NEUMANN (all [M,N] with the leading dimension of C unless noted)
   const float* lam;        // device scalar: log weight decay of this layer, or null
-  const bf16* w16;         // EPI_SGD: bf16 weights the gradient was taken at, leading dimension ldw16
+  const op16* w16;         // EPI_SGD: op16 weights the gradient was taken at, leading dimension ldw16
   int64_t ldw16;
   float step;              // EPI_SGD: learning rate; EPI_NEUMANN: alpha
   const float* t_in;       // EPI_NEUMANN: the HVP direction = the partial sum so far (may alias C)
@@ -50,7 +51,7 @@ struct GemmDesc {
 
 // ---- activation functions shared by the matrix-product epilogues and the row kernels ----
 // Standard normal density and distribution function.  The distribution function uses the rational
-// approximation 7.1.26 of Abramowitz & Stegun for erf (|error| <= 1.5e-7, far below the bf16 rounding of
+// approximation 7.1.26 of Abramowitz & Stegun for erf (|error| <= 1.5e-7, far below the op16 rounding of
 // every quantity it feeds): no branches, one reciprocal and one exponential, and exp(-x^2) with
 // x = a / sqrt(2) is the density's own exponential, so a kernel that needs both evaluates it once.
 __device__ __forceinline__ float norm_pdf(float a) { return 0.3989422804014327f * __expf(-0.5f * a * a); }
@@ -85,31 +86,31 @@ __device__ __forceinline__ void gemm_epilogue_store(const GemmEpilogue& e, float
     case EPI_BIAS_ACT: {
       const float v = acc + e.bias[n];
       *cp = v;
-      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(act_f(e.act, v));
+      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = to_op16(act_f(e.act, v));
       break;
     }
     case EPI_ACT_BWD:
       if (cp) *cp = acc;
-      e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(acc * act_d1(e.act, e.a[j]));
+      e.out16[(int64_t)m * e.ld16 + n] = to_op16(acc * act_d1(e.act, e.a[j]));
       break;
     case EPI_R_FWD: {
       const float v = acc + e.bias[n];
       *cp = v;
-      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(act_d1(e.act, e.a[j]) * v);
+      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = to_op16(act_d1(e.act, e.a[j]) * v);
       break;
     }
     case EPI_R_BWD: {
       float v = acc * act_d1(e.act, e.a[j]);
       if (e.act != BETTY_ACT_RELU) v += e.dh[j] * act_d2(e.act, e.a[j]) * e.Ra[j];
-      e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(v);
+      e.out16[(int64_t)m * e.ld16 + n] = to_op16(v);
       break;
     }
     case EPI_SGD: {
       float gval = acc;
-      if (e.lam) gval += expf(*e.lam) * __bfloat162float(e.w16[(int64_t)m * e.ldw16 + n]);
+      if (e.lam) gval += expf(*e.lam) * from_op16(e.w16[(int64_t)m * e.ldw16 + n]);
       const float w = *cp - e.step * gval;
       *cp = w;
-      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(w);
+      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = to_op16(w);
       break;
     }
     case EPI_NEUMANN: {
@@ -119,7 +120,7 @@ __device__ __forceinline__ void gemm_epilogue_store(const GemmEpilogue& e, float
       if (e.lam) hu += expf(*e.lam) * ti;
       const float tn = e.s_in[jc] + (ti - e.step * hu);
       *cp = tn;
-      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = __float2bfloat16_rn(tn);
+      if (e.out16) e.out16[(int64_t)m * e.ld16 + n] = to_op16(tn);
       break;
     }
   }
@@ -137,10 +138,11 @@ betty_status gemm_tc_pair(Ctx& c, const GemmDesc& g, bool tr = true);   // two-S
 // path does not take.
 betty_status gemm_simt(Ctx& c, const GemmDesc& g);
 
-static inline GemmPair gemm_pair(const bf16* A, int64_t lda, bool ta, const bf16* B, int64_t ldb, bool tb, int K,
+static inline GemmPair gemm_pair(const op16* A, int64_t lda, bool ta, const op16* B, int64_t ldb, bool tb, int K,
                                  float alpha = 1.f) {
   GemmPair p; p.A = A; p.lda = lda; p.ta = ta; p.B = B; p.ldb = ldb; p.tb = tb; p.K = K; p.alpha = alpha;
   return p;
 }
 
+}  // namespace BETTY_FAM
 }  // namespace betty

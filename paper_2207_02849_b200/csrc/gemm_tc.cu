@@ -12,9 +12,10 @@
 #include "gemm.cuh"
 
 namespace betty {
+namespace BETTY_FAM {
 
 static constexpr int TC_BM = 128;
-static constexpr int TC_BK = 64;            // 64 bf16 = one 128-byte swizzle row
+static constexpr int TC_BK = 64;            // 64 op16 = one 128-byte swizzle row
 static constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;
 static constexpr uint32_t TC_SPIN = 1u << 24;
 static constexpr int TC_THREADS = 320;      // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: epilogue
@@ -80,12 +81,14 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   d |= (uint64_t)2 << 61;
   return d;
 }
-// Instruction descriptor for kind::f16: fp32 accumulator, bf16 operands, majors, optional negation of A.
+// Instruction descriptor for kind::f16: fp32 accumulator, op16 operands, majors, optional negation of A.
 __device__ __forceinline__ uint32_t instr_desc(int a_mn, int b_mn, int neg_a, int n, int m) {
   uint32_t d = 0;
   d |= 1u << 4;                 // D format: F32
-  d |= 1u << 7;                 // A format: BF16
-  d |= 1u << 10;                // B format: BF16
+#ifndef BETTY_FP16_OPERANDS
+  d |= 1u << 7;                 // A format: BF16 (0: F16)
+  d |= 1u << 10;                // B format: BF16 (0: F16)
+#endif
   d |= (uint32_t)(neg_a & 1) << 13;
   d |= (uint32_t)(a_mn & 1) << 15;
   d |= (uint32_t)(b_mn & 1) << 16;
@@ -118,7 +121,7 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
   if (g.vec_ok && nb + 32 <= g.N) {
     float* crow = g.C ? g.C + (int64_t)m * g.ldc + nb : nullptr;
     const int64_t jb = (int64_t)m * g.N + nb;
-    bf16* orow = e.out16 ? e.out16 + (int64_t)m * e.ld16 + nb : nullptr;
+    op16* orow = e.out16 ? e.out16 + (int64_t)m * e.ld16 + nb : nullptr;
 #pragma unroll
     for (int j8 = 0; j8 < 32; j8 += 8) {
       float v[8], o[8];
@@ -152,9 +155,9 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
         float wv[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         if (e.lam) {
           const uint4 wq = *(const uint4*)(e.w16 + (int64_t)m * e.ldw16 + nb + j8);
-          const __nv_bfloat162* wp = (const __nv_bfloat162*)&wq;
+          const op16x2* wp = (const op16x2*)&wq;
 #pragma unroll
-          for (int k = 0; k < 4; ++k) { const float2 f = __bfloat1622float2(wp[k]); wv[2 * k] = f.x; wv[2 * k + 1] = f.y; }
+          for (int k = 0; k < 4; ++k) { const float2 f = from_op16x2(wp[k]); wv[2 * k] = f.x; wv[2 * k + 1] = f.y; }
         }
 #pragma unroll
         for (int k = 0; k < 8; ++k) { v[k] = cv[k] - e.step * (v[k] + kap * wv[k]); o[k] = v[k]; }
@@ -186,9 +189,9 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
         *(float4*)(crow + j8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
       }
       if (orow && e.mode != EPI_STORE) {
-        __nv_bfloat162 ob[4];
+        op16x2 ob[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) ob[k] = __floats2bfloat162_rn(o[2 * k], o[2 * k + 1]);
+        for (int k = 0; k < 4; ++k) ob[k] = to_op16x2(o[2 * k], o[2 * k + 1]);
         *(uint4*)(orow + j8) = *(uint4*)ob;
       }
     }
@@ -202,7 +205,7 @@ __device__ __forceinline__ void epilogue_row32(const TcArgs& g, int m, int nb, c
 // Transposed accumulator (tr): the host swapped the operand roles, so this thread's accumulator lane is
 // column n of C and r holds rows mb .. mb+31 of that column.  For a fixed row the 32 lanes of a warp
 // touch 32 consecutive elements of C and of every epilogue input: each access is one full 128-byte
-// line per warp (64 bytes for the bf16 outputs) instead of 32 separate lines.
+// line per warp (64 bytes for the op16 outputs) instead of 32 separate lines.
 // C is [MC, NC] = [g.N, g.M] here.  Every load of a batch of rows is issued before the first use: the
 // epilogue is bound by bytes in flight per SM (eight warps), so a batch is as deep as the registers
 // allow (all 32 rows; 16 when three inputs are read).  Mode and activation are compile-time
@@ -220,7 +223,7 @@ __device__ __forceinline__ void epilogue_t32_rows(const TcArgs& g, int n, int mb
   const float* qp = e.Ra ? e.Ra + (int64_t)mb * NC + n : nullptr;
   const float* tp = e.t_in ? e.t_in + (int64_t)mb * g.ldc + n : nullptr;
   const float* sp = e.s_in ? e.s_in + (int64_t)mb * g.ldc + n : nullptr;
-  bf16* op = e.out16 ? e.out16 + (int64_t)mb * e.ld16 + n : nullptr;
+  op16* op = e.out16 ? e.out16 + (int64_t)mb * e.ld16 + n : nullptr;
   const int rows = MC - mb;     // > 0; FULL: >= 32, and no per-row guards, so that the rows' dependency chains interleave
   const bool second = MODE == EPI_R_BWD && ACT != BETTY_ACT_RELU;
 #pragma unroll
@@ -245,38 +248,38 @@ __device__ __forceinline__ void epilogue_t32_rows(const TcArgs& g, int n, int mb
       if (FULL || j < rows) {
         const float acc = __uint_as_float(r[j]);
         float* c1 = cp + (int64_t)j * g.ldc;
-        bf16* o1 = op + (int64_t)j * e.ld16;
+        op16* o1 = op + (int64_t)j * e.ld16;
         if (MODE == EPI_STORE) *c1 = acc + g.beta * x0[k];
         if (MODE == EPI_BIAS_ACT) {
           const float v = acc + bias;
           *c1 = v;
-          if (op) *o1 = __float2bfloat16_rn(act_f(ACT, v));
+          if (op) *o1 = to_op16(act_f(ACT, v));
         }
         if (MODE == EPI_R_FWD) {
           const float v = acc + bias;
           *c1 = v;
-          if (op) *o1 = __float2bfloat16_rn(act_d1(ACT, x0[k]) * v);
+          if (op) *o1 = to_op16(act_d1(ACT, x0[k]) * v);
         }
         if (MODE == EPI_ACT_BWD) {
           if (cp) *c1 = acc;
-          *o1 = __float2bfloat16_rn(acc * act_d1(ACT, x0[k]));
+          *o1 = to_op16(acc * act_d1(ACT, x0[k]));
         }
         if (MODE == EPI_R_BWD) {
           float v = acc * act_d1(ACT, x0[k]);
           if (second) v += x1[k] * act_d2(ACT, x0[k]) * x2[k];
-          *o1 = __float2bfloat16_rn(v);
+          *o1 = to_op16(v);
         }
         if (MODE == EPI_SGD) {
-          // the bf16 weights the gradient was taken at (w16) are the rounded master weights: no second read
-          const float wq = __bfloat162float(__float2bfloat16_rn(x0[k]));
+          // the op16 weights the gradient was taken at (w16) are the rounded master weights: no second read
+          const float wq = from_op16(to_op16(x0[k]));
           const float w = x0[k] - e.step * (acc + kap * wq);
           *c1 = w;
-          if (op) *o1 = __float2bfloat16_rn(w);
+          if (op) *o1 = to_op16(w);
         }
         if (MODE == EPI_NEUMANN) {
           const float tn = x1[k] + (x0[k] - e.step * (acc + kap * x0[k]));
           *c1 = tn;
-          if (op) *o1 = __float2bfloat16_rn(tn);
+          if (op) *o1 = to_op16(tn);
         }
       }
     }
@@ -760,16 +763,21 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D bf16 tensor map over a row-major matrix [outer, inner] with leading dimension ld (elements)
-static bool make_map(CUtensorMap* tm, const bf16* base, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+// 2-D op16 tensor map over a row-major matrix [outer, inner] with leading dimension ld (elements)
+static bool make_map(CUtensorMap* tm, const op16* base, int64_t inner, int64_t outer, int64_t ld, int box_inner,
                      int box_outer) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(bf16)};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(op16)};
   cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
   cuuint32_t estr[2] = {1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+#ifdef BETTY_FP16_OPERANDS
+  const CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+#else
+  const CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+#endif
+  return fn(tm, dtype, 2, (void*)base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -883,4 +891,5 @@ betty_status gemm_tc(Ctx& c, const GemmDesc& g0, bool tr) {
   return launch_tc<128>(c, g0, tr);
 }
 
+}  // namespace BETTY_FAM
 }  // namespace betty

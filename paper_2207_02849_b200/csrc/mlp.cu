@@ -3,11 +3,12 @@
 // three-level configuration.  Gradients are hand-written reverse sweeps; Hessian-vector products
 // are R-operator (forward-over-reverse) passes that reuse a cached base forward/backward pass;
 // mixed second derivatives are a directional forward pass followed by the weight net's reverse
-// sweep.  Matrices are bf16 (rounded copies of the fp32 master), accumulation is fp32.
+// sweep.  Matrices are op16 (rounded copies of the fp32 master), accumulation is fp32.
 #include "ops.cuh"
 #include "gemm.cuh"
 
 namespace betty {
+namespace BETTY_FAM {
 
 static constexpr int MAXL = 16;
 static constexpr int WN_H = 100;
@@ -26,26 +27,26 @@ __device__ __forceinline__ float fd_eps(const float* vnorm2, float eps0) {
 }
 
 // ------------------------------------------------------------------ elementwise / row kernels
-// dst[r, c] = bf16(scale * src[r, c]); scale = eps0/|v| when vnorm2 is given, else 1.  Pad columns are zeroed.
-__global__ void k_cast_rows(const float* src, bf16* dst, int64_t rows, int64_t cols, int64_t ld, const float* vnorm2,
+// dst[r, c] = op16(scale * src[r, c]); scale = eps0/|v| when vnorm2 is given, else 1.  Pad columns are zeroed.
+__global__ void k_cast_rows(const float* src, op16* dst, int64_t rows, int64_t cols, int64_t ld, const float* vnorm2,
                             float eps0) {
   pdl_enter();
   const float s = vnorm2 ? fd_eps(vnorm2, eps0) : 1.f;
   const int64_t total = rows * ld;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / ld, c = i - r * ld;
-    dst[i] = __float2bfloat16_rn(c < cols ? s * src[r * cols + c] : 0.f);
+    dst[i] = to_op16(c < cols ? s * src[r * cols + c] : 0.f);
   }
 }
-// a += bias; h = act(a) as bf16 (hidden layers)
-__global__ void k_bias_act(float* a, const float* bias, bf16* h, int64_t rows, int64_t N, int64_t ldh, int act) {
+// a += bias; h = act(a) as op16 (hidden layers)
+__global__ void k_bias_act(float* a, const float* bias, op16* h, int64_t rows, int64_t N, int64_t ldh, int act) {
   pdl_enter();
   const int64_t total = rows * N;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / N, n = i - r * N;
     const float v = a[i] + bias[n];
     a[i] = v;
-    if (h) h[r * ldh + n] = __float2bfloat16_rn(act_f(act, v));
+    if (h) h[r * ldh + n] = to_op16(act_f(act, v));
   }
 }
 // one warp per row: p = softmax(z), ell = -log p[y]
@@ -70,15 +71,17 @@ __global__ void k_softmax_ce(const float* z, const int32_t* y, float* p, float* 
   }
 }
 // delta = coef_i * (p - onehot(y))
-__global__ void k_delta_top(const float* p, const int32_t* y, const float* coef, float scale, bf16* delta, int64_t B,
-                            int64_t C, int64_t ld) {
+// lscale (nullable): device loss scale multiplied into every delta (betty_level.loss_scale)
+__global__ void k_delta_top(const float* p, const int32_t* y, const float* coef, float scale, op16* delta, int64_t B,
+                            int64_t C, int64_t ld, const float* lscale) {
   pdl_enter();
+  const float S = lscale ? *lscale : 1.f;
   const int64_t total = B * ld;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / ld, c = i - r * ld;
     float v = 0.f;
-    if (c < C) v = (coef ? coef[r] : scale) * (p[r * C + c] - (c == y[r] ? 1.f : 0.f));
-    delta[i] = __float2bfloat16_rn(v);
+    if (c < C) v = S * ((coef ? coef[r] : scale) * (p[r * C + c] - (c == y[r] ? 1.f : 0.f)));
+    delta[i] = to_op16(v);
   }
 }
 // Column sums sum_i d[i, n] (bias gradients), with the consumer fused in.  Block = 32 columns (16 lanes x 2
@@ -88,7 +91,7 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
 //   mode 2: out[n] = s_in[n] + t_in[n] - step * sum   (one Horner step of the Neumann series; out may alias t_in)
 struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; };
 static constexpr int CS_COLS = 32, CS_GROUPS = 64;
-__global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
+__global__ void __launch_bounds__(1024) k_colsum_bf16(const op16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
   pdl_enter();
   __shared__ float sh[CS_GROUPS][CS_COLS + 1];
   const int cx = threadIdx.x & 15, rg = threadIdx.x >> 4;
@@ -97,15 +100,15 @@ __global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, 
   if (n < N) {
     constexpr int U = 16;
     for (int64_t i0 = rg; i0 < B; i0 += CS_GROUPS * U) {
-      __nv_bfloat162 v[U];
+      op16x2 v[U];
 #pragma unroll
       for (int k2 = 0; k2 < U; ++k2) {
         const int64_t i = i0 + CS_GROUPS * k2;
-        v[k2] = i < B ? *(const __nv_bfloat162*)(d + i * ld + n) : __floats2bfloat162_rn(0.f, 0.f);
+        v[k2] = i < B ? *(const op16x2*)(d + i * ld + n) : to_op16x2(0.f, 0.f);
       }
 #pragma unroll
       for (int k2 = 0; k2 < U; ++k2) {   // same order as a plain loop over the rows
-        const float2 f = __bfloat1622float2(v[k2]);
+        const float2 f = from_op16x2(v[k2]);
         a0 += f.x; a1 += f.y;
       }
     }
@@ -125,16 +128,16 @@ __global__ void __launch_bounds__(1024) k_colsum_bf16(const bf16* d, int64_t B, 
   }
 }
 // delta_prev = dh * act'(a)
-__global__ void k_act_backward(const float* dh, const float* a, bf16* dprev, int64_t B, int64_t N, int64_t ld, int act) {
+__global__ void k_act_backward(const float* dh, const float* a, op16* dprev, int64_t B, int64_t N, int64_t ld, int act) {
   pdl_enter();
   const int64_t total = B * ld;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / ld, n = i - r * ld;
-    dprev[i] = __float2bfloat16_rn(n < N ? dh[r * N + n] * act_d1(act, a[r * N + n]) : 0.f);
+    dprev[i] = to_op16(n < N ? dh[r * N + n] * act_d1(act, a[r * N + n]) : 0.f);
   }
 }
 // Ra += c ; Rh = act'(a) * Ra
-__global__ void k_r_act_forward(float* Ra, const float* cdir, const float* a, bf16* Rh, int64_t B, int64_t N,
+__global__ void k_r_act_forward(float* Ra, const float* cdir, const float* a, op16* Rh, int64_t B, int64_t N,
                                 int64_t ldh, int act) {
   pdl_enter();
   const int64_t total = B * N;
@@ -142,11 +145,11 @@ __global__ void k_r_act_forward(float* Ra, const float* cdir, const float* a, bf
     const int64_t r = i / N, n = i - r * N;
     const float v = Ra[i] + cdir[n];
     Ra[i] = v;
-    if (Rh) Rh[r * ldh + n] = __float2bfloat16_rn(act_d1(act, a[i]) * v);
+    if (Rh) Rh[r * ldh + n] = to_op16(act_d1(act, a[i]) * v);
   }
 }
 // one warp per row: Rdelta = coef_i * (p.*Ra - p * (p . Ra))
-__global__ void k_r_delta_top(const float* p, const float* Ra, const float* coef, float scale, bf16* Rd, int64_t B,
+__global__ void k_r_delta_top(const float* p, const float* Ra, const float* coef, float scale, op16* Rd, int64_t B,
                               int64_t C, int64_t ld) {
   pdl_enter();
   const int lane = threadIdx.x & 31;
@@ -159,11 +162,11 @@ __global__ void k_r_delta_top(const float* p, const float* Ra, const float* coef
   for (int64_t c = lane; c < ld; c += 32) {
     float v = 0.f;
     if (c < C) { const float pc = p[row * C + c]; v = k * (pc * Ra[row * C + c] - pc * s); }
-    Rd[row * ld + c] = __float2bfloat16_rn(v);
+    Rd[row * ld + c] = to_op16(v);
   }
 }
 // Rdelta_prev = Rdh * act'(a) + dh * act''(a) * Ra
-__global__ void k_r_act_backward(const float* Rdh, const float* dh, const float* a, const float* Ra, bf16* Rdprev,
+__global__ void k_r_act_backward(const float* Rdh, const float* dh, const float* a, const float* Ra, op16* Rdprev,
                                  int64_t B, int64_t N, int64_t ld, int act) {
   pdl_enter();
   const int64_t total = B * ld;
@@ -175,7 +178,7 @@ __global__ void k_r_act_backward(const float* Rdh, const float* dh, const float*
       v = Rdh[j] * act_d1(act, a[j]);
       if (act != BETTY_ACT_RELU) v += dh[j] * act_d2(act, a[j]) * Ra[j];
     }
-    Rdprev[i] = __float2bfloat16_rn(v);
+    Rdprev[i] = to_op16(v);
   }
 }
 // one warp per row: d_i = sum_c (p - onehot) * Ra
@@ -189,14 +192,15 @@ __global__ void k_jvp_rows(const float* p, const int32_t* y, const float* Ra, fl
   for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
   if (lane == 0) d[row] = s;
 }
-// out[r, c] += exp(lam) * W[r, c]   (out contiguous [rows, cols]; W bf16 with leading dimension ldw)
-__global__ void k_wd_add_bf16(float* out, const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* lam) {
+// out[r, c] += exp(lam) * W[r, c]   (out contiguous [rows, cols]; W op16 with leading dimension ldw)
+__global__ void k_wd_add_bf16(float* out, const op16* W, int64_t rows, int64_t cols, int64_t ldw, const float* lam,
+                              const float* lscale) {
   pdl_enter();
-  const float k = expf(*lam);
+  const float k = expf(*lam) * (lscale ? *lscale : 1.f);     // a scaled gradient takes a scaled decay term
   const int64_t total = rows * cols;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / cols, c = i - r * cols;
-    out[i] += k * __bfloat162float(W[r * ldw + c]);
+    out[i] += k * from_op16(W[r * ldw + c]);
   }
 }
 __global__ void k_wd_add_f32(float* out, const float* u, int64_t n, const float* lam) {
@@ -209,7 +213,7 @@ __global__ void k_wd_add_f32(float* out, const float* u, int64_t n, const float*
 // that draws the last ticket adds the per-block sums in a fixed order (one warp: strided partial sums, then a
 // shuffle tree), so the result does not depend on scheduling.
 static constexpr int LD_MAX_BLOCKS = 128;
-__global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
+__global__ void k_layer_dot(const op16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
                             float scale, float* out, int accumulate, double* partial, unsigned* counter) {
   pdl_enter();
   __shared__ double sh[32];
@@ -218,7 +222,7 @@ __global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t l
   const int64_t total = rows * cols;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / cols, c = i - r * cols;
-    const float w = __bfloat162float(W[r * ldw + c]);
+    const float w = from_op16(W[r * ldw + c]);
     acc += (double)w * (double)(q ? q[i] : w);
   }
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
@@ -245,7 +249,7 @@ __global__ void k_layer_dot(const bf16* W, int64_t rows, int64_t cols, int64_t l
     }
   }
 }
-static betty_status layer_dot(Ctx& c, const bf16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
+static betty_status layer_dot(Ctx& c, const op16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
                               float scale, float* out, bool accumulate) {
   int64_t nb = (rows * cols + 256 * 16 - 1) / (256 * 16);
   nb = nb < 1 ? 1 : (nb > LD_MAX_BLOCKS ? LD_MAX_BLOCKS : nb);
@@ -354,10 +358,10 @@ __global__ void k_wn_backward(const float* theta, const float* dir, const float*
 }
 
 // ------------------------------------------------------------------ finite-difference pieces
-// da_tot = da + sign*eps*c.  Hidden layer: hp = act(a + da_tot) -> bf16, dh = hp - act(a) -> bf16.
+// da_tot = da + sign*eps*c.  Hidden layer: hp = act(a + da_tot) -> op16, dh = hp - act(a) -> op16.
 // Output layer: z = a + da_tot (fp32).
 __global__ void k_fd_act(const float* a, const float* da, const float* cdir, const float* vnorm2, float eps0, float sign,
-                         bf16* hpm, bf16* dhd, float* zpm, int64_t B, int64_t N, int64_t ldh, int act) {
+                         op16* hpm, op16* dhd, float* zpm, int64_t B, int64_t N, int64_t ldh, int act) {
   pdl_enter();
   const float e = sign * fd_eps(vnorm2, eps0);
   const int64_t total = B * N;
@@ -366,8 +370,8 @@ __global__ void k_fd_act(const float* a, const float* da, const float* cdir, con
     const float d = da[i] + e * cdir[n];
     if (zpm) { zpm[i] = a[i] + d; continue; }
     const float h0 = act_f(act, a[i]), hp = act_f(act, a[i] + d);
-    hpm[r * ldh + n] = __float2bfloat16_rn(hp);
-    dhd[r * ldh + n] = __float2bfloat16_rn(hp - h0);
+    hpm[r * ldh + n] = to_op16(hp);
+    dhd[r * ldh + n] = to_op16(hp - h0);
   }
 }
 __global__ void k_fd_combine(float* out, const float* gp, const float* gm, const float* vnorm2, float eps0, float alpha,
@@ -387,28 +391,28 @@ struct Net {
   int64_t w[MAXL + 1];
   int64_t woff[MAXL], boff[MAXL], ldw[MAXL];
   const float* master;
-  bf16* W[MAXL];
+  op16* W[MAXL];
 };
 struct Pass {
   int64_t B;
   const int32_t* y;
-  const bf16* h[MAXL];   // h[l]: input of layer l
+  const op16* h[MAXL];   // h[l]: input of layer l
   int64_t ldh[MAXL];
   float* a[MAXL];        // pre-activations [B, w[l+1]]
   float* p;              // softmax [B, C]
   float* ell;            // per-sample cross-entropy
-  bf16* delta[MAXL];     // dC/da_l, leading dimension ld8(w[l+1])
+  op16* delta[MAXL];     // dC/da_l, leading dimension ld8(w[l+1])
   float* dh[MAXL];       // dC/dh_l (input side of layer l), l >= 1, fp32 [B, w[l]]
 };
-struct MlpHvpCache {
+struct HvpCache {
   Net net;
   Pass pass;
   const float* coef;     // per-sample top coefficient (r_i/B) or null (1/B)
   const float* lam;      // device per-layer log weight decay or null
   const betty_level* theta;
-  // bf16 copies of a direction's matrices that outlive one HVP (series solves): the weight-HVP epilogues
+  // op16 copies of a direction's matrices that outlive one HVP (series solves): the weight-HVP epilogues
   // of iteration k leave the rounded next term here, so that iteration k+1 starts without a cast pass
-  bf16* dir16[MAXL];     // null: every R-forward pass rounds its direction into scratch of its own
+  op16* dir16[MAXL];     // null: every R-forward pass rounds its direction into scratch of its own
   const float* dir16_of; // the fp32 vector that dir16 currently mirrors, or null
 };
 
@@ -433,19 +437,19 @@ static betty_status net_layout(const betty_level* M, Net& n) {
 }
 
 // contiguous case (ld == cols, cols % 8 == 0): 8 elements per thread, 2 x float4 in, 1 x 16 bytes out
-__global__ void k_cast_dense8(const float* src, bf16* dst, int64_t n8, const float* vnorm2, float eps0) {
+__global__ void k_cast_dense8(const float* src, op16* dst, int64_t n8, const float* vnorm2, float eps0) {
   pdl_enter();
   const float s = vnorm2 ? fd_eps(vnorm2, eps0) : 1.f;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
     const float4 a = ((const float4*)src)[2 * i], b = ((const float4*)src)[2 * i + 1];
-    __nv_bfloat162 o[4];
-    o[0] = __floats2bfloat162_rn(s * a.x, s * a.y); o[1] = __floats2bfloat162_rn(s * a.z, s * a.w);
-    o[2] = __floats2bfloat162_rn(s * b.x, s * b.y); o[3] = __floats2bfloat162_rn(s * b.z, s * b.w);
+    op16x2 o[4];
+    o[0] = to_op16x2(s * a.x, s * a.y); o[1] = to_op16x2(s * a.z, s * a.w);
+    o[2] = to_op16x2(s * b.x, s * b.y); o[3] = to_op16x2(s * b.z, s * b.w);
     ((uint4*)dst)[i] = *(uint4*)o;
   }
 }
 
-static betty_status cast_matrix(Ctx& c, const float* src, bf16* dst, int64_t rows, int64_t cols, int64_t ld,
+static betty_status cast_matrix(Ctx& c, const float* src, op16* dst, int64_t rows, int64_t cols, int64_t ld,
                                 const float* vnorm2 = nullptr, float eps0 = 0.f) {
   if (ld == cols && (cols & 7) == 0 && ((((uintptr_t)src) & 15) == 0)) {
     const int64_t n8 = rows * cols / 8;
@@ -457,15 +461,15 @@ static betty_status cast_matrix(Ctx& c, const float* src, bf16* dst, int64_t row
   return BETTY_OK;
 }
 
-// bf16 compute copy of the classifier's matrices (the single quantisation point)
+// op16 compute copy of the classifier's matrices (the single quantisation point)
 static betty_status net_setup(Ctx& c, const betty_level* M, Net& n) {
   BETTY_TRY(net_layout(M, n));
   if (c.shared.master == M->params) {
-    for (int l = 0; l < n.L; ++l) n.W[l] = c.shared.W[l];
+    for (int l = 0; l < n.L; ++l) n.W[l] = (op16*)c.shared.W[l];
     return BETTY_OK;
   }
   for (int l = 0; l < n.L; ++l) {
-    BETTY_ALLOC(Wl, bf16, c, (size_t)(n.w[l + 1] * n.ldw[l]));
+    BETTY_ALLOC(Wl, op16, c, (size_t)(n.w[l + 1] * n.ldw[l]));
     n.W[l] = Wl;
     BETTY_TRY(cast_matrix(c, n.master + n.woff[l], Wl, n.w[l + 1], n.w[l], n.ldw[l]));
   }
@@ -491,21 +495,21 @@ static betty_status forward(Ctx& c, const Net& n, const betty_level* D, Pass& ps
   ps.B = D->n;
   ps.y = (const int32_t*)D->y;
   const int64_t B = ps.B;
-  ps.h[0] = (const bf16*)D->X;
+  ps.h[0] = (const op16*)D->X;
   ps.ldh[0] = D->d;
   for (int l = 0; l < n.L; ++l) {
     const int64_t N = n.w[l + 1];
     BETTY_ALLOC(al, float, c, (size_t)(B * N));
     ps.a[l] = al;
-    bf16* hn = nullptr;
+    op16* hn = nullptr;
     if (l < n.L - 1) {
       ps.ldh[l + 1] = ld8(N);
-      hn = c.arena.alloc<bf16>((size_t)(B * ps.ldh[l + 1]));
+      hn = c.arena.alloc<op16>((size_t)(B * ps.ldh[l + 1]));
       if (!hn) return BETTY_ERR_WORKSPACE;
-      if (ps.ldh[l + 1] != N) cudaMemsetAsync(hn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(bf16), c.stream);
+      if (ps.ldh[l + 1] != N) cudaMemsetAsync(hn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(op16), c.stream);
       ps.h[l + 1] = hn;
     }
-    // a_l = h_l W_l^T + b_l (kept in fp32 for the derivative passes), h_{l+1} = act(a_l) in bf16: one kernel
+    // a_l = h_l W_l^T + b_l (kept in fp32 for the derivative passes), h_{l+1} = act(a_l) in op16: one kernel
     GemmDesc g = {}; g.M = (int)B; g.N = (int)N; g.npairs = 1; g.C = al; g.ldc = N; g.beta = 0.f;
     g.p[0] = gemm_pair(ps.h[l], ps.ldh[l], false, n.W[l], n.ldw[l], true, (int)n.w[l]);
     g.epi.mode = EPI_BIAS_ACT; g.epi.act = n.act; g.epi.bias = n.master + n.boff[l];
@@ -528,7 +532,8 @@ struct GradSink {
   bool sgd;                // instead of storing the gradient, take the step  master -= lr * grad  in the epilogue
   float lr;
   float* master;           // sgd: parameters to update in place
-  bf16* const* Wnext;      // sgd: per-layer bf16 copies of the updated matrices (for the next step), or null
+  op16* const* Wnext;      // sgd: per-layer op16 copies of the updated matrices (for the next step), or null
+  const float* lscale;     // device loss scale: every delta, and with it the whole gradient, is multiplied by it (null: 1)
 };
 
 // Reverse sweep from delta_top = coef_i (p - onehot).  Always leaves delta[l] (and dh[l] for smooth
@@ -538,9 +543,9 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
   const int64_t C = n.w[n.L];
   {
     const int64_t ld = ld8(C);
-    BETTY_ALLOC(dt, bf16, c, (size_t)(B * ld));
+    BETTY_ALLOC(dt, op16, c, (size_t)(B * ld));
     ps.delta[n.L - 1] = dt;
-    launch_pdl(k_delta_top, dim3(grid_for(B * ld)), dim3(256), 0, c.stream, ps.p, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld);
+    launch_pdl(k_delta_top, dim3(grid_for(B * ld)), dim3(256), 0, c.stream, ps.p, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld, sink.lscale);
     BETTY_LAUNCH_CHECK();
   }
   for (int l = n.L - 1; l >= 0; --l) {
@@ -560,14 +565,14 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       }
       BETTY_TRY(gemm(c, g));
       if (!sink.sgd && sink.lam) {
-        launch_pdl(k_wd_add_bf16, dim3(grid_for(N * K)), dim3(256), 0, c.stream, sink.gflat + n.woff[l], n.W[l], N, K, n.ldw[l], sink.lam + l);
+        launch_pdl(k_wd_add_bf16, dim3(grid_for(N * K)), dim3(256), 0, c.stream, sink.gflat + n.woff[l], n.W[l], N, K, n.ldw[l], sink.lam + l, sink.lscale);
         BETTY_LAUNCH_CHECK();
       }
       launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, ps.delta[l], B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
     }
     if (l > 0) {
-      // dh = delta_l W_l ; delta_{l-1} = dh * act'(a_{l-1}) in bf16: one kernel.  dh itself is kept
+      // dh = delta_l W_l ; delta_{l-1} = dh * act'(a_{l-1}) in op16: one kernel.  dh itself is kept
       // only for an R-operator pass over an activation with a second derivative.
       float* dh = nullptr;
       if (keep_dh && n.act != BETTY_ACT_RELU) {
@@ -576,8 +581,8 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       }
       ps.dh[l] = dh;
       const int64_t ldp = ld8(K);
-      BETTY_ALLOC(dp, bf16, c, (size_t)(B * ldp));
-      if (ldp != K) cudaMemsetAsync(dp, 0, (size_t)(B * ldp) * sizeof(bf16), c.stream);
+      BETTY_ALLOC(dp, op16, c, (size_t)(B * ldp));
+      if (ldp != K) cudaMemsetAsync(dp, 0, (size_t)(B * ldp) * sizeof(op16), c.stream);
       ps.delta[l - 1] = dp;
       GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.npairs = 1; g.C = dh; g.ldc = K; g.beta = 0.f;
       g.p[0] = gemm_pair(ps.delta[l], ldd, false, n.W[l], n.ldw[l], false, (int)N);
@@ -593,28 +598,28 @@ static inline GradSink grad_into(float* gflat, const float* lam) {
 
 // Directional derivative of the forward pass along `dir` (flat, same layout as the parameters).
 struct RPass {
-  bf16* U[MAXL];
+  op16* U[MAXL];
   float* Ra[MAXL];
-  const bf16* Rh[MAXL];   // Rh[0] == nullptr (inputs do not move)
+  const op16* Rh[MAXL];   // Rh[0] == nullptr (inputs do not move)
 };
-static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* dir, RPass& rp, MlpHvpCache* keep) {
+static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* dir, RPass& rp, HvpCache* keep) {
   const int64_t B = ps.B;
   rp.Rh[0] = nullptr;
   const bool kept = keep && keep->dir16[0];
   const bool fresh = kept && keep->dir16_of == dir;      // the kept copies already mirror this direction
   for (int l = 0; l < n.L; ++l) {
     const int64_t N = n.w[l + 1], K = n.w[l];
-    bf16* Ul = kept ? keep->dir16[l] : c.arena.alloc<bf16>((size_t)(N * n.ldw[l]));
+    op16* Ul = kept ? keep->dir16[l] : c.arena.alloc<op16>((size_t)(N * n.ldw[l]));
     if (!Ul) return BETTY_ERR_WORKSPACE;
     rp.U[l] = Ul;
     if (!fresh) BETTY_TRY(cast_matrix(c, dir + n.woff[l], Ul, N, K, n.ldw[l]));
     BETTY_ALLOC(Ra, float, c, (size_t)(B * N));
     rp.Ra[l] = Ra;
-    bf16* Rhn = nullptr;
+    op16* Rhn = nullptr;
     if (l < n.L - 1) {
-      Rhn = c.arena.alloc<bf16>((size_t)(B * ps.ldh[l + 1]));
+      Rhn = c.arena.alloc<op16>((size_t)(B * ps.ldh[l + 1]));
       if (!Rhn) return BETTY_ERR_WORKSPACE;
-      if (ps.ldh[l + 1] != N) cudaMemsetAsync(Rhn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(bf16), c.stream);
+      if (ps.ldh[l + 1] != N) cudaMemsetAsync(Rhn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(op16), c.stream);
       rp.Rh[l + 1] = Rhn;
     }
     // Ra_l = h_l U_l^T + Rh_l W_l^T + c_l ; Rh_{l+1} = act'(a_l) * Ra_l: one kernel
@@ -658,10 +663,14 @@ betty_status mlpfam_validate(const betty_level* L) {
   Net n;
   BETTY_TRY(net_layout(P.mlp, n));
   if (L->n < 0 || L->d != n.w[0]) return BETTY_ERR_SHAPE;
+#ifdef BETTY_FP16_OPERANDS
+  if (L->x_dtype != BETTY_F16) return BETTY_ERR_DTYPE;
+#else
   if (L->x_dtype != BETTY_BF16) return BETTY_ERR_DTYPE;
+#endif
   if (L->n > 0 && (!L->X || !L->y)) return BETTY_ERR_INVALID_ARG;
   if (!aligned16(L->X) || !aligned16(P.mlp->params)) return BETTY_ERR_ALIGNMENT;
-  if (L->d % 8 != 0) return BETTY_ERR_ALIGNMENT;     // bf16 rows must start on 16-byte boundaries
+  if (L->d % 8 != 0) return BETTY_ERR_ALIGNMENT;     // op16 rows must start on 16-byte boundaries
   if (P.theta && (P.theta->n_params != WN_P || !P.theta->params)) return BETTY_ERR_SHAPE;
   if (P.lam && (P.lam->n_params != n.L || !P.lam->params)) return BETTY_ERR_SHAPE;
   if (L->loss == BETTY_LOSS_WEIGHTNET_DETECT) {
@@ -739,7 +748,9 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
     if (wrt == P.mlp) {
       const float* coef;
       BETTY_TRY(reweight_coef(c, P, ps, &coef));
-      BETTY_TRY(backward(c, n, ps, coef, grad_into(out, P.lam ? P.lam->params : nullptr)));
+      GradSink sink = grad_into(out, P.lam ? P.lam->params : nullptr);
+      sink.lscale = c.loss_scale;       // set by a loss-scaled lower step only
+      BETTY_TRY(backward(c, n, ps, coef, sink));
     } else {
       BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, ps, nullptr, nullptr, s1, nullptr));
       BETTY_TRY(wn_backward(c, P.theta, nullptr, ps, s1, nullptr, 0.f, nullptr, out));
@@ -758,8 +769,8 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
 }
 
 betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache) {
-  static thread_local MlpHvpCache store;   // host-side bookkeeping only; device state lives in the workspace
-  MlpHvpCache& h = store;
+  static thread_local HvpCache store;   // host-side bookkeeping only; device state lives in the workspace
+  HvpCache& h = store;
   const Parts P = parts_of(L);
   h.theta = P.theta;
   h.lam = P.lam ? P.lam->params : nullptr;
@@ -774,7 +785,7 @@ betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache)
   } else if (!(L->loss == BETTY_LOSS_WEIGHTNET_DETECT && L->param_kind == BETTY_PARAM_WEIGHTNET)) {
     return BETTY_ERR_UNSUPPORTED;
   }
-  *cache = &h;
+  *cache = (MlpHvpCache*)&h;     // handed out as an opaque handle
   return BETTY_OK;
 }
 
@@ -786,7 +797,7 @@ struct SeriesSink { const float* v; float alpha; float* out; };
 
 // H u.  Without a sink the product is written to Hu; with one, u is the partial sum so far and the
 // Horner step is applied inside the weight-gradient products and bias column sums (Hu is not used).
-static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* u, float* Hu,
+static betty_status hvp_impl(Ctx& c, const betty_level* L, HvpCache* h, const float* u, float* Hu,
                              const SeriesSink* sink) {
   const size_t mark = c.arena.mark();
   const Net& n = h->net;
@@ -809,25 +820,25 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
   RPass rp;
   BETTY_TRY(rforward(c, n, ps, u, rp, h));
   const int64_t C = n.w[n.L];
-  bf16* Rd;
+  op16* Rd;
   {
     const int64_t ld = ld8(C);
-    Rd = c.arena.alloc<bf16>((size_t)(B * ld));
+    Rd = c.arena.alloc<op16>((size_t)(B * ld));
     if (!Rd) return BETTY_ERR_WORKSPACE;
     launch_pdl(k_r_delta_top, dim3(grid_for(B * 32)), dim3(256), 0, c.stream, ps.p, rp.Ra[n.L - 1], h->coef, B > 0 ? 1.f / (float)B : 0.f, Rd,
                                                          B, C, ld);
     BETTY_LAUNCH_CHECK();
   }
-  const bool leave16 = sink && h->dir16[0];     // the weight-HVP epilogues also leave the bf16 copy of the new partial sum in dir16
+  const bool leave16 = sink && h->dir16[0];     // the weight-HVP epilogues also leave the op16 copy of the new partial sum in dir16
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
-    bf16* Rdp = nullptr;
+    op16* Rdp = nullptr;
     if (l > 0) {  // R dh = Rdelta W_l + delta_l U_l ; Rdelta_{l-1} = Rdh*act' + dh*act''*Ra
       // (before this layer's weight product, whose epilogue may overwrite U_l with the next term)
       const int64_t ldp = ld8(K);
-      Rdp = c.arena.alloc<bf16>((size_t)(B * ldp));
+      Rdp = c.arena.alloc<op16>((size_t)(B * ldp));
       if (!Rdp) return BETTY_ERR_WORKSPACE;
-      if (ldp != K) cudaMemsetAsync(Rdp, 0, (size_t)(B * ldp) * sizeof(bf16), c.stream);
+      if (ldp != K) cudaMemsetAsync(Rdp, 0, (size_t)(B * ldp) * sizeof(op16), c.stream);
       GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.C = nullptr; g.ldc = K; g.beta = 0.f; g.npairs = 2;
       g.p[0] = gemm_pair(Rd, ldd, false, n.W[l], n.ldw[l], false, (int)N);
       g.p[1] = gemm_pair(ps.delta[l], ldd, false, rp.U[l], n.ldw[l], false, (int)N);
@@ -866,13 +877,14 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, MlpHvpCache* h, const
   return BETTY_OK;
 }
 
-// Gives the HVPs of a series solve persistent storage for the bf16 copy of the current term (allocated
+// Gives the HVPs of a series solve persistent storage for the op16 copy of the current term (allocated
 // at the arena's current top: call it after mlpfam_hvp_begin and before the first HVP of the solve).
-betty_status mlpfam_hvp_keep_direction(Ctx& c, MlpHvpCache* h) {
+betty_status mlpfam_hvp_keep_direction(Ctx& c, MlpHvpCache* handle) {
+  HvpCache* h = (HvpCache*)handle;
   if (!h || h->dir16[0]) return BETTY_OK;
   const Net& n = h->net;
   for (int l = 0; l < n.L; ++l) {
-    h->dir16[l] = c.arena.alloc<bf16>((size_t)(n.w[l + 1] * n.ldw[l]));
+    h->dir16[l] = c.arena.alloc<op16>((size_t)(n.w[l + 1] * n.ldw[l]));
     if (!h->dir16[l]) { h->dir16[0] = nullptr; return BETTY_ERR_WORKSPACE; }
   }
   h->dir16_of = nullptr;
@@ -880,17 +892,18 @@ betty_status mlpfam_hvp_keep_direction(Ctx& c, MlpHvpCache* h) {
 }
 
 betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* u, float* Hu) {
-  return hvp_impl(c, L, h, u, Hu, nullptr);
+  return hvp_impl(c, L, (HvpCache*)h, u, Hu, nullptr);
 }
 
 betty_status mlpfam_hvp_series(Ctx& c, const betty_level* L, MlpHvpCache* h, const float* s, const float* v, float alpha,
                                float* s_out) {
   SeriesSink sink = {v, alpha, s_out};
-  return hvp_impl(c, L, h, s, nullptr, &sink);
+  return hvp_impl(c, L, (HvpCache*)h, s, nullptr, &sink);
 }
 
-betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* h, const betty_level* wrt, const float* q,
+betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* handle, const betty_level* wrt, const float* q,
                           float* out) {
+  HvpCache* h = (HvpCache*)handle;
   const size_t mark = c.arena.mark();
   const Parts P = parts_of(L);
   const Net& n = h->net;
@@ -930,15 +943,15 @@ betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int fi
   const size_t mark = c.arena.mark();
   const Parts P = parts_of(L);
   // The gradient step is taken inside the weight-gradient products' epilogues, which also write the
-  // bf16 copy of the updated matrices for the next step: one cast at the start, none afterwards.
+  // op16 copy of the updated matrices for the next step: one cast at the start, none afterwards.
   Net n;
   BETTY_TRY(net_setup(c, P.mlp, n));
-  bf16* alt[MAXL];
+  op16* alt[MAXL];
   for (int l = 0; l < n.L; ++l) {
     const size_t cnt = (size_t)(n.w[l + 1] * n.ldw[l]);
-    alt[l] = c.arena.alloc<bf16>(cnt);
+    alt[l] = c.arena.alloc<op16>(cnt);
     if (!alt[l]) return BETTY_ERR_WORKSPACE;
-    if (n.ldw[l] != n.w[l]) cudaMemsetAsync(alt[l], 0, cnt * sizeof(bf16), c.stream);
+    if (n.ldw[l] != n.w[l]) cudaMemsetAsync(alt[l], 0, cnt * sizeof(op16), c.stream);
   }
   for (int s = 0; s < n_steps; ++s) {
     const size_t m2 = c.arena.mark();
@@ -950,7 +963,7 @@ betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int fi
     sink.lam = P.lam ? P.lam->params : nullptr;
     sink.sgd = true; sink.lr = lr_at(L, first_step + s); sink.master = L->params; sink.Wnext = alt;
     BETTY_TRY(backward(c, n, ps, coef, sink));
-    for (int l = 0; l < n.L; ++l) { bf16* t = n.W[l]; n.W[l] = alt[l]; alt[l] = t; }
+    for (int l = 0; l < n.L; ++l) { op16* t = n.W[l]; n.W[l] = alt[l]; alt[l] = t; }
     c.arena.release(m2);
   }
   c.arena.release(mark);
@@ -959,7 +972,7 @@ betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int fi
 
 // Finite difference of dC/dc at x +- eps v.  For the weight-net constraint the two perturbed forward
 // passes carry the perturbation separately from the base activations (base + delta operands), so that
-// an eps*v far below bf16 resolution of the weights survives the bf16 matrix products.
+// an eps*v far below op16 resolution of the weights survives the op16 matrix products.
 betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
                        float eps0, float alpha, float* out, bool accumulate) {
   if (L->loss != BETTY_LOSS_MLP_CE_REWEIGHT) return BETTY_ERR_UNSUPPORTED;
@@ -979,9 +992,9 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
   if (!P.theta || wrt != P.theta) return BETTY_ERR_INVALID_ARG;
   BETTY_TRY(forward(c, n, L, ps));
   const int64_t B = ps.B, C = n.w[n.L];
-  bf16* E[MAXL];
+  op16* E[MAXL];
   for (int l = 0; l < n.L; ++l) {
-    E[l] = c.arena.alloc<bf16>((size_t)(n.w[l + 1] * n.ldw[l]));
+    E[l] = c.arena.alloc<op16>((size_t)(n.w[l + 1] * n.ldw[l]));
     if (!E[l]) return BETTY_ERR_WORKSPACE;
     BETTY_TRY(cast_matrix(c, v + n.woff[l], E[l], n.w[l + 1], n.w[l], n.ldw[l], vnorm2, eps0));
   }
@@ -995,8 +1008,8 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
   for (int sgn = 0; sgn < 2; ++sgn) {
     const float sign = sgn == 0 ? 1.f : -1.f;
     const size_t m2 = c.arena.mark();
-    const bf16* hp = ps.h[0];      // perturbed input of the layer (layer 0: the data itself)
-    const bf16* dh = nullptr;      // its difference from the base input
+    const op16* hp = ps.h[0];      // perturbed input of the layer (layer 0: the data itself)
+    const op16* dh = nullptr;      // its difference from the base input
     for (int l = 0; l < n.L; ++l) {
       const int64_t N = n.w[l + 1], K = n.w[l];
       BETTY_ALLOC(da, float, c, (size_t)(B * N));
@@ -1006,11 +1019,11 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
       BETTY_TRY(gemm(c, g));
       if (l < n.L - 1) {
         const size_t cnt = (size_t)(B * ps.ldh[l + 1]);
-        BETTY_ALLOC(hn, bf16, c, cnt);
-        BETTY_ALLOC(dn, bf16, c, cnt);
+        BETTY_ALLOC(hn, op16, c, cnt);
+        BETTY_ALLOC(dn, op16, c, cnt);
         if (ps.ldh[l + 1] != N) {
-          cudaMemsetAsync(hn, 0, cnt * sizeof(bf16), c.stream);
-          cudaMemsetAsync(dn, 0, cnt * sizeof(bf16), c.stream);
+          cudaMemsetAsync(hn, 0, cnt * sizeof(op16), c.stream);
+          cudaMemsetAsync(dn, 0, cnt * sizeof(op16), c.stream);
         }
         launch_pdl(k_fd_act, dim3(grid_for(B * N)), dim3(256), 0, c.stream, ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, hn, dn, nullptr, B, N,
                                                        ps.ldh[l + 1], n.act);
@@ -1034,4 +1047,5 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
   return BETTY_OK;
 }
 
+}  // namespace BETTY_FAM
 }  // namespace betty

@@ -87,23 +87,28 @@ static inline float lr_at(const betty_level* L, int step_in_call) {
   return L->lr;
 }
 
-struct MlpHvpCache;  // base forward/backward state shared by the HVPs of one solve
-betty_status mlpfam_validate(const betty_level* L);
-size_t mlpfam_workspace(const betty_level* L);
-betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);
-betty_status mlpfam_share_weights(Ctx& c, const betty_level* M);
-void mlpfam_unshare_weights(Ctx& c);
-betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache);
-betty_status mlpfam_hvp_keep_direction(Ctx& c, MlpHvpCache* cache);
-betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* u, float* Hu);
-// One Neumann-series iteration with the update fused into the HVP's weight-gradient products:
-// One Horner step of the Neumann series: s_out = v + (s - alpha * H s)   (s_out == s allowed)
-betty_status mlpfam_hvp_series(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* s, const float* v, float alpha,
-                               float* s_out);
-betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* cache, const betty_level* wrt, const float* q,
-                          float* out);
-betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step = 0);
-betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
-                       float eps0, float alpha, float* out, bool accumulate);
+struct MlpHvpCache;  // opaque handle: base forward/backward state shared by the HVPs of one solve
+
+// The MLP families exist once per 16-bit operand type (see common.cuh): identical declarations in two namespaces.
+#define BETTY_DECLARE_MLP_FAMILY(NS)                                                                                   \
+  namespace NS {                                                                                                       \
+  betty_status mlpfam_validate(const betty_level* L);                                                                  \
+  size_t mlpfam_workspace(const betty_level* L);                                                                       \
+  betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out);                          \
+  betty_status mlpfam_share_weights(Ctx& c, const betty_level* M);                                                     \
+  void mlpfam_unshare_weights(Ctx& c);                                                                                 \
+  betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache);                                    \
+  betty_status mlpfam_hvp_keep_direction(Ctx& c, MlpHvpCache* cache);                                                  \
+  betty_status mlpfam_hvp(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* u, float* Hu);                \
+  betty_status mlpfam_hvp_series(Ctx& c, const betty_level* L, MlpHvpCache* cache, const float* s, const float* v, float alpha, \
+                                 float* s_out);                                                                        \
+  betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* cache, const betty_level* wrt, const float* q,  \
+                            float* out);                                                                               \
+  betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step = 0);                       \
+  betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,    \
+                         float eps0, float alpha, float* out, bool accumulate);                                        \
+  }
+BETTY_DECLARE_MLP_FAMILY(fam_bf16)
+BETTY_DECLARE_MLP_FAMILY(fam_f16)
 
 }  // namespace betty

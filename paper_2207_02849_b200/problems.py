@@ -37,11 +37,15 @@ def _act(name):
     return bt.ACT_RELU if name == "relu" else bt.ACT_GELU
 
 
-def reweight_levels(inp):
-    theta = bt.Level(bt.LOSS_MLP_CE, bt.PARAM_WEIGHTNET, dev(inp.theta), X=dev(inp.val.X, torch.bfloat16),
+def reweight_levels(inp, operand_dtype=torch.bfloat16):
+    """operand_dtype: torch.bfloat16 (default) or torch.float16, the type of the batches and of the classifier's
+    matrix-product operands."""
+    theta = bt.Level(bt.LOSS_MLP_CE, bt.PARAM_WEIGHTNET, dev(inp.theta), X=dev(inp.val.X, operand_dtype),
                      y=dev(inp.val.y))
-    w = bt.Level(bt.LOSS_MLP_CE_REWEIGHT, bt.PARAM_MLP, dev(inp.w), X=dev(inp.train.X, torch.bfloat16),
+    w = bt.Level(bt.LOSS_MLP_CE_REWEIGHT, bt.PARAM_MLP, dev(inp.w), X=dev(inp.train.X, operand_dtype),
                  y=dev(inp.train.y), widths=inp.widths, activation=_act(inp.activation), lr=inp.lr)
+    if operand_dtype == torch.float16:
+        w.set_precision(bt.BETTY_F16)
     w.set_constraints([theta])
     theta.set_constraints([w])
     return w, theta
