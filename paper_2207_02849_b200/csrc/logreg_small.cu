@@ -541,6 +541,227 @@ __global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(8192 / CPT, 1) k
   cluster_barrier();    // no CTA may leave while a neighbour can still send to it
 }
 
+// The hypergradient (mode 1) and ITD-RMAD (mode 2) loops in the same wide-row form: CPT columns of a row per
+// thread on 8192 / CPT threads.  One register array serves both matrices: it holds the training rows during
+// the training passes and is refilled from global memory (256 KB at most, L2-resident) around the single pass
+// over the validation rows, so a thread never keeps two row slices alive.  Same passes, same exchange, same
+// solver arithmetic in the same order as k_logreg_small; only the number of threads that share a row differs.
+template <int TPR, int CPT, class Post>
+__device__ __forceinline__ bool wide_pass(const float (&x)[CPT], float yv, bool has, int family, float inv_n, int kind,
+                                          const float* vv, const float* wt, float* part, float* cpart, uint64_t* bar,
+                                          uint32_t parity, Post post, uint32_t rank) {
+  constexpr int SW_T = 8192 / CPT, d = CPT * TPR;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cb = CPT * (tid & (TPR - 1));
+  float s0 = 0.f, s1 = 0.f, z0 = 0.f, z1 = 0.f;
+#pragma unroll
+  for (int k = 0; k < CPT / 4; ++k) {
+    const float4 v = *(const float4*)(vv + cb + 4 * k);
+    s0 += x[4 * k] * v.x + x[4 * k + 1] * v.y;
+    s1 += x[4 * k + 2] * v.z + x[4 * k + 3] * v.w;
+    if (kind == 2) {
+      const float4 u = *(const float4*)(wt + cb + 4 * k);
+      z0 += x[4 * k] * u.x + x[4 * k + 1] * u.y;
+      z1 += x[4 * k + 2] * u.z + x[4 * k + 3] * u.w;
+    }
+  }
+  float sdot = s0 + s1, zdot = z0 + z1;
+#pragma unroll
+  for (int o = TPR >> 1; o > 0; o >>= 1) {
+    sdot += __shfl_xor_sync(0xffffffffu, sdot, o);
+    if (kind == 2) zdot += __shfl_xor_sync(0xffffffffu, zdot, o);
+  }
+  float cf = 0.f;
+  if (has) {
+    if (kind == 0) cf = family == 0 ? -yv * sigm(-yv * sdot) * inv_n : (sdot - yv);
+    else if (kind == 1) cf = yv * sdot;
+    else { const float sg = sigm(zdot); cf = (family == 0 ? sg * (1.f - sg) * inv_n : 1.f) * sdot; }
+  }
+  float col[CPT];
+#pragma unroll
+  for (int k = 0; k < CPT; ++k) col[k] = cf * x[k];
+  int off = 0;
+  bool writer = true;
+  WarpColumnSum<TPR, CPT, CPT>::run(col, lane, off, writer);
+  constexpr int NF = CPT / (32 / TPR) > 0 ? CPT / (32 / TPR) : 1;
+  if (writer) {
+#pragma unroll
+    for (int i = 0; i < NF; ++i) part[warp * SM_PS + cb + off + i] = col[i];
+  }
+  __syncthreads();
+  return exchange_cols(part, SW_T / 32, d, cpart, bar, parity, post, rank);
+}
+
+template <int TPR, int CPT>
+__global__ void __cluster_dims__(SM_CL, 1, 1) __launch_bounds__(8192 / CPT, 1) k_logreg_small_wide(SmallArgs a) {
+  constexpr int SW_T = 8192 / CPT, d = CPT * TPR;
+  __shared__ __align__(16) float vec[SM_NVEC * SM_MAXD];
+  __shared__ __align__(16) float part[(SW_T / 32) * SM_PS];
+  __shared__ float cpart[2 * SM_CL * SM_MAXD];
+  __shared__ float red[32];
+  __shared__ __align__(8) uint64_t xbar[2];
+  extern __shared__ __align__(16) float traj[];     // [n_steps][d] stored iterates (ITD-RMAD)
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const int tid = threadIdx.x;
+  float *w = vec, *lam = vec + SM_MAXD, *v = vec + 3 * SM_MAXD, *q = vec + 4 * SM_MAXD, *r = vec + 5 * SM_MAXD,
+        *p = vec + 6 * SM_MAXD, *h = vec + 7 * SM_MAXD, *t = vec + 8 * SM_MAXD;
+  const int R = a.rows_per_cta, Rv = a.rows_per_cta_v, row = tid / TPR, cb = CPT * (tid & (TPR - 1));
+  const int64_t r0 = (int64_t)rank * R, r0v = (int64_t)rank * Rv;
+  int rows = (int)(a.n - r0 < R ? a.n - r0 : R); if (rows < 0) rows = 0;
+  int rowsv = (int)(a.nv - r0v < Rv ? a.nv - r0v : Rv); if (rowsv < 0) rowsv = 0;
+  const bool has = row < rows, hasv = row < rowsv;
+  float x[CPT];
+  float yreg = 0.f, curvreg = 0.f;
+  // this thread's CPT columns of its row of the training (which = 0) or validation (which = 1) matrix
+  auto load_row = [&](int which) {
+    const bool present = which == 0 ? has : hasv;
+#pragma unroll
+    for (int k = 0; k < CPT; ++k) x[k] = 0.f;
+    yreg = 0.f;
+    if (present) {
+      const float* base = which == 0 ? a.X + (r0 + row) * d : a.Xv + (r0v + row) * d;
+      const float4* src = (const float4*)(base + cb);
+#pragma unroll
+      for (int k = 0; k < CPT / 4; ++k) { const float4 u = src[k]; x[4 * k] = u.x; x[4 * k + 1] = u.y; x[4 * k + 2] = u.z; x[4 * k + 3] = u.w; }
+      yreg = which == 0 ? a.y[r0 + row] : a.yv[r0v + row];
+    }
+  };
+  for (int j = tid; j < d; j += SW_T) { w[j] = a.w[j]; lam[j] = a.lam[j]; }
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_u32(&xbar[0])));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_u32(&xbar[1])));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  cluster_barrier();    // every CTA of the cluster is running, its barriers set up, before anyone sends to it
+  const float inv_n = a.n > 0 ? 1.f / (float)a.n : 0.f, inv_nv = a.nv > 0 ? 1.f / (float)a.nv : 0.f;
+  int pb = 0; uint32_t ph = 0; bool alive = true;
+  auto train_pass = [&](int kind, const float* vv, const float* wt, auto post) {
+    const bool ok = wide_pass<TPR, CPT>(x, kind == 0 ? yreg : curvreg, has, a.family, inv_n, kind, vv, wt, part,
+                                        cpart + pb * SM_CL * SM_MAXD, &xbar[pb], (ph >> pb) & 1u, post, rank);
+    alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
+  };
+  // gradient of the upper cost at vv over the validation rows: the row registers are lent to them for one pass
+  auto valid_pass = [&](const float* vv, float* res) {
+    load_row(1);
+    const bool ok = wide_pass<TPR, CPT>(x, yreg, hasv, a.family_up, inv_nv, 0, vv, nullptr, part,
+                                        cpart + pb * SM_CL * SM_MAXD, &xbar[pb], (ph >> pb) & 1u,
+                                        [res](int j, float sum) { res[j] = sum; }, rank);
+    alive = alive && ok; ph ^= 1u << pb; pb ^= 1;
+    load_row(0);
+  };
+
+  if (a.mode == 2) {
+    // ITD-RMAD: unrolled steps with every iterate kept on chip, then the reverse sweep (see k_logreg_small)
+    const float lr = a.lr;
+    load_row(0);
+    for (int s = 0; s < a.n_steps && alive; ++s) {
+      float* ws = traj + (size_t)s * d;
+      train_pass(0, w, nullptr, [=](int j, float gsum) { const float wj = w[j]; ws[j] = wj; w[j] = wj - lr * (gsum + lam[j] * wj); });
+    }
+    valid_pass(w, v);
+    for (int j = tid; j < d; j += SW_T) q[j] = 0.f;
+    __syncthreads();
+    for (int s = a.n_steps - 1; s >= 0 && alive; --s) {
+      const float* wt = traj + (size_t)s * d;
+      train_pass(2, v, wt, [=](int j, float hsum) {
+        const float aj = v[j];
+        q[j] -= lr * (wt[j] * aj);
+        v[j] = aj - lr * (hsum + lam[j] * aj);
+      });
+    }
+    if (rank == 0)
+      for (int j = tid; j < d; j += SW_T) { a.out[j] = q[j]; a.w[j] = w[j]; }
+  } else {
+    valid_pass(w, v);          // leaves the training rows in the registers
+    if (a.method == BETTY_FD) {
+      const float nv2 = vdot(v, v, d, red);
+      for (int j = tid; j < d; j += SW_T) {
+        float o = 0.f;
+        if (nv2 > 0.f) {
+          const double eps = (double)a.eps0 / sqrt((double)nv2);
+          const double wp = (double)w[j] + eps * (double)v[j], wm = (double)w[j] - eps * (double)v[j];
+          o = (float)(-(double)a.alpha * (0.5 * wp * wp - 0.5 * wm * wm) / (2.0 * eps));
+        }
+        if (rank == 0) a.out[j] = o;
+      }
+    } else {
+      {   // curvature weight of this thread's row at the current w (constant over the solve)
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < CPT / 4; ++k) {
+          const float4 u = *(const float4*)(w + cb + 4 * k);
+          s += x[4 * k] * u.x + x[4 * k + 1] * u.y + x[4 * k + 2] * u.z + x[4 * k + 3] * u.w;
+        }
+#pragma unroll
+        for (int o = TPR >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const float sg = sigm(s);
+        curvreg = a.family == 0 ? sg * (1.f - sg) * inv_n : 1.f;
+      }
+      float qscale = 1.f;
+      if (a.method == BETTY_NEUMANN) {
+        for (int j = tid; j < d; j += SW_T) { t[j] = v[j]; q[j] = v[j]; }
+        __syncthreads();
+        for (int k = 0; k < a.K && alive; ++k) {
+          const float alpha = a.alpha;
+          train_pass(1, t, nullptr, [=](int j, float hsum) {
+            const float tn = t[j] - alpha * (hsum + lam[j] * t[j]);
+            t[j] = tn; q[j] += tn;
+          });
+        }
+        qscale = a.alpha;
+      } else {
+        for (int j = tid; j < d; j += SW_T) { q[j] = 0.f; r[j] = v[j]; p[j] = v[j]; }
+        __syncthreads();
+        float rho = vdot(r, r, d, red);
+        const float stop = a.tol * a.tol * rho;
+        int iters = 0, status = 0;
+        bool active = rho > stop;
+        if (!isfinite(rho)) { status = BETTY_ERR_NONFINITE; active = false; }
+        for (int k = 0; k < a.K && active; ++k) {
+          train_pass(1, p, nullptr, [=](int j, float hsum) { h[j] = hsum + lam[j] * p[j]; });
+          if (!alive) break;
+          const float gamma = vdot(p, h, d, red);
+          if (!isfinite(gamma)) { status = BETTY_ERR_NONFINITE; break; }
+          if (!(gamma > 0.f)) { status = BETTY_ERR_BREAKDOWN; break; }
+          const float al = rho / gamma;
+          float rr = 0.f;
+          if (tid < d) {
+            q[tid] += al * p[tid];
+            const float rn = r[tid] - al * h[tid];
+            r[tid] = rn; rr = rn * rn;
+          }
+          const float rho_new = vsum(rr, d, red);
+          const float beta = rho_new / rho;
+          for (int j = tid; j < d; j += SW_T) p[j] = r[j] + beta * p[j];
+          __syncthreads();
+          rho = rho_new;
+          ++iters;
+          if (!isfinite(rho)) { status = BETTY_ERR_NONFINITE; break; }
+          if (rho <= stop) break;
+        }
+        if (rank == 0 && tid == 0) {
+          a.sb->cg_iters = iters;
+          if (status) record_status(a.sb, status);
+        }
+      }
+      if (rank == 0)
+        for (int j = tid; j < d; j += SW_T) a.out[j] = -qscale * w[j] * q[j];
+    }
+  }
+  if (!alive && tid == 0) record_status(a.sb, BETTY_ERR_TIMEOUT);
+  cluster_barrier();    // no CTA may leave while a neighbour can still send to it
+}
+
+template <int TPR, int CPT>
+static betty_status launch_wide(Ctx& c, const SmallArgs& a, size_t traj_bytes) {
+  static SmemLimit limit = {};      // per form and per device
+  if (traj_bytes > 0) BETTY_TRY(ensure_dynamic_smem(k_logreg_small_wide<TPR, CPT>, limit, traj_bytes));
+  k_logreg_small_wide<TPR, CPT><<<SM_CL, 8192 / CPT, traj_bytes, c.stream>>>(a);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
 static size_t small_smem_bytes(int R, int Rv, int d, int64_t traj_floats) {
   size_t floats = (size_t)R * d + (size_t)Rv * d + R + Rv + R + (R > Rv ? R : Rv) + (size_t)SM_NVEC * SM_MAXD + 32 * SM_PS +
                   2 * SM_CL * SM_MAXD + 32 + (size_t)traj_floats;
@@ -577,6 +798,19 @@ static betty_status launch_small(Ctx& c, SmallArgs& a) {
     }
     BETTY_LAUNCH_CHECK();
     return BETTY_OK;
+  }
+  // hypergradient and ITD-RMAD modes: the wide-row form under the same conditions (power-of-two width of at
+  // least 16, at most 8192 / d rows of either matrix per CTA), as long as the stored iterates fit beside its
+  // 43 KB of static shared memory
+  const size_t traj_bytes = a.mode == 2 ? (size_t)a.n_steps * a.d * sizeof(float) : 0;
+  if (a.mode != 0 && a.in_regs && a.d >= 16 && traj_bytes <= 160 * 1024) {
+    switch (a.d) {
+      case 16: return launch_wide<1, 16>(c, a, traj_bytes);
+      case 32: return launch_wide<1, 32>(c, a, traj_bytes);
+      case 64: return launch_wide<1, 64>(c, a, traj_bytes);
+      case 128: return launch_wide<2, 64>(c, a, traj_bytes);
+      default: return launch_wide<8, 32>(c, a, traj_bytes);   // d = 256
+    }
   }
   const size_t smem = small_smem_bytes(a.rows_per_cta, a.rows_per_cta_v, a.d, a.mode == 2 ? (int64_t)a.n_steps * a.d : 0);
   static SmemLimit limit = {};      // per device
