@@ -19,6 +19,10 @@ quadratic        1/2 |A w - b|^2 of a constraining w          (upper loss for th
 mlp_ce_reweight  App. A "Classifier": mean_i r_i * CE_i with r_i = sigmoid(weightnet(CE_i
                  detached)), plus 1/2 sum_l exp(lambda_l) |W_l|^2 when a log-weight-decay
                  constraint is attached
+                 With a label-correction constraint attached (App. A "Correcting & Reweighting" listing) the
+                 per-sample loss is the cross-entropy against the corrected soft label, see cn_forward.
+mlp_ce_correct   App. A "Correct": mean CE of a constraining classifier on this level's batch plus the
+                 mean CE of the correction net's own soft labels (its linear + softmax part) on the same batch
 mlp_ce           App. A "Reweight": plain mean cross-entropy of a constraining classifier
 weightnet_detect mean_j (sigmoid(weightnet(CE_j(w))) - clean_j)^2 + mu/2 |theta|^2, where the
                  per-sample loss is NOT detached (w is a constraining parameter of this cost)
@@ -39,7 +43,7 @@ WN_H = 100  # hidden width of the 1-100-1 weight net (App. C, "Meta-Weight-Netwo
 @dataclass(eq=False)
 class Level:
     loss: str
-    param_kind: str                    # 'vector' | 'mlp' | 'weightnet' | 'logwd'
+    param_kind: str                    # 'vector' | 'mlp' | 'weightnet' | 'logwd' | 'correctnet'
     params: np.ndarray                 # flat fp64 (master copy)
     X: Optional[np.ndarray] = None
     y: Optional[np.ndarray] = None
@@ -201,9 +205,10 @@ def _onehot(y, C):
     return e
 
 
-def _mlp_backward(Ws, h, a, delta_top, act):
+def _mlp_backward(Ws, h, a, delta_top, act, extra_dh_last=None):
     """Reverse sweep from delta_top = dC/d(logits).  Returns gW, gb and the per-layer
-    delta_l = dC/da_l and dh_l = dC/dh_l (dh[l] pairs with a[l-1])."""
+    delta_l = dC/da_l and dh_l = dC/dh_l (dh[l] pairs with a[l-1]).  extra_dh_last: a further
+    dependence of the cost on the last hidden activation (the input of the top layer), added to its dh."""
     L = len(Ws)
     gW, gb, deltas, dhs = [None] * L, [None] * L, [None] * L, [None] * L
     delta = delta_top
@@ -213,6 +218,8 @@ def _mlp_backward(Ws, h, a, delta_top, act):
         gb[l] = delta.sum(axis=0)
         if l > 0:
             dhs[l] = delta @ Ws[l]
+            if l == L - 1 and extra_dh_last is not None:
+                dhs[l] = dhs[l] + extra_dh_last
             delta = dhs[l] * _act_d1(act, a[l - 1])
     return gW, gb, deltas, dhs
 
@@ -256,6 +263,85 @@ def wn_grad_s(theta, ell, hid, mask):
 def wn_ds_dell(theta, mask):
     a1, b1, a2, b2 = wn_unpack(theta)
     return (mask * (a1 * a2)[None, :]).sum(axis=1)
+
+
+# ------------------------------------------------------------------ label-correction net
+# Sec. 5.1 / App. C "Correct Network": it "takes the penultimate activation from the classification network, and
+# outputs soft labels through the linear layer and the softmax layer", and these are "interpolated with the
+# original labels via the reweighting scheme which is achieved with 2-layer MLP".  Reading: with h the last
+# hidden activation of the classifier (width H) and y the given label,
+#     s   = softmax(A h + a0)                       soft label, A [C, H]
+#     rho = sigmoid(a2 . relu(A1 h + b1) + b2)      interpolation weight; hidden width 100 like the weight net;
+#                                                   the paper does not name the MLP's input: the same h
+#     new = rho * onehot(y) + (1 - rho) * s
+# alpha = [A, a0, A1, b1, a2, b2] flat, C*H + C + 100*H + 201 parameters.
+def cn_size(H, C):
+    return C * H + C + WN_H * H + 2 * WN_H + 1
+
+
+def cn_unpack(alpha, H, C):
+    o = 0
+    A = alpha[o:o + C * H].reshape(C, H); o += C * H
+    a0 = alpha[o:o + C]; o += C
+    A1 = alpha[o:o + WN_H * H].reshape(WN_H, H); o += WN_H * H
+    b1 = alpha[o:o + WN_H]; o += WN_H
+    a2 = alpha[o:o + WN_H]; o += WN_H
+    b2 = alpha[o]; o += 1
+    assert o == alpha.size, "correction-net vector does not match the classifier's widths"
+    return A, a0, A1, b1, a2, b2
+
+
+def cn_forward(alpha, hlast, y, C):
+    """Returns s, rho, new labels and the hidden pieces (mask, hid) for the backward formulas."""
+    A, a0, A1, b1, a2, b2 = cn_unpack(alpha, hlast.shape[1], C)
+    t = hlast @ A.T + a0
+    ts = t - t.max(axis=1, keepdims=True)
+    s = np.exp(ts) / np.exp(ts).sum(axis=1, keepdims=True)
+    pre = hlast @ A1.T + b1
+    mask = (pre > 0.0).astype(np.float64)
+    hid = pre * mask
+    rho = expit(hid @ a2 + b2)
+    new = rho[:, None] * _onehot(y, C) + (1.0 - rho)[:, None] * s
+    return s, rho, new, mask, hid
+
+
+def _cn_sample_derivs(alpha, hlast, y, C, logp, s, rho, mask):
+    """Per-sample derivatives of l_i = -sum_c new_c log p_c with respect to the correction net's two
+    pre-activations: dt = dl/d(A h + a0) [B, C] and dpre = dl/d(A1 h + b1) [B, 100], plus dm = dl/dm [B]."""
+    A, a0, A1, b1, a2, b2 = cn_unpack(alpha, hlast.shape[1], C)
+    g = -(1.0 - rho)[:, None] * logp                                  # dl/ds
+    dt = s * (g - (s * g).sum(axis=1, keepdims=True))                 # back through the softmax
+    D = -logp[np.arange(y.shape[0]), y] + (s * logp).sum(axis=1)      # dl/drho = -<onehot - s, log p>
+    dm = D * rho * (1.0 - rho)
+    dpre = mask * a2[None, :] * dm[:, None]
+    return dt, dpre, dm
+
+
+def _cn_pack_grad(coef, dt, dpre, dm, hlast, hid):
+    """sum_i coef_i * d l_i / d alpha from the per-sample pieces."""
+    gt, gp = coef[:, None] * dt, coef[:, None] * dpre
+    return np.concatenate([(gt.T @ hlast).reshape(-1), gt.sum(axis=0), (gp.T @ hlast).reshape(-1), gp.sum(axis=0),
+                           ((coef * dm)[:, None] * hid).sum(axis=0), [np.sum(coef * dm)]])
+
+
+def _log_softmax(z):
+    zs = z - z.max(axis=1, keepdims=True)
+    return zs - np.log(np.exp(zs).sum(axis=1, keepdims=True))
+
+
+def _corrected(L: Level, over, h, a, y):
+    """Soft-label loss pieces of a classifier cost with a correction net attached, else None."""
+    G = _find_constraint(L, "correctnet", required=False) if L.loss == "mlp_ce_reweight" else None
+    if G is None:
+        return None
+    if len(h) < 2:
+        raise ValueError("label correction needs a hidden layer")
+    al = _p(G, over)
+    C = a[-1].shape[1]
+    logp = _log_softmax(a[-1])
+    s, rho, new, mask, hid = cn_forward(al, h[-1], y, C)
+    ell = -(new * logp).sum(axis=1)
+    return dict(level=G, alpha=al, logp=logp, s=s, rho=rho, new=new, mask=mask, hid=hid, ell=ell, hlast=h[-1])
 
 
 # ------------------------------------------------------------------ per-family evaluation
@@ -350,8 +436,16 @@ def cost(L: Level, over=None, r_fixed=None, ell_fixed=None) -> float:
     if L.loss == "mlp_ce":
         _, _, _, _, _, _, ell = _mlp_ce_state(L, over)
         return float(ell.mean())
+    if L.loss == "mlp_ce_correct":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        y = np.asarray(L.y, dtype=np.int64)
+        s, _, _, _, _ = cn_forward(_p(_find(L, "correctnet"), over), h[-1], y, a[-1].shape[1])
+        return float(ell.mean() - np.log(s[np.arange(y.shape[0]), y]).mean())
     if L.loss == "mlp_ce_reweight":
         M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        cn = _corrected(L, over, h, a, np.asarray(L.y, dtype=np.int64))
+        if cn is not None:
+            ell = cn["ell"]
         if ell_fixed is not None:
             ell = np.asarray(ell_fixed, dtype=np.float64)
         r = _reweight_r(L, ell, over)[0] if r_fixed is None else np.asarray(r_fixed)
@@ -400,11 +494,45 @@ def grad(L: Level, wrt: Level, over=None) -> np.ndarray:
         delta = (p - _onehot(np.asarray(L.y, np.int64), p.shape[1])) / B
         gW, gb, _, _ = _mlp_backward(Ws, h, a, delta, M.activation)
         return mlp_pack(gW, gb)
+    if L.loss == "mlp_ce_correct":
+        M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
+        G = _find(L, "correctnet")
+        al = _p(G, over)
+        y = np.asarray(L.y, dtype=np.int64)
+        B, C = L.X.shape[0], p.shape[1]
+        s, _, _, _, _ = cn_forward(al, h[-1], y, C)
+        dt = (s - _onehot(y, C)) / B                                  # d(mean CE of the soft label)/d(A h + a0)
+        if wrt is G:
+            out = np.zeros(al.size)
+            H = h[-1].shape[1]
+            out[:C * H] = (dt.T @ h[-1]).reshape(-1)
+            out[C * H:C * H + C] = dt.sum(axis=0)
+            return out
+        if wrt is M:
+            A = cn_unpack(al, h[-1].shape[1], C)[0]
+            delta = (p - _onehot(y, C)) / B
+            gW, gb, _, _ = _mlp_backward(Ws, h, a, delta, M.activation, extra_dh_last=dt @ A)
+            return mlp_pack(gW, gb)
+        return np.zeros(n_out)
     if L.loss == "mlp_ce_reweight":
         M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
         B = L.X.shape[0]
+        y = np.asarray(L.y, np.int64)
+        cn = _corrected(L, over, h, a, y)
+        if cn is not None:
+            ell = cn["ell"]
         r, wn = _reweight_r(L, ell, over)
         kap, lamL = _kappas(L, over, len(Ws))
+        if cn is not None and (wrt is L or wrt is cn["level"]):
+            dt, dpre, dm = _cn_sample_derivs(cn["alpha"], cn["hlast"], y, p.shape[1], cn["logp"], cn["s"], cn["rho"], cn["mask"])
+            if wrt is cn["level"]:
+                return _cn_pack_grad(r / B, dt, dpre, dm, cn["hlast"], cn["hid"])
+            A, _, A1, _, _, _ = cn_unpack(cn["alpha"], cn["hlast"].shape[1], p.shape[1])
+            delta = (r / B)[:, None] * (p - cn["new"])               # the soft label sums to one
+            extra = (r / B)[:, None] * (dt @ A + dpre @ A1)          # the label itself moves with h (not detached)
+            gW, gb, _, _ = _mlp_backward(Ws, h, a, delta, M.activation, extra_dh_last=extra)
+            gW = [g + k * W for g, k, W in zip(gW, kap, Ws)]
+            return mlp_pack(gW, gb)
         if wrt is L:
             delta = (r / B)[:, None] * (p - _onehot(np.asarray(L.y, np.int64), p.shape[1]))
             gW, gb, _, _ = _mlp_backward(Ws, h, a, delta, M.activation)
@@ -460,6 +588,8 @@ def hvp(L: Level, u: np.ndarray, over=None) -> np.ndarray:
         lam = _p(_find_constraint(L, "vector"), over)
         return L.X.T @ (L.X @ u) + lam * u
     if L.loss == "mlp_ce_reweight":
+        if _find_constraint(L, "correctnet", required=False) is not None:
+            raise ValueError("second derivatives are not offered with label correction (the paper pairs it with AID-FD)")
         # R-operator (forward-over-reverse) through the classifier, r_i held constant.
         M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
         act = M.activation
@@ -512,6 +642,8 @@ def mixed_vjp(L: Level, wrt: Level, q: np.ndarray, over=None) -> np.ndarray:
             return _p(L, over) * q
         raise ValueError("unknown constraint")
     if L.loss == "mlp_ce_reweight":
+        if _find_constraint(L, "correctnet", required=False) is not None:
+            raise ValueError("second derivatives are not offered with label correction (the paper pairs it with AID-FD)")
         M, Ws, bs, h, a, p, ell = _mlp_ce_state(L, over)
         B = L.X.shape[0]
         r, wn = _reweight_r(L, ell, over)

@@ -44,3 +44,16 @@ def three_levels(inp, bf16=True, quant="operands"):
                y=inp.D3.y, aux=inp.D3.clean.astype(np.float64), mu=0.0, constraints=[P2, P1])
     P1.constraints = [P2, P3]
     return P1, P2, P3
+
+
+def correct_reweight_levels(inp, bf16=True, quant="operands"):
+    """Classifier with corrected and reweighted labels below; the reweighting net (plain CE on the clean
+    batch) and the correction net (CE of the classifier + CE of its own soft labels on the clean batch) above."""
+    theta = Level(loss="mlp_ce", param_kind="weightnet", params=inp.theta, X=inp.val.X, y=inp.val.y)
+    alpha = Level(loss="mlp_ce_correct", param_kind="correctnet", params=inp.alpha, X=inp.val.X, y=inp.val.y)
+    w = Level(loss="mlp_ce_reweight", param_kind="mlp", params=inp.w, X=inp.train.X, y=inp.train.y,
+              widths=inp.widths, activation=inp.activation, lr=inp.lr, bf16=bf16, quant=quant,
+              constraints=[theta, alpha])
+    theta.constraints = [w]
+    alpha.constraints = [w]
+    return w, theta, alpha

@@ -178,6 +178,48 @@ def reweight_bilevel(seed: int, widths, B: int, noise: float, *, activation: str
         lower_steps=lower_steps, K=K, alpha=alpha)
 
 
+def correctnet_size(H: int, C: int) -> int:
+    """Parameters of the label-correction net on a classifier with last hidden width H and C classes:
+    a linear layer H -> C for the soft labels and an H-100-1 net for the interpolation weight."""
+    return C * H + C + WEIGHTNET_HIDDEN * H + 2 * WEIGHTNET_HIDDEN + 1
+
+
+def correctnet_init(seed: int, stream: int, H: int, C: int) -> np.ndarray:
+    """[A (C x H), a0 (C), A1 (100 x H), b1 (100), a2 (100), b2]: matrices ~ N(0, 1/fan_in), biases 0."""
+    Hd = WEIGHTNET_HIDDEN
+    A = normal_f32(seed, stream, (C * H,)) * np.float32(1.0 / np.sqrt(H))
+    A1 = normal_f32(seed, stream + 1, (Hd * H,)) * np.float32(1.0 / np.sqrt(H))
+    a2 = normal_f32(seed, stream + 2, (Hd,)) * np.float32(1.0 / np.sqrt(Hd))
+    return np.concatenate([A, np.zeros(C, np.float32), A1, np.zeros(Hd, np.float32), a2, np.zeros(1, np.float32)]).astype(np.float32)
+
+
+@dataclass
+class CorrectReweight:
+    """The extended bilevel program of the paper's noisy-label experiment: one classifier below, a
+    reweighting net and a label-correction net above it, both trained on the clean batch."""
+    widths: tuple
+    activation: str
+    w: np.ndarray
+    theta: np.ndarray        # reweighting net (301)
+    alpha: np.ndarray        # correction net
+    train: ClassBatch
+    val: ClassBatch
+    lr: float = 0.1
+    eps0: float = 0.01
+    fd_alpha: float = 1.0
+
+
+def correct_reweight(seed: int, widths, B: int, noise: float, *, activation: str = "relu",
+                     Bv: int | None = None) -> CorrectReweight:
+    widths = tuple(int(w) for w in widths)
+    T = teacher(seed, widths[0], widths[-1])
+    return CorrectReweight(
+        widths=widths, activation=activation, w=mlp_init(seed, 100, widths), theta=weightnet_init(seed, 200),
+        alpha=correctnet_init(seed, 210, widths[-2], widths[-1]),
+        train=class_batch(seed, 20, B, widths[0], widths[-1], noise, T),
+        val=class_batch(seed, 30, Bv or B, widths[0], widths[-1], 0.0, T))
+
+
 @dataclass
 class ThreeLevel:
     """Three-level chain: P1 classifier w (loss reweighted CE + per-layer exp(lambda) weight

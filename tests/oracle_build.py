@@ -1,2 +1,4 @@
 """Test-side names for the oracle's level builders."""
-from oracle.problems import logreg_levels, quadratic_levels, reweight_levels, three_levels  # noqa: F401
+from oracle.problems import (  # noqa: F401
+    correct_reweight_levels, logreg_levels, quadratic_levels, reweight_levels, three_levels,
+)
