@@ -73,6 +73,12 @@ typedef enum {
    * cross-entropy of sample i, r_i = sigmoid(weightnet(l_i; theta)) with l_i detached: derivatives
    * w.r.t. the MLP treat r_i as constants, derivatives w.r.t. theta treat l_i as data.
    * r_i = 1 without a WEIGHTNET constraint; no decay term without a LOGWD constraint.
+   * With a CORRECTNET constraint alpha (the extended bilevel program of Sec. 5.1) l_i is the cross-entropy against
+   * the corrected soft label  new_i = rho_i onehot(y_i) + (1 - rho_i) s_i,  s_i = softmax(A h_i + a0),
+   * rho_i = sigmoid(a2 . relu(A1 h_i + b1) + b2),  h_i the last hidden activation (width H >= 1 hidden layer needed);
+   * the label is not detached from the classifier.  Gradients (all participants), lower steps and the finite-
+   * difference hypergradient are offered; Hessian-vector and mixed products return BETTY_ERR_UNSUPPORTED (the paper
+   * pairs this program with AID-FD).  Limits: at most 1024 classes, H <= 8192, no loss scaling.
    * X bf16 [n,d], y int32 class ids. */
   BETTY_LOSS_MLP_CE_REWEIGHT = 4,
   /* App. A "Reweight": C = (1/B) sum_i l_i of the first MLP constraint on this level's batch. */
@@ -80,14 +86,21 @@ typedef enum {
   /* C = (1/B) sum_j (sigmoid(weightnet(l_j(w); theta)) - aux_j)^2 + mu/2 |theta|^2 with theta the
    * WEIGHTNET participant and w the MLP participant (own block or constraints); l_j is NOT
    * detached.  aux fp32 [n] in {0,1} (1 = label is clean).  X bf16 [n,d], y int32. */
-  BETTY_LOSS_WEIGHTNET_DETECT = 6
+  BETTY_LOSS_WEIGHTNET_DETECT = 6,
+  /* App. A "Correct" (Sec. 5.1, correcting and reweighting corrupted labels): own block CORRECTNET alpha, constraint
+   * MLP w.  C = (1/B) sum_j l_j(w) + (1/B) sum_j CE(softmax(A h_j + a0), y_j) on this level's (clean) batch, h_j the
+   * classifier's last hidden activation: the classifier's cross-entropy plus that of the correction net's own soft
+   * labels.  X in the classifier's operand type [n,d], y int32. */
+  BETTY_LOSS_MLP_CE_CORRECT = 7
 } betty_loss;
 
 typedef enum {
   BETTY_PARAM_VECTOR = 0,    /* plain vector (logistic/quadratic w, per-feature weight decay) */
   BETTY_PARAM_MLP = 1,       /* classifier weights, layout above */
   BETTY_PARAM_WEIGHTNET = 2, /* 301 parameters of the 1-100-1 weight net */
-  BETTY_PARAM_LOGWD = 3      /* per-layer log weight decay, one per MLP layer */
+  BETTY_PARAM_LOGWD = 3,     /* per-layer log weight decay, one per MLP layer */
+  BETTY_PARAM_CORRECTNET = 4 /* label-correction net on a classifier with last hidden width H and C classes:
+                              * [A (C x H), a0 (C), A1 (100 x H), b1 (100), a2 (100), b2], C*H + C + 100*H + 201 floats */
 } betty_param_kind;
 
 typedef enum { BETTY_NEUMANN = 0, BETTY_CG = 1, BETTY_FD = 2 } betty_method;

@@ -16,8 +16,8 @@ BETTY_OK = 0
  BETTY_ERR_CUDA, BETTY_ERR_NONFINITE, BETTY_ERR_BREAKDOWN, BETTY_ERR_TIMEOUT,
  BETTY_ERR_UNSUPPORTED, BETTY_ERR_CAPACITY) = range(1, 12)
 (LOSS_LOGREG_WD, LOSS_LOGREG, LOSS_QUADRATIC_WD, LOSS_QUADRATIC, LOSS_MLP_CE_REWEIGHT, LOSS_MLP_CE,
- LOSS_WEIGHTNET_DETECT) = range(7)
-PARAM_VECTOR, PARAM_MLP, PARAM_WEIGHTNET, PARAM_LOGWD = range(4)
+ LOSS_WEIGHTNET_DETECT, LOSS_MLP_CE_CORRECT) = range(8)
+PARAM_VECTOR, PARAM_MLP, PARAM_WEIGHTNET, PARAM_LOGWD, PARAM_CORRECTNET = range(5)
 BETTY_NEUMANN, BETTY_CG, BETTY_FD = range(3)
 ACT_RELU, ACT_GELU = range(2)
 BETTY_F32, BETTY_BF16, BETTY_I32, BETTY_F16 = range(4)

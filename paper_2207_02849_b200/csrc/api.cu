@@ -260,7 +260,7 @@ static betty_status validate_level(const betty_level* L) {
   for (int i = 0; i < L->n_constraints; ++i)
     if (!L->constraints[i]) return BETTY_ERR_INVALID_ARG;
   if (L->n_params < 0 || (L->n_params > 0 && !L->params)) return BETTY_ERR_INVALID_ARG;
-  if (L->param_kind < BETTY_PARAM_VECTOR || L->param_kind > BETTY_PARAM_LOGWD) return BETTY_ERR_INVALID_ARG;
+  if (L->param_kind < BETTY_PARAM_VECTOR || L->param_kind > BETTY_PARAM_CORRECTNET) return BETTY_ERR_INVALID_ARG;
   if (L->optimizer < BETTY_OPT_GD || L->optimizer > BETTY_OPT_ADAM) return BETTY_ERR_INVALID_ARG;
   if (L->optimizer != BETTY_OPT_GD && !L->opt_state) return BETTY_ERR_INVALID_ARG;
   if (L->precision != 0 && L->precision != BETTY_BF16 && L->precision != BETTY_F16) return BETTY_ERR_DTYPE;

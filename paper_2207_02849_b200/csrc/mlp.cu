@@ -360,8 +360,10 @@ __global__ void k_wn_backward(const float* theta, const float* dir, const float*
 // ------------------------------------------------------------------ finite-difference pieces
 // da_tot = da + sign*eps*c.  Hidden layer: hp = act(a + da_tot) -> op16, dh = hp - act(a) -> op16.
 // Output layer: z = a + da_tot (fp32).
+// hp32 (nullable, [B, N]): the perturbed activation in fp32, i.e. the rounded base value plus the displacement
+// (what a consumer that is not a matrix product, the label-correction net, evaluates at).
 __global__ void k_fd_act(const float* a, const float* da, const float* cdir, const float* vnorm2, float eps0, float sign,
-                         op16* hpm, op16* dhd, float* zpm, int64_t B, int64_t N, int64_t ldh, int act) {
+                         op16* hpm, op16* dhd, float* zpm, int64_t B, int64_t N, int64_t ldh, int act, float* hp32) {
   pdl_enter();
   const float e = sign * fd_eps(vnorm2, eps0);
   const int64_t total = B * N;
@@ -372,6 +374,7 @@ __global__ void k_fd_act(const float* a, const float* da, const float* cdir, con
     const float h0 = act_f(act, a[i]), hp = act_f(act, a[i] + d);
     hpm[r * ldh + n] = to_op16(hp);
     dhd[r * ldh + n] = to_op16(hp - h0);
+    if (hp32) hp32[i] = from_op16(to_op16(h0)) + (hp - h0);
   }
 }
 __global__ void k_fd_combine(float* out, const float* gp, const float* gm, const float* vnorm2, float eps0, float alpha,
@@ -381,6 +384,194 @@ __global__ void k_fd_combine(float* out, const float* gp, const float* gm, const
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     const float base = accumulate ? out[i] : 0.f;
     out[i] = e > 0.f ? base - alpha * (gp[i] - gm[i]) / (2.f * e) : base;
+  }
+}
+
+
+// ------------------------------------------------------------------ label-correction net
+// (Sec. 5.1 "Correcting & reweighting corrupted labels", its App. A listing and the App. C description.)  With h
+// the classifier's last hidden activation (width H, as the matrix products see it) and y the given label:
+//     s = softmax(A h + a0),   rho = sigmoid(a2 . relu(A1 h + b1) + b2),   new = rho onehot(y) + (1 - rho) s,
+// alpha = [A (C x H), a0 (C), A1 (100 x H), b1 (100), a2 (100), b2].  The classifier's per-sample loss becomes
+// l_i = -sum_c new_ic log p_ic, and the label is not detached from h.  The net is small (C + 100 outputs per sample):
+// it runs on CUDA cores in fp32, one block per sample, every reduction in a fixed order.
+static constexpr int CN_T = 128;          // threads per sample
+static constexpr int CN_MAX_C = 1024;
+static constexpr int CN_MAX_H = 8192;
+struct CnOff { int64_t A, a0, A1, b1, a2, b2, total; };
+__host__ __device__ static inline CnOff cn_offsets(int64_t H, int64_t C) {
+  CnOff o; o.A = 0; o.a0 = C * H; o.A1 = o.a0 + C; o.b1 = o.A1 + WN_H * H; o.a2 = o.b1 + WN_H; o.b2 = o.a2 + WN_H; o.total = o.b2 + 1;
+  return o;
+}
+// sum over the block, same value in every thread; fixed order (warp trees, then the warps in index order)
+__device__ __forceinline__ float cn_block_sum(float v, float* sh) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < CN_T / 32; ++i) t += sh[i];
+  __syncthreads();
+  return t;
+}
+__device__ __forceinline__ float cn_block_max(float v, float* sh) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = -INFINITY;
+  for (int i = 0; i < CN_T / 32; ++i) t = fmaxf(t, sh[i]);
+  __syncthreads();
+  return t;
+}
+// One block per sample.  h16 (operand type, leading dimension ldh) or h32 ([B, H]) is the last hidden activation;
+// z the logits.  Writes hl32 (fp32 copy of h, unless it is h32 itself), logp, s, hid, rho, the new labels and the
+// soft-label loss ell.  Dynamic shared memory: H + 2 C + 100 floats.
+__global__ void __launch_bounds__(CN_T) k_cn_forward(const float* alpha, const op16* h16, int64_t ldh, const float* h32,
+                                                     const float* z, const int32_t* y, int64_t H, int64_t C, float* hl32,
+                                                     float* logp, float* s, float* hid, float* rho, float* newlab, float* ell) {
+  pdl_enter();
+  extern __shared__ float cn_sm[];
+  __shared__ float red[CN_T / 32];
+  float* hrow = cn_sm; float* tb = hrow + H; float* lp = tb + C; float* hd = lp + C;
+  const int64_t row = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const CnOff o = cn_offsets(H, C);
+  for (int64_t j = tid; j < H; j += CN_T) {
+    const float v = h32 ? h32[row * H + j] : from_op16(h16[row * ldh + j]);
+    hrow[j] = v;
+    if (hl32 && !h32) hl32[row * H + j] = v;
+  }
+  // log-softmax of the logits
+  const float* zr = z + row * C;
+  float mx = -INFINITY;
+  for (int64_t c = tid; c < C; c += CN_T) mx = fmaxf(mx, zr[c]);
+  mx = cn_block_max(mx, red);          // also orders the writes of hrow before the reads below
+  float se = 0.f;
+  for (int64_t c = tid; c < C; c += CN_T) se += expf(zr[c] - mx);
+  const float lse = logf(cn_block_sum(se, red));
+  for (int64_t c = tid; c < C; c += CN_T) { const float v = zr[c] - mx - lse; lp[c] = v; logp[row * C + c] = v; }
+  // the C + 100 outputs of the two linear maps: one warp per output, lanes along H
+  for (int64_t e = warp; e < C + WN_H; e += CN_T / 32) {
+    const float* wrow = e < C ? alpha + o.A + e * H : alpha + o.A1 + (e - C) * H;
+    float acc = 0.f;
+    for (int64_t j = lane; j < H; j += 32) acc += wrow[j] * hrow[j];
+#pragma unroll
+    for (int sh = 16; sh > 0; sh >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sh);
+    if (lane == 0) {
+      if (e < C) tb[e] = acc + alpha[o.a0 + e];
+      else hd[e - C] = fmaxf(acc + alpha[o.b1 + (e - C)], 0.f);
+    }
+  }
+  __syncthreads();
+  float tm = -INFINITY;
+  for (int64_t c = tid; c < C; c += CN_T) tm = fmaxf(tm, tb[c]);
+  tm = cn_block_max(tm, red);
+  float ts = 0.f;
+  for (int64_t c = tid; c < C; c += CN_T) ts += expf(tb[c] - tm);
+  ts = cn_block_sum(ts, red);
+  const float m = cn_block_sum(tid < WN_H ? alpha[o.a2 + tid] * hd[tid] : 0.f, red) + alpha[o.b2];
+  const float r = 1.f / (1.f + expf(-m));
+  int32_t yy = y[row];
+  yy = yy < 0 ? 0 : (yy >= C ? (int32_t)C - 1 : yy);
+  float le = 0.f;
+  for (int64_t c = tid; c < C; c += CN_T) {
+    const float sc = expf(tb[c] - tm) / ts;
+    const float nw = (c == yy ? r : 0.f) + (1.f - r) * sc;
+    s[row * C + c] = sc;
+    newlab[row * C + c] = nw;
+    le -= nw * lp[c];
+  }
+  le = cn_block_sum(le, red);
+  if (tid < WN_H) hid[row * WN_H + tid] = hd[tid];
+  if (tid == 0) { rho[row] = r; ell[row] = le; }
+}
+// Per-sample derivatives of the loss with respect to the net's two pre-activations, times coef_i (or `scale`
+// when coef is null).  mode 0: the classifier's soft-label loss (dt = s (g - <s, g>), g = -(1 - rho) log p;
+// dm = (-log p_y + <s, log p>) rho (1 - rho); dpre = relu' a2 dm).  mode 1: the correction problem's own term,
+// the mean cross-entropy of the soft label against y (dt = s - onehot; nothing through the interpolation net).
+// G32 [B, C + 101] = [dt, dpre, dm]; G16 [B, ldg] = [dt, dpre] in the operand type (pad columns zero).
+__global__ void __launch_bounds__(CN_T) k_cn_sample_grad(int mode, const float* alpha, const float* logp, const float* s,
+                                                         const float* hid, const float* rho, const int32_t* y,
+                                                         const float* coef, float scale, int64_t H, int64_t C, float* G32,
+                                                         op16* G16, int64_t ldg) {
+  pdl_enter();
+  __shared__ float red[CN_T / 32];
+  const int64_t row = blockIdx.x;
+  const int tid = threadIdx.x;
+  const CnOff o = cn_offsets(H, C);
+  const float cf = coef ? coef[row] : scale;
+  const float r = rho[row];
+  int32_t yy = y[row];
+  yy = yy < 0 ? 0 : (yy >= C ? (int32_t)C - 1 : yy);
+  const int64_t W = C + WN_H + 1;
+  float sg = 0.f, sl = 0.f;
+  if (mode == 0) {
+    for (int64_t c = tid; c < C; c += CN_T) {
+      const float sc = s[row * C + c], l = logp[row * C + c];
+      sg += sc * (-(1.f - r) * l);
+      sl += sc * l;
+    }
+    sg = cn_block_sum(sg, red);
+    sl = cn_block_sum(sl, red);
+  }
+  const float dm = mode == 0 ? (-logp[row * C + yy] + sl) * r * (1.f - r) : 0.f;
+  for (int64_t c = tid; c < C; c += CN_T) {
+    const float sc = s[row * C + c];
+    const float dt = mode == 0 ? sc * (-(1.f - r) * logp[row * C + c] - sg) : sc - (c == yy ? 1.f : 0.f);
+    G32[row * W + c] = cf * dt;
+    G16[row * ldg + c] = to_op16(cf * dt);
+  }
+  for (int64_t k = tid; k < ldg - C; k += CN_T) {
+    float v = 0.f;
+    if (k < WN_H && mode == 0) v = cf * ((hid[row * WN_H + k] > 0.f ? alpha[o.a2 + k] : 0.f) * dm);
+    if (k < WN_H) G32[row * W + C + k] = v;
+    G16[row * ldg + C + k] = to_op16(v);
+  }
+  if (tid == 0) G32[row * W + C + WN_H] = cf * dm;
+}
+// out[e] = sum_i (derivative pieces of sample i) for every parameter e of the net, samples in index order, fp64.
+__global__ void k_cn_param_grad(const float* G32, const float* hl32, const float* hid, int64_t B, int64_t H, int64_t C, float* out) {
+  pdl_enter();
+  const CnOff o = cn_offsets(H, C);
+  const int64_t W = C + WN_H + 1;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < o.total; e += (int64_t)gridDim.x * blockDim.x) {
+    int64_t gcol; const float* other; int64_t ostride, ocol;      // out[e] = sum_i G32[i, gcol] * other[i * ostride + ocol]
+    if (e < o.a0) { gcol = e / H; other = hl32; ostride = H; ocol = e - gcol * H; }
+    else if (e < o.A1) { gcol = e - o.a0; other = nullptr; ostride = 0; ocol = 0; }
+    else if (e < o.b1) { const int64_t k = (e - o.A1) / H; gcol = C + k; other = hl32; ostride = H; ocol = (e - o.A1) - k * H; }
+    else if (e < o.a2) { gcol = C + (e - o.b1); other = nullptr; ostride = 0; ocol = 0; }
+    else if (e < o.b2) { gcol = C + WN_H; other = hid; ostride = WN_H; ocol = e - o.a2; }
+    else { gcol = C + WN_H; other = nullptr; ostride = 0; ocol = 0; }
+    double acc = 0.0;
+    for (int64_t i = 0; i < B; ++i) acc += (double)G32[i * W + gcol] * (other ? (double)other[i * ostride + ocol] : 1.0);
+    out[e] = (float)acc;
+  }
+}
+// M16 [(C + 100), ldm] = [A; A1] in the operand type: the second operand of the term the label's dependence on h
+// adds to the last hidden layer's delta (a matrix product like the others)
+__global__ void k_cn_cast_maps(const float* alpha, int64_t H, int64_t C, op16* M16, int64_t ldm) {
+  pdl_enter();
+  const CnOff o = cn_offsets(H, C);
+  const int64_t total = (C + WN_H) * ldm;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / ldm, j = i - r * ldm;
+    float v = 0.f;
+    if (j < H) v = r < C ? alpha[o.A + r * H + j] : alpha[o.A1 + (r - C) * H + j];
+    M16[i] = to_op16(v);
+  }
+}
+// delta = S * coef_i * (p - new label)
+__global__ void k_delta_top_soft(const float* p, const float* newlab, const float* coef, float scale, op16* delta, int64_t B,
+                                 int64_t C, int64_t ld, const float* lscale) {
+  pdl_enter();
+  const float S = lscale ? *lscale : 1.f;
+  const int64_t total = B * ld;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / ld, c = i - r * ld;
+    float v = 0.f;
+    if (c < C) v = S * ((coef ? coef[r] : scale) * (p[r * C + c] - newlab[r * C + c]));
+    delta[i] = to_op16(v);
   }
 }
 
@@ -414,6 +605,19 @@ struct HvpCache {
   // of iteration k leave the rounded next term here, so that iteration k+1 starts without a cast pass
   op16* dir16[MAXL];     // null: every R-forward pass rounds its direction into scratch of its own
   const float* dir16_of; // the fp32 vector that dir16 currently mirrors, or null
+};
+
+// Label-correction state of one pass (see the kernels above) and what a reverse sweep needs from it.
+struct CorrPass {
+  const betty_level* G;     // the correction net's level
+  int64_t H, C;
+  float *hl32, *logp, *s, *hid, *rho, *newlab;
+};
+struct CorrBack {
+  const float* newlab;      // soft labels for the top delta (null: the given labels)
+  const op16* G16; int64_t ldg;    // coef_i [dt_i, dpre_i], operand type
+  const op16* M16; int64_t ldm;    // [A; A1], operand type
+  int64_t Kc;               // C + 100
 };
 
 static betty_status net_layout(const betty_level* M, Net& n) {
@@ -538,14 +742,18 @@ struct GradSink {
 
 // Reverse sweep from delta_top = coef_i (p - onehot).  Always leaves delta[l] (and dh[l] for smooth
 // activations) in `ps` for an R-operator pass.
-static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, const GradSink& sink, bool keep_dh = false) {
+static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, const GradSink& sink, bool keep_dh = false,
+                             const CorrBack* cb = nullptr) {
   const int64_t B = ps.B;
   const int64_t C = n.w[n.L];
   {
     const int64_t ld = ld8(C);
     BETTY_ALLOC(dt, op16, c, (size_t)(B * ld));
     ps.delta[n.L - 1] = dt;
-    launch_pdl(k_delta_top, dim3(grid_for(B * ld)), dim3(256), 0, c.stream, ps.p, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld, sink.lscale);
+    if (cb && cb->newlab)
+      launch_pdl(k_delta_top_soft, dim3(grid_for(B * ld)), dim3(256), 0, c.stream, ps.p, cb->newlab, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld, sink.lscale);
+    else
+      launch_pdl(k_delta_top, dim3(grid_for(B * ld)), dim3(256), 0, c.stream, ps.p, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld, sink.lscale);
     BETTY_LAUNCH_CHECK();
   }
   for (int l = n.L - 1; l >= 0; --l) {
@@ -586,6 +794,8 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       ps.delta[l - 1] = dp;
       GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.npairs = 1; g.C = dh; g.ldc = K; g.beta = 0.f;
       g.p[0] = gemm_pair(ps.delta[l], ldd, false, n.W[l], n.ldw[l], false, (int)N);
+      // corrected labels move with the last hidden activation: one more product into the same accumulator
+      if (cb && cb->G16 && l == n.L - 1) g.p[g.npairs++] = gemm_pair(cb->G16, cb->ldg, false, cb->M16, cb->ldm, false, (int)cb->Kc);
       g.epi.mode = EPI_ACT_BWD; g.epi.act = n.act; g.epi.a = ps.a[l - 1]; g.epi.out16 = dp; g.epi.ld16 = ldp;
       BETTY_TRY(gemm(c, g));
     }
@@ -640,10 +850,14 @@ struct Parts {
   const betty_level* mlp;
   const betty_level* theta;   // weight net or null
   const betty_level* lam;     // log weight decay or null
+  const betty_level* corr;    // label-correction net or null
 };
 static Parts parts_of(const betty_level* L) {
   Parts p;
   p.mlp = find_participant(L, BETTY_PARAM_MLP);
+  p.corr = nullptr;
+  if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) p.corr = find_constraint(L, BETTY_PARAM_CORRECTNET);
+  if (L->loss == BETTY_LOSS_MLP_CE_CORRECT) p.corr = find_participant(L, BETTY_PARAM_CORRECTNET);
   if (L->loss == BETTY_LOSS_WEIGHTNET_DETECT) {
     p.theta = find_participant(L, BETTY_PARAM_WEIGHTNET);
     p.lam = nullptr;
@@ -671,6 +885,14 @@ betty_status mlpfam_validate(const betty_level* L) {
   if (L->n > 0 && (!L->X || !L->y)) return BETTY_ERR_INVALID_ARG;
   if (!aligned16(L->X) || !aligned16(P.mlp->params)) return BETTY_ERR_ALIGNMENT;
   if (L->d % 8 != 0) return BETTY_ERR_ALIGNMENT;     // op16 rows must start on 16-byte boundaries
+  if (L->loss == BETTY_LOSS_MLP_CE_CORRECT && !P.corr) return BETTY_ERR_INVALID_ARG;
+  if (P.corr) {
+    if (n.L < 2) return BETTY_ERR_SHAPE;                       // the net reads a hidden activation
+    const int64_t H = n.w[n.L - 1], C = n.w[n.L];
+    if (C > CN_MAX_C || H > CN_MAX_H) return BETTY_ERR_UNSUPPORTED;
+    if (!P.corr->params || P.corr->n_params != cn_offsets(H, C).total) return BETTY_ERR_SHAPE;
+    if (P.mlp->loss_scale) return BETTY_ERR_UNSUPPORTED;        // loss scaling is not offered together with label correction
+  }
   if (P.theta && (P.theta->n_params != WN_P || !P.theta->params)) return BETTY_ERR_SHAPE;
   if (P.lam && (P.lam->n_params != n.L || !P.lam->params)) return BETTY_ERR_SHAPE;
   if (L->loss == BETTY_LOSS_WEIGHTNET_DETECT) {
@@ -686,7 +908,12 @@ size_t mlpfam_workspace(const betty_level* L) {
   size_t S = 0;
   for (int l = 0; l <= P.mlp->n_layers; ++l) S += (size_t)ld8(P.mlp->widths[l]) + 8;
   const size_t B = (size_t)(L->n > 0 ? L->n : 1);
-  return 24 * (size_t)P.mlp->n_params + 96 * B * S + 64 * 256 * (size_t)(P.mlp->n_layers + 4) + (1 << 20);
+  size_t extra = 0;
+  if (P.corr && P.mlp->n_layers >= 2) {
+    const size_t H = (size_t)P.mlp->widths[P.mlp->n_layers - 1], C = (size_t)P.mlp->widths[P.mlp->n_layers];
+    extra = 16 * (size_t)P.corr->n_params + 64 * B * (H + 2 * C + 256) + (1 << 16);
+  }
+  return 24 * (size_t)P.mlp->n_params + 96 * B * S + 64 * 256 * (size_t)(P.mlp->n_layers + 4) + (1 << 20) + extra;
 }
 
 // per-sample scalar through the weight net
@@ -726,10 +953,64 @@ static betty_status reweight_coef(Ctx& c, const Parts& P, const Pass& ps, const 
   return BETTY_OK;
 }
 
+// ---- label-correction net: host side
+// Runs the net on the pass's last hidden activation (or on h32, a perturbed copy) and logits (or z), and replaces
+// the pass's per-sample losses by the soft-label losses.
+static betty_status corr_forward(Ctx& c, const Net& n, Pass& ps, const betty_level* G, CorrPass& cp, const float* h32 = nullptr,
+                                 const float* z = nullptr) {
+  const int64_t B = ps.B, H = n.w[n.L - 1], C = n.w[n.L];
+  cp.G = G; cp.H = H; cp.C = C;
+  const size_t nb = (size_t)(B > 0 ? B : 1);
+  cp.hl32 = h32 ? const_cast<float*>(h32) : c.arena.alloc<float>(nb * H);
+  cp.logp = c.arena.alloc<float>(nb * C);
+  cp.s = c.arena.alloc<float>(nb * C);
+  cp.hid = c.arena.alloc<float>(nb * WN_H);
+  cp.rho = c.arena.alloc<float>(nb);
+  cp.newlab = c.arena.alloc<float>(nb * C);
+  if (!cp.hl32 || !cp.logp || !cp.s || !cp.hid || !cp.rho || !cp.newlab) return BETTY_ERR_WORKSPACE;
+  if (B <= 0) return BETTY_OK;
+  const size_t smem = (size_t)(H + 2 * C + WN_H) * sizeof(float);
+  launch_pdl(k_cn_forward, dim3((unsigned)B), dim3(CN_T), smem, c.stream, (const float*)G->params, ps.h[n.L - 1], ps.ldh[n.L - 1], h32,
+             z ? z : (const float*)ps.a[n.L - 1], ps.y, H, C, cp.hl32, cp.logp, cp.s, cp.hid, cp.rho, cp.newlab, ps.ell);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+// coef_i times the per-sample derivatives (mode: see k_cn_sample_grad); G32 for the parameter gradient, G16 for the
+// reverse sweep's extra product
+static betty_status corr_sample_grad(Ctx& c, int mode, const CorrPass& cp, const Pass& ps, const float* coef, float** G32,
+                                     op16** G16, int64_t* ldg) {
+  const int64_t B = ps.B, W = cp.C + WN_H + 1;
+  *ldg = ld8(cp.C + WN_H);
+  const size_t nb = (size_t)(B > 0 ? B : 1);
+  *G32 = c.arena.alloc<float>(nb * W);
+  *G16 = c.arena.alloc<op16>(nb * (size_t)*ldg);
+  if (!*G32 || !*G16) return BETTY_ERR_WORKSPACE;
+  if (B <= 0) return BETTY_OK;
+  launch_pdl(k_cn_sample_grad, dim3((unsigned)B), dim3(CN_T), 0, c.stream, mode, (const float*)cp.G->params, (const float*)cp.logp,
+             (const float*)cp.s, (const float*)cp.hid, (const float*)cp.rho, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, cp.H, cp.C, *G32,
+             *G16, *ldg);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+static betty_status corr_param_grad(Ctx& c, const CorrPass& cp, const Pass& ps, const float* G32, float* out) {
+  const int64_t total = cn_offsets(cp.H, cp.C).total;
+  launch_pdl(k_cn_param_grad, dim3(grid_for(total)), dim3(256), 0, c.stream, G32, (const float*)cp.hl32, (const float*)cp.hid, ps.B, cp.H, cp.C, out);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+static betty_status corr_maps(Ctx& c, const betty_level* G, int64_t H, int64_t C, op16** M16, int64_t* ldm) {
+  *ldm = ld8(H);
+  *M16 = c.arena.alloc<op16>((size_t)((C + WN_H) * *ldm));
+  if (!*M16) return BETTY_ERR_WORKSPACE;
+  launch_pdl(k_cn_cast_maps, dim3(grid_for((C + WN_H) * *ldm)), dim3(256), 0, c.stream, (const float*)G->params, H, C, *M16, *ldm);
+  BETTY_LAUNCH_CHECK();
+  return BETTY_OK;
+}
+
 betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, float* out) {
   const Parts P = parts_of(L);
   const size_t mark = c.arena.mark();
-  const bool touches = (wrt == P.mlp) || (P.theta && wrt == P.theta) || (P.lam && wrt == P.lam);
+  const bool touches = (wrt == P.mlp) || (P.theta && wrt == P.theta) || (P.lam && wrt == P.lam) || (P.corr && wrt == P.corr);
   if (!touches) return vec_zero(c, out, wrt->n_params);
   Net n; Pass ps;
   BETTY_TRY(net_setup(c, P.mlp, n));
@@ -742,15 +1023,47 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
   }
   BETTY_TRY(forward(c, n, L, ps));
   BETTY_ALLOC(s1, float, c, (size_t)(ps.B > 0 ? ps.B : 1));
+  CorrPass cp;
+  if (P.corr) BETTY_TRY(corr_forward(c, n, ps, P.corr, cp));      // ps.ell now holds the soft-label losses
   if (L->loss == BETTY_LOSS_MLP_CE) {
     BETTY_TRY(backward(c, n, ps, nullptr, grad_into(out, nullptr)));
+  } else if (L->loss == BETTY_LOSS_MLP_CE_CORRECT) {
+    // mean CE of the classifier + mean CE of the correction net's own soft labels, both against the given labels
+    float* G32; op16* G16; int64_t ldg;
+    BETTY_TRY(corr_sample_grad(c, 1, cp, ps, nullptr, &G32, &G16, &ldg));
+    if (wrt == P.corr) {
+      BETTY_TRY(corr_param_grad(c, cp, ps, G32, out));
+    } else {
+      CorrBack cb = {};
+      cb.G16 = G16; cb.ldg = ldg; cb.Kc = cp.C + WN_H;
+      op16* M16;
+      BETTY_TRY(corr_maps(c, P.corr, cp.H, cp.C, &M16, &cb.ldm));
+      cb.M16 = M16;
+      BETTY_TRY(backward(c, n, ps, nullptr, grad_into(out, nullptr), false, &cb));
+    }
   } else if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
-    if (wrt == P.mlp) {
+    if (wrt == P.mlp || (P.corr && wrt == P.corr)) {
       const float* coef;
       BETTY_TRY(reweight_coef(c, P, ps, &coef));
-      GradSink sink = grad_into(out, P.lam ? P.lam->params : nullptr);
-      sink.lscale = c.loss_scale;       // set by a loss-scaled lower step only
-      BETTY_TRY(backward(c, n, ps, coef, sink));
+      CorrBack cb = {};
+      float* G32 = nullptr;
+      if (P.corr) {
+        op16* G16;
+        BETTY_TRY(corr_sample_grad(c, 0, cp, ps, coef, &G32, &G16, &cb.ldg));
+        cb.newlab = cp.newlab; cb.G16 = G16; cb.Kc = cp.C + WN_H;
+      }
+      if (P.corr && wrt == P.corr) {
+        BETTY_TRY(corr_param_grad(c, cp, ps, G32, out));
+      } else {
+        if (P.corr) {
+          op16* M16;
+          BETTY_TRY(corr_maps(c, P.corr, cp.H, cp.C, &M16, &cb.ldm));
+          cb.M16 = M16;
+        }
+        GradSink sink = grad_into(out, P.lam ? P.lam->params : nullptr);
+        sink.lscale = c.loss_scale;       // set by a loss-scaled lower step only
+        BETTY_TRY(backward(c, n, ps, coef, sink, false, P.corr ? &cb : nullptr));
+      }
     } else {
       BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, ps, nullptr, nullptr, s1, nullptr));
       BETTY_TRY(wn_backward(c, P.theta, nullptr, ps, s1, nullptr, 0.f, nullptr, out));
@@ -772,6 +1085,7 @@ betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache)
   static thread_local HvpCache store;   // host-side bookkeeping only; device state lives in the workspace
   HvpCache& h = store;
   const Parts P = parts_of(L);
+  if (P.corr) return BETTY_ERR_UNSUPPORTED;     // second derivatives are not offered with label correction (the paper pairs it with AID-FD)
   h.theta = P.theta;
   h.lam = P.lam ? P.lam->params : nullptr;
   h.coef = nullptr;
@@ -946,6 +1260,12 @@ betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int fi
   // op16 copy of the updated matrices for the next step: one cast at the start, none afterwards.
   Net n;
   BETTY_TRY(net_setup(c, P.mlp, n));
+  CorrBack cb = {};
+  if (P.corr) {       // the correction net does not move during the classifier's steps: its maps are cast once
+    op16* M16;
+    BETTY_TRY(corr_maps(c, P.corr, n.w[n.L - 1], n.w[n.L], &M16, &cb.ldm));
+    cb.M16 = M16; cb.Kc = n.w[n.L] + WN_H;
+  }
   op16* alt[MAXL];
   for (int l = 0; l < n.L; ++l) {
     const size_t cnt = (size_t)(n.w[l + 1] * n.ldw[l]);
@@ -957,12 +1277,19 @@ betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int fi
     const size_t m2 = c.arena.mark();
     Pass ps;
     BETTY_TRY(forward(c, n, L, ps));
+    CorrPass cp;
+    if (P.corr) BETTY_TRY(corr_forward(c, n, ps, P.corr, cp));
     const float* coef;
     BETTY_TRY(reweight_coef(c, P, ps, &coef));
+    if (P.corr) {
+      float* G32; op16* G16;
+      BETTY_TRY(corr_sample_grad(c, 0, cp, ps, coef, &G32, &G16, &cb.ldg));
+      cb.newlab = cp.newlab; cb.G16 = G16;
+    }
     GradSink sink = {};
     sink.lam = P.lam ? P.lam->params : nullptr;
     sink.sgd = true; sink.lr = lr_at(L, first_step + s); sink.master = L->params; sink.Wnext = alt;
-    BETTY_TRY(backward(c, n, ps, coef, sink));
+    BETTY_TRY(backward(c, n, ps, coef, sink, false, P.corr ? &cb : nullptr));
     for (int l = 0; l < n.L; ++l) { op16* t = n.W[l]; n.W[l] = alt[l]; alt[l] = t; }
     c.arena.release(m2);
   }
@@ -989,16 +1316,24 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
     c.arena.release(mark);
     return BETTY_OK;
   }
-  if (!P.theta || wrt != P.theta) return BETTY_ERR_INVALID_ARG;
+  const bool wrt_theta = P.theta && wrt == P.theta, wrt_corr = P.corr && wrt == P.corr;
+  if (!wrt_theta && !wrt_corr) return BETTY_ERR_INVALID_ARG;
   BETTY_TRY(forward(c, n, L, ps));
   const int64_t B = ps.B, C = n.w[n.L];
+  // the label-correction net is evaluated at the perturbed last hidden activation, in fp32
+  float* hlast_p = nullptr;
+  if (P.corr) {
+    hlast_p = c.arena.alloc<float>((size_t)((B > 0 ? B : 1) * n.w[n.L - 1]));
+    if (!hlast_p) return BETTY_ERR_WORKSPACE;
+  }
+  const int64_t n_out = wrt->n_params, gstride = (n_out + 63) & ~int64_t(63);
   op16* E[MAXL];
   for (int l = 0; l < n.L; ++l) {
     E[l] = c.arena.alloc<op16>((size_t)(n.w[l + 1] * n.ldw[l]));
     if (!E[l]) return BETTY_ERR_WORKSPACE;
     BETTY_TRY(cast_matrix(c, v + n.woff[l], E[l], n.w[l + 1], n.w[l], n.ldw[l], vnorm2, eps0));
   }
-  BETTY_ALLOC(G, float, c, 2 * 512);
+  BETTY_ALLOC(G, float, c, (size_t)(2 * gstride));
   BETTY_ALLOC(zpm, float, c, (size_t)(B * C));
   BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
   Pass pp = ps;   // perturbed pass: reuses y/B, gets its own p/ell
@@ -1026,22 +1361,32 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
           cudaMemsetAsync(dn, 0, cnt * sizeof(op16), c.stream);
         }
         launch_pdl(k_fd_act, dim3(grid_for(B * N)), dim3(256), 0, c.stream, ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, hn, dn, nullptr, B, N,
-                                                       ps.ldh[l + 1], n.act);
+                                                       ps.ldh[l + 1], n.act, (P.corr && l == n.L - 2) ? hlast_p : (float*)nullptr);
         BETTY_LAUNCH_CHECK();
         hp = hn; dh = dn;
       } else {
         launch_pdl(k_fd_act, dim3(grid_for(B * N)), dim3(256), 0, c.stream, ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, nullptr, nullptr, zpm,
-                                                       B, N, 0, n.act);
+                                                       B, N, 0, n.act, (float*)nullptr);
         BETTY_LAUNCH_CHECK();
       }
     }
     launch_pdl(k_softmax_ce, dim3(grid_for(B * 32)), dim3(256), 0, c.stream, zpm, ps.y, pp.p, pp.ell, B, C);
     BETTY_LAUNCH_CHECK();
-    BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, pp, nullptr, nullptr, s1, nullptr));
-    BETTY_TRY(wn_backward(c, P.theta, nullptr, pp, s1, nullptr, 0.f, nullptr, G + 512 * sgn));
+    CorrPass cpp;
+    if (P.corr) BETTY_TRY(corr_forward(c, n, pp, P.corr, cpp, hlast_p, zpm));     // pp.ell: soft-label losses at x +- eps v
+    if (wrt_theta) {
+      BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, pp, nullptr, nullptr, s1, nullptr));
+      BETTY_TRY(wn_backward(c, P.theta, nullptr, pp, s1, nullptr, 0.f, nullptr, G + gstride * sgn));
+    } else {
+      const float* coefp;
+      BETTY_TRY(reweight_coef(c, P, pp, &coefp));
+      float* G32; op16* G16; int64_t ldg;
+      BETTY_TRY(corr_sample_grad(c, 0, cpp, pp, coefp, &G32, &G16, &ldg));
+      BETTY_TRY(corr_param_grad(c, cpp, pp, G32, G + gstride * sgn));
+    }
     c.arena.release(m2);
   }
-  launch_pdl(k_fd_combine, dim3(grid_for(WN_P)), dim3(256), 0, c.stream, out, G, G + 512, vnorm2, eps0, alpha, accumulate ? 1 : 0, WN_P);
+  launch_pdl(k_fd_combine, dim3(grid_for(n_out)), dim3(256), 0, c.stream, out, G, G + gstride, vnorm2, eps0, alpha, accumulate ? 1 : 0, n_out);
   BETTY_LAUNCH_CHECK();
   c.arena.release(mark);
   return BETTY_OK;

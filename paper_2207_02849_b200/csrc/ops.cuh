@@ -20,7 +20,8 @@ static inline bool is_vector_family(int loss) {
          loss == BETTY_LOSS_QUADRATIC;
 }
 static inline bool is_mlp_family(int loss) {
-  return loss == BETTY_LOSS_MLP_CE_REWEIGHT || loss == BETTY_LOSS_MLP_CE || loss == BETTY_LOSS_WEIGHTNET_DETECT;
+  return loss == BETTY_LOSS_MLP_CE_REWEIGHT || loss == BETTY_LOSS_MLP_CE || loss == BETTY_LOSS_WEIGHTNET_DETECT ||
+         loss == BETTY_LOSS_MLP_CE_CORRECT;
 }
 
 // logreg.cu

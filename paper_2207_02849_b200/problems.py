@@ -62,3 +62,17 @@ def three_levels(inp):
     P2.set_constraints([P1])
     P3.set_constraints([P2, P1])
     return P1, P2, P3
+
+
+def correct_reweight_levels(inp):
+    """The extended bilevel program of the noisy-label experiment: classifier below (labels corrected and
+    reweighted), the reweighting net and the label-correction net above, both on the clean batch."""
+    Xv, yv = dev(inp.val.X, torch.bfloat16), dev(inp.val.y)
+    theta = bt.Level(bt.LOSS_MLP_CE, bt.PARAM_WEIGHTNET, dev(inp.theta), X=Xv, y=yv)
+    alpha = bt.Level(bt.LOSS_MLP_CE_CORRECT, bt.PARAM_CORRECTNET, dev(inp.alpha), X=Xv, y=yv)
+    w = bt.Level(bt.LOSS_MLP_CE_REWEIGHT, bt.PARAM_MLP, dev(inp.w), X=dev(inp.train.X, torch.bfloat16),
+                 y=dev(inp.train.y), widths=inp.widths, activation=_act(inp.activation), lr=inp.lr)
+    w.set_constraints([theta, alpha])
+    theta.set_constraints([w])
+    alpha.set_constraints([w])
+    return w, theta, alpha

@@ -3,7 +3,7 @@ import numpy as np
 import torch
 
 from paper_2207_02849_b200.problems import (  # noqa: F401
-    dev, logreg_levels, quadratic_levels, reweight_levels, three_levels,
+    correct_reweight_levels, dev, logreg_levels, quadratic_levels, reweight_levels, three_levels,
 )
 
 
