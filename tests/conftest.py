@@ -32,8 +32,9 @@ _PARITY = {}
 
 @pytest.fixture
 def parity_record():
-    """record(name, value): keeps a measured parity error; the session writes all of them to
-    gpurun_out/parity_errors.json (the figures quoted in the documentation come from that file)."""
+    """record(name, value): keeps a measured parity error.  When the environment variable BETTY_PARITY_LOG names
+    a file, the session merges all recorded errors into it as JSON (the figures quoted in the documentation
+    come from such a file)."""
     def record(name, value):
         _PARITY[name] = float(value)
         return float(value)
@@ -41,12 +42,11 @@ def parity_record():
 
 
 def pytest_sessionfinish(session, exitstatus):
-    if not _PARITY:
+    path = os.environ.get("BETTY_PARITY_LOG")
+    if not _PARITY or not path:
         return
-    out = os.path.join(ROOT, "gpurun_out")
     try:
-        os.makedirs(out, exist_ok=True)
-        path = os.path.join(out, "parity_errors.json")
+        os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
         old = {}
         if os.path.exists(path):
             with open(path) as f:
