@@ -44,15 +44,18 @@ class DeviceAllReduce:
     """The callable a data-parallel `Level` hands to the library: sums `count` floats at a device address
     over the ranks, ordered on the stream the library is enqueuing on."""
 
-    def __init__(self, group=None):
+    def __init__(self, group=None, single_rank_too: bool = False):
+        """single_rank_too: issue the collective even in a job of one rank (it then changes nothing; useful to
+        exercise the exchange itself on one GPU)."""
         self.group = group
+        self.single_rank_too = single_rank_too
         self.calls = 0
         self.floats = 0
 
     def __call__(self, ptr: int, count: int, stream: int) -> None:
         self.calls += 1
         self.floats += count
-        if not (dist.is_initialized() and dist.get_world_size(self.group) > 1):
+        if not dist.is_initialized() or (dist.get_world_size(self.group) <= 1 and not self.single_rank_too):
             return
         t = torch.as_tensor(_RawDeviceBuffer(ptr, count), device=torch.device("cuda", torch.cuda.current_device()))
         with torch.cuda.stream(torch.cuda.ExternalStream(stream) if stream else torch.cuda.default_stream()):

@@ -47,6 +47,46 @@ def test_single_rank_with_the_hook_attached_matches_the_oracle():
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
 
+def test_the_nccl_exchange_runs_on_the_library_buffers():
+    """A one-rank NCCL job on this GPU: the collective is issued on the raw device buffers the library hands to
+    the callback, on the stream the library is enqueuing on (a sum over one rank changes nothing, so the results
+    must still equal the oracle's)."""
+    import os
+    import socket
+    import torch.distributed as dist
+    import paper_2207_02849_b200 as bt
+    from paper_2207_02849_b200 import data_parallel as dp
+    from tests import cuda_build as cb
+    if dist.is_initialized():
+        pytest.skip("a process group already exists in this process")
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        inp = si.logreg_bilevel(7, 1500, 4096, 300)
+        w, lam = cb.logreg_levels(inp)
+        ow, olam = ob.logreg_levels(inp)
+        ar = dp.DeviceAllReduce(single_rank_too=True)
+        dp.shard_level(w, 1500, 0, 1, ar)
+        dp.shard_level(lam, 300, 0, 1, ar)
+        ws = bt.Workspace([w, lam])
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):                      # not the default stream: the exchange must follow the library's
+            bt.betty_lower_step(w, 3, ws)
+            out = torch.empty(4096, device="cuda")
+            bt.betty_hypergrad_cg(w, lam, lam, 5, 0.0, out, ws)
+            side.synchronize()
+        oracle.lower_step(ow, 3)
+        assert cb.rel_l2(w.params, ow.params) < 1e-4
+        assert cb.rel_l2(out, oracle.hypergrad_cg(ow, olam, olam, 5, 0.0)) < 1e-4
+        assert ar.calls == 3 + 2 + 5 + 1
+        assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+    finally:
+        dist.destroy_process_group()
+
+
 class _TwoThreadAllReduce:
     """Sum over two host threads that share one GPU (see the module docstring)."""
 
