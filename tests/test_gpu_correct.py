@@ -74,6 +74,27 @@ def test_corrected_costs_match_oracle(act, widths, B, parity_record):
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
 
+def test_corrected_costs_at_configuration_3_size(parity_record):
+    """The data-reweighting configuration's classifier (3072 -> 1024 -> 10, batch 512, 40% label noise) with the
+    correction net attached (112,851 parameters): both upper problems' finite-difference hypergradients."""
+    import paper_2207_02849_b200 as bt
+    from tests import cuda_build as cb
+    inp = si.correct_reweight(si.BASE_SEED + 3, (3072, 1024, 10), 512, 0.4, activation="relu")
+    w, th, al = cb.correct_reweight_levels(inp)
+    ow, oth, oal = ob.correct_reweight_levels(inp)
+    ws = bt.Workspace([w, th, al])
+    ga, gt = _vec(inp.alpha.size), _vec(si.WEIGHTNET_PARAMS)
+    bt.betty_hypergrad_fd(w, al, al, 0.01, 1.0, ga, ws)
+    assert parity_record("correct/config3-size/fd_alpha", cb.rel_l2(ga, oracle.hypergrad_fd(ow, oal, oal, 0.01, 1.0))) < TOL
+    bt.betty_hypergrad_fd(w, th, th, 0.01, 1.0, gt, ws)
+    assert parity_record("correct/config3-size/fd_theta", cb.rel_l2(gt, oracle.hypergrad_fd(ow, oth, oth, 0.01, 1.0))) < TOL
+    bt.betty_lower_step(w, 1, ws)
+    oracle.lower_step(ow, 1)
+    w0 = inp.w.astype(np.float64)
+    assert parity_record("correct/config3-size/lower_update", cb.rel_l2(w.params.double().cpu().numpy() - w0, ow.params - w0)) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
 def test_extended_bilevel_program_runs_through_the_schedule():
     """Sec. 5.1's program as its App. A listing wires it: two upper problems (reweight, correct), each with an
     upper-to-lower edge into the classifier and a lower-to-upper edge out of it, finite-difference Jacobians,

@@ -62,6 +62,25 @@ def test_fp16_primitives_and_hypergradients_match_oracle(act, widths, B, parity_
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
 
 
+def test_config3_shape_in_half_precision(parity_record):
+    """Configuration 3's problem (3072 -> 1024 -> 10, batch 512) with binary16 operands: one lower step, then the
+    finite-difference and Neumann hypergradients."""
+    inp = si.config3()
+    for b in (inp.train, inp.val):
+        b.X = torch.from_numpy(np.ascontiguousarray(b.X, dtype=np.float32)).half().float().numpy()
+    bt, cb, w, th, ow, oth = _levels(inp)
+    ws = bt.Workspace([w, th])
+    bt.betty_lower_step(w, inp.lower_steps, ws)
+    oracle.lower_step(ow, inp.lower_steps)
+    assert parity_record("fp16/config3/lower_update", _update_err(cb, w, ow, inp.w)) < TOL
+    out = torch.empty(si.WEIGHTNET_PARAMS, device="cuda")
+    bt.betty_hypergrad_fd(w, th, th, inp.eps0, inp.fd_alpha, out, ws)
+    assert parity_record("fp16/config3/fd", cb.rel_l2(out, oracle.hypergrad_fd(ow, oth, oth, inp.eps0, inp.fd_alpha))) < TOL
+    bt.betty_hypergrad_neumann(w, th, th, inp.K, inp.alpha, out, ws)
+    assert parity_record("fp16/config3/neumann", cb.rel_l2(out, oracle.hypergrad_neumann(ow, oth, oth, inp.K, inp.alpha))) < TOL
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
 def test_dynamic_loss_scaling_skips_overflowing_steps_like_the_oracle():
     inp = _inputs(103, (64, 96, 10), 128, "relu")
     bt, cb, w, th, ow, oth = _levels(inp)
