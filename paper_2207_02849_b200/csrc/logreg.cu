@@ -264,7 +264,14 @@ __global__ void k_logreg_finalize(const float* partials, int nparts, int64_t d, 
   if (j < d) {
     const int per = (nparts + 7) / 8;
     const int c0 = sl * per, c1 = min(nparts, c0 + per);
-    for (int c = c0; c < c1; ++c) acc += partials[(size_t)c * d + j];
+    // same order of additions as a plain loop; eight loads are in flight at a time (the kernel is latency-bound)
+    for (int c = c0; c < c1; c += 8) {
+      float v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = c + k < c1 ? __ldcg(partials + (size_t)(c + k) * d + j) : 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc += v[k];
+    }
   }
   sh[sl][cx] = acc;
   __syncthreads();
@@ -305,8 +312,17 @@ __global__ void k_logreg_finalize(const float* partials, int nparts, int64_t d, 
   if (threadIdx.x == 0) { *tl.counter = 0u; s_active = st->active; s_rho = st->rho; }
   __syncthreads();
   if (!s_active) return;                         // the solve has stopped: h was stored, nothing else moves
+  // gamma: the per-block terms, a few per thread in index order, then a fixed tree (warp shuffles, warps in order):
+  // the order depends on the grid alone, and every thread ends with the same value
   double gsum = 0.0;
-  for (unsigned i = 0; i < gridDim.x; ++i) gsum += ((volatile double*)tl.partials)[i];   // same order in every thread
+  for (unsigned i = threadIdx.x; i < gridDim.x; i += blockDim.x) gsum += __ldcg(tl.partials + i);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) gsum += __shfl_xor_sync(0xffffffffu, gsum, o);
+  if (cx == 0) shd[sl] = gsum;
+  __syncthreads();
+  gsum = 0.0;
+  for (int i = 0; i < 8; ++i) gsum += shd[i];
+  __syncthreads();
   const float gamma = (float)gsum;
   if (!isfinite(gsum) || !(gsum > 0.0)) {
     if (threadIdx.x == 0) {
@@ -320,12 +336,27 @@ __global__ void k_logreg_finalize(const float* partials, int nparts, int64_t d, 
   const float a = rho / gamma;
   const float* h = out;
   double rr = 0.0;
-  for (int64_t i = threadIdx.x; i < d; i += blockDim.x) {
-    const float pi = tl.p[i];
-    tl.q[i] += a * pi;
-    const float ri = tl.r[i] - a * __ldcg(h + i);
-    tl.r[i] = ri;
-    rr += (double)ri * (double)ri;
+  // one block walks the whole vector: eight elements per thread at a time, every load of a batch issued before its
+  // first use (the loop is bound by load latency, not by bytes)
+  constexpr int TB = 8;
+  for (int64_t base = 0; base < d; base += (int64_t)blockDim.x * TB) {
+    float pv[TB], qv[TB], rv[TB], hv[TB];
+#pragma unroll
+    for (int k = 0; k < TB; ++k) {
+      const int64_t i = base + threadIdx.x + (int64_t)k * blockDim.x;
+      const bool in = i < d;
+      pv[k] = in ? tl.p[i] : 0.f; qv[k] = in ? tl.q[i] : 0.f; rv[k] = in ? tl.r[i] : 0.f; hv[k] = in ? __ldcg(h + i) : 0.f;
+    }
+#pragma unroll
+    for (int k = 0; k < TB; ++k) {
+      const int64_t i = base + threadIdx.x + (int64_t)k * blockDim.x;
+      if (i < d) {
+        tl.q[i] = qv[k] + a * pv[k];
+        const float ri = rv[k] - a * hv[k];
+        tl.r[i] = ri;
+        rr += (double)ri * (double)ri;
+      }
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) rr += __shfl_xor_sync(0xffffffffu, rr, o);
@@ -335,7 +366,19 @@ __global__ void k_logreg_finalize(const float* partials, int nparts, int64_t d, 
   for (int i = 0; i < 8; ++i) rsum += shd[i];
   const float rho_new = (float)rsum;
   const float beta = rho_new / rho;
-  for (int64_t i = threadIdx.x; i < d; i += blockDim.x) tl.p[i] = tl.r[i] + beta * tl.p[i];
+  for (int64_t base = 0; base < d; base += (int64_t)blockDim.x * TB) {
+    float pv[TB], rv[TB];
+#pragma unroll
+    for (int k = 0; k < TB; ++k) {
+      const int64_t i = base + threadIdx.x + (int64_t)k * blockDim.x;
+      pv[k] = i < d ? tl.p[i] : 0.f; rv[k] = i < d ? tl.r[i] : 0.f;      // r: this thread's own stores of the loop above
+    }
+#pragma unroll
+    for (int k = 0; k < TB; ++k) {
+      const int64_t i = base + threadIdx.x + (int64_t)k * blockDim.x;
+      if (i < d) tl.p[i] = rv[k] + beta * pv[k];
+    }
+  }
   if (threadIdx.x == 0) {
     st->gamma = gamma;
     st->rho_new = rho_new;
