@@ -147,19 +147,39 @@ __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
         if (HVP) pt[r] += v.x * uv[k].x + v.y * uv[k].y + v.z * uv[k].z + v.w * uv[k].w;
       }
     }
-#pragma unroll
-    for (int r = 0; r < LR_R; ++r) {
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        if (NEEDZ) pz[r] += __shfl_xor_sync(0xffffffffu, pz[r], o);
-        if (HVP) pt[r] += __shfl_xor_sync(0xffffffffu, pt[r], o);
+    float* rb = red + buf * (LR_WARPS * 2 * LR_R);
+    static_assert(LR_R == 2, "the halving butterfly below is written for two rows per tile");
+    // Sums over the warp by a butterfly that halves what a lane keeps at every round where it still holds more than
+    // one value: 6 shuffles for the four sums of the full HVP form (20 with one full butterfly per sum), 5 for two.
+    if (NEEDZ && HVP) {
+      const bool up1 = (lane & 16) != 0, up2 = (lane & 8) != 0;
+      // round 1: lanes with bit 4 clear keep row 0's sums, the others row 1's
+      float k0 = up1 ? pz[1] : pz[0], k1 = up1 ? pt[1] : pt[0];
+      const float s0 = up1 ? pz[0] : pz[1], s1 = up1 ? pt[0] : pt[1];
+      k0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+      k1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+      // round 2: lanes with bit 3 clear keep the x.w sum, the others the x.u sum
+      float v = up2 ? k1 : k0;
+      v += __shfl_xor_sync(0xffffffffu, up2 ? k0 : k1, 8);
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      v += __shfl_xor_sync(0xffffffffu, v, 2);
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      if ((lane & 7) == 0) rb[warp * 2 * LR_R + 2 * (lane >> 4) + ((lane >> 3) & 1)] = v;
+    } else {
+      const bool up1 = (lane & 16) != 0;
+      const float a0 = NEEDZ ? pz[0] : pt[0], a1 = NEEDZ ? pz[1] : pt[1];
+      float v = up1 ? a1 : a0;
+      v += __shfl_xor_sync(0xffffffffu, up1 ? a0 : a1, 16);
+      v += __shfl_xor_sync(0xffffffffu, v, 8);
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      v += __shfl_xor_sync(0xffffffffu, v, 2);
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      if ((lane & 15) == 0) {
+        rb[warp * 2 * LR_R + 2 * (lane >> 4) + (NEEDZ ? 0 : 1)] = v;
+        rb[warp * 2 * LR_R + 2 * (lane >> 4) + (NEEDZ ? 1 : 0)] = 0.f;
       }
     }
-    float* rb = red + buf * (LR_WARPS * 2 * LR_R);
-    if (lane == 0) {
-#pragma unroll
-      for (int r = 0; r < LR_R; ++r) { rb[warp * 2 * LR_R + 2 * r] = pz[r]; rb[warp * 2 * LR_R + 2 * r + 1] = pt[r]; }
-    }
+
     // every thread has copied its part of stage s into registers; the same barrier makes the
     // verdict on an expired wait uniform across the CTA
     if (__syncthreads_or(!landed)) { timed_out = true; break; }
