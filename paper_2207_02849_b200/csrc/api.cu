@@ -73,6 +73,26 @@ int current_sm_count() {
   return n;
 }
 
+SideLane* side_lane(cudaStream_t main) {
+  static thread_local SideLane lanes[MAX_DEVICES];
+  static thread_local unsigned char state[MAX_DEVICES];   // 0: not tried, 1: made, 2: could not be made
+  const int dev = current_device();
+  if (dev < 0) return nullptr;
+  if (state[dev] == 1) return &lanes[dev];
+  if (state[dev] == 2) return nullptr;
+  // nothing is created while the caller's stream is being captured: that call runs in program order
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(main, &cap) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+  if (cap != cudaStreamCaptureStatusNone) return nullptr;
+  SideLane& ln = lanes[dev];
+  bool ok = cudaStreamCreateWithFlags(&ln.stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&ln.fork, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&ln.join, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) { (void)cudaGetLastError(); state[dev] = 2; return nullptr; }
+  state[dev] = 1;
+  return &ln;
+}
+
 // ------------------------------------------------------------------ small kernels
 // out (+)= scale * x
 __global__ void k_scale_into(float* out, const float* x, float scale, int accumulate, int64_t n) {

@@ -126,8 +126,9 @@ struct Ctx {
   int sm_count;
   SharedWeights shared;
   const float* loss_scale;   // device loss scale of the lower step in progress (betty_level.loss_scale), else null
+  bool on_side;              // launches currently go to the side stream (see SideWork)
   __host__ Ctx(void* ws, size_t ws_bytes, void* s)
-      : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(current_sm_count()), loss_scale(nullptr) {
+      : stream((cudaStream_t)s), arena(ws, ws_bytes), sm_count(current_sm_count()), loss_scale(nullptr), on_side(false) {
     shared.master = nullptr;
   }
 };
@@ -180,6 +181,55 @@ static inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.attrs = attr; cfg.numAttrs = 1;
   (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // errors surface in BETTY_LAUNCH_CHECK
 }
+
+// ---- side stream ----
+// A reverse sweep is a chain (the product that carries delta to the layer below) with work hanging off it
+// that nothing in the chain waits for: each layer's weight-gradient product, its regulariser term and its
+// bias column sums.  Launched on the caller's stream they lengthen the chain; launched on a second stream
+// they run beside it and fill the SMs a one-wave product leaves idle.  The second stream and two events
+// belong to the library (one set per host thread and device, made at the first call outside a stream
+// capture and kept for the life of the process); they hold no device memory.  Dependencies are stated with
+// event record / wait pairs, which a stream capture turns into graph edges, so that a captured call
+// replays with the same concurrency.
+struct SideLane { cudaStream_t stream; cudaEvent_t fork, join; };
+// the calling thread's lane on the current device; null when there is none and none can be made now
+// (no device, a failed creation, or `main` is being captured and the lane does not exist yet)
+SideLane* side_lane(cudaStream_t main);
+
+// Scope of one fork/join region.  begin() ... end() brackets launches that go to the side stream; they start
+// after everything launched on the caller's stream before begin().  join() (also run by the destructor, so that
+// an early error return leaves no work behind) makes the caller's stream wait for the side stream.  All memory
+// the side work touches must stay allocated until the join.  Without a lane everything stays on the caller's
+// stream, in program order.
+class SideWork {
+ public:
+  explicit SideWork(Ctx& c) : c_(c), lane_(c.on_side ? nullptr : side_lane(c.stream)), main_(c.stream), used_(false), ok_(true) {}
+  ~SideWork() { (void)join(); }
+  SideWork(const SideWork&) = delete;
+  SideWork& operator=(const SideWork&) = delete;
+  void begin() {
+    if (!lane_) return;
+    ok_ = ok_ && cudaEventRecord(lane_->fork, main_) == cudaSuccess &&
+          cudaStreamWaitEvent(lane_->stream, lane_->fork, 0) == cudaSuccess;
+    c_.stream = lane_->stream; c_.on_side = true; used_ = true;
+  }
+  void end() { c_.stream = main_; if (lane_) c_.on_side = false; }
+  betty_status join() {
+    end();
+    if (used_) {
+      ok_ = ok_ && cudaEventRecord(lane_->join, lane_->stream) == cudaSuccess &&
+            cudaStreamWaitEvent(main_, lane_->join, 0) == cudaSuccess;
+      used_ = false;
+    }
+    if (!ok_) { (void)cudaGetLastError(); return BETTY_ERR_CUDA; }
+    return BETTY_OK;
+  }
+ private:
+  Ctx& c_;
+  SideLane* lane_;
+  cudaStream_t main_;
+  bool used_, ok_;
+};
 
 // ---- vector kernels (vec.cu); all vectors fp32, scalars stay on the device ----
 betty_status vec_zero(Ctx& c, float* x, int64_t n);

@@ -756,9 +756,14 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       launch_pdl(k_delta_top, dim3(grid_for(B * ld)), dim3(256), 0, c.stream, ps.p, ps.y, coef, B > 0 ? 1.f / (float)B : 0.f, dt, B, C, ld, sink.lscale);
     BETTY_LAUNCH_CHECK();
   }
+  // The chain is delta_L -> delta_{L-1} -> ... ; each layer's parameter gradient hangs off it and goes to the
+  // side stream.  (A gradient step there writes the master matrix and the *other* op16 copy, never the copy
+  // the chain's product for the same layer reads.)
+  SideWork side(c);
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
     if (sink.gflat || sink.sgd) {
+      side.begin();
       GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.npairs = 1; g.ldc = K; g.beta = 0.f;
       g.p[0] = gemm_pair(ps.delta[l], ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
       ColsumSink cs = {};
@@ -778,6 +783,7 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       }
       launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, ps.delta[l], B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
+      side.end();
     }
     if (l > 0) {
       // dh = delta_l W_l ; delta_{l-1} = dh * act'(a_{l-1}) in op16: one kernel.  dh itself is kept
@@ -800,7 +806,7 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       BETTY_TRY(gemm(c, g));
     }
   }
-  return BETTY_OK;
+  return side.join();
 }
 static inline GradSink grad_into(float* gflat, const float* lam) {
   GradSink s = {}; s.gflat = gflat; s.lam = lam; return s;
@@ -1144,6 +1150,9 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, HvpCache* h, const fl
     BETTY_LAUNCH_CHECK();
   }
   const bool leave16 = sink && h->dir16[0];     // the weight-HVP epilogues also leave the op16 copy of the new partial sum in dir16
+  // The chain is Rdelta_L -> Rdelta_{L-1} -> ... ; each layer's weight product goes to the side stream once the
+  // chain's product of the same layer has been launched (it reads the U_l that the weight product may overwrite).
+  SideWork side(c);
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
     op16* Rdp = nullptr;
@@ -1161,6 +1170,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, HvpCache* h, const fl
       BETTY_TRY(gemm(c, g));
     }
     {  // R gW_l = Rdelta^T h_l + delta_l^T Rh_l + exp(lam_l) U_l
+      side.begin();
       GemmDesc g = {}; g.M = (int)N; g.N = (int)K; g.ldc = K; g.beta = 0.f; g.npairs = 0;
       g.p[g.npairs++] = gemm_pair(Rd, ldd, true, ps.h[l], ps.ldh[l], false, (int)B);
       if (l > 0) g.p[g.npairs++] = gemm_pair(ps.delta[l], ldd, true, rp.Rh[l], ps.ldh[l], false, (int)B);
@@ -1183,9 +1193,11 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, HvpCache* h, const fl
       }
       launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, Rd, B, N, ldd, cs);
       BETTY_LAUNCH_CHECK();
+      side.end();
     }
     if (l > 0) Rd = Rdp;
   }
+  BETTY_TRY(side.join());
   if (leave16) h->dir16_of = sink->out;
   c.arena.release(mark);
   return BETTY_OK;
