@@ -49,21 +49,37 @@ __global__ void k_bias_act(float* a, const float* bias, op16* h, int64_t rows, i
     if (h) h[r * ldh + n] = to_op16(act_f(act, v));
   }
 }
-// one warp per row: p = softmax(z), ell = -log p[y]
+// one warp per row: p = softmax(z), ell = -log p[y].  Rows of up to 1024 classes are held in registers
+// (32 values per lane, every load issued before the first use); longer rows are read three times.
 __global__ void k_softmax_ce(const float* z, const int32_t* y, float* p, float* ell, int64_t B, int64_t C) {
   pdl_enter();
   const int lane = threadIdx.x & 31;
   const int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
   if (row >= B) return;
   const float* zr = z + row * C;
-  float mx = -INFINITY;
-  for (int64_t c = lane; c < C; c += 32) mx = fmaxf(mx, zr[c]);
-  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  float s = 0.f;
-  for (int64_t c = lane; c < C; c += 32) s += expf(zr[c] - mx);
-  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  const float ls = logf(s);
-  for (int64_t c = lane; c < C; c += 32) p[row * C + c] = expf(zr[c] - mx - ls);
+  float mx = -INFINITY, s = 0.f, ls;
+  if (C <= 1024) {
+    float v[32];
+    const int nk = (int)((C + 31) >> 5);      // uniform: rounds of 32 classes this row has
+#pragma unroll
+    for (int k = 0; k < 32; ++k) { const int64_t c = lane + 32 * k; v[k] = (k < nk && c < C) ? zr[c] : -INFINITY; }
+#pragma unroll
+    for (int k = 0; k < 32; ++k) if (k < nk) mx = fmaxf(mx, v[k]);
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+#pragma unroll
+    for (int k = 0; k < 32; ++k) if (k < nk && lane + 32 * k < C) s += expf(v[k] - mx);     // same order as the loop below
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    ls = logf(s);
+#pragma unroll
+    for (int k = 0; k < 32; ++k) { const int64_t c = lane + 32 * k; if (k < nk && c < C) p[row * C + c] = expf(v[k] - mx - ls); }
+  } else {
+    for (int64_t c = lane; c < C; c += 32) mx = fmaxf(mx, zr[c]);
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int64_t c = lane; c < C; c += 32) s += expf(zr[c] - mx);
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    ls = logf(s);
+    for (int64_t c = lane; c < C; c += 32) p[row * C + c] = expf(zr[c] - mx - ls);
+  }
   if (lane == 0) {
     int32_t yy = y[row];
     yy = yy < 0 ? 0 : (yy >= C ? (int32_t)C - 1 : yy);     // class ids are validated on the host side of a dataset; clamp

@@ -69,3 +69,51 @@ def test_reweighting_step_replays_identically():
     g.replay()
     torch.cuda.synchronize()
     assert torch.equal(out, direct)
+
+
+def test_one_stream_order_and_two_stream_order_give_the_same_bits():
+    """The MLP families fork weight-gradient work to a second stream that each host thread gets at its
+    first call outside a capture.  A thread whose first call is captured has none and launches
+    everything in program order on the captured stream; both orders must give identical bits."""
+    import threading
+    import paper_2207_02849_b200 as bt
+    from tests import cuda_build as cb
+    inp = si.reweight_bilevel(67, (72, 136, 64, 10), 200, 0.4, activation="gelu")
+    w, th = cb.reweight_levels(inp)
+    w0 = w.params.clone()
+    ws = bt.Workspace([w, th])
+    out = torch.empty(si.WEIGHTNET_PARAMS, dtype=torch.float32, device="cuda")
+
+    def step():
+        w.params.copy_(w0)
+        bt.betty_lower_step(w, 2, ws)
+        bt.betty_hypergrad_neumann(w, th, th, 3, 0.01, out, ws)
+
+    step()          # this thread has made calls before: two streams
+    step()
+    torch.cuda.synchronize()
+    direct_out, direct_w = out.clone(), w.params.clone()
+    got = {}
+
+    def worker():
+        try:
+            torch.cuda.set_device(0)
+            s = torch.cuda.Stream()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s, capture_error_mode="thread_local"):
+                step()
+            out.zero_()
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            got["out"], got["w"] = out.clone(), w.params.clone()
+        except Exception as e:      # surfaces in the asserting thread
+            got["error"] = e
+
+    t = threading.Thread(target=worker)
+    t.start()
+    t.join()
+    assert "error" not in got, got.get("error")
+    assert torch.equal(got["out"], direct_out)
+    assert torch.equal(got["w"], direct_w)
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
