@@ -203,7 +203,9 @@ SideLane* side_lane(cudaStream_t main);
 // stream, in program order.
 class SideWork {
  public:
-  explicit SideWork(Ctx& c) : c_(c), lane_(c.on_side ? nullptr : side_lane(c.stream)), main_(c.stream), used_(false), ok_(true) {}
+  // enable = false: a scope that forks nothing (everything in program order on the caller's stream)
+  explicit SideWork(Ctx& c, bool enable = true)
+      : c_(c), lane_((c.on_side || !enable) ? nullptr : side_lane(c.stream)), main_(c.stream), used_(false), ok_(true) {}
   ~SideWork() { (void)join(); }
   SideWork(const SideWork&) = delete;
   SideWork& operator=(const SideWork&) = delete;
