@@ -443,20 +443,18 @@ class ThreeLevelWorkload:
         self.bt, self.torch = bt, torch
         self.P = cb.three_levels(self.inp)
         self.w0 = self.P[0].params.clone()
-        self.u = torch.empty(self.inp.w.size, dtype=torch.float32, device="cuda")
-        self.vt = torch.empty(self.inp.theta.size, dtype=torch.float32, device="cuda")
         self.out = torch.empty(self.inp.lam.size, dtype=torch.float32, device="cuda")
         self.ws = bt.Workspace(list(self.P))
         self.cfgm = bt.MethodCfg(bt.BETTY_NEUMANN, K=self.inp.K, alpha=self.inp.alpha)
+        self.u2l = [(2, 0), (1, 0)]              # lambda and theta constrain the classifier
+        self.l2u = [(0, 1), (0, 2), (1, 2)]      # w* constrains P2 and P3, theta* constrains P3
 
     def step(self):
         bt, (P1, P2, P3) = self.bt, self.P
         P1.params.copy_(self.w0)
         bt.betty_lower_step(P1, 1, self.ws)
-        bt.betty_grad(P3, P1, self.u, self.ws)
-        bt.betty_grad(P3, P2, self.vt, self.ws)
-        bt.betty_chain_levels(list(self.P), [0, 1], [self.cfgm], self.vt, self.u, True, self.ws)
-        bt.betty_chain_levels(list(self.P), [2, 0], [self.cfgm], self.u, self.out, False, self.ws)
+        # Eq. 2 over the program's dataflow graph, both paths from lambda merged at the w* node: one call
+        bt.betty_hypergrad_graph(list(self.P), self.u2l, self.l2u, 2, [self.cfgm] * 3, self.out, self.ws)
 
     def setup_host(self):
         torch = self.torch

@@ -620,16 +620,24 @@ static betty_status graph_hypergrad(Ctx& c, const betty_level* const* levels, co
   for (int i = 0; i < g.n_l2u; ++i)
     if (g.l2u[i].to == k) is_target[g.l2u[i].from] = true;     // L_k: the lower problems that call k
   GraphEval e = {&c, levels, &g, k, is_target, per_level, u, state};
-  BETTY_TRY(level_grad(c, levels[k], levels[k], out));          // direct gradient
-  for (int i = 0; i < g.n_u2l; ++i) {
+  // No parameter changes during this evaluation, and every pass through a classifier evaluates it at the
+  // same matrices: the first MLP level's matrices are rounded to operand precision once, not once per pass.
+  const betty_level* mlp = nullptr;
+  for (int i = 0; i < g.n && !mlp; ++i)
+    if (levels[i] && levels[i]->param_kind == BETTY_PARAM_MLP) mlp = levels[i];
+  const bool share = mlp && !c.shared.master;
+  if (share) BETTY_TRY(mlpfam_share_weights(c, mlp));
+  betty_status rc = level_grad(c, levels[k], levels[k], out);          // direct gradient
+  for (int i = 0; i < g.n_u2l && rc == BETTY_OK; ++i) {
     if (g.u2l[i].from != k) continue;
     const int c0 = g.u2l[i].to;
     if (c0 == k) continue;
-    BETTY_TRY(eval_node(e, c0));
-    if (!u[c0]) continue;
-    BETTY_TRY(brj(c, levels[c0], levels[k], u[c0], per_level[c0], out, true));
+    rc = eval_node(e, c0);
+    if (rc != BETTY_OK || !u[c0]) continue;
+    rc = brj(c, levels[c0], levels[k], u[c0], per_level[c0], out, true);
   }
-  return BETTY_OK;
+  if (share) mlpfam_unshare_weights(c);
+  return rc;
 }
 
 // Execution of Sec. 3.3: a problem takes one gradient step when called; after every unroll_steps of

@@ -153,12 +153,12 @@ __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
     // one value: 6 shuffles for the four sums of the full HVP form (20 with one full butterfly per sum), 5 for two.
     if (NEEDZ && HVP) {
       const bool up1 = (lane & 16) != 0, up2 = (lane & 8) != 0;
-      // round 1: lanes with bit 4 clear keep row 0's sums, the others row 1's
+      // first halving: lanes with bit 4 clear keep row 0's sums, the others row 1's
       float k0 = up1 ? pz[1] : pz[0], k1 = up1 ? pt[1] : pt[0];
       const float s0 = up1 ? pz[0] : pz[1], s1 = up1 ? pt[0] : pt[1];
       k0 += __shfl_xor_sync(0xffffffffu, s0, 16);
       k1 += __shfl_xor_sync(0xffffffffu, s1, 16);
-      // round 2: lanes with bit 3 clear keep the x.w sum, the others the x.u sum
+      // second halving: lanes with bit 3 clear keep the x.w sum, the others the x.u sum
       float v = up2 ? k1 : k0;
       v += __shfl_xor_sync(0xffffffffu, up2 ? k0 : k1, 8);
       v += __shfl_xor_sync(0xffffffffu, v, 4);
@@ -181,7 +181,7 @@ __global__ void __launch_bounds__(LR_THREADS, 2) k_logreg_stream(LrArgs a) {
     }
 
     // every thread has copied its part of stage s into registers; the same barrier makes the
-    // verdict on an expired wait uniform across the CTA
+    // decision about an expired wait uniform across the CTA
     if (__syncthreads_or(!landed)) { timed_out = true; break; }
     if (tid == 0) {
       const int64_t tn = t + (int64_t)LR_S * gridDim.x;

@@ -217,6 +217,10 @@ def test_config4_full_size(bt, parity_record):
     bt.betty_chain_levels([P1, P2, P3], [0, 1], [cfg], v_t, u, True, ws)
     bt.betty_chain_levels([P1, P2, P3], [2, 0], [cfg], u, out, False, ws)
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+    # the same quantity from the dataflow graph in one call (both paths from lambda, merged at the w* node)
+    out_g = _vec(inp.lam.size)
+    bt.betty_hypergrad_graph([P1, P2, P3], [(2, 0), (1, 0)], [(0, 1), (0, 2), (1, 2)], 2, [cfg, cfg, cfg], out_g, ws)
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
     for quant in ("operands", "weights"):
         O1, O2, O3 = ob.three_levels(inp, quant=quant)
         oracle.lower_step(O1, 1)
@@ -226,6 +230,8 @@ def test_config4_full_size(bt, parity_record):
         assert parity_record(f"config4/{quant}/u", cb.rel_l2(u, ou)) < (TOL if quant == "operands" else TOL_INTERMEDIATE_PLAIN)
         assert parity_record(f"config4/{quant}/chain", cb.rel_l2(out, ref)) < TOL
         assert parity_record(f"config4/{quant}/chain_max", cb.rel_max(out, ref)) < TOL     # each of the three components
+        assert parity_record(f"config4/{quant}/graph", cb.rel_l2(out_g, ref)) < TOL
+        assert cb.rel_max(out_g, ref) < TOL
 
 
 def test_config5_reduced_width(bt):
