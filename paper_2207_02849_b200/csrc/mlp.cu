@@ -276,7 +276,7 @@ static betty_status layer_dot(Ctx& c, const op16* W, int64_t rows, int64_t cols,
   const size_t mark = c.arena.mark();
   BETTY_ALLOC(partial, double, c, (size_t)nb);
   BETTY_ALLOC(counter, unsigned, c, 8);
-  if (cudaMemsetAsync(counter, 0, 32, c.stream) != cudaSuccess) return BETTY_ERR_CUDA;
+  BETTY_TRY(vec_zero(c, (float*)counter, 8));     // a kernel, not a memset: keeps the programmatic launch chain unbroken
   launch_pdl(k_layer_dot, dim3((unsigned)nb), dim3(256), 0, c.stream, W, rows, cols, ldw, q, lam, scale, out, accumulate ? 1 : 0, partial, counter);
   BETTY_LAUNCH_CHECK();
   c.arena.release(mark);
@@ -730,7 +730,7 @@ static betty_status forward(Ctx& c, const Net& n, const betty_level* D, Pass& ps
       ps.ldh[l + 1] = ld8(N);
       hn = c.arena.alloc<op16>((size_t)(B * ps.ldh[l + 1]));
       if (!hn) return BETTY_ERR_WORKSPACE;
-      if (ps.ldh[l + 1] != N) cudaMemsetAsync(hn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(op16), c.stream);
+      if (ps.ldh[l + 1] != N) BETTY_TRY(vec_zero(c, (float*)hn, (int64_t)((size_t)(B * ps.ldh[l + 1])) / 2));
       ps.h[l + 1] = hn;
     }
     // a_l = h_l W_l^T + b_l (kept in fp32 for the derivative passes), h_{l+1} = act(a_l) in op16: one kernel
@@ -816,7 +816,7 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       ps.dh[l] = dh;
       const int64_t ldp = ld8(K);
       BETTY_ALLOC(dp, op16, c, (size_t)(B * ldp));
-      if (ldp != K) cudaMemsetAsync(dp, 0, (size_t)(B * ldp) * sizeof(op16), c.stream);
+      if (ldp != K) BETTY_TRY(vec_zero(c, (float*)dp, (int64_t)((size_t)(B * ldp)) / 2));
       ps.delta[l - 1] = dp;
       GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.npairs = 1; g.C = dh; g.ldc = K; g.beta = 0.f;
       g.p[0] = gemm_pair(ps.delta[l], ldd, false, n.W[l], n.ldw[l], false, (int)N);
@@ -855,7 +855,7 @@ static betty_status rforward(Ctx& c, const Net& n, const Pass& ps, const float* 
     if (l < n.L - 1) {
       Rhn = c.arena.alloc<op16>((size_t)(B * ps.ldh[l + 1]));
       if (!Rhn) return BETTY_ERR_WORKSPACE;
-      if (ps.ldh[l + 1] != N) cudaMemsetAsync(Rhn, 0, (size_t)(B * ps.ldh[l + 1]) * sizeof(op16), c.stream);
+      if (ps.ldh[l + 1] != N) BETTY_TRY(vec_zero(c, (float*)Rhn, (int64_t)((size_t)(B * ps.ldh[l + 1])) / 2));
       rp.Rh[l + 1] = Rhn;
     }
     // Ra_l = h_l U_l^T + Rh_l W_l^T + c_l ; Rh_{l+1} = act'(a_l) * Ra_l: one kernel
@@ -961,7 +961,7 @@ static betty_status wn_backward(Ctx& c, const betty_level* theta, const float* d
   const size_t mark = c.arena.mark();
   BETTY_ALLOC(partial, double, c, (size_t)nb * WN_STRIDE);
   BETTY_ALLOC(counter, unsigned, c, 8);
-  if (cudaMemsetAsync(counter, 0, 32, c.stream) != cudaSuccess) return BETTY_ERR_CUDA;
+  BETTY_TRY(vec_zero(c, (float*)counter, 8));     // a kernel, not a memset: keeps the programmatic launch chain unbroken
   launch_pdl(k_wn_backward, dim3(nb), dim3(128), 0, c.stream, theta->params, dir, ps.ell, cA, cB, ps.B, mu, muvec, out, accumulate ? 1 : 0,
                                           out_scale, partial, counter);
   BETTY_LAUNCH_CHECK();
@@ -1181,7 +1181,7 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, HvpCache* h, const fl
       const int64_t ldp = ld8(K);
       Rdp = c.arena.alloc<op16>((size_t)(B * ldp));
       if (!Rdp) return BETTY_ERR_WORKSPACE;
-      if (ldp != K) cudaMemsetAsync(Rdp, 0, (size_t)(B * ldp) * sizeof(op16), c.stream);
+      if (ldp != K) BETTY_TRY(vec_zero(c, (float*)Rdp, (int64_t)((size_t)(B * ldp)) / 2));
       GemmDesc g = {}; g.M = (int)B; g.N = (int)K; g.C = nullptr; g.ldc = K; g.beta = 0.f; g.npairs = 2;
       g.p[0] = gemm_pair(Rd, ldd, false, n.W[l], n.ldw[l], false, (int)N);
       g.p[1] = gemm_pair(ps.delta[l], ldd, false, rp.U[l], n.ldw[l], false, (int)N);
@@ -1303,7 +1303,7 @@ betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int fi
     const size_t cnt = (size_t)(n.w[l + 1] * n.ldw[l]);
     alt[l] = c.arena.alloc<op16>(cnt);
     if (!alt[l]) return BETTY_ERR_WORKSPACE;
-    if (n.ldw[l] != n.w[l]) cudaMemsetAsync(alt[l], 0, cnt * sizeof(op16), c.stream);
+    if (n.ldw[l] != n.w[l]) BETTY_TRY(vec_zero(c, (float*)alt[l], (int64_t)(cnt) / 2));
   }
   for (int s = 0; s < n_steps; ++s) {
     const size_t m2 = c.arena.mark();
@@ -1389,8 +1389,8 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
         BETTY_ALLOC(hn, op16, c, cnt);
         BETTY_ALLOC(dn, op16, c, cnt);
         if (ps.ldh[l + 1] != N) {
-          cudaMemsetAsync(hn, 0, cnt * sizeof(op16), c.stream);
-          cudaMemsetAsync(dn, 0, cnt * sizeof(op16), c.stream);
+          BETTY_TRY(vec_zero(c, (float*)hn, (int64_t)(cnt) / 2));
+          BETTY_TRY(vec_zero(c, (float*)dn, (int64_t)(cnt) / 2));
         }
         launch_pdl(k_fd_act, dim3(grid_for(B * N)), dim3(256), 0, c.stream, ps.a[l], da, v + n.boff[l], vnorm2, eps0, sign, hn, dn, nullptr, B, N,
                                                        ps.ldh[l + 1], n.act, (P.corr && l == n.L - 2) ? hlast_p : (float*)nullptr);

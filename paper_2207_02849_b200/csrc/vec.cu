@@ -137,8 +137,7 @@ __global__ void k_dot(const float* x, const float* y, int64_t n, float* result, 
 
 betty_status vec_reduce_init(Ctx& c, float* partials) {
   unsigned* counter = (unsigned*)((double*)partials + DOT_MAX_BLOCKS);
-  if (cudaMemsetAsync(counter, 0, 32, c.stream) != cudaSuccess) return BETTY_ERR_CUDA;
-  return BETTY_OK;
+  return vec_zero(c, (float*)counter, 8);     // a kernel, not a memset: keeps the programmatic launch chain unbroken
 }
 
 betty_status vec_dot(Ctx& c, const float* x, const float* y, int64_t n, float* result, float* partials) {
