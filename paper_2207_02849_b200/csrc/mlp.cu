@@ -337,21 +337,31 @@ __global__ void k_wn_backward(const float* theta, const float* dir, const float*
   const int64_t per = (B + gridDim.x - 1) / gridDim.x;
   const int64_t i0 = blockIdx.x * per, i1 = (i0 + per < B) ? i0 + per : B;
   double ga1 = 0.0, gb1 = 0.0, ga2 = 0.0, gb2 = 0.0;
-  if (k < WN_H) {
-    const float a1 = theta[k], b1 = theta[WN_H + k], a2 = theta[2 * WN_H + k];
-    const float da1 = dir ? dir[k] : 0.f, db1 = dir ? dir[WN_H + k] : 0.f, da2 = dir ? dir[2 * WN_H + k] : 0.f;
-    for (int64_t i = i0; i < i1; ++i) {
-      const float l = ell[i], ca = cA[i], cb = cB ? cB[i] : 0.f;
-      const float pre = a1 * l + b1;
-      if (pre > 0.f) {
-        const float t = ca * a2 + cb * da2;
-        ga1 += (double)(l * t);
-        gb1 += (double)t;
-        ga2 += (double)(ca * pre + cb * (l * da1 + db1));
+  const bool unit = k < WN_H;
+  const float a1 = unit ? theta[k] : 0.f, b1 = unit ? theta[WN_H + k] : 0.f, a2 = unit ? theta[2 * WN_H + k] : 0.f;
+  const float da1 = (unit && dir) ? dir[k] : 0.f, db1 = (unit && dir) ? dir[WN_H + k] : 0.f, da2 = (unit && dir) ? dir[2 * WN_H + k] : 0.f;
+  // the block's samples pass through shared memory 128 at a time (one coalesced load per array instead of one
+  // broadcast load per sample and thread); every thread still adds its samples in index order
+  __shared__ float s_l[128], s_a[128], s_b[128];
+  for (int64_t c0 = i0; c0 < i1; c0 += 128) {
+    const int cnt = (int)((i1 - c0 < 128) ? i1 - c0 : 128);
+    __syncthreads();
+    if (k < cnt) { s_l[k] = ell[c0 + k]; s_a[k] = cA[c0 + k]; s_b[k] = cB ? cB[c0 + k] : 0.f; }
+    __syncthreads();
+    if (unit) {
+      for (int i = 0; i < cnt; ++i) {
+        const float l = s_l[i], ca = s_a[i], cb = s_b[i];
+        const float pre = a1 * l + b1;
+        if (pre > 0.f) {
+          const float t = ca * a2 + cb * da2;
+          ga1 += (double)(l * t);
+          gb1 += (double)t;
+          ga2 += (double)(ca * pre + cb * (l * da1 + db1));
+        }
       }
+    } else if (k == WN_H) {
+      for (int i = 0; i < cnt; ++i) gb2 += (double)s_a[i];
     }
-  } else if (k == WN_H) {
-    for (int64_t i = i0; i < i1; ++i) gb2 += (double)cA[i];
   }
   double* mine = partial + (size_t)blockIdx.x * WN_STRIDE;
   if (k < WN_H) { mine[k] = ga1; mine[WN_H + k] = gb1; mine[2 * WN_H + k] = ga2; }
@@ -363,9 +373,16 @@ __global__ void k_wn_backward(const float* theta, const float* dir, const float*
   __syncthreads();
   if (!is_last) return;
   __threadfence();
+  // block order, eight loads in flight at a time (L2 loads: the partial sums were written by other SMs)
   auto total = [&](int idx) {
     double t = 0.0;
-    for (unsigned bb = 0; bb < gridDim.x; ++bb) t += ((volatile double*)partial)[(size_t)bb * WN_STRIDE + idx];
+    for (unsigned b0 = 0; b0 < gridDim.x; b0 += 8) {
+      double v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = b0 + u < gridDim.x ? __ldcg(partial + (size_t)(b0 + u) * WN_STRIDE + idx) : 0.0;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) if (b0 + u < gridDim.x) t += v[u];
+    }
     return t;
   };
   auto put = [&](int idx) {
