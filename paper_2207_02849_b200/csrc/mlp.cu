@@ -968,9 +968,11 @@ static betty_status wn_sample(Ctx& c, int mode, const betty_level* theta, const 
   BETTY_LAUNCH_CHECK();
   return BETTY_OK;
 }
+// keep_scratch: the partial-sum scratch stays allocated (for a caller that runs this on the side stream and
+// releases the arena only after the join)
 static betty_status wn_backward(Ctx& c, const betty_level* theta, const float* dir, const Pass& ps, const float* cA,
                                 const float* cB, float mu, const float* muvec, float* out, bool accumulate = false,
-                                float out_scale = 1.f) {
+                                float out_scale = 1.f, bool keep_scratch = false) {
   // 64 samples per block: the block that comes last reads every block's 301 partial sums, so few blocks
   // keep that second phase short (batch 1024: 16 blocks)
   int nb = (int)((ps.B + 63) / 64);
@@ -982,7 +984,7 @@ static betty_status wn_backward(Ctx& c, const betty_level* theta, const float* d
   launch_pdl(k_wn_backward, dim3(nb), dim3(128), 0, c.stream, theta->params, dir, ps.ell, cA, cB, ps.B, mu, muvec, out, accumulate ? 1 : 0,
                                           out_scale, partial, counter);
   BETTY_LAUNCH_CHECK();
-  c.arena.release(mark);
+  if (!keep_scratch) c.arena.release(mark);
   return BETTY_OK;
 }
 
@@ -1369,12 +1371,8 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
   if (!wrt_theta && !wrt_corr) return BETTY_ERR_INVALID_ARG;
   BETTY_TRY(forward(c, n, L, ps));
   const int64_t B = ps.B, C = n.w[n.L];
-  // the label-correction net is evaluated at the perturbed last hidden activation, in fp32
-  float* hlast_p = nullptr;
-  if (P.corr) {
-    hlast_p = c.arena.alloc<float>((size_t)((B > 0 ? B : 1) * n.w[n.L - 1]));
-    if (!hlast_p) return BETTY_ERR_WORKSPACE;
-  }
+  // The two perturbed passes (x + eps v and x - eps v) share nothing but read-only inputs: each gets buffers of
+  // its own, the second runs on the side stream beside the first, and nothing is released before the join.
   const int64_t n_out = wrt->n_params, gstride = (n_out + 63) & ~int64_t(63);
   op16* E[MAXL];
   for (int l = 0; l < n.L; ++l) {
@@ -1383,15 +1381,24 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
     BETTY_TRY(cast_matrix(c, v + n.woff[l], E[l], n.w[l + 1], n.w[l], n.ldw[l], vnorm2, eps0));
   }
   BETTY_ALLOC(G, float, c, (size_t)(2 * gstride));
-  BETTY_ALLOC(zpm, float, c, (size_t)(B * C));
-  BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
-  Pass pp = ps;   // perturbed pass: reuses y/B, gets its own p/ell
-  BETTY_ALLOC(p2, float, c, (size_t)(B * C));
-  BETTY_ALLOC(ell2, float, c, (size_t)(B > 0 ? B : 1));
-  pp.p = p2; pp.ell = ell2;
-  for (int sgn = 0; sgn < 2; ++sgn) {
+  SideWork side(c);
+  for (int pass = 0; pass < 2; ++pass) {
+    // the side stream's pass is launched first: it starts after what is on the caller's stream at that moment
+    const int sgn = 1 - pass;
     const float sign = sgn == 0 ? 1.f : -1.f;
-    const size_t m2 = c.arena.mark();
+    if (sgn == 1) side.begin();
+    // the label-correction net is evaluated at the perturbed last hidden activation, in fp32
+    float* hlast_p = nullptr;
+    if (P.corr) {
+      hlast_p = c.arena.alloc<float>((size_t)((B > 0 ? B : 1) * n.w[n.L - 1]));
+      if (!hlast_p) return BETTY_ERR_WORKSPACE;
+    }
+    BETTY_ALLOC(zpm, float, c, (size_t)(B * C));
+    BETTY_ALLOC(s1, float, c, (size_t)(B > 0 ? B : 1));
+    Pass pp = ps;   // perturbed pass: reuses y/B, gets its own p/ell
+    BETTY_ALLOC(p2, float, c, (size_t)(B * C));
+    BETTY_ALLOC(ell2, float, c, (size_t)(B > 0 ? B : 1));
+    pp.p = p2; pp.ell = ell2;
     const op16* hp = ps.h[0];      // perturbed input of the layer (layer 0: the data itself)
     const op16* dh = nullptr;      // its difference from the base input
     for (int l = 0; l < n.L; ++l) {
@@ -1425,7 +1432,7 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
     if (P.corr) BETTY_TRY(corr_forward(c, n, pp, P.corr, cpp, hlast_p, zpm));     // pp.ell: soft-label losses at x +- eps v
     if (wrt_theta) {
       BETTY_TRY(wn_sample(c, WN_REWEIGHT_TGRAD, P.theta, nullptr, pp, nullptr, nullptr, s1, nullptr));
-      BETTY_TRY(wn_backward(c, P.theta, nullptr, pp, s1, nullptr, 0.f, nullptr, G + gstride * sgn));
+      BETTY_TRY(wn_backward(c, P.theta, nullptr, pp, s1, nullptr, 0.f, nullptr, G + gstride * sgn, false, 1.f, true));
     } else {
       const float* coefp;
       BETTY_TRY(reweight_coef(c, P, pp, &coefp));
@@ -1433,8 +1440,9 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
       BETTY_TRY(corr_sample_grad(c, 0, cpp, pp, coefp, &G32, &G16, &ldg));
       BETTY_TRY(corr_param_grad(c, cpp, pp, G32, G + gstride * sgn));
     }
-    c.arena.release(m2);
+    if (sgn == 1) side.end();
   }
+  BETTY_TRY(side.join());
   launch_pdl(k_fd_combine, dim3(grid_for(n_out)), dim3(256), 0, c.stream, out, G, G + gstride, vnorm2, eps0, alpha, accumulate ? 1 : 0, n_out);
   BETTY_LAUNCH_CHECK();
   c.arena.release(mark);
