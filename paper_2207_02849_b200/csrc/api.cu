@@ -344,8 +344,9 @@ static betty_status step_grad(Ctx& c, const betty_level* L, float* out) {
 }
 
 // (d x*/d c)^T v by the configured approximation; out (+)= result.
+// pre: the base pass of an MLP-family level (mlpfam_hvp_begin) made by the caller, or null
 static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v,
-                        const betty_method_cfg& cfg, float* out, bool accumulate) {
+                        const betty_method_cfg& cfg, float* out, bool accumulate, MlpHvpCache* pre = nullptr) {
   if (!is_participant(L, wrt) || wrt == L) return BETTY_ERR_INVALID_ARG;
   const int64_t n = L->n_params, nc = wrt->n_params;
   const bool vecfam = is_vector_family(L->loss);
@@ -374,8 +375,8 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
   }
   if (cfg.method != BETTY_NEUMANN && cfg.method != BETTY_CG) return BETTY_ERR_INVALID_ARG;
   if (cfg.K < 0) return BETTY_ERR_INVALID_ARG;
-  MlpHvpCache* cache = nullptr;
-  if (!vecfam) BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
+  MlpHvpCache* cache = pre;
+  if (!vecfam && !cache) BETTY_TRY(mlpfam_hvp_begin(c, L, &cache));
   // logistic levels: the per-row curvature at the (fixed) lower parameters is shared by the solve's HVPs
   VecHvpCache vcache = {nullptr, false};
   if (vecfam && L->n > 0 && cfg.K > 1) vcache.curv = c.arena.alloc<float>((size_t)L->n);
@@ -468,9 +469,26 @@ static betty_status hypergrad(const betty_level* lower, const betty_level* upper
   BETTY_ALLOC(v, float, c, (size_t)lower->n_params);
   // the upper gradient and the Jacobian product both evaluate costs at the lower level's present parameters
   BETTY_TRY(mlpfam_share_weights(c, lower));
-  BETTY_TRY(level_grad(c, upper, lower, v));     // dC_u / d theta_lower
-  BETTY_TRY(level_grad(c, upper, wrt, out));     // direct gradient
-  const betty_status rc = brj(c, lower, wrt, v, cfg, out, true);
+  // An MLP-family lower level's base pass (forward and delta chain on its own batch, what every HVP of the solve
+  // starts from) does not depend on the upper level's gradients: it runs on the side stream beside them.  Its
+  // buffers sit below everything the gradients allocate and release, and stay until the call returns.
+  const bool series = cfg.method == BETTY_NEUMANN || cfg.method == BETTY_CG;
+  const bool early = series && cfg.K >= 0 && is_mlp_family(lower->loss) && !lower->comm && !upper->comm;
+  MlpHvpCache* pre = nullptr;
+  betty_status rc = BETTY_OK;
+  {
+    SideWork side(c, early);
+    if (early) {
+      side.begin();
+      rc = mlpfam_hvp_begin(c, lower, &pre);
+      side.end();
+    }
+    if (rc == BETTY_OK) rc = level_grad(c, upper, lower, v);     // dC_u / d theta_lower
+    if (rc == BETTY_OK) rc = level_grad(c, upper, wrt, out);     // direct gradient
+    const betty_status rj = side.join();
+    if (rc == BETTY_OK) rc = rj;
+  }
+  if (rc == BETTY_OK) rc = brj(c, lower, wrt, v, cfg, out, true, pre);
   mlpfam_unshare_weights(c);
   return rc;
 }
