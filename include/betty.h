@@ -27,10 +27,12 @@
  *    need to be preserved between calls, but calls sharing one `ws` must not overlap in time.
  *  - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and return without
  *    synchronising.  The MLP families also use one stream of the library's own (made once per host
- *    thread and device, never destroyed, no device memory): work that nothing in a reverse sweep's
- *    chain waits for (weight-gradient products, bias sums) runs there, forked from and joined back
- *    into `stream` with events inside the call, so the caller sees ordinary stream order and a
- *    stream capture of a call records the same dependencies.  The first MLP-family call of a
+ *    thread and device, never destroyed, no device memory): independent pieces of a call (the
+ *    weight-gradient products and bias sums beside a reverse sweep's chain, one of the two
+ *    perturbed passes of a finite difference, a lower level's base pass beside the upper level's
+ *    gradients) run there, forked from and joined back into `stream` with events inside the call,
+ *    so the caller sees ordinary stream order and a stream capture of a call records the same
+ *    dependencies.  The first MLP-family call of a
  *    thread should not be made under a capture (it then runs without the second stream).  Argument errors are returned immediately and nothing is enqueued.
  *    Conditions found on the device (non-finite values, CG breakdown, an expired bounded wait)
  *    are recorded in the status block and reported by betty_poll_status.

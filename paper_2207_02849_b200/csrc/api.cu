@@ -599,7 +599,17 @@ static void dfs_paths(const Graph& g, int k, const bool* is_target, int* stack, 
 struct GraphEval {
   Ctx* c; const betty_level* const* levels; const Graph* g; int k; const bool* is_target;
   const betty_method_cfg* cfg; float** u; int* state;   // state: 0 new, 1 in progress, 2 done (u may stay null: no target above)
+  float** tgrad;           // dC_k / d theta_c of the target nodes, where already evaluated (else null)
+  MlpHvpCache** pre;       // base passes of MLP-family nodes, where already made (else null)
 };
+// The nodes an evaluation from k will visit below child c0 (each once), in the order their Jacobian products run.
+static void collect_nodes(const Graph& g, int k, int cnode, bool* seen, int* order, int& n) {
+  if (seen[cnode]) return;
+  seen[cnode] = true;
+  for (int i = 0; i < g.n_l2u; ++i)
+    if (g.l2u[i].from == cnode && g.l2u[i].to != k) collect_nodes(g, k, g.l2u[i].to, seen, order, n);
+  order[n++] = cnode;
+}
 static betty_status eval_node(GraphEval& e, int cnode) {
   if (e.state[cnode] == 2) return BETTY_OK;
   if (e.state[cnode] == 1) return BETTY_ERR_INVALID_ARG;      // cycle among lower-to-upper edges
@@ -607,9 +617,12 @@ static betty_status eval_node(GraphEval& e, int cnode) {
   float* acc = nullptr;
   const int64_t nc = e.levels[cnode]->n_params;
   if (e.is_target[cnode]) {
-    acc = e.c->arena.alloc<float>((size_t)nc);
-    if (!acc) return BETTY_ERR_WORKSPACE;
-    BETTY_TRY(level_grad(*e.c, e.levels[e.k], e.levels[cnode], acc));
+    acc = e.tgrad[cnode];
+    if (!acc) {
+      acc = e.c->arena.alloc<float>((size_t)nc);
+      if (!acc) return BETTY_ERR_WORKSPACE;
+      BETTY_TRY(level_grad(*e.c, e.levels[e.k], e.levels[cnode], acc));
+    }
   }
   for (int i = 0; i < e.g->n_l2u; ++i) {
     if (e.g->l2u[i].from != cnode) continue;
@@ -623,7 +636,7 @@ static betty_status eval_node(GraphEval& e, int cnode) {
       if (!acc) return BETTY_ERR_WORKSPACE;
       accumulate = false;
     }
-    BETTY_TRY(brj(*e.c, e.levels[nx], e.levels[cnode], e.u[nx], e.cfg[nx], acc, accumulate));
+    BETTY_TRY(brj(*e.c, e.levels[nx], e.levels[cnode], e.u[nx], e.cfg[nx], acc, accumulate, e.pre[nx]));
   }
   e.u[cnode] = acc;
   e.state[cnode] = 2;
@@ -637,7 +650,9 @@ static betty_status graph_hypergrad(Ctx& c, const betty_level* const* levels, co
   int state[256] = {0};
   for (int i = 0; i < g.n_l2u; ++i)
     if (g.l2u[i].to == k) is_target[g.l2u[i].from] = true;     // L_k: the lower problems that call k
-  GraphEval e = {&c, levels, &g, k, is_target, per_level, u, state};
+  float* tgrad[256] = {nullptr};
+  MlpHvpCache* pre[256] = {nullptr};
+  GraphEval e = {&c, levels, &g, k, is_target, per_level, u, state, tgrad, pre};
   // No parameter changes during this evaluation, and every pass through a classifier evaluates it at the
   // same matrices: the first MLP level's matrices are rounded to operand precision once, not once per pass.
   const betty_level* mlp = nullptr;
@@ -645,14 +660,52 @@ static betty_status graph_hypergrad(Ctx& c, const betty_level* const* levels, co
     if (levels[i] && levels[i]->param_kind == BETTY_PARAM_MLP) mlp = levels[i];
   const bool share = mlp && !c.shared.master;
   if (share) BETTY_TRY(mlpfam_share_weights(c, mlp));
-  betty_status rc = level_grad(c, levels[k], levels[k], out);          // direct gradient
+  // What does not depend on anything computed here runs first, on two streams: the base passes of the MLP-family
+  // nodes whose Jacobian products use a series solve (side stream; at most as many as the per-thread cache slots),
+  // beside the gradients of C_k with respect to k's own parameters and to the target nodes (caller's stream).
+  // Everything the side stream touches is allocated before the gradients' scratch and stays until the call returns.
+  int order[256], n_ord = 0;
+  {
+    bool seen[256] = {false};
+    for (int i = 0; i < g.n_u2l; ++i)
+      if (g.u2l[i].from == k && g.u2l[i].to != k) collect_nodes(g, k, g.u2l[i].to, seen, order, n_ord);
+  }
+  bool plain = !levels[k]->comm;
+  for (int i = 0; i < n_ord; ++i) plain = plain && !levels[order[i]]->comm;
+  betty_status rc = BETTY_OK;
+  {
+    SideWork side(c, plain && n_ord > 0);
+    if (plain) {
+      side.begin();
+      int made = 0;
+      for (int i = 0; i < n_ord && made < MLP_HVP_CACHE_SLOTS; ++i) {
+        const betty_level* L = levels[order[i]];
+        const betty_method_cfg& m = per_level[order[i]];
+        if (!is_mlp_family(L->loss) || (m.method != BETTY_NEUMANN && m.method != BETTY_CG) || m.K < 0) continue;
+        // a pass that cannot be made here is left to the Jacobian product, which reports why
+        if (mlpfam_hvp_begin(c, L, &pre[order[i]]) != BETTY_OK) pre[order[i]] = nullptr;
+        ++made;
+      }
+      side.end();
+    }
+    rc = level_grad(c, levels[k], levels[k], out);          // direct gradient
+    for (int i = 0; i < n_ord && rc == BETTY_OK && plain; ++i) {
+      const int t = order[i];
+      if (!is_target[t]) continue;
+      tgrad[t] = c.arena.alloc<float>((size_t)levels[t]->n_params);
+      if (!tgrad[t]) { rc = BETTY_ERR_WORKSPACE; break; }
+      rc = level_grad(c, levels[k], levels[t], tgrad[t]);
+    }
+    const betty_status rj = side.join();
+    if (rc == BETTY_OK) rc = rj;
+  }
   for (int i = 0; i < g.n_u2l && rc == BETTY_OK; ++i) {
     if (g.u2l[i].from != k) continue;
     const int c0 = g.u2l[i].to;
     if (c0 == k) continue;
     rc = eval_node(e, c0);
     if (rc != BETTY_OK || !u[c0]) continue;
-    rc = brj(c, levels[c0], levels[k], u[c0], per_level[c0], out, true);
+    rc = brj(c, levels[c0], levels[k], u[c0], per_level[c0], out, true, pre[c0]);
   }
   if (share) mlpfam_unshare_weights(c);
   return rc;

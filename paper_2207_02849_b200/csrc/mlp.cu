@@ -1127,8 +1127,9 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
 }
 
 betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache) {
-  static thread_local HvpCache store;   // host-side bookkeeping only; device state lives in the workspace
-  HvpCache& h = store;
+  static thread_local HvpCache store[MLP_HVP_CACHE_SLOTS];   // host-side bookkeeping only; device state lives in the workspace
+  static thread_local unsigned next_slot = 0;
+  HvpCache& h = store[next_slot++ % MLP_HVP_CACHE_SLOTS];
   const Parts P = parts_of(L);
   if (P.corr) return BETTY_ERR_UNSUPPORTED;     // second derivatives are not offered with label correction (the paper pairs it with AID-FD)
   h.theta = P.theta;

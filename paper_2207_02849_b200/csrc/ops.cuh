@@ -89,6 +89,9 @@ static inline float lr_at(const betty_level* L, int step_in_call) {
 }
 
 struct MlpHvpCache;  // opaque handle: base forward/backward state shared by the HVPs of one solve
+// base passes (mlpfam_hvp_begin) a host thread may hold at once: handles are slots of a per-thread ring, and the
+// oldest is reused by the call after this many
+static constexpr int MLP_HVP_CACHE_SLOTS = 8;
 
 // The MLP families exist once per 16-bit operand type (see common.cuh): identical declarations in two namespaces.
 #define BETTY_DECLARE_MLP_FAMILY(NS)                                                                                   \
