@@ -45,8 +45,11 @@ static betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps,
   return BETTY_MLP_DISPATCH(L, mlpfam_lower_step(c, L, n_steps, first_step));
 }
 static betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
-                              float eps0, float alpha, float* out, bool accumulate) {
-  return BETTY_MLP_DISPATCH(L, mlpfam_fd(c, L, wrt, v, vnorm2, eps0, alpha, out, accumulate));
+                              float eps0, float alpha, float* out, bool accumulate, MlpHvpCache* pre) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_fd(c, L, wrt, v, vnorm2, eps0, alpha, out, accumulate, pre));
+}
+static betty_status mlpfam_fd_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache) {
+  return BETTY_MLP_DISPATCH(L, mlpfam_fd_begin(c, L, cache));
 }
 
 std::mutex& smem_limit_mutex() {
@@ -364,7 +367,7 @@ static betty_status brj(Ctx& c, const betty_level* L, const betty_level* wrt, co
     }
     const bool acc_local = accumulate && !L->comm;
     rc = vecfam ? vecfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, dst, acc_local)
-                : mlpfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, dst, acc_local);
+                : mlpfam_fd(c, L, wrt, v, &st->vnorm2, cfg.eps0, cfg.alpha, dst, acc_local, pre);
     if (rc == BETTY_OK && L->comm) {
       BETTY_TRY(dp_reduce(c, L, dst, nc));
       launch_pdl(k_scale_into, dim3(ew_grid(nc)), dim3(256), 0, c.stream, out, (const float*)dst, 1.f, accumulate ? 1 : 0, nc);
@@ -472,15 +475,17 @@ static betty_status hypergrad(const betty_level* lower, const betty_level* upper
   // An MLP-family lower level's base pass (forward and delta chain on its own batch, what every HVP of the solve
   // starts from) does not depend on the upper level's gradients: it runs on the side stream beside them.  Its
   // buffers sit below everything the gradients allocate and release, and stay until the call returns.
-  const bool series = cfg.method == BETTY_NEUMANN || cfg.method == BETTY_CG;
-  const bool early = series && cfg.K >= 0 && is_mlp_family(lower->loss) && !lower->comm && !upper->comm;
+  // (For a finite difference the base pass is the forward pass alone; with respect to a weight decay it needs none.)
+  const bool series = (cfg.method == BETTY_NEUMANN || cfg.method == BETTY_CG) && cfg.K >= 0;
+  const bool fd = cfg.method == BETTY_FD && lower->loss == BETTY_LOSS_MLP_CE_REWEIGHT && wrt->param_kind != BETTY_PARAM_LOGWD;
+  const bool early = (series || fd) && is_mlp_family(lower->loss) && !lower->comm && !upper->comm;
   MlpHvpCache* pre = nullptr;
   betty_status rc = BETTY_OK;
   {
     SideWork side(c, early);
     if (early) {
       side.begin();
-      rc = mlpfam_hvp_begin(c, lower, &pre);
+      rc = fd ? mlpfam_fd_begin(c, lower, &pre) : mlpfam_hvp_begin(c, lower, &pre);
       side.end();
     }
     if (rc == BETTY_OK) rc = level_grad(c, upper, lower, v);     // dC_u / d theta_lower

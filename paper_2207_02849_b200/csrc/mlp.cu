@@ -1126,10 +1126,13 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
   return BETTY_OK;
 }
 
-betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache) {
+static HvpCache& next_cache_slot() {
   static thread_local HvpCache store[MLP_HVP_CACHE_SLOTS];   // host-side bookkeeping only; device state lives in the workspace
   static thread_local unsigned next_slot = 0;
-  HvpCache& h = store[next_slot++ % MLP_HVP_CACHE_SLOTS];
+  return store[next_slot++ % MLP_HVP_CACHE_SLOTS];
+}
+betty_status mlpfam_hvp_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache) {
+  HvpCache& h = next_cache_slot();
   const Parts P = parts_of(L);
   if (P.corr) return BETTY_ERR_UNSUPPORTED;     // second derivatives are not offered with label correction (the paper pairs it with AID-FD)
   h.theta = P.theta;
@@ -1352,13 +1355,27 @@ betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int fi
 // Finite difference of dC/dc at x +- eps v.  For the weight-net constraint the two perturbed forward
 // passes carry the perturbation separately from the base activations (base + delta operands), so that
 // an eps*v far below op16 resolution of the weights survives the op16 matrix products.
+// The part of mlpfam_fd that does not depend on the direction: the classifier's forward pass at the unperturbed
+// parameters.  Its buffers stay allocated (the handle is a slot of the per-thread ring of base passes).
+betty_status mlpfam_fd_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache) {
+  if (L->loss != BETTY_LOSS_MLP_CE_REWEIGHT) return BETTY_ERR_UNSUPPORTED;
+  HvpCache& h = next_cache_slot();
+  const Parts P = parts_of(L);
+  BETTY_TRY(net_setup(c, P.mlp, h.net));
+  BETTY_TRY(forward(c, h.net, L, h.pass));
+  *cache = (MlpHvpCache*)&h;
+  return BETTY_OK;
+}
+
+// pre: the forward pass made by mlpfam_fd_begin, or null
 betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,
-                       float eps0, float alpha, float* out, bool accumulate) {
+                       float eps0, float alpha, float* out, bool accumulate, MlpHvpCache* pre) {
   if (L->loss != BETTY_LOSS_MLP_CE_REWEIGHT) return BETTY_ERR_UNSUPPORTED;
   const Parts P = parts_of(L);
   const size_t mark = c.arena.mark();
   Net n; Pass ps;
-  BETTY_TRY(net_setup(c, P.mlp, n));
+  if (pre) n = ((HvpCache*)pre)->net;
+  else BETTY_TRY(net_setup(c, P.mlp, n));
   if (P.lam && wrt == P.lam) {
     // dC/d(lam_l) = 1/2 exp(lam_l)|W_l|^2 is quadratic in W: its central difference is exactly
     // exp(lam_l) <W_l, V_l> for every eps, which is what is evaluated.
@@ -1370,7 +1387,8 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
   }
   const bool wrt_theta = P.theta && wrt == P.theta, wrt_corr = P.corr && wrt == P.corr;
   if (!wrt_theta && !wrt_corr) return BETTY_ERR_INVALID_ARG;
-  BETTY_TRY(forward(c, n, L, ps));
+  if (pre) ps = ((HvpCache*)pre)->pass;
+  else BETTY_TRY(forward(c, n, L, ps));
   const int64_t B = ps.B, C = n.w[n.L];
   // The two perturbed passes (x + eps v and x - eps v) share nothing but read-only inputs: each gets buffers of
   // its own, the second runs on the side stream beside the first, and nothing is released before the join.

@@ -109,8 +109,9 @@ static constexpr int MLP_HVP_CACHE_SLOTS = 8;
   betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* cache, const betty_level* wrt, const float* q,  \
                             float* out);                                                                               \
   betty_status mlpfam_lower_step(Ctx& c, const betty_level* L, int n_steps, int first_step = 0);                       \
+  betty_status mlpfam_fd_begin(Ctx& c, const betty_level* L, MlpHvpCache** cache);                                     \
   betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, const float* v, const float* vnorm2,    \
-                         float eps0, float alpha, float* out, bool accumulate);                                        \
+                         float eps0, float alpha, float* out, bool accumulate, MlpHvpCache* pre);                      \
   }
 BETTY_DECLARE_MLP_FAMILY(fam_bf16)
 BETTY_DECLARE_MLP_FAMILY(fam_f16)
