@@ -117,3 +117,50 @@ def test_one_stream_order_and_two_stream_order_give_the_same_bits():
     assert torch.equal(got["out"], direct_out)
     assert torch.equal(got["w"], direct_w)
     assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
+
+
+@pytest.mark.parametrize("problem", ["fd", "neumann", "three_levels"])
+def test_two_stream_steps_repeat_bit_for_bit(problem):
+    """The calls fork independent work to a second stream (weight-gradient products beside the delta
+    chain, the two finite-difference passes, a lower level's base pass beside the upper gradients).  A
+    missing dependency between the streams would show as results that change from replay to replay:
+    30 replays of one captured step must all give the bits of the directly launched step."""
+    import paper_2207_02849_b200 as bt
+    from tests import cuda_build as cb
+    if problem == "three_levels":
+        inp = si.three_level(83, (48, 72, 40, 10), 160, 0.3, activation="gelu")
+        P = cb.three_levels(inp)
+        w0 = P[0].params.clone()
+        ws = bt.Workspace(list(P))
+        out = torch.empty(inp.lam.size, dtype=torch.float32, device="cuda")
+        cfg = bt.MethodCfg(bt.BETTY_NEUMANN, K=3, alpha=0.01)
+
+        def step():
+            P[0].params.copy_(w0)
+            bt.betty_lower_step(P[0], 1, ws)
+            bt.betty_hypergrad_graph(list(P), [(2, 0), (1, 0)], [(0, 1), (0, 2), (1, 2)], 2, [cfg] * 3, out, ws)
+    else:
+        inp = si.reweight_bilevel(79, (72, 136, 64, 10), 200, 0.4, activation="gelu")
+        w, th = cb.reweight_levels(inp)
+        w0 = w.params.clone()
+        ws = bt.Workspace([w, th])
+        out = torch.empty(si.WEIGHTNET_PARAMS, dtype=torch.float32, device="cuda")
+
+        def step():
+            w.params.copy_(w0)
+            bt.betty_lower_step(w, 2, ws)
+            if problem == "fd":
+                bt.betty_hypergrad_fd(w, th, th, 0.01, 1.0, out, ws)
+            else:
+                bt.betty_hypergrad_neumann(w, th, th, 3, 0.01, out, ws)
+
+    step()
+    torch.cuda.synchronize()
+    direct = out.clone()
+    g = _capture(step)
+    for _ in range(30):
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, direct)
+    assert bt.betty_poll_status(ws)[0] == bt.BETTY_OK
