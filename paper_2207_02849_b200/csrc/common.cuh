@@ -207,6 +207,7 @@ class SideWork {
   explicit SideWork(Ctx& c, bool enable = true)
       : c_(c), lane_((c.on_side || !enable) ? nullptr : side_lane(c.stream)), main_(c.stream), used_(false), ok_(true) {}
   ~SideWork() { (void)join(); }
+  bool forks() const { return lane_ != nullptr; }   // false: everything stays on the caller's stream
   SideWork(const SideWork&) = delete;
   SideWork& operator=(const SideWork&) = delete;
   void begin() {

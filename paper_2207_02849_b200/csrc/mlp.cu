@@ -111,11 +111,10 @@ __global__ void k_delta_top(const float* p, const int32_t* y, const float* coef,
 //   mode 2: out[n] = s_in[n] + t_in[n] - step * sum   (one Horner step of the Neumann series; out may alias t_in)
 struct ColsumSink { int mode; float step; float* out; const float* t_in; const float* s_in; };
 static constexpr int CS_COLS = 32, CS_GROUPS = 64;
-__global__ void __launch_bounds__(1024) k_colsum_bf16(const op16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
-  pdl_enter();
-  __shared__ float sh[CS_GROUPS][CS_COLS + 1];
+__device__ __forceinline__ void colsum_block(const op16* d, int64_t B, int64_t N, int64_t ld, const ColsumSink& k,
+                                             int64_t block, float (*sh)[CS_COLS + 1]) {
   const int cx = threadIdx.x & 15, rg = threadIdx.x >> 4;
-  const int64_t n = blockIdx.x * CS_COLS + 2 * cx;
+  const int64_t n = block * CS_COLS + 2 * cx;
   float a0 = 0.f, a1 = 0.f;
   if (n < N) {
     constexpr int U = 16;
@@ -136,7 +135,7 @@ __global__ void __launch_bounds__(1024) k_colsum_bf16(const op16* d, int64_t B, 
   sh[rg][2 * cx] = a0; sh[rg][2 * cx + 1] = a1;
   __syncthreads();
   if (threadIdx.x < CS_COLS) {
-    const int64_t nn = blockIdx.x * CS_COLS + threadIdx.x;
+    const int64_t nn = block * CS_COLS + threadIdx.x;
     if (nn < N) {
       float t = 0.f;
 #pragma unroll
@@ -147,6 +146,39 @@ __global__ void __launch_bounds__(1024) k_colsum_bf16(const op16* d, int64_t B, 
     }
   }
 }
+__global__ void __launch_bounds__(1024) k_colsum_bf16(const op16* d, int64_t B, int64_t N, int64_t ld, ColsumSink k) {
+  pdl_enter();
+  __shared__ float sh[CS_GROUPS][CS_COLS + 1];
+  colsum_block(d, B, N, ld, k, blockIdx.x, sh);
+}
+// The column sums of several layers in one launch (a reverse sweep that runs on one stream takes them together
+// after its last product): block b belongs to the job whose block range contains it.
+struct ColsumJob { const op16* d; int64_t B, N, ld; ColsumSink k; int first_block; };
+struct ColsumJobs { int n; ColsumJob j[MAXL]; };
+__global__ void __launch_bounds__(1024) k_colsum_multi(const __grid_constant__ ColsumJobs jobs) {
+  pdl_enter();
+  __shared__ float sh[CS_GROUPS][CS_COLS + 1];
+  int i = jobs.n - 1;
+  while (i > 0 && (int)blockIdx.x < jobs.j[i].first_block) --i;
+  const ColsumJob& job = jobs.j[i];
+  colsum_block(job.d, job.B, job.N, job.ld, job.k, (int64_t)blockIdx.x - job.first_block, sh);
+}
+// collects a sweep's column sums; launch() takes them all in one kernel
+struct ColsumBatch {
+  ColsumJobs jobs; int blocks;
+  ColsumBatch() : blocks(0) { jobs.n = 0; }
+  void add(const op16* d, int64_t B, int64_t N, int64_t ld, const ColsumSink& k) {
+    ColsumJob& j = jobs.j[jobs.n++];
+    j.d = d; j.B = B; j.N = N; j.ld = ld; j.k = k; j.first_block = blocks;
+    blocks += (int)((N + CS_COLS - 1) / CS_COLS);
+  }
+  betty_status launch(Ctx& c) {
+    if (jobs.n == 0) return BETTY_OK;
+    launch_pdl(k_colsum_multi, dim3((unsigned)blocks), dim3(1024), 0, c.stream, jobs);
+    BETTY_LAUNCH_CHECK();
+    return BETTY_OK;
+  }
+};
 // delta_prev = dh * act'(a)
 __global__ void k_act_backward(const float* dh, const float* a, op16* dprev, int64_t B, int64_t N, int64_t ld, int act) {
   pdl_enter();
@@ -797,6 +829,8 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
   // side stream.  (A gradient step there writes the master matrix and the *other* op16 copy, never the copy
   // the chain's product for the same layer reads.)
   SideWork side(c, n.L >= SIDE_MIN_LAYERS);
+  const bool one_stream = !side.forks();
+  ColsumBatch colsums;
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
     if (sink.gflat || sink.sgd) {
@@ -818,8 +852,12 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
         launch_pdl(k_wd_add_bf16, dim3(grid_for(N * K)), dim3(256), 0, c.stream, sink.gflat + n.woff[l], n.W[l], N, K, n.ldw[l], sink.lam + l, sink.lscale);
         BETTY_LAUNCH_CHECK();
       }
-      launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, ps.delta[l], B, N, ldd, cs);
-      BETTY_LAUNCH_CHECK();
+      if (one_stream) {
+        colsums.add(ps.delta[l], B, N, ldd, cs);      // taken together after the last product
+      } else {
+        launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, ps.delta[l], B, N, ldd, cs);
+        BETTY_LAUNCH_CHECK();
+      }
       side.end();
     }
     if (l > 0) {
@@ -843,6 +881,7 @@ static betty_status backward(Ctx& c, const Net& n, Pass& ps, const float* coef, 
       BETTY_TRY(gemm(c, g));
     }
   }
+  BETTY_TRY(colsums.launch(c));
   return side.join();
 }
 static inline GradSink grad_into(float* gflat, const float* lam) {
@@ -1196,6 +1235,8 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, HvpCache* h, const fl
   // The chain is Rdelta_L -> Rdelta_{L-1} -> ... ; each layer's weight product goes to the side stream once the
   // chain's product of the same layer has been launched (it reads the U_l that the weight product may overwrite).
   SideWork side(c, n.L >= SIDE_MIN_LAYERS);
+  const bool one_stream = !side.forks();
+  ColsumBatch colsums;
   for (int l = n.L - 1; l >= 0; --l) {
     const int64_t N = n.w[l + 1], K = n.w[l], ldd = ld8(N);
     op16* Rdp = nullptr;
@@ -1234,12 +1275,17 @@ static betty_status hvp_impl(Ctx& c, const betty_level* L, HvpCache* h, const fl
         launch_pdl(k_wd_add_f32, dim3(grid_for(N * K)), dim3(256), 0, c.stream, Hu + n.woff[l], u + n.woff[l], N * K, h->lam + l);
         BETTY_LAUNCH_CHECK();
       }
-      launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, Rd, B, N, ldd, cs);
-      BETTY_LAUNCH_CHECK();
+      if (one_stream) {
+        colsums.add(Rd, B, N, ldd, cs);
+      } else {
+        launch_pdl(k_colsum_bf16, dim3((unsigned)((N + CS_COLS - 1) / CS_COLS)), dim3(1024), 0, c.stream, Rd, B, N, ldd, cs);
+        BETTY_LAUNCH_CHECK();
+      }
       side.end();
     }
     if (l > 0) Rd = Rdp;
   }
+  BETTY_TRY(colsums.launch(c));
   BETTY_TRY(side.join());
   if (leave16) h->dir16_of = sink->out;
   c.arena.release(mark);
