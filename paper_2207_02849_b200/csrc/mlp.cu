@@ -265,14 +265,15 @@ __global__ void k_wd_add_f32(float* out, const float* u, int64_t n, const float*
 // that draws the last ticket adds the per-block sums in a fixed order (one warp: strided partial sums, then a
 // shuffle tree), so the result does not depend on scheduling.
 static constexpr int LD_MAX_BLOCKS = 128;
-__global__ void k_layer_dot(const op16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
-                            float scale, float* out, int accumulate, double* partial, unsigned* counter) {
-  pdl_enter();
+// block `blk` of `nblk` blocks working on one matrix
+__device__ __forceinline__ void layer_dot_block(const op16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
+                                                float scale, float* out, int accumulate, double* partial, unsigned* counter,
+                                                unsigned blk, unsigned nblk) {
   __shared__ double sh[32];
   __shared__ bool is_last;
   double acc = 0.0;
   const int64_t total = rows * cols;
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+  for (int64_t i = blk * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)nblk * blockDim.x) {
     const int64_t r = i / cols, c = i - r * cols;
     const float w = from_op16(W[r * ldw + c]);
     acc += (double)w * (double)(q ? q[i] : w);
@@ -283,16 +284,16 @@ __global__ void k_layer_dot(const op16* W, int64_t rows, int64_t cols, int64_t l
   if (threadIdx.x == 0) {
     double t = 0.0;
     for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += sh[i];
-    partial[blockIdx.x] = t;
+    partial[blk] = t;
     __threadfence();
-    is_last = atomicAdd(counter, 1u) == gridDim.x - 1;
+    is_last = atomicAdd(counter, 1u) == nblk - 1;
   }
   __syncthreads();
   if (is_last && threadIdx.x < 32) {
     // second phase by one warp: lane l adds blocks l, l+32, ... in order, then a fixed shuffle tree
     __threadfence();
     double tot = 0.0;
-    for (unsigned bb = threadIdx.x; bb < gridDim.x; bb += 32) tot += ((volatile double*)partial)[bb];
+    for (unsigned bb = threadIdx.x; bb < nblk; bb += 32) tot += ((volatile double*)partial)[bb];
     for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
     if (threadIdx.x == 0) {
       const float v = scale * expf(*lam) * (float)tot;
@@ -301,20 +302,18 @@ __global__ void k_layer_dot(const op16* W, int64_t rows, int64_t cols, int64_t l
     }
   }
 }
-static betty_status layer_dot(Ctx& c, const op16* W, int64_t rows, int64_t cols, int64_t ldw, const float* q, const float* lam,
-                              float scale, float* out, bool accumulate) {
-  int64_t nb = (rows * cols + 256 * 16 - 1) / (256 * 16);
-  nb = nb < 1 ? 1 : (nb > LD_MAX_BLOCKS ? LD_MAX_BLOCKS : nb);
-  const size_t mark = c.arena.mark();
-  BETTY_ALLOC(partial, double, c, (size_t)nb);
-  BETTY_ALLOC(counter, unsigned, c, 8);
-  BETTY_TRY(vec_zero(c, (float*)counter, 8));     // a kernel, not a memset: keeps the programmatic launch chain unbroken
-  launch_pdl(k_layer_dot, dim3((unsigned)nb), dim3(256), 0, c.stream, W, rows, cols, ldw, q, lam, scale, out, accumulate ? 1 : 0, partial, counter);
-  BETTY_LAUNCH_CHECK();
-  c.arena.release(mark);
-  return BETTY_OK;
+// All layers of a net in one launch: block b belongs to the job whose block range contains it; every job has partial
+// sums, a ticket counter and an output of its own.
+struct LayerDotJob { const op16* W; int64_t rows, cols, ldw; const float* q; const float* lam; float* out; double* partial; unsigned* counter; int first_block, n_blocks; };
+struct LayerDotJobs { int n; float scale; int accumulate; LayerDotJob j[MAXL]; };
+__global__ void k_layer_dot_multi(const __grid_constant__ LayerDotJobs jobs) {
+  pdl_enter();
+  int i = jobs.n - 1;
+  while (i > 0 && (int)blockIdx.x < jobs.j[i].first_block) --i;
+  const LayerDotJob& t = jobs.j[i];
+  layer_dot_block(t.W, t.rows, t.cols, t.ldw, t.q, t.lam, jobs.scale, t.out, jobs.accumulate, t.partial, t.counter,
+                  blockIdx.x - (unsigned)t.first_block, (unsigned)t.n_blocks);
 }
-
 // ------------------------------------------------------------------ weight net 1-100-1
 enum WnMode { WN_REWEIGHT_COEF = 0, WN_REWEIGHT_TGRAD, WN_REWEIGHT_TMIXED, WN_DETECT_TGRAD, WN_DETECT_WGRAD,
               WN_DETECT_THVP, WN_DETECT_WMIXED };
@@ -688,6 +687,32 @@ struct CorrBack {
   const op16* M16; int64_t ldm;    // [A; A1], operand type
   int64_t Kc;               // C + 100
 };
+
+// out[l] (+)= scale * exp(lam[l]) * <W_l, q_l> for every layer (q == nullptr: <W_l, W_l>): one zeroing kernel for all
+// ticket counters and one launch for all layers.
+static betty_status layer_dots(Ctx& c, const Net& n, const float* q, const float* lam, float scale, float* out, bool accumulate) {
+  const size_t mark = c.arena.mark();
+  LayerDotJobs jobs;
+  jobs.n = n.L; jobs.scale = scale; jobs.accumulate = accumulate ? 1 : 0;
+  BETTY_ALLOC(counters, unsigned, c, (size_t)(8 * n.L));
+  int blocks = 0;
+  for (int l = 0; l < n.L; ++l) {
+    const int64_t rows = n.w[l + 1], cols = n.w[l];
+    int64_t nb = (rows * cols + 256 * 16 - 1) / (256 * 16);
+    nb = nb < 1 ? 1 : (nb > LD_MAX_BLOCKS ? LD_MAX_BLOCKS : nb);
+    BETTY_ALLOC(partial, double, c, (size_t)nb);
+    LayerDotJob& t = jobs.j[l];
+    t.W = n.W[l]; t.rows = rows; t.cols = cols; t.ldw = n.ldw[l];
+    t.q = q ? q + n.woff[l] : nullptr; t.lam = lam + l; t.out = out + l;
+    t.partial = partial; t.counter = counters + 8 * l; t.first_block = blocks; t.n_blocks = (int)nb;
+    blocks += (int)nb;
+  }
+  BETTY_TRY(vec_zero(c, (float*)counters, 8 * n.L));
+  launch_pdl(k_layer_dot_multi, dim3((unsigned)blocks), dim3(256), 0, c.stream, jobs);
+  BETTY_LAUNCH_CHECK();
+  c.arena.release(mark);
+  return BETTY_OK;
+}
 
 static betty_status net_layout(const betty_level* M, Net& n) {
   if (M->param_kind != BETTY_PARAM_MLP || M->n_layers < 1 || M->n_layers > MAXL || !M->widths) return BETTY_ERR_INVALID_ARG;
@@ -1099,9 +1124,7 @@ betty_status mlpfam_grad(Ctx& c, const betty_level* L, const betty_level* wrt, f
   Net n; Pass ps;
   BETTY_TRY(net_setup(c, P.mlp, n));
   if (P.lam && wrt == P.lam) {
-    for (int l = 0; l < n.L; ++l) {
-      BETTY_TRY(layer_dot(c, n.W[l], n.w[l + 1], n.w[l], n.ldw[l], nullptr, P.lam->params + l, 0.5f, out + l, false));
-    }
+    BETTY_TRY(layer_dots(c, n, nullptr, P.lam->params, 0.5f, out, false));
     c.arena.release(mark);
     return BETTY_OK;
   }
@@ -1326,9 +1349,7 @@ betty_status mlpfam_mixed(Ctx& c, const betty_level* L, MlpHvpCache* handle, con
   const int64_t B = ps.B;
   if (L->loss == BETTY_LOSS_MLP_CE_REWEIGHT) {
     if (P.lam && wrt == P.lam) {
-      for (int l = 0; l < n.L; ++l) {
-        BETTY_TRY(layer_dot(c, n.W[l], n.w[l + 1], n.w[l], n.ldw[l], q + n.woff[l], P.lam->params + l, 1.f, out + l, false));
-      }
+      BETTY_TRY(layer_dots(c, n, q, P.lam->params, 1.f, out, false));
     } else if (P.theta && wrt == P.theta) {
       RPass rp;
       BETTY_TRY(rforward(c, n, ps, q, rp, h));
@@ -1425,9 +1446,7 @@ betty_status mlpfam_fd(Ctx& c, const betty_level* L, const betty_level* wrt, con
   if (P.lam && wrt == P.lam) {
     // dC/d(lam_l) = 1/2 exp(lam_l)|W_l|^2 is quadratic in W: its central difference is exactly
     // exp(lam_l) <W_l, V_l> for every eps, which is what is evaluated.
-    for (int l = 0; l < n.L; ++l) {
-      BETTY_TRY(layer_dot(c, n.W[l], n.w[l + 1], n.w[l], n.ldw[l], v + n.woff[l], P.lam->params + l, -alpha, out + l, accumulate));
-    }
+    BETTY_TRY(layer_dots(c, n, v, P.lam->params, -alpha, out, accumulate));
     c.arena.release(mark);
     return BETTY_OK;
   }
